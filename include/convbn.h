@@ -1,0 +1,181 @@
+/*
+ * convbn.h - C ABI of the B200 (sm_100a) Tune-mode Convolution-BatchNorm library.
+ *
+ * One ConvBN block (paper Sec. 3.1): a convolution with weight omega and optional bias b,
+ * followed by a BatchNorm layer with FROZEN running statistics mu_hat / var_hat and affine
+ * parameters gamma / beta.  Per output channel co:
+ *
+ *     r[co] = 1 / sqrt(var_hat[co] + eps)          s[co] = gamma[co] r[co]
+ *     omega'[co,:] = s[co] omega[co,:]             b'[co] = (b[co] - mu_hat[co]) s[co] + beta[co]
+ *
+ * Conventions common to every entry point
+ *   - The descriptor is read on the host.  EVERY OTHER POINTER IS A DEVICE POINTER (memory the
+ *     current device can access) unless the argument is explicitly called "host".
+ *   - The caller owns every buffer.  The library allocates no device memory, keeps no
+ *     reference to a buffer after the call's kernels have run, and never writes the running
+ *     statistics.  Work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = the
+ *     default stream) and the call returns without synchronising.
+ *   - Activations x / z / dz / dx / y have dtype `desc.dtype` and layout `desc.layout`:
+ *         CONVBN_NCHW: [N][C][H][W]   weight: [C_out][C_in/G][kh][kw]
+ *         CONVBN_NHWC: [N][H][W][C]   weight: [C_out][kh][kw][C_in/G]
+ *     Weights passed in have the activation dtype.  b, gamma, beta, run_mean, run_var and
+ *     every parameter gradient (dw in the weight's layout, db, dgamma, dbeta) are fp32.
+ *     Supported pairs: (F32, NCHW) and (BF16, NHWC); others return CONVBN_EUNSUPPORTED.
+ *   - Convolution hyper-parameters follow the usual deep-learning convention (the paper
+ *     states only a kernel size): cross-correlation, zero padding, floor output size
+ *     H_out = (H_in + 2 pad_h - dil_h (kh-1) - 1) / stride_h + 1, contiguous channel groups.
+ *   - Activation and weight pointers must be 16-byte aligned, fp32 vectors 4-byte aligned.
+ *   - `workspace` is scratch of at least convbn_workspace_bytes(desc, phase) bytes, 256-byte
+ *     aligned; its contents are undefined after the call.  Calls that share a workspace must
+ *     not overlap on the device.
+ *   - Return value: a convbn_status.  Descriptor, pointer, alignment and workspace problems are
+ *     found on the host before anything is launched.  A launch failure gives CONVBN_ECUDA.
+ *     Device-side waits are bounded; one that expires sets a device error word which
+ *     convbn_check() reports as CONVBN_ETIMEOUT.
+ *   - Arithmetic: products of the storage type, fp32 accumulation, per-channel work in fp32,
+ *     one rounding to the storage type when an activation is written.  Results are
+ *     run-to-run deterministic (fixed reduction order, no floating-point atomics).
+ */
+#ifndef CONVBN_H_
+#define CONVBN_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CONVBN_OK = 0,
+    CONVBN_EINVAL = 1,       /* bad descriptor or NULL pointer                      */
+    CONVBN_EUNSUPPORTED = 2, /* dtype / layout pair not implemented                 */
+    CONVBN_EWORKSPACE = 3,   /* workspace missing or too small                      */
+    CONVBN_EALIGN = 4,       /* pointer not aligned as required                     */
+    CONVBN_ECUDA = 5,        /* CUDA runtime / driver call failed                   */
+    CONVBN_ETIMEOUT = 6      /* a bounded device-side wait expired                  */
+} convbn_status;
+
+typedef enum { CONVBN_F32 = 0, CONVBN_BF16 = 1 } convbn_dtype;
+typedef enum { CONVBN_NCHW = 0, CONVBN_NHWC = 1 } convbn_layout;
+typedef enum { CONVBN_MODE_TUNE = 0, CONVBN_MODE_EVAL = 1, CONVBN_MODE_DEPLOY = 2 } convbn_mode;
+
+typedef enum {
+    CONVBN_PHASE_TUNE_FWD = 0,
+    CONVBN_PHASE_TUNE_BWD_DATA = 1,
+    CONVBN_PHASE_TUNE_BWD_WEIGHT = 2,
+    CONVBN_PHASE_EVAL_FWD = 3,
+    CONVBN_PHASE_EVAL_BWD = 4,
+    CONVBN_PHASE_DEPLOY_FWD = 5,
+    CONVBN_PHASE_DEPLOY_BWD = 6,
+    CONVBN_PHASE_COUNT = 7
+} convbn_phase;
+
+/* Problem description (paper Sec. 3.1 and the shape annotations of Appendix C; stride, padding,
+ * dilation and groups as in the convention above).  Plain data, read on the host. */
+typedef struct convbn_desc {
+    int n, c_in, h_in, w_in;   /* X is [N, C_in, H_in, W_in] logically                  */
+    int c_out, kh, kw;         /* omega is [C_out, C_in/groups, kh, kw] logically        */
+    int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, groups;
+    int dtype;                 /* convbn_dtype of activations and weights               */
+    int layout;                /* convbn_layout                                         */
+    double eps;                /* BatchNorm epsilon, added to the variance under the root */
+} convbn_desc;
+
+/* Output extent of the convolution (floor convention).  Host only.
+ * CONVBN_EINVAL if the descriptor is inconsistent or the output would be empty. */
+int convbn_out_shape(const convbn_desc *desc, int *h_out, int *w_out);
+
+/* Bytes of the opaque `saved` buffer that a forward call of `mode` (convbn_mode) writes for its
+ * backward calls - the activation kept beside X (Sec. 3.3 / 3.4, Appendix M memory analysis):
+ *   TUNE   : three fp32 vectors s, b', r (omega' is re-formed from omega in backward, it is
+ *            never kept; no pre-normalisation tensor exists)
+ *   EVAL   : the pre-normalisation output Y, N C_out H_out W_out elements of desc.dtype
+ *   DEPLOY : 0
+ * Returns 0 for an invalid descriptor. */
+size_t convbn_saved_bytes(const convbn_desc *desc, int mode);
+
+/* Scratch bytes a call of `phase` (convbn_phase) needs.  0 for an invalid descriptor/phase. */
+size_t convbn_workspace_bytes(const convbn_desc *desc, int phase);
+
+/* ---- Tune mode (Sec. 3.4; Table 2, Tune row) --------------------------------------------- */
+
+/* Forward: forms s, b' and omega' from the CURRENT parameters ("on the fly"), then
+ *     Z = omega' (*) X + b'.
+ * in : x [activation], w [weight], b [C_out] or NULL (= no conv bias), gamma, beta, run_mean,
+ *      run_var [C_out]
+ * out: z [N, C_out, H_out, W_out]; saved (convbn_saved_bytes(desc, TUNE) bytes, 16-byte aligned) */
+int convbn_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const float *b,
+                    const float *gamma, const float *beta, const float *run_mean,
+                    const float *run_var, void *z, void *saved, void *workspace,
+                    size_t workspace_bytes, void *stream);
+
+/* Backward, data:  dX = omega'_rot (*) dZ  (the transposed convolution of dZ with omega').
+ * in : dz, w (the same omega given to the forward), saved (from convbn_tune_fwd)
+ * out: dx, same shape as x.  Every element of dx is written. */
+int convbn_tune_bwd_data(const convbn_desc *desc, const void *dz, const void *w,
+                         const void *saved, void *dx, void *workspace, size_t workspace_bytes,
+                         void *stream);
+
+/* Backward, parameters:
+ *     domega' = dZ (.) X                      (cross-correlation over N, H_out, W_out)
+ *     domega  = s domega'                     dbeta = sum dZ        db = s dbeta
+ *     dgamma  = r ( sum_{ci,r,q} domega' omega + dbeta (b - mu_hat) )
+ * in : dz, x, w, b (NULL iff the conv has no bias), run_mean, saved
+ * out: dw [weight layout, fp32], db [C_out] (must be NULL iff b is NULL), dgamma, dbeta [C_out] */
+int convbn_tune_bwd_weight(const convbn_desc *desc, const void *dz, const void *x,
+                           const void *w, const float *b, const float *run_mean,
+                           const void *saved, float *dw, float *db, float *dgamma,
+                           float *dbeta, void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---- Eval mode comparator (Sec. 3.1; Table 2, Eval row) ---------------------------------- */
+
+/* Y = omega (*) X + b is written to `y_saved` (the activation Eval mode keeps), then
+ * Z = gamma (Y - mu_hat) r + beta.  y_saved: convbn_saved_bytes(desc, EVAL) bytes. */
+int convbn_eval_fwd(const convbn_desc *desc, const void *x, const void *w, const float *b,
+                    const float *gamma, const float *beta, const float *run_mean,
+                    const float *run_var, void *z, void *y_saved, void *workspace,
+                    size_t workspace_bytes, void *stream);
+
+/* dY = s dZ; dX = omega_rot (*) dY; domega = dY (.) X; db = sum dY;
+ * dgamma = sum dZ (Y - mu_hat) r; dbeta = sum dZ.   db may be NULL. */
+int convbn_eval_bwd(const convbn_desc *desc, const void *dz, const void *x, const void *y_saved,
+                    const void *w, const float *gamma, const float *run_mean,
+                    const float *run_var, void *dx, float *dw, float *db, float *dgamma,
+                    float *dbeta, void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---- Deploy mode comparator (Sec. 3.3; Table 2, Deploy row; Appendix C) -------------------- */
+
+/* Once for all: w_fused = omega' (weight dtype and layout), b_fused = b' (fp32). */
+int convbn_deploy_prepare(const convbn_desc *desc, const void *w, const float *b,
+                          const float *gamma, const float *beta, const float *run_mean,
+                          const float *run_var, void *w_fused, float *b_fused, void *stream);
+
+/* Z = omega' (*) X + b' */
+int convbn_deploy_fwd(const convbn_desc *desc, const void *x, const void *w_fused,
+                      const float *b_fused, void *z, void *workspace, size_t workspace_bytes,
+                      void *stream);
+
+/* dX = omega'_rot (*) dZ; domega' = dZ (.) X; db' = sum dZ.  Gradients go to the FUSED
+ * parameters only (which is what makes this mode unstable for training, Sec. 3.3). */
+int convbn_deploy_bwd(const convbn_desc *desc, const void *dz, const void *x,
+                      const void *w_fused, void *dx, float *dw_fused, float *db_fused,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---- housekeeping -------------------------------------------------------------------------- */
+
+/* Synchronises `stream`, then reads and clears the device error word of the current device.
+ * CONVBN_OK, CONVBN_ETIMEOUT (a bounded wait in a kernel gave up; outputs of that call are
+ * invalid) or CONVBN_ECUDA (the stream reported an error). */
+int convbn_check(void *stream);
+
+/* Static, NUL-terminated description of a status code. */
+const char *convbn_status_string(int status);
+
+/* Name of the kernel family the last call of `phase` selected on this thread ("direct",
+ * "umma", "depthwise", ...), for logs and tests.  Static string, never NULL. */
+const char *convbn_last_kernel(int phase);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CONVBN_H_ */

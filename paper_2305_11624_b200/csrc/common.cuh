@@ -1,0 +1,65 @@
+// Shared device/host declarations of the ConvBN library: the kernel-side problem record,
+// tensor index helpers for the two memory layouts, storage-type conversion and error plumbing.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/convbn.h"
+
+namespace convbn {
+
+// Problem sizes as the kernels see them (derived once on the host from convbn_desc).
+struct Problem {
+    int n, c_in, h_in, w_in, c_out, kh, kw;
+    int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, groups;
+    int h_out, w_out;
+    int cg;        // input channels per group
+    int cog;       // output channels per group
+    int kdim;      // cg * kh * kw : length of one weight row
+    long long p;   // n * h_out * w_out : output pixels
+    long long pin; // n * h_in * w_in : input pixels
+    float eps;
+};
+
+// Layout tags (match convbn_layout).
+struct NCHW { static constexpr int id = CONVBN_NCHW; };
+struct NHWC { static constexpr int id = CONVBN_NHWC; };
+
+template <class L>
+__host__ __device__ __forceinline__ long long act_idx(int n, int c, int h, int w, int C, int H, int W) {
+    if (L::id == CONVBN_NCHW) return (((long long)n * C + c) * H + h) * W + w;
+    return (((long long)n * H + h) * W + w) * C + c;
+}
+
+// Weight element (co, ci, r, q) of a [C_out][Cg][kh][kw] (NCHW) or [C_out][kh][kw][Cg] (NHWC) tensor.
+template <class L>
+__host__ __device__ __forceinline__ long long w_idx(int co, int ci, int r, int q, int cg, int kh, int kw) {
+    if (L::id == CONVBN_NCHW) return (((long long)co * cg + ci) * kh + r) * kw + q;
+    return (((long long)co * kh + r) * kw + q) * cg + ci;
+}
+
+// Position k within a weight row -> (ci, r, q) for the layout's row order.
+template <class L>
+__host__ __device__ __forceinline__ void w_row_decode(int k, int cg, int kh, int kw, int &ci, int &r, int &q) {
+    if (L::id == CONVBN_NCHW) { q = k % kw; int t = k / kw; r = t % kh; ci = t / kh; }
+    else { ci = k % cg; int t = k / cg; q = t % kw; r = t / kw; }
+}
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <class T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// Device error word: kernels that give up on a bounded wait OR a non-zero code into it.  The word
+// lives in one translation unit; kernels elsewhere get its device address as an argument.
+enum : int { ERRW_TIMEOUT = 1 };
+cudaError_t error_word_address(int **dev_ptr);          // address on the current device
+cudaError_t read_and_clear_error_word(int *host_value); // synchronous
+
+static inline int ceil_div_i(long long a, long long b) { return (int)((a + b - 1) / b); }
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace convbn

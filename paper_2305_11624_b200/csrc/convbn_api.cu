@@ -1,0 +1,352 @@
+// C ABI of the ConvBN library: host-side validation, workspace planning, kernel selection.
+// Every step of every entry point runs in this library's own kernels; there is no CPU path.
+#include <stdint.h>
+#include <string.h>
+
+#include "kernels.h"
+
+using namespace convbn;
+
+namespace {
+
+thread_local const char *t_last_kernel[CONVBN_PHASE_COUNT] = {"none", "none", "none", "none",
+                                                              "none", "none", "none"};
+
+inline bool aligned(const void *p, size_t a) { return ((uintptr_t)p % a) == 0; }
+inline size_t elem_size(int dtype) { return dtype == CONVBN_F32 ? 4 : 2; }
+
+int make_problem(const convbn_desc *d, Problem *pb) {
+    if (!d) return CONVBN_EINVAL;
+    if (d->n <= 0 || d->c_in <= 0 || d->h_in <= 0 || d->w_in <= 0 || d->c_out <= 0 || d->kh <= 0 ||
+        d->kw <= 0 || d->stride_h <= 0 || d->stride_w <= 0 || d->pad_h < 0 || d->pad_w < 0 ||
+        d->dil_h <= 0 || d->dil_w <= 0 || d->groups <= 0)
+        return CONVBN_EINVAL;
+    if (d->c_in % d->groups || d->c_out % d->groups) return CONVBN_EINVAL;
+    if (!(d->eps >= 0.0)) return CONVBN_EINVAL;
+    const long long eh = (long long)d->h_in + 2LL * d->pad_h - (long long)d->dil_h * (d->kh - 1) - 1;
+    const long long ew = (long long)d->w_in + 2LL * d->pad_w - (long long)d->dil_w * (d->kw - 1) - 1;
+    if (eh < 0 || ew < 0) return CONVBN_EINVAL;
+    if (d->dtype != CONVBN_F32 && d->dtype != CONVBN_BF16) return CONVBN_EINVAL;
+    if (d->layout != CONVBN_NCHW && d->layout != CONVBN_NHWC) return CONVBN_EINVAL;
+    pb->n = d->n; pb->c_in = d->c_in; pb->h_in = d->h_in; pb->w_in = d->w_in;
+    pb->c_out = d->c_out; pb->kh = d->kh; pb->kw = d->kw;
+    pb->stride_h = d->stride_h; pb->stride_w = d->stride_w; pb->pad_h = d->pad_h; pb->pad_w = d->pad_w;
+    pb->dil_h = d->dil_h; pb->dil_w = d->dil_w; pb->groups = d->groups;
+    pb->h_out = (int)(eh / d->stride_h) + 1;
+    pb->w_out = (int)(ew / d->stride_w) + 1;
+    pb->cg = d->c_in / d->groups;
+    pb->cog = d->c_out / d->groups;
+    const long long kdim = (long long)pb->cg * d->kh * d->kw;
+    pb->p = (long long)d->n * pb->h_out * pb->w_out;
+    pb->pin = (long long)d->n * d->h_in * d->w_in;
+    // keep every element count inside 2^40 and every row inside int
+    if (kdim > (1LL << 30) || pb->p * d->c_out > (1LL << 40) || pb->pin * d->c_in > (1LL << 40))
+        return CONVBN_EINVAL;
+    pb->kdim = (int)kdim;
+    pb->eps = (float)d->eps;
+    return CONVBN_OK;
+}
+
+int check_pair(const convbn_desc *d) {
+    if ((d->dtype == CONVBN_F32 && d->layout == CONVBN_NCHW) ||
+        (d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC))
+        return CONVBN_OK;
+    return CONVBN_EUNSUPPORTED;
+}
+
+// Workspace carve-up of one phase.  Offsets are multiples of 256 bytes.
+struct Plan {
+    size_t total = 0;
+    size_t w_scaled = 0;   // omega' (storage dtype, weight layout)
+    size_t partials = 0;   // [splits][C_out][kdim] fp32
+    size_t bsum = 0;       // [bsplits][C_out] fp32
+    size_t part_g = 0;     // [bsplits][C_out] fp32 (Eval backward)
+    size_t dy = 0;         // Eval backward: s dZ, storage dtype
+    size_t vec3 = 0;       // Eval forward: [s | beta - mean s | r]
+    int splits = 1, bsplits = 1;
+};
+
+Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
+    Plan pl;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    const size_t wbytes = (size_t)pb.c_out * pb.kdim * elem_size(d->dtype);
+    const size_t wrows = (size_t)pb.c_out * pb.kdim;
+    pl.splits = direct_wgrad_splits(pb);
+    pl.bsplits = channel_sum_splits(pb);
+    switch (phase) {
+        case CONVBN_PHASE_TUNE_FWD:
+        case CONVBN_PHASE_TUNE_BWD_DATA:
+            pl.w_scaled = take(wbytes);
+            break;
+        case CONVBN_PHASE_TUNE_BWD_WEIGHT:
+        case CONVBN_PHASE_DEPLOY_BWD:
+            pl.partials = take(wrows * pl.splits * sizeof(float));
+            pl.bsum = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
+            break;
+        case CONVBN_PHASE_EVAL_FWD:
+            pl.vec3 = take(3 * (size_t)pb.c_out * sizeof(float));
+            break;
+        case CONVBN_PHASE_EVAL_BWD:
+            pl.dy = take((size_t)pb.p * pb.c_out * elem_size(d->dtype));
+            pl.part_g = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
+            pl.bsum = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
+            pl.partials = take(wrows * pl.splits * sizeof(float));
+            break;
+        default:
+            break;
+    }
+    pl.total = off;
+    return pl;
+}
+
+int check_ws(const Plan &pl, const void *ws, size_t ws_bytes) {
+    if (pl.total == 0) return CONVBN_OK;
+    if (!ws || ws_bytes < pl.total) return CONVBN_EWORKSPACE;
+    if (!aligned(ws, 256)) return CONVBN_EALIGN;
+    return CONVBN_OK;
+}
+
+#define CK(expr) do { int _s = (expr); if (_s != CONVBN_OK) return _s; } while (0)
+#define CU(expr) do { if ((expr) != cudaSuccess) return CONVBN_ECUDA; } while (0)
+
+inline char *at(void *ws, size_t off) { return (char *)ws + off; }
+
+// Shared by Tune and Deploy backward-weight: conv weight gradient partials + per-channel dZ sums.
+int run_wgrad_partials(const convbn_desc *d, const Problem &pb, const Plan &pl, const void *dz,
+                       const void *x, void *ws, cudaStream_t st) {
+    CU(launch_direct_wgrad(pb, d->dtype, d->layout, dz, x, (float *)at(ws, pl.partials), pl.splits, st));
+    CU(launch_channel_sum_partial(pb, d->dtype, d->layout, dz, (float *)at(ws, pl.bsum), pl.bsplits, st));
+    return CONVBN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int convbn_out_shape(const convbn_desc *desc, int *h_out, int *w_out) {
+    Problem pb;
+    if (!h_out || !w_out) return CONVBN_EINVAL;
+    CK(make_problem(desc, &pb));
+    *h_out = pb.h_out;
+    *w_out = pb.w_out;
+    return CONVBN_OK;
+}
+
+size_t convbn_saved_bytes(const convbn_desc *desc, int mode) {
+    Problem pb;
+    if (make_problem(desc, &pb) != CONVBN_OK) return 0;
+    switch (mode) {
+        case CONVBN_MODE_TUNE: return 3 * (size_t)pb.c_out * sizeof(float);
+        case CONVBN_MODE_EVAL: return (size_t)pb.p * pb.c_out * elem_size(desc->dtype);
+        default: return 0;
+    }
+}
+
+size_t convbn_workspace_bytes(const convbn_desc *desc, int phase) {
+    Problem pb;
+    if (phase < 0 || phase >= CONVBN_PHASE_COUNT) return 0;
+    if (make_problem(desc, &pb) != CONVBN_OK) return 0;
+    return make_plan(desc, pb, phase).total;
+}
+
+int convbn_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const float *b,
+                    const float *gamma, const float *beta, const float *run_mean,
+                    const float *run_var, void *z, void *saved, void *workspace,
+                    size_t workspace_bytes, void *stream) {
+    Problem pb;
+    CK(make_problem(desc, &pb));
+    CK(check_pair(desc));
+    if (!x || !w || !gamma || !beta || !run_mean || !run_var || !z || !saved) return CONVBN_EINVAL;
+    if (!aligned(x, 16) || !aligned(w, 16) || !aligned(z, 16) || !aligned(saved, 16) ||
+        !aligned(b, 4) || !aligned(gamma, 4) || !aligned(beta, 4) || !aligned(run_mean, 4) ||
+        !aligned(run_var, 4))
+        return CONVBN_EALIGN;
+    const Plan pl = make_plan(desc, pb, CONVBN_PHASE_TUNE_FWD);
+    CK(check_ws(pl, workspace, workspace_bytes));
+    cudaStream_t st = (cudaStream_t)stream;
+    float *vec3 = (float *)saved;
+    void *wf = at(workspace, pl.w_scaled);
+    CU(launch_reparam(pb, desc->dtype, desc->layout, w, b, gamma, beta, run_mean, run_var, vec3, wf,
+                      nullptr, st));
+    CU(launch_direct_fwd(pb, desc->dtype, desc->layout, x, wf, vec3 + pb.c_out, z, st));
+    t_last_kernel[CONVBN_PHASE_TUNE_FWD] = "direct";
+    return CONVBN_OK;
+}
+
+int convbn_tune_bwd_data(const convbn_desc *desc, const void *dz, const void *w, const void *saved,
+                         void *dx, void *workspace, size_t workspace_bytes, void *stream) {
+    Problem pb;
+    CK(make_problem(desc, &pb));
+    CK(check_pair(desc));
+    if (!dz || !w || !saved || !dx) return CONVBN_EINVAL;
+    if (!aligned(dz, 16) || !aligned(w, 16) || !aligned(saved, 16) || !aligned(dx, 16))
+        return CONVBN_EALIGN;
+    const Plan pl = make_plan(desc, pb, CONVBN_PHASE_TUNE_BWD_DATA);
+    CK(check_ws(pl, workspace, workspace_bytes));
+    cudaStream_t st = (cudaStream_t)stream;
+    void *wf = at(workspace, pl.w_scaled);
+    CU(launch_rescale_weight(pb, desc->dtype, w, (const float *)saved, wf, st));
+    CU(launch_direct_dgrad(pb, desc->dtype, desc->layout, dz, wf, dx, st));
+    t_last_kernel[CONVBN_PHASE_TUNE_BWD_DATA] = "direct";
+    return CONVBN_OK;
+}
+
+int convbn_tune_bwd_weight(const convbn_desc *desc, const void *dz, const void *x, const void *w,
+                           const float *b, const float *run_mean, const void *saved, float *dw,
+                           float *db, float *dgamma, float *dbeta, void *workspace,
+                           size_t workspace_bytes, void *stream) {
+    Problem pb;
+    CK(make_problem(desc, &pb));
+    CK(check_pair(desc));
+    if (!dz || !x || !w || !run_mean || !saved || !dw || !dgamma || !dbeta) return CONVBN_EINVAL;
+    if ((b == nullptr) != (db == nullptr)) return CONVBN_EINVAL;
+    if (!aligned(dz, 16) || !aligned(x, 16) || !aligned(w, 16) || !aligned(saved, 16) ||
+        !aligned(dw, 16) || !aligned(b, 4) || !aligned(run_mean, 4) || !aligned(db, 4) ||
+        !aligned(dgamma, 4) || !aligned(dbeta, 4))
+        return CONVBN_EALIGN;
+    const Plan pl = make_plan(desc, pb, CONVBN_PHASE_TUNE_BWD_WEIGHT);
+    CK(check_ws(pl, workspace, workspace_bytes));
+    cudaStream_t st = (cudaStream_t)stream;
+    CK(run_wgrad_partials(desc, pb, pl, dz, x, workspace, st));
+    CU(launch_wgrad_epilogue(pb, desc->dtype, (const float *)at(workspace, pl.partials), pl.splits,
+                             (const float *)at(workspace, pl.bsum), pl.bsplits, w,
+                             (const float *)saved, b, run_mean, dw, db, dgamma, dbeta, st));
+    t_last_kernel[CONVBN_PHASE_TUNE_BWD_WEIGHT] = "direct";
+    return CONVBN_OK;
+}
+
+int convbn_eval_fwd(const convbn_desc *desc, const void *x, const void *w, const float *b,
+                    const float *gamma, const float *beta, const float *run_mean,
+                    const float *run_var, void *z, void *y_saved, void *workspace,
+                    size_t workspace_bytes, void *stream) {
+    Problem pb;
+    CK(make_problem(desc, &pb));
+    CK(check_pair(desc));
+    if (!x || !w || !gamma || !beta || !run_mean || !run_var || !z || !y_saved) return CONVBN_EINVAL;
+    if (!aligned(x, 16) || !aligned(w, 16) || !aligned(z, 16) || !aligned(y_saved, 16) ||
+        !aligned(b, 4) || !aligned(gamma, 4) || !aligned(beta, 4) || !aligned(run_mean, 4) ||
+        !aligned(run_var, 4))
+        return CONVBN_EALIGN;
+    const Plan pl = make_plan(desc, pb, CONVBN_PHASE_EVAL_FWD);
+    CK(check_ws(pl, workspace, workspace_bytes));
+    cudaStream_t st = (cudaStream_t)stream;
+    float *vec3 = (float *)at(workspace, pl.vec3);
+    // BN acts on Y, which already holds the conv bias: shift = beta - mean s
+    CU(launch_reparam(pb, desc->dtype, desc->layout, w, nullptr, gamma, beta, run_mean, run_var, vec3,
+                      nullptr, nullptr, st));
+    CU(launch_direct_fwd(pb, desc->dtype, desc->layout, x, w, b, y_saved, st));
+    CU(launch_bn_eval_fwd(pb, desc->dtype, desc->layout, y_saved, vec3, z, st));
+    t_last_kernel[CONVBN_PHASE_EVAL_FWD] = "direct";
+    return CONVBN_OK;
+}
+
+int convbn_eval_bwd(const convbn_desc *desc, const void *dz, const void *x, const void *y_saved,
+                    const void *w, const float *gamma, const float *run_mean, const float *run_var,
+                    void *dx, float *dw, float *db, float *dgamma, float *dbeta, void *workspace,
+                    size_t workspace_bytes, void *stream) {
+    Problem pb;
+    CK(make_problem(desc, &pb));
+    CK(check_pair(desc));
+    if (!dz || !x || !y_saved || !w || !gamma || !run_mean || !run_var || !dx || !dw || !dgamma || !dbeta)
+        return CONVBN_EINVAL;
+    if (!aligned(dz, 16) || !aligned(x, 16) || !aligned(y_saved, 16) || !aligned(w, 16) ||
+        !aligned(dx, 16) || !aligned(dw, 16) || !aligned(gamma, 4) || !aligned(run_mean, 4) ||
+        !aligned(run_var, 4) || !aligned(db, 4) || !aligned(dgamma, 4) || !aligned(dbeta, 4))
+        return CONVBN_EALIGN;
+    const Plan pl = make_plan(desc, pb, CONVBN_PHASE_EVAL_BWD);
+    CK(check_ws(pl, workspace, workspace_bytes));
+    cudaStream_t st = (cudaStream_t)stream;
+    void *dy = at(workspace, pl.dy);
+    float *pg = (float *)at(workspace, pl.part_g), *pbm = (float *)at(workspace, pl.bsum);
+    CU(launch_bn_eval_bwd(pb, desc->dtype, desc->layout, dz, y_saved, gamma, run_mean, run_var, dy, pg,
+                          pbm, pl.bsplits, st));
+    CU(launch_bn_eval_finish(pb, pg, pbm, pl.bsplits, gamma, run_var, db, dgamma, dbeta, st));
+    CU(launch_direct_dgrad(pb, desc->dtype, desc->layout, dy, w, dx, st));
+    CU(launch_direct_wgrad(pb, desc->dtype, desc->layout, dy, x, (float *)at(workspace, pl.partials),
+                           pl.splits, st));
+    CU(launch_wgrad_epilogue(pb, desc->dtype, (const float *)at(workspace, pl.partials), pl.splits,
+                             nullptr, 0, w, nullptr, nullptr, nullptr, dw, nullptr, nullptr, nullptr, st));
+    t_last_kernel[CONVBN_PHASE_EVAL_BWD] = "direct";
+    return CONVBN_OK;
+}
+
+int convbn_deploy_prepare(const convbn_desc *desc, const void *w, const float *b, const float *gamma,
+                          const float *beta, const float *run_mean, const float *run_var,
+                          void *w_fused, float *b_fused, void *stream) {
+    Problem pb;
+    CK(make_problem(desc, &pb));
+    CK(check_pair(desc));
+    if (!w || !gamma || !beta || !run_mean || !run_var || !w_fused || !b_fused) return CONVBN_EINVAL;
+    if (!aligned(w, 16) || !aligned(w_fused, 16) || !aligned(b, 4) || !aligned(gamma, 4) ||
+        !aligned(beta, 4) || !aligned(run_mean, 4) || !aligned(run_var, 4) || !aligned(b_fused, 4))
+        return CONVBN_EALIGN;
+    CU(launch_reparam(pb, desc->dtype, desc->layout, w, b, gamma, beta, run_mean, run_var, nullptr,
+                      w_fused, b_fused, (cudaStream_t)stream));
+    return CONVBN_OK;
+}
+
+int convbn_deploy_fwd(const convbn_desc *desc, const void *x, const void *w_fused,
+                      const float *b_fused, void *z, void *workspace, size_t workspace_bytes,
+                      void *stream) {
+    Problem pb;
+    CK(make_problem(desc, &pb));
+    CK(check_pair(desc));
+    if (!x || !w_fused || !b_fused || !z) return CONVBN_EINVAL;
+    if (!aligned(x, 16) || !aligned(w_fused, 16) || !aligned(z, 16) || !aligned(b_fused, 4))
+        return CONVBN_EALIGN;
+    const Plan pl = make_plan(desc, pb, CONVBN_PHASE_DEPLOY_FWD);
+    CK(check_ws(pl, workspace, workspace_bytes));
+    CU(launch_direct_fwd(pb, desc->dtype, desc->layout, x, w_fused, b_fused, z, (cudaStream_t)stream));
+    t_last_kernel[CONVBN_PHASE_DEPLOY_FWD] = "direct";
+    return CONVBN_OK;
+}
+
+int convbn_deploy_bwd(const convbn_desc *desc, const void *dz, const void *x, const void *w_fused,
+                      void *dx, float *dw_fused, float *db_fused, void *workspace,
+                      size_t workspace_bytes, void *stream) {
+    Problem pb;
+    CK(make_problem(desc, &pb));
+    CK(check_pair(desc));
+    if (!dz || !x || !w_fused || !dx || !dw_fused || !db_fused) return CONVBN_EINVAL;
+    if (!aligned(dz, 16) || !aligned(x, 16) || !aligned(w_fused, 16) || !aligned(dx, 16) ||
+        !aligned(dw_fused, 16) || !aligned(db_fused, 4))
+        return CONVBN_EALIGN;
+    const Plan pl = make_plan(desc, pb, CONVBN_PHASE_DEPLOY_BWD);
+    CK(check_ws(pl, workspace, workspace_bytes));
+    cudaStream_t st = (cudaStream_t)stream;
+    CU(launch_direct_dgrad(pb, desc->dtype, desc->layout, dz, w_fused, dx, st));
+    CK(run_wgrad_partials(desc, pb, pl, dz, x, workspace, st));
+    CU(launch_wgrad_epilogue(pb, desc->dtype, (const float *)at(workspace, pl.partials), pl.splits,
+                             (const float *)at(workspace, pl.bsum), pl.bsplits, w_fused, nullptr, nullptr,
+                             nullptr, dw_fused, db_fused, nullptr, nullptr, st));
+    t_last_kernel[CONVBN_PHASE_DEPLOY_BWD] = "direct";
+    return CONVBN_OK;
+}
+
+int convbn_check(void *stream) {
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return CONVBN_ECUDA;
+    int word = 0;
+    if (read_and_clear_error_word(&word) != cudaSuccess) return CONVBN_ECUDA;
+    return (word & ERRW_TIMEOUT) ? CONVBN_ETIMEOUT : CONVBN_OK;
+}
+
+const char *convbn_status_string(int status) {
+    switch (status) {
+        case CONVBN_OK: return "ok";
+        case CONVBN_EINVAL: return "invalid descriptor or NULL pointer";
+        case CONVBN_EUNSUPPORTED: return "dtype/layout pair not supported";
+        case CONVBN_EWORKSPACE: return "workspace missing or too small";
+        case CONVBN_EALIGN: return "pointer not aligned as required";
+        case CONVBN_ECUDA: return "CUDA call failed";
+        case CONVBN_ETIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown status";
+    }
+}
+
+const char *convbn_last_kernel(int phase) {
+    if (phase < 0 || phase >= CONVBN_PHASE_COUNT) return "none";
+    return t_last_kernel[phase];
+}
+
+}  // extern "C"

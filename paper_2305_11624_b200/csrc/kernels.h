@@ -1,0 +1,64 @@
+// Host-side launchers of every kernel family.  Each returns the cudaError_t of its launch.
+#pragma once
+
+#include "common.cuh"
+
+namespace convbn {
+
+// ---- per-output-channel reparameterisation (Sec. 3.3 definitions of omega', b') -------------
+// Writes, each if its pointer is non-NULL:
+//   vec3      : [s | b' | r]  (3 * C_out floats)
+//   w_scaled  : omega' in the layout of w, storage dtype
+//   b_fused   : b' alone (C_out floats)
+// scale_weights = false copies omega unscaled (s = 1 for the weight only; used by Eval mode).
+cudaError_t launch_reparam(const Problem &pb, int dtype, int layout, const void *w, const float *b,
+                           const float *gamma, const float *beta, const float *mean,
+                           const float *var, float *vec3, void *w_scaled, float *b_fused,
+                           cudaStream_t st);
+
+// omega' = s omega re-formed from the saved scale vector (first C_out floats of vec3).
+cudaError_t launch_rescale_weight(const Problem &pb, int dtype, const void *w, const float *vec3,
+                                  void *w_scaled, cudaStream_t st);
+
+// ---- direct (one thread per output element) convolution kernels, any shape -----------------
+cudaError_t launch_direct_fwd(const Problem &pb, int dtype, int layout, const void *x,
+                              const void *w, const float *bias, void *z, cudaStream_t st);
+cudaError_t launch_direct_dgrad(const Problem &pb, int dtype, int layout, const void *dz,
+                                const void *w, void *dx, cudaStream_t st);
+int direct_wgrad_splits(const Problem &pb);
+// partials: [splits][C_out][kdim] fp32, row order of the weight layout
+cudaError_t launch_direct_wgrad(const Problem &pb, int dtype, int layout, const void *dz,
+                                const void *x, float *partials, int splits, cudaStream_t st);
+
+// ---- per-channel reductions (Appendix B: backward of a broadcast is a sum) -------------------
+int channel_sum_splits(const Problem &pb);
+// part: [splits][C_out] partial sums of t over pixel slices
+cudaError_t launch_channel_sum_partial(const Problem &pb, int dtype, int layout, const void *t,
+                                       float *part, int splits, cudaStream_t st);
+
+// Finishes the parameter gradients from fp32 partials (fixed summation order):
+//   dwf = sum_splits partials;  dsum = sum_splits bsum_part
+//   tune mode  (vec3 != NULL): dw = s dwf; dbeta = dsum; db = s dsum;
+//                              dgamma = r (sum_k dwf w + dsum (b - mean))
+//   plain mode (vec3 == NULL): dw = dwf; db = dsum (if db != NULL)
+cudaError_t launch_wgrad_epilogue(const Problem &pb, int dtype, const float *partials, int splits,
+                                  const float *bsum_part, int bsplits, const void *w,
+                                  const float *vec3, const float *b, const float *mean, float *dw,
+                                  float *db, float *dgamma, float *dbeta, cudaStream_t st);
+
+// ---- Eval-mode elementwise BatchNorm (Sec. 3.1) ---------------------------------------------
+// z = gamma (y - mean) r + beta
+cudaError_t launch_bn_eval_fwd(const Problem &pb, int dtype, int layout, const void *y,
+                               const float *vec3_eval /* [s | beta - mean s | r] */, void *z,
+                               cudaStream_t st);
+// dy = s dz; part_g[split][c] = sum dz (y - mean) r; part_b[split][c] = sum dz
+cudaError_t launch_bn_eval_bwd(const Problem &pb, int dtype, int layout, const void *dz,
+                               const void *y, const float *gamma, const float *mean,
+                               const float *var, void *dy, float *part_g, float *part_b,
+                               int splits, cudaStream_t st);
+// dgamma = sum part_g; dbeta = sum part_b; db = s dbeta (if db != NULL)
+cudaError_t launch_bn_eval_finish(const Problem &pb, const float *part_g, const float *part_b,
+                                  int splits, const float *gamma, const float *var, float *db,
+                                  float *dgamma, float *dbeta, cudaStream_t st);
+
+}  // namespace convbn

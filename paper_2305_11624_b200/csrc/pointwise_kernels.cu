@@ -1,0 +1,307 @@
+// Per-channel and elementwise kernels: on-the-fly reparameterisation (omega', b'), per-channel
+// sums, the parameter-gradient epilogue of Tune mode, and the Eval-mode BatchNorm passes.
+#include "kernels.h"
+
+namespace convbn {
+
+__device__ int g_error_word = 0;
+
+cudaError_t error_word_address(int **dev_ptr) {
+    return cudaGetSymbolAddress((void **)dev_ptr, g_error_word);
+}
+
+cudaError_t read_and_clear_error_word(int *host_value) {
+    cudaError_t e = cudaMemcpyFromSymbol(host_value, g_error_word, sizeof(int));
+    if (e != cudaSuccess) return e;
+    const int zero = 0;
+    return cudaMemcpyToSymbol(g_error_word, &zero, sizeof(int));
+}
+
+template <class F>
+static cudaError_t by_type(int dtype, F f) {
+    if (dtype == CONVBN_F32) return f((float *)0);
+    if (dtype == CONVBN_BF16) return f((__nv_bfloat16 *)0);
+    return cudaErrorInvalidValue;
+}
+
+// ---- omega' = s omega, b' = (b - mu_hat) s + beta  (Sec. 3.3 definitions, used per step in Tune) ----
+// One block row per output channel (blockIdx.y = co); the weight row keeps its memory order, so
+// the kernel is layout-agnostic.
+template <class T>
+__global__ void __launch_bounds__(256) reparam_kernel(int c_out, int kdim, float eps,
+                                                      const T *__restrict__ w,
+                                                      const float *__restrict__ b,
+                                                      const float *__restrict__ gamma,
+                                                      const float *__restrict__ beta,
+                                                      const float *__restrict__ mean,
+                                                      const float *__restrict__ var,
+                                                      float *__restrict__ vec3,
+                                                      T *__restrict__ w_scaled,
+                                                      float *__restrict__ b_fused) {
+    const int co = blockIdx.y;
+    const float r = 1.0f / sqrtf(var[co] + eps);
+    const float s = gamma[co] * r;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        const float bf = ((b ? b[co] : 0.f) - mean[co]) * s + beta[co];
+        if (vec3) { vec3[co] = s; vec3[c_out + co] = bf; vec3[2 * c_out + co] = r; }
+        if (b_fused) b_fused[co] = bf;
+    }
+    if (w_scaled) {
+        const long long base = (long long)co * kdim;
+        for (int k = blockIdx.x * blockDim.x + threadIdx.x; k < kdim; k += gridDim.x * blockDim.x)
+            w_scaled[base + k] = from_f32<T>(s * to_f32(w[base + k]));
+    }
+}
+
+cudaError_t launch_reparam(const Problem &pb, int dtype, int layout, const void *w, const float *b,
+                           const float *gamma, const float *beta, const float *mean,
+                           const float *var, float *vec3, void *w_scaled, float *b_fused,
+                           cudaStream_t st) {
+    (void)layout;
+    return by_type(dtype, [&](auto *tp) {
+        using T = typename std::remove_pointer<decltype(tp)>::type;
+        int gx = (pb.kdim + 255) / 256;
+        if (gx > 8) gx = 8;
+        if (!w_scaled) gx = 1;
+        dim3 grid(gx, pb.c_out);
+        reparam_kernel<T><<<grid, 256, 0, st>>>(pb.c_out, pb.kdim, pb.eps, (const T *)w, b, gamma,
+                                                beta, mean, var, vec3, (T *)w_scaled, b_fused);
+        return cudaGetLastError();
+    });
+}
+
+template <class T>
+__global__ void __launch_bounds__(256) rescale_weight_kernel(int kdim, const T *__restrict__ w,
+                                                             const float *__restrict__ s_vec,
+                                                             T *__restrict__ w_scaled) {
+    const int co = blockIdx.y;
+    const float s = s_vec[co];
+    const long long base = (long long)co * kdim;
+    for (int k = blockIdx.x * blockDim.x + threadIdx.x; k < kdim; k += gridDim.x * blockDim.x)
+        w_scaled[base + k] = from_f32<T>(s * to_f32(w[base + k]));
+}
+
+cudaError_t launch_rescale_weight(const Problem &pb, int dtype, const void *w, const float *vec3,
+                                  void *w_scaled, cudaStream_t st) {
+    return by_type(dtype, [&](auto *tp) {
+        using T = typename std::remove_pointer<decltype(tp)>::type;
+        int gx = (pb.kdim + 255) / 256;
+        if (gx > 8) gx = 8;
+        rescale_weight_kernel<T><<<dim3(gx, pb.c_out), 256, 0, st>>>(pb.kdim, (const T *)w, vec3, (T *)w_scaled);
+        return cudaGetLastError();
+    });
+}
+
+// ---- per-channel partial sums over pixel slices (Appendix B) --------------------------------
+template <class T, class L>
+__global__ void __launch_bounds__(256) channel_sum_partial_kernel(int c_out, int h_out, int w_out,
+                                                                  long long p, const T *__restrict__ t,
+                                                                  float *__restrict__ part, int splits) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= c_out) return;
+    const int split = blockIdx.y;
+    const long long per = (p + splits - 1) / splits;
+    const long long p0 = split * per, p1 = min(p, p0 + per);
+    float acc = 0.f;
+    if (L::id == CONVBN_NHWC) {
+        for (long long q = p0; q < p1; ++q) acc += to_f32(t[q * c_out + c]);
+    } else {
+        const long long hw = (long long)h_out * w_out;
+        for (long long q = p0; q < p1; ++q) {
+            const long long n = q / hw, i = q % hw;
+            acc += to_f32(t[(n * c_out + c) * hw + i]);
+        }
+    }
+    part[(long long)split * c_out + c] = acc;
+}
+
+int channel_sum_splits(const Problem &pb) {
+    long long want = (148LL * 2048 + pb.c_out - 1) / pb.c_out;
+    long long cap = pb.p / 16;
+    if (cap < 1) cap = 1;
+    if (want > cap) want = cap;
+    if (want > 2048) want = 2048;
+    return (int)(want < 1 ? 1 : want);
+}
+
+cudaError_t launch_channel_sum_partial(const Problem &pb, int dtype, int layout, const void *t,
+                                       float *part, int splits, cudaStream_t st) {
+    const int threads = pb.c_out >= 256 ? 256 : ((pb.c_out + 31) / 32) * 32;
+    dim3 grid((pb.c_out + threads - 1) / threads, splits);
+    if (dtype == CONVBN_F32 && layout == CONVBN_NCHW)
+        channel_sum_partial_kernel<float, NCHW><<<grid, threads, 0, st>>>(
+            pb.c_out, pb.h_out, pb.w_out, pb.p, (const float *)t, part, splits);
+    else if (dtype == CONVBN_BF16 && layout == CONVBN_NHWC)
+        channel_sum_partial_kernel<__nv_bfloat16, NHWC><<<grid, threads, 0, st>>>(
+            pb.c_out, pb.h_out, pb.w_out, pb.p, (const __nv_bfloat16 *)t, part, splits);
+    else
+        return cudaErrorInvalidValue;
+    return cudaGetLastError();
+}
+
+// ---- parameter-gradient epilogue (Table 2, Tune row: domega, db, dgamma, dbeta) -------------
+// One block per output channel.  Partials are added in split order, then the row dot product
+// sum_k domega'[co,k] omega[co,k] is reduced over the block in a fixed tree order.
+template <class T>
+__global__ void __launch_bounds__(256) wgrad_epilogue_kernel(int c_out, int kdim,
+                                                             const float *__restrict__ partials, int splits,
+                                                             const float *__restrict__ bsum_part, int bsplits,
+                                                             const T *__restrict__ w,
+                                                             const float *__restrict__ vec3,
+                                                             const float *__restrict__ b,
+                                                             const float *__restrict__ mean,
+                                                             float *__restrict__ dw, float *__restrict__ db,
+                                                             float *__restrict__ dgamma,
+                                                             float *__restrict__ dbeta) {
+    __shared__ float red[256];
+    const int co = blockIdx.x;
+    const long long rows = (long long)c_out * kdim;
+    const float s = vec3 ? vec3[co] : 1.f;
+    float dot = 0.f;
+    for (int k = threadIdx.x; k < kdim; k += blockDim.x) {
+        const long long o = (long long)co * kdim + k;
+        float acc = 0.f;
+        for (int sp = 0; sp < splits; ++sp) acc += partials[sp * rows + o];
+        dw[o] = s * acc;
+        if (vec3) dot = fmaf(acc, to_f32(w[o]), dot);
+    }
+    float bs = 0.f;
+    if (bsum_part)
+        for (int sp = threadIdx.x; sp < bsplits; sp += blockDim.x) bs += bsum_part[(long long)sp * c_out + co];
+    // two fixed-order block reductions: dot, then bs
+    red[threadIdx.x] = dot;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) { if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o]; __syncthreads(); }
+    const float dot_all = red[0];
+    __syncthreads();
+    red[threadIdx.x] = bs;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) { if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o]; __syncthreads(); }
+    if (threadIdx.x == 0) {
+        const float dsum = red[0];
+        if (vec3) {
+            const float r = vec3[2 * c_out + co];
+            dbeta[co] = dsum;
+            if (db) db[co] = s * dsum;
+            dgamma[co] = r * (dot_all + dsum * ((b ? b[co] : 0.f) - mean[co]));
+        } else if (db) {
+            db[co] = dsum;
+        }
+    }
+}
+
+cudaError_t launch_wgrad_epilogue(const Problem &pb, int dtype, const float *partials, int splits,
+                                  const float *bsum_part, int bsplits, const void *w,
+                                  const float *vec3, const float *b, const float *mean, float *dw,
+                                  float *db, float *dgamma, float *dbeta, cudaStream_t st) {
+    return by_type(dtype, [&](auto *tp) {
+        using T = typename std::remove_pointer<decltype(tp)>::type;
+        wgrad_epilogue_kernel<T><<<pb.c_out, 256, 0, st>>>(pb.c_out, pb.kdim, partials, splits,
+                                                           bsum_part, bsplits, (const T *)w, vec3, b,
+                                                           mean, dw, db, dgamma, dbeta);
+        return cudaGetLastError();
+    });
+}
+
+// ---- Eval-mode BatchNorm, forward: z = s y + (beta - mean s)  (Sec. 3.1) ----------------------
+template <class T, class L>
+__global__ void __launch_bounds__(256) bn_eval_fwd_kernel(int c_out, long long hw, long long total,
+                                                          const T *__restrict__ y,
+                                                          const float *__restrict__ vec3,
+                                                          T *__restrict__ z) {
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        const int c = L::id == CONVBN_NHWC ? (int)(i % c_out) : (int)((i / hw) % c_out);
+        z[i] = from_f32<T>(fmaf(vec3[c], to_f32(y[i]), vec3[c_out + c]));
+    }
+}
+
+cudaError_t launch_bn_eval_fwd(const Problem &pb, int dtype, int layout, const void *y,
+                               const float *vec3, void *z, cudaStream_t st) {
+    const long long total = pb.p * pb.c_out, hw = (long long)pb.h_out * pb.w_out;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148 * 32) blocks = 148 * 32;
+    if (dtype == CONVBN_F32 && layout == CONVBN_NCHW)
+        bn_eval_fwd_kernel<float, NCHW><<<(int)blocks, 256, 0, st>>>(pb.c_out, hw, total, (const float *)y, vec3, (float *)z);
+    else if (dtype == CONVBN_BF16 && layout == CONVBN_NHWC)
+        bn_eval_fwd_kernel<__nv_bfloat16, NHWC><<<(int)blocks, 256, 0, st>>>(
+            pb.c_out, hw, total, (const __nv_bfloat16 *)y, vec3, (__nv_bfloat16 *)z);
+    else
+        return cudaErrorInvalidValue;
+    return cudaGetLastError();
+}
+
+// ---- Eval-mode BatchNorm, backward (Table 2, Eval row) ---------------------------------------
+// dy = s dz, and per pixel slice: part_g = sum dz (y - mean) r, part_b = sum dz.
+template <class T, class L>
+__global__ void __launch_bounds__(256) bn_eval_bwd_kernel(int c_out, int h_out, int w_out, long long p,
+                                                          float eps, const T *__restrict__ dz,
+                                                          const T *__restrict__ y,
+                                                          const float *__restrict__ gamma,
+                                                          const float *__restrict__ mean,
+                                                          const float *__restrict__ var,
+                                                          T *__restrict__ dy, float *__restrict__ part_g,
+                                                          float *__restrict__ part_b, int splits) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= c_out) return;
+    const int split = blockIdx.y;
+    const long long per = (p + splits - 1) / splits;
+    const long long p0 = split * per, p1 = min(p, p0 + per);
+    const float r = 1.0f / sqrtf(var[c] + eps), s = gamma[c] * r, m = mean[c];
+    const long long hw = (long long)h_out * w_out;
+    float ag = 0.f, ab = 0.f;
+    for (long long q = p0; q < p1; ++q) {
+        const long long i = L::id == CONVBN_NHWC ? q * c_out + c : ((q / hw) * c_out + c) * hw + q % hw;
+        const float d = to_f32(dz[i]);
+        dy[i] = from_f32<T>(s * d);
+        ag = fmaf(d, (to_f32(y[i]) - m) * r, ag);
+        ab += d;
+    }
+    part_g[(long long)split * c_out + c] = ag;
+    part_b[(long long)split * c_out + c] = ab;
+}
+
+cudaError_t launch_bn_eval_bwd(const Problem &pb, int dtype, int layout, const void *dz, const void *y,
+                               const float *gamma, const float *mean, const float *var, void *dy,
+                               float *part_g, float *part_b, int splits, cudaStream_t st) {
+    const int threads = pb.c_out >= 256 ? 256 : ((pb.c_out + 31) / 32) * 32;
+    dim3 grid((pb.c_out + threads - 1) / threads, splits);
+    if (dtype == CONVBN_F32 && layout == CONVBN_NCHW)
+        bn_eval_bwd_kernel<float, NCHW><<<grid, threads, 0, st>>>(
+            pb.c_out, pb.h_out, pb.w_out, pb.p, pb.eps, (const float *)dz, (const float *)y, gamma, mean,
+            var, (float *)dy, part_g, part_b, splits);
+    else if (dtype == CONVBN_BF16 && layout == CONVBN_NHWC)
+        bn_eval_bwd_kernel<__nv_bfloat16, NHWC><<<grid, threads, 0, st>>>(
+            pb.c_out, pb.h_out, pb.w_out, pb.p, pb.eps, (const __nv_bfloat16 *)dz,
+            (const __nv_bfloat16 *)y, gamma, mean, var, (__nv_bfloat16 *)dy, part_g, part_b, splits);
+    else
+        return cudaErrorInvalidValue;
+    return cudaGetLastError();
+}
+
+__global__ void bn_eval_finish_kernel(int c_out, float eps, const float *__restrict__ part_g,
+                                      const float *__restrict__ part_b, int splits,
+                                      const float *__restrict__ gamma, const float *__restrict__ var,
+                                      float *__restrict__ db, float *__restrict__ dgamma,
+                                      float *__restrict__ dbeta) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= c_out) return;
+    float g = 0.f, bsum = 0.f;
+    for (int sp = 0; sp < splits; ++sp) {
+        g += part_g[(long long)sp * c_out + c];
+        bsum += part_b[(long long)sp * c_out + c];
+    }
+    dgamma[c] = g;
+    dbeta[c] = bsum;
+    if (db) db[c] = gamma[c] / sqrtf(var[c] + eps) * bsum;
+}
+
+cudaError_t launch_bn_eval_finish(const Problem &pb, const float *part_g, const float *part_b,
+                                  int splits, const float *gamma, const float *var, float *db,
+                                  float *dgamma, float *dbeta, cudaStream_t st) {
+    bn_eval_finish_kernel<<<(pb.c_out + 127) / 128, 128, 0, st>>>(pb.c_out, pb.eps, part_g, part_b, splits,
+                                                                 gamma, var, db, dgamma, dbeta);
+    return cudaGetLastError();
+}
+
+}  // namespace convbn

@@ -1,0 +1,124 @@
+"""GPU parity: the CUDA library against the fp64 CPU oracle, element by element on the same
+seeded inputs, through the C ABI.  Small shapes span several tiles, ragged tails and the
+degenerate cases; the benchmark configurations run at full size."""
+import numpy as np
+import pytest
+
+import parity
+from oracle import oracle as O
+from paper_2305_11624_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+L = I.LayerSpec
+
+SMALL = [
+    # fp32 NCHW (direct kernels)
+    L("f32_bias", 2, 16, 16, 16, 32, 3, 3, pad=1, dtype="f32", layout="nchw", bias=True),
+    L("f32_s2_g2", 3, 8, 13, 11, 12, 3, 3, stride=2, pad=1, groups=2, dtype="f32", layout="nchw", bias=True),
+    L("f32_dil", 1, 5, 12, 9, 7, 3, 3, pad=2, dil=2, dtype="f32", layout="nchw"),
+    L("f32_1x1", 2, 7, 5, 5, 3, 1, 1, dtype="f32", layout="nchw", bias=True),
+    L("f32_one_pixel", 1, 4, 1, 1, 2, 3, 3, pad=1, dtype="f32", layout="nchw"),
+    # bf16 NHWC: tensor-core eligible shapes (channels multiple of 64) with ragged pixel counts
+    L("b_1x1_a", 3, 256, 9, 13, 64, 1, 1),
+    L("b_1x1_b", 2, 64, 17, 15, 256, 1, 1),
+    L("b_1x1_big", 1, 512, 20, 20, 192, 1, 1),
+    L("b_3x3_a", 2, 64, 20, 24, 64, 3, 3, pad=1),
+    L("b_3x3_b", 3, 128, 7, 7, 256, 3, 3, pad=1),
+    L("b_3x3_s2", 2, 128, 21, 18, 128, 3, 3, stride=2, pad=1),
+    L("b_3x3_nopad", 1, 64, 10, 11, 128, 3, 3),
+    L("b_5x5", 1, 64, 12, 12, 64, 5, 5, pad=2),
+    L("b_bias", 2, 64, 8, 8, 64, 3, 3, pad=1, bias=True),
+    # bf16 NHWC: shapes that do not fit the tensor-core tiles
+    L("b_odd_c", 2, 24, 9, 10, 40, 3, 3, pad=1),
+    L("b_stem_like", 2, 3, 30, 30, 64, 7, 7, stride=2, pad=3),
+    L("b_dil", 1, 64, 14, 14, 64, 3, 3, pad=2, dil=2),
+    # depthwise / grouped
+    L("b_dw", 2, 96, 14, 15, 96, 3, 3, pad=1, groups=96),
+    L("b_dw_s2", 1, 32, 9, 9, 32, 3, 3, stride=2, pad=1, groups=32),
+    L("b_grouped", 2, 256, 9, 9, 256, 3, 3, pad=1, groups=32),
+    L("b_grouped_cout2x", 1, 16, 6, 6, 32, 3, 3, pad=1, groups=4),
+]
+
+
+@pytest.mark.parametrize("spec", SMALL, ids=lambda s: s.name)
+def test_tune_small(spec):
+    t = parity.make_inputs(spec, 1234)
+    ref = parity.oracle_tune(spec, t)
+    got = parity.run_tune_gpu(spec, t)
+    parity.compare(got, ref, parity.TOL[spec.dtype], parity.TUNE_OUTPUTS, spec.name)
+
+
+FULL = [(ci, li, sp) for ci, layers in I.CONFIGS.items() for li, sp in enumerate(layers)]
+
+
+@pytest.mark.parametrize("ci,li,spec", FULL, ids=lambda v: v.name if isinstance(v, L) else None)
+def test_tune_benchmark_configs_full_size(ci, li, spec):
+    """All five configurations at full size, every element of every output tensor."""
+    t = parity.make_inputs(spec, I.config_seed(ci, li))
+    ref = parity.oracle_tune(spec, t)
+    got = parity.run_tune_gpu(spec, t)
+    errs = parity.compare(got, ref, parity.TOL[spec.dtype], parity.TUNE_OUTPUTS, spec.name)
+    print(spec.name, got["_kernels"], {k: "%.2e" % v for k, v in errs.items()})
+
+
+def test_tune_is_deterministic_and_leaves_inputs_alone():
+    from paper_2305_11624_b200.harness import Block
+    import torch
+    spec = L("det", 2, 64, 20, 24, 64, 3, 3, pad=1)
+    t = parity.make_inputs(spec, 5)
+    blk = Block(spec)
+    blk.load(t)
+    before = {k: getattr(blk, k).clone() for k in ("x", "w", "dz", "gamma", "beta", "mu_hat", "var_hat")}
+    outs = []
+    for _ in range(2):
+        blk.tune_step()
+        torch.cuda.synchronize()
+        outs.append({k: getattr(blk, k).clone() for k in ("z", "dx", "dw", "dgamma", "dbeta")})
+    for k in outs[0]:
+        assert torch.equal(outs[0][k], outs[1][k]), k
+    for k, v in before.items():
+        assert torch.equal(getattr(blk, k), v), k
+
+
+@pytest.mark.parametrize("spec", [SMALL[0], SMALL[8], SMALL[10], SMALL[17], SMALL[19]], ids=lambda s: s.name)
+def test_eval_and_deploy_comparators(spec):
+    """Eval and Deploy entry points against the oracle's Eval-row and Deploy-row equations, and
+    the paper's claim Z_eval = Z_deploy = Z_tune on the device outputs themselves."""
+    from paper_2305_11624_b200.harness import Block
+    from paper_2305_11624_b200 import convbn as C
+    tol = parity.TOL[spec.dtype]
+    t = parity.make_inputs(spec, 77)
+    s = parity.oracle_shape(spec)
+    p = dict(gamma=t["gamma"], beta=t["beta"], mu_hat=t["mu_hat"], var_hat=t["var_hat"])
+    ev = O.eval_forward(s, t["x"], t["w"], t["b"], **p)
+    ge = O.eval_backward(s, t["dz"], t["x"], ev["y"], t["w"], t["gamma"], t["mu_hat"], t["var_hat"],
+                         with_bias=spec.bias)
+    blk = Block(spec, modes=("tune", "eval", "deploy"))
+    blk.load(t)
+    blk.eval_fwd()
+    z_eval = blk.fetch("z")
+    assert O.rel_l2(blk.fetch("y_saved"), ev["y"]) <= tol
+    assert O.rel_l2(z_eval, ev["z"]) <= tol
+    blk.eval_bwd()
+    got = {k: blk.fetch(k) for k in ("dx", "dw", "dgamma", "dbeta")}
+    got["db"] = blk.fetch("db") if spec.bias else None
+    parity.compare(got, ge, 2 * tol if spec.dtype == "bf16" else tol, ("dx", "dw", "db", "dgamma", "dbeta"),
+                   spec.name + "/eval")
+    w_f, b_f = O.fold(s, t["w"], t["b"], **p)
+    gd = O.deploy_backward(s, t["dz"], t["x"], w_f)
+    blk.deploy_prepare(); blk.deploy_fwd()
+    z_dep = blk.fetch("z")
+    assert O.rel_l2(blk.fetch("w_fused"), w_f) <= tol
+    assert O.rel_l2(blk.fetch("b_fused"), b_f) <= 1e-5
+    assert O.rel_l2(z_dep, ev["z"]) <= tol
+    blk.deploy_bwd()
+    assert O.rel_l2(blk.fetch("dx"), gd["dx"]) <= tol
+    assert O.rel_l2(blk.fetch("dw_fused"), gd["dw_f"]) <= tol
+    assert O.rel_l2(blk.fetch("db_fused"), gd["db_f"]) <= tol
+    blk.tune_fwd()
+    z_tune = blk.fetch("z")
+    C.convbn_check()
+    assert O.rel_l2(z_tune, z_dep) <= tol and O.rel_l2(z_tune, z_eval) <= 2 * tol
+    assert blk.saved_bytes("tune") < blk.saved_bytes("eval")
+    assert blk.saved_bytes("tune") - blk.saved_bytes("deploy") == 3 * spec.c_out * 4
