@@ -161,6 +161,34 @@ int convbn_deploy_bwd(const convbn_desc *desc, const void *dz, const void *x,
                       const void *w_fused, void *dx, float *dw_fused, float *db_fused,
                       void *workspace, size_t workspace_bytes, void *stream);
 
+/* ---- one Tune-mode training step from HOST buffers ------------------------------------------- */
+
+/* Device bytes convbn_tune_step_host needs in `device_arena`.  0 for an invalid descriptor. */
+size_t convbn_host_step_arena_bytes(const convbn_desc *desc);
+
+/* Forward, backward-data and backward-weight of one block (the three Tune-row calls above, Sec. 3.4
+ * and Table 2) with every tensor in HOST memory: x, dz, w, b (NULL = no bias), gamma, beta,
+ * run_mean, run_var are host inputs; z, dx, dw, db (NULL iff b is NULL), dgamma, dbeta are host
+ * outputs, in the dtype / layout conventions above.  Copies are asynchronous on `stream` (use
+ * page-locked host memory for them to overlap); outputs are valid once the stream has been
+ * synchronised.  `device_arena` is caller-owned DEVICE scratch of at least
+ * convbn_host_step_arena_bytes(desc) bytes, 256-byte aligned. */
+int convbn_tune_step_host(const convbn_desc *desc, const void *x, const void *dz, const void *w,
+                          const float *b, const float *gamma, const float *beta,
+                          const float *run_mean, const float *run_var, void *z, void *dx, float *dw,
+                          float *db, float *dgamma, float *dbeta, void *device_arena,
+                          size_t arena_bytes, void *stream);
+
+/* ---- measurement aid (the paper has no counterpart) ------------------------------------------ */
+
+/* After convbn_profile_begin(), every kernel this library launches (from any thread) is bracketed
+ * by a pair of CUDA events on its stream.  convbn_profile_end() stops that, synchronises the
+ * device and writes one line per kernel family into `report` (host buffer, NUL-terminated,
+ * truncated to report_bytes): "<name> <launches> <total milliseconds>\n".  At most 65536
+ * launches are recorded between begin and end; later ones run unrecorded. */
+int convbn_profile_begin(void);
+int convbn_profile_end(char *report, size_t report_bytes);
+
 /* ---- housekeeping -------------------------------------------------------------------------- */
 
 /* Synchronises `stream`, then reads and clears the device error word of the current device.

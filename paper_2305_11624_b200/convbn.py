@@ -23,7 +23,8 @@ EXPORTS = (
     "convbn_out_shape", "convbn_saved_bytes", "convbn_workspace_bytes", "convbn_tune_fwd",
     "convbn_tune_bwd_data", "convbn_tune_bwd_weight", "convbn_eval_fwd", "convbn_eval_bwd",
     "convbn_deploy_prepare", "convbn_deploy_fwd", "convbn_deploy_bwd", "convbn_check",
-    "convbn_status_string", "convbn_last_kernel",
+    "convbn_status_string", "convbn_last_kernel", "convbn_host_step_arena_bytes",
+    "convbn_tune_step_host", "convbn_profile_begin", "convbn_profile_end",
 )
 
 
@@ -59,6 +60,7 @@ def lib():
         L = ctypes.CDLL(LIBRARY)
         L.convbn_saved_bytes.restype = ctypes.c_size_t
         L.convbn_workspace_bytes.restype = ctypes.c_size_t
+        L.convbn_host_step_arena_bytes.restype = ctypes.c_size_t
         L.convbn_status_string.restype = ctypes.c_char_p
         L.convbn_last_kernel.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -188,3 +190,34 @@ def convbn_deploy_bwd(desc, dz, x, w_fused, dx, dw_fused, db_fused, workspace=No
 
 def convbn_check(stream=None) -> None:
     _raise(lib().convbn_check(_stream(stream)), "convbn_check")
+
+
+def convbn_host_step_arena_bytes(desc: Desc) -> int:
+    return int(lib().convbn_host_step_arena_bytes(ctypes.byref(desc)))
+
+
+def convbn_tune_step_host(desc, x, dz, w, b, gamma, beta, run_mean, run_var, z, dx, dw, db, dgamma,
+                          dbeta, device_arena, arena_bytes: Optional[int] = None, stream=None):
+    """All tensors but ``device_arena`` are HOST tensors (page-locked for asynchronous copies)."""
+    ab = _nbytes(device_arena) if arena_bytes is None else arena_bytes
+    _raise(lib().convbn_tune_step_host(ctypes.byref(desc), _ptr(x), _ptr(dz), _ptr(w), _ptr(b),
+                                       _ptr(gamma), _ptr(beta), _ptr(run_mean), _ptr(run_var),
+                                       _ptr(z), _ptr(dx), _ptr(dw), _ptr(db), _ptr(dgamma),
+                                       _ptr(dbeta), _ptr(device_arena), ctypes.c_size_t(ab),
+                                       _stream(stream)),
+           "convbn_tune_step_host")
+
+
+def convbn_profile_begin() -> None:
+    _raise(lib().convbn_profile_begin(), "convbn_profile_begin")
+
+
+def convbn_profile_end() -> dict:
+    """{kernel family: (launches, total milliseconds)} since convbn_profile_begin()."""
+    buf = ctypes.create_string_buffer(1 << 16)
+    _raise(lib().convbn_profile_end(buf, ctypes.c_size_t(len(buf))), "convbn_profile_end")
+    out = {}
+    for line in buf.value.decode().splitlines():
+        name, count, ms = line.split()
+        out[name] = (int(count), float(ms))
+    return out

@@ -1,7 +1,13 @@
 // C ABI of the ConvBN library: host-side validation, workspace planning, kernel selection.
 // Every step of every entry point runs in this library's own kernels; there is no CPU path.
 #include <stdint.h>
+#include <stdio.h>
 #include <string.h>
+
+#include <map>
+#include <mutex>
+#include <string>
+#include <vector>
 
 #include "kernels.h"
 
@@ -100,6 +106,36 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
     return pl;
 }
 
+// Device arena of the host-buffer entry point: every tensor of one block plus saved + workspace.
+struct HostArena {
+    size_t total = 0, x = 0, dz = 0, w = 0, b = 0, gamma = 0, beta = 0, mean = 0, var = 0, z = 0, dx = 0,
+           dw = 0, db = 0, dgamma = 0, dbeta = 0, saved = 0, ws = 0;
+    size_t x_bytes = 0, z_bytes = 0, w_bytes = 0, dw_bytes = 0, ws_bytes = 0;
+};
+
+HostArena make_host_arena(const convbn_desc *d, const Problem &pb) {
+    HostArena a;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    const size_t es = elem_size(d->dtype), vb = (size_t)pb.c_out * sizeof(float);
+    a.x_bytes = (size_t)pb.pin * pb.c_in * es;
+    a.z_bytes = (size_t)pb.p * pb.c_out * es;
+    a.w_bytes = (size_t)pb.c_out * pb.kdim * es;
+    a.dw_bytes = (size_t)pb.c_out * pb.kdim * sizeof(float);
+    a.x = take(a.x_bytes); a.dz = take(a.z_bytes); a.w = take(a.w_bytes);
+    a.b = take(vb); a.gamma = take(vb); a.beta = take(vb); a.mean = take(vb); a.var = take(vb);
+    a.z = take(a.z_bytes); a.dx = take(a.x_bytes); a.dw = take(a.dw_bytes);
+    a.db = take(vb); a.dgamma = take(vb); a.dbeta = take(vb);
+    a.saved = take(3 * vb);
+    for (int ph = CONVBN_PHASE_TUNE_FWD; ph <= CONVBN_PHASE_TUNE_BWD_WEIGHT; ++ph) {
+        const size_t t = make_plan(d, pb, ph).total;
+        if (t > a.ws_bytes) a.ws_bytes = t;
+    }
+    a.ws = take(a.ws_bytes);
+    a.total = off;
+    return a;
+}
+
 int check_ws(const Plan &pl, const void *ws, size_t ws_bytes) {
     if (pl.total == 0) return CONVBN_OK;
     if (!ws || ws_bytes < pl.total) return CONVBN_EWORKSPACE;
@@ -107,6 +143,39 @@ int check_ws(const Plan &pl, const void *ws, size_t ws_bytes) {
     return CONVBN_OK;
 }
 
+// ---- optional per-kernel timing (CUDA events around every launch this library makes) ----------
+struct ProfRec { cudaEvent_t a, b; const char *name; };
+struct Profiler {
+    bool on = false;
+    std::vector<ProfRec> recs;
+};
+Profiler g_prof;
+std::mutex g_prof_mu;
+const size_t kProfCap = 1 << 16;
+
+struct ProfScope {
+    cudaStream_t st;
+    bool live = false;
+    ProfRec rec{};
+    ProfScope(const char *name, cudaStream_t s) : st(s) {
+        if (!g_prof.on) return;
+        std::lock_guard<std::mutex> lk(g_prof_mu);
+        if (!g_prof.on || g_prof.recs.size() >= kProfCap) return;
+        if (cudaEventCreate(&rec.a) != cudaSuccess) return;
+        if (cudaEventCreate(&rec.b) != cudaSuccess) { cudaEventDestroy(rec.a); return; }
+        rec.name = name;
+        cudaEventRecord(rec.a, st);
+        live = true;
+    }
+    ~ProfScope() {
+        if (!live) return;
+        cudaEventRecord(rec.b, st);
+        std::lock_guard<std::mutex> lk(g_prof_mu);
+        g_prof.recs.push_back(rec);
+    }
+};
+
+#define LAUNCH(name, call) do { ProfScope _ps(name, st); if ((call) != cudaSuccess) return CONVBN_ECUDA; } while (0)
 #define CK(expr) do { int _s = (expr); if (_s != CONVBN_OK) return _s; } while (0)
 #define CU(expr) do { if ((expr) != cudaSuccess) return CONVBN_ECUDA; } while (0)
 
@@ -115,8 +184,8 @@ inline char *at(void *ws, size_t off) { return (char *)ws + off; }
 // Shared by Tune and Deploy backward-weight: conv weight gradient partials + per-channel dZ sums.
 int run_wgrad_partials(const convbn_desc *d, const Problem &pb, const Plan &pl, const void *dz,
                        const void *x, void *ws, cudaStream_t st) {
-    CU(launch_direct_wgrad(pb, d->dtype, d->layout, dz, x, (float *)at(ws, pl.partials), pl.splits, st));
-    CU(launch_channel_sum_partial(pb, d->dtype, d->layout, dz, (float *)at(ws, pl.bsum), pl.bsplits, st));
+    LAUNCH("direct_wgrad", launch_direct_wgrad(pb, d->dtype, d->layout, dz, x, (float *)at(ws, pl.partials), pl.splits, st));
+    LAUNCH("channel_sum", launch_channel_sum_partial(pb, d->dtype, d->layout, dz, (float *)at(ws, pl.bsum), pl.bsplits, st));
     return CONVBN_OK;
 }
 
@@ -167,9 +236,9 @@ int convbn_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const
     cudaStream_t st = (cudaStream_t)stream;
     float *vec3 = (float *)saved;
     void *wf = at(workspace, pl.w_scaled);
-    CU(launch_reparam(pb, desc->dtype, desc->layout, w, b, gamma, beta, run_mean, run_var, vec3, wf,
+    LAUNCH("reparam", launch_reparam(pb, desc->dtype, desc->layout, w, b, gamma, beta, run_mean, run_var, vec3, wf,
                       nullptr, st));
-    CU(launch_direct_fwd(pb, desc->dtype, desc->layout, x, wf, vec3 + pb.c_out, z, st));
+    LAUNCH("direct_fwd", launch_direct_fwd(pb, desc->dtype, desc->layout, x, wf, vec3 + pb.c_out, z, st));
     t_last_kernel[CONVBN_PHASE_TUNE_FWD] = "direct";
     return CONVBN_OK;
 }
@@ -186,8 +255,8 @@ int convbn_tune_bwd_data(const convbn_desc *desc, const void *dz, const void *w,
     CK(check_ws(pl, workspace, workspace_bytes));
     cudaStream_t st = (cudaStream_t)stream;
     void *wf = at(workspace, pl.w_scaled);
-    CU(launch_rescale_weight(pb, desc->dtype, w, (const float *)saved, wf, st));
-    CU(launch_direct_dgrad(pb, desc->dtype, desc->layout, dz, wf, dx, st));
+    LAUNCH("rescale_weight", launch_rescale_weight(pb, desc->dtype, w, (const float *)saved, wf, st));
+    LAUNCH("direct_dgrad", launch_direct_dgrad(pb, desc->dtype, desc->layout, dz, wf, dx, st));
     t_last_kernel[CONVBN_PHASE_TUNE_BWD_DATA] = "direct";
     return CONVBN_OK;
 }
@@ -209,7 +278,7 @@ int convbn_tune_bwd_weight(const convbn_desc *desc, const void *dz, const void *
     CK(check_ws(pl, workspace, workspace_bytes));
     cudaStream_t st = (cudaStream_t)stream;
     CK(run_wgrad_partials(desc, pb, pl, dz, x, workspace, st));
-    CU(launch_wgrad_epilogue(pb, desc->dtype, (const float *)at(workspace, pl.partials), pl.splits,
+    LAUNCH("wgrad_epilogue", launch_wgrad_epilogue(pb, desc->dtype, (const float *)at(workspace, pl.partials), pl.splits,
                              (const float *)at(workspace, pl.bsum), pl.bsplits, w,
                              (const float *)saved, b, run_mean, dw, db, dgamma, dbeta, st));
     t_last_kernel[CONVBN_PHASE_TUNE_BWD_WEIGHT] = "direct";
@@ -233,10 +302,10 @@ int convbn_eval_fwd(const convbn_desc *desc, const void *x, const void *w, const
     cudaStream_t st = (cudaStream_t)stream;
     float *vec3 = (float *)at(workspace, pl.vec3);
     // BN acts on Y, which already holds the conv bias: shift = beta - mean s
-    CU(launch_reparam(pb, desc->dtype, desc->layout, w, nullptr, gamma, beta, run_mean, run_var, vec3,
+    LAUNCH("reparam", launch_reparam(pb, desc->dtype, desc->layout, w, nullptr, gamma, beta, run_mean, run_var, vec3,
                       nullptr, nullptr, st));
-    CU(launch_direct_fwd(pb, desc->dtype, desc->layout, x, w, b, y_saved, st));
-    CU(launch_bn_eval_fwd(pb, desc->dtype, desc->layout, y_saved, vec3, z, st));
+    LAUNCH("direct_fwd", launch_direct_fwd(pb, desc->dtype, desc->layout, x, w, b, y_saved, st));
+    LAUNCH("bn_eval_fwd", launch_bn_eval_fwd(pb, desc->dtype, desc->layout, y_saved, vec3, z, st));
     t_last_kernel[CONVBN_PHASE_EVAL_FWD] = "direct";
     return CONVBN_OK;
 }
@@ -259,13 +328,13 @@ int convbn_eval_bwd(const convbn_desc *desc, const void *dz, const void *x, cons
     cudaStream_t st = (cudaStream_t)stream;
     void *dy = at(workspace, pl.dy);
     float *pg = (float *)at(workspace, pl.part_g), *pbm = (float *)at(workspace, pl.bsum);
-    CU(launch_bn_eval_bwd(pb, desc->dtype, desc->layout, dz, y_saved, gamma, run_mean, run_var, dy, pg,
+    LAUNCH("bn_eval_bwd", launch_bn_eval_bwd(pb, desc->dtype, desc->layout, dz, y_saved, gamma, run_mean, run_var, dy, pg,
                           pbm, pl.bsplits, st));
-    CU(launch_bn_eval_finish(pb, pg, pbm, pl.bsplits, gamma, run_var, db, dgamma, dbeta, st));
-    CU(launch_direct_dgrad(pb, desc->dtype, desc->layout, dy, w, dx, st));
-    CU(launch_direct_wgrad(pb, desc->dtype, desc->layout, dy, x, (float *)at(workspace, pl.partials),
+    LAUNCH("bn_eval_finish", launch_bn_eval_finish(pb, pg, pbm, pl.bsplits, gamma, run_var, db, dgamma, dbeta, st));
+    LAUNCH("direct_dgrad", launch_direct_dgrad(pb, desc->dtype, desc->layout, dy, w, dx, st));
+    LAUNCH("direct_wgrad", launch_direct_wgrad(pb, desc->dtype, desc->layout, dy, x, (float *)at(workspace, pl.partials),
                            pl.splits, st));
-    CU(launch_wgrad_epilogue(pb, desc->dtype, (const float *)at(workspace, pl.partials), pl.splits,
+    LAUNCH("wgrad_epilogue", launch_wgrad_epilogue(pb, desc->dtype, (const float *)at(workspace, pl.partials), pl.splits,
                              nullptr, 0, w, nullptr, nullptr, nullptr, dw, nullptr, nullptr, nullptr, st));
     t_last_kernel[CONVBN_PHASE_EVAL_BWD] = "direct";
     return CONVBN_OK;
@@ -281,8 +350,9 @@ int convbn_deploy_prepare(const convbn_desc *desc, const void *w, const float *b
     if (!aligned(w, 16) || !aligned(w_fused, 16) || !aligned(b, 4) || !aligned(gamma, 4) ||
         !aligned(beta, 4) || !aligned(run_mean, 4) || !aligned(run_var, 4) || !aligned(b_fused, 4))
         return CONVBN_EALIGN;
-    CU(launch_reparam(pb, desc->dtype, desc->layout, w, b, gamma, beta, run_mean, run_var, nullptr,
-                      w_fused, b_fused, (cudaStream_t)stream));
+    cudaStream_t st = (cudaStream_t)stream;
+    LAUNCH("reparam", launch_reparam(pb, desc->dtype, desc->layout, w, b, gamma, beta, run_mean, run_var, nullptr,
+                      w_fused, b_fused, st));
     return CONVBN_OK;
 }
 
@@ -297,7 +367,8 @@ int convbn_deploy_fwd(const convbn_desc *desc, const void *x, const void *w_fuse
         return CONVBN_EALIGN;
     const Plan pl = make_plan(desc, pb, CONVBN_PHASE_DEPLOY_FWD);
     CK(check_ws(pl, workspace, workspace_bytes));
-    CU(launch_direct_fwd(pb, desc->dtype, desc->layout, x, w_fused, b_fused, z, (cudaStream_t)stream));
+    cudaStream_t st = (cudaStream_t)stream;
+    LAUNCH("direct_fwd", launch_direct_fwd(pb, desc->dtype, desc->layout, x, w_fused, b_fused, z, st));
     t_last_kernel[CONVBN_PHASE_DEPLOY_FWD] = "direct";
     return CONVBN_OK;
 }
@@ -315,9 +386,9 @@ int convbn_deploy_bwd(const convbn_desc *desc, const void *dz, const void *x, co
     const Plan pl = make_plan(desc, pb, CONVBN_PHASE_DEPLOY_BWD);
     CK(check_ws(pl, workspace, workspace_bytes));
     cudaStream_t st = (cudaStream_t)stream;
-    CU(launch_direct_dgrad(pb, desc->dtype, desc->layout, dz, w_fused, dx, st));
+    LAUNCH("direct_dgrad", launch_direct_dgrad(pb, desc->dtype, desc->layout, dz, w_fused, dx, st));
     CK(run_wgrad_partials(desc, pb, pl, dz, x, workspace, st));
-    CU(launch_wgrad_epilogue(pb, desc->dtype, (const float *)at(workspace, pl.partials), pl.splits,
+    LAUNCH("wgrad_epilogue", launch_wgrad_epilogue(pb, desc->dtype, (const float *)at(workspace, pl.partials), pl.splits,
                              (const float *)at(workspace, pl.bsum), pl.bsplits, w_fused, nullptr, nullptr,
                              nullptr, dw_fused, db_fused, nullptr, nullptr, st));
     t_last_kernel[CONVBN_PHASE_DEPLOY_BWD] = "direct";
@@ -329,6 +400,99 @@ int convbn_check(void *stream) {
     int word = 0;
     if (read_and_clear_error_word(&word) != cudaSuccess) return CONVBN_ECUDA;
     return (word & ERRW_TIMEOUT) ? CONVBN_ETIMEOUT : CONVBN_OK;
+}
+
+int convbn_profile_begin(void) {
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    for (auto &r : g_prof.recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    g_prof.recs.clear();
+    g_prof.on = true;
+    return CONVBN_OK;
+}
+
+int convbn_profile_end(char *report, size_t report_bytes) {
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    g_prof.on = false;
+    int status = CONVBN_OK;
+    if (cudaDeviceSynchronize() != cudaSuccess) status = CONVBN_ECUDA;
+    std::map<std::string, std::pair<long long, double>> agg;
+    for (auto &r : g_prof.recs) {
+        float ms = 0.f;
+        if (status == CONVBN_OK && cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess) {
+            auto &e = agg[r.name];
+            e.first += 1;
+            e.second += ms;
+        }
+        cudaEventDestroy(r.a);
+        cudaEventDestroy(r.b);
+    }
+    g_prof.recs.clear();
+    if (report && report_bytes) {
+        size_t off = 0;
+        report[0] = 0;
+        for (auto &kv : agg) {
+            int n = snprintf(report + off, report_bytes - off, "%s %lld %.6f\n", kv.first.c_str(),
+                             kv.second.first, kv.second.second);
+            if (n < 0 || (size_t)n >= report_bytes - off) { report[off] = 0; break; }
+            off += (size_t)n;
+        }
+    }
+    return status;
+}
+
+size_t convbn_host_step_arena_bytes(const convbn_desc *desc) {
+    Problem pb;
+    if (make_problem(desc, &pb) != CONVBN_OK) return 0;
+    return make_host_arena(desc, pb).total;
+}
+
+int convbn_tune_step_host(const convbn_desc *desc, const void *x, const void *dz, const void *w,
+                          const float *b, const float *gamma, const float *beta,
+                          const float *run_mean, const float *run_var, void *z, void *dx, float *dw,
+                          float *db, float *dgamma, float *dbeta, void *device_arena,
+                          size_t arena_bytes, void *stream) {
+    Problem pb;
+    CK(make_problem(desc, &pb));
+    CK(check_pair(desc));
+    if (!x || !dz || !w || !gamma || !beta || !run_mean || !run_var || !z || !dx || !dw || !dgamma || !dbeta)
+        return CONVBN_EINVAL;
+    if ((b == nullptr) != (db == nullptr)) return CONVBN_EINVAL;
+    const HostArena ar = make_host_arena(desc, pb);
+    if (!device_arena || arena_bytes < ar.total) return CONVBN_EWORKSPACE;
+    if (!aligned(device_arena, 256)) return CONVBN_EALIGN;
+    cudaStream_t st = (cudaStream_t)stream;
+    char *d = (char *)device_arena;
+    const size_t vb = (size_t)pb.c_out * sizeof(float);
+    auto h2d = [&](size_t off, const void *src, size_t bytes) {
+        return cudaMemcpyAsync(d + off, src, bytes, cudaMemcpyHostToDevice, st);
+    };
+    auto d2h = [&](void *dst, size_t off, size_t bytes) {
+        return cudaMemcpyAsync(dst, d + off, bytes, cudaMemcpyDeviceToHost, st);
+    };
+    CU(h2d(ar.x, x, ar.x_bytes));
+    CU(h2d(ar.w, w, ar.w_bytes));
+    CU(h2d(ar.gamma, gamma, vb));
+    CU(h2d(ar.beta, beta, vb));
+    CU(h2d(ar.mean, run_mean, vb));
+    CU(h2d(ar.var, run_var, vb));
+    if (b) CU(h2d(ar.b, b, vb));
+    const float *db_dev = b ? (const float *)(d + ar.b) : nullptr;
+    CK(convbn_tune_fwd(desc, d + ar.x, d + ar.w, db_dev, (const float *)(d + ar.gamma),
+                       (const float *)(d + ar.beta), (const float *)(d + ar.mean),
+                       (const float *)(d + ar.var), d + ar.z, d + ar.saved, d + ar.ws, ar.ws_bytes, stream));
+    CU(d2h(z, ar.z, ar.z_bytes));
+    CU(h2d(ar.dz, dz, ar.z_bytes));
+    CK(convbn_tune_bwd_data(desc, d + ar.dz, d + ar.w, d + ar.saved, d + ar.dx, d + ar.ws, ar.ws_bytes, stream));
+    CU(d2h(dx, ar.dx, ar.x_bytes));
+    CK(convbn_tune_bwd_weight(desc, d + ar.dz, d + ar.x, d + ar.w, db_dev, (const float *)(d + ar.mean),
+                              d + ar.saved, (float *)(d + ar.dw), b ? (float *)(d + ar.db) : nullptr,
+                              (float *)(d + ar.dgamma), (float *)(d + ar.dbeta), d + ar.ws, ar.ws_bytes,
+                              stream));
+    CU(d2h(dw, ar.dw, ar.dw_bytes));
+    CU(d2h(dgamma, ar.dgamma, vb));
+    CU(d2h(dbeta, ar.dbeta, vb));
+    if (db) CU(d2h(db, ar.db, vb));
+    return CONVBN_OK;
 }
 
 const char *convbn_status_string(int status) {
