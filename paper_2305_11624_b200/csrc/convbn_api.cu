@@ -18,6 +18,39 @@ namespace {
 thread_local const char *t_last_kernel[CONVBN_PHASE_COUNT] = {"none", "none", "none", "none",
                                                               "none", "none", "none"};
 
+// ---- optional per-kernel timing (CUDA events around every launch this library makes) ----------
+struct ProfRec { cudaEvent_t a, b; std::string name; };
+thread_local char t_prof_tag[96] = "";   // shape key of the API call in progress
+struct Profiler {
+    bool on = false;
+    std::vector<ProfRec> recs;
+};
+Profiler g_prof;
+std::mutex g_prof_mu;
+const size_t kProfCap = 1 << 16;
+
+struct ProfScope {
+    cudaStream_t st;
+    bool live = false;
+    ProfRec rec{};
+    ProfScope(const char *name, cudaStream_t s) : st(s) {
+        if (!g_prof.on) return;
+        std::lock_guard<std::mutex> lk(g_prof_mu);
+        if (!g_prof.on || g_prof.recs.size() >= kProfCap) return;
+        if (cudaEventCreate(&rec.a) != cudaSuccess) return;
+        if (cudaEventCreate(&rec.b) != cudaSuccess) { cudaEventDestroy(rec.a); return; }
+        rec.name = std::string(name) + "@" + t_prof_tag;
+        cudaEventRecord(rec.a, st);
+        live = true;
+    }
+    ~ProfScope() {
+        if (!live) return;
+        cudaEventRecord(rec.b, st);
+        std::lock_guard<std::mutex> lk(g_prof_mu);
+        g_prof.recs.push_back(rec);
+    }
+};
+
 inline bool aligned(const void *p, size_t a) { return ((uintptr_t)p % a) == 0; }
 inline size_t elem_size(int dtype) { return dtype == CONVBN_F32 ? 4 : 2; }
 
@@ -50,6 +83,9 @@ int make_problem(const convbn_desc *d, Problem *pb) {
         return CONVBN_EINVAL;
     pb->kdim = (int)kdim;
     pb->eps = (float)d->eps;
+    if (g_prof.on)
+        snprintf(t_prof_tag, sizeof(t_prof_tag), "n%d_c%d_%dx%d_o%d_k%dx%d_s%d_g%d", d->n, d->c_in,
+                 d->h_in, d->w_in, d->c_out, d->kh, d->kw, d->stride_h, d->groups);
     return CONVBN_OK;
 }
 
@@ -142,38 +178,6 @@ int check_ws(const Plan &pl, const void *ws, size_t ws_bytes) {
     if (!aligned(ws, 256)) return CONVBN_EALIGN;
     return CONVBN_OK;
 }
-
-// ---- optional per-kernel timing (CUDA events around every launch this library makes) ----------
-struct ProfRec { cudaEvent_t a, b; const char *name; };
-struct Profiler {
-    bool on = false;
-    std::vector<ProfRec> recs;
-};
-Profiler g_prof;
-std::mutex g_prof_mu;
-const size_t kProfCap = 1 << 16;
-
-struct ProfScope {
-    cudaStream_t st;
-    bool live = false;
-    ProfRec rec{};
-    ProfScope(const char *name, cudaStream_t s) : st(s) {
-        if (!g_prof.on) return;
-        std::lock_guard<std::mutex> lk(g_prof_mu);
-        if (!g_prof.on || g_prof.recs.size() >= kProfCap) return;
-        if (cudaEventCreate(&rec.a) != cudaSuccess) return;
-        if (cudaEventCreate(&rec.b) != cudaSuccess) { cudaEventDestroy(rec.a); return; }
-        rec.name = name;
-        cudaEventRecord(rec.a, st);
-        live = true;
-    }
-    ~ProfScope() {
-        if (!live) return;
-        cudaEventRecord(rec.b, st);
-        std::lock_guard<std::mutex> lk(g_prof_mu);
-        g_prof.recs.push_back(rec);
-    }
-};
 
 #define LAUNCH(name, call) do { ProfScope _ps(name, st); if ((call) != cudaSuccess) return CONVBN_ECUDA; } while (0)
 #define CK(expr) do { int _s = (expr); if (_s != CONVBN_OK) return _s; } while (0)
