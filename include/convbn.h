@@ -52,7 +52,8 @@ typedef enum {
     CONVBN_EWORKSPACE = 3,   /* workspace missing or too small                      */
     CONVBN_EALIGN = 4,       /* pointer not aligned as required                     */
     CONVBN_ECUDA = 5,        /* CUDA runtime / driver call failed                   */
-    CONVBN_ETIMEOUT = 6      /* a bounded device-side wait expired                  */
+    CONVBN_ETIMEOUT = 6,     /* a bounded device-side wait expired                  */
+    CONVBN_ECAPACITY = 7     /* problem too large for the library's built-in scratch */
 } convbn_status;
 
 typedef enum { CONVBN_F32 = 0, CONVBN_BF16 = 1 } convbn_dtype;
@@ -126,6 +127,32 @@ int convbn_tune_bwd_weight(const convbn_desc *desc, const void *dz, const void *
                            const void *w, const float *b, const float *run_mean,
                            const void *saved, float *dw, float *db, float *dgamma,
                            float *dbeta, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Parameter gradients for callers that cannot allocate device memory (the paper has no counterpart
+ * of this call; it exists for integration reasons only).
+ *
+ * convbn_tune_bwd_weight needs a scratch buffer for its partial sums, and somebody has to allocate
+ * it.  Some users of this library cannot: code that runs where cudaMalloc is forbidden or would
+ * stall the device (inside another framework's memory-pool callback, in a plug-in whose host owns
+ * all device memory, in a real-time loop that must not touch the allocator).  For them this call
+ * computes exactly what convbn_tune_bwd_weight computes, with the same kernels and the same
+ * argument meaning, but takes no workspace: the scratch is a fixed 16 MiB array compiled into the
+ * library (each GPU that loads the library holds those 16 MiB until the process ends).  The call
+ * itself performs no cudaMalloc / cudaFree and calls no allocating routine.
+ *
+ *   - Limit: if convbn_workspace_bytes(desc, CONVBN_PHASE_TUNE_BWD_WEIGHT) exceeds 16 MiB
+ *     (16 * 2^20 bytes) the call returns CONVBN_ECAPACITY and launches nothing.
+ *   - The first call on each device looks up the array's device address (a runtime query, made with
+ *     that device current).  Make that first call before starting any stream capture.
+ *   - All calls share the one array.  It still holds the previous call's partial sums when a call
+ *     starts; that is harmless, because every word the kernels read is first written by the same
+ *     call, so nothing needs to be zeroed.  But two calls that overlap on the GPU (different
+ *     streams, or different host threads without ordering) would overwrite each other's partial
+ *     sums: callers must serialise them on the device. */
+int convbn_tune_bwd_weight_noalloc(const convbn_desc *desc, const void *dz, const void *x,
+                                   const void *w, const float *b, const float *run_mean,
+                                   const void *saved, float *dw, float *db, float *dgamma,
+                                   float *dbeta, void *stream);
 
 /* ---- Eval mode comparator (Sec. 3.1; Table 2, Eval row) ---------------------------------- */
 

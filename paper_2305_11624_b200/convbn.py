@@ -12,7 +12,7 @@ from typing import Optional
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIBRARY = os.path.join(_HERE, "libconvbn.so")
 
-OK, EINVAL, EUNSUPPORTED, EWORKSPACE, EALIGN, ECUDA, ETIMEOUT = range(7)
+OK, EINVAL, EUNSUPPORTED, EWORKSPACE, EALIGN, ECUDA, ETIMEOUT, ECAPACITY = range(8)
 F32, BF16 = 0, 1
 NCHW, NHWC = 0, 1
 MODE_TUNE, MODE_EVAL, MODE_DEPLOY = 0, 1, 2
@@ -25,6 +25,7 @@ EXPORTS = (
     "convbn_deploy_prepare", "convbn_deploy_fwd", "convbn_deploy_bwd", "convbn_check",
     "convbn_status_string", "convbn_last_kernel", "convbn_host_step_arena_bytes",
     "convbn_tune_step_host", "convbn_profile_begin", "convbn_profile_end",
+    "convbn_tune_bwd_weight_noalloc",
 )
 
 
@@ -143,6 +144,18 @@ def convbn_tune_bwd_weight(desc, dz, x, w, b, run_mean, saved, dw, db, dgamma, d
                                         _ptr(dgamma), _ptr(dbeta), _ptr(workspace),
                                         ctypes.c_size_t(wb), _stream(stream)),
            "convbn_tune_bwd_weight")
+
+
+def convbn_tune_bwd_weight_noalloc(desc, dz, x, w, b, run_mean, saved, dw, db, dgamma, dbeta,
+                                   stream=None):
+    """Same results as convbn_tune_bwd_weight for callers that must not allocate device memory:
+    no workspace argument, the library's built-in 16 MiB scratch array is used instead.  Raises
+    ConvBNError(ECAPACITY) when the layer needs more scratch than that.  Calls sharing a device
+    must not overlap on it."""
+    _raise(lib().convbn_tune_bwd_weight_noalloc(ctypes.byref(desc), _ptr(dz), _ptr(x), _ptr(w),
+                                                _ptr(b), _ptr(run_mean), _ptr(saved), _ptr(dw),
+                                                _ptr(db), _ptr(dgamma), _ptr(dbeta), _stream(stream)),
+           "convbn_tune_bwd_weight_noalloc")
 
 
 def convbn_eval_fwd(desc, x, w, b, gamma, beta, run_mean, run_var, z, y_saved, workspace=None,

@@ -499,6 +499,53 @@ int convbn_tune_step_host(const convbn_desc *desc, const void *x, const void *dz
     return CONVBN_OK;
 }
 
+// ---- parameter gradients without any caller-provided scratch -------------------------------------
+// Built-in scratch of convbn_tune_bwd_weight_noalloc.  It is part of the library image: every GPU
+// that loads the library carries these bytes until the process exits.  In host code the name below
+// is only a host-side handle of the symbol, never a device address, so the host asks the runtime for
+// the real address once per device and hands that to the kernels.
+#define CONVBN_NOALLOC_SCRATCH_BYTES (16u << 20)
+static __device__ __align__(256) unsigned char g_noalloc_scratch[CONVBN_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+const int kMaxDevices = 64;
+void *g_noalloc_ptr[kMaxDevices] = {nullptr};
+std::mutex g_noalloc_mu;
+
+// Device address of the built-in scratch on the CURRENT device (looked up on first use there).
+int noalloc_scratch_address(void **out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CONVBN_ECUDA;
+    std::lock_guard<std::mutex> lk(g_noalloc_mu);
+    if (!g_noalloc_ptr[dev]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress((void **)&ptr, g_noalloc_scratch) != cudaSuccess || !ptr)
+            return CONVBN_ECUDA;
+        g_noalloc_ptr[dev] = ptr;
+    }
+    *out = g_noalloc_ptr[dev];
+    return CONVBN_OK;
+}
+}  // namespace
+
+int convbn_tune_bwd_weight_noalloc(const convbn_desc *desc, const void *dz, const void *x,
+                                   const void *w, const float *b, const float *run_mean,
+                                   const void *saved, float *dw, float *db, float *dgamma,
+                                   float *dbeta, void *stream) {
+    Problem pb;
+    CK(make_problem(desc, &pb));
+    CK(check_pair(desc));
+    const size_t need = make_plan(desc, pb, CONVBN_PHASE_TUNE_BWD_WEIGHT).total;
+    if (need > (size_t)CONVBN_NOALLOC_SCRATCH_BYTES) return CONVBN_ECAPACITY;
+    void *scratch = nullptr;
+    CK(noalloc_scratch_address(&scratch));
+    // Same kernels as convbn_tune_bwd_weight, with the built-in array standing in for the caller's
+    // workspace.  Every scratch word those kernels read is written earlier in the same call, so
+    // nothing left over from a previous call has to be cleared.
+    return convbn_tune_bwd_weight(desc, dz, x, w, b, run_mean, saved, dw, db, dgamma, dbeta, scratch,
+                                  (size_t)CONVBN_NOALLOC_SCRATCH_BYTES, stream);
+}
+
 const char *convbn_status_string(int status) {
     switch (status) {
         case CONVBN_OK: return "ok";
@@ -508,6 +555,7 @@ const char *convbn_status_string(int status) {
         case CONVBN_EALIGN: return "pointer not aligned as required";
         case CONVBN_ECUDA: return "CUDA call failed";
         case CONVBN_ETIMEOUT: return "a bounded device-side wait expired";
+        case CONVBN_ECAPACITY: return "problem needs more scratch than the built-in 16 MiB array holds";
         default: return "unknown status";
     }
 }
