@@ -2,6 +2,7 @@
 // Every step of every entry point runs in this library's own kernels; there is no CPU path.
 #include <stdint.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <map>
@@ -121,8 +122,12 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
         case CONVBN_PHASE_TUNE_BWD_DATA:
             pl.w_scaled = take(wbytes);
             break;
-        case CONVBN_PHASE_TUNE_BWD_WEIGHT:
         case CONVBN_PHASE_DEPLOY_BWD:
+            pl.w_scaled = take(wbytes);
+            pl.partials = take(wrows * pl.splits * sizeof(float));
+            pl.bsum = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
+            break;
+        case CONVBN_PHASE_TUNE_BWD_WEIGHT:
             pl.partials = take(wrows * pl.splits * sizeof(float));
             pl.bsum = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
             break;
@@ -131,6 +136,7 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
             break;
         case CONVBN_PHASE_EVAL_BWD:
             pl.dy = take((size_t)pb.p * pb.c_out * elem_size(d->dtype));
+            pl.w_scaled = take(wbytes);
             pl.part_g = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
             pl.bsum = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
             pl.partials = take(wrows * pl.splits * sizeof(float));
@@ -184,6 +190,64 @@ int check_ws(const Plan &pl, const void *ws, size_t ws_bytes) {
 #define CU(expr) do { if ((expr) != cudaSuccess) return CONVBN_ECUDA; } while (0)
 
 inline char *at(void *ws, size_t off) { return (char *)ws + off; }
+
+bool force_direct() {
+    static const bool v = [] { const char *e = getenv("CONVBN_FORCE_DIRECT"); return e && e[0] == '1'; }();
+    return v;
+}
+
+// Tensor-core eligibility of the forward convolution and its GEMM shape.
+bool umma_fwd_shape(const convbn_desc *d, const Problem &pb, UmmaConvShape *s) {
+    if (force_direct() || d->dtype != CONVBN_BF16 || d->layout != CONVBN_NHWC || pb.groups != 1) return false;
+    *s = UmmaConvShape{pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.c_out, pb.kh, pb.kw,
+                       -pb.pad_h, -pb.pad_w, pb.stride_h, pb.stride_w, pb.dil_h, pb.dil_w};
+    return umma_conv_eligible(*s);
+}
+
+// Backward data as a stride-1 convolution of dZ with the rotated, channel-swapped omega'.
+bool umma_dgrad_shape(const convbn_desc *d, const Problem &pb, UmmaConvShape *s) {
+    if (force_direct() || d->dtype != CONVBN_BF16 || d->layout != CONVBN_NHWC || pb.groups != 1) return false;
+    if (pb.stride_h != 1 || pb.stride_w != 1) return false;
+    *s = UmmaConvShape{pb.n, pb.h_out, pb.w_out, pb.c_out, pb.h_in, pb.w_in, pb.c_in, pb.kh, pb.kw,
+                       pb.pad_h - (pb.kh - 1) * pb.dil_h, pb.pad_w - (pb.kw - 1) * pb.dil_w, 1, 1, pb.dil_h,
+                       pb.dil_w};
+    return umma_conv_eligible(*s);
+}
+
+// Forward convolution with whatever weights / bias the mode folded: tensor cores when eligible.
+int run_conv_fwd(const convbn_desc *d, const Problem &pb, const void *x, const void *w, const float *bias,
+                 void *z, cudaStream_t st, const char **which) {
+    UmmaConvShape s;
+    if (umma_fwd_shape(d, pb, &s)) {
+        LAUNCH("umma_fwd", launch_umma_conv(s, x, w, bias, z, st));
+        *which = "umma";
+    } else {
+        LAUNCH("direct_fwd", launch_direct_fwd(pb, d->dtype, d->layout, x, w, bias, z, st));
+        *which = "direct";
+    }
+    return CONVBN_OK;
+}
+
+// Backward data.  `scale` (C_out floats or NULL) is folded into the weights on the way:
+// w_scratch receives omega' in the layout the chosen kernel wants.
+int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, const void *w, const float *scale,
+                   void *w_scratch, void *dx, cudaStream_t st, const char **which) {
+    UmmaConvShape s;
+    if (umma_dgrad_shape(d, pb, &s)) {
+        LAUNCH("reparam_dgrad", launch_reparam_dgrad(pb, w, scale, w_scratch, st));
+        LAUNCH("umma_dgrad", launch_umma_conv(s, dz, w_scratch, nullptr, dx, st));
+        *which = "umma";
+    } else {
+        const void *wd = w;
+        if (scale) {
+            LAUNCH("rescale_weight", launch_rescale_weight(pb, d->dtype, w, scale, w_scratch, st));
+            wd = w_scratch;
+        }
+        LAUNCH("direct_dgrad", launch_direct_dgrad(pb, d->dtype, d->layout, dz, wd, dx, st));
+        *which = "direct";
+    }
+    return CONVBN_OK;
+}
 
 // Shared by Tune and Deploy backward-weight: conv weight gradient partials + per-channel dZ sums.
 int run_wgrad_partials(const convbn_desc *d, const Problem &pb, const Plan &pl, const void *dz,
@@ -242,8 +306,7 @@ int convbn_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const
     void *wf = at(workspace, pl.w_scaled);
     LAUNCH("reparam", launch_reparam(pb, desc->dtype, desc->layout, w, b, gamma, beta, run_mean, run_var, vec3, wf,
                       nullptr, st));
-    LAUNCH("direct_fwd", launch_direct_fwd(pb, desc->dtype, desc->layout, x, wf, vec3 + pb.c_out, z, st));
-    t_last_kernel[CONVBN_PHASE_TUNE_FWD] = "direct";
+    CK(run_conv_fwd(desc, pb, x, wf, vec3 + pb.c_out, z, st, &t_last_kernel[CONVBN_PHASE_TUNE_FWD]));
     return CONVBN_OK;
 }
 
@@ -259,9 +322,8 @@ int convbn_tune_bwd_data(const convbn_desc *desc, const void *dz, const void *w,
     CK(check_ws(pl, workspace, workspace_bytes));
     cudaStream_t st = (cudaStream_t)stream;
     void *wf = at(workspace, pl.w_scaled);
-    LAUNCH("rescale_weight", launch_rescale_weight(pb, desc->dtype, w, (const float *)saved, wf, st));
-    LAUNCH("direct_dgrad", launch_direct_dgrad(pb, desc->dtype, desc->layout, dz, wf, dx, st));
-    t_last_kernel[CONVBN_PHASE_TUNE_BWD_DATA] = "direct";
+    CK(run_conv_dgrad(desc, pb, dz, w, (const float *)saved, wf, dx, st,
+                      &t_last_kernel[CONVBN_PHASE_TUNE_BWD_DATA]));
     return CONVBN_OK;
 }
 
@@ -308,9 +370,8 @@ int convbn_eval_fwd(const convbn_desc *desc, const void *x, const void *w, const
     // BN acts on Y, which already holds the conv bias: shift = beta - mean s
     LAUNCH("reparam", launch_reparam(pb, desc->dtype, desc->layout, w, nullptr, gamma, beta, run_mean, run_var, vec3,
                       nullptr, nullptr, st));
-    LAUNCH("direct_fwd", launch_direct_fwd(pb, desc->dtype, desc->layout, x, w, b, y_saved, st));
+    CK(run_conv_fwd(desc, pb, x, w, b, y_saved, st, &t_last_kernel[CONVBN_PHASE_EVAL_FWD]));
     LAUNCH("bn_eval_fwd", launch_bn_eval_fwd(pb, desc->dtype, desc->layout, y_saved, vec3, z, st));
-    t_last_kernel[CONVBN_PHASE_EVAL_FWD] = "direct";
     return CONVBN_OK;
 }
 
@@ -335,12 +396,12 @@ int convbn_eval_bwd(const convbn_desc *desc, const void *dz, const void *x, cons
     LAUNCH("bn_eval_bwd", launch_bn_eval_bwd(pb, desc->dtype, desc->layout, dz, y_saved, gamma, run_mean, run_var, dy, pg,
                           pbm, pl.bsplits, st));
     LAUNCH("bn_eval_finish", launch_bn_eval_finish(pb, pg, pbm, pl.bsplits, gamma, run_var, db, dgamma, dbeta, st));
-    LAUNCH("direct_dgrad", launch_direct_dgrad(pb, desc->dtype, desc->layout, dy, w, dx, st));
+    CK(run_conv_dgrad(desc, pb, dy, w, nullptr, at(workspace, pl.w_scaled), dx, st,
+                      &t_last_kernel[CONVBN_PHASE_EVAL_BWD]));
     LAUNCH("direct_wgrad", launch_direct_wgrad(pb, desc->dtype, desc->layout, dy, x, (float *)at(workspace, pl.partials),
                            pl.splits, st));
     LAUNCH("wgrad_epilogue", launch_wgrad_epilogue(pb, desc->dtype, (const float *)at(workspace, pl.partials), pl.splits,
                              nullptr, 0, w, nullptr, nullptr, nullptr, dw, nullptr, nullptr, nullptr, st));
-    t_last_kernel[CONVBN_PHASE_EVAL_BWD] = "direct";
     return CONVBN_OK;
 }
 
@@ -372,8 +433,7 @@ int convbn_deploy_fwd(const convbn_desc *desc, const void *x, const void *w_fuse
     const Plan pl = make_plan(desc, pb, CONVBN_PHASE_DEPLOY_FWD);
     CK(check_ws(pl, workspace, workspace_bytes));
     cudaStream_t st = (cudaStream_t)stream;
-    LAUNCH("direct_fwd", launch_direct_fwd(pb, desc->dtype, desc->layout, x, w_fused, b_fused, z, st));
-    t_last_kernel[CONVBN_PHASE_DEPLOY_FWD] = "direct";
+    CK(run_conv_fwd(desc, pb, x, w_fused, b_fused, z, st, &t_last_kernel[CONVBN_PHASE_DEPLOY_FWD]));
     return CONVBN_OK;
 }
 
@@ -390,12 +450,12 @@ int convbn_deploy_bwd(const convbn_desc *desc, const void *dz, const void *x, co
     const Plan pl = make_plan(desc, pb, CONVBN_PHASE_DEPLOY_BWD);
     CK(check_ws(pl, workspace, workspace_bytes));
     cudaStream_t st = (cudaStream_t)stream;
-    LAUNCH("direct_dgrad", launch_direct_dgrad(pb, desc->dtype, desc->layout, dz, w_fused, dx, st));
+    CK(run_conv_dgrad(desc, pb, dz, w_fused, nullptr, at(workspace, pl.w_scaled), dx, st,
+                      &t_last_kernel[CONVBN_PHASE_DEPLOY_BWD]));
     CK(run_wgrad_partials(desc, pb, pl, dz, x, workspace, st));
     LAUNCH("wgrad_epilogue", launch_wgrad_epilogue(pb, desc->dtype, (const float *)at(workspace, pl.partials), pl.splits,
                              (const float *)at(workspace, pl.bsum), pl.bsplits, w_fused, nullptr, nullptr,
                              nullptr, dw_fused, db_fused, nullptr, nullptr, st));
-    t_last_kernel[CONVBN_PHASE_DEPLOY_BWD] = "direct";
     return CONVBN_OK;
 }
 

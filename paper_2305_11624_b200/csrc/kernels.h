@@ -30,6 +30,23 @@ int direct_wgrad_splits(const Problem &pb);
 cudaError_t launch_direct_wgrad(const Problem &pb, int dtype, int layout, const void *dz,
                                 const void *x, float *partials, int splits, cudaStream_t st);
 
+// ---- tensor-core implicit-GEMM convolution (bf16 NHWC, groups = 1) -----------------------------
+// out[n,ho,wo,:cn] = bias + sum over taps (r,q) and channels c of
+//     act[n, lower_h + ho stride_h + r dil_h, lower_w + wo stride_w + q dil_w, c] * wmat[:, (r taps_w + q) ca + c]
+// with zeros outside the activation tensor.  wmat is a row-major [cn][taps_h taps_w ca] bf16 matrix.
+struct UmmaConvShape {
+    int n, ha, wa, ca;       // activation tensor [n][ha][wa][ca]
+    int ho, wo, cn;          // output tensor [n][ho][wo][cn]
+    int taps_h, taps_w, lower_h, lower_w, stride_h, stride_w, dil_h, dil_w;
+};
+bool umma_conv_eligible(const UmmaConvShape &s);
+cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void *wmat, const float *bias,
+                             void *out, cudaStream_t st);
+// Weight operand of the backward-data GEMM: w_t[ci][taps-1-tap][co] = s[co] w[co][tap][ci]
+// (s_vec == NULL: unscaled).  bf16, groups = 1.
+cudaError_t launch_reparam_dgrad(const Problem &pb, const void *w, const float *s_vec, void *w_t,
+                                 cudaStream_t st);
+
 // ---- per-channel reductions (Appendix B: backward of a broadcast is a sum) -------------------
 int channel_sum_splits(const Problem &pb);
 // part: [splits][C_out] partial sums of t over pixel slices

@@ -92,6 +92,36 @@ cudaError_t launch_rescale_weight(const Problem &pb, int dtype, const void *w, c
     });
 }
 
+// omega' re-laid-out for the backward-data GEMM (dX = omega'_rot (*) dZ, Sec. 3.2.1): output channel
+// becomes the contiguous (reduction) index and the taps are rotated by 180 degrees.
+__global__ void __launch_bounds__(256) reparam_dgrad_kernel(int c_out, int c_in, int taps,
+                                                            const __nv_bfloat16 *__restrict__ w,
+                                                            const float *__restrict__ s_vec,
+                                                            __nv_bfloat16 *__restrict__ w_t) {
+    __shared__ float tile[32][33];
+    const int tap = blockIdx.z, co0 = blockIdx.y * 32, ci0 = blockIdx.x * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int j = ty; j < 32; j += 8) {
+        const int co = co0 + j, ci = ci0 + tx;
+        if (co < c_out && ci < c_in)
+            tile[j][tx] = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((long long)co * taps + tap) * c_in + ci]);
+    }
+    __syncthreads();
+    for (int j = ty; j < 32; j += 8) {
+        const int ci = ci0 + j, co = co0 + tx;
+        if (co < c_out && ci < c_in)
+            w_t[((long long)ci * taps + (taps - 1 - tap)) * c_out + co] = __float2bfloat16_rn(tile[tx][j]);
+    }
+}
+
+cudaError_t launch_reparam_dgrad(const Problem &pb, const void *w, const float *s_vec, void *w_t,
+                                 cudaStream_t st) {
+    dim3 grid((pb.c_in + 31) / 32, (pb.c_out + 31) / 32, pb.kh * pb.kw);
+    reparam_dgrad_kernel<<<grid, 256, 0, st>>>(pb.c_out, pb.c_in, pb.kh * pb.kw, (const __nv_bfloat16 *)w, s_vec,
+                                               (__nv_bfloat16 *)w_t);
+    return cudaGetLastError();
+}
+
 // ---- per-channel partial sums over pixel slices (Appendix B) --------------------------------
 template <class T, class L>
 __global__ void __launch_bounds__(256) channel_sum_partial_kernel(int c_out, int h_out, int w_out,
