@@ -289,7 +289,7 @@ def run_ours(args):
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         full = layers[0].n
-        times, fl, cores = oracle_step_time(args.workload, full, 2)
+        times, fl, cores = oracle_step_time(args.workload, full, 2)  # ~2 x 3 s on 16 cores
         cpu = {"value": fl / min(times) / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": "one full step (all %d samples of every layer) of the fp64 oracle, best of 2, %.1f s"
                          % (full, min(times))}

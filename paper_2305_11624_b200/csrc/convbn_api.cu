@@ -97,6 +97,11 @@ int check_pair(const convbn_desc *d) {
     return CONVBN_EUNSUPPORTED;
 }
 
+bool force_direct() {
+    static const bool v = [] { const char *e = getenv("CONVBN_FORCE_DIRECT"); return e && e[0] == '1'; }();
+    return v;
+}
+
 // Workspace carve-up of one phase.  Offsets are multiples of 256 bytes.
 struct Plan {
     size_t total = 0;
@@ -106,7 +111,10 @@ struct Plan {
     size_t part_g = 0;     // [bsplits][C_out] fp32 (Eval backward)
     size_t dy = 0;         // Eval backward: s dZ, storage dtype
     size_t vec3 = 0;       // Eval forward: [s | beta - mean s | r]
+    size_t dotpart = 0;    // [kt][C_out] fp32 (tensor-core weight-gradient path)
     int splits = 1, bsplits = 1;
+    bool umma_wgrad = false;
+    UmmaWgradPlan uw;
 };
 
 Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
@@ -117,6 +125,14 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
     const size_t wrows = (size_t)pb.c_out * pb.kdim;
     pl.splits = direct_wgrad_splits(pb);
     pl.bsplits = channel_sum_splits(pb);
+    pl.umma_wgrad = !force_direct() && d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC &&
+                    umma_wgrad_eligible(pb);
+    size_t part_bytes = wrows * pl.splits * sizeof(float), dot_bytes = 0;
+    if (pl.umma_wgrad) {
+        pl.uw = umma_wgrad_plan(pb);
+        part_bytes = wrows * pl.uw.splits * sizeof(float);
+        dot_bytes = (size_t)pl.uw.kt * pb.c_out * sizeof(float);
+    }
     switch (phase) {
         case CONVBN_PHASE_TUNE_FWD:
         case CONVBN_PHASE_TUNE_BWD_DATA:
@@ -124,12 +140,14 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
             break;
         case CONVBN_PHASE_DEPLOY_BWD:
             pl.w_scaled = take(wbytes);
-            pl.partials = take(wrows * pl.splits * sizeof(float));
+            pl.partials = take(part_bytes);
             pl.bsum = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
+            pl.dotpart = take(dot_bytes);
             break;
         case CONVBN_PHASE_TUNE_BWD_WEIGHT:
-            pl.partials = take(wrows * pl.splits * sizeof(float));
+            pl.partials = take(part_bytes);
             pl.bsum = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
+            pl.dotpart = take(dot_bytes);
             break;
         case CONVBN_PHASE_EVAL_FWD:
             pl.vec3 = take(3 * (size_t)pb.c_out * sizeof(float));
@@ -139,7 +157,8 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
             pl.w_scaled = take(wbytes);
             pl.part_g = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
             pl.bsum = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
-            pl.partials = take(wrows * pl.splits * sizeof(float));
+            pl.partials = take(part_bytes);
+            pl.dotpart = take(dot_bytes);
             break;
         default:
             break;
@@ -190,11 +209,6 @@ int check_ws(const Plan &pl, const void *ws, size_t ws_bytes) {
 #define CU(expr) do { if ((expr) != cudaSuccess) return CONVBN_ECUDA; } while (0)
 
 inline char *at(void *ws, size_t off) { return (char *)ws + off; }
-
-bool force_direct() {
-    static const bool v = [] { const char *e = getenv("CONVBN_FORCE_DIRECT"); return e && e[0] == '1'; }();
-    return v;
-}
 
 // Tensor-core eligibility of the forward convolution and its GEMM shape.
 bool umma_fwd_shape(const convbn_desc *d, const Problem &pb, UmmaConvShape *s) {
@@ -249,11 +263,31 @@ int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, cons
     return CONVBN_OK;
 }
 
-// Shared by Tune and Deploy backward-weight: conv weight gradient partials + per-channel dZ sums.
-int run_wgrad_partials(const convbn_desc *d, const Problem &pb, const Plan &pl, const void *dz,
-                       const void *x, void *ws, cudaStream_t st) {
-    LAUNCH("direct_wgrad", launch_direct_wgrad(pb, d->dtype, d->layout, dz, x, (float *)at(ws, pl.partials), pl.splits, st));
-    LAUNCH("channel_sum", launch_channel_sum_partial(pb, d->dtype, d->layout, dz, (float *)at(ws, pl.bsum), pl.bsplits, st));
+// Parameter gradients from dZ and X, shared by all modes.
+//   vec3 != NULL (Tune): dw = s domega', dbeta, db = s dbeta, dgamma          (Table 2, Tune row)
+//   vec3 == NULL        : dw = domega', db = sum dZ if db != NULL               (Deploy / Eval rows)
+int run_param_grads(const convbn_desc *d, const Problem &pb, const Plan &pl, const void *dz, const void *x,
+                    const void *w, const float *vec3, const float *b, const float *mean, float *dw, float *db,
+                    float *dgamma, float *dbeta, void *ws, cudaStream_t st, const char **which) {
+    float *partials = (float *)at(ws, pl.partials), *bsum = (float *)at(ws, pl.bsum);
+    const bool need_bsum = vec3 || db;
+    if (need_bsum)
+        LAUNCH("channel_sum", launch_channel_sum_partial(pb, d->dtype, d->layout, dz, bsum, pl.bsplits, st));
+    if (pl.umma_wgrad) {
+        float *dotpart = (float *)at(ws, pl.dotpart);
+        LAUNCH("umma_wgrad", launch_umma_wgrad(pb, pl.uw, dz, x, partials, st));
+        LAUNCH("wgrad_epilogue_t", launch_wgrad_epilogue_t(pb, pl.uw, partials, w, vec3, dw, dotpart, st));
+        if (need_bsum)
+            LAUNCH("param_finish", launch_param_finish(pb, pl.uw, dotpart, bsum, pl.bsplits, vec3, b, mean, db,
+                                                       dgamma, dbeta, st));
+        *which = "umma";
+    } else {
+        LAUNCH("direct_wgrad", launch_direct_wgrad(pb, d->dtype, d->layout, dz, x, partials, pl.splits, st));
+        LAUNCH("wgrad_epilogue", launch_wgrad_epilogue(pb, d->dtype, partials, pl.splits, need_bsum ? bsum : nullptr,
+                                                       need_bsum ? pl.bsplits : 0, w, vec3, b, mean, dw, db, dgamma,
+                                                       dbeta, st));
+        *which = "direct";
+    }
     return CONVBN_OK;
 }
 
@@ -343,11 +377,8 @@ int convbn_tune_bwd_weight(const convbn_desc *desc, const void *dz, const void *
     const Plan pl = make_plan(desc, pb, CONVBN_PHASE_TUNE_BWD_WEIGHT);
     CK(check_ws(pl, workspace, workspace_bytes));
     cudaStream_t st = (cudaStream_t)stream;
-    CK(run_wgrad_partials(desc, pb, pl, dz, x, workspace, st));
-    LAUNCH("wgrad_epilogue", launch_wgrad_epilogue(pb, desc->dtype, (const float *)at(workspace, pl.partials), pl.splits,
-                             (const float *)at(workspace, pl.bsum), pl.bsplits, w,
-                             (const float *)saved, b, run_mean, dw, db, dgamma, dbeta, st));
-    t_last_kernel[CONVBN_PHASE_TUNE_BWD_WEIGHT] = "direct";
+    CK(run_param_grads(desc, pb, pl, dz, x, w, (const float *)saved, b, run_mean, dw, db, dgamma, dbeta,
+                       workspace, st, &t_last_kernel[CONVBN_PHASE_TUNE_BWD_WEIGHT]));
     return CONVBN_OK;
 }
 
@@ -398,10 +429,9 @@ int convbn_eval_bwd(const convbn_desc *desc, const void *dz, const void *x, cons
     LAUNCH("bn_eval_finish", launch_bn_eval_finish(pb, pg, pbm, pl.bsplits, gamma, run_var, db, dgamma, dbeta, st));
     CK(run_conv_dgrad(desc, pb, dy, w, nullptr, at(workspace, pl.w_scaled), dx, st,
                       &t_last_kernel[CONVBN_PHASE_EVAL_BWD]));
-    LAUNCH("direct_wgrad", launch_direct_wgrad(pb, desc->dtype, desc->layout, dy, x, (float *)at(workspace, pl.partials),
-                           pl.splits, st));
-    LAUNCH("wgrad_epilogue", launch_wgrad_epilogue(pb, desc->dtype, (const float *)at(workspace, pl.partials), pl.splits,
-                             nullptr, 0, w, nullptr, nullptr, nullptr, dw, nullptr, nullptr, nullptr, st));
+    const char *unused = nullptr;
+    CK(run_param_grads(desc, pb, pl, dy, x, w, nullptr, nullptr, nullptr, dw, nullptr, nullptr, nullptr, workspace,
+                       st, &unused));
     return CONVBN_OK;
 }
 
@@ -452,10 +482,9 @@ int convbn_deploy_bwd(const convbn_desc *desc, const void *dz, const void *x, co
     cudaStream_t st = (cudaStream_t)stream;
     CK(run_conv_dgrad(desc, pb, dz, w_fused, nullptr, at(workspace, pl.w_scaled), dx, st,
                       &t_last_kernel[CONVBN_PHASE_DEPLOY_BWD]));
-    CK(run_wgrad_partials(desc, pb, pl, dz, x, workspace, st));
-    LAUNCH("wgrad_epilogue", launch_wgrad_epilogue(pb, desc->dtype, (const float *)at(workspace, pl.partials), pl.splits,
-                             (const float *)at(workspace, pl.bsum), pl.bsplits, w_fused, nullptr, nullptr,
-                             nullptr, dw_fused, db_fused, nullptr, nullptr, st));
+    const char *unused = nullptr;
+    CK(run_param_grads(desc, pb, pl, dz, x, w_fused, nullptr, nullptr, nullptr, dw_fused, db_fused, nullptr, nullptr,
+                       workspace, st, &unused));
     return CONVBN_OK;
 }
 

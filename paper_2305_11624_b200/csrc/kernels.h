@@ -47,6 +47,27 @@ cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void
 cudaError_t launch_reparam_dgrad(const Problem &pb, const void *w, const float *s_vec, void *w_t,
                                  cudaStream_t st);
 
+// ---- tensor-core weight gradient (bf16 NHWC, groups = 1, channels multiples of 64) ---------------
+struct UmmaWgradPlan {
+    int splits = 1;           // pixel slices = partial tiles
+    long long per_split = 0;  // pixels per slice
+    int kt = 1;               // k ranges of the epilogue (rows of dotpart)
+};
+bool umma_wgrad_eligible(const Problem &pb);
+UmmaWgradPlan umma_wgrad_plan(const Problem &pb);
+// partials: [splits][kdim][C_out] fp32 (k-major: the transpose of the weight layout)
+cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const void *dz, const void *x,
+                              float *partials, cudaStream_t st);
+// dw[co][k] = scale[co] * sum_splits partials (scale = first C_out floats of vec3, 1 if NULL);
+// dotpart[kt][C_out] = per-k-range pieces of sum_k (sum_splits partials) w[co][k]  (only if vec3)
+cudaError_t launch_wgrad_epilogue_t(const Problem &pb, const UmmaWgradPlan &pl, const float *partials,
+                                    const void *w, const float *vec3, float *dw, float *dotpart,
+                                    cudaStream_t st);
+// dbeta, db, dgamma from dotpart and the per-channel dZ sums (tune mode), or db = sum dZ (vec3 NULL).
+cudaError_t launch_param_finish(const Problem &pb, const UmmaWgradPlan &pl, const float *dotpart,
+                                const float *bsum_part, int bsplits, const float *vec3, const float *b,
+                                const float *mean, float *db, float *dgamma, float *dbeta, cudaStream_t st);
+
 // ---- per-channel reductions (Appendix B: backward of a broadcast is a sum) -------------------
 int channel_sum_splits(const Problem &pb);
 // part: [splits][C_out] partial sums of t over pixel slices

@@ -10,6 +10,16 @@
 #include <stdint.h>
 
 namespace convbn {
+
+// Host helpers (umma_conv.cu): tensor maps over bf16 tensors, 128-byte swizzle, zero fill.
+// Row-major matrix [rows][cols], box = box_rows x box_cols.
+bool make_tmap_matrix_bf16(CUtensorMap *tm, const void *base, long long rows, long long cols, int box_rows,
+                           int box_cols);
+// NHWC tensor in im2col mode: `pixels` output positions x `channels` channels per load.
+bool make_tmap_im2col_bf16(CUtensorMap *tm, const void *base, int n, int h, int w, int c, int lower_h,
+                           int lower_w, int upper_h, int upper_w, int stride_h, int stride_w, int pixels,
+                           int channels);
+
 namespace ptx {
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {

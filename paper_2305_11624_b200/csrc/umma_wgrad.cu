@@ -1,0 +1,346 @@
+// Weight-gradient implicit GEMM on the sm_100a tensor cores:  domega' = dZ (.) X  (Sec. 3.2.1; Table 2,
+// Tune row), the reduction over all N H_out W_out output pixels.
+//
+// GEMM view: D[k][co] = sum_p Xcol[p][k] dZ[p][co] with k = (tap, ci).  Both operands have the
+// reduction index p as their slow axis in NHWC memory, so both are fed to tcgen05.mma as MN-major
+// tiles: the A tile is two [64 pixels][64 channels] im2col loads of X (two consecutive 64-wide slices
+// of k), the B tile is BN/64 plain [64 pixels][64 channels] boxes of dZ.  The pixel range is cut into
+// `splits` slices (grid.z); every CTA accumulates its slice in tensor memory in fp32 and writes one
+// fp32 partial tile part[split][k][co].  A second kernel adds the slices in fixed order and forms
+// domega, dgamma, ... from the fp32 sums (never from rounded values).
+#include "kernels.h"
+#include "sm100_ptx.cuh"
+
+namespace convbn {
+
+using namespace ptx;
+
+constexpr int kWM = 128;          // k rows per tile (two 64-channel slices)
+constexpr int kWP = 64;           // pixels per stage (reduction depth per stage)
+constexpr int kWUmmaK = 16;
+constexpr int kWMaxStages = 8;
+constexpr int kWThreads = 192;
+constexpr uint32_t kChunkBytes = kWP * 64 * 2;   // one [64 pixels][64 channels] bf16 box
+
+struct WgradGemm {
+    int ho, wo, c_in, c_out, taps_w;
+    int lower_h, lower_w, stride_h, stride_w, dil_h, dil_w;
+    int kdim;               // taps * c_in
+    long long p;            // output pixels
+    long long per_split;    // pixels per slice (multiple of 64)
+    int stages;
+};
+
+struct WgradSmemCtl {
+    uint64_t full[kWMaxStages];
+    uint64_t empty[kWMaxStages];
+    uint64_t tmem_full;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_constant__ CUtensorMap tm_x,
+                                                              const __grid_constant__ CUtensorMap tm_dz,
+                                                              const WgradGemm g, float *__restrict__ partials,
+                                                              int *err) {
+    extern __shared__ uint8_t smem_raw[];
+    constexpr uint32_t kABytes = 2 * kChunkBytes, kBBytes = (BN / 64) * kChunkBytes, kStageBytes = kABytes + kBBytes;
+    uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    WgradSmemCtl *ctl = (WgradSmemCtl *)(tiles + (size_t)g.stages * kStageBytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int stages = g.stages;
+    const int k0 = blockIdx.x * kWM;                    // first k row of this tile
+    const int n0 = blockIdx.y * BN;                     // first output channel
+    const long long p0 = (long long)blockIdx.z * g.per_split;
+    const long long p1 = p0 + g.per_split < g.p ? p0 + g.per_split : g.p;
+    const int num_kb = (int)((p1 - p0 + kWP - 1) / kWP);
+    const int a_chunks = (k0 + 64 < g.kdim) ? 2 : 1;    // second 64-slice may fall beyond K
+    int b_chunks = (g.c_out - n0) / 64;
+    if (b_chunks > BN / 64) b_chunks = BN / 64;
+    volatile int *abort_flag = &ctl->abort_flag;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
+        mbar_init(&ctl->tmem_full, 1);
+        ctl->abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(&ctl->tmem_base, BN);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        if (elect_one()) {
+            prefetch_tensormap(&tm_x);
+            prefetch_tensormap(&tm_dz);
+            const uint32_t tx_bytes = (uint32_t)(a_chunks + b_chunks) * kChunkBytes;
+            int issued = 0;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % stages;
+                const uint32_t ph = (uint32_t)(kb / stages) & 1u;
+                if (!mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag)) {
+                    atomicOr(err, ERRW_TIMEOUT);
+                    ctl->abort_flag = 1;
+                    break;
+                }
+                const long long pp = p0 + (long long)kb * kWP;
+                const int wo0 = (int)(pp % g.wo);
+                const long long t = pp / g.wo;
+                const int ho0 = (int)(t % g.ho), img0 = (int)(t / g.ho);
+                const int base_w = g.lower_w + wo0 * g.stride_w, base_h = g.lower_h + ho0 * g.stride_h;
+                uint8_t *a_dst = tiles + (size_t)s * kStageBytes, *b_dst = a_dst + kABytes;
+                mbar_arrive_expect_tx(&ctl->full[s], tx_bytes);
+                for (int j = 0; j < a_chunks; ++j) {
+                    const int kk = k0 + j * 64;                  // k = tap * c_in + ci
+                    const int tap = kk / g.c_in, ci0 = kk - tap * g.c_in;
+                    const int r = tap / g.taps_w, q = tap - r * g.taps_w;
+                    tma_load_im2col_4d(a_dst + j * kChunkBytes, &tm_x, &ctl->full[s], ci0, base_w, base_h, img0,
+                                       (uint16_t)(q * g.dil_w), (uint16_t)(r * g.dil_h));
+                }
+                for (int j = 0; j < b_chunks; ++j)
+                    tma_load_2d(b_dst + j * kChunkBytes, &tm_dz, &ctl->full[s], n0 + j * 64, (int)pp);
+                ++issued;
+            }
+            if (ctl->abort_flag) {
+                const int first = issued > stages ? issued - stages : 0;
+                for (int kb = first; kb < issued; ++kb)
+                    mbar_wait_bounded(&ctl->full[kb % stages], (uint32_t)(kb / stages) & 1u, nullptr, 200000000ull);
+            }
+        }
+    } else if (warp == 1) {
+        if (elect_one()) {
+            constexpr uint32_t idesc = idesc_bf16_f32(kWM, BN, 1, 1);   // both operands MN-major
+            bool ok = true;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % stages;
+                const uint32_t ph = (uint32_t)(kb / stages) & 1u;
+                if (!mbar_wait_bounded(&ctl->full[s], ph, abort_flag)) {
+                    atomicOr(err, ERRW_TIMEOUT);
+                    ctl->abort_flag = 1;
+                    ok = false;
+                    break;
+                }
+                tc_fence_after_sync();
+                const uint32_t a_addr = smem_u32(tiles + (size_t)s * kStageBytes), b_addr = a_addr + kABytes;
+#pragma unroll
+                for (int k = 0; k < kWP / kWUmmaK; ++k) {
+                    // 16 pixels = two groups of 8 rows (1024 B apart); 64-channel slices 8192 B apart
+                    const uint64_t ad = smem_desc_sw128(a_addr + k * kWUmmaK * 128, kChunkBytes, 1024);
+                    const uint64_t bd = smem_desc_sw128(b_addr + k * kWUmmaK * 128, kChunkBytes, 1024);
+                    umma_bf16_ss(tmem_base, ad, bd, idesc, (kb | k) ? 1u : 0u);
+                }
+                umma_commit(&ctl->empty[s]);
+            }
+            if (ok) umma_commit(&ctl->tmem_full);
+        }
+    } else {
+        const int quarter = warp & 3;
+        const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->tmem_full, 0, abort_flag));
+        if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+        if (ok) {
+            tc_fence_after_sync();
+            const int k = k0 + quarter * 32 + lane;
+            const bool row_ok = k < g.kdim;
+            float *orow = partials + ((size_t)blockIdx.z * g.kdim + (row_ok ? k : 0)) * g.c_out + n0;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                if (n0 + c0 >= g.c_out) break;
+                uint32_t v[32];
+                tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
+                tmem_ld_wait();
+                if (row_ok) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4)
+                        *(uint4 *)(orow + c0 + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                }
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, BN);
+}
+
+bool umma_wgrad_eligible(const Problem &pb) {
+    if (pb.groups != 1 || pb.c_in % 64 || pb.c_out % 64) return false;
+    if (pb.pad_h > 128 || pb.pad_w > 128) return false;
+    if ((pb.kh - 1) * pb.dil_h > 255 || (pb.kw - 1) * pb.dil_w > 255) return false;
+    if (pb.stride_h > 8 || pb.stride_w > 8) return false;
+    if (pb.p >= (1LL << 31)) return false;
+    return true;
+}
+
+static int wgrad_bn(const Problem &pb) { return pb.c_out >= 256 ? 256 : (pb.c_out >= 128 ? 128 : 64); }
+
+UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
+    UmmaWgradPlan pl;
+    const int bn = wgrad_bn(pb);
+    const long long m_tiles = (pb.kdim + kWM - 1) / kWM, n_tiles = (pb.c_out + bn - 1) / bn;
+    const long long target = bn == 256 ? 148 : 296;
+    long long splits = (target + m_tiles * n_tiles - 1) / (m_tiles * n_tiles);
+    const long long max_splits = (pb.p + 4 * kWP - 1) / (4 * kWP);     // at least 256 pixels per slice
+    if (splits > max_splits) splits = max_splits;
+    if (splits < 1) splits = 1;
+    long long per = (pb.p + splits - 1) / splits;
+    per = (per + kWP - 1) / kWP * kWP;
+    pl.per_split = per;
+    pl.splits = (int)((pb.p + per - 1) / per);
+    int kt = (int)(296 / (pb.c_out / 32));
+    const int kt_max = (pb.kdim + 31) / 32;
+    if (kt > kt_max) kt = kt_max;
+    if (kt < 1) kt = 1;
+    pl.kt = kt;
+    return pl;
+}
+
+template <int BN>
+static cudaError_t launch_w(const CUtensorMap &tx, const CUtensorMap &tdz, WgradGemm g, const UmmaWgradPlan &pl,
+                            const Problem &pb, float *partials, int *err, cudaStream_t st) {
+    constexpr size_t stage = 2 * kChunkBytes + (BN / 64) * kChunkBytes;
+    int stages = BN == 256 ? 4 : 4;
+    const long long max_kb = (pl.per_split + kWP - 1) / kWP;
+    if (stages > max_kb) stages = (int)max_kb;
+    g.stages = stages;
+    size_t smem = stages * stage + 1024 + sizeof(WgradSmemCtl);
+    const size_t floor_smem = (size_t)(228 * 1024) / (512 / BN + 1) + 1024;
+    if (smem < floor_smem) smem = floor_smem;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(umma_wgrad_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             210 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    dim3 grid((unsigned)((pb.kdim + kWM - 1) / kWM), (unsigned)((pb.c_out + BN - 1) / BN), (unsigned)pl.splits);
+    umma_wgrad_kernel<BN><<<grid, kWThreads, smem, st>>>(tx, tdz, g, partials, err);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const void *dz, const void *x,
+                              float *partials, cudaStream_t st) {
+    WgradGemm g;
+    g.ho = pb.h_out; g.wo = pb.w_out; g.c_in = pb.c_in; g.c_out = pb.c_out; g.taps_w = pb.kw;
+    g.lower_h = -pb.pad_h; g.lower_w = -pb.pad_w; g.stride_h = pb.stride_h; g.stride_w = pb.stride_w;
+    g.dil_h = pb.dil_h; g.dil_w = pb.dil_w; g.kdim = pb.kdim; g.p = pb.p; g.per_split = pl.per_split; g.stages = 1;
+    const int upper_h = g.lower_h + (pb.h_out - 1) * pb.stride_h - (pb.h_in - 1);
+    const int upper_w = g.lower_w + (pb.w_out - 1) * pb.stride_w - (pb.w_in - 1);
+    CUtensorMap tx, tdz;
+    if (!make_tmap_im2col_bf16(&tx, x, pb.n, pb.h_in, pb.w_in, pb.c_in, g.lower_h, g.lower_w, upper_h, upper_w,
+                               pb.stride_h, pb.stride_w, kWP, 64))
+        return cudaErrorInvalidValue;
+    if (!make_tmap_matrix_bf16(&tdz, dz, pb.p, pb.c_out, kWP, 64)) return cudaErrorInvalidValue;
+    int *err = nullptr;
+    cudaError_t e = error_word_address(&err);
+    if (e != cudaSuccess) return e;
+    const int bn = wgrad_bn(pb);
+    if (bn == 64) return launch_w<64>(tx, tdz, g, pl, pb, partials, err, st);
+    if (bn == 128) return launch_w<128>(tx, tdz, g, pl, pb, partials, err, st);
+    return launch_w<256>(tx, tdz, g, pl, pb, partials, err, st);
+}
+
+// ---- epilogue over k-major partials ------------------------------------------------------------
+// part[split][k][co] -> dw[co][k] = scale[co] * sum_split part;  dotpart[kt][co] = sum over this block's
+// k range of (sum_split part) * w[co][k].  Block = 32 output channels x one k range; 32 x 8 threads.
+__global__ void __launch_bounds__(256) wgrad_epilogue_t_kernel(int c_out, int kdim, const float *__restrict__ part,
+                                                              int splits, int kper,
+                                                              const __nv_bfloat16 *__restrict__ w,
+                                                              const float *__restrict__ vec3,
+                                                              float *__restrict__ dw, float *__restrict__ dotpart) {
+    __shared__ float tile[32][33];
+    __shared__ float wtile[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int co0 = blockIdx.x * 32;
+    const int kbeg = blockIdx.y * kper, kend = min(kdim, kbeg + kper);
+    const size_t slice = (size_t)kdim * c_out;
+    float dot[4] = {0.f, 0.f, 0.f, 0.f};
+    float sc[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) sc[j] = vec3 ? vec3[co0 + ty + 8 * j] : 1.f;
+    for (int kb = kbeg; kb < kend; kb += 32) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int kl = ty + 8 * j, k = kb + kl;
+            float acc = 0.f;
+            if (k < kend) {
+                const float *src = part + (size_t)k * c_out + co0 + tx;
+                for (int sp = 0; sp < splits; ++sp) acc += src[sp * slice];
+            }
+            tile[kl][tx] = acc;
+            const int kr = kb + tx;          // w[co0 + kl][kb + tx], coalesced along k
+            wtile[kl][tx] = (vec3 && kr < kend) ? __bfloat162float(w[(size_t)(co0 + kl) * kdim + kr]) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int cl = ty + 8 * j, k = kb + tx;
+            if (k < kend) {
+                const float v = tile[tx][cl];
+                dw[(size_t)(co0 + cl) * kdim + k] = sc[j] * v;
+                dot[j] = fmaf(v, wtile[cl][tx], dot[j]);
+            }
+        }
+        __syncthreads();
+    }
+    if (dotpart) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float d = dot[j];
+            for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+            if (tx == 0) dotpart[(size_t)blockIdx.y * c_out + co0 + ty + 8 * j] = d;
+        }
+    }
+}
+
+// dbeta = sum dZ; db = s dbeta; dgamma = r (sum_k domega' omega + dbeta (b - mu_hat))   (Table 2, Tune row)
+// plain mode (vec3 == NULL): db = sum dZ only.
+__global__ void param_finish_kernel(int c_out, const float *__restrict__ dotpart, int kt,
+                                    const float *__restrict__ bsum_part, int bsplits,
+                                    const float *__restrict__ vec3, const float *__restrict__ b,
+                                    const float *__restrict__ mean, float *__restrict__ db,
+                                    float *__restrict__ dgamma, float *__restrict__ dbeta) {
+    const int co = blockIdx.x * blockDim.x + threadIdx.x;
+    if (co >= c_out) return;
+    float dsum = 0.f;
+    for (int sp = 0; sp < bsplits; ++sp) dsum += bsum_part[(size_t)sp * c_out + co];
+    if (!vec3) {
+        if (db) db[co] = dsum;
+        return;
+    }
+    float dot = 0.f;
+    for (int t = 0; t < kt; ++t) dot += dotpart[(size_t)t * c_out + co];
+    const float s = vec3[co], r = vec3[2 * c_out + co];
+    dbeta[co] = dsum;
+    if (db) db[co] = s * dsum;
+    dgamma[co] = r * (dot + dsum * ((b ? b[co] : 0.f) - mean[co]));
+}
+
+cudaError_t launch_wgrad_epilogue_t(const Problem &pb, const UmmaWgradPlan &pl, const float *partials,
+                                    const void *w, const float *vec3, float *dw, float *dotpart,
+                                    cudaStream_t st) {
+    int kper = (pb.kdim + pl.kt - 1) / pl.kt;
+    kper = (kper + 31) / 32 * 32;
+    const int kt = (pb.kdim + kper - 1) / kper;
+    dim3 grid(pb.c_out / 32, kt);
+    wgrad_epilogue_t_kernel<<<grid, 256, 0, st>>>(pb.c_out, pb.kdim, partials, pl.splits, kper,
+                                                  (const __nv_bfloat16 *)w, vec3, dw, vec3 ? dotpart : nullptr);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_param_finish(const Problem &pb, const UmmaWgradPlan &pl, const float *dotpart,
+                                const float *bsum_part, int bsplits, const float *vec3, const float *b,
+                                const float *mean, float *db, float *dgamma, float *dbeta, cudaStream_t st) {
+    int kper = (pb.kdim + pl.kt - 1) / pl.kt;
+    kper = (kper + 31) / 32 * 32;
+    const int kt = (pb.kdim + kper - 1) / kper;
+    param_finish_kernel<<<(pb.c_out + 127) / 128, 128, 0, st>>>(pb.c_out, dotpart, kt, bsum_part, bsplits, vec3, b,
+                                                               mean, db, dgamma, dbeta);
+    return cudaGetLastError();
+}
+
+}  // namespace convbn
