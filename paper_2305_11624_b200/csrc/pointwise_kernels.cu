@@ -145,17 +145,63 @@ __global__ void __launch_bounds__(256) channel_sum_partial_kernel(int c_out, int
     part[(long long)split * c_out + c] = acc;
 }
 
+// NHWC bf16 with C a multiple of 8: the tensor is a flat array of 16-byte vectors (8 channels);
+// the block size is a multiple of C/8, so a thread always sees the same 8 channels.  Per-thread
+// sums are combined per channel in thread order (fixed), one partial row per block.
+__global__ void __launch_bounds__(256) channel_sum_nhwc8_kernel(int c_out, long long p, int pix_per_block,
+                                                                const uint4 *__restrict__ t,
+                                                                float *__restrict__ part) {
+    __shared__ float red[256][9];
+    const int v = c_out / 8;                       // vectors per pixel
+    const long long vec0 = (long long)blockIdx.x * pix_per_block * v;
+    long long vec1 = vec0 + (long long)pix_per_block * v;
+    if (vec1 > p * v) vec1 = p * v;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (long long i = vec0 + threadIdx.x; i < vec1; i += blockDim.x) {
+        const uint4 q = t[i];
+        const uint32_t u[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            acc[2 * e] += __uint_as_float(u[e] << 16);
+            acc[2 * e + 1] += __uint_as_float(u[e] & 0xFFFF0000u);
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) red[threadIdx.x][e] = acc[e];
+    __syncthreads();
+    if ((int)threadIdx.x < c_out && (int)threadIdx.x < 256) {
+        for (int c = threadIdx.x; c < c_out; c += blockDim.x) {
+            const int g = c / 8, e = c % 8;
+            float s = 0.f;
+            for (int th = g; th < (int)blockDim.x; th += v) s += red[th][e];
+            part[(long long)blockIdx.x * c_out + c] = s;
+        }
+    }
+}
+
+static bool channel_sum_fast(const Problem &pb, int dtype, int layout) {
+    return dtype == CONVBN_BF16 && layout == CONVBN_NHWC && pb.c_out % 8 == 0 && pb.c_out / 8 <= 256;
+}
+
 int channel_sum_splits(const Problem &pb) {
-    long long want = (148LL * 2048 + pb.c_out - 1) / pb.c_out;
-    long long cap = pb.p / 16;
-    if (cap < 1) cap = 1;
+    // shared by both kernels: about four blocks per SM, at least 64 pixels each
+    long long want = 592;
+    long long cap = (pb.p + 63) / 64;
     if (want > cap) want = cap;
-    if (want > 2048) want = 2048;
-    return (int)(want < 1 ? 1 : want);
+    if (want < 1) want = 1;
+    const long long per = (pb.p + want - 1) / want;
+    return (int)((pb.p + per - 1) / per);
 }
 
 cudaError_t launch_channel_sum_partial(const Problem &pb, int dtype, int layout, const void *t,
                                        float *part, int splits, cudaStream_t st) {
+    if (channel_sum_fast(pb, dtype, layout)) {
+        const int v = pb.c_out / 8;
+        const int block = (256 / v) * v;
+        const long long per = (pb.p + splits - 1) / splits;
+        channel_sum_nhwc8_kernel<<<splits, block, 0, st>>>(pb.c_out, pb.p, (int)per, (const uint4 *)t, part);
+        return cudaGetLastError();
+    }
     const int threads = pb.c_out >= 256 ? 256 : ((pb.c_out + 31) / 32) * 32;
     dim3 grid((pb.c_out + threads - 1) / threads, splits);
     if (dtype == CONVBN_F32 && layout == CONVBN_NCHW)

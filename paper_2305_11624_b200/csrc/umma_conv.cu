@@ -39,11 +39,16 @@ struct ConvGemm {
 struct ConvSmemCtl {
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
-    uint64_t tmem_full;
+    uint64_t tmem_full[2];     // MMA issuer -> epilogue, one per accumulator buffer
+    uint64_t tmem_empty[2];    // epilogue -> MMA issuer (4 arrivals: one per epilogue warp)
     uint32_t tmem_base;
     int abort_flag;
 };
 
+// Persistent: CTA b works on tiles b, b + gridDim.x, ...; tile t covers output pixels
+// [128 (t / n_tiles), +128) and output channels [BN (t % n_tiles), +BN).  The accumulator is
+// double-buffered in tensor memory (2 x BN columns), so the MMAs of a tile overlap the epilogue of
+// the tile before, and the TMA ring runs ahead across tile boundaries.
 template <int BN>
 __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_constant__ CUtensorMap tm_act,
                                                                 const __grid_constant__ CUtensorMap tm_w,
@@ -57,18 +62,18 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
     const int stages = g.stages;
     const int cchunks = g.ca / kBK;
     const int num_kb = g.taps_h * g.taps_w * cchunks;
-    const long long m0 = (long long)blockIdx.x * kBM;
-    const int n0 = blockIdx.y * BN;
+    const int n_tiles = (g.cn + BN - 1) / BN;
+    const long long total_tiles = ((g.p + kBM - 1) / kBM) * n_tiles;
     volatile int *abort_flag = &ctl->abort_flag;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
-        mbar_init(&ctl->tmem_full, 1);
+        for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tmem_full[a], 1); mbar_init(&ctl->tmem_empty[a], 4); }
         ctl->abort_flag = 0;
         fence_barrier_init();
     }
     if (warp == 1) {
-        tmem_alloc(&ctl->tmem_base, BN);
+        tmem_alloc(&ctl->tmem_base, 2 * BN);
         tmem_relinquish();
     }
     tc_fence_before_sync();
@@ -81,86 +86,120 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
         if (elect_one()) {
             prefetch_tensormap(&tm_act);
             prefetch_tensormap(&tm_w);
-            const int wo0 = (int)(m0 % g.wo);
-            const long long t = m0 / g.wo;
-            const int ho0 = (int)(t % g.ho), img0 = (int)(t / g.ho);
-            const int base_w = g.lower_w + wo0 * g.stride_w, base_h = g.lower_h + ho0 * g.stride_h;
-            int issued = 0;
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % stages;
-                const uint32_t ph = (uint32_t)(kb / stages) & 1u;
-                if (!mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag)) {
-                    atomicOr(err, ERRW_TIMEOUT);
-                    ctl->abort_flag = 1;
-                    break;
+            long long it = 0;
+            bool ok = true;
+            for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                const long long m0 = (t / n_tiles) * kBM;
+                const int n0 = (int)(t % n_tiles) * BN;
+                const int wo0 = (int)(m0 % g.wo);
+                const long long tq = m0 / g.wo;
+                const int ho0 = (int)(tq % g.ho), img0 = (int)(tq / g.ho);
+                const int base_w = g.lower_w + wo0 * g.stride_w, base_h = g.lower_h + ho0 * g.stride_h;
+                int tap = 0, cc = 0;
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = (int)(it % stages);
+                    const uint32_t ph = (uint32_t)(it / stages) & 1u;
+                    if (!mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag)) {
+                        atomicOr(err, ERRW_TIMEOUT);
+                        ctl->abort_flag = 1;
+                        ok = false;
+                        break;
+                    }
+                    const int r = tap / g.taps_w, q = tap - r * g.taps_w;
+                    uint8_t *a_dst = tiles + (size_t)s * kStageBytes, *b_dst = a_dst + kABytes;
+                    mbar_arrive_expect_tx(&ctl->full[s], kStageBytes);
+                    tma_load_im2col_4d(a_dst, &tm_act, &ctl->full[s], cc * kBK, base_w, base_h, img0,
+                                       (uint16_t)(q * g.dil_w), (uint16_t)(r * g.dil_h));
+                    tma_load_2d(b_dst, &tm_w, &ctl->full[s], kb * kBK, n0);
+                    if (++cc == cchunks) { cc = 0; ++tap; }
                 }
-                const int tap = kb / cchunks, cc = kb - tap * cchunks;
-                const int r = tap / g.taps_w, q = tap - r * g.taps_w;
-                uint8_t *a_dst = tiles + (size_t)s * kStageBytes, *b_dst = a_dst + kABytes;
-                mbar_arrive_expect_tx(&ctl->full[s], kStageBytes);
-                tma_load_im2col_4d(a_dst, &tm_act, &ctl->full[s], cc * kBK, base_w, base_h, img0,
-                                   (uint16_t)(q * g.dil_w), (uint16_t)(r * g.dil_h));
-                tma_load_2d(b_dst, &tm_w, &ctl->full[s], kb * kBK, n0);
-                ++issued;
             }
-            if (ctl->abort_flag) {
+            if (!ok) {
                 // Let the copies already issued land (bounded) before the CTA may exit.
-                const int first = issued > stages ? issued - stages : 0;
-                for (int kb = first; kb < issued; ++kb)
-                    mbar_wait_bounded(&ctl->full[kb % stages], (uint32_t)(kb / stages) & 1u, nullptr, 200000000ull);
+                const long long first = it > stages ? it - stages : 0;
+                for (long long j = first; j < it; ++j)
+                    mbar_wait_bounded(&ctl->full[j % stages], (uint32_t)(j / stages) & 1u, nullptr, 200000000ull);
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (elect_one()) {
             constexpr uint32_t idesc = idesc_bf16_f32(kBM, BN, 0, 0);
+            long long it = 0;
+            uint32_t i = 0;
             bool ok = true;
-            for (int kb = 0; kb < num_kb && ok; ++kb) {
-                const int s = kb % stages;
-                const uint32_t ph = (uint32_t)(kb / stages) & 1u;
-                if (!mbar_wait_bounded(&ctl->full[s], ph, abort_flag)) {
-                    atomicOr(err, ERRW_TIMEOUT);
-                    ctl->abort_flag = 1;
-                    ok = false;
-                    break;
-                }
+            for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++i) {
+                const uint32_t acc = i & 1u;
+                if (!mbar_wait_bounded(&ctl->tmem_empty[acc], ((i >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after_sync();
-                const uint32_t a_addr = smem_u32(tiles + (size_t)s * kStageBytes), b_addr = a_addr + kABytes;
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = (int)(it % stages);
+                    const uint32_t ph = (uint32_t)(it / stages) & 1u;
+                    if (!mbar_wait_bounded(&ctl->full[s], ph, abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t a_addr = smem_u32(tiles + (size_t)s * kStageBytes), b_addr = a_addr + kABytes;
 #pragma unroll
-                for (int k = 0; k < kBK / kUmmaK; ++k) {
-                    const uint64_t ad = smem_desc_sw128(a_addr + k * kUmmaK * 2, 16, 1024);
-                    const uint64_t bd = smem_desc_sw128(b_addr + k * kUmmaK * 2, 16, 1024);
-                    umma_bf16_ss(tmem_base, ad, bd, idesc, (kb | k) ? 1u : 0u);
+                    for (int k = 0; k < kBK / kUmmaK; ++k) {
+                        const uint64_t ad = smem_desc_sw128(a_addr + k * kUmmaK * 2, 16, 1024);
+                        const uint64_t bd = smem_desc_sw128(b_addr + k * kUmmaK * 2, 16, 1024);
+                        umma_bf16_ss(d_tmem, ad, bd, idesc, (kb | k) ? 1u : 0u);
+                    }
+                    umma_commit(&ctl->empty[s]);
                 }
-                umma_commit(&ctl->empty[s]);
+                if (ok) umma_commit(&ctl->tmem_full[acc]);
             }
-            if (ok) umma_commit(&ctl->tmem_full);
+            if (!ok) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
         }
     } else {
         // ---------------- epilogue: tensor memory -> registers -> bf16 -> global ----------------
-        const int quarter = warp & 3;                      // lanes this warp may read
-        const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->tmem_full, 0, abort_flag));
-        if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
-        if (ok) {
+        const int quarter = warp & 3;                      // tensor-memory lanes this warp may read
+        uint32_t i = 0;
+        for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x, ++i) {
+            const uint32_t acc = i & 1u;
+            const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->tmem_full[acc], (i >> 1) & 1u, abort_flag));
+            if (!ok) {
+                if (lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+                break;
+            }
             tc_fence_after_sync();
+            const long long m0 = (t / n_tiles) * kBM;
+            const int n0 = (int)(t % n_tiles) * BN;
             const long long m = m0 + quarter * 32 + lane;
             const bool row_ok = m < g.p;
             __nv_bfloat16 *orow = out + (size_t)(row_ok ? m : 0) * g.cn + n0;
+            const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
+            const bool bias_vec = bias && (((uintptr_t)bias & 15) == 0);
+            int ncols = g.cn - n0;                          // valid columns of this tile (multiple of 8)
+            if (ncols > BN) ncols = BN;
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
-                if (n0 + c0 >= g.cn) break;                 // warp-uniform
                 uint32_t v[32];
-                tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
-                tmem_ld_wait();
-                if (row_ok) {
+                if (c0 < ncols) {
+                    tmem_ld_32x32(t_row + (uint32_t)c0, v);
+                    tmem_ld_wait();
+                }
+                if (c0 + 32 >= BN) {
+                    // every column of this accumulator has been read: hand the buffer back
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ctl->tmem_empty[acc]);
+                }
+                if (row_ok && c0 < ncols) {
 #pragma unroll
                     for (int j = 0; j < 32; j += 8) {
-                        if (n0 + c0 + j < g.cn) {           // cn is a multiple of 8
+                        if (c0 + j < ncols) {
                             float f[8];
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) {
-                                f[e] = __uint_as_float(v[j + e]);
-                                if (bias) f[e] += __ldg(bias + n0 + c0 + j + e);
+                            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[j + e]);
+                            if (bias && !bias_vec) {
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) f[e] += __ldg(bias + n0 + c0 + j + e);
+                            } else if (bias) {
+                                const float4 b0 = __ldg((const float4 *)(bias + n0 + c0 + j));
+                                const float4 b1 = __ldg((const float4 *)(bias + n0 + c0 + j + 4));
+                                f[0] += b0.x; f[1] += b0.y; f[2] += b0.z; f[3] += b0.w;
+                                f[4] += b1.x; f[5] += b1.y; f[6] += b1.z; f[7] += b1.w;
                             }
                             uint4 pk;
                             __nv_bfloat162 h;
@@ -177,7 +216,7 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem_base, BN);
+    if (warp == 1) tmem_dealloc(tmem_base, 2 * BN);
 }
 
 // ---- host side: tensor maps and launch ---------------------------------------------------------
@@ -250,21 +289,27 @@ bool umma_conv_eligible(const UmmaConvShape &s) {
     return true;
 }
 
+static int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            n = v;
+        else
+            n = 148;
+    }
+    return n;
+}
+
 template <int BN>
 static cudaError_t launch_bn(const CUtensorMap &ta, const CUtensorMap &tw, ConvGemm g, const float *bias,
                              void *out, int *err, cudaStream_t st) {
     constexpr size_t stage = (size_t)kBM * kBK * 2 + (size_t)BN * kBK * 2;
-    const int num_kb = g.taps_h * g.taps_w * (g.ca / kBK);
-    int stages = (int)((96 * 1024) / stage);
-    if (stages > num_kb) stages = num_kb;
+    int stages = (int)((192 * 1024) / stage);          // one CTA per SM owns the shared memory
     if (stages > kMaxStages) stages = kMaxStages;
-    if (stages < 1) stages = 1;
     g.stages = stages;
-    // Tensor memory has 512 columns per SM and every CTA takes BN of them: ask for enough shared
-    // memory that no more than 512 / BN CTAs are resident, so an allocation never has to wait.
-    size_t smem = stages * stage + 1024 + sizeof(ConvSmemCtl);
-    const size_t floor_smem = (size_t)(228 * 1024) / (512 / BN + 1) + 1024;
-    if (smem < floor_smem) smem = floor_smem;
+    const size_t smem = stages * stage + 1024 + sizeof(ConvSmemCtl);
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(umma_conv_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -272,9 +317,27 @@ static cudaError_t launch_bn(const CUtensorMap &ta, const CUtensorMap &tw, ConvG
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    dim3 grid((unsigned)((g.p + kBM - 1) / kBM), (unsigned)((g.cn + BN - 1) / BN));
+    const long long total = ((g.p + kBM - 1) / kBM) * ((g.cn + BN - 1) / BN);
+    const unsigned grid = (unsigned)(total < sm_count() ? total : sm_count());
     umma_conv_kernel<BN><<<grid, kConvThreads, smem, st>>>(ta, tw, g, bias, (__nv_bfloat16 *)out, err);
     return cudaGetLastError();
+}
+
+// Tile width: fewest rounds of tiles over the SMs, weighted by the time of one tile (N = 64 tiles are
+// bound by shared-memory operand bandwidth, about 1.5x slower per column than wider ones).
+static int pick_bn(long long tiles_m, int cn) {
+    int best = 64;
+    double best_cost = 1e30;
+    const int cand[3] = {256, 128, 64};
+    for (int c = 0; c < 3; ++c) {
+        const int bn = cand[c];
+        if (bn > 64 && cn <= bn / 2) continue;
+        const long long tiles = tiles_m * ((cn + bn - 1) / bn);
+        const long long rounds = (tiles + sm_count() - 1) / sm_count();
+        const double cost = (double)rounds * bn * (bn == 64 ? 1.5 : 1.0);
+        if (cost < best_cost) { best_cost = cost; best = bn; }
+    }
+    return best;
 }
 
 cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void *wmat, const float *bias,
@@ -287,11 +350,7 @@ cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void
     const int upper_h = s.lower_h + (s.ho - 1) * s.stride_h - (s.ha - 1);
     const int upper_w = s.lower_w + (s.wo - 1) * s.stride_w - (s.wa - 1);
     const long long tiles_m = (g.p + kBM - 1) / kBM;
-    int bn = 64;
-    if (s.cn > 64) {
-        bn = (s.cn >= 256 && tiles_m * ((s.cn + 255) / 256) >= 148) ? 256 : 128;
-        if (bn == 128 && tiles_m * ((s.cn + 127) / 128) < 148) bn = 64;
-    }
+    const int bn = pick_bn(tiles_m, s.cn);
     CUtensorMap ta, tw;
     if (!make_tmap_im2col_bf16(&ta, act, s.n, s.ha, s.wa, s.ca, s.lower_h, s.lower_w, upper_h, upper_w, s.stride_h,
                                s.stride_w, kBM, kBK))

@@ -182,7 +182,7 @@ UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
     UmmaWgradPlan pl;
     const int bn = wgrad_bn(pb);
     const long long m_tiles = (pb.kdim + kWM - 1) / kWM, n_tiles = (pb.c_out + bn - 1) / bn;
-    const long long target = bn == 256 ? 148 : 296;
+    const long long target = 148;
     long long splits = (target + m_tiles * n_tiles - 1) / (m_tiles * n_tiles);
     const long long max_splits = (pb.p + 4 * kWP - 1) / (4 * kWP);     // at least 256 pixels per slice
     if (splits > max_splits) splits = max_splits;
@@ -191,11 +191,7 @@ UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
     per = (per + kWP - 1) / kWP * kWP;
     pl.per_split = per;
     pl.splits = (int)((pb.p + per - 1) / per);
-    int kt = (int)(296 / (pb.c_out / 32));
-    const int kt_max = (pb.kdim + 31) / 32;
-    if (kt > kt_max) kt = kt_max;
-    if (kt < 1) kt = 1;
-    pl.kt = kt;
+    pl.kt = (pb.kdim + 7) / 8;        // epilogue blocks along k (8 rows each) = rows of dotpart
     return pl;
 }
 
@@ -245,75 +241,73 @@ cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
 }
 
 // ---- epilogue over k-major partials ------------------------------------------------------------
-// part[split][k][co] -> dw[co][k] = scale[co] * sum_split part;  dotpart[kt][co] = sum over this block's
-// k range of (sum_split part) * w[co][k].  Block = 32 output channels x one k range; 32 x 8 threads.
+// part[split][k][co] -> dw[co][k] = scale[co] * sum_split part;  dotpart[blockIdx.y][co] = sum over the
+// block's 8 k rows of (sum_split part) * w[co][k].  Block = 32 output channels x 8 k rows.
 __global__ void __launch_bounds__(256) wgrad_epilogue_t_kernel(int c_out, int kdim, const float *__restrict__ part,
-                                                              int splits, int kper,
-                                                              const __nv_bfloat16 *__restrict__ w,
+                                                              int splits, const __nv_bfloat16 *__restrict__ w,
                                                               const float *__restrict__ vec3,
                                                               float *__restrict__ dw, float *__restrict__ dotpart) {
-    __shared__ float tile[32][33];
-    __shared__ float wtile[32][33];
+    __shared__ float tile[8][33];
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    const int co0 = blockIdx.x * 32;
-    const int kbeg = blockIdx.y * kper, kend = min(kdim, kbeg + kper);
+    const int co0 = blockIdx.x * 32, k0 = blockIdx.y * 8;
     const size_t slice = (size_t)kdim * c_out;
-    float dot[4] = {0.f, 0.f, 0.f, 0.f};
-    float sc[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) sc[j] = vec3 ? vec3[co0 + ty + 8 * j] : 1.f;
-    for (int kb = kbeg; kb < kend; kb += 32) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int kl = ty + 8 * j, k = kb + kl;
-            float acc = 0.f;
-            if (k < kend) {
-                const float *src = part + (size_t)k * c_out + co0 + tx;
-                for (int sp = 0; sp < splits; ++sp) acc += src[sp * slice];
+    {
+        const int k = k0 + ty;
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        if (k < kdim) {
+            const float *src = part + (size_t)k * c_out + co0 + tx;
+            int sp = 0;
+            for (; sp + 4 <= splits; sp += 4) {
+                a0 += src[(size_t)sp * slice];
+                a1 += src[(size_t)(sp + 1) * slice];
+                a2 += src[(size_t)(sp + 2) * slice];
+                a3 += src[(size_t)(sp + 3) * slice];
             }
-            tile[kl][tx] = acc;
-            const int kr = kb + tx;          // w[co0 + kl][kb + tx], coalesced along k
-            wtile[kl][tx] = (vec3 && kr < kend) ? __bfloat162float(w[(size_t)(co0 + kl) * kdim + kr]) : 0.f;
+            for (; sp < splits; ++sp) a0 += src[(size_t)sp * slice];
         }
-        __syncthreads();
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int cl = ty + 8 * j, k = kb + tx;
-            if (k < kend) {
-                const float v = tile[tx][cl];
-                dw[(size_t)(co0 + cl) * kdim + k] = sc[j] * v;
-                dot[j] = fmaf(v, wtile[cl][tx], dot[j]);
-            }
-        }
-        __syncthreads();
+        tile[ty][tx] = (a0 + a1) + (a2 + a3);
+    }
+    __syncthreads();
+    const int kk = threadIdx.x & 7, cl = threadIdx.x >> 3, k = k0 + kk, co = co0 + cl;
+    float d = 0.f;
+    if (k < kdim) {
+        const float v = tile[kk][cl];
+        const size_t o = (size_t)co * kdim + k;
+        dw[o] = (vec3 ? vec3[co] : 1.f) * v;
+        if (dotpart) d = v * __bfloat162float(w[o]);
     }
     if (dotpart) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            float d = dot[j];
-            for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
-            if (tx == 0) dotpart[(size_t)blockIdx.y * c_out + co0 + ty + 8 * j] = d;
-        }
+        d += __shfl_xor_sync(0xffffffffu, d, 1);
+        d += __shfl_xor_sync(0xffffffffu, d, 2);
+        d += __shfl_xor_sync(0xffffffffu, d, 4);
+        if (kk == 0) dotpart[(size_t)blockIdx.y * c_out + co] = d;
     }
 }
 
-// dbeta = sum dZ; db = s dbeta; dgamma = r (sum_k domega' omega + dbeta (b - mu_hat))   (Table 2, Tune row)
-// plain mode (vec3 == NULL): db = sum dZ only.
-__global__ void param_finish_kernel(int c_out, const float *__restrict__ dotpart, int kt,
-                                    const float *__restrict__ bsum_part, int bsplits,
-                                    const float *__restrict__ vec3, const float *__restrict__ b,
-                                    const float *__restrict__ mean, float *__restrict__ db,
-                                    float *__restrict__ dgamma, float *__restrict__ dbeta) {
-    const int co = blockIdx.x * blockDim.x + threadIdx.x;
+// One warp per output channel: dbeta = sum dZ; db = s dbeta;
+// dgamma = r (sum_k domega' omega + dbeta (b - mu_hat))   (Table 2, Tune row).
+// Plain mode (vec3 == NULL): db = sum dZ only.  Lanes add strided pieces, then a fixed shuffle tree.
+__global__ void __launch_bounds__(256) param_finish_kernel(int c_out, const float *__restrict__ dotpart, int kt,
+                                                          const float *__restrict__ bsum_part, int bsplits,
+                                                          const float *__restrict__ vec3,
+                                                          const float *__restrict__ b,
+                                                          const float *__restrict__ mean, float *__restrict__ db,
+                                                          float *__restrict__ dgamma, float *__restrict__ dbeta) {
+    const int co = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (co >= c_out) return;
-    float dsum = 0.f;
-    for (int sp = 0; sp < bsplits; ++sp) dsum += bsum_part[(size_t)sp * c_out + co];
+    float dsum = 0.f, dot = 0.f;
+    for (int sp = lane; sp < bsplits; sp += 32) dsum += bsum_part[(size_t)sp * c_out + co];
+    if (vec3)
+        for (int t = lane; t < kt; t += 32) dot += dotpart[(size_t)t * c_out + co];
+    for (int o = 16; o > 0; o >>= 1) {
+        dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
+        dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    }
+    if (lane) return;
     if (!vec3) {
         if (db) db[co] = dsum;
         return;
     }
-    float dot = 0.f;
-    for (int t = 0; t < kt; ++t) dot += dotpart[(size_t)t * c_out + co];
     const float s = vec3[co], r = vec3[2 * c_out + co];
     dbeta[co] = dsum;
     if (db) db[co] = s * dsum;
@@ -323,11 +317,8 @@ __global__ void param_finish_kernel(int c_out, const float *__restrict__ dotpart
 cudaError_t launch_wgrad_epilogue_t(const Problem &pb, const UmmaWgradPlan &pl, const float *partials,
                                     const void *w, const float *vec3, float *dw, float *dotpart,
                                     cudaStream_t st) {
-    int kper = (pb.kdim + pl.kt - 1) / pl.kt;
-    kper = (kper + 31) / 32 * 32;
-    const int kt = (pb.kdim + kper - 1) / kper;
-    dim3 grid(pb.c_out / 32, kt);
-    wgrad_epilogue_t_kernel<<<grid, 256, 0, st>>>(pb.c_out, pb.kdim, partials, pl.splits, kper,
+    dim3 grid(pb.c_out / 32, pl.kt);
+    wgrad_epilogue_t_kernel<<<grid, 256, 0, st>>>(pb.c_out, pb.kdim, partials, pl.splits,
                                                   (const __nv_bfloat16 *)w, vec3, dw, vec3 ? dotpart : nullptr);
     return cudaGetLastError();
 }
@@ -335,11 +326,8 @@ cudaError_t launch_wgrad_epilogue_t(const Problem &pb, const UmmaWgradPlan &pl, 
 cudaError_t launch_param_finish(const Problem &pb, const UmmaWgradPlan &pl, const float *dotpart,
                                 const float *bsum_part, int bsplits, const float *vec3, const float *b,
                                 const float *mean, float *db, float *dgamma, float *dbeta, cudaStream_t st) {
-    int kper = (pb.kdim + pl.kt - 1) / pl.kt;
-    kper = (kper + 31) / 32 * 32;
-    const int kt = (pb.kdim + kper - 1) / kper;
-    param_finish_kernel<<<(pb.c_out + 127) / 128, 128, 0, st>>>(pb.c_out, dotpart, kt, bsum_part, bsplits, vec3, b,
-                                                               mean, db, dgamma, dbeta);
+    param_finish_kernel<<<(pb.c_out + 7) / 8, 256, 0, st>>>(pb.c_out, dotpart, pl.kt, bsum_part, bsplits, vec3, b,
+                                                           mean, db, dgamma, dbeta);
     return cudaGetLastError();
 }
 
