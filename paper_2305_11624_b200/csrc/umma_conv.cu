@@ -24,6 +24,8 @@ constexpr int kBK = 64;        // K elements per stage = one 128-byte swizzle ro
 constexpr int kUmmaK = 16;     // K per tcgen05.mma of kind::f16
 constexpr int kMaxStages = 8;
 constexpr int kConvThreads = 192;
+constexpr uint32_t kStagingWarpBytes = 32 * 128;              // [32 rows][64 bf16]
+constexpr uint32_t kStagingBytes = 4 * 2 * kStagingWarpBytes; // 4 epilogue warps, double-buffered
 
 struct ConvGemm {
     int ho, wo;              // output spatial extent
@@ -52,12 +54,15 @@ struct ConvSmemCtl {
 template <int BN>
 __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_constant__ CUtensorMap tm_act,
                                                                 const __grid_constant__ CUtensorMap tm_w,
+                                                                const __grid_constant__ CUtensorMap tm_out,
                                                                 const ConvGemm g, const float *__restrict__ bias,
-                                                                __nv_bfloat16 *__restrict__ out, int *err) {
+                                                                int *err) {
     extern __shared__ uint8_t smem_raw[];
     constexpr uint32_t kABytes = kBM * kBK * 2, kBBytes = BN * kBK * 2, kStageBytes = kABytes + kBBytes;
     uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    ConvSmemCtl *ctl = (ConvSmemCtl *)(tiles + (size_t)g.stages * kStageBytes);
+    uint8_t *staging = tiles + (size_t)g.stages * kStageBytes;         // 4 warps x 2 x [32 rows][128 B]
+    ConvSmemCtl *ctl = (ConvSmemCtl *)(staging + kStagingBytes);
+    float *bias_s = (float *)(((uintptr_t)(ctl + 1) + 15) & ~(uintptr_t)15);   // cn floats
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int stages = g.stages;
     const int cchunks = g.ca / kBK;
@@ -76,6 +81,8 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
         tmem_alloc(&ctl->tmem_base, 2 * BN);
         tmem_relinquish();
     }
+    if (bias)
+        for (int c = threadIdx.x; c < g.cn; c += kConvThreads) bias_s[c] = bias[c];
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -152,9 +159,12 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
             if (!ok) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
         }
     } else {
-        // ---------------- epilogue: tensor memory -> registers -> bf16 -> global ----------------
+        // ---------------- epilogue: tensor memory -> registers -> bf16 -> shared -> TMA store --------
+        // Each warp owns 32 accumulator rows and two private [32 rows][64 columns] staging buffers
+        // (128-byte swizzle), so only warp-level synchronisation is needed.
         const int quarter = warp & 3;                      // tensor-memory lanes this warp may read
-        uint32_t i = 0;
+        uint8_t *stage_buf = staging + (size_t)quarter * 2 * kStagingWarpBytes;
+        uint32_t i = 0, sbuf = 0;
         for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x, ++i) {
             const uint32_t acc = i & 1u;
             const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->tmem_full[acc], (i >> 1) & 1u, abort_flag));
@@ -165,54 +175,59 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
             tc_fence_after_sync();
             const long long m0 = (t / n_tiles) * kBM;
             const int n0 = (int)(t % n_tiles) * BN;
-            const long long m = m0 + quarter * 32 + lane;
-            const bool row_ok = m < g.p;
-            __nv_bfloat16 *orow = out + (size_t)(row_ok ? m : 0) * g.cn + n0;
             const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
-            const bool bias_vec = bias && (((uintptr_t)bias & 15) == 0);
-            int ncols = g.cn - n0;                          // valid columns of this tile (multiple of 8)
+            int ncols = g.cn - n0;                          // valid columns of this tile
             if (ncols > BN) ncols = BN;
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t v[32];
+            for (int c0 = 0; c0 < BN; c0 += 64) {
+                uint32_t v[64];
                 if (c0 < ncols) {
-                    tmem_ld_32x32(t_row + (uint32_t)c0, v);
+                    tmem_ld_32x32(t_row + (uint32_t)c0, *(uint32_t(*)[32]) & v[0]);
+                    tmem_ld_32x32(t_row + (uint32_t)c0 + 32, *(uint32_t(*)[32]) & v[32]);
                     tmem_ld_wait();
                 }
-                if (c0 + 32 >= BN) {
+                if (c0 + 64 >= BN) {
                     // every column of this accumulator has been read: hand the buffer back
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&ctl->tmem_empty[acc]);
                 }
-                if (row_ok && c0 < ncols) {
+                if (c0 < ncols) {
+                    uint8_t *buf = stage_buf + (size_t)sbuf * kStagingWarpBytes;
+                    // the store issued two groups ago read this buffer: wait until it no longer does
+                    if (lane == 0) tma_store_wait_read<1>();
+                    __syncwarp();
+                    uint8_t *row = buf + lane * 128;
 #pragma unroll
-                    for (int j = 0; j < 32; j += 8) {
-                        if (c0 + j < ncols) {
-                            float f[8];
+                    for (int j = 0; j < 64; j += 8) {
+                        float f[8];
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[j + e]);
-                            if (bias && !bias_vec) {
-#pragma unroll
-                                for (int e = 0; e < 8; ++e) f[e] += __ldg(bias + n0 + c0 + j + e);
-                            } else if (bias) {
-                                const float4 b0 = __ldg((const float4 *)(bias + n0 + c0 + j));
-                                const float4 b1 = __ldg((const float4 *)(bias + n0 + c0 + j + 4));
-                                f[0] += b0.x; f[1] += b0.y; f[2] += b0.z; f[3] += b0.w;
-                                f[4] += b1.x; f[5] += b1.y; f[6] += b1.z; f[7] += b1.w;
-                            }
-                            uint4 pk;
-                            __nv_bfloat162 h;
-                            h = __floats2bfloat162_rn(f[0], f[1]); pk.x = *(uint32_t *)&h;
-                            h = __floats2bfloat162_rn(f[2], f[3]); pk.y = *(uint32_t *)&h;
-                            h = __floats2bfloat162_rn(f[4], f[5]); pk.z = *(uint32_t *)&h;
-                            h = __floats2bfloat162_rn(f[6], f[7]); pk.w = *(uint32_t *)&h;
-                            *(uint4 *)(orow + c0 + j) = pk;
+                        for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[j + e]);
+                        if (bias) {
+                            const float4 b0 = *(const float4 *)(bias_s + n0 + c0 + j);
+                            const float4 b1 = *(const float4 *)(bias_s + n0 + c0 + j + 4);
+                            f[0] += b0.x; f[1] += b0.y; f[2] += b0.z; f[3] += b0.w;
+                            f[4] += b1.x; f[5] += b1.y; f[6] += b1.z; f[7] += b1.w;
                         }
+                        uint4 pk;
+                        __nv_bfloat162 h;
+                        h = __floats2bfloat162_rn(f[0], f[1]); pk.x = *(uint32_t *)&h;
+                        h = __floats2bfloat162_rn(f[2], f[3]); pk.y = *(uint32_t *)&h;
+                        h = __floats2bfloat162_rn(f[4], f[5]); pk.z = *(uint32_t *)&h;
+                        h = __floats2bfloat162_rn(f[6], f[7]); pk.w = *(uint32_t *)&h;
+                        *(uint4 *)(row + ((((j >> 3) ^ (lane & 7)) & 7) << 4)) = pk;
                     }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&tm_out, buf, n0 + c0, (int)(m0 + quarter * 32));
+                        tma_store_commit();
+                    }
+                    sbuf ^= 1u;
                 }
             }
         }
+        if (lane == 0) tma_store_wait_all<0>();             // global writes done before the CTA exits
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -281,7 +296,7 @@ bool make_tmap_im2col_bf16(CUtensorMap *tm, const void *base, int n, int h, int 
 }
 
 bool umma_conv_eligible(const UmmaConvShape &s) {
-    if (s.ca % kBK || s.cn % 8 || s.cn < 8) return false;
+    if (s.ca % kBK || s.cn % 8 || s.cn < 64 || s.cn > 4096) return false;
     if (s.lower_h < -128 || s.lower_h > 127 || s.lower_w < -128 || s.lower_w > 127) return false;
     if ((s.taps_h - 1) * s.dil_h > 255 || (s.taps_w - 1) * s.dil_w > 255) return false;
     if (s.stride_h > 8 || s.stride_w > 8) return false;
@@ -303,23 +318,24 @@ static int sm_count() {
 }
 
 template <int BN>
-static cudaError_t launch_bn(const CUtensorMap &ta, const CUtensorMap &tw, ConvGemm g, const float *bias,
-                             void *out, int *err, cudaStream_t st) {
+static cudaError_t launch_bn(const CUtensorMap &ta, const CUtensorMap &tw, const CUtensorMap &tout, ConvGemm g,
+                             const float *bias, int *err, cudaStream_t st) {
     constexpr size_t stage = (size_t)kBM * kBK * 2 + (size_t)BN * kBK * 2;
-    int stages = (int)((192 * 1024) / stage);          // one CTA per SM owns the shared memory
+    const size_t fixed = 1024 + kStagingBytes + sizeof(ConvSmemCtl) + (size_t)g.cn * sizeof(float) + 16;
+    int stages = (int)((220 * 1024 - fixed) / stage);  // one CTA per SM owns the shared memory
     if (stages > kMaxStages) stages = kMaxStages;
     g.stages = stages;
-    const size_t smem = stages * stage + 1024 + sizeof(ConvSmemCtl);
+    const size_t smem = stages * stage + fixed;
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(umma_conv_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             200 * 1024);
+                                             224 * 1024);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
     const long long total = ((g.p + kBM - 1) / kBM) * ((g.cn + BN - 1) / BN);
     const unsigned grid = (unsigned)(total < sm_count() ? total : sm_count());
-    umma_conv_kernel<BN><<<grid, kConvThreads, smem, st>>>(ta, tw, g, bias, (__nv_bfloat16 *)out, err);
+    umma_conv_kernel<BN><<<grid, kConvThreads, smem, st>>>(ta, tw, tout, g, bias, err);
     return cudaGetLastError();
 }
 
@@ -351,7 +367,8 @@ cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void
     const int upper_w = s.lower_w + (s.wo - 1) * s.stride_w - (s.wa - 1);
     const long long tiles_m = (g.p + kBM - 1) / kBM;
     const int bn = pick_bn(tiles_m, s.cn);
-    CUtensorMap ta, tw;
+    CUtensorMap ta, tw, tout;
+    if (!make_tmap_matrix_bf16(&tout, out, g.p, s.cn, 32, 64)) return cudaErrorInvalidValue;
     if (!make_tmap_im2col_bf16(&ta, act, s.n, s.ha, s.wa, s.ca, s.lower_h, s.lower_w, upper_h, upper_w, s.stride_h,
                                s.stride_w, kBM, kBK))
         return cudaErrorInvalidValue;
@@ -360,9 +377,9 @@ cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void
     int *err = nullptr;
     cudaError_t e = error_word_address(&err);
     if (e != cudaSuccess) return e;
-    if (bn == 64) return launch_bn<64>(ta, tw, g, bias, out, err, st);
-    if (bn == 128) return launch_bn<128>(ta, tw, g, bias, out, err, st);
-    return launch_bn<256>(ta, tw, g, bias, out, err, st);
+    if (bn == 64) return launch_bn<64>(ta, tw, tout, g, bias, err, st);
+    if (bn == 128) return launch_bn<128>(ta, tw, tout, g, bias, err, st);
+    return launch_bn<256>(ta, tw, tout, g, bias, err, st);
 }
 
 }  // namespace convbn
