@@ -23,9 +23,9 @@ constexpr int kBM = 128;       // output pixels per tile (UMMA M)
 constexpr int kBK = 64;        // K elements per stage = one 128-byte swizzle row of bf16
 constexpr int kUmmaK = 16;     // K per tcgen05.mma of kind::f16
 constexpr int kMaxStages = 8;
-constexpr int kConvThreads = 192;
+constexpr int kConvThreads = 320;                             // TMA warp, MMA warp, 2 x 4 epilogue warps
 constexpr uint32_t kStagingWarpBytes = 32 * 128;              // [32 rows][64 bf16]
-constexpr uint32_t kStagingBytes = 4 * 2 * kStagingWarpBytes; // 4 epilogue warps, double-buffered
+constexpr uint32_t kStagingBytes = 8 * 2 * kStagingWarpBytes; // 8 epilogue warps, double-buffered
 
 struct ConvGemm {
     int ho, wo;              // output spatial extent
@@ -93,19 +93,22 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
         if (elect_one()) {
             prefetch_tensormap(&tm_act);
             prefetch_tensormap(&tm_w);
-            long long it = 0;
+            uint32_t it = 0;                         // k-blocks issued so far
+            int s = 0;                               // ring slot and its phase, advanced incrementally
+            uint32_t ph = 0;
             bool ok = true;
             for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const long long m0 = (t / n_tiles) * kBM;
-                const int n0 = (int)(t % n_tiles) * BN;
-                const int wo0 = (int)(m0 % g.wo);
-                const long long tq = m0 / g.wo;
-                const int ho0 = (int)(tq % g.ho), img0 = (int)(tq / g.ho);
+                // 32-bit arithmetic: 64-bit divisions cost this single thread about a microsecond per tile
+                const uint32_t tt = (uint32_t)t, mt = tt / (uint32_t)n_tiles;
+                const uint32_t m0 = mt * kBM;
+                const int n0 = (int)(tt - mt * (uint32_t)n_tiles) * BN;
+                const uint32_t tq = m0 / (uint32_t)g.wo;
+                const int wo0 = (int)(m0 - tq * (uint32_t)g.wo);
+                const uint32_t img = tq / (uint32_t)g.ho;
+                const int ho0 = (int)(tq - img * (uint32_t)g.ho), img0 = (int)img;
                 const int base_w = g.lower_w + wo0 * g.stride_w, base_h = g.lower_h + ho0 * g.stride_h;
                 int tap = 0, cc = 0;
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const int s = (int)(it % stages);
-                    const uint32_t ph = (uint32_t)(it / stages) & 1u;
                     if (!mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag)) {
                         atomicOr(err, ERRW_TIMEOUT);
                         ctl->abort_flag = 1;
@@ -119,20 +122,22 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                                        (uint16_t)(q * g.dil_w), (uint16_t)(r * g.dil_h));
                     tma_load_2d(b_dst, &tm_w, &ctl->full[s], kb * kBK, n0);
                     if (++cc == cchunks) { cc = 0; ++tap; }
+                    if (++s == stages) { s = 0; ph ^= 1u; }
                 }
             }
             if (!ok) {
                 // Let the copies already issued land (bounded) before the CTA may exit.
-                const long long first = it > stages ? it - stages : 0;
-                for (long long j = first; j < it; ++j)
-                    mbar_wait_bounded(&ctl->full[j % stages], (uint32_t)(j / stages) & 1u, nullptr, 200000000ull);
+                const uint32_t first = it > (uint32_t)stages ? it - stages : 0;
+                for (uint32_t j = first; j < it; ++j)
+                    mbar_wait_bounded(&ctl->full[j % stages], (j / stages) & 1u, nullptr, 200000000ull);
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (elect_one()) {
             constexpr uint32_t idesc = idesc_bf16_f32(kBM, BN, 0, 0);
-            long long it = 0;
+            int s = 0;
+            uint32_t ph = 0;
             uint32_t i = 0;
             bool ok = true;
             for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++i) {
@@ -140,9 +145,7 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                 if (!mbar_wait_bounded(&ctl->tmem_empty[acc], ((i >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * BN;
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const int s = (int)(it % stages);
-                    const uint32_t ph = (uint32_t)(it / stages) & 1u;
+                for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait_bounded(&ctl->full[s], ph, abort_flag)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint32_t a_addr = smem_u32(tiles + (size_t)s * kStageBytes), b_addr = a_addr + kABytes;
@@ -153,6 +156,7 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                         umma_bf16_ss(d_tmem, ad, bd, idesc, (kb | k) ? 1u : 0u);
                     }
                     umma_commit(&ctl->empty[s]);
+                    if (++s == stages) { s = 0; ph ^= 1u; }
                 }
                 if (ok) umma_commit(&ctl->tmem_full[acc]);
             }
@@ -160,21 +164,24 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
         }
     } else {
         // ---------------- epilogue: tensor memory -> registers -> bf16 -> shared -> TMA store --------
-        // Each warp owns 32 accumulator rows and two private [32 rows][64 columns] staging buffers
-        // (128-byte swizzle), so only warp-level synchronisation is needed.
+        // Two groups of four warps; group e drains accumulator buffer e, i.e. every other tile of this
+        // CTA, so two tiles are in their epilogue at once.  Each warp owns 32 accumulator rows and two
+        // private [32 rows][64 columns] staging buffers (128-byte swizzle): warp-level sync only.
         const int quarter = warp & 3;                      // tensor-memory lanes this warp may read
-        uint8_t *stage_buf = staging + (size_t)quarter * 2 * kStagingWarpBytes;
-        uint32_t i = 0, sbuf = 0;
-        for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x, ++i) {
-            const uint32_t acc = i & 1u;
+        const uint32_t egroup = (uint32_t)(warp - 2) >> 2; // 0: warps 2-5, 1: warps 6-9
+        uint8_t *stage_buf = staging + (size_t)(warp - 2) * 2 * kStagingWarpBytes;
+        uint32_t i = egroup, sbuf = 0;
+        for (long long t = blockIdx.x + (long long)egroup * gridDim.x; t < total_tiles; t += 2LL * gridDim.x, i += 2) {
+            const uint32_t acc = egroup;
             const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->tmem_full[acc], (i >> 1) & 1u, abort_flag));
             if (!ok) {
                 if (lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
                 break;
             }
             tc_fence_after_sync();
-            const long long m0 = (t / n_tiles) * kBM;
-            const int n0 = (int)(t % n_tiles) * BN;
+            const uint32_t tt = (uint32_t)t, mt = tt / (uint32_t)n_tiles;
+            const uint32_t m0 = mt * kBM;
+            const int n0 = (int)(tt - mt * (uint32_t)n_tiles) * BN;
             const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
             int ncols = g.cn - n0;                          // valid columns of this tile
             if (ncols > BN) ncols = BN;
@@ -301,6 +308,7 @@ bool umma_conv_eligible(const UmmaConvShape &s) {
     if ((s.taps_h - 1) * s.dil_h > 255 || (s.taps_w - 1) * s.dil_w > 255) return false;
     if (s.stride_h > 8 || s.stride_w > 8) return false;
     if ((long long)s.taps_h * s.taps_w * s.ca > (1 << 24)) return false;
+    if ((long long)s.n * s.ho * s.wo >= (1LL << 31) - 256) return false;
     return true;
 }
 

@@ -80,19 +80,20 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
             prefetch_tensormap(&tm_x);
             prefetch_tensormap(&tm_dz);
             const uint32_t tx_bytes = (uint32_t)(a_chunks + b_chunks) * kChunkBytes;
-            int issued = 0;
+            int issued = 0, s = 0;
+            uint32_t ph = 0;
             for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % stages;
-                const uint32_t ph = (uint32_t)(kb / stages) & 1u;
                 if (!mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag)) {
                     atomicOr(err, ERRW_TIMEOUT);
                     ctl->abort_flag = 1;
                     break;
                 }
-                const long long pp = p0 + (long long)kb * kWP;
-                const int wo0 = (int)(pp % g.wo);
-                const long long t = pp / g.wo;
-                const int ho0 = (int)(t % g.ho), img0 = (int)(t / g.ho);
+                // 32-bit arithmetic on purpose (64-bit divisions would dominate this thread's loop)
+                const uint32_t pp = (uint32_t)p0 + (uint32_t)kb * kWP;
+                const uint32_t t = pp / (uint32_t)g.wo;
+                const int wo0 = (int)(pp - t * (uint32_t)g.wo);
+                const uint32_t img = t / (uint32_t)g.ho;
+                const int ho0 = (int)(t - img * (uint32_t)g.ho), img0 = (int)img;
                 const int base_w = g.lower_w + wo0 * g.stride_w, base_h = g.lower_h + ho0 * g.stride_h;
                 uint8_t *a_dst = tiles + (size_t)s * kStageBytes, *b_dst = a_dst + kABytes;
                 mbar_arrive_expect_tx(&ctl->full[s], tx_bytes);
@@ -106,6 +107,7 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
                 for (int j = 0; j < b_chunks; ++j)
                     tma_load_2d(b_dst + j * kChunkBytes, &tm_dz, &ctl->full[s], n0 + j * 64, (int)pp);
                 ++issued;
+                if (++s == stages) { s = 0; ph ^= 1u; }
             }
             if (ctl->abort_flag) {
                 const int first = issued > stages ? issued - stages : 0;
@@ -117,9 +119,9 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
         if (elect_one()) {
             constexpr uint32_t idesc = idesc_bf16_f32(kWM, BN, 1, 1);   // both operands MN-major
             bool ok = true;
+            int s = 0;
+            uint32_t ph = 0;
             for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % stages;
-                const uint32_t ph = (uint32_t)(kb / stages) & 1u;
                 if (!mbar_wait_bounded(&ctl->full[s], ph, abort_flag)) {
                     atomicOr(err, ERRW_TIMEOUT);
                     ctl->abort_flag = 1;
@@ -136,6 +138,7 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
                     umma_bf16_ss(tmem_base, ad, bd, idesc, (kb | k) ? 1u : 0u);
                 }
                 umma_commit(&ctl->empty[s]);
+                if (++s == stages) { s = 0; ph ^= 1u; }
             }
             if (ok) umma_commit(&ctl->tmem_full);
         }
