@@ -90,47 +90,46 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
-        if (elect_one()) {
-            prefetch_tensormap(&tm_act);
-            prefetch_tensormap(&tm_w);
-            uint32_t it = 0;                         // k-blocks issued so far
-            int s = 0;                               // ring slot and its phase, advanced incrementally
-            uint32_t ph = 0;
-            bool ok = true;
-            for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                // 32-bit arithmetic: 64-bit divisions cost this single thread about a microsecond per tile
-                const uint32_t tt = (uint32_t)t, mt = tt / (uint32_t)n_tiles;
-                const uint32_t m0 = mt * kBM;
-                const int n0 = (int)(tt - mt * (uint32_t)n_tiles) * BN;
-                const uint32_t tq = m0 / (uint32_t)g.wo;
-                const int wo0 = (int)(m0 - tq * (uint32_t)g.wo);
-                const uint32_t img = tq / (uint32_t)g.ho;
-                const int ho0 = (int)(tq - img * (uint32_t)g.ho), img0 = (int)img;
-                const int base_w = g.lower_w + wo0 * g.stride_w, base_h = g.lower_h + ho0 * g.stride_h;
-                int tap = 0, cc = 0;
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    if (!mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag)) {
-                        atomicOr(err, ERRW_TIMEOUT);
-                        ctl->abort_flag = 1;
-                        ok = false;
-                        break;
-                    }
-                    const int r = tap / g.taps_w, q = tap - r * g.taps_w;
-                    uint8_t *a_dst = tiles + (size_t)s * kStageBytes, *b_dst = a_dst + kABytes;
+        // The whole warp runs the loop; lane 0 arms the barrier and loads the activation tile, lane 1
+        // loads the weight tile, so the two copies are issued in parallel.
+        if (lane == 0) { prefetch_tensormap(&tm_act); prefetch_tensormap(&tm_w); }
+        uint32_t it = 0;                         // k-blocks issued so far
+        int s = 0;                               // ring slot and its phase, advanced incrementally
+        uint32_t ph = 0;
+        bool ok = true;
+        for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            // 32-bit arithmetic: 64-bit divisions would cost about a microsecond per tile here
+            const uint32_t tt = (uint32_t)t, mt = tt / (uint32_t)n_tiles;
+            const uint32_t m0 = mt * kBM;
+            const int n0 = (int)(tt - mt * (uint32_t)n_tiles) * BN;
+            const uint32_t tq = m0 / (uint32_t)g.wo;
+            const int wo0 = (int)(m0 - tq * (uint32_t)g.wo);
+            const uint32_t img = tq / (uint32_t)g.ho;
+            const int ho0 = (int)(tq - img * (uint32_t)g.ho), img0 = (int)img;
+            const int base_w = g.lower_w + wo0 * g.stride_w, base_h = g.lower_h + ho0 * g.stride_h;
+            int r = 0, q = 0, cc = 0;
+            for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag));
+                if (!ok) break;
+                uint8_t *a_dst = tiles + (size_t)s * kStageBytes, *b_dst = a_dst + kABytes;
+                if (lane == 0) {
                     mbar_arrive_expect_tx(&ctl->full[s], kStageBytes);
                     tma_load_im2col_4d(a_dst, &tm_act, &ctl->full[s], cc * kBK, base_w, base_h, img0,
                                        (uint16_t)(q * g.dil_w), (uint16_t)(r * g.dil_h));
+                } else if (lane == 1) {
                     tma_load_2d(b_dst, &tm_w, &ctl->full[s], kb * kBK, n0);
-                    if (++cc == cchunks) { cc = 0; ++tap; }
-                    if (++s == stages) { s = 0; ph ^= 1u; }
                 }
+                if (++cc == cchunks) { cc = 0; if (++q == g.taps_w) { q = 0; ++r; } }
+                if (++s == stages) { s = 0; ph ^= 1u; }
             }
-            if (!ok) {
-                // Let the copies already issued land (bounded) before the CTA may exit.
-                const uint32_t first = it > (uint32_t)stages ? it - stages : 0;
-                for (uint32_t j = first; j < it; ++j)
-                    mbar_wait_bounded(&ctl->full[j % stages], (j / stages) & 1u, nullptr, 200000000ull);
-            }
+        }
+        if (!ok && lane == 0) {
+            atomicOr(err, ERRW_TIMEOUT);
+            ctl->abort_flag = 1;
+            // Let the copies already issued land (bounded) before the CTA may exit.
+            const uint32_t first = it > (uint32_t)stages ? it - stages : 0;
+            for (uint32_t j = first; j < it; ++j)
+                mbar_wait_bounded(&ctl->full[j % stages], (j / stages) & 1u, nullptr, 200000000ull);
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------

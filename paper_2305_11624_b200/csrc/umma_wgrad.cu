@@ -76,44 +76,46 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
     const uint32_t tmem_base = ctl->tmem_base;
 
     if (warp == 0) {
-        if (elect_one()) {
-            prefetch_tensormap(&tm_x);
-            prefetch_tensormap(&tm_dz);
-            const uint32_t tx_bytes = (uint32_t)(a_chunks + b_chunks) * kChunkBytes;
-            int issued = 0, s = 0;
-            uint32_t ph = 0;
-            for (int kb = 0; kb < num_kb; ++kb) {
-                if (!mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag)) {
-                    atomicOr(err, ERRW_TIMEOUT);
-                    ctl->abort_flag = 1;
-                    break;
-                }
-                // 32-bit arithmetic on purpose (64-bit divisions would dominate this thread's loop)
-                const uint32_t pp = (uint32_t)p0 + (uint32_t)kb * kWP;
-                const uint32_t t = pp / (uint32_t)g.wo;
-                const int wo0 = (int)(pp - t * (uint32_t)g.wo);
-                const uint32_t img = t / (uint32_t)g.ho;
-                const int ho0 = (int)(t - img * (uint32_t)g.ho), img0 = (int)img;
-                const int base_w = g.lower_w + wo0 * g.stride_w, base_h = g.lower_h + ho0 * g.stride_h;
-                uint8_t *a_dst = tiles + (size_t)s * kStageBytes, *b_dst = a_dst + kABytes;
-                mbar_arrive_expect_tx(&ctl->full[s], tx_bytes);
-                for (int j = 0; j < a_chunks; ++j) {
-                    const int kk = k0 + j * 64;                  // k = tap * c_in + ci
-                    const int tap = kk / g.c_in, ci0 = kk - tap * g.c_in;
-                    const int r = tap / g.taps_w, q = tap - r * g.taps_w;
-                    tma_load_im2col_4d(a_dst + j * kChunkBytes, &tm_x, &ctl->full[s], ci0, base_w, base_h, img0,
-                                       (uint16_t)(q * g.dil_w), (uint16_t)(r * g.dil_h));
-                }
-                for (int j = 0; j < b_chunks; ++j)
-                    tma_load_2d(b_dst + j * kChunkBytes, &tm_dz, &ctl->full[s], n0 + j * 64, (int)pp);
-                ++issued;
-                if (++s == stages) { s = 0; ph ^= 1u; }
-            }
-            if (ctl->abort_flag) {
-                const int first = issued > stages ? issued - stages : 0;
-                for (int kb = first; kb < issued; ++kb)
-                    mbar_wait_bounded(&ctl->full[kb % stages], (uint32_t)(kb / stages) & 1u, nullptr, 200000000ull);
-            }
+        // The whole warp runs the loop; lanes 0-1 load the two X slices, lanes 2.. the dZ boxes.
+        if (lane == 0) { prefetch_tensormap(&tm_x); prefetch_tensormap(&tm_dz); }
+        const uint32_t tx_bytes = (uint32_t)(a_chunks + b_chunks) * kChunkBytes;
+        // this lane's X slice: k = tap * c_in + ci is fixed for the whole CTA
+        const int kk = k0 + (lane & 1) * 64;
+        const int tap = kk / g.c_in, ci0 = kk - tap * g.c_in;
+        const int tr = tap / g.taps_w, tq = tap - tr * g.taps_w;
+        const uint16_t off_w = (uint16_t)(tq * g.dil_w), off_h = (uint16_t)(tr * g.dil_h);
+        int issued = 0, s = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        // pixel coordinates of the slice start, advanced by 64 pixels per stage without divisions
+        uint32_t pp = (uint32_t)p0;
+        uint32_t t0 = pp / (uint32_t)g.wo;
+        int wo0 = (int)(pp - t0 * (uint32_t)g.wo);
+        uint32_t img = t0 / (uint32_t)g.ho;
+        int ho0 = (int)(t0 - img * (uint32_t)g.ho);
+        for (int kb = 0; kb < num_kb; ++kb) {
+            ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag));
+            if (!ok) break;
+            const int base_w = g.lower_w + wo0 * g.stride_w, base_h = g.lower_h + ho0 * g.stride_h;
+            uint8_t *a_dst = tiles + (size_t)s * kStageBytes, *b_dst = a_dst + kABytes;
+            if (lane == 0) mbar_arrive_expect_tx(&ctl->full[s], tx_bytes);
+            if (lane < a_chunks)
+                tma_load_im2col_4d(a_dst + lane * kChunkBytes, &tm_x, &ctl->full[s], ci0, base_w, base_h, (int)img,
+                                   off_w, off_h);
+            else if (lane >= 2 && lane - 2 < b_chunks)
+                tma_load_2d(b_dst + (lane - 2) * kChunkBytes, &tm_dz, &ctl->full[s], n0 + (lane - 2) * 64, (int)pp);
+            ++issued;
+            if (++s == stages) { s = 0; ph ^= 1u; }
+            pp += kWP;
+            wo0 += kWP;
+            while (wo0 >= g.wo) { wo0 -= g.wo; if (++ho0 == g.ho) { ho0 = 0; ++img; } }
+        }
+        if (!ok && lane == 0) {
+            atomicOr(err, ERRW_TIMEOUT);
+            ctl->abort_flag = 1;
+            const int first = issued > stages ? issued - stages : 0;
+            for (int kb = first; kb < issued; ++kb)
+                mbar_wait_bounded(&ctl->full[kb % stages], (uint32_t)(kb / stages) & 1u, nullptr, 200000000ull);
         }
     } else if (warp == 1) {
         if (elect_one()) {
