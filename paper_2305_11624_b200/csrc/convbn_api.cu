@@ -113,7 +113,7 @@ struct Plan {
     size_t vec3 = 0;       // Eval forward: [s | beta - mean s | r]
     size_t dotpart = 0;    // [kt][C_out] fp32 (tensor-core weight-gradient path)
     int splits = 1, bsplits = 1;
-    bool umma_wgrad = false;
+    bool umma_wgrad = false, dw_wgrad = false;
     UmmaWgradPlan uw;
 };
 
@@ -128,6 +128,12 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
     pl.umma_wgrad = !force_direct() && d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC &&
                     umma_wgrad_eligible(pb);
     size_t part_bytes = wrows * pl.splits * sizeof(float), dot_bytes = 0;
+    pl.dw_wgrad = !force_direct() && d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && dw_eligible(pb) &&
+                  dw_wgrad_supported(pb);
+    if (pl.dw_wgrad) {
+        pl.splits = dw_wgrad_splits(pb);
+        part_bytes = wrows * pl.splits * sizeof(float);
+    }
     if (pl.umma_wgrad) {
         pl.uw = umma_wgrad_plan(pb);
         part_bytes = wrows * pl.uw.splits * sizeof(float);
@@ -210,6 +216,10 @@ int check_ws(const Plan &pl, const void *ws, size_t ws_bytes) {
 
 inline char *at(void *ws, size_t off) { return (char *)ws + off; }
 
+bool dw_path(const convbn_desc *d, const Problem &pb) {
+    return !force_direct() && d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && dw_eligible(pb);
+}
+
 // Tensor-core eligibility of the forward convolution and its GEMM shape.
 bool umma_fwd_shape(const convbn_desc *d, const Problem &pb, UmmaConvShape *s) {
     if (force_direct() || d->dtype != CONVBN_BF16 || d->layout != CONVBN_NHWC || pb.groups != 1) return false;
@@ -235,6 +245,9 @@ int run_conv_fwd(const convbn_desc *d, const Problem &pb, const void *x, const v
     if (umma_fwd_shape(d, pb, &s)) {
         LAUNCH("umma_fwd", launch_umma_conv(s, x, w, bias, z, st));
         *which = "umma";
+    } else if (dw_path(d, pb)) {
+        LAUNCH("dw_fwd", launch_dw_fwd(pb, x, w, bias, z, st));
+        *which = "depthwise";
     } else {
         LAUNCH("direct_fwd", launch_direct_fwd(pb, d->dtype, d->layout, x, w, bias, z, st));
         *which = "direct";
@@ -251,6 +264,14 @@ int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, cons
         LAUNCH("reparam_dgrad", launch_reparam_dgrad(pb, w, scale, w_scratch, st));
         LAUNCH("umma_dgrad", launch_umma_conv(s, dz, w_scratch, nullptr, dx, st));
         *which = "umma";
+    } else if (dw_path(d, pb)) {
+        const void *wd = w;
+        if (scale) {
+            LAUNCH("rescale_weight", launch_rescale_weight(pb, d->dtype, w, scale, w_scratch, st));
+            wd = w_scratch;
+        }
+        LAUNCH("dw_dgrad", launch_dw_dgrad(pb, dz, wd, dx, st));
+        *which = "depthwise";
     } else {
         const void *wd = w;
         if (scale) {
@@ -282,11 +303,14 @@ int run_param_grads(const convbn_desc *d, const Problem &pb, const Plan &pl, con
                                                        dgamma, dbeta, st));
         *which = "umma";
     } else {
-        LAUNCH("direct_wgrad", launch_direct_wgrad(pb, d->dtype, d->layout, dz, x, partials, pl.splits, st));
+        if (pl.dw_wgrad)
+            LAUNCH("dw_wgrad", launch_dw_wgrad(pb, dz, x, partials, pl.splits, st));
+        else
+            LAUNCH("direct_wgrad", launch_direct_wgrad(pb, d->dtype, d->layout, dz, x, partials, pl.splits, st));
         LAUNCH("wgrad_epilogue", launch_wgrad_epilogue(pb, d->dtype, partials, pl.splits, need_bsum ? bsum : nullptr,
                                                        need_bsum ? pl.bsplits : 0, w, vec3, b, mean, dw, db, dgamma,
                                                        dbeta, st));
-        *which = "direct";
+        *which = pl.dw_wgrad ? "depthwise" : "direct";
     }
     return CONVBN_OK;
 }

@@ -1,0 +1,313 @@
+// Depthwise ConvBN kernels (groups = C_in = C_out), bf16 NHWC, C a multiple of 8.
+// Depthwise convolution has about 4.5 FLOP per byte: it is a streaming problem, so these kernels use
+// the plain ALUs with 128-bit (8-channel) coalesced accesses along C and keep fp32 accumulators in
+// registers; neighbouring taps are served by L1.
+//   forward        Z[n,h,w,c]  = b'[c] + sum_{r,q} omega'[c,r,q] X[n, h s - p + r d, w s - p + q d, c]   (Sec. 3.1/3.3)
+//   backward data  dX = omega'_rot (*) dZ   (Sec. 3.2.1), gathered per dX element
+//   backward weight domega'[c,r,q] = sum_{n,h,w} dZ[n,h,w,c] X[n, ...]   (Sec. 3.2.1), per-slice partials
+#include "kernels.h"
+
+namespace convbn {
+
+namespace {
+
+constexpr int kMaxTaps = 49;   // up to 7 x 7
+
+struct DwShape {
+    int n, c, h_in, w_in, h_out, w_out, kh, kw, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w;
+};
+
+__device__ __forceinline__ void unpack8(const uint4 &q, float (&f)[8]) {
+    const uint32_t u[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        f[2 * e] = __uint_as_float(u[e] << 16);
+        f[2 * e + 1] = __uint_as_float(u[e] & 0xFFFF0000u);
+    }
+}
+
+__device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
+    uint4 q;
+    __nv_bfloat162 h;
+    h = __floats2bfloat162_rn(f[0], f[1]); q.x = *(uint32_t *)&h;
+    h = __floats2bfloat162_rn(f[2], f[3]); q.y = *(uint32_t *)&h;
+    h = __floats2bfloat162_rn(f[4], f[5]); q.z = *(uint32_t *)&h;
+    h = __floats2bfloat162_rn(f[6], f[7]); q.w = *(uint32_t *)&h;
+    return q;
+}
+
+// Stage the block's weights in shared memory as fp32 [tap][C] (global layout is [C][tap]).
+__device__ __forceinline__ void stage_weights(float *w_s, const __nv_bfloat16 *w, int taps, int c) {
+    for (int i = threadIdx.x; i < taps * c; i += blockDim.x) {
+        const int ch = i % c, t = i / c;
+        w_s[i] = __bfloat162float(w[(size_t)ch * taps + t]);
+    }
+    __syncthreads();
+}
+
+// One thread: 8 channels x TW consecutive output columns of one output row.  For unit stride and
+// dilation along W the TW + kw - 1 input vectors of a row are loaded once and reused by all taps.
+template <int TW, int KW>
+__global__ void __launch_bounds__(256) dw_fwd_kernel(DwShape s, const uint4 *__restrict__ x,
+                                                     const __nv_bfloat16 *__restrict__ w,
+                                                     const float *__restrict__ bias, uint4 *__restrict__ z) {
+    extern __shared__ float w_s[];                   // [taps][C]
+    const int v = s.c / 8;
+    stage_weights(w_s, w, s.kh * s.kw, s.c);
+    const uint32_t wgroups = (uint32_t)(s.w_out + TW - 1) / TW;
+    const uint32_t total = (uint32_t)s.n * s.h_out * wgroups * v;
+    for (uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        uint32_t t = idx / (uint32_t)v;
+        const int cv = (int)(idx - t * (uint32_t)v);
+        const uint32_t t1 = t / wgroups;
+        const int wg = (int)(t - t1 * wgroups);
+        const uint32_t n = t1 / (uint32_t)s.h_out;
+        const int ho = (int)(t1 - n * (uint32_t)s.h_out);
+        const int wo0 = wg * TW;
+        float acc[TW][8];
+#pragma unroll
+        for (int j = 0; j < TW; ++j)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[j][e] = bias ? bias[cv * 8 + e] : 0.f;
+        for (int r = 0; r < s.kh; ++r) {
+            const int hi = ho * s.stride_h - s.pad_h + r * s.dil_h;
+            if (hi < 0 || hi >= s.h_in) continue;
+            const uint4 *xrow = x + ((size_t)(n * s.h_in + hi) * s.w_in) * v + cv;
+            if (KW > 0) {
+                // unit stride / dilation along W, kw == KW: sliding window in registers
+                uint4 seg[TW + (KW > 0 ? KW : 1) - 1];
+                const int wi0 = wo0 - s.pad_w;
+#pragma unroll
+                for (int j = 0; j < TW + KW - 1; ++j) {
+                    const int wi = wi0 + j;
+                    seg[j] = (wi >= 0 && wi < s.w_in) ? __ldg(xrow + (size_t)wi * v) : make_uint4(0, 0, 0, 0);
+                }
+#pragma unroll
+                for (int q = 0; q < KW; ++q) {
+                    float wv[8];
+                    const float *wp = w_s + (r * KW + q) * s.c + cv * 8;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) wv[e] = wp[e];
+#pragma unroll
+                    for (int j = 0; j < TW; ++j) {
+                        float xv[8];
+                        unpack8(seg[j + q], xv);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc[j][e] = fmaf(xv[e], wv[e], acc[j][e]);
+                    }
+                }
+            } else {
+                for (int q = 0; q < s.kw; ++q) {
+                    float wv[8];
+                    const float *wp = w_s + (r * s.kw + q) * s.c + cv * 8;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) wv[e] = wp[e];
+#pragma unroll
+                    for (int j = 0; j < TW; ++j) {
+                        const int wi = (wo0 + j) * s.stride_w - s.pad_w + q * s.dil_w;
+                        if (wi >= 0 && wi < s.w_in && wo0 + j < s.w_out) {
+                            float xv[8];
+                            unpack8(__ldg(xrow + (size_t)wi * v), xv);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) acc[j][e] = fmaf(xv[e], wv[e], acc[j][e]);
+                        }
+                    }
+                }
+            }
+        }
+        uint4 *zrow = z + ((size_t)(n * s.h_out + ho) * s.w_out + wo0) * v + cv;
+#pragma unroll
+        for (int j = 0; j < TW; ++j)
+            if (wo0 + j < s.w_out) zrow[(size_t)j * v] = pack8(acc[j]);
+    }
+}
+
+// dX[n,h,w,c] = sum over taps with (h + p - r d) divisible by the stride of omega'[c,r,q] dZ[n,ho,wo,c].
+__global__ void __launch_bounds__(256) dw_dgrad_kernel(DwShape s, const uint4 *__restrict__ dz,
+                                                       const __nv_bfloat16 *__restrict__ w,
+                                                       uint4 *__restrict__ dx) {
+    extern __shared__ float w_s[];
+    const int v = s.c / 8;
+    stage_weights(w_s, w, s.kh * s.kw, s.c);
+    const uint32_t total = (uint32_t)s.n * s.h_in * s.w_in * v;
+    for (uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        uint32_t t = idx / (uint32_t)v;
+        const int cv = (int)(idx - t * (uint32_t)v);
+        const uint32_t t1 = t / (uint32_t)s.w_in;
+        const int wq = (int)(t - t1 * (uint32_t)s.w_in);
+        const uint32_t n = t1 / (uint32_t)s.h_in;
+        const int h = (int)(t1 - n * (uint32_t)s.h_in);
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int r = 0; r < s.kh; ++r) {
+            const int hs = h + s.pad_h - r * s.dil_h;
+            if (hs < 0 || hs % s.stride_h) continue;
+            const int ho = hs / s.stride_h;
+            if (ho >= s.h_out) continue;
+            for (int q = 0; q < s.kw; ++q) {
+                const int ws = wq + s.pad_w - q * s.dil_w;
+                if (ws < 0 || ws % s.stride_w) continue;
+                const int wo = ws / s.stride_w;
+                if (wo >= s.w_out) continue;
+                float dv[8];
+                unpack8(__ldg(dz + ((size_t)(n * s.h_out + ho) * s.w_out + wo) * v + cv), dv);
+                const float *wp = w_s + (r * s.kw + q) * s.c + cv * 8;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] = fmaf(dv[e], wp[e], acc[e]);
+            }
+        }
+        dx[idx] = pack8(acc);
+    }
+}
+
+// Per-slice partials of domega': block = (C/8 channel vectors) x (pixel lanes); every thread keeps
+// taps x 8 fp32 sums for its channels over the pixels it visits, then the pixel lanes are added in
+// lane order through shared memory.  part[split][c][tap].
+template <int TAPS>
+__global__ void __launch_bounds__(256) dw_wgrad_kernel(DwShape s, const uint4 *__restrict__ dz,
+                                                       const uint4 *__restrict__ x, float *__restrict__ part,
+                                                       uint32_t pix_per_block) {
+    extern __shared__ float red[];                   // [lanes][v][8]
+    const int v = s.c / 8, lanes = blockDim.x / v;
+    const int cv = threadIdx.x % v, pl = threadIdx.x / v;
+    const uint32_t p_total = (uint32_t)s.n * s.h_out * s.w_out;
+    const uint32_t p0 = blockIdx.x * pix_per_block;
+    const uint32_t p1 = p0 + pix_per_block < p_total ? p0 + pix_per_block : p_total;
+    float acc[TAPS][8];
+#pragma unroll
+    for (int t = 0; t < TAPS; ++t)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[t][e] = 0.f;
+    for (uint32_t p = p0 + pl; p < p1; p += lanes) {
+        const uint32_t t2 = p / (uint32_t)s.w_out;
+        const int wo = (int)(p - t2 * (uint32_t)s.w_out);
+        const uint32_t n = t2 / (uint32_t)s.h_out;
+        const int ho = (int)(t2 - n * (uint32_t)s.h_out);
+        float dv[8];
+        unpack8(__ldg(dz + (size_t)p * v + cv), dv);
+#pragma unroll
+        for (int t = 0; t < TAPS; ++t) {
+            const int r = t / s.kw, q = t - r * s.kw;
+            const int hi = ho * s.stride_h - s.pad_h + r * s.dil_h;
+            const int wi = wo * s.stride_w - s.pad_w + q * s.dil_w;
+            if (hi >= 0 && hi < s.h_in && wi >= 0 && wi < s.w_in) {
+                float xv[8];
+                unpack8(__ldg(x + ((size_t)(n * s.h_in + hi) * s.w_in + wi) * v + cv), xv);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[t][e] = fmaf(dv[e], xv[e], acc[t][e]);
+            }
+        }
+    }
+#pragma unroll
+    for (int t = 0; t < TAPS; ++t) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) red[((size_t)pl * v + cv) * 8 + e] = acc[t][e];
+        __syncthreads();
+        for (int i = threadIdx.x; i < s.c; i += blockDim.x) {
+            const int g = i / 8, e = i % 8;
+            float sum = 0.f;
+            for (int l = 0; l < lanes; ++l) sum += red[((size_t)l * v + g) * 8 + e];
+            part[((size_t)blockIdx.x * s.c + i) * TAPS + t] = sum;
+        }
+        __syncthreads();
+    }
+}
+
+DwShape dw_shape(const Problem &pb) {
+    return DwShape{pb.n, pb.c_in, pb.h_in, pb.w_in, pb.h_out, pb.w_out, pb.kh, pb.kw, pb.stride_h, pb.stride_w,
+                   pb.pad_h, pb.pad_w, pb.dil_h, pb.dil_w};
+}
+
+int dw_grid(long long total) {
+    long long b = (total + 255) / 256;
+    const long long cap = 148LL * 32;
+    return (int)(b < 1 ? 1 : (b > cap ? cap : b));
+}
+
+template <class K>
+cudaError_t set_smem_once(K kernel, bool *done) {
+    if (*done) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+    if (e == cudaSuccess) *done = true;
+    return e;
+}
+
+}  // namespace
+
+bool dw_eligible(const Problem &pb) {
+    return pb.groups == pb.c_in && pb.c_in == pb.c_out && pb.c_in % 8 == 0 && pb.c_in / 8 <= 256 &&
+           pb.kh * pb.kw <= kMaxTaps && (size_t)pb.kh * pb.kw * pb.c_in * sizeof(float) <= 96 * 1024 &&
+           pb.pin * pb.c_in < (1LL << 31) && pb.p * pb.c_out < (1LL << 31);
+}
+
+cudaError_t launch_dw_fwd(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
+                          cudaStream_t st) {
+    const DwShape s = dw_shape(pb);
+    const size_t smem = (size_t)pb.kh * pb.kw * pb.c_in * sizeof(float);
+    const long long total = (long long)pb.n * pb.h_out * ((pb.w_out + 3) / 4) * (pb.c_in / 8);
+    const bool unit_w = pb.stride_w == 1 && pb.dil_w == 1;
+    static bool a3 = false, a5 = false, a0 = false;
+    cudaError_t e;
+    if (unit_w && pb.kw == 3) {
+        if ((e = set_smem_once(dw_fwd_kernel<4, 3>, &a3)) != cudaSuccess) return e;
+        dw_fwd_kernel<4, 3><<<dw_grid(total), 256, smem, st>>>(s, (const uint4 *)x, (const __nv_bfloat16 *)w, bias,
+                                                                (uint4 *)z);
+    } else if (unit_w && pb.kw == 5) {
+        if ((e = set_smem_once(dw_fwd_kernel<4, 5>, &a5)) != cudaSuccess) return e;
+        dw_fwd_kernel<4, 5><<<dw_grid(total), 256, smem, st>>>(s, (const uint4 *)x, (const __nv_bfloat16 *)w, bias,
+                                                                (uint4 *)z);
+    } else {
+        if ((e = set_smem_once(dw_fwd_kernel<4, 0>, &a0)) != cudaSuccess) return e;
+        dw_fwd_kernel<4, 0><<<dw_grid(total), 256, smem, st>>>(s, (const uint4 *)x, (const __nv_bfloat16 *)w, bias,
+                                                                (uint4 *)z);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_dw_dgrad(const Problem &pb, const void *dz, const void *w, void *dx, cudaStream_t st) {
+    const DwShape s = dw_shape(pb);
+    const size_t smem = (size_t)pb.kh * pb.kw * pb.c_in * sizeof(float);
+    static bool attr = false;
+    cudaError_t e = set_smem_once(dw_dgrad_kernel, &attr);
+    if (e != cudaSuccess) return e;
+    const long long total = pb.pin * (pb.c_in / 8);
+    dw_dgrad_kernel<<<dw_grid(total), 256, smem, st>>>(s, (const uint4 *)dz, (const __nv_bfloat16 *)w, (uint4 *)dx);
+    return cudaGetLastError();
+}
+
+int dw_wgrad_splits(const Problem &pb) {
+    long long want = 148 * 8;
+    const long long cap = (pb.p + 63) / 64;
+    if (want > cap) want = cap;
+    if (want < 1) want = 1;
+    const long long per = (pb.p + want - 1) / want;
+    return (int)((pb.p + per - 1) / per);
+}
+
+template <int TAPS>
+static cudaError_t launch_dw_wgrad_t(const Problem &pb, const void *dz, const void *x, float *part, int splits,
+                                     cudaStream_t st) {
+    const DwShape s = dw_shape(pb);
+    const int v = pb.c_in / 8;
+    const int block = (256 / v) * v;
+    const size_t smem = (size_t)block * 8 * sizeof(float);
+    const long long per = (pb.p + splits - 1) / splits;
+    dw_wgrad_kernel<TAPS><<<splits, block, smem, st>>>(s, (const uint4 *)dz, (const uint4 *)x, part, (uint32_t)per);
+    return cudaGetLastError();
+}
+
+bool dw_wgrad_supported(const Problem &pb) {
+    const int t = pb.kh * pb.kw;
+    return t == 9 || t == 25 || t == 1;
+}
+
+cudaError_t launch_dw_wgrad(const Problem &pb, const void *dz, const void *x, float *part, int splits,
+                            cudaStream_t st) {
+    switch (pb.kh * pb.kw) {
+        case 1: return launch_dw_wgrad_t<1>(pb, dz, x, part, splits, st);
+        case 9: return launch_dw_wgrad_t<9>(pb, dz, x, part, splits, st);
+        case 25: return launch_dw_wgrad_t<25>(pb, dz, x, part, splits, st);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace convbn

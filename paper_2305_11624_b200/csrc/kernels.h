@@ -68,6 +68,17 @@ cudaError_t launch_param_finish(const Problem &pb, const UmmaWgradPlan &pl, cons
                                 const float *bsum_part, int bsplits, const float *vec3, const float *b,
                                 const float *mean, float *db, float *dgamma, float *dbeta, cudaStream_t st);
 
+// ---- depthwise (groups = C_in = C_out) bandwidth kernels, bf16 NHWC, C multiple of 8 -----------
+bool dw_eligible(const Problem &pb);
+bool dw_wgrad_supported(const Problem &pb);     // tap counts the register-tiled kernel is built for
+cudaError_t launch_dw_fwd(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
+                          cudaStream_t st);
+cudaError_t launch_dw_dgrad(const Problem &pb, const void *dz, const void *w, void *dx, cudaStream_t st);
+int dw_wgrad_splits(const Problem &pb);
+// part: [splits][C][taps] fp32 (the layout of the direct weight-gradient partials)
+cudaError_t launch_dw_wgrad(const Problem &pb, const void *dz, const void *x, float *part, int splits,
+                            cudaStream_t st);
+
 // ---- per-channel reductions (Appendix B: backward of a broadcast is a sum) -------------------
 int channel_sum_splits(const Problem &pb);
 // part: [splits][C_out] partial sums of t over pixel slices
