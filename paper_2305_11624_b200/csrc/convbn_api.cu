@@ -102,6 +102,10 @@ bool force_direct() {
     return v;
 }
 
+bool grouped_path(const convbn_desc *d, const Problem &pb) {
+    return !force_direct() && d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && grouped_bd_eligible(pb);
+}
+
 // Workspace carve-up of one phase.  Offsets are multiples of 256 bytes.
 struct Plan {
     size_t total = 0;
@@ -113,7 +117,8 @@ struct Plan {
     size_t vec3 = 0;       // Eval forward: [s | beta - mean s | r]
     size_t dotpart = 0;    // [kt][C_out] fp32 (tensor-core weight-gradient path)
     int splits = 1, bsplits = 1;
-    bool umma_wgrad = false, dw_wgrad = false;
+    size_t wbd = 0;        // block-diagonal expanded weights [C_out][taps][64], storage dtype
+    bool umma_wgrad = false, dw_wgrad = false, grouped_wgrad = false;
     UmmaWgradPlan uw;
 };
 
@@ -134,6 +139,13 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
         pl.splits = dw_wgrad_splits(pb);
         part_bytes = wrows * pl.splits * sizeof(float);
     }
+    const bool grouped = grouped_path(d, pb);
+    const size_t wbd_bytes = grouped ? (size_t)pb.c_out * pb.kh * pb.kw * 64 * elem_size(d->dtype) : 0;
+    pl.grouped_wgrad = grouped;
+    if (grouped) {
+        pl.uw = umma_wgrad_plan(pb);
+        part_bytes = (size_t)pl.uw.splits * (pb.c_out / 64) * pb.kh * pb.kw * 64 * 64 * sizeof(float);
+    }
     if (pl.umma_wgrad) {
         pl.uw = umma_wgrad_plan(pb);
         part_bytes = wrows * pl.uw.splits * sizeof(float);
@@ -143,9 +155,14 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
         case CONVBN_PHASE_TUNE_FWD:
         case CONVBN_PHASE_TUNE_BWD_DATA:
             pl.w_scaled = take(wbytes);
+            pl.wbd = take(wbd_bytes);
+            break;
+        case CONVBN_PHASE_DEPLOY_FWD:
+            pl.wbd = take(wbd_bytes);
             break;
         case CONVBN_PHASE_DEPLOY_BWD:
             pl.w_scaled = take(wbytes);
+            pl.wbd = take(wbd_bytes);
             pl.partials = take(part_bytes);
             pl.bsum = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
             pl.dotpart = take(dot_bytes);
@@ -157,10 +174,12 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
             break;
         case CONVBN_PHASE_EVAL_FWD:
             pl.vec3 = take(3 * (size_t)pb.c_out * sizeof(float));
+            pl.wbd = take(wbd_bytes);
             break;
         case CONVBN_PHASE_EVAL_BWD:
             pl.dy = take((size_t)pb.p * pb.c_out * elem_size(d->dtype));
             pl.w_scaled = take(wbytes);
+            pl.wbd = take(wbd_bytes);
             pl.part_g = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
             pl.bsum = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
             pl.partials = take(part_bytes);
@@ -240,9 +259,17 @@ bool umma_dgrad_shape(const convbn_desc *d, const Problem &pb, UmmaConvShape *s)
 
 // Forward convolution with whatever weights / bias the mode folded: tensor cores when eligible.
 int run_conv_fwd(const convbn_desc *d, const Problem &pb, const void *x, const void *w, const float *bias,
-                 void *z, cudaStream_t st, const char **which) {
+                 void *z, void *wbd_scratch, cudaStream_t st, const char **which) {
     UmmaConvShape s;
-    if (umma_fwd_shape(d, pb, &s)) {
+    if (grouped_path(d, pb)) {
+        // block-diagonal GEMM: expand the (already folded) weights, then the dense tensor-core kernel
+        s = UmmaConvShape{pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.c_out, pb.kh, pb.kw,
+                          -pb.pad_h, -pb.pad_w, pb.stride_h, pb.stride_w, pb.dil_h, pb.dil_w, 1};
+        if (!umma_conv_eligible(s)) return CONVBN_EUNSUPPORTED;
+        LAUNCH("expand_blockdiag", launch_expand_blockdiag(pb, w, nullptr, wbd_scratch, false, st));
+        LAUNCH("grouped_fwd", launch_umma_conv(s, x, wbd_scratch, bias, z, st));
+        *which = "grouped-umma";
+    } else if (umma_fwd_shape(d, pb, &s)) {
         LAUNCH("umma_fwd", launch_umma_conv(s, x, w, bias, z, st));
         *which = "umma";
     } else if (dw_path(d, pb)) {
@@ -258,19 +285,38 @@ int run_conv_fwd(const convbn_desc *d, const Problem &pb, const void *x, const v
 // Backward data.  `scale` (C_out floats or NULL) is folded into the weights on the way:
 // w_scratch receives omega' in the layout the chosen kernel wants.
 int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, const void *w, const float *scale,
-                   void *w_scratch, void *dx, cudaStream_t st, const char **which) {
+                   void *w_scratch, void *wbd_scratch, void *dx, cudaStream_t st, const char **which) {
     UmmaConvShape s;
-    if (umma_dgrad_shape(d, pb, &s)) {
+    if (grouped_path(d, pb) && pb.stride_h == 1 && pb.stride_w == 1) {
+        s = UmmaConvShape{pb.n, pb.h_out, pb.w_out, pb.c_out, pb.h_in, pb.w_in, pb.c_in, pb.kh, pb.kw,
+                          pb.pad_h - (pb.kh - 1) * pb.dil_h, pb.pad_w - (pb.kw - 1) * pb.dil_w, 1, 1, pb.dil_h,
+                          pb.dil_w, 1};
+        if (!umma_conv_eligible(s)) return CONVBN_EUNSUPPORTED;
+        LAUNCH("expand_blockdiag", launch_expand_blockdiag(pb, w, scale, wbd_scratch, true, st));
+        LAUNCH("grouped_dgrad", launch_umma_conv(s, dz, wbd_scratch, nullptr, dx, st));
+        *which = "grouped-umma";
+    } else if (umma_dgrad_shape(d, pb, &s)) {
         LAUNCH("reparam_dgrad", launch_reparam_dgrad(pb, w, scale, w_scratch, st));
         LAUNCH("umma_dgrad", launch_umma_conv(s, dz, w_scratch, nullptr, dx, st));
         *which = "umma";
     } else if (dw_path(d, pb)) {
-        const void *wd = w;
-        if (scale) {
-            LAUNCH("rescale_weight", launch_rescale_weight(pb, d->dtype, w, scale, w_scratch, st));
-            wd = w_scratch;
+        if (pb.stride_h == 1 && pb.stride_w == 1) {
+            // dX = omega'_rot (*) dZ is itself a stride-1 depthwise convolution of dZ with the rotated
+            // taps and padding (k-1) d - p: run the forward kernel on the mirrored problem.
+            LAUNCH("rescale_weight", launch_rescale_weight(pb, d->dtype, w, scale, w_scratch, st, true));
+            Problem mp = pb;
+            mp.h_in = pb.h_out; mp.w_in = pb.w_out; mp.h_out = pb.h_in; mp.w_out = pb.w_in;
+            mp.pad_h = (pb.kh - 1) * pb.dil_h - pb.pad_h; mp.pad_w = (pb.kw - 1) * pb.dil_w - pb.pad_w;
+            mp.p = pb.pin; mp.pin = pb.p;
+            LAUNCH("dw_dgrad", launch_dw_fwd(mp, dz, w_scratch, nullptr, dx, st));
+        } else {
+            const void *wd = w;
+            if (scale) {
+                LAUNCH("rescale_weight", launch_rescale_weight(pb, d->dtype, w, scale, w_scratch, st));
+                wd = w_scratch;
+            }
+            LAUNCH("dw_dgrad", launch_dw_dgrad(pb, dz, wd, dx, st));
         }
-        LAUNCH("dw_dgrad", launch_dw_dgrad(pb, dz, wd, dx, st));
         *which = "depthwise";
     } else {
         const void *wd = w;
@@ -294,7 +340,13 @@ int run_param_grads(const convbn_desc *d, const Problem &pb, const Plan &pl, con
     const bool need_bsum = vec3 || db;
     if (need_bsum)
         LAUNCH("channel_sum", launch_channel_sum_partial(pb, d->dtype, d->layout, dz, bsum, pl.bsplits, st));
-    if (pl.umma_wgrad) {
+    if (pl.grouped_wgrad) {
+        LAUNCH("grouped_wgrad", launch_umma_wgrad(pb, pl.uw, dz, x, partials, st));
+        LAUNCH("wgrad_epilogue_bd", launch_wgrad_epilogue_bd(pb, partials, pl.uw.splits, need_bsum ? bsum : nullptr,
+                                                             need_bsum ? pl.bsplits : 0, w, vec3, b, mean, dw, db,
+                                                             dgamma, dbeta, st));
+        *which = "grouped-umma";
+    } else if (pl.umma_wgrad) {
         float *dotpart = (float *)at(ws, pl.dotpart);
         LAUNCH("umma_wgrad", launch_umma_wgrad(pb, pl.uw, dz, x, partials, st));
         LAUNCH("wgrad_epilogue_t", launch_wgrad_epilogue_t(pb, pl.uw, partials, w, vec3, dw, dotpart, st));
@@ -364,7 +416,7 @@ int convbn_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const
     void *wf = at(workspace, pl.w_scaled);
     LAUNCH("reparam", launch_reparam(pb, desc->dtype, desc->layout, w, b, gamma, beta, run_mean, run_var, vec3, wf,
                       nullptr, st));
-    CK(run_conv_fwd(desc, pb, x, wf, vec3 + pb.c_out, z, st, &t_last_kernel[CONVBN_PHASE_TUNE_FWD]));
+    CK(run_conv_fwd(desc, pb, x, wf, vec3 + pb.c_out, z, at(workspace, pl.wbd), st, &t_last_kernel[CONVBN_PHASE_TUNE_FWD]));
     return CONVBN_OK;
 }
 
@@ -380,7 +432,7 @@ int convbn_tune_bwd_data(const convbn_desc *desc, const void *dz, const void *w,
     CK(check_ws(pl, workspace, workspace_bytes));
     cudaStream_t st = (cudaStream_t)stream;
     void *wf = at(workspace, pl.w_scaled);
-    CK(run_conv_dgrad(desc, pb, dz, w, (const float *)saved, wf, dx, st,
+    CK(run_conv_dgrad(desc, pb, dz, w, (const float *)saved, wf, at(workspace, pl.wbd), dx, st,
                       &t_last_kernel[CONVBN_PHASE_TUNE_BWD_DATA]));
     return CONVBN_OK;
 }
@@ -425,7 +477,7 @@ int convbn_eval_fwd(const convbn_desc *desc, const void *x, const void *w, const
     // BN acts on Y, which already holds the conv bias: shift = beta - mean s
     LAUNCH("reparam", launch_reparam(pb, desc->dtype, desc->layout, w, nullptr, gamma, beta, run_mean, run_var, vec3,
                       nullptr, nullptr, st));
-    CK(run_conv_fwd(desc, pb, x, w, b, y_saved, st, &t_last_kernel[CONVBN_PHASE_EVAL_FWD]));
+    CK(run_conv_fwd(desc, pb, x, w, b, y_saved, at(workspace, pl.wbd), st, &t_last_kernel[CONVBN_PHASE_EVAL_FWD]));
     LAUNCH("bn_eval_fwd", launch_bn_eval_fwd(pb, desc->dtype, desc->layout, y_saved, vec3, z, st));
     return CONVBN_OK;
 }
@@ -451,7 +503,7 @@ int convbn_eval_bwd(const convbn_desc *desc, const void *dz, const void *x, cons
     LAUNCH("bn_eval_bwd", launch_bn_eval_bwd(pb, desc->dtype, desc->layout, dz, y_saved, gamma, run_mean, run_var, dy, pg,
                           pbm, pl.bsplits, st));
     LAUNCH("bn_eval_finish", launch_bn_eval_finish(pb, pg, pbm, pl.bsplits, gamma, run_var, db, dgamma, dbeta, st));
-    CK(run_conv_dgrad(desc, pb, dy, w, nullptr, at(workspace, pl.w_scaled), dx, st,
+    CK(run_conv_dgrad(desc, pb, dy, w, nullptr, at(workspace, pl.w_scaled), at(workspace, pl.wbd), dx, st,
                       &t_last_kernel[CONVBN_PHASE_EVAL_BWD]));
     const char *unused = nullptr;
     CK(run_param_grads(desc, pb, pl, dy, x, w, nullptr, nullptr, nullptr, dw, nullptr, nullptr, nullptr, workspace,
@@ -487,7 +539,7 @@ int convbn_deploy_fwd(const convbn_desc *desc, const void *x, const void *w_fuse
     const Plan pl = make_plan(desc, pb, CONVBN_PHASE_DEPLOY_FWD);
     CK(check_ws(pl, workspace, workspace_bytes));
     cudaStream_t st = (cudaStream_t)stream;
-    CK(run_conv_fwd(desc, pb, x, w_fused, b_fused, z, st, &t_last_kernel[CONVBN_PHASE_DEPLOY_FWD]));
+    CK(run_conv_fwd(desc, pb, x, w_fused, b_fused, z, at(workspace, pl.wbd), st, &t_last_kernel[CONVBN_PHASE_DEPLOY_FWD]));
     return CONVBN_OK;
 }
 
@@ -504,7 +556,7 @@ int convbn_deploy_bwd(const convbn_desc *desc, const void *dz, const void *x, co
     const Plan pl = make_plan(desc, pb, CONVBN_PHASE_DEPLOY_BWD);
     CK(check_ws(pl, workspace, workspace_bytes));
     cudaStream_t st = (cudaStream_t)stream;
-    CK(run_conv_dgrad(desc, pb, dz, w_fused, nullptr, at(workspace, pl.w_scaled), dx, st,
+    CK(run_conv_dgrad(desc, pb, dz, w_fused, nullptr, at(workspace, pl.w_scaled), at(workspace, pl.wbd), dx, st,
                       &t_last_kernel[CONVBN_PHASE_DEPLOY_BWD]));
     const char *unused = nullptr;
     CK(run_param_grads(desc, pb, pl, dz, x, w_fused, nullptr, nullptr, nullptr, dw_fused, db_fused, nullptr, nullptr,

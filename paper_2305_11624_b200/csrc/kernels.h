@@ -16,9 +16,10 @@ cudaError_t launch_reparam(const Problem &pb, int dtype, int layout, const void 
                            const float *var, float *vec3, void *w_scaled, float *b_fused,
                            cudaStream_t st);
 
-// omega' = s omega re-formed from the saved scale vector (first C_out floats of vec3).
+// omega' = s omega re-formed from the saved scale vector (first C_out floats of vec3; NULL = 1).
+// reverse_row writes each weight row back to front (the 180-degree tap rotation when C_in/G = 1).
 cudaError_t launch_rescale_weight(const Problem &pb, int dtype, const void *w, const float *vec3,
-                                  void *w_scaled, cudaStream_t st);
+                                  void *w_scaled, cudaStream_t st, bool reverse_row = false);
 
 // ---- direct (one thread per output element) convolution kernels, any shape -----------------
 cudaError_t launch_direct_fwd(const Problem &pb, int dtype, int layout, const void *x,
@@ -38,6 +39,9 @@ struct UmmaConvShape {
     int n, ha, wa, ca;       // activation tensor [n][ha][wa][ca]
     int ho, wo, cn;          // output tensor [n][ho][wo][cn]
     int taps_h, taps_w, lower_h, lower_w, stride_h, stride_w, dil_h, dil_w;
+    // 1: grouped convolution run as a block-diagonal GEMM: output channels [64 b, 64 b + 64) read only
+    // activation channels [64 b, 64 b + 64) and wmat is [cn][taps * 64] (zeros outside a channel's group).
+    int blockdiag = 0;
 };
 bool umma_conv_eligible(const UmmaConvShape &s);
 cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void *wmat, const float *bias,
@@ -78,6 +82,21 @@ int dw_wgrad_splits(const Problem &pb);
 // part: [splits][C][taps] fp32 (the layout of the direct weight-gradient partials)
 cudaError_t launch_dw_wgrad(const Problem &pb, const void *dz, const void *x, float *part, int splits,
                             cudaStream_t st);
+
+// ---- grouped convolution on the tensor cores as a block-diagonal GEMM ----------------------------
+// For C_in/G = C_out/G = cg dividing 64 and C a multiple of 64, every 64-channel block is a dense
+// 64 -> 64 convolution whose weight matrix is zero outside the cg x cg diagonal blocks.
+bool grouped_bd_eligible(const Problem &pb);
+// wbd[co][tap][64]: omega (scaled by s_vec[co] if given) placed at its group's columns, zeros elsewhere.
+// transpose_flip = true builds the backward-data operand instead: wbd[ci][taps-1-tap][64 output channels].
+cudaError_t launch_expand_blockdiag(const Problem &pb, const void *w, const float *s_vec, void *wbd,
+                                    bool transpose_flip, cudaStream_t st);
+// Parameter-gradient epilogue over block-diagonal partials part[split][block][tap * 64 + ci][64 co]:
+// same outputs as launch_wgrad_epilogue.
+cudaError_t launch_wgrad_epilogue_bd(const Problem &pb, const float *partials, int splits,
+                                     const float *bsum_part, int bsplits, const void *w, const float *vec3,
+                                     const float *b, const float *mean, float *dw, float *db, float *dgamma,
+                                     float *dbeta, cudaStream_t st);
 
 // ---- per-channel reductions (Appendix B: backward of a broadcast is a sum) -------------------
 int channel_sum_splits(const Problem &pb);

@@ -73,21 +73,22 @@ cudaError_t launch_reparam(const Problem &pb, int dtype, int layout, const void 
 template <class T>
 __global__ void __launch_bounds__(256) rescale_weight_kernel(int kdim, const T *__restrict__ w,
                                                              const float *__restrict__ s_vec,
-                                                             T *__restrict__ w_scaled) {
+                                                             T *__restrict__ w_scaled, int reverse_row) {
     const int co = blockIdx.y;
-    const float s = s_vec[co];
+    const float s = s_vec ? s_vec[co] : 1.f;
     const long long base = (long long)co * kdim;
     for (int k = blockIdx.x * blockDim.x + threadIdx.x; k < kdim; k += gridDim.x * blockDim.x)
-        w_scaled[base + k] = from_f32<T>(s * to_f32(w[base + k]));
+        w_scaled[base + (reverse_row ? kdim - 1 - k : k)] = from_f32<T>(s * to_f32(w[base + k]));
 }
 
 cudaError_t launch_rescale_weight(const Problem &pb, int dtype, const void *w, const float *vec3,
-                                  void *w_scaled, cudaStream_t st) {
+                                  void *w_scaled, cudaStream_t st, bool reverse_row) {
     return by_type(dtype, [&](auto *tp) {
         using T = typename std::remove_pointer<decltype(tp)>::type;
         int gx = (pb.kdim + 255) / 256;
         if (gx > 8) gx = 8;
-        rescale_weight_kernel<T><<<dim3(gx, pb.c_out), 256, 0, st>>>(pb.kdim, (const T *)w, vec3, (T *)w_scaled);
+        rescale_weight_kernel<T><<<dim3(gx, pb.c_out), 256, 0, st>>>(pb.kdim, (const T *)w, vec3, (T *)w_scaled,
+                                                                     reverse_row ? 1 : 0);
         return cudaGetLastError();
     });
 }

@@ -36,6 +36,7 @@ struct ConvGemm {
     int stride_h, stride_w, dil_h, dil_w;
     long long p;             // output pixels n * ho * wo
     int stages;
+    int blockdiag;           // grouped conv as block-diagonal GEMM: tile n0 reads channels [n0, n0 + 64) only
 };
 
 struct ConvSmemCtl {
@@ -65,7 +66,7 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
     float *bias_s = (float *)(((uintptr_t)(ctl + 1) + 15) & ~(uintptr_t)15);   // cn floats
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int stages = g.stages;
-    const int cchunks = g.ca / kBK;
+    const int cchunks = g.blockdiag ? 1 : g.ca / kBK;
     const int num_kb = g.taps_h * g.taps_w * cchunks;
     const int n_tiles = (g.cn + BN - 1) / BN;
     const long long total_tiles = ((g.p + kBM - 1) / kBM) * n_tiles;
@@ -114,7 +115,7 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                 uint8_t *a_dst = tiles + (size_t)s * kStageBytes, *b_dst = a_dst + kABytes;
                 if (lane == 0) {
                     mbar_arrive_expect_tx(&ctl->full[s], kStageBytes);
-                    tma_load_im2col_4d(a_dst, &tm_act, &ctl->full[s], cc * kBK, base_w, base_h, img0,
+                    tma_load_im2col_4d(a_dst, &tm_act, &ctl->full[s], (g.blockdiag ? n0 : 0) + cc * kBK, base_w, base_h, img0,
                                        (uint16_t)(q * g.dil_w), (uint16_t)(r * g.dil_h));
                 } else if (lane == 1) {
                     tma_load_2d(b_dst, &tm_w, &ctl->full[s], kb * kBK, n0);
@@ -303,6 +304,7 @@ bool make_tmap_im2col_bf16(CUtensorMap *tm, const void *base, int n, int h, int 
 
 bool umma_conv_eligible(const UmmaConvShape &s) {
     if (s.ca % kBK || s.cn % 8 || s.cn < 64 || s.cn > 4096) return false;
+    if (s.blockdiag && (s.ca != s.cn)) return false;
     if (s.lower_h < -128 || s.lower_h > 127 || s.lower_w < -128 || s.lower_w > 127) return false;
     if ((s.taps_h - 1) * s.dil_h > 255 || (s.taps_w - 1) * s.dil_w > 255) return false;
     if (s.stride_h > 8 || s.stride_w > 8) return false;
@@ -369,17 +371,18 @@ cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void
     g.ho = s.ho; g.wo = s.wo; g.cn = s.cn; g.ca = s.ca; g.taps_h = s.taps_h; g.taps_w = s.taps_w;
     g.lower_h = s.lower_h; g.lower_w = s.lower_w; g.stride_h = s.stride_h; g.stride_w = s.stride_w;
     g.dil_h = s.dil_h; g.dil_w = s.dil_w; g.p = (long long)s.n * s.ho * s.wo; g.stages = 1;
+    g.blockdiag = s.blockdiag;
     // The bounding box of base pixels has ho x wo positions: upper = lower + (out-1) stride - (in-1).
     const int upper_h = s.lower_h + (s.ho - 1) * s.stride_h - (s.ha - 1);
     const int upper_w = s.lower_w + (s.wo - 1) * s.stride_w - (s.wa - 1);
     const long long tiles_m = (g.p + kBM - 1) / kBM;
-    const int bn = pick_bn(tiles_m, s.cn);
+    const int bn = s.blockdiag ? 64 : pick_bn(tiles_m, s.cn);
     CUtensorMap ta, tw, tout;
     if (!make_tmap_matrix_bf16(&tout, out, g.p, s.cn, 32, 64)) return cudaErrorInvalidValue;
     if (!make_tmap_im2col_bf16(&ta, act, s.n, s.ha, s.wa, s.ca, s.lower_h, s.lower_w, upper_h, upper_w, s.stride_h,
                                s.stride_w, kBM, kBK))
         return cudaErrorInvalidValue;
-    if (!make_tmap_matrix_bf16(&tw, wmat, s.cn, (long long)s.taps_h * s.taps_w * s.ca, bn, kBK))
+    if (!make_tmap_matrix_bf16(&tw, wmat, s.cn, (long long)s.taps_h * s.taps_w * (s.blockdiag ? 64 : s.ca), bn, kBK))
         return cudaErrorInvalidValue;
     int *err = nullptr;
     cudaError_t e = error_word_address(&err);

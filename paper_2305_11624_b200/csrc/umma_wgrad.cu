@@ -29,6 +29,7 @@ struct WgradGemm {
     long long p;            // output pixels
     long long per_split;    // pixels per slice (multiple of 64)
     int stages;
+    int blockdiag;          // grouped conv: c_in = 64 here, k rows are (tap, channel of block blockIdx.y)
 };
 
 struct WgradSmemCtl {
@@ -81,7 +82,7 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
         const uint32_t tx_bytes = (uint32_t)(a_chunks + b_chunks) * kChunkBytes;
         // this lane's X slice: k = tap * c_in + ci is fixed for the whole CTA
         const int kk = k0 + (lane & 1) * 64;
-        const int tap = kk / g.c_in, ci0 = kk - tap * g.c_in;
+        const int tap = kk / g.c_in, ci0 = kk - tap * g.c_in + (g.blockdiag ? n0 : 0);
         const int tr = tap / g.taps_w, tq = tap - tr * g.taps_w;
         const uint16_t off_w = (uint16_t)(tq * g.dil_w), off_h = (uint16_t)(tr * g.dil_h);
         int issued = 0, s = 0;
@@ -152,7 +153,9 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
             tc_fence_after_sync();
             const int k = k0 + quarter * 32 + lane;
             const bool row_ok = k < g.kdim;
-            float *orow = partials + ((size_t)blockIdx.z * g.kdim + (row_ok ? k : 0)) * g.c_out + n0;
+            float *orow = g.blockdiag
+                              ? partials + (((size_t)blockIdx.z * gridDim.y + blockIdx.y) * g.kdim + (row_ok ? k : 0)) * 64
+                              : partials + ((size_t)blockIdx.z * g.kdim + (row_ok ? k : 0)) * g.c_out + n0;
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 if (n0 + c0 >= g.c_out) break;
@@ -172,6 +175,15 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
     if (warp == 1) tmem_dealloc(tmem_base, BN);
 }
 
+bool grouped_bd_eligible(const Problem &pb) {
+    if (pb.groups <= 1 || pb.cg != pb.cog || pb.cg < 2 || 64 % pb.cg || pb.c_in % 64) return false;
+    if (pb.pad_h > 128 || pb.pad_w > 128) return false;
+    if ((pb.kh - 1) * pb.dil_h > 255 || (pb.kw - 1) * pb.dil_w > 255) return false;
+    if (pb.stride_h > 8 || pb.stride_w > 8) return false;
+    if (pb.p >= (1LL << 31) - 256 || pb.pin >= (1LL << 31) - 256) return false;
+    return true;
+}
+
 bool umma_wgrad_eligible(const Problem &pb) {
     if (pb.groups != 1 || pb.c_in % 64 || pb.c_out % 64) return false;
     if (pb.pad_h > 128 || pb.pad_w > 128) return false;
@@ -185,8 +197,10 @@ static int wgrad_bn(const Problem &pb) { return pb.c_out >= 256 ? 256 : (pb.c_ou
 
 UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
     UmmaWgradPlan pl;
-    const int bn = wgrad_bn(pb);
-    const long long m_tiles = (pb.kdim + kWM - 1) / kWM, n_tiles = (pb.c_out + bn - 1) / bn;
+    const bool bd = pb.groups > 1;
+    const int bn = bd ? 64 : wgrad_bn(pb);
+    const long long kd = bd ? (long long)pb.kh * pb.kw * 64 : pb.kdim;
+    const long long m_tiles = (kd + kWM - 1) / kWM, n_tiles = (pb.c_out + bn - 1) / bn;
     const long long target = 148;
     long long splits = (target + m_tiles * n_tiles - 1) / (m_tiles * n_tiles);
     const long long max_splits = (pb.p + 4 * kWP - 1) / (4 * kWP);     // at least 256 pixels per slice
@@ -218,7 +232,7 @@ static cudaError_t launch_w(const CUtensorMap &tx, const CUtensorMap &tdz, Wgrad
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    dim3 grid((unsigned)((pb.kdim + kWM - 1) / kWM), (unsigned)((pb.c_out + BN - 1) / BN), (unsigned)pl.splits);
+    dim3 grid((unsigned)((g.kdim + kWM - 1) / kWM), (unsigned)((pb.c_out + BN - 1) / BN), (unsigned)pl.splits);
     umma_wgrad_kernel<BN><<<grid, kWThreads, smem, st>>>(tx, tdz, g, partials, err);
     return cudaGetLastError();
 }
@@ -229,6 +243,8 @@ cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
     g.ho = pb.h_out; g.wo = pb.w_out; g.c_in = pb.c_in; g.c_out = pb.c_out; g.taps_w = pb.kw;
     g.lower_h = -pb.pad_h; g.lower_w = -pb.pad_w; g.stride_h = pb.stride_h; g.stride_w = pb.stride_w;
     g.dil_h = pb.dil_h; g.dil_w = pb.dil_w; g.kdim = pb.kdim; g.p = pb.p; g.per_split = pl.per_split; g.stages = 1;
+    g.blockdiag = pb.groups > 1 ? 1 : 0;
+    if (g.blockdiag) { g.c_in = 64; g.kdim = pb.kh * pb.kw * 64; }
     const int upper_h = g.lower_h + (pb.h_out - 1) * pb.stride_h - (pb.h_in - 1);
     const int upper_w = g.lower_w + (pb.w_out - 1) * pb.stride_w - (pb.w_in - 1);
     CUtensorMap tx, tdz;
@@ -239,7 +255,7 @@ cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
     int *err = nullptr;
     cudaError_t e = error_word_address(&err);
     if (e != cudaSuccess) return e;
-    const int bn = wgrad_bn(pb);
+    const int bn = g.blockdiag ? 64 : wgrad_bn(pb);
     if (bn == 64) return launch_w<64>(tx, tdz, g, pl, pb, partials, err, st);
     if (bn == 128) return launch_w<128>(tx, tdz, g, pl, pb, partials, err, st);
     return launch_w<256>(tx, tdz, g, pl, pb, partials, err, st);
