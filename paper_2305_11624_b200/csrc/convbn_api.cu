@@ -257,6 +257,27 @@ bool umma_dgrad_shape(const convbn_desc *d, const Problem &pb, UmmaConvShape *s)
     return umma_conv_eligible(*s);
 }
 
+// Taps of one residue class of a strided backward-data pass (unit dilation): r = r_max - stride m for
+// m = 0 .. count-1, read at output offset off_min + m relative to the class coordinate.
+struct ClassTaps { int count, r_max, off_min; };
+ClassTaps class_taps(int a, int pad, int k, int stride) {
+    ClassTaps c{0, 0, 0};
+    const int r0 = (a + pad) % stride;                 // smallest tap with (a + pad - r) divisible by stride
+    if (r0 >= k) return c;
+    c.count = (k - 1 - r0) / stride + 1;
+    c.r_max = r0 + (c.count - 1) * stride;
+    c.off_min = (a + pad - c.r_max) / stride;          // exact, may be negative
+    return c;
+}
+
+bool strided_dgrad_ok(const convbn_desc *d, const Problem &pb) {
+    if (force_direct() || d->dtype != CONVBN_BF16 || d->layout != CONVBN_NHWC || pb.groups != 1) return false;
+    if (pb.stride_h == 1 && pb.stride_w == 1) return false;
+    if (pb.dil_h != 1 || pb.dil_w != 1 || pb.stride_h > 4 || pb.stride_w > 4) return false;
+    return pb.c_out % 64 == 0 && pb.c_in % 8 == 0 && pb.c_in >= 64 && pb.c_in <= 4096 &&
+           pb.pin < (1LL << 31) - 256;
+}
+
 // Forward convolution with whatever weights / bias the mode folded: tensor cores when eligible.
 int run_conv_fwd(const convbn_desc *d, const Problem &pb, const void *x, const void *w, const float *bias,
                  void *z, void *wbd_scratch, cudaStream_t st, const char **which) {
@@ -295,6 +316,39 @@ int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, cons
         LAUNCH("expand_blockdiag", launch_expand_blockdiag(pb, w, scale, wbd_scratch, true, st));
         LAUNCH("grouped_dgrad", launch_umma_conv(s, dz, wbd_scratch, nullptr, dx, st));
         *which = "grouped-umma";
+    } else if (strided_dgrad_ok(d, pb)) {
+        // Strided backward data, one stride-1 GEMM per residue class (a, b) of the input position:
+        // rows h = stride_h i + a only meet taps r with (a + pad_h - r) divisible by stride_h, at output
+        // row i + (a + pad_h - r) / stride_h; no multiplication by inserted zeros.
+        bool any_empty = false;
+        for (int a = 0; a < pb.stride_h && !any_empty; ++a) any_empty = class_taps(a, pb.pad_h, pb.kh, pb.stride_h).count == 0;
+        for (int b2 = 0; b2 < pb.stride_w && !any_empty; ++b2) any_empty = class_taps(b2, pb.pad_w, pb.kw, pb.stride_w).count == 0;
+        if (any_empty &&
+            cudaMemsetAsync(dx, 0, (size_t)pb.pin * pb.c_in * elem_size(d->dtype), st) != cudaSuccess)
+            return CONVBN_ECUDA;
+        size_t woff = 0;
+        for (int a = 0; a < pb.stride_h && a < pb.h_in; ++a)
+            for (int b2 = 0; b2 < pb.stride_w && b2 < pb.w_in; ++b2) {
+                const ClassTaps ch = class_taps(a, pb.pad_h, pb.kh, pb.stride_h);
+                const ClassTaps cw = class_taps(b2, pb.pad_w, pb.kw, pb.stride_w);
+                if (ch.count == 0 || cw.count == 0) continue;
+                char *wc = (char *)w_scratch + woff;
+                woff += (size_t)ch.count * cw.count * pb.c_in * pb.c_out * elem_size(d->dtype);
+                UmmaConvShape cs{pb.n, pb.h_out, pb.w_out, pb.c_out,
+                                 (pb.h_in - a + pb.stride_h - 1) / pb.stride_h,
+                                 (pb.w_in - b2 + pb.stride_w - 1) / pb.stride_w, pb.c_in, ch.count, cw.count,
+                                 ch.off_min, cw.off_min, 1, 1, 1, 1, 0};
+                cs.out_sn = (long long)pb.h_in * pb.w_in * pb.c_in;
+                cs.out_sh = pb.stride_h * pb.w_in * pb.c_in;
+                cs.out_sw = pb.stride_w * pb.c_in;
+                if (!umma_conv_eligible(cs)) return CONVBN_EUNSUPPORTED;
+                LAUNCH("reparam_dgrad", launch_reparam_dgrad_class(pb, w, scale, wc, ch.count, cw.count, ch.r_max,
+                                                                   cw.r_max, pb.stride_h, pb.stride_w, st));
+                LAUNCH("umma_dgrad", launch_umma_conv(cs, dz, wc, nullptr,
+                                                      (char *)dx + ((size_t)a * pb.w_in + b2) * pb.c_in *
+                                                                       elem_size(d->dtype), st));
+            }
+        *which = "umma-strided";
     } else if (umma_dgrad_shape(d, pb, &s)) {
         LAUNCH("reparam_dgrad", launch_reparam_dgrad(pb, w, scale, w_scratch, st));
         LAUNCH("umma_dgrad", launch_umma_conv(s, dz, w_scratch, nullptr, dx, st));

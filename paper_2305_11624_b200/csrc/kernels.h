@@ -42,6 +42,10 @@ struct UmmaConvShape {
     // 1: grouped convolution run as a block-diagonal GEMM: output channels [64 b, 64 b + 64) read only
     // activation channels [64 b, 64 b + 64) and wmat is [cn][taps * 64] (zeros outside a channel's group).
     int blockdiag = 0;
+    // Strided output, used when out_sw != 0 (no bias in this mode): output pixel (n, i, j) is written at
+    // out + n out_sn + i out_sh + j out_sw (elements) instead of densely.
+    long long out_sn = 0;
+    int out_sh = 0, out_sw = 0;
 };
 bool umma_conv_eligible(const UmmaConvShape &s);
 cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void *wmat, const float *bias,
@@ -50,6 +54,10 @@ cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void
 // (s_vec == NULL: unscaled).  bf16, groups = 1.
 cudaError_t launch_reparam_dgrad(const Problem &pb, const void *w, const float *s_vec, void *w_t,
                                  cudaStream_t st);
+// One parity class of a strided backward-data pass: w_t[ci][mh][mw][co] = s[co] w[co][r][q][ci] with
+// r = r_max - step_h mh, q = q_max - step_w mw for mh < th, mw < tw.
+cudaError_t launch_reparam_dgrad_class(const Problem &pb, const void *w, const float *s_vec, void *w_t, int th,
+                                       int tw, int r_max, int q_max, int step_h, int step_w, cudaStream_t st);
 
 // ---- tensor-core weight gradient (bf16 NHWC, groups = 1, channels multiples of 64) ---------------
 struct UmmaWgradPlan {

@@ -115,6 +115,38 @@ __global__ void __launch_bounds__(256) reparam_dgrad_kernel(int c_out, int c_in,
     }
 }
 
+__global__ void __launch_bounds__(256) reparam_dgrad_class_kernel(int c_out, int c_in, int kw, int tw, int r_max,
+                                                                  int q_max, int step_h, int step_w, int ctaps,
+                                                                  const __nv_bfloat16 *__restrict__ w,
+                                                                  const float *__restrict__ s_vec,
+                                                                  __nv_bfloat16 *__restrict__ w_t, int taps) {
+    __shared__ float tile[32][33];
+    const int ct = blockIdx.z, mh = ct / tw, mw = ct - mh * tw;
+    const int tap = (r_max - step_h * mh) * kw + (q_max - step_w * mw);
+    const int co0 = blockIdx.y * 32, ci0 = blockIdx.x * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int j = ty; j < 32; j += 8) {
+        const int co = co0 + j, ci = ci0 + tx;
+        if (co < c_out && ci < c_in)
+            tile[j][tx] = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((long long)co * taps + tap) * c_in + ci]);
+    }
+    __syncthreads();
+    for (int j = ty; j < 32; j += 8) {
+        const int ci = ci0 + j, co = co0 + tx;
+        if (co < c_out && ci < c_in)
+            w_t[((long long)ci * ctaps + ct) * c_out + co] = __float2bfloat16_rn(tile[tx][j]);
+    }
+}
+
+cudaError_t launch_reparam_dgrad_class(const Problem &pb, const void *w, const float *s_vec, void *w_t, int th,
+                                       int tw, int r_max, int q_max, int step_h, int step_w, cudaStream_t st) {
+    dim3 grid((pb.c_in + 31) / 32, (pb.c_out + 31) / 32, th * tw);
+    reparam_dgrad_class_kernel<<<grid, 256, 0, st>>>(pb.c_out, pb.c_in, pb.kw, tw, r_max, q_max, step_h, step_w,
+                                                     th * tw, (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t,
+                                                     pb.kh * pb.kw);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_reparam_dgrad(const Problem &pb, const void *w, const float *s_vec, void *w_t,
                                  cudaStream_t st) {
     dim3 grid((pb.c_in + 31) / 32, (pb.c_out + 31) / 32, pb.kh * pb.kw);

@@ -37,6 +37,11 @@ struct ConvGemm {
     long long p;             // output pixels n * ho * wo
     int stages;
     int blockdiag;           // grouped conv as block-diagonal GEMM: tile n0 reads channels [n0, n0 + 64) only
+    // Strided output (one parity class of a strided backward-data pass): pixel (img, i, j) of the
+    // class goes to out_strided + img out_sn + i out_sh + j out_sw (elements).  NULL: dense TMA stores.
+    __nv_bfloat16 *out_strided;
+    long long out_sn;
+    int out_sh, out_sw;
 };
 
 struct ConvSmemCtl {
@@ -185,6 +190,15 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
             const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
             int ncols = g.cn - n0;                          // valid columns of this tile
             if (ncols > BN) ncols = BN;
+            __nv_bfloat16 *srow = nullptr;                  // strided mode: this thread's output pixel
+            if (g.out_strided) {
+                const uint32_t m = m0 + quarter * 32 + lane;
+                if ((long long)m < g.p) {
+                    const uint32_t tq = m / (uint32_t)g.wo, img = tq / (uint32_t)g.ho;
+                    srow = g.out_strided + (size_t)img * g.out_sn + (size_t)(tq - img * (uint32_t)g.ho) * g.out_sh +
+                           (size_t)(m - tq * (uint32_t)g.wo) * g.out_sw + n0;
+                }
+            }
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 64) {
                 uint32_t v[64];
@@ -199,7 +213,22 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&ctl->tmem_empty[acc]);
                 }
-                if (c0 < ncols) {
+                if (c0 < ncols && g.out_strided) {
+                    if (srow) {
+#pragma unroll
+                        for (int j = 0; j < 64; j += 8) {
+                            if (c0 + j < ncols) {
+                                uint4 pk;
+                                __nv_bfloat162 h;
+                                h = __floats2bfloat162_rn(__uint_as_float(v[j]), __uint_as_float(v[j + 1])); pk.x = *(uint32_t *)&h;
+                                h = __floats2bfloat162_rn(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])); pk.y = *(uint32_t *)&h;
+                                h = __floats2bfloat162_rn(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5])); pk.z = *(uint32_t *)&h;
+                                h = __floats2bfloat162_rn(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7])); pk.w = *(uint32_t *)&h;
+                                *(uint4 *)(srow + c0 + j) = pk;
+                            }
+                        }
+                    }
+                } else if (c0 < ncols) {
                     uint8_t *buf = stage_buf + (size_t)sbuf * kStagingWarpBytes;
                     // the store issued two groups ago read this buffer: wait until it no longer does
                     if (lane == 0) tma_store_wait_read<1>();
@@ -372,13 +401,16 @@ cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void
     g.lower_h = s.lower_h; g.lower_w = s.lower_w; g.stride_h = s.stride_h; g.stride_w = s.stride_w;
     g.dil_h = s.dil_h; g.dil_w = s.dil_w; g.p = (long long)s.n * s.ho * s.wo; g.stages = 1;
     g.blockdiag = s.blockdiag;
+    g.out_strided = s.out_sw ? (__nv_bfloat16 *)out : nullptr;
+    g.out_sn = s.out_sn; g.out_sh = s.out_sh; g.out_sw = s.out_sw;
     // The bounding box of base pixels has ho x wo positions: upper = lower + (out-1) stride - (in-1).
     const int upper_h = s.lower_h + (s.ho - 1) * s.stride_h - (s.ha - 1);
     const int upper_w = s.lower_w + (s.wo - 1) * s.stride_w - (s.wa - 1);
     const long long tiles_m = (g.p + kBM - 1) / kBM;
     const int bn = s.blockdiag ? 64 : pick_bn(tiles_m, s.cn);
     CUtensorMap ta, tw, tout;
-    if (!make_tmap_matrix_bf16(&tout, out, g.p, s.cn, 32, 64)) return cudaErrorInvalidValue;
+    // (in strided mode the output map is encoded but never used: every row is stored by its thread)
+    if (!make_tmap_matrix_bf16(&tout, out, s.out_sw ? 32 : g.p, s.cn, 32, 64)) return cudaErrorInvalidValue;
     if (!make_tmap_im2col_bf16(&ta, act, s.n, s.ha, s.wa, s.ca, s.lower_h, s.lower_w, upper_h, upper_w, s.stride_h,
                                s.stride_w, kBM, kBK))
         return cudaErrorInvalidValue;
