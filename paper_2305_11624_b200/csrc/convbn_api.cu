@@ -116,7 +116,7 @@ struct Plan {
     size_t dy = 0;         // Eval backward: s dZ, storage dtype
     size_t vec3 = 0;       // Eval forward: [s | beta - mean s | r]
     size_t dotpart = 0;    // [kt][C_out] fp32 (tensor-core weight-gradient path)
-    int splits = 1, bsplits = 1;
+    int splits = 1, bsplits = 1, bn_splits = 1;
     size_t wbd = 0;        // block-diagonal expanded weights [C_out][taps][64], storage dtype
     bool umma_wgrad = false, dw_wgrad = false, grouped_wgrad = false;
     UmmaWgradPlan uw;
@@ -130,6 +130,7 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
     const size_t wrows = (size_t)pb.c_out * pb.kdim;
     pl.splits = direct_wgrad_splits(pb);
     pl.bsplits = channel_sum_splits(pb);
+    pl.bn_splits = pl.bsplits;                      // pixel slices of the Eval-mode BatchNorm backward
     pl.umma_wgrad = !force_direct() && d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC &&
                     umma_wgrad_eligible(pb);
     size_t part_bytes = wrows * pl.splits * sizeof(float), dot_bytes = 0;
@@ -144,10 +145,12 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
     pl.grouped_wgrad = grouped;
     if (grouped) {
         pl.uw = umma_wgrad_plan(pb);
+        pl.bsplits = pl.uw.splits;
         part_bytes = (size_t)pl.uw.splits * (pb.c_out / 64) * pb.kh * pb.kw * 64 * 64 * sizeof(float);
     }
     if (pl.umma_wgrad) {
         pl.uw = umma_wgrad_plan(pb);
+        pl.bsplits = pl.uw.splits;
         part_bytes = wrows * pl.uw.splits * sizeof(float);
         dot_bytes = (size_t)pl.uw.kt * pb.c_out * sizeof(float);
     }
@@ -180,8 +183,8 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
             pl.dy = take((size_t)pb.p * pb.c_out * elem_size(d->dtype));
             pl.w_scaled = take(wbytes);
             pl.wbd = take(wbd_bytes);
-            pl.part_g = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
-            pl.bsum = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
+            pl.part_g = take((size_t)pl.bn_splits * pb.c_out * sizeof(float));
+            pl.bsum = take((size_t)(pl.bn_splits > pl.bsplits ? pl.bn_splits : pl.bsplits) * pb.c_out * sizeof(float));
             pl.partials = take(part_bytes);
             pl.dotpart = take(dot_bytes);
             break;
@@ -392,17 +395,18 @@ int run_param_grads(const convbn_desc *d, const Problem &pb, const Plan &pl, con
                     float *dgamma, float *dbeta, void *ws, cudaStream_t st, const char **which) {
     float *partials = (float *)at(ws, pl.partials), *bsum = (float *)at(ws, pl.bsum);
     const bool need_bsum = vec3 || db;
-    if (need_bsum)
+    const bool tc = pl.grouped_wgrad || pl.umma_wgrad;      // tensor-core paths sum dZ inside the GEMM
+    if (need_bsum && !tc)
         LAUNCH("channel_sum", launch_channel_sum_partial(pb, d->dtype, d->layout, dz, bsum, pl.bsplits, st));
     if (pl.grouped_wgrad) {
-        LAUNCH("grouped_wgrad", launch_umma_wgrad(pb, pl.uw, dz, x, partials, st));
+        LAUNCH("grouped_wgrad", launch_umma_wgrad(pb, pl.uw, dz, x, partials, bsum, st));
         LAUNCH("wgrad_epilogue_bd", launch_wgrad_epilogue_bd(pb, partials, pl.uw.splits, need_bsum ? bsum : nullptr,
                                                              need_bsum ? pl.bsplits : 0, w, vec3, b, mean, dw, db,
                                                              dgamma, dbeta, st));
         *which = "grouped-umma";
     } else if (pl.umma_wgrad) {
         float *dotpart = (float *)at(ws, pl.dotpart);
-        LAUNCH("umma_wgrad", launch_umma_wgrad(pb, pl.uw, dz, x, partials, st));
+        LAUNCH("umma_wgrad", launch_umma_wgrad(pb, pl.uw, dz, x, partials, bsum, st));
         LAUNCH("wgrad_epilogue_t", launch_wgrad_epilogue_t(pb, pl.uw, partials, w, vec3, dw, dotpart, st));
         if (need_bsum)
             LAUNCH("param_finish", launch_param_finish(pb, pl.uw, dotpart, bsum, pl.bsplits, vec3, b, mean, db,
@@ -555,8 +559,8 @@ int convbn_eval_bwd(const convbn_desc *desc, const void *dz, const void *x, cons
     void *dy = at(workspace, pl.dy);
     float *pg = (float *)at(workspace, pl.part_g), *pbm = (float *)at(workspace, pl.bsum);
     LAUNCH("bn_eval_bwd", launch_bn_eval_bwd(pb, desc->dtype, desc->layout, dz, y_saved, gamma, run_mean, run_var, dy, pg,
-                          pbm, pl.bsplits, st));
-    LAUNCH("bn_eval_finish", launch_bn_eval_finish(pb, pg, pbm, pl.bsplits, gamma, run_var, db, dgamma, dbeta, st));
+                          pbm, pl.bn_splits, st));
+    LAUNCH("bn_eval_finish", launch_bn_eval_finish(pb, pg, pbm, pl.bn_splits, gamma, run_var, db, dgamma, dbeta, st));
     CK(run_conv_dgrad(desc, pb, dy, w, nullptr, at(workspace, pl.w_scaled), at(workspace, pl.wbd), dx, st,
                       &t_last_kernel[CONVBN_PHASE_EVAL_BWD]));
     const char *unused = nullptr;

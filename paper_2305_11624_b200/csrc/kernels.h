@@ -68,8 +68,9 @@ struct UmmaWgradPlan {
 bool umma_wgrad_eligible(const Problem &pb);
 UmmaWgradPlan umma_wgrad_plan(const Problem &pb);
 // partials: [splits][kdim][C_out] fp32 (k-major: the transpose of the weight layout)
+// bsum    : [splits][C_out] fp32 per-slice sums of dZ over pixels (from a ones row in the GEMM)
 cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const void *dz, const void *x,
-                              float *partials, cudaStream_t st);
+                              float *partials, float *bsum, cudaStream_t st);
 // dw[co][k] = scale[co] * sum_splits partials (scale = first C_out floats of vec3, 1 if NULL);
 // dotpart[kt][C_out] = per-k-range pieces of sum_k (sum_splits partials) w[co][k]  (only if vec3)
 cudaError_t launch_wgrad_epilogue_t(const Problem &pb, const UmmaWgradPlan &pl, const float *partials,

@@ -44,7 +44,7 @@ template <int BN>
 __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_constant__ CUtensorMap tm_x,
                                                               const __grid_constant__ CUtensorMap tm_dz,
                                                               const WgradGemm g, float *__restrict__ partials,
-                                                              int *err) {
+                                                              float *__restrict__ bsum, int *err) {
     extern __shared__ uint8_t smem_raw[];
     constexpr uint32_t kABytes = 2 * kChunkBytes, kBBytes = (BN / 64) * kChunkBytes, kStageBytes = kABytes + kBBytes;
     uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -56,7 +56,11 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
     const long long p0 = (long long)blockIdx.z * g.per_split;
     const long long p1 = p0 + g.per_split < g.p ? p0 + g.per_split : g.p;
     const int num_kb = (int)((p1 - p0 + kWP - 1) / kWP);
-    const int a_chunks = (k0 + 64 < g.kdim) ? 2 : 1;    // second 64-slice may fall beyond K
+    // The list of 64-row slices is the K / 64 real ones followed by one slice of constant ones: its
+    // accumulator rows are sum_p dZ[p][co], the per-channel sums needed for dbeta (Table 2), for free.
+    const int nch = g.kdim / 64, c_first = k0 / 64;
+    const int a_chunks = nch - c_first >= 2 ? 2 : (nch - c_first >= 1 ? 1 : 0);   // slices loaded by TMA
+    const int ones_slot = (c_first == nch) ? 0 : (c_first + 1 == nch ? 1 : -1);
     int b_chunks = (g.c_out - n0) / 64;
     if (b_chunks > BN / 64) b_chunks = BN / 64;
     volatile int *abort_flag = &ctl->abort_flag;
@@ -70,6 +74,15 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
     if (warp == 1) {
         tmem_alloc(&ctl->tmem_base, BN);
         tmem_relinquish();
+    }
+    if (ones_slot >= 0) {
+        // bf16 1.0 everywhere (invariant under the swizzle); TMA never writes this slice
+        const uint4 ones = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
+        for (int s = 0; s < stages; ++s) {
+            uint4 *dst = (uint4 *)(tiles + (size_t)s * kStageBytes + (size_t)ones_slot * kChunkBytes);
+            for (int i = threadIdx.x; i < (int)(kChunkBytes / 16); i += kWThreads) dst[i] = ones;
+        }
+        fence_proxy_async_smem();
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -153,6 +166,8 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
             tc_fence_after_sync();
             const int k = k0 + quarter * 32 + lane;
             const bool row_ok = k < g.kdim;
+            const bool sum_row = (k == g.kdim);             // first row of the ones slice
+            float *brow = bsum + (size_t)blockIdx.z * g.c_out + n0;
             float *orow = g.blockdiag
                               ? partials + (((size_t)blockIdx.z * gridDim.y + blockIdx.y) * g.kdim + (row_ok ? k : 0)) * 64
                               : partials + ((size_t)blockIdx.z * g.kdim + (row_ok ? k : 0)) * g.c_out + n0;
@@ -166,6 +181,10 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
 #pragma unroll
                     for (int j = 0; j < 32; j += 4)
                         *(uint4 *)(orow + c0 + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                } else if (sum_row) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4)
+                        *(uint4 *)(brow + c0 + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
                 }
             }
         }
@@ -200,7 +219,7 @@ UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
     const bool bd = pb.groups > 1;
     const int bn = bd ? 64 : wgrad_bn(pb);
     const long long kd = bd ? (long long)pb.kh * pb.kw * 64 : pb.kdim;
-    const long long m_tiles = (kd + kWM - 1) / kWM, n_tiles = (pb.c_out + bn - 1) / bn;
+    const long long m_tiles = (kd / 64 + 1 + 1) / 2, n_tiles = (pb.c_out + bn - 1) / bn;   // + the ones slice
     const long long target = 148;
     long long splits = (target + m_tiles * n_tiles - 1) / (m_tiles * n_tiles);
     const long long max_splits = (pb.p + 4 * kWP - 1) / (4 * kWP);     // at least 256 pixels per slice
@@ -216,7 +235,7 @@ UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
 
 template <int BN>
 static cudaError_t launch_w(const CUtensorMap &tx, const CUtensorMap &tdz, WgradGemm g, const UmmaWgradPlan &pl,
-                            const Problem &pb, float *partials, int *err, cudaStream_t st) {
+                            const Problem &pb, float *partials, float *bsum, int *err, cudaStream_t st) {
     constexpr size_t stage = 2 * kChunkBytes + (BN / 64) * kChunkBytes;
     int stages = BN == 256 ? 4 : 4;
     const long long max_kb = (pl.per_split + kWP - 1) / kWP;
@@ -232,13 +251,13 @@ static cudaError_t launch_w(const CUtensorMap &tx, const CUtensorMap &tdz, Wgrad
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    dim3 grid((unsigned)((g.kdim + kWM - 1) / kWM), (unsigned)((pb.c_out + BN - 1) / BN), (unsigned)pl.splits);
-    umma_wgrad_kernel<BN><<<grid, kWThreads, smem, st>>>(tx, tdz, g, partials, err);
+    dim3 grid((unsigned)((g.kdim / 64 + 2) / 2), (unsigned)((pb.c_out + BN - 1) / BN), (unsigned)pl.splits);
+    umma_wgrad_kernel<BN><<<grid, kWThreads, smem, st>>>(tx, tdz, g, partials, bsum, err);
     return cudaGetLastError();
 }
 
 cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const void *dz, const void *x,
-                              float *partials, cudaStream_t st) {
+                              float *partials, float *bsum, cudaStream_t st) {
     WgradGemm g;
     g.ho = pb.h_out; g.wo = pb.w_out; g.c_in = pb.c_in; g.c_out = pb.c_out; g.taps_w = pb.kw;
     g.lower_h = -pb.pad_h; g.lower_w = -pb.pad_w; g.stride_h = pb.stride_h; g.stride_w = pb.stride_w;
@@ -256,9 +275,9 @@ cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
     cudaError_t e = error_word_address(&err);
     if (e != cudaSuccess) return e;
     const int bn = g.blockdiag ? 64 : wgrad_bn(pb);
-    if (bn == 64) return launch_w<64>(tx, tdz, g, pl, pb, partials, err, st);
-    if (bn == 128) return launch_w<128>(tx, tdz, g, pl, pb, partials, err, st);
-    return launch_w<256>(tx, tdz, g, pl, pb, partials, err, st);
+    if (bn == 64) return launch_w<64>(tx, tdz, g, pl, pb, partials, bsum, err, st);
+    if (bn == 128) return launch_w<128>(tx, tdz, g, pl, pb, partials, bsum, err, st);
+    return launch_w<256>(tx, tdz, g, pl, pb, partials, bsum, err, st);
 }
 
 // ---- epilogue over k-major partials ------------------------------------------------------------
