@@ -116,6 +116,7 @@ struct Plan {
     size_t dy = 0;         // Eval backward: s dZ, storage dtype
     size_t vec3 = 0;       // Eval forward: [s | beta - mean s | r]
     size_t dotpart = 0;    // [kt][C_out] fp32 (tensor-core weight-gradient path)
+    size_t counters = 0;   // C_out / 32 words (fused epilogue)
     int splits = 1, bsplits = 1, bn_splits = 1;
     size_t wbd = 0;        // block-diagonal expanded weights [C_out][taps][64], storage dtype
     bool umma_wgrad = false, dw_wgrad = false, grouped_wgrad = false;
@@ -169,11 +170,13 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
             pl.partials = take(part_bytes);
             pl.bsum = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
             pl.dotpart = take(dot_bytes);
+            pl.counters = take(dot_bytes ? (size_t)(pb.c_out / 32 + 1) * sizeof(unsigned int) : 0);
             break;
         case CONVBN_PHASE_TUNE_BWD_WEIGHT:
             pl.partials = take(part_bytes);
             pl.bsum = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
             pl.dotpart = take(dot_bytes);
+            pl.counters = take(dot_bytes ? (size_t)(pb.c_out / 32 + 1) * sizeof(unsigned int) : 0);
             break;
         case CONVBN_PHASE_EVAL_FWD:
             pl.vec3 = take(3 * (size_t)pb.c_out * sizeof(float));
@@ -187,6 +190,7 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
             pl.bsum = take((size_t)(pl.bn_splits > pl.bsplits ? pl.bn_splits : pl.bsplits) * pb.c_out * sizeof(float));
             pl.partials = take(part_bytes);
             pl.dotpart = take(dot_bytes);
+            pl.counters = take(dot_bytes ? (size_t)(pb.c_out / 32 + 1) * sizeof(unsigned int) : 0);
             break;
         default:
             break;
@@ -399,18 +403,18 @@ int run_param_grads(const convbn_desc *d, const Problem &pb, const Plan &pl, con
     if (need_bsum && !tc)
         LAUNCH("channel_sum", launch_channel_sum_partial(pb, d->dtype, d->layout, dz, bsum, pl.bsplits, st));
     if (pl.grouped_wgrad) {
-        LAUNCH("grouped_wgrad", launch_umma_wgrad(pb, pl.uw, dz, x, partials, bsum, st));
+        LAUNCH("grouped_wgrad", launch_umma_wgrad(pb, pl.uw, dz, x, partials, bsum, nullptr, st));
         LAUNCH("wgrad_epilogue_bd", launch_wgrad_epilogue_bd(pb, partials, pl.uw.splits, need_bsum ? bsum : nullptr,
                                                              need_bsum ? pl.bsplits : 0, w, vec3, b, mean, dw, db,
                                                              dgamma, dbeta, st));
         *which = "grouped-umma";
     } else if (pl.umma_wgrad) {
         float *dotpart = (float *)at(ws, pl.dotpart);
-        LAUNCH("umma_wgrad", launch_umma_wgrad(pb, pl.uw, dz, x, partials, bsum, st));
-        LAUNCH("wgrad_epilogue_t", launch_wgrad_epilogue_t(pb, pl.uw, partials, w, vec3, dw, dotpart, st));
-        if (need_bsum)
-            LAUNCH("param_finish", launch_param_finish(pb, pl.uw, dotpart, bsum, pl.bsplits, vec3, b, mean, db,
-                                                       dgamma, dbeta, st));
+        unsigned int *counters = (unsigned int *)at(ws, pl.counters);
+        LAUNCH("umma_wgrad", launch_umma_wgrad(pb, pl.uw, dz, x, partials, bsum, counters, st));
+        LAUNCH("wgrad_epilogue_fused", launch_wgrad_epilogue_fused(pb, pl.uw, partials, bsum, w, vec3, b, mean, dw,
+                                                                   dotpart, counters, db, dgamma, dbeta, need_bsum,
+                                                                   st));
         *which = "umma";
     } else {
         if (pl.dw_wgrad)

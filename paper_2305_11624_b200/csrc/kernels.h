@@ -69,17 +69,16 @@ bool umma_wgrad_eligible(const Problem &pb);
 UmmaWgradPlan umma_wgrad_plan(const Problem &pb);
 // partials: [splits][kdim][C_out] fp32 (k-major: the transpose of the weight layout)
 // bsum    : [splits][C_out] fp32 per-slice sums of dZ over pixels (from a ones row in the GEMM)
+// counters: C_out / 32 words zeroed for the fused epilogue (may be NULL)
 cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const void *dz, const void *x,
-                              float *partials, float *bsum, cudaStream_t st);
-// dw[co][k] = scale[co] * sum_splits partials (scale = first C_out floats of vec3, 1 if NULL);
-// dotpart[kt][C_out] = per-k-range pieces of sum_k (sum_splits partials) w[co][k]  (only if vec3)
-cudaError_t launch_wgrad_epilogue_t(const Problem &pb, const UmmaWgradPlan &pl, const float *partials,
-                                    const void *w, const float *vec3, float *dw, float *dotpart,
-                                    cudaStream_t st);
-// dbeta, db, dgamma from dotpart and the per-channel dZ sums (tune mode), or db = sum dZ (vec3 NULL).
-cudaError_t launch_param_finish(const Problem &pb, const UmmaWgradPlan &pl, const float *dotpart,
-                                const float *bsum_part, int bsplits, const float *vec3, const float *b,
-                                const float *mean, float *db, float *dgamma, float *dbeta, cudaStream_t st);
+                              float *partials, float *bsum, unsigned int *counters, cudaStream_t st);
+// Everything after the GEMM in one kernel: dw[co][k] = scale[co] * sum_splits partials (scale = first
+// C_out floats of vec3, 1 if NULL); with need_sums also dbeta, db, dgamma (vec3 given) or db = sum dZ.
+// dotpart: [kt][C_out] scratch; counters: C_out / 32 zeroed words.
+cudaError_t launch_wgrad_epilogue_fused(const Problem &pb, const UmmaWgradPlan &pl, const float *partials,
+                                        const float *bsum, const void *w, const float *vec3, const float *b,
+                                        const float *mean, float *dw, float *dotpart, unsigned int *counters,
+                                        float *db, float *dgamma, float *dbeta, bool need_sums, cudaStream_t st);
 
 // ---- depthwise (groups = C_in = C_out) bandwidth kernels, bf16 NHWC, C multiple of 8 -----------
 bool dw_eligible(const Problem &pb);

@@ -44,7 +44,9 @@ template <int BN>
 __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_constant__ CUtensorMap tm_x,
                                                               const __grid_constant__ CUtensorMap tm_dz,
                                                               const WgradGemm g, float *__restrict__ partials,
-                                                              float *__restrict__ bsum, int *err) {
+                                                              float *__restrict__ bsum,
+                                                              unsigned int *__restrict__ counters, int ncounters,
+                                                              int *err) {
     extern __shared__ uint8_t smem_raw[];
     constexpr uint32_t kABytes = 2 * kChunkBytes, kBBytes = (BN / 64) * kChunkBytes, kStageBytes = kABytes + kBBytes;
     uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -75,6 +77,9 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
         tmem_alloc(&ctl->tmem_base, BN);
         tmem_relinquish();
     }
+    // counters of the epilogue kernel that runs after this one start from zero
+    if (counters && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
+        for (int i = threadIdx.x; i < ncounters; i += kWThreads) counters[i] = 0u;
     if (ones_slot >= 0) {
         // bf16 1.0 everywhere (invariant under the swizzle); TMA never writes this slice
         const uint4 ones = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
@@ -235,7 +240,8 @@ UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
 
 template <int BN>
 static cudaError_t launch_w(const CUtensorMap &tx, const CUtensorMap &tdz, WgradGemm g, const UmmaWgradPlan &pl,
-                            const Problem &pb, float *partials, float *bsum, int *err, cudaStream_t st) {
+                            const Problem &pb, float *partials, float *bsum, unsigned int *counters, int *err,
+                            cudaStream_t st) {
     constexpr size_t stage = 2 * kChunkBytes + (BN / 64) * kChunkBytes;
     int stages = BN == 256 ? 4 : 4;
     const long long max_kb = (pl.per_split + kWP - 1) / kWP;
@@ -252,12 +258,12 @@ static cudaError_t launch_w(const CUtensorMap &tx, const CUtensorMap &tdz, Wgrad
         attr_done = true;
     }
     dim3 grid((unsigned)((g.kdim / 64 + 2) / 2), (unsigned)((pb.c_out + BN - 1) / BN), (unsigned)pl.splits);
-    umma_wgrad_kernel<BN><<<grid, kWThreads, smem, st>>>(tx, tdz, g, partials, bsum, err);
+    umma_wgrad_kernel<BN><<<grid, kWThreads, smem, st>>>(tx, tdz, g, partials, bsum, counters, pb.c_out / 32, err);
     return cudaGetLastError();
 }
 
 cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const void *dz, const void *x,
-                              float *partials, float *bsum, cudaStream_t st) {
+                              float *partials, float *bsum, unsigned int *counters, cudaStream_t st) {
     WgradGemm g;
     g.ho = pb.h_out; g.wo = pb.w_out; g.c_in = pb.c_in; g.c_out = pb.c_out; g.taps_w = pb.kw;
     g.lower_h = -pb.pad_h; g.lower_w = -pb.pad_w; g.stride_h = pb.stride_h; g.stride_w = pb.stride_w;
@@ -275,99 +281,106 @@ cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
     cudaError_t e = error_word_address(&err);
     if (e != cudaSuccess) return e;
     const int bn = g.blockdiag ? 64 : wgrad_bn(pb);
-    if (bn == 64) return launch_w<64>(tx, tdz, g, pl, pb, partials, bsum, err, st);
-    if (bn == 128) return launch_w<128>(tx, tdz, g, pl, pb, partials, bsum, err, st);
-    return launch_w<256>(tx, tdz, g, pl, pb, partials, bsum, err, st);
+    if (bn == 64) return launch_w<64>(tx, tdz, g, pl, pb, partials, bsum, counters, err, st);
+    if (bn == 128) return launch_w<128>(tx, tdz, g, pl, pb, partials, bsum, counters, err, st);
+    return launch_w<256>(tx, tdz, g, pl, pb, partials, bsum, counters, err, st);
 }
 
 // ---- epilogue over k-major partials ------------------------------------------------------------
-// part[split][k][co] -> dw[co][k] = scale[co] * sum_split part;  dotpart[blockIdx.y][co] = sum over the
-// block's 8 k rows of (sum_split part) * w[co][k].  Block = 32 output channels x 8 k rows.
-__global__ void __launch_bounds__(256) wgrad_epilogue_t_kernel(int c_out, int kdim, const float *__restrict__ part,
-                                                              int splits, const __nv_bfloat16 *__restrict__ w,
-                                                              const float *__restrict__ vec3,
-                                                              float *__restrict__ dw, float *__restrict__ dotpart) {
-    __shared__ float tile[8][33];
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+// One kernel finishes every parameter gradient (Table 2, Tune row) from the fp32 partial tiles:
+//   block (bx, by): 32 output channels x 8 k rows, 4 lanes over the pixel slices (1024 threads)
+//     acc[k][co] = sum_split part[split][k][co]        (each lane a strided subset, lanes added in order)
+//     dw[co][k]  = s[co] acc                           (transposed through shared memory)
+//     dotpart[by][co] = sum over the block's k rows of acc * w[co][k]
+//   the LAST block to finish for a group of 32 channels (a counter per group, zeroed by the GEMM
+//   kernel) adds dotpart over all k blocks and bsum over all slices, lanes strided + a fixed shuffle
+//   tree, so the result does not depend on which block came last:
+//     dbeta = sum dZ,  db = s dbeta,  dgamma = r (sum_k domega' omega + dbeta (b - mu_hat))
+//   plain mode (vec3 == NULL): dw = acc, db = sum dZ if requested.
+__global__ void __launch_bounds__(1024) wgrad_epilogue_fused_kernel(
+    int c_out, int kdim, const float *__restrict__ part, int splits, const float *__restrict__ bsum, int bsplits,
+    const __nv_bfloat16 *__restrict__ w, const float *__restrict__ vec3, const float *__restrict__ b,
+    const float *__restrict__ mean, float *__restrict__ dw, float *__restrict__ dotpart,
+    unsigned int *__restrict__ counters, float *__restrict__ db, float *__restrict__ dgamma,
+    float *__restrict__ dbeta, int need_sums) {
+    __shared__ float tile[4][8][33];
+    __shared__ int is_last;
+    const int tx = threadIdx.x & 31, ty = (threadIdx.x >> 5) & 7, tz = threadIdx.x >> 8;
     const int co0 = blockIdx.x * 32, k0 = blockIdx.y * 8;
     const size_t slice = (size_t)kdim * c_out;
     {
         const int k = k0 + ty;
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        float a0 = 0.f, a1 = 0.f;
         if (k < kdim) {
             const float *src = part + (size_t)k * c_out + co0 + tx;
-            int sp = 0;
-            for (; sp + 4 <= splits; sp += 4) {
+            int sp = tz;
+            for (; sp + 4 < splits; sp += 8) {
                 a0 += src[(size_t)sp * slice];
-                a1 += src[(size_t)(sp + 1) * slice];
-                a2 += src[(size_t)(sp + 2) * slice];
-                a3 += src[(size_t)(sp + 3) * slice];
+                a1 += src[(size_t)(sp + 4) * slice];
             }
-            for (; sp < splits; ++sp) a0 += src[(size_t)sp * slice];
+            if (sp < splits) a0 += src[(size_t)sp * slice];
         }
-        tile[ty][tx] = (a0 + a1) + (a2 + a3);
+        tile[tz][ty][tx] = a0 + a1;
     }
     __syncthreads();
-    const int kk = threadIdx.x & 7, cl = threadIdx.x >> 3, k = k0 + kk, co = co0 + cl;
-    float d = 0.f;
-    if (k < kdim) {
-        const float v = tile[kk][cl];
-        const size_t o = (size_t)co * kdim + k;
-        dw[o] = (vec3 ? vec3[co] : 1.f) * v;
-        if (dotpart) d = v * __bfloat162float(w[o]);
+    if (threadIdx.x < 256) {
+        const int kk = threadIdx.x & 7, cl = threadIdx.x >> 3, k = k0 + kk, co = co0 + cl;
+        float d = 0.f;
+        if (k < kdim) {
+            const float v = (tile[0][kk][cl] + tile[1][kk][cl]) + (tile[2][kk][cl] + tile[3][kk][cl]);
+            const size_t o = (size_t)co * kdim + k;
+            dw[o] = (vec3 ? vec3[co] : 1.f) * v;
+            if (vec3) d = v * __bfloat162float(w[o]);
+        }
+        if (vec3) {
+            d += __shfl_xor_sync(0xffffffffu, d, 1);
+            d += __shfl_xor_sync(0xffffffffu, d, 2);
+            d += __shfl_xor_sync(0xffffffffu, d, 4);
+            if (kk == 0) dotpart[(size_t)blockIdx.y * c_out + co] = d;
+        }
     }
-    if (dotpart) {
-        d += __shfl_xor_sync(0xffffffffu, d, 1);
-        d += __shfl_xor_sync(0xffffffffu, d, 2);
-        d += __shfl_xor_sync(0xffffffffu, d, 4);
-        if (kk == 0) dotpart[(size_t)blockIdx.y * c_out + co] = d;
+    if (!need_sums) return;
+    // ---- last block of this channel group finishes the per-channel quantities ----
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int done = atomicAdd(&counters[blockIdx.x], 1u);
+        is_last = (done == gridDim.y - 1);
     }
-}
-
-// One warp per output channel: dbeta = sum dZ; db = s dbeta;
-// dgamma = r (sum_k domega' omega + dbeta (b - mu_hat))   (Table 2, Tune row).
-// Plain mode (vec3 == NULL): db = sum dZ only.  Lanes add strided pieces, then a fixed shuffle tree.
-__global__ void __launch_bounds__(256) param_finish_kernel(int c_out, const float *__restrict__ dotpart, int kt,
-                                                          const float *__restrict__ bsum_part, int bsplits,
-                                                          const float *__restrict__ vec3,
-                                                          const float *__restrict__ b,
-                                                          const float *__restrict__ mean, float *__restrict__ db,
-                                                          float *__restrict__ dgamma, float *__restrict__ dbeta) {
-    const int co = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-    if (co >= c_out) return;
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const int warp = threadIdx.x >> 5, lane = tx;
+    const int co = co0 + warp;                      // 32 warps, one per channel
     float dsum = 0.f, dot = 0.f;
-    for (int sp = lane; sp < bsplits; sp += 32) dsum += bsum_part[(size_t)sp * c_out + co];
+    for (int sp = lane; sp < bsplits; sp += 32) dsum += __ldcg(bsum + (size_t)sp * c_out + co);
     if (vec3)
-        for (int t = lane; t < kt; t += 32) dot += dotpart[(size_t)t * c_out + co];
+        for (int t = lane; t < (int)gridDim.y; t += 32) dot += __ldcg(dotpart + (size_t)t * c_out + co);
     for (int o = 16; o > 0; o >>= 1) {
         dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
         dot += __shfl_xor_sync(0xffffffffu, dot, o);
     }
-    if (lane) return;
-    if (!vec3) {
-        if (db) db[co] = dsum;
-        return;
+    if (lane == 0) {
+        if (!vec3) {
+            if (db) db[co] = dsum;
+        } else {
+            const float s = vec3[co], r = vec3[2 * c_out + co];
+            dbeta[co] = dsum;
+            if (db) db[co] = s * dsum;
+            dgamma[co] = r * (dot + dsum * ((b ? b[co] : 0.f) - mean[co]));
+        }
     }
-    const float s = vec3[co], r = vec3[2 * c_out + co];
-    dbeta[co] = dsum;
-    if (db) db[co] = s * dsum;
-    dgamma[co] = r * (dot + dsum * ((b ? b[co] : 0.f) - mean[co]));
+    if (threadIdx.x == 0) counters[blockIdx.x] = 0;   // leave the counter clean for the next call
 }
 
-cudaError_t launch_wgrad_epilogue_t(const Problem &pb, const UmmaWgradPlan &pl, const float *partials,
-                                    const void *w, const float *vec3, float *dw, float *dotpart,
-                                    cudaStream_t st) {
+cudaError_t launch_wgrad_epilogue_fused(const Problem &pb, const UmmaWgradPlan &pl, const float *partials,
+                                        const float *bsum, const void *w, const float *vec3, const float *b,
+                                        const float *mean, float *dw, float *dotpart, unsigned int *counters,
+                                        float *db, float *dgamma, float *dbeta, bool need_sums, cudaStream_t st) {
     dim3 grid(pb.c_out / 32, pl.kt);
-    wgrad_epilogue_t_kernel<<<grid, 256, 0, st>>>(pb.c_out, pb.kdim, partials, pl.splits,
-                                                  (const __nv_bfloat16 *)w, vec3, dw, vec3 ? dotpart : nullptr);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_param_finish(const Problem &pb, const UmmaWgradPlan &pl, const float *dotpart,
-                                const float *bsum_part, int bsplits, const float *vec3, const float *b,
-                                const float *mean, float *db, float *dgamma, float *dbeta, cudaStream_t st) {
-    param_finish_kernel<<<(pb.c_out + 7) / 8, 256, 0, st>>>(pb.c_out, dotpart, pl.kt, bsum_part, bsplits, vec3, b,
-                                                           mean, db, dgamma, dbeta);
+    wgrad_epilogue_fused_kernel<<<grid, 1024, 0, st>>>(pb.c_out, pb.kdim, partials, pl.splits, bsum, pl.splits,
+                                                       (const __nv_bfloat16 *)w, vec3, b, mean, dw, dotpart, counters,
+                                                       db, dgamma, dbeta, need_sums ? 1 : 0);
     return cudaGetLastError();
 }
 
