@@ -476,6 +476,15 @@ int convbn_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const
     cudaStream_t st = (cudaStream_t)stream;
     float *vec3 = (float *)saved;
     void *wf = at(workspace, pl.w_scaled);
+    UmmaConvShape us;
+    if (!grouped_path(desc, pb) && umma_fwd_shape(desc, pb, &us)) {
+        // dense tensor-core path: s, b' and the saved vectors are formed inside the GEMM kernel and s is
+        // applied to the fp32 accumulator, so one launch does the whole forward pass
+        const BnFold fold{gamma, beta, run_mean, run_var, b, pb.eps, vec3};
+        LAUNCH("umma_fwd", launch_umma_conv(us, x, w, nullptr, z, st, &fold));
+        t_last_kernel[CONVBN_PHASE_TUNE_FWD] = "umma";
+        return CONVBN_OK;
+    }
     LAUNCH("reparam", launch_reparam(pb, desc->dtype, desc->layout, w, b, gamma, beta, run_mean, run_var, vec3, wf,
                       nullptr, st));
     CK(run_conv_fwd(desc, pb, x, wf, vec3 + pb.c_out, z, at(workspace, pl.wbd), st, &t_last_kernel[CONVBN_PHASE_TUNE_FWD]));

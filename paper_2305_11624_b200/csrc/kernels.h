@@ -48,8 +48,16 @@ struct UmmaConvShape {
     int out_sh = 0, out_sw = 0;
 };
 bool umma_conv_eligible(const UmmaConvShape &s);
+// BatchNorm parameters for in-kernel reparameterisation: the kernel forms s and b' per output channel,
+// computes out = s * (wmat (*) act) + b' and (CTA 0) writes [s | b' | r] to vec3 (3 cn floats, may be NULL).
+struct BnFold {
+    const float *gamma, *beta, *mean, *var, *b;   // b may be NULL
+    float eps;
+    float *vec3;
+};
+// fold != NULL replaces `bias` (dense output mode only).
 cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void *wmat, const float *bias,
-                             void *out, cudaStream_t st);
+                             void *out, cudaStream_t st, const BnFold *fold = nullptr);
 // Weight operand of the backward-data GEMM: w_t[ci][taps-1-tap][co] = s[co] w[co][tap][ci]
 // (s_vec == NULL: unscaled).  bf16, groups = 1.
 cudaError_t launch_reparam_dgrad(const Problem &pb, const void *w, const float *s_vec, void *w_t,
@@ -64,6 +72,7 @@ struct UmmaWgradPlan {
     int splits = 1;           // pixel slices = partial tiles
     long long per_split = 0;  // pixels per slice
     int kt = 1;               // k ranges of the epilogue (rows of dotpart)
+    int kr = 8;               // k rows per epilogue block (8 or 2)
 };
 bool umma_wgrad_eligible(const Problem &pb);
 UmmaWgradPlan umma_wgrad_plan(const Problem &pb);

@@ -42,6 +42,7 @@ struct ConvGemm {
     __nv_bfloat16 *out_strided;
     long long out_sn;
     int out_sh, out_sw;
+    BnFold fold;             // fold.gamma != NULL: scale and shift formed in the kernel from the BN parameters
 };
 
 struct ConvSmemCtl {
@@ -69,6 +70,8 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
     uint8_t *staging = tiles + (size_t)g.stages * kStageBytes;         // 4 warps x 2 x [32 rows][128 B]
     ConvSmemCtl *ctl = (ConvSmemCtl *)(staging + kStagingBytes);
     float *bias_s = (float *)(((uintptr_t)(ctl + 1) + 15) & ~(uintptr_t)15);   // cn floats
+    float *scale_s = bias_s + g.cn;                                            // cn floats (fold mode)
+    const bool fold = g.fold.gamma != nullptr;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int stages = g.stages;
     const int cchunks = g.blockdiag ? 1 : g.ca / kBK;
@@ -87,8 +90,22 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
         tmem_alloc(&ctl->tmem_base, 2 * BN);
         tmem_relinquish();
     }
-    if (bias)
+    if (fold) {
+        // On-the-fly reparameterisation (Sec. 3.3 / 3.4): s = gamma / sqrt(var + eps), b' = (b - mu) s + beta.
+        // s multiplies the fp32 accumulator (the associative law of Sec. 3.2.2), so omega is used unrounded.
+        for (int c = threadIdx.x; c < g.cn; c += kConvThreads) {
+            const float r = 1.0f / sqrtf(g.fold.var[c] + g.fold.eps);
+            const float sc = g.fold.gamma[c] * r;
+            const float bf = ((g.fold.b ? g.fold.b[c] : 0.f) - g.fold.mean[c]) * sc + g.fold.beta[c];
+            scale_s[c] = sc;
+            bias_s[c] = bf;
+            if (blockIdx.x == 0 && g.fold.vec3) {
+                g.fold.vec3[c] = sc; g.fold.vec3[g.cn + c] = bf; g.fold.vec3[2 * g.cn + c] = r;
+            }
+        }
+    } else if (bias) {
         for (int c = threadIdx.x; c < g.cn; c += kConvThreads) bias_s[c] = bias[c];
+    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -239,7 +256,13 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                         float f[8];
 #pragma unroll
                         for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[j + e]);
-                        if (bias) {
+                        if (fold) {
+                            const float4 s0 = *(const float4 *)(scale_s + n0 + c0 + j);
+                            const float4 s1 = *(const float4 *)(scale_s + n0 + c0 + j + 4);
+                            f[0] *= s0.x; f[1] *= s0.y; f[2] *= s0.z; f[3] *= s0.w;
+                            f[4] *= s1.x; f[5] *= s1.y; f[6] *= s1.z; f[7] *= s1.w;
+                        }
+                        if (bias || fold) {
                             const float4 b0 = *(const float4 *)(bias_s + n0 + c0 + j);
                             const float4 b1 = *(const float4 *)(bias_s + n0 + c0 + j + 4);
                             f[0] += b0.x; f[1] += b0.y; f[2] += b0.z; f[3] += b0.w;
@@ -359,7 +382,7 @@ template <int BN>
 static cudaError_t launch_bn(const CUtensorMap &ta, const CUtensorMap &tw, const CUtensorMap &tout, ConvGemm g,
                              const float *bias, int *err, cudaStream_t st) {
     constexpr size_t stage = (size_t)kBM * kBK * 2 + (size_t)BN * kBK * 2;
-    const size_t fixed = 1024 + kStagingBytes + sizeof(ConvSmemCtl) + (size_t)g.cn * sizeof(float) + 16;
+    const size_t fixed = 1024 + kStagingBytes + sizeof(ConvSmemCtl) + 2 * (size_t)g.cn * sizeof(float) + 16;
     int stages = (int)((220 * 1024 - fixed) / stage);  // one CTA per SM owns the shared memory
     if (stages > kMaxStages) stages = kMaxStages;
     g.stages = stages;
@@ -395,12 +418,13 @@ static int pick_bn(long long tiles_m, int cn) {
 }
 
 cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void *wmat, const float *bias,
-                             void *out, cudaStream_t st) {
+                             void *out, cudaStream_t st, const BnFold *fold) {
     ConvGemm g;
     g.ho = s.ho; g.wo = s.wo; g.cn = s.cn; g.ca = s.ca; g.taps_h = s.taps_h; g.taps_w = s.taps_w;
     g.lower_h = s.lower_h; g.lower_w = s.lower_w; g.stride_h = s.stride_h; g.stride_w = s.stride_w;
     g.dil_h = s.dil_h; g.dil_w = s.dil_w; g.p = (long long)s.n * s.ho * s.wo; g.stages = 1;
     g.blockdiag = s.blockdiag;
+    g.fold = fold ? *fold : BnFold{nullptr, nullptr, nullptr, nullptr, nullptr, 0.f, nullptr};
     g.out_strided = s.out_sw ? (__nv_bfloat16 *)out : nullptr;
     g.out_sn = s.out_sn; g.out_sh = s.out_sh; g.out_sw = s.out_sw;
     // The bounding box of base pixels has ho x wo positions: upper = lower + (out-1) stride - (in-1).

@@ -234,7 +234,8 @@ UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
     per = (per + kWP - 1) / kWP * kWP;
     pl.per_split = per;
     pl.splits = (int)((pb.p + per - 1) / per);
-    pl.kt = (pb.kdim + 7) / 8;        // epilogue blocks along k (8 rows each) = rows of dotpart
+    pl.kr = pl.splits > 16 ? 2 : 8;   // k rows per epilogue block
+    pl.kt = (pb.kdim + pl.kr - 1) / pl.kr;   // epilogue blocks along k = rows of dotpart
     return pl;
 }
 
@@ -288,7 +289,8 @@ cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
 
 // ---- epilogue over k-major partials ------------------------------------------------------------
 // One kernel finishes every parameter gradient (Table 2, Tune row) from the fp32 partial tiles:
-//   block (bx, by): 32 output channels x 8 k rows, 4 lanes over the pixel slices (1024 threads)
+//   block (bx, by): 32 output channels x KR k rows x SL lanes over the pixel slices (KR SL = 32,
+//   1024 threads): (8, 4) when there are few slices, (2, 16) when there are many
 //     acc[k][co] = sum_split part[split][k][co]        (each lane a strided subset, lanes added in order)
 //     dw[co][k]  = s[co] acc                           (transposed through shared memory)
 //     dotpart[by][co] = sum over the block's k rows of acc * w[co][k]
@@ -297,16 +299,18 @@ cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
 //   tree, so the result does not depend on which block came last:
 //     dbeta = sum dZ,  db = s dbeta,  dgamma = r (sum_k domega' omega + dbeta (b - mu_hat))
 //   plain mode (vec3 == NULL): dw = acc, db = sum dZ if requested.
+template <int KR, int SL>
 __global__ void __launch_bounds__(1024) wgrad_epilogue_fused_kernel(
     int c_out, int kdim, const float *__restrict__ part, int splits, const float *__restrict__ bsum, int bsplits,
     const __nv_bfloat16 *__restrict__ w, const float *__restrict__ vec3, const float *__restrict__ b,
     const float *__restrict__ mean, float *__restrict__ dw, float *__restrict__ dotpart,
     unsigned int *__restrict__ counters, float *__restrict__ db, float *__restrict__ dgamma,
     float *__restrict__ dbeta, int need_sums) {
-    __shared__ float tile[4][8][33];
+    static_assert(KR * SL == 32, "one block is 32 x 32 threads");
+    __shared__ float tile[SL][KR][33];
     __shared__ int is_last;
-    const int tx = threadIdx.x & 31, ty = (threadIdx.x >> 5) & 7, tz = threadIdx.x >> 8;
-    const int co0 = blockIdx.x * 32, k0 = blockIdx.y * 8;
+    const int tx = threadIdx.x & 31, ty = (threadIdx.x >> 5) % KR, tz = (threadIdx.x >> 5) / KR;
+    const int co0 = blockIdx.x * 32, k0 = blockIdx.y * KR;
     const size_t slice = (size_t)kdim * c_out;
     {
         const int k = k0 + ty;
@@ -314,28 +318,29 @@ __global__ void __launch_bounds__(1024) wgrad_epilogue_fused_kernel(
         if (k < kdim) {
             const float *src = part + (size_t)k * c_out + co0 + tx;
             int sp = tz;
-            for (; sp + 4 < splits; sp += 8) {
+            for (; sp + SL < splits; sp += 2 * SL) {
                 a0 += src[(size_t)sp * slice];
-                a1 += src[(size_t)(sp + 4) * slice];
+                a1 += src[(size_t)(sp + SL) * slice];
             }
             if (sp < splits) a0 += src[(size_t)sp * slice];
         }
         tile[tz][ty][tx] = a0 + a1;
     }
     __syncthreads();
-    if (threadIdx.x < 256) {
-        const int kk = threadIdx.x & 7, cl = threadIdx.x >> 3, k = k0 + kk, co = co0 + cl;
+    if (threadIdx.x < 32 * KR) {
+        const int kk = threadIdx.x % KR, cl = threadIdx.x / KR, k = k0 + kk, co = co0 + cl;
         float d = 0.f;
         if (k < kdim) {
-            const float v = (tile[0][kk][cl] + tile[1][kk][cl]) + (tile[2][kk][cl] + tile[3][kk][cl]);
+            float v = 0.f;
+#pragma unroll
+            for (int z = 0; z < SL; ++z) v += tile[z][kk][cl];
             const size_t o = (size_t)co * kdim + k;
             dw[o] = (vec3 ? vec3[co] : 1.f) * v;
             if (vec3) d = v * __bfloat162float(w[o]);
         }
         if (vec3) {
-            d += __shfl_xor_sync(0xffffffffu, d, 1);
-            d += __shfl_xor_sync(0xffffffffu, d, 2);
-            d += __shfl_xor_sync(0xffffffffu, d, 4);
+#pragma unroll
+            for (int o = 1; o < KR; o <<= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
             if (kk == 0) dotpart[(size_t)blockIdx.y * c_out + co] = d;
         }
     }
@@ -377,10 +382,14 @@ cudaError_t launch_wgrad_epilogue_fused(const Problem &pb, const UmmaWgradPlan &
                                         const float *bsum, const void *w, const float *vec3, const float *b,
                                         const float *mean, float *dw, float *dotpart, unsigned int *counters,
                                         float *db, float *dgamma, float *dbeta, bool need_sums, cudaStream_t st) {
-    dim3 grid(pb.c_out / 32, pl.kt);
-    wgrad_epilogue_fused_kernel<<<grid, 1024, 0, st>>>(pb.c_out, pb.kdim, partials, pl.splits, bsum, pl.splits,
-                                                       (const __nv_bfloat16 *)w, vec3, b, mean, dw, dotpart, counters,
-                                                       db, dgamma, dbeta, need_sums ? 1 : 0);
+    if (pl.kr == 8)
+        wgrad_epilogue_fused_kernel<8, 4><<<dim3(pb.c_out / 32, pl.kt), 1024, 0, st>>>(
+            pb.c_out, pb.kdim, partials, pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw,
+            dotpart, counters, db, dgamma, dbeta, need_sums ? 1 : 0);
+    else
+        wgrad_epilogue_fused_kernel<2, 16><<<dim3(pb.c_out / 32, pl.kt), 1024, 0, st>>>(
+            pb.c_out, pb.kdim, partials, pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw,
+            dotpart, counters, db, dgamma, dbeta, need_sums ? 1 : 0);
     return cudaGetLastError();
 }
 
