@@ -234,7 +234,7 @@ UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
     per = (per + kWP - 1) / kWP * kWP;
     pl.per_split = per;
     pl.splits = (int)((pb.p + per - 1) / per);
-    pl.kr = pl.splits > 16 ? 2 : 8;   // k rows per epilogue block
+    pl.kr = pl.splits > 64 ? 2 : 8;   // k rows per epilogue block
     pl.kt = (pb.kdim + pl.kr - 1) / pl.kr;   // epilogue blocks along k = rows of dotpart
     return pl;
 }
