@@ -224,23 +224,59 @@ def run_ours(args):
     sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    C.convbn_profile_begin()
+
+    def max_over_ranks(v):
+        if world > 1:
+            t = torch.tensor([v], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+        return v
+
+    # ---- timed region: K steps, each a replay of the CUDA graph of one step (one graph per buffer
+    # set), so the layers' ~15 launches per step cost no host time; --no-graph times eager calls.
+    graphs, launch_mode = None, "eager library calls"
+    if not args.no_graph:
+        try:
+            graphs = []
+            for si in range(sets):
+                gr = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gr):
+                    for b in blocks[si]:
+                        b.tune_step()
+                graphs.append(gr)
+            for gr in graphs:
+                gr.replay()
+            torch.cuda.synchronize()
+            launch_mode = "CUDA graph replay (one captured step per buffer set)"
+        except Exception as exc:  # capture unsupported: say so and time eager calls
+            graphs, launch_mode = None, "eager library calls (graph capture failed: %r)" % (exc,)
     barrier()
     e0.record(stream)
     for i in range(args.steps):
-        step(args.warmup + i)
+        if graphs:
+            graphs[(args.warmup + i) % sets].replay()
+        else:
+            step(args.warmup + i)
     e1.record(stream)
     barrier()
+    ms = max_over_ranks(e0.elapsed_time(e1))
+    value = world * step_flops * args.steps / (ms * 1e-3) / 1e12
+
+    # ---- second pass, same K steps as eager calls with a CUDA-event pair around every kernel: the
+    # per-kernel durations behind the roofline object (events cannot be read back out of a graph)
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    C.convbn_profile_begin()
+    barrier()
+    f0.record(stream)
+    for i in range(args.steps):
+        step(args.warmup + i)
+    f1.record(stream)
+    barrier()
     prof = C.convbn_profile_end()
+    eager_ms = max_over_ranks(f0.elapsed_time(f1))
     sampler.stop_flag.set()
     sampler.join()
     C.convbn_check()
-    ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * step_flops * args.steps / (ms * 1e-3) / 1e12
 
     # ---- roofline of the dominant kernel -----------------------------------------------------
     peaks, peak_src = load_peaks()
@@ -303,7 +339,11 @@ def run_ours(args):
                            "layers": [b.spec.name for b in blocks[0]],
                            "l2": "step footprint %.0f MB of activations > L2; %d rotating buffer sets"
                                  % (footprint / 1e6, sets),
-                           "flops_per_step": step_flops, "parallelism": "replicas x%d" % world},
+                           "flops_per_step": step_flops, "parallelism": "replicas x%d" % world,
+                           "launch": launch_mode},
+                "eager": {"ms_per_step": eager_ms / args.steps,
+                          "value": world * step_flops * args.steps / (eager_ms * 1e-3) / 1e12,
+                          "note": "same steps as plain library calls with per-kernel CUDA events (source of `kernels` and `roofline`)"},
                 "clocks": sampler.summary(), "e2e": e2e,
                 "gpu_launches": sum(k["launches"] for k in kernels),
                 "roofline": roofline, "cpu_baseline": cpu, "kernels": kernels[:12],
@@ -367,6 +407,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--ref-batch", type=int, default=4, help="samples per step of the reference arm")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="time eager library calls instead of graph replays")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":

@@ -6,8 +6,22 @@ namespace convbn {
 
 __device__ int g_error_word = 0;
 
+// The address is looked up once per device and cached, so launches make no runtime query
+// (which also keeps them legal while a stream is being captured, after one warm-up call).
 cudaError_t error_word_address(int **dev_ptr) {
-    return cudaGetSymbolAddress((void **)dev_ptr, g_error_word);
+    static int *cache[64] = {nullptr};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaGetSymbolAddress((void **)dev_ptr, g_error_word);
+    if (!cache[dev]) {
+        int *p = nullptr;
+        e = cudaGetSymbolAddress((void **)&p, g_error_word);
+        if (e != cudaSuccess) return e;
+        cache[dev] = p;
+    }
+    *dev_ptr = cache[dev];
+    return cudaSuccess;
 }
 
 cudaError_t read_and_clear_error_word(int *host_value) {
