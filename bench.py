@@ -62,6 +62,12 @@ def kernel_bytes(kind, spec, out_hw):
     raise KeyError(kind)
 
 
+# DRAM bytes (read + write) per launch from the ncu capture summarised in
+# profiles/config1_gemm_kernels_ncu_full.md; None for kernels changed or not captured since.
+NCU_TRAFFIC = {("umma_fwd", "c1a"): 51.84e6, ("umma_dgrad", "c1a"): 13.66e6, ("umma_wgrad", "c1a"): 65.16e6,
+               ("umma_fwd", "c1b"): 12.97e6, ("umma_dgrad", "c1b"): 12.97e6, ("umma_wgrad", "c1b"): 25.71e6,
+               ("umma_fwd", "c1c"): 13.77e6, ("umma_dgrad", "c1c"): 52.17e6, ("umma_wgrad", "c1c"): 65.37e6}
+
 KIND_OF = {"direct_fwd": "fwd", "direct_dgrad": "dgrad", "direct_wgrad": "wgrad",
            "umma_fwd": "fwd", "umma_dgrad": "dgrad", "umma_wgrad": "wgrad",
            "dw_fwd": "fwd", "dw_dgrad": "dgrad", "dw_wgrad": "wgrad",
@@ -77,7 +83,7 @@ def shape_tag(spec):
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons of one GPU through NVML (read-only) while running."""
 
-    def __init__(self, uuid, period=0.05):
+    def __init__(self, uuid, period=0.01):
         super().__init__(daemon=True)
         self.period, self.stop_flag = period, threading.Event()
         self.sm, self.reasons, self.sm_max, self.ok = [], set(), None, False
@@ -305,12 +311,13 @@ def run_ours(args):
             if tensor_bound:
                 ach = fl / dur / 1e12
                 roofline = {"bound": "tensor", "achieved": ach, "peak": tc, "unit": "TFLOP/s",
-                            "frac": ach / tc, "traffic": None,
+                            "frac": ach / tc, "traffic": NCU_TRAFFIC.get((top["kernel"], top["layer"])),
                             "peak_source": peak_src + " bf16 sustained (kernel timed inside a long step)"}
             else:
                 ach = by / dur / 1e9
                 roofline = {"bound": "hbm", "achieved": ach, "peak": hbm, "unit": "GB/s",
-                            "frac": ach / hbm, "traffic": None, "peak_source": peak_src + " copy bandwidth"}
+                            "frac": ach / hbm, "traffic": NCU_TRAFFIC.get((top["kernel"], top["layer"])),
+                            "peak_source": peak_src + " copy bandwidth"}
             roofline.update({"kernel": top["kernel"], "layer": top["layer"], "us_per_launch": dur * 1e6,
                              "algorithmic_bytes": by, "algorithmic_flops": fl, "share_of_step": top["share"]})
     for k in kernels:
@@ -399,8 +406,8 @@ def run_e2e(args, torch, C, blks, dev, stream, world, step_flops):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=1, choices=sorted(WORKLOAD_NAMES))
     ap.add_argument("--buffer-sets", type=int, default=2)
