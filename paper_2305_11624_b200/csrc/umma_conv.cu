@@ -42,6 +42,7 @@ struct ConvGemm {
     __nv_bfloat16 *out_strided;
     long long out_sn;
     int out_sh, out_sw;
+    int resident;            // 1: the CTA's whole weight slab [BN][K] stays in shared memory (loaded once)
     BnFold fold;             // fold.gamma != NULL: scale and shift formed in the kernel from the BN parameters
 };
 
@@ -50,6 +51,7 @@ struct ConvSmemCtl {
     uint64_t empty[kMaxStages];
     uint64_t tmem_full[2];     // MMA issuer -> epilogue, one per accumulator buffer
     uint64_t tmem_empty[2];    // epilogue -> MMA issuer (4 arrivals: one per epilogue warp)
+    uint64_t bfull;            // resident weight slab has landed
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -65,24 +67,43 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                                                                 const ConvGemm g, const float *__restrict__ bias,
                                                                 int *err) {
     extern __shared__ uint8_t smem_raw[];
-    constexpr uint32_t kABytes = kBM * kBK * 2, kBBytes = BN * kBK * 2, kStageBytes = kABytes + kBBytes;
+    constexpr uint32_t kABytes = kBM * kBK * 2, kBBytes = BN * kBK * 2;
+    const int cchunks = g.blockdiag ? 1 : g.ca / kBK;
+    const int num_kb = g.taps_h * g.taps_w * cchunks;
+    // Ring slots hold the activation tile and, unless the weights are resident, the weight tile.
+    const uint32_t kStageBytes = g.resident ? kABytes : kABytes + kBBytes;
     uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t *staging = tiles + (size_t)g.stages * kStageBytes;         // 4 warps x 2 x [32 rows][128 B]
+    uint8_t *slab = tiles + (size_t)g.stages * kStageBytes;            // resident weights: num_kb x [BN][64]
+    uint8_t *staging = slab + (g.resident ? (size_t)num_kb * kBBytes : 0);   // 8 warps x 2 x [32 rows][128 B]
     ConvSmemCtl *ctl = (ConvSmemCtl *)(staging + kStagingBytes);
     float *bias_s = (float *)(((uintptr_t)(ctl + 1) + 15) & ~(uintptr_t)15);   // cn floats
     float *scale_s = bias_s + g.cn;                                            // cn floats (fold mode)
     const bool fold = g.fold.gamma != nullptr;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int stages = g.stages;
-    const int cchunks = g.blockdiag ? 1 : g.ca / kBK;
-    const int num_kb = g.taps_h * g.taps_w * cchunks;
-    const int n_tiles = (g.cn + BN - 1) / BN;
-    const long long total_tiles = ((g.p + kBM - 1) / kBM) * n_tiles;
+    const uint32_t n_tiles = (uint32_t)(g.cn + BN - 1) / BN;
+    const uint32_t m_tiles = (uint32_t)((g.p + kBM - 1) / kBM);
+    const uint32_t total_tiles = m_tiles * n_tiles;
+    // Tile i of this CTA.  Resident weights: the CTA keeps one n-tile (blockIdx.x % n_tiles) and walks
+    // m-tiles; otherwise tiles are dealt round-robin with the n-tiles of an m-tile on neighbouring CTAs.
+    auto tile_of = [&](uint32_t i, uint32_t &mt, uint32_t &nt) -> bool {
+        if (g.resident) {
+            nt = blockIdx.x % n_tiles;
+            mt = blockIdx.x / n_tiles + i * (gridDim.x / n_tiles);
+            return mt < m_tiles;
+        }
+        const uint32_t t = blockIdx.x + i * gridDim.x;
+        if (t >= total_tiles) return false;
+        mt = t / n_tiles;
+        nt = t - mt * n_tiles;
+        return true;
+    };
     volatile int *abort_flag = &ctl->abort_flag;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tmem_full[a], 1); mbar_init(&ctl->tmem_empty[a], 4); }
+        mbar_init(&ctl->bfull, 1);
         ctl->abort_flag = 0;
         fence_barrier_init();
     }
@@ -120,11 +141,16 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
         int s = 0;                               // ring slot and its phase, advanced incrementally
         uint32_t ph = 0;
         bool ok = true;
-        for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        if (g.resident && lane == 1) {
+            const int n0 = (int)(blockIdx.x % n_tiles) * BN;
+            mbar_arrive_expect_tx(&ctl->bfull, (uint32_t)num_kb * kBBytes);
+            for (int kb = 0; kb < num_kb; ++kb) tma_load_2d(slab + (size_t)kb * kBBytes, &tm_w, &ctl->bfull, kb * kBK, n0);
+        }
+        uint32_t mt, nt;
+        for (uint32_t i = 0; ok && tile_of(i, mt, nt); ++i) {
             // 32-bit arithmetic: 64-bit divisions would cost about a microsecond per tile here
-            const uint32_t tt = (uint32_t)t, mt = tt / (uint32_t)n_tiles;
             const uint32_t m0 = mt * kBM;
-            const int n0 = (int)(tt - mt * (uint32_t)n_tiles) * BN;
+            const int n0 = (int)nt * BN;
             const uint32_t tq = m0 / (uint32_t)g.wo;
             const int wo0 = (int)(m0 - tq * (uint32_t)g.wo);
             const uint32_t img = tq / (uint32_t)g.ho;
@@ -136,10 +162,10 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                 if (!ok) break;
                 uint8_t *a_dst = tiles + (size_t)s * kStageBytes, *b_dst = a_dst + kABytes;
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(&ctl->full[s], kStageBytes);
+                    mbar_arrive_expect_tx(&ctl->full[s], kStageBytes);   // (activation + weight tile) or activation only
                     tma_load_im2col_4d(a_dst, &tm_act, &ctl->full[s], (g.blockdiag ? n0 : 0) + cc * kBK, base_w, base_h, img0,
                                        (uint16_t)(q * g.dil_w), (uint16_t)(r * g.dil_h));
-                } else if (lane == 1) {
+                } else if (lane == 1 && !g.resident) {
                     tma_load_2d(b_dst, &tm_w, &ctl->full[s], kb * kBK, n0);
                 }
                 if (++cc == cchunks) { cc = 0; if (++q == g.taps_w) { q = 0; ++r; } }
@@ -160,9 +186,13 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
             constexpr uint32_t idesc = idesc_bf16_f32(kBM, BN, 0, 0);
             int s = 0;
             uint32_t ph = 0;
-            uint32_t i = 0;
             bool ok = true;
-            for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++i) {
+            if (g.resident) {
+                ok = mbar_wait_bounded(&ctl->bfull, 0, abort_flag);
+                tc_fence_after_sync();
+            }
+            uint32_t mt, nt;
+            for (uint32_t i = 0; ok && tile_of(i, mt, nt); ++i) {
                 const uint32_t acc = i & 1u;
                 if (!mbar_wait_bounded(&ctl->tmem_empty[acc], ((i >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after_sync();
@@ -170,7 +200,8 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait_bounded(&ctl->full[s], ph, abort_flag)) { ok = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t a_addr = smem_u32(tiles + (size_t)s * kStageBytes), b_addr = a_addr + kABytes;
+                    const uint32_t a_addr = smem_u32(tiles + (size_t)s * kStageBytes);
+                    const uint32_t b_addr = g.resident ? smem_u32(slab + (size_t)kb * kBBytes) : a_addr + kABytes;
 #pragma unroll
                     for (int k = 0; k < kBK / kUmmaK; ++k) {
                         const uint64_t ad = smem_desc_sw128(a_addr + k * kUmmaK * 2, 16, 1024);
@@ -192,8 +223,8 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
         const int quarter = warp & 3;                      // tensor-memory lanes this warp may read
         const uint32_t egroup = (uint32_t)(warp - 2) >> 2; // 0: warps 2-5, 1: warps 6-9
         uint8_t *stage_buf = staging + (size_t)(warp - 2) * 2 * kStagingWarpBytes;
-        uint32_t i = egroup, sbuf = 0;
-        for (long long t = blockIdx.x + (long long)egroup * gridDim.x; t < total_tiles; t += 2LL * gridDim.x, i += 2) {
+        uint32_t sbuf = 0, mt, nt;
+        for (uint32_t i = egroup; tile_of(i, mt, nt); i += 2) {
             const uint32_t acc = egroup;
             const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->tmem_full[acc], (i >> 1) & 1u, abort_flag));
             if (!ok) {
@@ -201,9 +232,8 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                 break;
             }
             tc_fence_after_sync();
-            const uint32_t tt = (uint32_t)t, mt = tt / (uint32_t)n_tiles;
             const uint32_t m0 = mt * kBM;
-            const int n0 = (int)(tt - mt * (uint32_t)n_tiles) * BN;
+            const int n0 = (int)nt * BN;
             const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
             int ncols = g.cn - n0;                          // valid columns of this tile
             if (ncols > BN) ncols = BN;
@@ -381,8 +411,22 @@ static int sm_count() {
 template <int BN>
 static cudaError_t launch_bn(const CUtensorMap &ta, const CUtensorMap &tw, const CUtensorMap &tout, ConvGemm g,
                              const float *bias, int *err, cudaStream_t st) {
-    constexpr size_t stage = (size_t)kBM * kBK * 2 + (size_t)BN * kBK * 2;
-    const size_t fixed = 1024 + kStagingBytes + sizeof(ConvSmemCtl) + 2 * (size_t)g.cn * sizeof(float) + 16;
+    const size_t a_bytes = (size_t)kBM * kBK * 2, b_bytes = (size_t)BN * kBK * 2;
+    size_t fixed = 1024 + kStagingBytes + sizeof(ConvSmemCtl) + 2 * (size_t)g.cn * sizeof(float) + 16;
+    const int num_kb = g.taps_h * g.taps_w * (g.blockdiag ? 1 : g.ca / kBK);
+    const long long m_tiles = (g.p + kBM - 1) / kBM, n_tiles = (g.cn + BN - 1) / BN;
+    long long grid_l = m_tiles * n_tiles < sm_count() ? m_tiles * n_tiles : sm_count();
+    // Weights stay resident when the CTA's slab fits beside at least four activation slots and the
+    // grid can give every CTA one fixed n-tile.
+    const size_t slab = (size_t)num_kb * b_bytes;
+    g.resident = 0;
+    if (slab <= 104 * 1024 && fixed + slab + 4 * a_bytes <= 220 * 1024 && m_tiles * n_tiles >= sm_count() &&
+        n_tiles <= sm_count()) {
+        g.resident = 1;
+        grid_l = sm_count() - sm_count() % n_tiles;
+        fixed += slab;
+    }
+    const size_t stage = g.resident ? a_bytes : a_bytes + b_bytes;
     int stages = (int)((220 * 1024 - fixed) / stage);  // one CTA per SM owns the shared memory
     if (stages > kMaxStages) stages = kMaxStages;
     g.stages = stages;
@@ -394,8 +438,7 @@ static cudaError_t launch_bn(const CUtensorMap &ta, const CUtensorMap &tw, const
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    const long long total = ((g.p + kBM - 1) / kBM) * ((g.cn + BN - 1) / BN);
-    const unsigned grid = (unsigned)(total < sm_count() ? total : sm_count());
+    const unsigned grid = (unsigned)grid_l;
     umma_conv_kernel<BN><<<grid, kConvThreads, smem, st>>>(ta, tw, tout, g, bias, err);
     return cudaGetLastError();
 }
