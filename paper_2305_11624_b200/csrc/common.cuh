@@ -59,6 +59,32 @@ enum : int { ERRW_TIMEOUT = 1 };
 cudaError_t error_word_address(int **dev_ptr);          // address on the current device
 cudaError_t read_and_clear_error_word(int *host_value); // synchronous
 
+// ---- programmatic dependent launch -------------------------------------------------------------
+// Kernels launched through launch_pdl may start while the kernel before them in the stream is still
+// running: their set-up (barriers, tensor memory, descriptor prefetch) then overlaps its tail.  They
+// call pdl_wait() before their first access to global memory, which returns only once every earlier
+// kernel has completed and flushed; launched the plain way, pdl_wait() returns at once.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+bool pdl_enabled();   // false when CONVBN_NO_PDL=1
+
+template <class... KArgs, class... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl_enabled() ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 static inline int ceil_div_i(long long a, long long b) { return (int)((a + b - 1) / b); }
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 

@@ -1,10 +1,17 @@
 // Per-channel and elementwise kernels: on-the-fly reparameterisation (omega', b'), per-channel
 // sums, the parameter-gradient epilogue of Tune mode, and the Eval-mode BatchNorm passes.
+#include <stdlib.h>
+
 #include "kernels.h"
 
 namespace convbn {
 
 __device__ int g_error_word = 0;
+
+bool pdl_enabled() {
+    static const bool v = [] { const char *e = getenv("CONVBN_NO_PDL"); return !(e && e[0] == '1'); }();
+    return v;
+}
 
 // The address is looked up once per device and cached, so launches make no runtime query
 // (which also keeps them legal while a stream is being captured, after one warm-up call).
@@ -114,6 +121,8 @@ __global__ void __launch_bounds__(256) reparam_dgrad_kernel(int c_out, int c_in,
                                                             const float *__restrict__ s_vec,
                                                             __nv_bfloat16 *__restrict__ w_t) {
     __shared__ float tile[32][33];
+    pdl_wait();
+    pdl_launch_dependents();
     const int tap = blockIdx.z, co0 = blockIdx.y * 32, ci0 = blockIdx.x * 32;
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
     for (int j = ty; j < 32; j += 8) {
@@ -135,6 +144,8 @@ __global__ void __launch_bounds__(256) reparam_dgrad_class_kernel(int c_out, int
                                                                   const float *__restrict__ s_vec,
                                                                   __nv_bfloat16 *__restrict__ w_t, int taps) {
     __shared__ float tile[32][33];
+    pdl_wait();
+    pdl_launch_dependents();
     const int ct = blockIdx.z, mh = ct / tw, mw = ct - mh * tw;
     const int tap = (r_max - step_h * mh) * kw + (q_max - step_w * mw);
     const int co0 = blockIdx.y * 32, ci0 = blockIdx.x * 32;
@@ -155,18 +166,15 @@ __global__ void __launch_bounds__(256) reparam_dgrad_class_kernel(int c_out, int
 cudaError_t launch_reparam_dgrad_class(const Problem &pb, const void *w, const float *s_vec, void *w_t, int th,
                                        int tw, int r_max, int q_max, int step_h, int step_w, cudaStream_t st) {
     dim3 grid((pb.c_in + 31) / 32, (pb.c_out + 31) / 32, th * tw);
-    reparam_dgrad_class_kernel<<<grid, 256, 0, st>>>(pb.c_out, pb.c_in, pb.kw, tw, r_max, q_max, step_h, step_w,
-                                                     th * tw, (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t,
-                                                     pb.kh * pb.kw);
-    return cudaGetLastError();
+    return launch_pdl(reparam_dgrad_class_kernel, grid, dim3(256), 0, st, pb.c_out, pb.c_in, pb.kw, tw, r_max, q_max,
+                      step_h, step_w, th * tw, (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t, pb.kh * pb.kw);
 }
 
 cudaError_t launch_reparam_dgrad(const Problem &pb, const void *w, const float *s_vec, void *w_t,
                                  cudaStream_t st) {
     dim3 grid((pb.c_in + 31) / 32, (pb.c_out + 31) / 32, pb.kh * pb.kw);
-    reparam_dgrad_kernel<<<grid, 256, 0, st>>>(pb.c_out, pb.c_in, pb.kh * pb.kw, (const __nv_bfloat16 *)w, s_vec,
-                                               (__nv_bfloat16 *)w_t);
-    return cudaGetLastError();
+    return launch_pdl(reparam_dgrad_kernel, grid, dim3(256), 0, st, pb.c_out, pb.c_in, pb.kh * pb.kw,
+                      (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t);
 }
 
 // ---- per-channel partial sums over pixel slices (Appendix B) --------------------------------

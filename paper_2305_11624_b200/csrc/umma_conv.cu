@@ -111,6 +111,10 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
         tmem_alloc(&ctl->tmem_base, 2 * BN);
         tmem_relinquish();
     }
+    // Everything above touched only this CTA's own shared / tensor memory.  Global memory (inputs that
+    // an earlier kernel may still be writing, outputs it may still be reading) comes after this wait.
+    pdl_wait();
+    pdl_launch_dependents();
     if (fold) {
         // On-the-fly reparameterisation (Sec. 3.3 / 3.4): s = gamma / sqrt(var + eps), b' = (b - mu) s + beta.
         // s multiplies the fp32 accumulator (the associative law of Sec. 3.2.2), so omega is used unrounded.
@@ -439,8 +443,7 @@ static cudaError_t launch_bn(const CUtensorMap &ta, const CUtensorMap &tw, const
         attr_done = true;
     }
     const unsigned grid = (unsigned)grid_l;
-    umma_conv_kernel<BN><<<grid, kConvThreads, smem, st>>>(ta, tw, tout, g, bias, err);
-    return cudaGetLastError();
+    return launch_pdl(umma_conv_kernel<BN>, dim3(grid), dim3(kConvThreads), smem, st, ta, tw, tout, g, bias, err);
 }
 
 // Tile width: fewest rounds of tiles over the SMs, weighted by the time of one tile (N = 64 tiles are

@@ -77,6 +77,8 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
         tmem_alloc(&ctl->tmem_base, BN);
         tmem_relinquish();
     }
+    pdl_wait();                 // global memory only after every earlier kernel has finished
+    pdl_launch_dependents();
     // counters of the epilogue kernel that runs after this one start from zero
     if (counters && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
         for (int i = threadIdx.x; i < ncounters; i += kWThreads) counters[i] = 0u;
@@ -259,8 +261,8 @@ static cudaError_t launch_w(const CUtensorMap &tx, const CUtensorMap &tdz, Wgrad
         attr_done = true;
     }
     dim3 grid((unsigned)((g.kdim / 64 + 2) / 2), (unsigned)((pb.c_out + BN - 1) / BN), (unsigned)pl.splits);
-    umma_wgrad_kernel<BN><<<grid, kWThreads, smem, st>>>(tx, tdz, g, partials, bsum, counters, pb.c_out / 32, err);
-    return cudaGetLastError();
+    return launch_pdl(umma_wgrad_kernel<BN>, grid, dim3(kWThreads), smem, st, tx, tdz, g, partials, bsum, counters,
+                      pb.c_out / 32, err);
 }
 
 cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const void *dz, const void *x,
@@ -309,6 +311,8 @@ __global__ void __launch_bounds__(1024) wgrad_epilogue_fused_kernel(
     static_assert(KR * SL == 32, "one block is 32 x 32 threads");
     __shared__ float tile[SL][KR][33];
     __shared__ int is_last;
+    pdl_wait();
+    pdl_launch_dependents();
     const int tx = threadIdx.x & 31, ty = (threadIdx.x >> 5) % KR, tz = (threadIdx.x >> 5) / KR;
     const int co0 = blockIdx.x * 32, k0 = blockIdx.y * KR;
     const size_t slice = (size_t)kdim * c_out;
@@ -382,15 +386,15 @@ cudaError_t launch_wgrad_epilogue_fused(const Problem &pb, const UmmaWgradPlan &
                                         const float *bsum, const void *w, const float *vec3, const float *b,
                                         const float *mean, float *dw, float *dotpart, unsigned int *counters,
                                         float *db, float *dgamma, float *dbeta, bool need_sums, cudaStream_t st) {
+    const dim3 grid(pb.c_out / 32, pl.kt);
+    const int ns = need_sums ? 1 : 0;
     if (pl.kr == 8)
-        wgrad_epilogue_fused_kernel<8, 4><<<dim3(pb.c_out / 32, pl.kt), 1024, 0, st>>>(
-            pb.c_out, pb.kdim, partials, pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw,
-            dotpart, counters, db, dgamma, dbeta, need_sums ? 1 : 0);
-    else
-        wgrad_epilogue_fused_kernel<2, 16><<<dim3(pb.c_out / 32, pl.kt), 1024, 0, st>>>(
-            pb.c_out, pb.kdim, partials, pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw,
-            dotpart, counters, db, dgamma, dbeta, need_sums ? 1 : 0);
-    return cudaGetLastError();
+        return launch_pdl(wgrad_epilogue_fused_kernel<8, 4>, grid, dim3(1024), 0, st, pb.c_out, pb.kdim, partials,
+                          pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw, dotpart, counters, db,
+                          dgamma, dbeta, ns);
+    return launch_pdl(wgrad_epilogue_fused_kernel<2, 16>, grid, dim3(1024), 0, st, pb.c_out, pb.kdim, partials,
+                      pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw, dotpart, counters, db,
+                      dgamma, dbeta, ns);
 }
 
 }  // namespace convbn
