@@ -22,10 +22,10 @@ using namespace ptx;
 constexpr int kBM = 128;       // output pixels per tile (UMMA M)
 constexpr int kBK = 64;        // K elements per stage = one 128-byte swizzle row of bf16
 constexpr int kUmmaK = 16;     // K per tcgen05.mma of kind::f16
-constexpr int kMaxStages = 8;
+constexpr int kMaxStages = 12;
 constexpr int kConvThreads = 320;                             // TMA warp, MMA warp, 2 x 4 epilogue warps
 constexpr uint32_t kStagingWarpBytes = 32 * 128;              // [32 rows][64 bf16]
-constexpr uint32_t kStagingBytes = 8 * 2 * kStagingWarpBytes; // 8 epilogue warps, double-buffered
+constexpr uint32_t kStagingBytes = 8 * kStagingWarpBytes;     // one buffer per epilogue warp
 
 struct ConvGemm {
     int ho, wo;              // output spatial extent
@@ -226,8 +226,8 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
         // private [32 rows][64 columns] staging buffers (128-byte swizzle): warp-level sync only.
         const int quarter = warp & 3;                      // tensor-memory lanes this warp may read
         const uint32_t egroup = (uint32_t)(warp - 2) >> 2; // 0: warps 2-5, 1: warps 6-9
-        uint8_t *stage_buf = staging + (size_t)(warp - 2) * 2 * kStagingWarpBytes;
-        uint32_t sbuf = 0, mt, nt;
+        uint8_t *stage_buf = staging + (size_t)(warp - 2) * kStagingWarpBytes;
+        uint32_t mt, nt;
         for (uint32_t i = egroup; tile_of(i, mt, nt); i += 2) {
             const uint32_t acc = egroup;
             const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->tmem_full[acc], (i >> 1) & 1u, abort_flag));
@@ -280,9 +280,10 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                         }
                     }
                 } else if (c0 < ncols) {
-                    uint8_t *buf = stage_buf + (size_t)sbuf * kStagingWarpBytes;
-                    // the store issued two groups ago read this buffer: wait until it no longer does
-                    if (lane == 0) tma_store_wait_read<1>();
+                    uint8_t *buf = stage_buf;
+                    // the previous store read this buffer: wait until it no longer does (shared memory
+                    // is better spent on ring slots than on a second staging buffer)
+                    if (lane == 0) tma_store_wait_read<0>();
                     __syncwarp();
                     uint8_t *row = buf + lane * 128;
 #pragma unroll
@@ -316,7 +317,6 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                         tma_store_2d(&tm_out, buf, n0 + c0, (int)(m0 + quarter * 32));
                         tma_store_commit();
                     }
-                    sbuf ^= 1u;
                 }
             }
         }
