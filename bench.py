@@ -68,7 +68,7 @@ NCU_TRAFFIC = {("umma_fwd", "c1a"): 51.84e6, ("umma_dgrad", "c1a"): 13.66e6, ("u
                ("umma_fwd", "c1b"): 12.97e6, ("umma_dgrad", "c1b"): 12.97e6, ("umma_wgrad", "c1b"): 25.71e6,
                ("umma_fwd", "c1c"): 13.77e6, ("umma_dgrad", "c1c"): 52.17e6, ("umma_wgrad", "c1c"): 65.37e6}
 
-KIND_OF = {"direct_fwd": "fwd", "direct_dgrad": "dgrad", "direct_wgrad": "wgrad",
+KIND_OF = {"strip_fwd": "fwd", "strip_dgrad": "dgrad", "direct_fwd": "fwd", "direct_dgrad": "dgrad", "direct_wgrad": "wgrad",
            "umma_fwd": "fwd", "umma_dgrad": "dgrad", "umma_wgrad": "wgrad",
            "dw_fwd": "fwd", "dw_dgrad": "dgrad", "dw_wgrad": "wgrad",
            "grouped_fwd": "fwd", "grouped_dgrad": "dgrad", "grouped_wgrad": "wgrad",

@@ -298,8 +298,13 @@ int run_conv_fwd(const convbn_desc *d, const Problem &pb, const void *x, const v
         LAUNCH("grouped_fwd", launch_umma_conv(s, x, wbd_scratch, bias, z, st));
         *which = "grouped-umma";
     } else if (umma_fwd_shape(d, pb, &s)) {
-        LAUNCH("umma_fwd", launch_umma_conv(s, x, w, bias, z, st));
-        *which = "umma";
+        if (umma_strip_eligible(s)) {
+            LAUNCH("strip_fwd", launch_umma_strip_conv(s, x, w, bias, z, st));
+            *which = "umma-strip";
+        } else {
+            LAUNCH("umma_fwd", launch_umma_conv(s, x, w, bias, z, st));
+            *which = "umma";
+        }
     } else if (dw_path(d, pb)) {
         LAUNCH("dw_fwd", launch_dw_fwd(pb, x, w, bias, z, st));
         *which = "depthwise";
@@ -358,8 +363,13 @@ int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, cons
         *which = "umma-strided";
     } else if (umma_dgrad_shape(d, pb, &s)) {
         LAUNCH("reparam_dgrad", launch_reparam_dgrad(pb, w, scale, w_scratch, st));
-        LAUNCH("umma_dgrad", launch_umma_conv(s, dz, w_scratch, nullptr, dx, st));
-        *which = "umma";
+        if (umma_strip_eligible(s)) {
+            LAUNCH("strip_dgrad", launch_umma_strip_conv(s, dz, w_scratch, nullptr, dx, st));
+            *which = "umma-strip";
+        } else {
+            LAUNCH("umma_dgrad", launch_umma_conv(s, dz, w_scratch, nullptr, dx, st));
+            *which = "umma";
+        }
     } else if (dw_path(d, pb)) {
         if (pb.stride_h == 1 && pb.stride_w == 1) {
             // dX = omega'_rot (*) dZ is itself a stride-1 depthwise convolution of dZ with the rotated
@@ -481,8 +491,13 @@ int convbn_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const
         // dense tensor-core path: s, b' and the saved vectors are formed inside the GEMM kernel and s is
         // applied to the fp32 accumulator, so one launch does the whole forward pass
         const BnFold fold{gamma, beta, run_mean, run_var, b, pb.eps, vec3};
-        LAUNCH("umma_fwd", launch_umma_conv(us, x, w, nullptr, z, st, &fold));
-        t_last_kernel[CONVBN_PHASE_TUNE_FWD] = "umma";
+        if (umma_strip_eligible(us)) {
+            LAUNCH("strip_fwd", launch_umma_strip_conv(us, x, w, nullptr, z, st, &fold));
+            t_last_kernel[CONVBN_PHASE_TUNE_FWD] = "umma-strip";
+        } else {
+            LAUNCH("umma_fwd", launch_umma_conv(us, x, w, nullptr, z, st, &fold));
+            t_last_kernel[CONVBN_PHASE_TUNE_FWD] = "umma";
+        }
         return CONVBN_OK;
     }
     LAUNCH("reparam", launch_reparam(pb, desc->dtype, desc->layout, w, b, gamma, beta, run_mean, run_var, vec3, wf,

@@ -58,6 +58,11 @@ struct BnFold {
 // fold != NULL replaces `bias` (dense output mode only).
 cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void *wmat, const float *bias,
                              void *out, cudaStream_t st, const BnFold *fold = nullptr);
+// Stride-1 multi-tap convolutions with the input patch staged once per tile (see umma_strip.cu): same
+// contract as launch_umma_conv (dense output mode, groups = 1).  Eligibility depends on the image size.
+bool umma_strip_eligible(const UmmaConvShape &s);
+cudaError_t launch_umma_strip_conv(const UmmaConvShape &s, const void *act, const void *wmat, const float *bias,
+                                   void *out, cudaStream_t st, const BnFold *fold = nullptr);
 // Weight operand of the backward-data GEMM: w_t[ci][taps-1-tap][co] = s[co] w[co][tap][ci]
 // (s_vec == NULL: unscaled).  bf16, groups = 1.
 cudaError_t launch_reparam_dgrad(const Problem &pb, const void *w, const float *s_vec, void *w_t,

@@ -89,6 +89,14 @@ __device__ __forceinline__ void tma_load_2d(void *smem_dst, const CUtensorMap *m
         ::"r"(smem_u32(smem_dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y)
         : "memory");
 }
+// Tiled 4-D box (c, w, h, n); coordinates outside the tensor read zeros (c must stay 16-byte aligned).
+__device__ __forceinline__ void tma_load_4d(void *smem_dst, const CUtensorMap *map, uint64_t *bar, int c, int w,
+                                            int h, int n) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(smem_dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(c), "r"(w), "r"(h), "r"(n)
+        : "memory");
+}
 // im2col mode over an NHWC tensor: (c, w, h, n) is the first pixel's base coordinate, (off_w, off_h)
 // the filter-tap offset added to every pixel of the column.
 __device__ __forceinline__ void tma_load_im2col_4d(void *smem_dst, const CUtensorMap *map, uint64_t *bar, int c,

@@ -1,0 +1,389 @@
+// Stride-1 k x k convolution on the sm_100a tensor cores with the input staged ONCE per tile.
+//
+// The im2col kernel (umma_conv.cu) reloads every input pixel once per filter tap; for 3x3 layers that
+// is 9x the input through L2 and the TMA ring's latency bounds the kernel.  Here a tile is R output
+// rows x CW output columns of one image.  Its (R + kh - 1) x (CW + kw - 1) input patch is loaded by
+// one tiled TMA copy per 64-channel chunk into shared memory as a flat list of pixels, 128 bytes
+// each, 128-byte swizzled.  Number the tile's outputs, halo columns included, as "virtual pixels"
+// v = i Wt + j (Wt = CW + kw - 1): tap (r, q) of virtual pixel v reads patch pixel v + r Wt + q, so the
+// A operand of tap (r, q) for 128 consecutive virtual pixels is the SAME shared memory, read from a
+// start address shifted by (r Wt + q) pixels.  All taps of a chunk are issued from one copy.
+// Junk virtual pixels (j >= CW or i >= R) are computed and dropped.
+//
+//   forward        Z  = omega' (*) X + b'   (Sec. 3.1 / 3.3)   activation X,  weights omega'
+//   backward data  dX = omega'_rot (*) dZ   (Sec. 3.2.1)       activation dZ, rotated / swapped omega'
+//
+// Warps: 0 patch loader, 1 weight-tile loader (ring), 2 MMA issuer and tensor-memory owner,
+// 3-10 epilogue (two per tensor-memory lane quarter).  Every wait is bounded.
+#include "kernels.h"
+#include "sm100_ptx.cuh"
+
+namespace convbn {
+
+using namespace ptx;
+
+constexpr int kSThreads = 352;
+constexpr int kSBStages = 4;          // weight-tile ring depth
+
+struct StripGemm {
+    int n, ho, wo, cn, ca, kh, kw, lower_h, lower_w;
+    int R, CW, Wt, rows_in, nmb;      // tile rows / columns, patch width, patch rows, M blocks of 128
+    int tiles_h, tiles_w;
+    uint32_t strip_bytes;             // one patch buffer (multiple of 1024)
+    int nacc;                         // accumulator sets in tensor memory (1 or 2)
+    uint32_t tmem_cols;
+    __nv_bfloat16 *out;
+    BnFold fold;
+};
+
+struct StripCtl {
+    uint64_t strip_full[2], strip_empty[2];
+    uint64_t b_full[kSBStages], b_empty[kSBStages];
+    uint64_t tmem_full[2], tmem_empty[2];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid_constant__ CUtensorMap tm_act,
+                                                                   const __grid_constant__ CUtensorMap tm_w,
+                                                                   const StripGemm g, const float *__restrict__ bias,
+                                                                   int *err) {
+    extern __shared__ uint8_t smem_raw[];
+    constexpr uint32_t kBBytes = BN * 64 * 2;
+    uint8_t *strips = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *bring = strips + 2 * (size_t)g.strip_bytes;
+    StripCtl *ctl = (StripCtl *)(bring + (size_t)kSBStages * kBBytes);
+    float *bias_s = (float *)(((uintptr_t)(ctl + 1) + 15) & ~(uintptr_t)15);
+    float *scale_s = bias_s + g.cn;
+    const bool fold = g.fold.gamma != nullptr;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int cchunks = g.ca / 64, taps = g.kh * g.kw;
+    const uint32_t n_tiles = (uint32_t)g.cn / BN;
+    const uint32_t sp_tiles = (uint32_t)g.n * g.tiles_h * g.tiles_w;
+    const uint32_t total_tiles = sp_tiles * n_tiles;
+    volatile int *abort_flag = &ctl->abort_flag;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&ctl->strip_full[s], 1); mbar_init(&ctl->strip_empty[s], 1);
+            mbar_init(&ctl->tmem_full[s], 1); mbar_init(&ctl->tmem_empty[s], 8);
+        }
+        for (int s = 0; s < kSBStages; ++s) { mbar_init(&ctl->b_full[s], 1); mbar_init(&ctl->b_empty[s], 1); }
+        ctl->abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 2) {
+        tmem_alloc(&ctl->tmem_base, g.tmem_cols);
+        tmem_relinquish();
+    }
+    pdl_wait();
+    pdl_launch_dependents();
+    if (fold) {
+        for (int c = threadIdx.x; c < g.cn; c += kSThreads) {
+            const float r = 1.0f / sqrtf(g.fold.var[c] + g.fold.eps);
+            const float sc = g.fold.gamma[c] * r;
+            const float bf = ((g.fold.b ? g.fold.b[c] : 0.f) - g.fold.mean[c]) * sc + g.fold.beta[c];
+            scale_s[c] = sc;
+            bias_s[c] = bf;
+            if (blockIdx.x == 0 && g.fold.vec3) {
+                g.fold.vec3[c] = sc; g.fold.vec3[g.cn + c] = bf; g.fold.vec3[2 * g.cn + c] = r;
+            }
+        }
+    } else if (bias) {
+        for (int c = threadIdx.x; c < g.cn; c += kSThreads) bias_s[c] = bias[c];
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    // tile t -> (image, tile row, tile column, n-tile); n-tiles of one patch sit on neighbouring CTAs
+    auto decode = [&](uint32_t t, int &img, int &h0, int &w0, int &n0) {
+        const uint32_t sp = t / n_tiles;
+        n0 = (int)(t - sp * n_tiles) * BN;
+        const uint32_t a = sp / (uint32_t)g.tiles_w;
+        w0 = (int)(sp - a * (uint32_t)g.tiles_w) * g.CW;
+        const uint32_t b = a / (uint32_t)g.tiles_h;
+        h0 = (int)(a - b * (uint32_t)g.tiles_h) * g.R;
+        img = (int)b;
+    };
+
+    if (warp == 0) {
+        // ---------------- patch loader: one TMA copy per (tile, channel chunk) ----------------
+        if (elect_one()) {
+            prefetch_tensormap(&tm_act);
+            int sb = 0;
+            uint32_t ph = 0;
+            const uint32_t bytes = (uint32_t)g.rows_in * g.Wt * 128u;
+            bool ok = true;
+            for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                int img, h0, w0, n0;
+                decode(t, img, h0, w0, n0);
+                for (int cc = 0; cc < cchunks; ++cc) {
+                    if (!mbar_wait_bounded(&ctl->strip_empty[sb], ph ^ 1u, abort_flag)) { ok = false; break; }
+                    mbar_arrive_expect_tx(&ctl->strip_full[sb], bytes);
+                    tma_load_4d(strips + (size_t)sb * g.strip_bytes, &tm_act, &ctl->strip_full[sb], cc * 64,
+                                w0 + g.lower_w, h0 + g.lower_h, img);
+                    if (++sb == 2) { sb = 0; ph ^= 1u; }
+                }
+            }
+            if (!ok) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+            // an issued copy always completes; give the last ones time to land before the CTA can exit
+            if (!ok) for (int s = 0; s < 2; ++s) mbar_wait_bounded(&ctl->strip_full[s], 0, nullptr, 2000000ull);
+        }
+    } else if (warp == 1) {
+        // ---------------- weight-tile loader ----------------
+        if (elect_one()) {
+            prefetch_tensormap(&tm_w);
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                const int n0 = (int)(t % n_tiles) * BN;
+                for (int cc = 0; cc < cchunks && ok; ++cc)
+                    for (int tap = 0; tap < taps; ++tap) {
+                        if (!mbar_wait_bounded(&ctl->b_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+                        mbar_arrive_expect_tx(&ctl->b_full[s], kBBytes);
+                        tma_load_2d(bring + (size_t)s * kBBytes, &tm_w, &ctl->b_full[s], tap * g.ca + cc * 64, n0);
+                        if (++s == kSBStages) { s = 0; ph ^= 1u; }
+                    }
+            }
+            if (!ok) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+            if (!ok) for (int q = 0; q < kSBStages; ++q) mbar_wait_bounded(&ctl->b_full[q], 0, nullptr, 2000000ull);
+        }
+    } else if (warp == 2) {
+        // ---------------- MMA issuer ----------------
+        if (elect_one()) {
+            constexpr uint32_t idesc = idesc_bf16_f32(128, BN, 0, 0);
+            int sb = 0, s = 0;
+            uint32_t sph = 0, bph = 0, i = 0;
+            bool ok = true;
+            for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++i) {
+                const uint32_t a = i % (uint32_t)g.nacc, use = i / (uint32_t)g.nacc;
+                if (!mbar_wait_bounded(&ctl->tmem_empty[a], (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d0 = tmem_base + a * (uint32_t)(g.nmb * BN);
+                for (int cc = 0; cc < cchunks && ok; ++cc) {
+                    if (!mbar_wait_bounded(&ctl->strip_full[sb], sph, abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t patch = smem_u32(strips + (size_t)sb * g.strip_bytes);
+                    int r = 0, q = 0;
+                    for (int tap = 0; tap < taps; ++tap) {
+                        if (!mbar_wait_bounded(&ctl->b_full[s], bph, abort_flag)) { ok = false; break; }
+                        tc_fence_after_sync();
+                        const uint32_t b_addr = smem_u32(bring + (size_t)s * kBBytes);
+                        const uint32_t shift = (uint32_t)(r * g.Wt + q) * 128u;
+                        for (int mb = 0; mb < g.nmb; ++mb) {
+                            const uint32_t a_addr = patch + (uint32_t)mb * (128u * 128u) + shift;
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                umma_bf16_ss(d0 + (uint32_t)(mb * BN), smem_desc_sw128(a_addr + k * 32, 16, 1024),
+                                             smem_desc_sw128(b_addr + k * 32, 16, 1024), idesc,
+                                             (cc | tap | k) ? 1u : 0u);
+                        }
+                        umma_commit(&ctl->b_empty[s]);
+                        if (++s == kSBStages) { s = 0; bph ^= 1u; }
+                        if (++q == g.kw) { q = 0; ++r; }
+                    }
+                    if (ok) umma_commit(&ctl->strip_empty[sb]);
+                    if (++sb == 2) { sb = 0; sph ^= 1u; }
+                }
+                if (ok) umma_commit(&ctl->tmem_full[a]);
+            }
+            if (!ok) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+        }
+    } else {
+        // ---------------- epilogue: tensor memory -> registers -> (scale, shift) -> bf16 -> global ----
+        const int quarter = warp & 3;
+        const int egroup = (warp - 3) >> 2;            // M blocks egroup, egroup + 2 of every tile
+        uint32_t i = 0;
+        for (uint32_t t = blockIdx.x; t < total_tiles; t += gridDim.x, ++i) {
+            const uint32_t a = i % (uint32_t)g.nacc, use = i / (uint32_t)g.nacc;
+            const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->tmem_full[a], use & 1u, abort_flag));
+            if (!ok) {
+                if (lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+                break;
+            }
+            tc_fence_after_sync();
+            int img, h0, w0, n0;
+            decode(t, img, h0, w0, n0);
+            for (int mb = egroup; mb < g.nmb; mb += 2) {
+                const uint32_t v = (uint32_t)mb * 128u + (uint32_t)(quarter * 32 + lane);
+                const uint32_t vi = v / (uint32_t)g.Wt;
+                const int ti = (int)vi, tj = (int)(v - vi * (uint32_t)g.Wt);
+                const int h = h0 + ti, wq = w0 + tj;
+                const bool valid = ti < g.R && tj < g.CW && h < g.ho && wq < g.wo;
+                __nv_bfloat16 *orow = g.out + ((size_t)((size_t)img * g.ho + (valid ? h : 0)) * g.wo + (valid ? wq : 0)) * g.cn + n0;
+                const uint32_t t_row = tmem_base + (a * (uint32_t)g.nmb + (uint32_t)mb) * BN + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    uint32_t vv[32];
+                    tmem_ld_32x32(t_row + (uint32_t)c0, vv);
+                    tmem_ld_wait();
+                    if (valid) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            float f[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(vv[j + e]);
+                            if (fold) {
+                                const float4 s0 = *(const float4 *)(scale_s + n0 + c0 + j);
+                                const float4 s1 = *(const float4 *)(scale_s + n0 + c0 + j + 4);
+                                f[0] *= s0.x; f[1] *= s0.y; f[2] *= s0.z; f[3] *= s0.w;
+                                f[4] *= s1.x; f[5] *= s1.y; f[6] *= s1.z; f[7] *= s1.w;
+                            }
+                            if (bias || fold) {
+                                const float4 b0 = *(const float4 *)(bias_s + n0 + c0 + j);
+                                const float4 b1 = *(const float4 *)(bias_s + n0 + c0 + j + 4);
+                                f[0] += b0.x; f[1] += b0.y; f[2] += b0.z; f[3] += b0.w;
+                                f[4] += b1.x; f[5] += b1.y; f[6] += b1.z; f[7] += b1.w;
+                            }
+                            uint4 pk;
+                            __nv_bfloat162 hh;
+                            hh = __floats2bfloat162_rn(f[0], f[1]); pk.x = *(uint32_t *)&hh;
+                            hh = __floats2bfloat162_rn(f[2], f[3]); pk.y = *(uint32_t *)&hh;
+                            hh = __floats2bfloat162_rn(f[4], f[5]); pk.z = *(uint32_t *)&hh;
+                            hh = __floats2bfloat162_rn(f[6], f[7]); pk.w = *(uint32_t *)&hh;
+                            *(uint4 *)(orow + c0 + j) = pk;
+                        }
+                    }
+                }
+            }
+            // this warp has read all it needs from the accumulator set
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->tmem_empty[a]);
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 2) tmem_dealloc(tmem_base, g.tmem_cols);
+}
+
+// ---- host side --------------------------------------------------------------------------------------
+namespace {
+
+struct StripPlan { bool ok = false; int bn = 64, R = 0, CW = 0, Wt = 0, nmb = 0, nacc = 2, tiles_w = 1 << 20; uint32_t strip_bytes = 0; size_t smem = 0; };
+
+StripPlan plan_strip(const UmmaConvShape &s) {
+    StripPlan best;
+    if (s.stride_h != 1 || s.stride_w != 1 || s.dil_h != 1 || s.dil_w != 1 || s.blockdiag || s.out_sw) return best;
+    if (s.taps_h * s.taps_w < 2 || s.ca % 64 || s.cn % 64 || s.cn > 4096 || s.wo < 14 || s.ho < 2) return best;
+    if ((long long)s.n * s.ho * s.wo >= (1LL << 30)) return best;
+    const int bn = (s.cn % 128 == 0) ? 128 : 64;
+    const int nmb_max = 512 / bn / 2;                      // two accumulator sets
+    const int tiles_w_min = (s.wo + (256 - s.taps_w + 1) - 1) / (256 - s.taps_w + 1);
+    double best_eff = 0.0, best_score = -1.0;
+    for (int tiles_w = tiles_w_min; tiles_w < tiles_w_min + 4; ++tiles_w) {
+    const int cw = (s.wo + tiles_w - 1) / tiles_w, wt = cw + s.taps_w - 1;
+    if (cw < 8) break;
+    for (int r = 1; r <= s.ho && r + s.taps_h - 1 <= 256; ++r) {
+        const int nmb = (r * wt + 127) / 128;
+        if (nmb > nmb_max) break;
+        const size_t px = (size_t)nmb * 128 + (size_t)(s.taps_h - 1) * wt + (s.taps_w - 1);
+        const uint32_t sbytes = (uint32_t)(((px * 128) + 1023) / 1024 * 1024);
+        const size_t smem = 1024 + 2 * (size_t)sbytes + (size_t)kSBStages * bn * 128 + sizeof(StripCtl) +
+                            2 * (size_t)s.cn * sizeof(float) + 32;
+        if (smem > 224 * 1024) break;
+        // useful fraction of the MMA rows, derated by the halo rows that are loaded again by the next tile
+        const int tiles_h = (s.ho + r - 1) / r;
+        const double eff = (double)s.ho * s.wo / ((double)tiles_h * tiles_w * nmb * 128.0);
+        // prefer the useful fraction; among equals fewer column tiles (less halo), then taller tiles
+        const double score = eff - 0.01 * (tiles_w - tiles_w_min) + 1e-4 * r;
+        if (score > best_score) {
+            best_score = score;
+            best_eff = eff;
+            best.ok = true; best.bn = bn; best.R = r; best.CW = cw; best.Wt = wt; best.nmb = nmb;
+            best.strip_bytes = sbytes; best.smem = smem; best.tiles_w = tiles_w;
+        }
+    }
+    }
+    if (best_eff < 0.70) best.ok = false;
+    return best;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// NHWC bf16 tensor as a 4-D tiled map (c, w, h, n): box = 64 channels x box_w x box_h x 1 image.
+bool make_tmap_nhwc_box(CUtensorMap *tm, const void *base, int n, int h, int w, int c, int box_w, int box_h) {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return false;
+        fn = (EncodeTiledFn)f;
+    }
+    cuuint64_t dims[4] = {(cuuint64_t)c, (cuuint64_t)w, (cuuint64_t)h, (cuuint64_t)n};
+    cuuint64_t strides[3] = {(cuuint64_t)c * 2, (cuuint64_t)w * c * 2, (cuuint64_t)h * w * c * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)box_w, (cuuint32_t)box_h, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int strip_sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0, v = 0;
+        n = (cudaGetDevice(&dev) == cudaSuccess &&
+             cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) ? v : 148;
+    }
+    return n;
+}
+
+template <int BN>
+cudaError_t launch_strip(const CUtensorMap &ta, const CUtensorMap &tw, const StripGemm &g, size_t smem,
+                         const float *bias, int *err, cudaStream_t st) {
+    static bool attr = false;
+    if (!attr) {
+        cudaError_t e = cudaFuncSetAttribute(umma_strip_conv_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             226 * 1024);
+        if (e != cudaSuccess) return e;
+        attr = true;
+    }
+    const long long total = (long long)g.n * g.tiles_h * g.tiles_w * (g.cn / BN);
+    const unsigned grid = (unsigned)(total < strip_sm_count() ? total : strip_sm_count());
+    return launch_pdl(umma_strip_conv_kernel<BN>, dim3(grid), dim3(kSThreads), smem, st, ta, tw, g, bias, err);
+}
+
+}  // namespace
+
+bool umma_strip_eligible(const UmmaConvShape &s) {
+    static const bool off = [] { const char *e = getenv("CONVBN_NO_STRIP"); return e && e[0] == '1'; }();
+    return !off && plan_strip(s).ok;
+}
+
+cudaError_t launch_umma_strip_conv(const UmmaConvShape &s, const void *act, const void *wmat, const float *bias,
+                                   void *out, cudaStream_t st, const BnFold *fold) {
+    const StripPlan pl = plan_strip(s);
+    if (!pl.ok) return cudaErrorInvalidValue;
+    StripGemm g;
+    g.n = s.n; g.ho = s.ho; g.wo = s.wo; g.cn = s.cn; g.ca = s.ca; g.kh = s.taps_h; g.kw = s.taps_w;
+    g.lower_h = s.lower_h; g.lower_w = s.lower_w;
+    g.R = pl.R; g.CW = pl.CW; g.Wt = pl.Wt; g.rows_in = pl.R + s.taps_h - 1; g.nmb = pl.nmb;
+    g.tiles_h = (s.ho + pl.R - 1) / pl.R; g.tiles_w = (s.wo + pl.CW - 1) / pl.CW;
+    g.strip_bytes = pl.strip_bytes;
+    g.nacc = 2;
+    int cols = 2 * pl.nmb * pl.bn, p2 = 32;
+    while (p2 < cols) p2 <<= 1;
+    g.tmem_cols = (uint32_t)p2;
+    g.out = (__nv_bfloat16 *)out;
+    g.fold = fold ? *fold : BnFold{nullptr, nullptr, nullptr, nullptr, nullptr, 0.f, nullptr};
+    CUtensorMap ta, tw;
+    if (!make_tmap_nhwc_box(&ta, act, s.n, s.ha, s.wa, s.ca, pl.Wt, g.rows_in)) return cudaErrorInvalidValue;
+    if (!make_tmap_matrix_bf16(&tw, wmat, s.cn, (long long)s.taps_h * s.taps_w * s.ca, pl.bn, 64))
+        return cudaErrorInvalidValue;
+    int *err = nullptr;
+    cudaError_t e = error_word_address(&err);
+    if (e != cudaSuccess) return e;
+    if (pl.bn == 64) return launch_strip<64>(ta, tw, g, pl.smem, bias, err, st);
+    return launch_strip<128>(ta, tw, g, pl.smem, bias, err, st);
+}
+
+}  // namespace convbn
