@@ -85,6 +85,16 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// Ask for the largest shared-memory carve-out for a kernel, once.  The tensor-core kernels need it;
+// the small kernels launched between them ask for the same split so that the SMs are not
+// re-partitioned (which drains them) at every kernel boundary of a training step.
+template <class K>
+inline void prefer_max_shared_once(K kernel, bool *done) {
+    if (*done) return;
+    cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    *done = true;
+}
+
 static inline int ceil_div_i(long long a, long long b) { return (int)((a + b - 1) / b); }
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 

@@ -166,6 +166,8 @@ __global__ void __launch_bounds__(256) reparam_dgrad_class_kernel(int c_out, int
 cudaError_t launch_reparam_dgrad_class(const Problem &pb, const void *w, const float *s_vec, void *w_t, int th,
                                        int tw, int r_max, int q_max, int step_h, int step_w, cudaStream_t st) {
     dim3 grid((pb.c_in + 31) / 32, (pb.c_out + 31) / 32, th * tw);
+    static bool carve = false;
+    prefer_max_shared_once(reparam_dgrad_class_kernel, &carve);
     return launch_pdl(reparam_dgrad_class_kernel, grid, dim3(256), 0, st, pb.c_out, pb.c_in, pb.kw, tw, r_max, q_max,
                       step_h, step_w, th * tw, (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t, pb.kh * pb.kw);
 }
@@ -173,6 +175,8 @@ cudaError_t launch_reparam_dgrad_class(const Problem &pb, const void *w, const f
 cudaError_t launch_reparam_dgrad(const Problem &pb, const void *w, const float *s_vec, void *w_t,
                                  cudaStream_t st) {
     dim3 grid((pb.c_in + 31) / 32, (pb.c_out + 31) / 32, pb.kh * pb.kw);
+    static bool carve = false;
+    prefer_max_shared_once(reparam_dgrad_kernel, &carve);
     return launch_pdl(reparam_dgrad_kernel, grid, dim3(256), 0, st, pb.c_out, pb.c_in, pb.kh * pb.kw,
                       (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t);
 }

@@ -442,6 +442,8 @@ static cudaError_t launch_bn(const CUtensorMap &ta, const CUtensorMap &tw, const
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
+    static bool carve = false;
+    prefer_max_shared_once(umma_conv_kernel<BN>, &carve);
     const unsigned grid = (unsigned)grid_l;
     return launch_pdl(umma_conv_kernel<BN>, dim3(grid), dim3(kConvThreads), smem, st, ta, tw, tout, g, bias, err);
 }

@@ -174,13 +174,15 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
                         tc_fence_after_sync();
                         const uint32_t b_addr = smem_u32(bring + (size_t)s * kBBytes);
                         const uint32_t shift = (uint32_t)(r * g.Wt + q) * 128u;
-                        for (int mb = 0; mb < g.nmb; ++mb) {
-                            const uint32_t a_addr = patch + (uint32_t)mb * (128u * 128u) + shift;
+                        // consecutive MMAs go to different accumulators (M blocks), so an MMA never has to
+                        // wait for the previous one's accumulator update
 #pragma unroll
-                            for (int k = 0; k < 4; ++k)
-                                umma_bf16_ss(d0 + (uint32_t)(mb * BN), smem_desc_sw128(a_addr + k * 32, 16, 1024),
-                                             smem_desc_sw128(b_addr + k * 32, 16, 1024), idesc,
-                                             (cc | tap | k) ? 1u : 0u);
+                        for (int k = 0; k < 4; ++k) {
+                            const uint64_t bd = smem_desc_sw128(b_addr + k * 32, 16, 1024);
+                            for (int mb = 0; mb < g.nmb; ++mb)
+                                umma_bf16_ss(d0 + (uint32_t)(mb * BN),
+                                             smem_desc_sw128(patch + (uint32_t)mb * (128u * 128u) + shift + k * 32, 16, 1024),
+                                             bd, idesc, (cc | tap | k) ? 1u : 0u);
                         }
                         umma_commit(&ctl->b_empty[s]);
                         if (++s == kSBStages) { s = 0; bph ^= 1u; }
@@ -347,6 +349,8 @@ cudaError_t launch_strip(const CUtensorMap &ta, const CUtensorMap &tw, const Str
         if (e != cudaSuccess) return e;
         attr = true;
     }
+    static bool carve = false;
+    prefer_max_shared_once(umma_strip_conv_kernel<BN>, &carve);
     const long long total = (long long)g.n * g.tiles_h * g.tiles_w * (g.cn / BN);
     const unsigned grid = (unsigned)(total < strip_sm_count() ? total : strip_sm_count());
     return launch_pdl(umma_strip_conv_kernel<BN>, dim3(grid), dim3(kSThreads), smem, st, ta, tw, g, bias, err);

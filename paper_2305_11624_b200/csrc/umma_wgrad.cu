@@ -260,6 +260,8 @@ static cudaError_t launch_w(const CUtensorMap &tx, const CUtensorMap &tdz, Wgrad
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
+    static bool carve = false;
+    prefer_max_shared_once(umma_wgrad_kernel<BN>, &carve);
     dim3 grid((unsigned)((g.kdim / 64 + 2) / 2), (unsigned)((pb.c_out + BN - 1) / BN), (unsigned)pl.splits);
     return launch_pdl(umma_wgrad_kernel<BN>, grid, dim3(kWThreads), smem, st, tx, tdz, g, partials, bsum, counters,
                       pb.c_out / 32, err);
@@ -388,6 +390,9 @@ cudaError_t launch_wgrad_epilogue_fused(const Problem &pb, const UmmaWgradPlan &
                                         float *db, float *dgamma, float *dbeta, bool need_sums, cudaStream_t st) {
     const dim3 grid(pb.c_out / 32, pl.kt);
     const int ns = need_sums ? 1 : 0;
+    static bool carve_a = false, carve_b = false;
+    prefer_max_shared_once(wgrad_epilogue_fused_kernel<8, 4>, &carve_a);
+    prefer_max_shared_once(wgrad_epilogue_fused_kernel<2, 16>, &carve_b);
     if (pl.kr == 8)
         return launch_pdl(wgrad_epilogue_fused_kernel<8, 4>, grid, dim3(1024), 0, st, pb.c_out, pb.kdim, partials,
                           pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw, dotpart, counters, db,
