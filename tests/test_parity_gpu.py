@@ -38,7 +38,29 @@ SMALL = [
     L("b_dw_s2", 1, 32, 9, 9, 32, 3, 3, stride=2, pad=1, groups=32),
     L("b_grouped", 2, 256, 9, 9, 256, 3, 3, pad=1, groups=32),
     L("b_grouped_cout2x", 1, 16, 6, 6, 32, 3, 3, pad=1, groups=4),
+    # strip kernel: column split (W > 256), BN = 128, ragged rows, 5x5, two channel chunks
+    L("b_strip_wide", 1, 64, 7, 300, 64, 3, 3, pad=1),
+    L("b_strip_bn128", 2, 128, 19, 33, 128, 3, 3, pad=1),
+    L("b_strip_5x5", 1, 64, 21, 40, 64, 5, 5, pad=2),
+    L("b_strip_1x3", 1, 64, 9, 30, 192, 1, 3, pad=0),
+    # strided backward data: 1x1 stride 2 (empty residue classes), 5x5 stride 2, stride 3
+    L("b_1x1_s2", 2, 64, 15, 14, 128, 1, 1, stride=2),
+    L("b_5x5_s2", 1, 64, 17, 19, 64, 5, 5, stride=2, pad=2),
+    L("b_3x3_s3", 1, 64, 20, 16, 64, 3, 3, stride=3, pad=1),
+    # grouped block-diagonal with other group widths; depthwise 5x5
+    L("b_grouped_cg4", 1, 64, 10, 12, 64, 3, 3, pad=1, groups=16),
+    L("b_grouped_cg32_s2", 2, 128, 11, 9, 128, 3, 3, stride=2, pad=1, groups=4),
+    L("b_dw_5x5", 1, 48, 11, 13, 48, 5, 5, pad=2, groups=48),
 ]
+
+EXPECTED_PATH = {   # the specialised kernels must actually be the ones that ran
+    "b_1x1_a": ("umma", "umma", "umma"), "b_3x3_a": ("umma-strip", "umma-strip", "umma"),
+    "b_3x3_s2": ("umma", "umma-strided", "umma"), "b_dw": ("depthwise", "depthwise", "depthwise"),
+    "b_grouped": ("grouped-umma", "grouped-umma", "grouped-umma"), "b_odd_c": ("direct", "direct", "direct"),
+    "b_strip_wide": ("umma-strip", "umma-strip", "umma"), "b_strip_bn128": ("umma-strip", "umma-strip", "umma"),
+    "b_1x1_s2": ("umma", "umma-strided", "umma"), "b_grouped_cg32_s2": ("grouped-umma", "direct", "grouped-umma"),
+    "f32_bias": ("direct", "direct", "direct"),
+}
 
 
 @pytest.mark.parametrize("spec", SMALL, ids=lambda s: s.name)
@@ -47,6 +69,8 @@ def test_tune_small(spec):
     ref = parity.oracle_tune(spec, t)
     got = parity.run_tune_gpu(spec, t)
     parity.compare(got, ref, parity.TOL[spec.dtype], parity.TUNE_OUTPUTS, spec.name)
+    if spec.name in EXPECTED_PATH:
+        assert got["_kernels"] == EXPECTED_PATH[spec.name], got["_kernels"]
 
 
 FULL = [(ci, li, sp) for ci, layers in I.CONFIGS.items() for li, sp in enumerate(layers)]
