@@ -122,71 +122,6 @@ __global__ void __launch_bounds__(256) dw_fwd_kernel(DwShape s, const uint4 *__r
     }
 }
 
-// Unit stride and dilation, KH x KW known at compile time: the thread's whole input window
-// (KH rows x (TW + KW - 1) vectors) is requested before any arithmetic, so one memory round trip
-// serves TW outputs; this is what lets a streaming kernel with few resident threads fill HBM.
-template <int TW, int KH, int KW>
-__global__ void __launch_bounds__(256, 1) dw_fwd_window_kernel(DwShape s, const uint4 *__restrict__ x,
-                                                               const __nv_bfloat16 *__restrict__ w,
-                                                               const float *__restrict__ bias,
-                                                               uint4 *__restrict__ z) {
-    extern __shared__ float w_s[];                   // [taps][C]
-    const int v = s.c / 8;
-    stage_weights(w_s, w, KH * KW, s.c);
-    const uint32_t wgroups = (uint32_t)(s.w_out + TW - 1) / TW;
-    const uint32_t total = (uint32_t)s.n * s.h_out * wgroups * v;
-    for (uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
-        uint32_t t = idx / (uint32_t)v;
-        const int cv = (int)(idx - t * (uint32_t)v);
-        const uint32_t t1 = t / wgroups;
-        const int wg = (int)(t - t1 * wgroups);
-        const uint32_t n = t1 / (uint32_t)s.h_out;
-        const int ho = (int)(t1 - n * (uint32_t)s.h_out);
-        const int wo0 = wg * TW, wi0 = wo0 - s.pad_w, hi0 = ho - s.pad_h;
-        uint4 seg[KH][TW + KW - 1];
-#pragma unroll
-        for (int r = 0; r < KH; ++r) {
-            const int hi = hi0 + r;
-            const bool row_ok = hi >= 0 && hi < s.h_in;
-            const uint4 *xrow = x + ((size_t)(n * s.h_in + (row_ok ? hi : 0)) * s.w_in) * v + cv;
-#pragma unroll
-            for (int j = 0; j < TW + KW - 1; ++j) {
-                const int wi = wi0 + j;
-                seg[r][j] = (row_ok && wi >= 0 && wi < s.w_in) ? __ldg(xrow + (size_t)wi * v) : make_uint4(0, 0, 0, 0);
-            }
-        }
-        float acc[TW][8];
-#pragma unroll
-        for (int j = 0; j < TW; ++j)
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[j][e] = bias ? bias[cv * 8 + e] : 0.f;
-#pragma unroll
-        for (int r = 0; r < KH; ++r) {
-#pragma unroll
-            for (int j = 0; j < TW + KW - 1; ++j) {
-                float xv[8];
-                unpack8(seg[r][j], xv);
-#pragma unroll
-                for (int q = 0; q < KW; ++q) {
-                    const int o = j - q;                 // output column fed by this vector through tap q
-                    if (o >= 0 && o < TW) {
-                        const float4 w0 = *(const float4 *)(w_s + (r * KW + q) * s.c + cv * 8);
-                        const float4 w1 = *(const float4 *)(w_s + (r * KW + q) * s.c + cv * 8 + 4);
-                        acc[o][0] = fmaf(xv[0], w0.x, acc[o][0]); acc[o][1] = fmaf(xv[1], w0.y, acc[o][1]);
-                        acc[o][2] = fmaf(xv[2], w0.z, acc[o][2]); acc[o][3] = fmaf(xv[3], w0.w, acc[o][3]);
-                        acc[o][4] = fmaf(xv[4], w1.x, acc[o][4]); acc[o][5] = fmaf(xv[5], w1.y, acc[o][5]);
-                        acc[o][6] = fmaf(xv[6], w1.z, acc[o][6]); acc[o][7] = fmaf(xv[7], w1.w, acc[o][7]);
-                    }
-                }
-            }
-        }
-        uint4 *zrow = z + ((size_t)(n * s.h_out + ho) * s.w_out + wo0) * v + cv;
-#pragma unroll
-        for (int j = 0; j < TW; ++j)
-            if (wo0 + j < s.w_out) zrow[(size_t)j * v] = pack8(acc[j]);
-    }
-}
-
 // dX[n,h,w,c] = sum over taps with (h + p - r d) divisible by the stride of omega'[c,r,q] dZ[n,ho,wo,c].
 __global__ void __launch_bounds__(256) dw_dgrad_kernel(DwShape s, const uint4 *__restrict__ dz,
                                                        const __nv_bfloat16 *__restrict__ w,
@@ -277,7 +212,7 @@ __global__ void __launch_bounds__(256) dw_wgrad_kernel(DwShape s, const uint4 *_
     }
 }
 
-// Unit stride / dilation, KH x KW known: like the forward window kernel, every thread requests the
+// Unit stride / dilation, KH x KW known at compile time: every thread requests the
 // KH x (TW + KW - 1) input window and TW dZ vectors of its item before any arithmetic.
 // Items are (image, output row, group of TW output columns); a block owns a contiguous item range.
 template <int TW, int KH, int KW>
@@ -385,13 +320,9 @@ cudaError_t launch_dw_fwd(const Problem &pb, const void *x, const void *w, const
     const size_t smem = (size_t)pb.kh * pb.kw * pb.c_in * sizeof(float);
     const long long total = (long long)pb.n * pb.h_out * ((pb.w_out + 3) / 4) * (pb.c_in / 8);
     const bool unit_w = pb.stride_w == 1 && pb.dil_w == 1;
-    static bool a3 = false, a5 = false, a0 = false, a33 = false;
+    static bool a3 = false, a5 = false, a0 = false;
     cudaError_t e;
-    if (unit_w && pb.stride_h == 1 && pb.dil_h == 1 && pb.kh == 3 && pb.kw == 3) {
-        if ((e = set_smem_once(dw_fwd_window_kernel<4, 3, 3>, &a33)) != cudaSuccess) return e;
-        dw_fwd_window_kernel<4, 3, 3><<<dw_grid(total), 256, smem, st>>>(s, (const uint4 *)x, (const __nv_bfloat16 *)w,
-                                                                         bias, (uint4 *)z);
-    } else if (unit_w && pb.kw == 3) {
+    if (unit_w && pb.kw == 3) {
         if ((e = set_smem_once(dw_fwd_kernel<4, 3>, &a3)) != cudaSuccess) return e;
         dw_fwd_kernel<4, 3><<<dw_grid(total), 256, smem, st>>>(s, (const uint4 *)x, (const __nv_bfloat16 *)w, bias,
                                                                 (uint4 *)z);
