@@ -134,6 +134,23 @@ class ClockSampler(threading.Thread):
                 "reasons": sorted(snake[r] for r in self.reasons)}
 
 
+# ---- multi-rank bookkeeping (replicas: every rank runs the whole workload on its own batch) -------
+def max_over_ranks(value, device=None):
+    """The slowest rank's time: MAX all-reduce over the default process group (identity for one rank)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(flops_per_step, steps, ms_max, world):
+    """Aggregate TFLOP/s of `world` replicas that each did `steps` steps within `ms_max` milliseconds."""
+    return world * flops_per_step * steps / (ms_max * 1e-3) / 1e12
+
+
 # ---- the CPU oracle, timed (reported baseline and the --impl reference arm) ----------------------
 def oracle_step_time(workload, batch, repeats, seed=7):
     """Seconds per Tune fwd+bwd step of the fp64 oracle on `batch` samples of every layer of the
@@ -231,13 +248,6 @@ def run_ours(args):
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
-    def max_over_ranks(v):
-        if world > 1:
-            t = torch.tensor([v], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            return float(t.item())
-        return v
-
     # ---- timed region: K steps, each a replay of the CUDA graph of one step (one graph per buffer
     # set), so the layers' ~15 launches per step cost no host time; --no-graph times eager calls.
     graphs, launch_mode = None, "eager library calls"
@@ -265,8 +275,8 @@ def run_ours(args):
             step(args.warmup + i)
     e1.record(stream)
     barrier()
-    ms = max_over_ranks(e0.elapsed_time(e1))
-    value = world * step_flops * args.steps / (ms * 1e-3) / 1e12
+    ms = max_over_ranks(e0.elapsed_time(e1), dev)
+    value = whole_job_value(step_flops, args.steps, ms, world)
 
     # ---- second pass, same K steps as eager calls with a CUDA-event pair around every kernel: the
     # per-kernel durations behind the roofline object (events cannot be read back out of a graph)
@@ -279,7 +289,7 @@ def run_ours(args):
     f1.record(stream)
     barrier()
     prof = C.convbn_profile_end()
-    eager_ms = max_over_ranks(f0.elapsed_time(f1))
+    eager_ms = max_over_ranks(f0.elapsed_time(f1), dev)
     sampler.stop_flag.set()
     sampler.join()
     C.convbn_check()
