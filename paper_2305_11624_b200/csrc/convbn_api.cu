@@ -102,6 +102,10 @@ bool force_direct() {
     return v;
 }
 
+bool stem_path(const convbn_desc *d, const Problem &pb) {
+    return !force_direct() && d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && stem_eligible(pb);
+}
+
 bool grouped_path(const convbn_desc *d, const Problem &pb) {
     return !force_direct() && d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && grouped_bd_eligible(pb);
 }
@@ -118,6 +122,8 @@ struct Plan {
     size_t dotpart = 0;    // [kt][C_out] fp32 (tensor-core weight-gradient path)
     size_t counters = 0;   // C_out / 32 words (fused epilogue)
     int splits = 1, bsplits = 1, bn_splits = 1;
+    size_t xpk = 0, wst = 0;   // small-C_in layers: packed input [n][hp][wp][8], expanded weights [C_out][kh][64]
+    bool stem = false;
     size_t wbd = 0;        // block-diagonal expanded weights [C_out][taps][64], storage dtype
     bool umma_wgrad = false, dw_wgrad = false, grouped_wgrad = false;
     UmmaWgradPlan uw;
@@ -141,6 +147,8 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
         pl.splits = dw_wgrad_splits(pb);
         part_bytes = wrows * pl.splits * sizeof(float);
     }
+    pl.stem = stem_path(d, pb);
+    const size_t xpk_bytes = pl.stem ? stem_packed_bytes(pb) : 0, wst_bytes = pl.stem ? stem_weight_bytes(pb) : 0;
     const bool grouped = grouped_path(d, pb);
     const size_t wbd_bytes = grouped ? (size_t)pb.c_out * pb.kh * pb.kw * 64 * elem_size(d->dtype) : 0;
     pl.grouped_wgrad = grouped;
@@ -160,9 +168,11 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
         case CONVBN_PHASE_TUNE_BWD_DATA:
             pl.w_scaled = take(wbytes);
             pl.wbd = take(wbd_bytes);
+            if (phase == CONVBN_PHASE_TUNE_FWD) { pl.xpk = take(xpk_bytes); pl.wst = take(wst_bytes); }
             break;
         case CONVBN_PHASE_DEPLOY_FWD:
             pl.wbd = take(wbd_bytes);
+            pl.xpk = take(xpk_bytes); pl.wst = take(wst_bytes);
             break;
         case CONVBN_PHASE_DEPLOY_BWD:
             pl.w_scaled = take(wbytes);
@@ -181,6 +191,7 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
         case CONVBN_PHASE_EVAL_FWD:
             pl.vec3 = take(3 * (size_t)pb.c_out * sizeof(float));
             pl.wbd = take(wbd_bytes);
+            pl.xpk = take(xpk_bytes); pl.wst = take(wst_bytes);
             break;
         case CONVBN_PHASE_EVAL_BWD:
             pl.dy = take((size_t)pb.p * pb.c_out * elem_size(d->dtype));
@@ -287,9 +298,17 @@ bool strided_dgrad_ok(const convbn_desc *d, const Problem &pb) {
 
 // Forward convolution with whatever weights / bias the mode folded: tensor cores when eligible.
 int run_conv_fwd(const convbn_desc *d, const Problem &pb, const void *x, const void *w, const float *bias,
-                 void *z, void *wbd_scratch, cudaStream_t st, const char **which) {
+                 void *z, const Plan &pl, void *ws, cudaStream_t st, const char **which) {
     UmmaConvShape s;
-    if (grouped_path(d, pb)) {
+    void *wbd_scratch = at(ws, pl.wbd);
+    if (pl.stem) {
+        // few input channels: repack X (8 channels per pixel, zero border) and run the tensor-core GEMM
+        // with one 64-wide K row (8 pixels x 8 channels) per filter row
+        LAUNCH("stem_pack", launch_stem_pack(pb, x, at(ws, pl.xpk), st));
+        LAUNCH("stem_expand", launch_stem_expand_weights(pb, w, nullptr, at(ws, pl.wst), st));
+        LAUNCH("stem_fwd", launch_stem_fwd(pb, at(ws, pl.xpk), at(ws, pl.wst), bias, z, st));
+        *which = "umma-stem";
+    } else if (grouped_path(d, pb)) {
         // block-diagonal GEMM: expand the (already folded) weights, then the dense tensor-core kernel
         s = UmmaConvShape{pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.c_out, pb.kh, pb.kw,
                           -pb.pad_h, -pb.pad_w, pb.stride_h, pb.stride_w, pb.dil_h, pb.dil_w, 1};
@@ -487,6 +506,14 @@ int convbn_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const
     float *vec3 = (float *)saved;
     void *wf = at(workspace, pl.w_scaled);
     UmmaConvShape us;
+    if (pl.stem) {
+        const BnFold fold{gamma, beta, run_mean, run_var, b, pb.eps, vec3};
+        LAUNCH("stem_pack", launch_stem_pack(pb, x, at(workspace, pl.xpk), st));
+        LAUNCH("stem_expand", launch_stem_expand_weights(pb, w, nullptr, at(workspace, pl.wst), st));
+        LAUNCH("stem_fwd", launch_stem_fwd(pb, at(workspace, pl.xpk), at(workspace, pl.wst), nullptr, z, st, &fold));
+        t_last_kernel[CONVBN_PHASE_TUNE_FWD] = "umma-stem";
+        return CONVBN_OK;
+    }
     if (!grouped_path(desc, pb) && umma_fwd_shape(desc, pb, &us)) {
         // dense tensor-core path: s, b' and the saved vectors are formed inside the GEMM kernel and s is
         // applied to the fp32 accumulator, so one launch does the whole forward pass
@@ -502,7 +529,7 @@ int convbn_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const
     }
     LAUNCH("reparam", launch_reparam(pb, desc->dtype, desc->layout, w, b, gamma, beta, run_mean, run_var, vec3, wf,
                       nullptr, st));
-    CK(run_conv_fwd(desc, pb, x, wf, vec3 + pb.c_out, z, at(workspace, pl.wbd), st, &t_last_kernel[CONVBN_PHASE_TUNE_FWD]));
+    CK(run_conv_fwd(desc, pb, x, wf, vec3 + pb.c_out, z, pl, workspace, st, &t_last_kernel[CONVBN_PHASE_TUNE_FWD]));
     return CONVBN_OK;
 }
 
@@ -563,7 +590,7 @@ int convbn_eval_fwd(const convbn_desc *desc, const void *x, const void *w, const
     // BN acts on Y, which already holds the conv bias: shift = beta - mean s
     LAUNCH("reparam", launch_reparam(pb, desc->dtype, desc->layout, w, nullptr, gamma, beta, run_mean, run_var, vec3,
                       nullptr, nullptr, st));
-    CK(run_conv_fwd(desc, pb, x, w, b, y_saved, at(workspace, pl.wbd), st, &t_last_kernel[CONVBN_PHASE_EVAL_FWD]));
+    CK(run_conv_fwd(desc, pb, x, w, b, y_saved, pl, workspace, st, &t_last_kernel[CONVBN_PHASE_EVAL_FWD]));
     LAUNCH("bn_eval_fwd", launch_bn_eval_fwd(pb, desc->dtype, desc->layout, y_saved, vec3, z, st));
     return CONVBN_OK;
 }
@@ -625,7 +652,7 @@ int convbn_deploy_fwd(const convbn_desc *desc, const void *x, const void *w_fuse
     const Plan pl = make_plan(desc, pb, CONVBN_PHASE_DEPLOY_FWD);
     CK(check_ws(pl, workspace, workspace_bytes));
     cudaStream_t st = (cudaStream_t)stream;
-    CK(run_conv_fwd(desc, pb, x, w_fused, b_fused, z, at(workspace, pl.wbd), st, &t_last_kernel[CONVBN_PHASE_DEPLOY_FWD]));
+    CK(run_conv_fwd(desc, pb, x, w_fused, b_fused, z, pl, workspace, st, &t_last_kernel[CONVBN_PHASE_DEPLOY_FWD]));
     return CONVBN_OK;
 }
 

@@ -94,6 +94,17 @@ cudaError_t launch_wgrad_epilogue_fused(const Problem &pb, const UmmaWgradPlan &
                                         const float *mean, float *dw, float *dotpart, unsigned int *counters,
                                         float *db, float *dgamma, float *dbeta, bool need_sums, cudaStream_t st);
 
+// ---- first-layer convolutions with C_in <= 8 (see stem_kernels.cu) -------------------------------
+bool stem_eligible(const Problem &pb);
+void stem_geometry(const Problem &pb, int *hp, int *wp);     // extent of the packed, zero-bordered input
+size_t stem_packed_bytes(const Problem &pb);                 // [n][hp][wp][8] bf16
+size_t stem_weight_bytes(const Problem &pb);                 // [C_out][kh][64] bf16
+cudaError_t launch_stem_pack(const Problem &pb, const void *x, void *x_packed, cudaStream_t st);
+cudaError_t launch_stem_expand_weights(const Problem &pb, const void *w, const float *s_vec, void *wst,
+                                       cudaStream_t st);
+cudaError_t launch_stem_fwd(const Problem &pb, const void *x_packed, const void *wst, const float *bias, void *out,
+                            cudaStream_t st, const BnFold *fold = nullptr);
+
 // ---- depthwise (groups = C_in = C_out) bandwidth kernels, bf16 NHWC, C multiple of 8 -----------
 bool dw_eligible(const Problem &pb);
 bool dw_wgrad_supported(const Problem &pb);     // tap counts the register-tiled kernel is built for

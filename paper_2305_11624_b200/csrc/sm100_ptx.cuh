@@ -20,6 +20,10 @@ bool make_tmap_im2col_bf16(CUtensorMap *tm, const void *base, int n, int h, int 
                            int lower_w, int upper_h, int upper_w, int stride_h, int stride_w, int pixels,
                            int channels);
 
+// General tiled map over bf16 data: rank <= 5, dims / byte strides (strides[0] unused) / box, 128-byte swizzle.
+bool make_tmap_tiled_bf16(CUtensorMap *tm, const void *base, int rank, const unsigned long long *dims,
+                          const unsigned long long *strides_bytes, const unsigned int *box);
+
 namespace ptx {
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
@@ -97,6 +101,13 @@ __device__ __forceinline__ void tma_load_4d(void *smem_dst, const CUtensorMap *m
         ::"r"(smem_u32(smem_dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(c), "r"(w), "r"(h), "r"(n)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_5d(void *smem_dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1,
+                                            int c2, int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(smem_u32(smem_dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        : "memory");
+}
 // im2col mode over an NHWC tensor: (c, w, h, n) is the first pixel's base coordinate, (off_w, off_h)
 // the filter-tap offset added to every pixel of the column.
 __device__ __forceinline__ void tma_load_im2col_4d(void *smem_dst, const CUtensorMap *map, uint64_t *bar, int c,
@@ -112,6 +123,12 @@ __device__ __forceinline__ void tma_load_im2col_4d(void *smem_dst, const CUtenso
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, const void *smem_src, int x, int y) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
                  ::"l"((uint64_t)map), "r"(smem_u32(smem_src)), "r"(x), "r"(y)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, const void *smem_src, int c0, int c1, int c2,
+                                             int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                 ::"l"((uint64_t)map), "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
                  : "memory");
 }
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }

@@ -42,6 +42,10 @@ struct ConvGemm {
     __nv_bfloat16 *out_strided;
     long long out_sn;
     int out_sh, out_sw;
+    // Small-C_in ("stem") mode: the activation map is a 5-D window view {64, wo, ho, r, n} of a packed,
+    // zero-bordered copy of X (8 channels per pixel; 8 pixels x 8 channels = one 128-byte K row per tap
+    // row r), tiles are stem_th x stem_tw output patches (stem_th * stem_tw = 128), the output map is 4-D.
+    int stem, stem_tw, stem_th, stem_tiles_w, stem_tiles_h;
     int resident;            // 1: the CTA's whole weight slab [BN][K] stays in shared memory (loaded once)
     BnFold fold;             // fold.gamma != NULL: scale and shift formed in the kernel from the BN parameters
 };
@@ -155,10 +159,20 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
             // 32-bit arithmetic: 64-bit divisions would cost about a microsecond per tile here
             const uint32_t m0 = mt * kBM;
             const int n0 = (int)nt * BN;
-            const uint32_t tq = m0 / (uint32_t)g.wo;
-            const int wo0 = (int)(m0 - tq * (uint32_t)g.wo);
-            const uint32_t img = tq / (uint32_t)g.ho;
-            const int ho0 = (int)(tq - img * (uint32_t)g.ho), img0 = (int)img;
+            uint32_t tq, img;
+            int wo0, ho0;
+            if (g.stem) {       // m-tile -> (image, patch row, patch column)
+                tq = mt / (uint32_t)g.stem_tiles_w;
+                wo0 = (int)(mt - tq * (uint32_t)g.stem_tiles_w) * g.stem_tw;
+                img = tq / (uint32_t)g.stem_tiles_h;
+                ho0 = (int)(tq - img * (uint32_t)g.stem_tiles_h) * g.stem_th;
+            } else {
+                tq = m0 / (uint32_t)g.wo;
+                wo0 = (int)(m0 - tq * (uint32_t)g.wo);
+                img = tq / (uint32_t)g.ho;
+                ho0 = (int)(tq - img * (uint32_t)g.ho);
+            }
+            const int img0 = (int)img;
             const int base_w = g.lower_w + wo0 * g.stride_w, base_h = g.lower_h + ho0 * g.stride_h;
             int r = 0, q = 0, cc = 0;
             for (int kb = 0; kb < num_kb; ++kb, ++it) {
@@ -167,6 +181,9 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                 uint8_t *a_dst = tiles + (size_t)s * kStageBytes, *b_dst = a_dst + kABytes;
                 if (lane == 0) {
                     mbar_arrive_expect_tx(&ctl->full[s], kStageBytes);   // (activation + weight tile) or activation only
+                    if (g.stem)
+                        tma_load_5d(a_dst, &tm_act, &ctl->full[s], 0, wo0, ho0, kb, img0);
+                    else
                     tma_load_im2col_4d(a_dst, &tm_act, &ctl->full[s], (g.blockdiag ? n0 : 0) + cc * kBK, base_w, base_h, img0,
                                        (uint16_t)(q * g.dil_w), (uint16_t)(r * g.dil_h));
                 } else if (lane == 1 && !g.resident) {
@@ -314,7 +331,15 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        tma_store_2d(&tm_out, buf, n0 + c0, (int)(m0 + quarter * 32));
+                        if (g.stem) {
+                            // this warp's 32 accumulator rows are (32 / stem_tw) patch rows of stem_tw pixels
+                            const uint32_t tq2 = mt / (uint32_t)g.stem_tiles_w, im2 = tq2 / (uint32_t)g.stem_tiles_h;
+                            tma_store_4d(&tm_out, buf, n0 + c0, (int)(mt - tq2 * (uint32_t)g.stem_tiles_w) * g.stem_tw,
+                                         (int)(tq2 - im2 * (uint32_t)g.stem_tiles_h) * g.stem_th + quarter * (32 / g.stem_tw),
+                                         (int)im2);
+                        } else {
+                            tma_store_2d(&tm_out, buf, n0 + c0, (int)(m0 + quarter * 32));
+                        }
                         tma_store_commit();
                     }
                 }
@@ -386,6 +411,18 @@ bool make_tmap_im2col_bf16(CUtensorMap *tm, const void *base, int n, int h, int 
                            upper, (cuuint32_t)channels, (cuuint32_t)pixels, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool make_tmap_tiled_bf16(CUtensorMap *tm, const void *base, int rank, const unsigned long long *dims,
+                          const unsigned long long *strides_bytes, const unsigned int *box) {
+    if (!load_encoders() || rank < 1 || rank > 5) return false;
+    cuuint64_t d[5], st[4];
+    cuuint32_t bx[5], es[5];
+    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
+    for (int i = 1; i < rank; ++i) st[i - 1] = strides_bytes[i];
+    return g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), d, st, bx,
+                          es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 bool umma_conv_eligible(const UmmaConvShape &s) {
@@ -472,6 +509,7 @@ cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void
     g.lower_h = s.lower_h; g.lower_w = s.lower_w; g.stride_h = s.stride_h; g.stride_w = s.stride_w;
     g.dil_h = s.dil_h; g.dil_w = s.dil_w; g.p = (long long)s.n * s.ho * s.wo; g.stages = 1;
     g.blockdiag = s.blockdiag;
+    g.stem = 0; g.stem_tw = g.stem_th = g.stem_tiles_w = g.stem_tiles_h = 1;
     g.fold = fold ? *fold : BnFold{nullptr, nullptr, nullptr, nullptr, nullptr, 0.f, nullptr};
     g.out_strided = s.out_sw ? (__nv_bfloat16 *)out : nullptr;
     g.out_sn = s.out_sn; g.out_sh = s.out_sh; g.out_sw = s.out_sw;
@@ -494,6 +532,46 @@ cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void
     if (bn == 64) return launch_bn<64>(ta, tw, tout, g, bias, err, st);
     if (bn == 128) return launch_bn<128>(ta, tw, tout, g, bias, err, st);
     return launch_bn<256>(ta, tw, tout, g, bias, err, st);
+}
+
+// Forward pass of a small-C_in layer on the packed input (see stem_kernels.cu): tiles of 8 x 16 output
+// pixels, K = kh rows of 64, weights resident.
+cudaError_t launch_stem_fwd(const Problem &pb, const void *x_packed, const void *wst, const float *bias, void *out,
+                            cudaStream_t st, const BnFold *fold) {
+    int hp, wp;
+    stem_geometry(pb, &hp, &wp);
+    ConvGemm g;
+    g.ho = pb.h_out; g.wo = pb.w_out; g.cn = pb.c_out; g.ca = 64; g.taps_h = pb.kh; g.taps_w = 1;
+    g.lower_h = g.lower_w = 0; g.stride_h = g.stride_w = g.dil_h = g.dil_w = 1;
+    g.stem = 1; g.stem_tw = 16; g.stem_th = 8;
+    g.stem_tiles_w = (pb.w_out + 15) / 16; g.stem_tiles_h = (pb.h_out + 7) / 8;
+    g.p = (long long)pb.n * g.stem_tiles_h * g.stem_tiles_w * kBM;      // m-tiles x 128 (patches, ragged edges clipped)
+    g.stages = 1; g.blockdiag = 0; g.out_strided = nullptr; g.out_sn = 0; g.out_sh = g.out_sw = 0;
+    g.fold = fold ? *fold : BnFold{nullptr, nullptr, nullptr, nullptr, nullptr, 0.f, nullptr};
+    CUtensorMap ta, tw, tout;
+    {   // overlapping windows: 64 elements (8 pixels x 8 channels) starting at every output column
+        const unsigned long long dims[5] = {64, (unsigned long long)pb.w_out, (unsigned long long)pb.h_out,
+                                            (unsigned long long)pb.kh, (unsigned long long)pb.n};
+        const unsigned long long str[5] = {0, (unsigned long long)pb.stride_w * 16,
+                                           (unsigned long long)pb.stride_h * wp * 16, (unsigned long long)wp * 16,
+                                           (unsigned long long)hp * wp * 16};
+        const unsigned int box[5] = {64, 16, 8, 1, 1};
+        if (!make_tmap_tiled_bf16(&ta, x_packed, 5, dims, str, box)) return cudaErrorInvalidValue;
+    }
+    {
+        const unsigned long long dims[4] = {(unsigned long long)pb.c_out, (unsigned long long)pb.w_out,
+                                            (unsigned long long)pb.h_out, (unsigned long long)pb.n};
+        const unsigned long long str[4] = {0, (unsigned long long)pb.c_out * 2,
+                                           (unsigned long long)pb.w_out * pb.c_out * 2,
+                                           (unsigned long long)pb.h_out * pb.w_out * pb.c_out * 2};
+        const unsigned int box[4] = {64, 16, 2, 1};
+        if (!make_tmap_tiled_bf16(&tout, out, 4, dims, str, box)) return cudaErrorInvalidValue;
+    }
+    if (!make_tmap_matrix_bf16(&tw, wst, pb.c_out, (long long)pb.kh * 64, 64, kBK)) return cudaErrorInvalidValue;
+    int *err = nullptr;
+    cudaError_t e = error_word_address(&err);
+    if (e != cudaSuccess) return e;
+    return launch_bn<64>(ta, tw, tout, g, bias, err, st);
 }
 
 }  // namespace convbn
