@@ -157,6 +157,12 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
         pl.bsplits = pl.uw.splits;
         part_bytes = (size_t)pl.uw.splits * (pb.c_out / 64) * pb.kh * pb.kw * 64 * 64 * sizeof(float);
     }
+    if (pl.stem) {
+        pl.umma_wgrad = false;
+        pl.uw = stem_wgrad_plan(pb);
+        pl.bsplits = pl.uw.splits;
+        part_bytes = (size_t)pl.uw.splits * pb.kh * 64 * pb.c_out * sizeof(float);
+    }
     if (pl.umma_wgrad) {
         pl.uw = umma_wgrad_plan(pb);
         pl.bsplits = pl.uw.splits;
@@ -177,12 +183,14 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
         case CONVBN_PHASE_DEPLOY_BWD:
             pl.w_scaled = take(wbytes);
             pl.wbd = take(wbd_bytes);
+            pl.xpk = take(xpk_bytes);
             pl.partials = take(part_bytes);
             pl.bsum = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
             pl.dotpart = take(dot_bytes);
             pl.counters = take(dot_bytes ? (size_t)(pb.c_out / 32 + 1) * sizeof(unsigned int) : 0);
             break;
         case CONVBN_PHASE_TUNE_BWD_WEIGHT:
+            pl.xpk = take(xpk_bytes);
             pl.partials = take(part_bytes);
             pl.bsum = take((size_t)pl.bsplits * pb.c_out * sizeof(float));
             pl.dotpart = take(dot_bytes);
@@ -197,6 +205,7 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
             pl.dy = take((size_t)pb.p * pb.c_out * elem_size(d->dtype));
             pl.w_scaled = take(wbytes);
             pl.wbd = take(wbd_bytes);
+            pl.xpk = take(xpk_bytes);
             pl.part_g = take((size_t)pl.bn_splits * pb.c_out * sizeof(float));
             pl.bsum = take((size_t)(pl.bn_splits > pl.bsplits ? pl.bn_splits : pl.bsplits) * pb.c_out * sizeof(float));
             pl.partials = take(part_bytes);
@@ -428,10 +437,16 @@ int run_param_grads(const convbn_desc *d, const Problem &pb, const Plan &pl, con
                     float *dgamma, float *dbeta, void *ws, cudaStream_t st, const char **which) {
     float *partials = (float *)at(ws, pl.partials), *bsum = (float *)at(ws, pl.bsum);
     const bool need_bsum = vec3 || db;
-    const bool tc = pl.grouped_wgrad || pl.umma_wgrad;      // tensor-core paths sum dZ inside the GEMM
+    const bool tc = pl.grouped_wgrad || pl.umma_wgrad || pl.stem;   // tensor-core paths sum dZ inside the GEMM
     if (need_bsum && !tc)
         LAUNCH("channel_sum", launch_channel_sum_partial(pb, d->dtype, d->layout, dz, bsum, pl.bsplits, st));
-    if (pl.grouped_wgrad) {
+    if (pl.stem) {
+        LAUNCH("stem_pack", launch_stem_pack(pb, x, at(ws, pl.xpk), st));
+        LAUNCH("stem_wgrad", launch_stem_wgrad(pb, pl.uw, dz, at(ws, pl.xpk), partials, bsum, st));
+        LAUNCH("wgrad_epilogue_stem", launch_wgrad_epilogue_stem(pb, pl.uw, partials, bsum, w, vec3, b, mean, dw, db,
+                                                                 dgamma, dbeta, need_bsum, st));
+        *which = "umma-stem";
+    } else if (pl.grouped_wgrad) {
         LAUNCH("grouped_wgrad", launch_umma_wgrad(pb, pl.uw, dz, x, partials, bsum, nullptr, st));
         LAUNCH("wgrad_epilogue_bd", launch_wgrad_epilogue_bd(pb, partials, pl.uw.splits, need_bsum ? bsum : nullptr,
                                                              need_bsum ? pl.bsplits : 0, w, vec3, b, mean, dw, db,

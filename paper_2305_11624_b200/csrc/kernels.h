@@ -102,6 +102,15 @@ size_t stem_weight_bytes(const Problem &pb);                 // [C_out][kh][64] 
 cudaError_t launch_stem_pack(const Problem &pb, const void *x, void *x_packed, cudaStream_t st);
 cudaError_t launch_stem_expand_weights(const Problem &pb, const void *w, const float *s_vec, void *wst,
                                        cudaStream_t st);
+// Weight gradient of a stem layer on the packed input: partials [splits][kh * 64][C_out] (padded k rows),
+// bsum [splits][C_out]; the epilogue gathers the real kh x kw x C_in entries.
+UmmaWgradPlan stem_wgrad_plan(const Problem &pb);
+cudaError_t launch_stem_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const void *dz, const void *x_packed,
+                              float *partials, float *bsum, cudaStream_t st);
+cudaError_t launch_wgrad_epilogue_stem(const Problem &pb, const UmmaWgradPlan &pl, const float *partials,
+                                       const float *bsum, const void *w, const float *vec3, const float *b,
+                                       const float *mean, float *dw, float *db, float *dgamma, float *dbeta,
+                                       bool need_sums, cudaStream_t st);
 cudaError_t launch_stem_fwd(const Problem &pb, const void *x_packed, const void *wst, const float *bias, void *out,
                             cudaStream_t st, const BnFold *fold = nullptr);
 

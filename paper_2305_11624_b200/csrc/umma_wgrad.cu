@@ -30,6 +30,9 @@ struct WgradGemm {
     long long per_split;    // pixels per slice (multiple of 64)
     int stages;
     int blockdiag;          // grouped conv: c_in = 64 here, k rows are (tap, channel of block blockIdx.y)
+    // Small-C_in ("stem") mode: tm_x is the 5-D window view of the packed input (one 64-wide slice per
+    // filter row), tm_dz a 4-D map of dZ; a "pixel block" is a 4 x 16 patch of output pixels.
+    int stem, stem_tiles_w, stem_tiles_h;
 };
 
 struct WgradSmemCtl {
@@ -120,6 +123,19 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
             const int base_w = g.lower_w + wo0 * g.stride_w, base_h = g.lower_h + ho0 * g.stride_h;
             uint8_t *a_dst = tiles + (size_t)s * kStageBytes, *b_dst = a_dst + kABytes;
             if (lane == 0) mbar_arrive_expect_tx(&ctl->full[s], tx_bytes);
+            if (g.stem) {
+                // pixel block -> (image, patch row, patch column) of 4 x 16 output pixels
+                const uint32_t blk = (uint32_t)(p0 / kWP) + (uint32_t)kb;
+                const uint32_t t1 = blk / (uint32_t)g.stem_tiles_w;
+                const int pw = (int)(blk - t1 * (uint32_t)g.stem_tiles_w) * 16;
+                const uint32_t im = t1 / (uint32_t)g.stem_tiles_h;
+                const int phh = (int)(t1 - im * (uint32_t)g.stem_tiles_h) * 4;
+                if (lane < a_chunks)
+                    tma_load_5d(a_dst + lane * kChunkBytes, &tm_x, &ctl->full[s], 0, pw, phh, c_first + lane, (int)im);
+                else if (lane >= 2 && lane - 2 < b_chunks)
+                    tma_load_4d(b_dst + (lane - 2) * kChunkBytes, &tm_dz, &ctl->full[s], n0 + (lane - 2) * 64, pw, phh,
+                                (int)im);
+            } else
             if (lane < a_chunks)
                 tma_load_im2col_4d(a_dst + lane * kChunkBytes, &tm_x, &ctl->full[s], ci0, base_w, base_h, (int)img,
                                    off_w, off_h);
@@ -274,6 +290,7 @@ cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
     g.lower_h = -pb.pad_h; g.lower_w = -pb.pad_w; g.stride_h = pb.stride_h; g.stride_w = pb.stride_w;
     g.dil_h = pb.dil_h; g.dil_w = pb.dil_w; g.kdim = pb.kdim; g.p = pb.p; g.per_split = pl.per_split; g.stages = 1;
     g.blockdiag = pb.groups > 1 ? 1 : 0;
+    g.stem = 0; g.stem_tiles_w = g.stem_tiles_h = 1;
     if (g.blockdiag) { g.c_in = 64; g.kdim = pb.kh * pb.kw * 64; }
     const int upper_h = g.lower_h + (pb.h_out - 1) * pb.stride_h - (pb.h_in - 1);
     const int upper_w = g.lower_w + (pb.w_out - 1) * pb.stride_w - (pb.w_in - 1);
@@ -400,6 +417,123 @@ cudaError_t launch_wgrad_epilogue_fused(const Problem &pb, const UmmaWgradPlan &
     return launch_pdl(wgrad_epilogue_fused_kernel<2, 16>, grid, dim3(1024), 0, st, pb.c_out, pb.kdim, partials,
                       pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw, dotpart, counters, db,
                       dgamma, dbeta, ns);
+}
+
+// ---- small-C_in ("stem") layers -------------------------------------------------------------------
+UmmaWgradPlan stem_wgrad_plan(const Problem &pb) {
+    UmmaWgradPlan pl;
+    const int bn = wgrad_bn(pb);
+    const long long patches = (long long)pb.n * ((pb.h_out + 3) / 4) * ((pb.w_out + 15) / 16);
+    const long long m_tiles = (pb.kh + 2) / 2, n_tiles = (pb.c_out + bn - 1) / bn;
+    long long splits = (148 + m_tiles * n_tiles - 1) / (m_tiles * n_tiles);
+    if (splits > (patches + 3) / 4) splits = (patches + 3) / 4;
+    if (splits < 1) splits = 1;
+    const long long per = (patches + splits - 1) / splits;
+    pl.per_split = per * kWP;                       // in pixels of 4 x 16 patches
+    pl.splits = (int)((patches + per - 1) / per);
+    pl.kr = 8; pl.kt = 1;
+    return pl;
+}
+
+// partials: [splits][kh * 64][C_out]; bsum: [splits][C_out]
+cudaError_t launch_stem_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const void *dz, const void *x_packed,
+                              float *partials, float *bsum, cudaStream_t st) {
+    int hp, wp;
+    stem_geometry(pb, &hp, &wp);
+    WgradGemm g;
+    g.ho = pb.h_out; g.wo = pb.w_out; g.c_in = 64; g.c_out = pb.c_out; g.taps_w = 1;
+    g.lower_h = g.lower_w = 0; g.stride_h = g.stride_w = g.dil_h = g.dil_w = 1;
+    g.kdim = pb.kh * 64;
+    g.stem = 1; g.stem_tiles_w = (pb.w_out + 15) / 16; g.stem_tiles_h = (pb.h_out + 3) / 4;
+    g.p = (long long)pb.n * g.stem_tiles_h * g.stem_tiles_w * kWP;
+    g.per_split = pl.per_split; g.stages = 1; g.blockdiag = 0;
+    CUtensorMap tx, tdz;
+    {
+        const unsigned long long dims[5] = {64, (unsigned long long)pb.w_out, (unsigned long long)pb.h_out,
+                                            (unsigned long long)pb.kh, (unsigned long long)pb.n};
+        const unsigned long long str[5] = {0, (unsigned long long)pb.stride_w * 16,
+                                           (unsigned long long)pb.stride_h * wp * 16, (unsigned long long)wp * 16,
+                                           (unsigned long long)hp * wp * 16};
+        const unsigned int box[5] = {64, 16, 4, 1, 1};
+        if (!make_tmap_tiled_bf16(&tx, x_packed, 5, dims, str, box)) return cudaErrorInvalidValue;
+    }
+    {
+        const unsigned long long dims[4] = {(unsigned long long)pb.c_out, (unsigned long long)pb.w_out,
+                                            (unsigned long long)pb.h_out, (unsigned long long)pb.n};
+        const unsigned long long str[4] = {0, (unsigned long long)pb.c_out * 2,
+                                           (unsigned long long)pb.w_out * pb.c_out * 2,
+                                           (unsigned long long)pb.h_out * pb.w_out * pb.c_out * 2};
+        const unsigned int box[4] = {64, 16, 4, 1};
+        if (!make_tmap_tiled_bf16(&tdz, dz, 4, dims, str, box)) return cudaErrorInvalidValue;
+    }
+    int *err = nullptr;
+    cudaError_t e = error_word_address(&err);
+    if (e != cudaSuccess) return e;
+    Problem q = pb;
+    q.kdim = g.kdim;                                   // grid: (kh + 2) / 2 row tiles
+    const int bn = wgrad_bn(pb);
+    if (bn == 64) return launch_w<64>(tx, tdz, g, pl, q, partials, bsum, nullptr, err, st);
+    if (bn == 128) return launch_w<128>(tx, tdz, g, pl, q, partials, bsum, nullptr, err, st);
+    return launch_w<256>(tx, tdz, g, pl, q, partials, bsum, nullptr, err, st);
+}
+
+// One block per output channel: gathers the kh x kw x C_in real entries out of the kh x 64 padded rows,
+// adds the slices in order and finishes domega, db, dgamma, dbeta (Table 2, Tune row) or the plain sums.
+__global__ void __launch_bounds__(256) wgrad_epilogue_stem_kernel(int c_out, int kh, int kw, int c_in,
+                                                                 const float *__restrict__ part, int splits,
+                                                                 const float *__restrict__ bsum,
+                                                                 const __nv_bfloat16 *__restrict__ w,
+                                                                 const float *__restrict__ vec3,
+                                                                 const float *__restrict__ b,
+                                                                 const float *__restrict__ mean,
+                                                                 float *__restrict__ dw, float *__restrict__ db,
+                                                                 float *__restrict__ dgamma,
+                                                                 float *__restrict__ dbeta, int need_sums) {
+    __shared__ float red[256];
+    const int co = blockIdx.x, kdim = kh * kw * c_in;
+    const size_t slice = (size_t)kh * 64 * c_out;
+    const float s = vec3 ? vec3[co] : 1.f;
+    float dot = 0.f;
+    for (int k = threadIdx.x; k < kdim; k += blockDim.x) {
+        const int c = k % c_in, t = k / c_in, q = t % kw, r = t / kw;
+        const size_t o = ((size_t)r * 64 + q * 8 + c) * c_out + co;
+        float acc = 0.f;
+        for (int sp = 0; sp < splits; ++sp) acc += part[(size_t)sp * slice + o];
+        dw[(size_t)co * kdim + k] = s * acc;
+        if (vec3) dot = fmaf(acc, __bfloat162float(w[(size_t)co * kdim + k]), dot);
+    }
+    float bs = 0.f;
+    if (need_sums)
+        for (int sp = threadIdx.x; sp < splits; sp += blockDim.x) bs += bsum[(size_t)sp * c_out + co];
+    red[threadIdx.x] = dot;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) { if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o]; __syncthreads(); }
+    const float dot_all = red[0];
+    __syncthreads();
+    red[threadIdx.x] = bs;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) { if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o]; __syncthreads(); }
+    if (threadIdx.x == 0 && need_sums) {
+        const float dsum = red[0];
+        if (vec3) {
+            const float r = vec3[2 * c_out + co];
+            dbeta[co] = dsum;
+            if (db) db[co] = s * dsum;
+            dgamma[co] = r * (dot_all + dsum * ((b ? b[co] : 0.f) - mean[co]));
+        } else if (db) {
+            db[co] = dsum;
+        }
+    }
+}
+
+cudaError_t launch_wgrad_epilogue_stem(const Problem &pb, const UmmaWgradPlan &pl, const float *partials,
+                                       const float *bsum, const void *w, const float *vec3, const float *b,
+                                       const float *mean, float *dw, float *db, float *dgamma, float *dbeta,
+                                       bool need_sums, cudaStream_t st) {
+    wgrad_epilogue_stem_kernel<<<pb.c_out, 256, 0, st>>>(pb.c_out, pb.kh, pb.kw, pb.c_in, partials, pl.splits, bsum,
+                                                         (const __nv_bfloat16 *)w, vec3, b, mean, dw, db, dgamma, dbeta,
+                                                         need_sums ? 1 : 0);
+    return cudaGetLastError();
 }
 
 }  // namespace convbn
