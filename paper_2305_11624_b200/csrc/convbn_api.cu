@@ -348,7 +348,10 @@ int run_conv_fwd(const convbn_desc *d, const Problem &pb, const void *x, const v
 int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, const void *w, const float *scale,
                    void *w_scratch, void *wbd_scratch, void *dx, cudaStream_t st, const char **which) {
     UmmaConvShape s;
-    if (grouped_path(d, pb) && pb.stride_h == 1 && pb.stride_w == 1) {
+    if (stem_path(d, pb) && stem_dgrad_eligible(pb)) {
+        LAUNCH("stem_dgrad", launch_stem_dgrad(pb, dz, w, scale, dx, st));
+        *which = "stem-simt";
+    } else if (grouped_path(d, pb) && pb.stride_h == 1 && pb.stride_w == 1) {
         s = UmmaConvShape{pb.n, pb.h_out, pb.w_out, pb.c_out, pb.h_in, pb.w_in, pb.c_in, pb.kh, pb.kw,
                           pb.pad_h - (pb.kh - 1) * pb.dil_h, pb.pad_w - (pb.kw - 1) * pb.dil_w, 1, 1, pb.dil_h,
                           pb.dil_w, 1};

@@ -102,6 +102,10 @@ size_t stem_weight_bytes(const Problem &pb);                 // [C_out][kh][64] 
 cudaError_t launch_stem_pack(const Problem &pb, const void *x, void *x_packed, cudaStream_t st);
 cudaError_t launch_stem_expand_weights(const Problem &pb, const void *w, const float *s_vec, void *wst,
                                        cudaStream_t st);
+// Backward data of a stem layer (fp32 FMA kernel; scale folded into the weights it stages).
+bool stem_dgrad_eligible(const Problem &pb);
+cudaError_t launch_stem_dgrad(const Problem &pb, const void *dz, const void *w, const float *s_vec, void *dx,
+                              cudaStream_t st);
 // Weight gradient of a stem layer on the packed input: partials [splits][kh * 64][C_out] (padded k rows),
 // bsum [splits][C_out]; the epilogue gathers the real kh x kw x C_in entries.
 UmmaWgradPlan stem_wgrad_plan(const Problem &pb);
