@@ -94,17 +94,18 @@ cudaError_t launch_stem_expand_weights(const Problem &pb, const void *w, const f
 // layer's input gradient is rarely needed, so this is an fp32 FMA kernel: blockIdx.y is the residue
 // class (h mod stride_h, w mod stride_w), so all lanes of a warp meet the same taps and read the
 // (scaled, fp32) weights from shared memory as broadcasts; dZ is read 8 channels (16 bytes) at a time.
+template <int CP>      // channels kept per thread: C_in rounded up to 4 or 8 (weights zero-padded)
 __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_in, int c_in, int h_out, int w_out,
                                                          int c_out, int kh, int kw, int stride_h, int stride_w,
                                                          int pad_h, int pad_w, const uint4 *__restrict__ dz,
                                                          const __nv_bfloat16 *__restrict__ w,
                                                          const float *__restrict__ s_vec,
                                                          __nv_bfloat16 *__restrict__ dx) {
-    extern __shared__ float w_s[];                  // [tap][co][c_in]
+    extern __shared__ float w_s[];                  // [tap][co][CP]
     const int taps = kh * kw;
-    for (int i = threadIdx.x; i < taps * c_out * c_in; i += blockDim.x) {
-        const int c = i % c_in, t = i / c_in, co = t % c_out, tap = t / c_out;
-        w_s[i] = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((size_t)co * taps + tap) * c_in + c]);
+    for (int i = threadIdx.x; i < taps * c_out * CP; i += blockDim.x) {
+        const int c = i % CP, t = i / CP, co = t % c_out, tap = t / c_out;
+        w_s[i] = c < c_in ? (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((size_t)co * taps + tap) * c_in + c]) : 0.f;
     }
     __syncthreads();
     const int a = blockIdx.y / stride_w, b = blockIdx.y % stride_w;
@@ -118,7 +119,9 @@ __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_
         const uint32_t img = t1 / (uint32_t)hi_n;
         const int i = (int)(t1 - img * (uint32_t)hi_n);
         const int h = i * stride_h + a, wq = j * stride_w + b;
-        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        float acc[CP];
+#pragma unroll
+        for (int c = 0; c < CP; ++c) acc[c] = 0.f;
         for (int r = (a + pad_h) % stride_h; r < kh; r += stride_h) {
             const int hs = h + pad_h - r;
             if (hs < 0) break;
@@ -130,35 +133,45 @@ __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_
                 const int wo = ws / stride_w;
                 if (wo >= w_out) continue;
                 const uint4 *src = dz + ((size_t)(img * h_out + ho) * w_out + wo) * v;
-                const float *wt = w_s + (size_t)(r * kw + q) * c_out * c_in;
+                const float *wt = w_s + (size_t)(r * kw + q) * c_out * CP;
                 for (int g8 = 0; g8 < v; ++g8) {
                     const uint4 qv = __ldg(src + g8);
                     const uint32_t u[4] = {qv.x, qv.y, qv.z, qv.w};
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
                         const float d = __uint_as_float((e & 1) ? (u[e >> 1] & 0xFFFF0000u) : (u[e >> 1] << 16));
-                        const float *wc = wt + (g8 * 8 + e) * c_in;
-                        for (int c = 0; c < c_in; ++c) acc[c] = fmaf(d, wc[c], acc[c]);
+                        const float4 *wc = (const float4 *)(wt + (g8 * 8 + e) * CP);
+#pragma unroll
+                        for (int c4 = 0; c4 < CP / 4; ++c4) {
+                            const float4 wv = wc[c4];
+                            acc[4 * c4] = fmaf(d, wv.x, acc[4 * c4]); acc[4 * c4 + 1] = fmaf(d, wv.y, acc[4 * c4 + 1]);
+                            acc[4 * c4 + 2] = fmaf(d, wv.z, acc[4 * c4 + 2]); acc[4 * c4 + 3] = fmaf(d, wv.w, acc[4 * c4 + 3]);
+                        }
                     }
                 }
             }
         }
         __nv_bfloat16 *dst = dx + ((size_t)(img * h_in + h) * w_in + wq) * c_in;
-        for (int c = 0; c < c_in; ++c) dst[c] = __float2bfloat16_rn(acc[c]);
+#pragma unroll
+        for (int c = 0; c < CP; ++c)
+            if (c < c_in) dst[c] = __float2bfloat16_rn(acc[c]);
     }
 }
 
 bool stem_dgrad_eligible(const Problem &pb) {
     return stem_eligible(pb) && pb.c_out % 8 == 0 &&
-           (size_t)pb.kh * pb.kw * pb.c_out * pb.c_in * sizeof(float) <= 160 * 1024;
+           (size_t)pb.kh * pb.kw * pb.c_out * (pb.c_in <= 4 ? 4 : 8) * sizeof(float) <= 160 * 1024;
 }
 
 cudaError_t launch_stem_dgrad(const Problem &pb, const void *dz, const void *w, const float *s_vec, void *dx,
                               cudaStream_t st) {
-    const size_t smem = (size_t)pb.kh * pb.kw * pb.c_out * pb.c_in * sizeof(float);
+    const int cp = pb.c_in <= 4 ? 4 : 8;
+    const size_t smem = (size_t)pb.kh * pb.kw * pb.c_out * cp * sizeof(float);
     static bool attr = false;
     if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(stem_dgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(stem_dgrad_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(stem_dgrad_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
         if (e != cudaSuccess) return e;
         attr = true;
     }
@@ -167,9 +180,16 @@ cudaError_t launch_stem_dgrad(const Problem &pb, const void *dz, const void *w, 
     long long bx = (per_class + 255) / 256;
     if (bx > 148 * 8) bx = 148 * 8;
     dim3 grid((unsigned)bx, (unsigned)(pb.stride_h * pb.stride_w));
-    stem_dgrad_kernel<<<grid, 256, smem, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.c_out, pb.kh,
-                                               pb.kw, pb.stride_h, pb.stride_w, pb.pad_h, pb.pad_w, (const uint4 *)dz,
-                                               (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)dx);
+    if (cp == 4)
+        stem_dgrad_kernel<4><<<grid, 256, smem, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.c_out,
+                                                      pb.kh, pb.kw, pb.stride_h, pb.stride_w, pb.pad_h, pb.pad_w,
+                                                      (const uint4 *)dz, (const __nv_bfloat16 *)w, s_vec,
+                                                      (__nv_bfloat16 *)dx);
+    else
+        stem_dgrad_kernel<8><<<grid, 256, smem, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.c_out,
+                                                      pb.kh, pb.kw, pb.stride_h, pb.stride_w, pb.pad_h, pb.pad_w,
+                                                      (const uint4 *)dz, (const __nv_bfloat16 *)w, s_vec,
+                                                      (__nv_bfloat16 *)dx);
     return cudaGetLastError();
 }
 

@@ -252,7 +252,7 @@ UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
     per = (per + kWP - 1) / kWP * kWP;
     pl.per_split = per;
     pl.splits = (int)((pb.p + per - 1) / per);
-    pl.kr = pl.splits > 64 ? 2 : 8;   // k rows per epilogue block
+    pl.kr = pl.splits > 64 ? 2 : (pl.splits <= 3 ? 32 : 8);   // k rows per epilogue block
     pl.kt = (pb.kdim + pl.kr - 1) / pl.kr;   // epilogue blocks along k = rows of dotpart
     return pl;
 }
@@ -410,6 +410,10 @@ cudaError_t launch_wgrad_epilogue_fused(const Problem &pb, const UmmaWgradPlan &
     static bool carve_a = false, carve_b = false;
     prefer_max_shared_once(wgrad_epilogue_fused_kernel<8, 4>, &carve_a);
     prefer_max_shared_once(wgrad_epilogue_fused_kernel<2, 16>, &carve_b);
+    if (pl.kr == 32)
+        return launch_pdl(wgrad_epilogue_fused_kernel<32, 1>, grid, dim3(1024), 0, st, pb.c_out, pb.kdim, partials,
+                          pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw, dotpart, counters, db,
+                          dgamma, dbeta, ns);
     if (pl.kr == 8)
         return launch_pdl(wgrad_epilogue_fused_kernel<8, 4>, grid, dim3(1024), 0, st, pb.c_out, pb.kdim, partials,
                           pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw, dotpart, counters, db,
