@@ -333,6 +333,42 @@ def run_ours(args):
     for k in kernels:
         k.pop("_tag")
 
+    # ---- Tune against the Eval- and Deploy-mode paths built from the same kernels (the paper's
+    # comparison: Table 2, Fig. 3), eager calls, forward + full backward of every layer per step
+    modes = None
+    if not args.no_modes and rank == 0:
+        mblocks = [Block(sp, device=dev, modes=("tune", "eval", "deploy")) for sp in layers]
+        for li, b in enumerate(mblocks):
+            b.randomize(I.config_seed(args.workload, li) + 17)
+            b.deploy_prepare()
+
+        def run_mode(m):
+            for b in mblocks:
+                if m == "tune":
+                    b.tune_step()
+                elif m == "eval":
+                    b.eval_fwd(); b.eval_bwd()
+                else:
+                    b.deploy_fwd(); b.deploy_bwd()
+
+        modes = {}
+        ksteps = max(3, min(args.steps, 50))
+        for m in ("tune", "eval", "deploy"):
+            for _ in range(3):
+                run_mode(m)
+            torch.cuda.synchronize()
+            m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            m0.record(stream)
+            for _ in range(ksteps):
+                run_mode(m)
+            m1.record(stream)
+            torch.cuda.synchronize()
+            modes[m] = {"ms_per_step": m0.elapsed_time(m1) / ksteps,
+                        "saved_bytes": sum(b.saved_bytes(m) for b in mblocks)}
+        modes["note"] = "eager calls, %d steps each; saved_bytes = X plus what the mode keeps for backward" % ksteps
+        C.convbn_check()
+        del mblocks
+
     # ---- end to end through the host-buffer entry point ---------------------------------------
     e2e = None
     if not args.no_e2e:
@@ -363,7 +399,7 @@ def run_ours(args):
                           "note": "same steps as plain library calls with per-kernel CUDA events (source of `kernels` and `roofline`)"},
                 "clocks": sampler.summary(), "e2e": e2e,
                 "gpu_launches": sum(k["launches"] for k in kernels),
-                "roofline": roofline, "cpu_baseline": cpu, "kernels": kernels[:12],
+                "roofline": roofline, "cpu_baseline": cpu, "modes": modes, "kernels": kernels[:12],
                 "activation_bytes": {b.spec.name: {m: b.saved_bytes(m) for m in ("tune", "eval", "deploy")}
                                      for b in blocks[0]}}
         print(json.dumps(line), flush=True)
@@ -424,6 +460,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--ref-batch", type=int, default=4, help="samples per step of the reference arm")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-modes", action="store_true", help="skip the Tune / Eval / Deploy comparison")
     ap.add_argument("--no-graph", action="store_true", help="time eager library calls instead of graph replays")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

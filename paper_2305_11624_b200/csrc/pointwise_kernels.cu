@@ -351,8 +351,96 @@ __global__ void __launch_bounds__(256) bn_eval_fwd_kernel(int c_out, long long h
     }
 }
 
+// bf16 NHWC with C a multiple of 8: 16-byte vectors; the block size is a multiple of C / 8, so a thread
+// keeps its 8 channels (and their scale / shift in registers) over its grid-stride loop.
+__global__ void __launch_bounds__(256) bn_eval_fwd_nhwc8_kernel(int c_out, long long vecs, const uint4 *__restrict__ y,
+                                                                const float *__restrict__ vec3,
+                                                                uint4 *__restrict__ z) {
+    const int v = c_out / 8, cv = threadIdx.x % v;
+    float sc[8], sh[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { sc[e] = vec3[cv * 8 + e]; sh[e] = vec3[c_out + cv * 8 + e]; }
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < vecs;
+         i += (long long)gridDim.x * blockDim.x) {
+        const uint4 q = y[i];
+        const uint32_t u[4] = {q.x, q.y, q.z, q.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float a = fmaf(sc[2 * e], __uint_as_float(u[e] << 16), sh[2 * e]);
+            const float b2 = fmaf(sc[2 * e + 1], __uint_as_float(u[e] & 0xFFFF0000u), sh[2 * e + 1]);
+            const __nv_bfloat162 h = __floats2bfloat162_rn(a, b2);
+            o[e] = *(const uint32_t *)&h;
+        }
+        z[i] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+// dy = s dz and per-block partial sums of dz (y - mean) r and dz, one partial row per block
+// (Table 2, Eval row); layout and block shape as above, lanes combined per channel in thread order.
+__global__ void __launch_bounds__(256) bn_eval_bwd_nhwc8_kernel(int c_out, long long p, int pix_per_block, float eps,
+                                                                const uint4 *__restrict__ dz,
+                                                                const uint4 *__restrict__ y,
+                                                                const float *__restrict__ gamma,
+                                                                const float *__restrict__ mean,
+                                                                const float *__restrict__ var,
+                                                                uint4 *__restrict__ dy, float *__restrict__ part_g,
+                                                                float *__restrict__ part_b) {
+    __shared__ float red[256][9];
+    const int v = c_out / 8, cv = threadIdx.x % v;
+    float s8[8], r8[8], m8[8], ag[8], ab[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        const int c = cv * 8 + e;
+        r8[e] = 1.0f / sqrtf(var[c] + eps);
+        s8[e] = gamma[c] * r8[e];
+        m8[e] = mean[c];
+        ag[e] = ab[e] = 0.f;
+    }
+    const long long vec0 = (long long)blockIdx.x * pix_per_block * v;
+    long long vec1 = vec0 + (long long)pix_per_block * v;
+    if (vec1 > p * v) vec1 = p * v;
+    for (long long i = vec0 + threadIdx.x; i < vec1; i += blockDim.x) {
+        const uint4 qd = dz[i], qy = y[i];
+        const uint32_t ud[4] = {qd.x, qd.y, qd.z, qd.w}, uy[4] = {qy.x, qy.y, qy.z, qy.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float d0 = __uint_as_float(ud[e] << 16), d1 = __uint_as_float(ud[e] & 0xFFFF0000u);
+            const float y0 = __uint_as_float(uy[e] << 16), y1 = __uint_as_float(uy[e] & 0xFFFF0000u);
+            ag[2 * e] = fmaf(d0, (y0 - m8[2 * e]) * r8[2 * e], ag[2 * e]);
+            ag[2 * e + 1] = fmaf(d1, (y1 - m8[2 * e + 1]) * r8[2 * e + 1], ag[2 * e + 1]);
+            ab[2 * e] += d0;
+            ab[2 * e + 1] += d1;
+            const __nv_bfloat162 h = __floats2bfloat162_rn(s8[2 * e] * d0, s8[2 * e + 1] * d1);
+            o[e] = *(const uint32_t *)&h;
+        }
+        dy[i] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+    for (int pass = 0; pass < 2; ++pass) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) red[threadIdx.x][e] = pass ? ab[e] : ag[e];
+        __syncthreads();
+        for (int c = threadIdx.x; c < c_out; c += blockDim.x) {
+            const int g = c / 8, e = c % 8;
+            float sum = 0.f;
+            for (int th = g; th < (int)blockDim.x; th += v) sum += red[th][e];
+            (pass ? part_b : part_g)[(long long)blockIdx.x * c_out + c] = sum;
+        }
+        __syncthreads();
+    }
+}
+
 cudaError_t launch_bn_eval_fwd(const Problem &pb, int dtype, int layout, const void *y,
                                const float *vec3, void *z, cudaStream_t st) {
+    if (channel_sum_fast(pb, dtype, layout)) {
+        const int v = pb.c_out / 8, block = (256 / v) * v;
+        const long long vecs = pb.p * v;
+        long long nb = (vecs + block - 1) / block;
+        if (nb > 148 * 16) nb = 148 * 16;
+        bn_eval_fwd_nhwc8_kernel<<<(int)nb, block, 0, st>>>(pb.c_out, vecs, (const uint4 *)y, vec3, (uint4 *)z);
+        return cudaGetLastError();
+    }
     const long long total = pb.p * pb.c_out, hw = (long long)pb.h_out * pb.w_out;
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 32) blocks = 148 * 32;
@@ -399,6 +487,14 @@ __global__ void __launch_bounds__(256) bn_eval_bwd_kernel(int c_out, int h_out, 
 cudaError_t launch_bn_eval_bwd(const Problem &pb, int dtype, int layout, const void *dz, const void *y,
                                const float *gamma, const float *mean, const float *var, void *dy,
                                float *part_g, float *part_b, int splits, cudaStream_t st) {
+    if (channel_sum_fast(pb, dtype, layout)) {
+        const int v = pb.c_out / 8, block = (256 / v) * v;
+        const long long per = (pb.p + splits - 1) / splits;
+        bn_eval_bwd_nhwc8_kernel<<<splits, block, 0, st>>>(pb.c_out, pb.p, (int)per, pb.eps, (const uint4 *)dz,
+                                                           (const uint4 *)y, gamma, mean, var, (uint4 *)dy, part_g,
+                                                           part_b);
+        return cudaGetLastError();
+    }
     const int threads = pb.c_out >= 256 ? 256 : ((pb.c_out + 31) / 32) * 32;
     dim3 grid((pb.c_out + threads - 1) / threads, splits);
     if (dtype == CONVBN_F32 && layout == CONVBN_NCHW)
