@@ -5,7 +5,9 @@ import numpy as np
 from oracle import oracle as O
 from paper_2305_11624_b200 import inputs as I
 
-# spec tolerances: relative L2 per output tensor against the fp64 oracle
+# Tolerances: relative L2 per output tensor against the fp64 oracle.  bf16: inputs, omega' (backward
+# data) and outputs are each rounded once to 8 mantissa bits (2^-9 = 2e-3 rms-ish each) -> 5e-3;
+# fp32: sums of <= a few thousand products in fp32 -> 1e-5.
 TOL = {"bf16": 5e-3, "f32": 1e-5}
 
 
