@@ -252,15 +252,10 @@ UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
     per = (per + kWP - 1) / kWP * kWP;
     pl.per_split = per;
     pl.splits = (int)((pb.p + per - 1) / per);
-    // k rows per epilogue block (the block's other 32 / kr lanes split the slices): the tallest block
-    // that still gives about two blocks per SM, with no more slice lanes than slices
-    pl.kr = 2;
-    const int cand[3] = {32, 8, 2};
-    for (int i = 0; i < 3; ++i) {
-        const int kr = cand[i], sl = 32 / kr;
-        if (sl > pl.splits && kr != 32) continue;
-        if ((long long)(pb.c_out / 32) * ((pb.kdim + kr - 1) / kr) >= 296 || kr == 2) { pl.kr = kr; break; }
-    }
+    // k rows per epilogue block (the block's other lanes split the slices): many slices -> 2 rows x 16
+    // lanes; few slices or very many blocks -> 32 rows x 1 lane (every block pays a fence and an atomic)
+    const long long blocks8 = (long long)(pb.c_out / 32) * ((pb.kdim + 7) / 8);
+    pl.kr = pl.splits > 64 ? 2 : ((pl.splits <= 8 || blocks8 > 1200) && blocks8 / 4 >= 148 ? 32 : 8);
     pl.kt = (pb.kdim + pl.kr - 1) / pl.kr;   // epilogue blocks along k = rows of dotpart
     return pl;
 }
