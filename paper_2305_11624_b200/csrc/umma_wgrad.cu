@@ -372,9 +372,9 @@ __global__ void __launch_bounds__(1024) wgrad_epilogue_fused_kernel(
     }
     if (!need_sums) return;
     // ---- last block of this channel group finishes the per-channel quantities ----
-    __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
+        __threadfence();        // after the barrier: orders the whole block's dw / dotpart writes before the count
         const unsigned int done = atomicAdd(&counters[blockIdx.x], 1u);
         is_last = (done == gridDim.y - 1);
     }
