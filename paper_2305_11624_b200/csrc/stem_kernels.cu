@@ -91,105 +91,157 @@ cudaError_t launch_stem_expand_weights(const Problem &pb, const void *w, const f
 // ---- backward data of a stem layer (plain ALUs) ---------------------------------------------------
 // dX[n,h,w,c] = sum over the taps that reach (h, w) and over co of omega'[co,r,q,c] dZ[n,ho,wo,co]
 // (Sec. 3.2.1).  With C_in <= 8 the GEMM N dimension is too narrow for the tensor cores, and the first
-// layer's input gradient is rarely needed, so this is an fp32 FMA kernel: blockIdx.y is the residue
-// class (h mod stride_h, w mod stride_w), so all lanes of a warp meet the same taps and read the
-// (scaled, fp32) weights from shared memory as broadcasts; dZ is read 8 channels (16 bytes) at a time.
-template <int CP>      // channels kept per thread: C_in rounded up to 4 or 8 (weights zero-padded)
+// layer's input gradient is rarely needed, so this is an fp32 FMA kernel.  blockIdx.y is the residue
+// class (h mod stride_h, w mod stride_w), so every lane meets the same taps.  Eight lanes share one
+// pixel: lane l of the eight takes the 8-channel chunks l, l+8, ... of dZ, so that a warp's 16-byte
+// loads cover four pixels' contiguous 128 bytes, and the eight partial sums meet in a butterfly.  The
+// (scaled, fp32) weights sit in shared memory as [tap][chunk/8][channel in chunk][chunk%8][CP], which
+// puts the eight lanes' 16-byte reads side by side.
+template <int CP, int CIN, int PX>   // CP: floats per weight vector (4 or 8); CIN: channels accumulated (<= CP);
+                                     // PX: pixels of one row and class per thread, which share each weight read
 __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_in, int c_in, int h_out, int w_out,
                                                          int c_out, int kh, int kw, int stride_h, int stride_w,
                                                          int pad_h, int pad_w, const uint4 *__restrict__ dz,
                                                          const __nv_bfloat16 *__restrict__ w,
                                                          const float *__restrict__ s_vec,
                                                          __nv_bfloat16 *__restrict__ dx) {
-    extern __shared__ float w_s[];                  // [tap][co][CP]
+    extern __shared__ float w_s[];
     const int taps = kh * kw;
-    for (int i = threadIdx.x; i < taps * c_out * CP; i += blockDim.x) {
-        const int c = i % CP, t = i / CP, co = t % c_out, tap = t / c_out;
-        w_s[i] = c < c_in ? (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((size_t)co * taps + tap) * c_in + c]) : 0.f;
+    const int v = c_out / 8, vo = (v + 7) / 8;
+    for (int i = threadIdx.x; i < taps * vo * 64 * CP; i += blockDim.x) {
+        const int c = i % CP;
+        int t = i / CP;
+        const int l = t % 8;
+        t /= 8;
+        const int e = t % 8;
+        t /= 8;
+        const int go = t % vo, tap = t / vo;
+        const int co = (go * 8 + l) * 8 + e;
+        w_s[i] = (co < c_out && c < c_in)
+                     ? (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((size_t)co * taps + tap) * c_in + c])
+                     : 0.f;
     }
     __syncthreads();
     const int a = blockIdx.y / stride_w, b = blockIdx.y % stride_w;
     if (a >= h_in || b >= w_in) return;
     const int hi_n = (h_in - a + stride_h - 1) / stride_h, wj_n = (w_in - b + stride_w - 1) / stride_w;
-    const uint32_t total = (uint32_t)n * hi_n * wj_n;
-    const int v = c_out / 8;
-    for (uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
-        const uint32_t t1 = idx / (uint32_t)wj_n;
-        const int j = (int)(idx - t1 * (uint32_t)wj_n);
+    const int wq_n = (wj_n + PX - 1) / PX;                     // groups of PX pixels along a row
+    const uint32_t total = (uint32_t)n * hi_n * wq_n;
+    const int l8 = threadIdx.x & 7;
+    const uint32_t gpb = blockDim.x >> 3;                      // pixel groups per block and pass
+    const int r0 = (a + pad_h) % stride_h, q0 = (b + pad_w) % stride_w;
+    const size_t tap_floats = (size_t)vo * 64 * CP;
+    for (uint32_t base = blockIdx.x * gpb; base < total; base += gridDim.x * gpb) {
+        uint32_t idx = base + (threadIdx.x >> 3);
+        const bool live = idx < total;
+        if (!live) idx = total - 1;                            // keeps the whole warp in the butterfly
+        const uint32_t t1 = idx / (uint32_t)wq_n;
+        const int j = (int)(idx - t1 * (uint32_t)wq_n) * PX;
         const uint32_t img = t1 / (uint32_t)hi_n;
         const int i = (int)(t1 - img * (uint32_t)hi_n);
         const int h = i * stride_h + a, wq = j * stride_w + b;
-        float acc[CP];
+        float acc[PX][CIN];
 #pragma unroll
-        for (int c = 0; c < CP; ++c) acc[c] = 0.f;
-        for (int r = (a + pad_h) % stride_h; r < kh; r += stride_h) {
-            const int hs = h + pad_h - r;
-            if (hs < 0) break;
-            const int ho = hs / stride_h;
-            if (ho >= h_out) continue;
-            for (int q = (b + pad_w) % stride_w; q < kw; q += stride_w) {
-                const int ws = wq + pad_w - q;
-                if (ws < 0) break;
-                const int wo = ws / stride_w;
-                if (wo >= w_out) continue;
-                const uint4 *src = dz + ((size_t)(img * h_out + ho) * w_out + wo) * v;
-                const float *wt = w_s + (size_t)(r * kw + q) * c_out * CP;
-                for (int g8 = 0; g8 < v; ++g8) {
-                    const uint4 qv = __ldg(src + g8);
-                    const uint32_t u[4] = {qv.x, qv.y, qv.z, qv.w};
+        for (int p = 0; p < PX; ++p)
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const float d = __uint_as_float((e & 1) ? (u[e >> 1] & 0xFFFF0000u) : (u[e >> 1] << 16));
-                        const float4 *wc = (const float4 *)(wt + (g8 * 8 + e) * CP);
+            for (int c = 0; c < CIN; ++c) acc[p][c] = 0.f;
+        for (int g8 = l8; g8 < v; g8 += 8) {
+            const float *wg = w_s + ((size_t)(g8 >> 3) * 64 + l8) * CP;
+            for (int r = r0; r < kh; r += stride_h) {
+                // h + pad_h - r and wq + pad_w - q are multiples of the stride inside a class, also when negative
+                const int ho = (h + pad_h - r) / stride_h;
+                if (ho < 0 || ho >= h_out) continue;
+                const uint4 *row = dz + ((size_t)(img * h_out + ho) * w_out) * v + g8;
+                for (int qb = q0; qb < kw; qb += 4 * stride_w) {
+                    // Four taps of one kernel row at a time: tap u of them pairs pixel p with output column
+                    // wo0 - u + p, so the PX + 3 columns from wo0 - 3 on serve all four taps.
+                    const int wo0 = (wq + pad_w - qb) / stride_w;
+                    const int nu = min(4, (kw - qb + stride_w - 1) / stride_w);
+                    uint4 win[PX + 3];
 #pragma unroll
-                        for (int c4 = 0; c4 < CP / 4; ++c4) {
-                            const float4 wv = wc[c4];
-                            acc[4 * c4] = fmaf(d, wv.x, acc[4 * c4]); acc[4 * c4 + 1] = fmaf(d, wv.y, acc[4 * c4 + 1]);
-                            acc[4 * c4 + 2] = fmaf(d, wv.z, acc[4 * c4 + 2]); acc[4 * c4 + 3] = fmaf(d, wv.w, acc[4 * c4 + 3]);
+                    for (int k = 0; k < PX + 3; ++k) {
+                        const int wk = wo0 - 3 + k;
+                        win[k] = (k >= 4 - nu && wk >= 0 && wk < w_out) ? __ldg(row + (size_t)wk * v)
+                                                                         : make_uint4(0u, 0u, 0u, 0u);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (u < nu) {                          // the same for every lane
+                            const float *wt = wg + (size_t)(r * kw + qb + u * stride_w) * tap_floats;
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                const float4 *wc = (const float4 *)(wt + e * 8 * CP);
+                                float wv[CP];
+#pragma unroll
+                                for (int c4 = 0; c4 < CP / 4; ++c4) {
+                                    const float4 f = wc[c4];
+                                    wv[4 * c4] = f.x; wv[4 * c4 + 1] = f.y; wv[4 * c4 + 2] = f.z; wv[4 * c4 + 3] = f.w;
+                                }
+#pragma unroll
+                                for (int p = 0; p < PX; ++p) {
+                                    const uint4 &qv = win[p - u + 3];
+                                    const uint32_t word = e < 2 ? qv.x : e < 4 ? qv.y : e < 6 ? qv.z : qv.w;
+                                    const float d = __uint_as_float((e & 1) ? (word & 0xFFFF0000u) : (word << 16));
+#pragma unroll
+                                    for (int c = 0; c < CIN; ++c) acc[p][c] = fmaf(d, wv[c], acc[p][c]);
+                                }
+                            }
                         }
                     }
                 }
             }
         }
-        __nv_bfloat16 *dst = dx + ((size_t)(img * h_in + h) * w_in + wq) * c_in;
 #pragma unroll
-        for (int c = 0; c < CP; ++c)
-            if (c < c_in) dst[c] = __float2bfloat16_rn(acc[c]);
+        for (int p = 0; p < PX; ++p) {
+            float mine = 0.f;
+#pragma unroll
+            for (int c = 0; c < CIN; ++c) {
+                float t = acc[p][c];
+                t += __shfl_xor_sync(0xFFFFFFFFu, t, 1);
+                t += __shfl_xor_sync(0xFFFFFFFFu, t, 2);
+                t += __shfl_xor_sync(0xFFFFFFFFu, t, 4);
+                if (l8 == c) mine = t;
+            }
+            if (live && j + p < wj_n && l8 < c_in)
+                dx[((size_t)(img * h_in + h) * w_in + wq + p * stride_w) * c_in + l8] = __float2bfloat16_rn(mine);
+        }
     }
 }
 
 bool stem_dgrad_eligible(const Problem &pb) {
     return stem_eligible(pb) && pb.c_out % 8 == 0 &&
-           (size_t)pb.kh * pb.kw * pb.c_out * (pb.c_in <= 4 ? 4 : 8) * sizeof(float) <= 160 * 1024;
+           (size_t)pb.kh * pb.kw * ((pb.c_out / 8 + 7) / 8) * 64 * (pb.c_in <= 4 ? 4 : 8) * sizeof(float) <= 160 * 1024;
 }
 
 cudaError_t launch_stem_dgrad(const Problem &pb, const void *dz, const void *w, const float *s_vec, void *dx,
                               cudaStream_t st) {
     const int cp = pb.c_in <= 4 ? 4 : 8;
-    const size_t smem = (size_t)pb.kh * pb.kw * pb.c_out * cp * sizeof(float);
+    const int vo = (pb.c_out / 8 + 7) / 8;
+    const size_t smem = (size_t)pb.kh * pb.kw * vo * 64 * cp * sizeof(float);
     static bool attr = false;
     if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(stem_dgrad_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(stem_dgrad_kernel<4, 3, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(stem_dgrad_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+            e = cudaFuncSetAttribute(stem_dgrad_kernel<4, 4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(stem_dgrad_kernel<8, 8, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
         if (e != cudaSuccess) return e;
         attr = true;
     }
     const long long per_class = (long long)pb.n * ((pb.h_in + pb.stride_h - 1) / pb.stride_h) *
                                 ((pb.w_in + pb.stride_w - 1) / pb.stride_w);
-    long long bx = (per_class + 255) / 256;
-    if (bx > 148 * 8) bx = 148 * 8;
+    long long bx = (per_class + 63) / 64;                      // at least 64 pixels per block and pass
+    if (bx > 148 * 4) bx = 148 * 4;
     dim3 grid((unsigned)bx, (unsigned)(pb.stride_h * pb.stride_w));
-    if (cp == 4)
-        stem_dgrad_kernel<4><<<grid, 256, smem, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.c_out,
-                                                      pb.kh, pb.kw, pb.stride_h, pb.stride_w, pb.pad_h, pb.pad_w,
-                                                      (const uint4 *)dz, (const __nv_bfloat16 *)w, s_vec,
-                                                      (__nv_bfloat16 *)dx);
-    else
-        stem_dgrad_kernel<8><<<grid, 256, smem, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.c_out,
-                                                      pb.kh, pb.kw, pb.stride_h, pb.stride_w, pb.pad_h, pb.pad_w,
-                                                      (const uint4 *)dz, (const __nv_bfloat16 *)w, s_vec,
-                                                      (__nv_bfloat16 *)dx);
+#define CONVBN_STEM_DGRAD(CP_, CIN_, PX_)                                                                           \
+    stem_dgrad_kernel<CP_, CIN_, PX_><<<grid, 256, smem, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out,     \
+                                                          pb.c_out, pb.kh, pb.kw, pb.stride_h, pb.stride_w,        \
+                                                          pb.pad_h, pb.pad_w, (const uint4 *)dz,                   \
+                                                          (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)dx)
+    if (pb.c_in == 3) CONVBN_STEM_DGRAD(4, 3, 8);
+    else if (cp == 4) CONVBN_STEM_DGRAD(4, 4, 4);
+    else CONVBN_STEM_DGRAD(8, 8, 4);
+#undef CONVBN_STEM_DGRAD
     return cudaGetLastError();
 }
 
