@@ -91,14 +91,15 @@ cudaError_t launch_stem_expand_weights(const Problem &pb, const void *w, const f
 // ---- backward data of a stem layer (plain ALUs) ---------------------------------------------------
 // dX[n,h,w,c] = sum over the taps that reach (h, w) and over co of omega'[co,r,q,c] dZ[n,ho,wo,co]
 // (Sec. 3.2.1).  With C_in <= 8 the GEMM N dimension is too narrow for the tensor cores, and the first
-// layer's input gradient is rarely needed, so this is an fp32 FMA kernel.  blockIdx.y is the residue
-// class (h mod stride_h, w mod stride_w), so every lane meets the same taps.  Eight lanes share one
-// pixel: lane l of the eight takes the 8-channel chunks l, l+8, ... of dZ, so that a warp's 16-byte
-// loads cover four pixels' contiguous 128 bytes, and the eight partial sums meet in a butterfly.  The
-// (scaled, fp32) weights sit in shared memory as [tap][chunk/8][channel in chunk][chunk%8][CP], which
-// puts the eight lanes' 16-byte reads side by side.
-template <int CP, int CIN, int PX>   // CP: floats per weight vector (4 or 8); CIN: channels accumulated (<= CP);
-                                     // PX: pixels of one row and class per thread, which share each weight read
+// layer's input gradient is rarely needed, so this is an fp32 FMA kernel.  A block works on one
+// residue class (h mod stride_h, w mod stride_w) at a time, so every lane meets the same taps.  Eight
+// lanes share a group of PX pixels of one row: lane l of the eight takes the 8-channel chunks l, l+8,
+// ... of dZ, so that a warp's 16-byte loads cover contiguous 128-byte pixels, and the eight partial
+// sums meet in a butterfly.  The (scaled, fp32) weights sit in shared memory as
+// [tap][chunk/8][channel in chunk][chunk%8][CP], which puts the eight lanes' 16-byte reads side by side;
+// each weight read serves PX pixels, and the PX + 3 columns of dZ that four taps of a kernel row need
+// are loaded and widened to fp32 once for all four.
+template <int CP, int CIN, int PX>   // CP: floats per weight vector (4 or 8); CIN: channels accumulated (<= CP)
 __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_in, int c_in, int h_out, int w_out,
                                                          int c_out, int kh, int kw, int stride_h, int stride_w,
                                                          int pad_h, int pad_w, const uint4 *__restrict__ dz,
@@ -108,6 +109,7 @@ __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_
     extern __shared__ float w_s[];
     const int taps = kh * kw;
     const int v = c_out / 8, vo = (v + 7) / 8;
+#pragma unroll 8
     for (int i = threadIdx.x; i < taps * vo * 64 * CP; i += blockDim.x) {
         const int c = i % CP;
         int t = i / CP;
@@ -122,16 +124,28 @@ __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_
                      : 0.f;
     }
     __syncthreads();
-    const int a = blockIdx.y / stride_w, b = blockIdx.y % stride_w;
-    if (a >= h_in || b >= w_in) return;
-    const int hi_n = (h_in - a + stride_h - 1) / stride_h, wj_n = (w_in - b + stride_w - 1) / stride_w;
-    const int wq_n = (wj_n + PX - 1) / PX;                     // groups of PX pixels along a row
-    const uint32_t total = (uint32_t)n * hi_n * wq_n;
     const int l8 = threadIdx.x & 7;
     const uint32_t gpb = blockDim.x >> 3;                      // pixel groups per block and pass
-    const int r0 = (a + pad_h) % stride_h, q0 = (b + pad_w) % stride_w;
     const size_t tap_floats = (size_t)vo * 64 * CP;
-    for (uint32_t base = blockIdx.x * gpb; base < total; base += gridDim.x * gpb) {
+    // Work items are (pass of gpb pixel groups, residue class).  A block owns a contiguous run of
+    // passes and visits every class of a pass before the next pass: the classes of one pass, and
+    // neighbouring passes, read the same rows of dZ, and every block meets the classes equally often
+    // although they have different tap counts.
+    const int wq_max = ((w_in + stride_w - 1) / stride_w + PX - 1) / PX;
+    const uint32_t ipc = ((uint32_t)n * ((h_in + stride_h - 1) / stride_h) * wq_max + gpb - 1) / gpb;
+    const uint32_t ncls = (uint32_t)(stride_h * stride_w);
+    const uint32_t run = (ipc + gridDim.x - 1) / gridDim.x;
+    const uint32_t pass_end = min(ipc, (blockIdx.x + 1) * run);
+    for (uint32_t item = blockIdx.x * run * ncls; item < pass_end * ncls; ++item) {
+        const int cls = (int)(item % ncls);
+        const uint32_t base = (item / ncls) * gpb;
+        const int a = cls / stride_w, b = cls % stride_w;
+        if (a >= h_in || b >= w_in) continue;
+        const int hi_n = (h_in - a + stride_h - 1) / stride_h, wj_n = (w_in - b + stride_w - 1) / stride_w;
+        const int wq_n = (wj_n + PX - 1) / PX;                 // groups of PX pixels along a row
+        const uint32_t total = (uint32_t)n * hi_n * wq_n;
+        if (base >= total) continue;
+        const int r0 = (a + pad_h) % stride_h, q0 = (b + pad_w) % stride_w;
         uint32_t idx = base + (threadIdx.x >> 3);
         const bool live = idx < total;
         if (!live) idx = total - 1;                            // keeps the whole warp in the butterfly
@@ -164,13 +178,20 @@ __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_
                         win[k] = (k >= 4 - nu && wk >= 0 && wk < w_out) ? __ldg(row + (size_t)wk * v)
                                                                          : make_uint4(0u, 0u, 0u, 0u);
                     }
+                    const float *wt = wg + (size_t)(r * kw + qb) * tap_floats;
+                    const size_t tap_step = (size_t)stride_w * tap_floats;
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        if (u < nu) {                          // the same for every lane
-                            const float *wt = wg + (size_t)(r * kw + qb + u * stride_w) * tap_floats;
+                    for (int e = 0; e < 8; ++e) {              // channel e of the lane's chunk, widened once
+                        float d[PX + 3];
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) {
-                                const float4 *wc = (const float4 *)(wt + e * 8 * CP);
+                        for (int k = 0; k < PX + 3; ++k) {
+                            const uint32_t word = e < 2 ? win[k].x : e < 4 ? win[k].y : e < 6 ? win[k].z : win[k].w;
+                            d[k] = __uint_as_float((e & 1) ? (word & 0xFFFF0000u) : (word << 16));
+                        }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            if (u < nu) {                      // the same for every lane
+                                const float4 *wc = (const float4 *)(wt + u * tap_step + e * 8 * CP);
                                 float wv[CP];
 #pragma unroll
                                 for (int c4 = 0; c4 < CP / 4; ++c4) {
@@ -178,13 +199,9 @@ __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_
                                     wv[4 * c4] = f.x; wv[4 * c4 + 1] = f.y; wv[4 * c4 + 2] = f.z; wv[4 * c4 + 3] = f.w;
                                 }
 #pragma unroll
-                                for (int p = 0; p < PX; ++p) {
-                                    const uint4 &qv = win[p - u + 3];
-                                    const uint32_t word = e < 2 ? qv.x : e < 4 ? qv.y : e < 6 ? qv.z : qv.w;
-                                    const float d = __uint_as_float((e & 1) ? (word & 0xFFFF0000u) : (word << 16));
+                                for (int p = 0; p < PX; ++p)
 #pragma unroll
-                                    for (int c = 0; c < CIN; ++c) acc[p][c] = fmaf(d, wv[c], acc[p][c]);
-                                }
+                                    for (int c = 0; c < CIN; ++c) acc[p][c] = fmaf(d[p - u + 3], wv[c], acc[p][c]);
                             }
                         }
                     }
@@ -228,11 +245,8 @@ cudaError_t launch_stem_dgrad(const Problem &pb, const void *dz, const void *w, 
         if (e != cudaSuccess) return e;
         attr = true;
     }
-    const long long per_class = (long long)pb.n * ((pb.h_in + pb.stride_h - 1) / pb.stride_h) *
-                                ((pb.w_in + pb.stride_w - 1) / pb.stride_w);
-    long long bx = (per_class + 63) / 64;                      // at least 64 pixels per block and pass
-    if (bx > 148 * 4) bx = 148 * 4;
-    dim3 grid((unsigned)bx, (unsigned)(pb.stride_h * pb.stride_w));
+    const long long passes = ((long long)pb.n * pb.h_in * pb.w_in + 63) / 64;
+    const unsigned grid = (unsigned)(passes < 148 * 2 ? passes : 148 * 2);   // two resident blocks per SM
 #define CONVBN_STEM_DGRAD(CP_, CIN_, PX_)                                                                           \
     stem_dgrad_kernel<CP_, CIN_, PX_><<<grid, 256, smem, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out,     \
                                                           pb.c_out, pb.kh, pb.kw, pb.stride_h, pb.stride_w,        \
