@@ -88,174 +88,164 @@ cudaError_t launch_stem_expand_weights(const Problem &pb, const void *w, const f
     return cudaGetLastError();
 }
 
-// ---- backward data of a stem layer (plain ALUs) ---------------------------------------------------
+// ---- backward data of a stem layer ------------------------------------------------------------------
 // dX[n,h,w,c] = sum over the taps that reach (h, w) and over co of omega'[co,r,q,c] dZ[n,ho,wo,co]
-// (Sec. 3.2.1).  With C_in <= 8 the GEMM N dimension is too narrow for the tensor cores, and the first
-// layer's input gradient is rarely needed, so this is an fp32 FMA kernel.  A block works on one
-// residue class (h mod stride_h, w mod stride_w) at a time, so every lane meets the same taps.  Eight
-// lanes share a group of PX pixels of one row: lane l of the eight takes the 8-channel chunks l, l+8,
-// ... of dZ, so that a warp's 16-byte loads cover contiguous 128-byte pixels, and the eight partial
-// sums meet in a butterfly.  The (scaled, fp32) weights sit in shared memory as
-// [tap][chunk/8][channel in chunk][chunk%8][CP], which puts the eight lanes' 16-byte reads side by side;
-// each weight read serves PX pixels, and the PX + 3 columns of dZ that four taps of a kernel row need
-// are loaded and widened to fp32 once for all four.
-template <int CP, int CIN, int PX>   // CP: floats per weight vector (4 or 8); CIN: channels accumulated (<= CP)
+// (Sec. 3.2.1).  As a GEMM this has N = C_in <= 8 columns: too narrow for a 128-row tcgen05 tile (its
+// smallest N is 16, and the A operand would stream through shared memory once per tap), so the kernel
+// uses warp-level m16n8k16 MMAs with fp32 accumulation instead.  One MMA tile is 16 consecutive pixels
+// of one row and one residue class (h mod stride_h, w mod stride_w), so that all of them meet the same
+// taps; K runs over 64 output channels per tap.  The contraction order over the channels is free as
+// long as A and B agree, which lets every lane fetch its A fragments with 16-byte loads straight from
+// dZ: lane (g, t) reads 8-channel chunks t and t + 4 of pixels g and g + 8, and k-step k takes word k
+// of each chunk.  The B fragments (the scaled weights, rounded to bf16) are laid out in shared memory
+// in exactly that order, one 32-bit word per lane and fragment register.
+__device__ __forceinline__ void mma_16x8x16_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                 uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+constexpr int STEM_DG_TILES = 2;     // 16-pixel tiles per warp and pass; they share the B fragments
+
 __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_in, int c_in, int h_out, int w_out,
                                                          int c_out, int kh, int kw, int stride_h, int stride_w,
                                                          int pad_h, int pad_w, const uint4 *__restrict__ dz,
                                                          const __nv_bfloat16 *__restrict__ w,
                                                          const float *__restrict__ s_vec,
                                                          __nv_bfloat16 *__restrict__ dx) {
-    extern __shared__ float w_s[];
+    extern __shared__ uint32_t wfrag[];    // [tap][64-channel block][k-step][b0/b1][lane]
     const int taps = kh * kw;
-    const int v = c_out / 8, vo = (v + 7) / 8;
-#pragma unroll 8
-    for (int i = threadIdx.x; i < taps * vo * 64 * CP; i += blockDim.x) {
-        const int c = i % CP;
-        int t = i / CP;
-        const int l = t % 8;
-        t /= 8;
-        const int e = t % 8;
-        t /= 8;
-        const int go = t % vo, tap = t / vo;
-        const int co = (go * 8 + l) * 8 + e;
-        w_s[i] = (co < c_out && c < c_in)
-                     ? (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((size_t)co * taps + tap) * c_in + c])
-                     : 0.f;
+    const int ncb = c_out / 64, v = c_out / 8;
+#pragma unroll 4
+    for (int i = threadIdx.x; i < taps * ncb * 256; i += blockDim.x) {
+        const int t = i & 3, g = (i >> 2) & 7, which = (i >> 5) & 1, k = (i >> 6) & 3;
+        const int cb = (i >> 8) % ncb, tap = (i >> 8) / ncb;
+        const int co = cb * 64 + which * 32 + 8 * t + 2 * k;
+        uint32_t word = 0u;
+        if (g < c_in) {
+            const float w0 = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((size_t)co * taps + tap) * c_in + g]);
+            const float w1 =
+                (s_vec ? s_vec[co + 1] : 1.f) * __bfloat162float(w[((size_t)(co + 1) * taps + tap) * c_in + g]);
+            word = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(w0)) |
+                   ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(w1)) << 16);
+        }
+        wfrag[i] = word;
     }
     __syncthreads();
-    const int l8 = threadIdx.x & 7;
-    const uint32_t gpb = blockDim.x >> 3;                      // pixel groups per block and pass
-    const size_t tap_floats = (size_t)vo * 64 * CP;
-    // Work items are (pass of gpb pixel groups, residue class).  A block owns a contiguous run of
-    // passes and visits every class of a pass before the next pass: the classes of one pass, and
-    // neighbouring passes, read the same rows of dZ, and every block meets the classes equally often
-    // although they have different tap counts.
-    const int wq_max = ((w_in + stride_w - 1) / stride_w + PX - 1) / PX;
-    const uint32_t ipc = ((uint32_t)n * ((h_in + stride_h - 1) / stride_h) * wq_max + gpb - 1) / gpb;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const uint32_t tpp = (blockDim.x >> 5) * STEM_DG_TILES;    // tiles per block and pass
+    // Work items are (pass of tpp tiles, residue class).  A block owns a contiguous run of passes and
+    // visits every class of a pass before the next pass: the classes of one pass, and neighbouring
+    // passes, read the same rows of dZ, and every block meets the classes equally often although they
+    // have different tap counts.
+    const int wt_max = ((w_in + stride_w - 1) / stride_w + 15) / 16;
+    const uint32_t ipc = ((uint32_t)n * ((h_in + stride_h - 1) / stride_h) * wt_max + tpp - 1) / tpp;
     const uint32_t ncls = (uint32_t)(stride_h * stride_w);
     const uint32_t run = (ipc + gridDim.x - 1) / gridDim.x;
     const uint32_t pass_end = min(ipc, (blockIdx.x + 1) * run);
     for (uint32_t item = blockIdx.x * run * ncls; item < pass_end * ncls; ++item) {
         const int cls = (int)(item % ncls);
-        const uint32_t base = (item / ncls) * gpb;
         const int a = cls / stride_w, b = cls % stride_w;
         if (a >= h_in || b >= w_in) continue;
         const int hi_n = (h_in - a + stride_h - 1) / stride_h, wj_n = (w_in - b + stride_w - 1) / stride_w;
-        const int wq_n = (wj_n + PX - 1) / PX;                 // groups of PX pixels along a row
-        const uint32_t total = (uint32_t)n * hi_n * wq_n;
-        if (base >= total) continue;
+        const int wt_n = (wj_n + 15) / 16;                     // tiles along a row
+        const uint32_t total = (uint32_t)n * hi_n * wt_n;
         const int r0 = (a + pad_h) % stride_h, q0 = (b + pad_w) % stride_w;
-        uint32_t idx = base + (threadIdx.x >> 3);
-        const bool live = idx < total;
-        if (!live) idx = total - 1;                            // keeps the whole warp in the butterfly
-        const uint32_t t1 = idx / (uint32_t)wq_n;
-        const int j = (int)(idx - t1 * (uint32_t)wq_n) * PX;
-        const uint32_t img = t1 / (uint32_t)hi_n;
-        const int i = (int)(t1 - img * (uint32_t)hi_n);
-        const int h = i * stride_h + a, wq = j * stride_w + b;
-        float acc[PX][CIN];
+        bool live[STEM_DG_TILES];
+        int img[STEM_DG_TILES], h[STEM_DG_TILES], j0[STEM_DG_TILES];
+        float acc[STEM_DG_TILES][4];
 #pragma unroll
-        for (int p = 0; p < PX; ++p)
+        for (int tl = 0; tl < STEM_DG_TILES; ++tl) {
+            const uint32_t idx = (item / ncls) * tpp + warp * STEM_DG_TILES + tl;
+            live[tl] = idx < total;
+            const uint32_t id = live[tl] ? idx : 0u;
+            const uint32_t t1 = id / (uint32_t)wt_n;
+            j0[tl] = (int)(id - t1 * (uint32_t)wt_n) * 16;
+            img[tl] = (int)(t1 / (uint32_t)hi_n);
+            h[tl] = (int)(t1 - (uint32_t)img[tl] * (uint32_t)hi_n) * stride_h + a;
 #pragma unroll
-            for (int c = 0; c < CIN; ++c) acc[p][c] = 0.f;
-        for (int g8 = l8; g8 < v; g8 += 8) {
-            const float *wg = w_s + ((size_t)(g8 >> 3) * 64 + l8) * CP;
+            for (int c = 0; c < 4; ++c) acc[tl][c] = 0.f;
+        }
+        if (!live[0]) continue;                                // tiles of a warp are consecutive
+        for (int cb = 0; cb < ncb; ++cb) {
             for (int r = r0; r < kh; r += stride_h) {
-                // h + pad_h - r and wq + pad_w - q are multiples of the stride inside a class, also when negative
-                const int ho = (h + pad_h - r) / stride_h;
-                if (ho < 0 || ho >= h_out) continue;
-                const uint4 *row = dz + ((size_t)(img * h_out + ho) * w_out) * v + g8;
-                for (int qb = q0; qb < kw; qb += 4 * stride_w) {
-                    // Four taps of one kernel row at a time: tap u of them pairs pixel p with output column
-                    // wo0 - u + p, so the PX + 3 columns from wo0 - 3 on serve all four taps.
-                    const int wo0 = (wq + pad_w - qb) / stride_w;
-                    const int nu = min(4, (kw - qb + stride_w - 1) / stride_w);
-                    uint4 win[PX + 3];
+                // h + pad_h - r and w + pad_w - q are multiples of the stride inside a class, also when negative
+                const uint4 *row[STEM_DG_TILES];
+                bool row_ok[STEM_DG_TILES];
 #pragma unroll
-                    for (int k = 0; k < PX + 3; ++k) {
-                        const int wk = wo0 - 3 + k;
-                        win[k] = (k >= 4 - nu && wk >= 0 && wk < w_out) ? __ldg(row + (size_t)wk * v)
-                                                                         : make_uint4(0u, 0u, 0u, 0u);
+                for (int tl = 0; tl < STEM_DG_TILES; ++tl) {
+                    const int ho = (h[tl] + pad_h - r) / stride_h;
+                    row_ok[tl] = live[tl] && ho >= 0 && ho < h_out;
+                    row[tl] = dz + ((size_t)(img[tl] * h_out + (row_ok[tl] ? ho : 0)) * w_out) * v + cb * 8 + t;
+                }
+                for (int q = q0; q < kw; q += stride_w) {
+                    uint4 alo[STEM_DG_TILES][2], ahi[STEM_DG_TILES][2];   // pixels g / g + 8, chunks t / t + 4
+#pragma unroll
+                    for (int tl = 0; tl < STEM_DG_TILES; ++tl) {
+                        const int wo = (j0[tl] * stride_w + b + pad_w - q) / stride_w + g;
+                        const bool lo_ok = row_ok[tl] && wo >= 0 && wo < w_out;
+                        const bool hi_ok = row_ok[tl] && wo + 8 >= 0 && wo + 8 < w_out;
+                        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+                        alo[tl][0] = lo_ok ? __ldg(row[tl] + (size_t)wo * v) : zero;
+                        alo[tl][1] = lo_ok ? __ldg(row[tl] + (size_t)wo * v + 4) : zero;
+                        ahi[tl][0] = hi_ok ? __ldg(row[tl] + (size_t)(wo + 8) * v) : zero;
+                        ahi[tl][1] = hi_ok ? __ldg(row[tl] + (size_t)(wo + 8) * v + 4) : zero;
                     }
-                    const float *wt = wg + (size_t)(r * kw + qb) * tap_floats;
-                    const size_t tap_step = (size_t)stride_w * tap_floats;
+                    const uint32_t *wf = wfrag + ((size_t)(r * kw + q) * ncb + cb) * 256 + lane;
+                    uint32_t bf[4][2];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {              // channel e of the lane's chunk, widened once
-                        float d[PX + 3];
+                    for (int k = 0; k < 4; ++k) {
+                        bf[k][0] = wf[k * 64];
+                        bf[k][1] = wf[k * 64 + 32];
+                    }
 #pragma unroll
-                        for (int k = 0; k < PX + 3; ++k) {
-                            const uint32_t word = e < 2 ? win[k].x : e < 4 ? win[k].y : e < 6 ? win[k].z : win[k].w;
-                            d[k] = __uint_as_float((e & 1) ? (word & 0xFFFF0000u) : (word << 16));
-                        }
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            if (u < nu) {                      // the same for every lane
-                                const float4 *wc = (const float4 *)(wt + u * tap_step + e * 8 * CP);
-                                float wv[CP];
-#pragma unroll
-                                for (int c4 = 0; c4 < CP / 4; ++c4) {
-                                    const float4 f = wc[c4];
-                                    wv[4 * c4] = f.x; wv[4 * c4 + 1] = f.y; wv[4 * c4 + 2] = f.z; wv[4 * c4 + 3] = f.w;
-                                }
-#pragma unroll
-                                for (int p = 0; p < PX; ++p)
-#pragma unroll
-                                    for (int c = 0; c < CIN; ++c) acc[p][c] = fmaf(d[p - u + 3], wv[c], acc[p][c]);
-                            }
+                    for (int tl = 0; tl < STEM_DG_TILES; ++tl) {
+                        if (row_ok[tl]) {                      // the same for the whole warp
+                            mma_16x8x16_bf16(acc[tl], alo[tl][0].x, ahi[tl][0].x, alo[tl][1].x, ahi[tl][1].x, bf[0][0], bf[0][1]);
+                            mma_16x8x16_bf16(acc[tl], alo[tl][0].y, ahi[tl][0].y, alo[tl][1].y, ahi[tl][1].y, bf[1][0], bf[1][1]);
+                            mma_16x8x16_bf16(acc[tl], alo[tl][0].z, ahi[tl][0].z, alo[tl][1].z, ahi[tl][1].z, bf[2][0], bf[2][1]);
+                            mma_16x8x16_bf16(acc[tl], alo[tl][0].w, ahi[tl][0].w, alo[tl][1].w, ahi[tl][1].w, bf[3][0], bf[3][1]);
                         }
                     }
                 }
             }
         }
+        // accumulator registers: (pixel g, channels 2t and 2t+1), (pixel g + 8, the same channels)
 #pragma unroll
-        for (int p = 0; p < PX; ++p) {
-            float mine = 0.f;
+        for (int tl = 0; tl < STEM_DG_TILES; ++tl) {
+            if (!live[tl]) continue;
 #pragma unroll
-            for (int c = 0; c < CIN; ++c) {
-                float t = acc[p][c];
-                t += __shfl_xor_sync(0xFFFFFFFFu, t, 1);
-                t += __shfl_xor_sync(0xFFFFFFFFu, t, 2);
-                t += __shfl_xor_sync(0xFFFFFFFFu, t, 4);
-                if (l8 == c) mine = t;
+            for (int half = 0; half < 2; ++half) {
+                const int j = j0[tl] + g + 8 * half;
+                if (j >= wj_n) continue;
+                __nv_bfloat16 *dst = dx + ((size_t)(img[tl] * h_in + h[tl]) * w_in + j * stride_w + b) * c_in;
+                if (2 * t < c_in) dst[2 * t] = __float2bfloat16_rn(acc[tl][2 * half]);
+                if (2 * t + 1 < c_in) dst[2 * t + 1] = __float2bfloat16_rn(acc[tl][2 * half + 1]);
             }
-            if (live && j + p < wj_n && l8 < c_in)
-                dx[((size_t)(img * h_in + h) * w_in + wq + p * stride_w) * c_in + l8] = __float2bfloat16_rn(mine);
         }
     }
 }
 
 bool stem_dgrad_eligible(const Problem &pb) {
-    return stem_eligible(pb) && pb.c_out % 8 == 0 &&
-           (size_t)pb.kh * pb.kw * ((pb.c_out / 8 + 7) / 8) * 64 * (pb.c_in <= 4 ? 4 : 8) * sizeof(float) <= 160 * 1024;
+    return stem_eligible(pb) && (size_t)pb.kh * pb.kw * (pb.c_out / 64) * 1024 <= 160 * 1024;
 }
 
 cudaError_t launch_stem_dgrad(const Problem &pb, const void *dz, const void *w, const float *s_vec, void *dx,
                               cudaStream_t st) {
-    const int cp = pb.c_in <= 4 ? 4 : 8;
-    const int vo = (pb.c_out / 8 + 7) / 8;
-    const size_t smem = (size_t)pb.kh * pb.kw * vo * 64 * cp * sizeof(float);
+    const size_t smem = (size_t)pb.kh * pb.kw * (pb.c_out / 64) * 1024;
     static bool attr = false;
     if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(stem_dgrad_kernel<4, 3, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(stem_dgrad_kernel<4, 4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(stem_dgrad_kernel<8, 8, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(stem_dgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
         if (e != cudaSuccess) return e;
         attr = true;
     }
-    const long long passes = ((long long)pb.n * pb.h_in * pb.w_in + 63) / 64;
-    const unsigned grid = (unsigned)(passes < 148 * 2 ? passes : 148 * 2);   // two resident blocks per SM
-#define CONVBN_STEM_DGRAD(CP_, CIN_, PX_)                                                                           \
-    stem_dgrad_kernel<CP_, CIN_, PX_><<<grid, 256, smem, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out,     \
-                                                          pb.c_out, pb.kh, pb.kw, pb.stride_h, pb.stride_w,        \
-                                                          pb.pad_h, pb.pad_w, (const uint4 *)dz,                   \
-                                                          (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)dx)
-    if (pb.c_in == 3) CONVBN_STEM_DGRAD(4, 3, 8);
-    else if (cp == 4) CONVBN_STEM_DGRAD(4, 4, 4);
-    else CONVBN_STEM_DGRAD(8, 8, 4);
-#undef CONVBN_STEM_DGRAD
+    const long long passes = ((long long)pb.n * pb.h_in * pb.w_in + 255) / 256;
+    const unsigned grid = (unsigned)(passes < 148 * 3 ? passes : 148 * 3);   // three resident blocks per SM
+    stem_dgrad_kernel<<<grid, 256, smem, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.c_out, pb.kh,
+                                               pb.kw, pb.stride_h, pb.stride_w, pb.pad_h, pb.pad_w, (const uint4 *)dz,
+                                               (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)dx);
     return cudaGetLastError();
 }
 
