@@ -106,15 +106,21 @@ __device__ __forceinline__ void mma_16x8x16_bf16(float (&c)[4], uint32_t a0, uin
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-constexpr int STEM_DG_TILES = 2;     // 16-pixel tiles per warp and pass; they share the B fragments
-
+// A warp owns 32 consecutive columns of one dZ row at a time (two MMA tiles).  With NU taps in a kernel
+// row of the class, tap u pairs output pixel j with dZ column j + const - u, so instead of loading
+// shifted A fragments per tap the warp keeps one accumulator per tap over the un-shifted columns and
+// applies the shifts once at the end, through a small shared-memory scratch: every A fragment is
+// loaded once per kernel row rather than once per tap, and 32 - (NU - 1) output pixels come out of
+// each 32-column window.
+template <int NU>      // taps per kernel row and class, rounded up to 1, 2, 4 or 8
 __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_in, int c_in, int h_out, int w_out,
                                                          int c_out, int kh, int kw, int stride_h, int stride_w,
                                                          int pad_h, int pad_w, const uint4 *__restrict__ dz,
                                                          const __nv_bfloat16 *__restrict__ w,
                                                          const float *__restrict__ s_vec,
                                                          __nv_bfloat16 *__restrict__ dx) {
-    extern __shared__ uint32_t wfrag[];    // [tap][64-channel block][k-step][b0/b1][lane]
+    extern __shared__ uint32_t wfrag[];    // [tap][64-channel block][k-step][b0/b1][lane], then the scratch
+    constexpr int OUTW = 32 - (NU - 1);    // output pixels per window
     const int taps = kh * kw;
     const int ncb = c_out / 64, v = c_out / 8;
 #pragma unroll 4
@@ -135,13 +141,14 @@ __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
-    const uint32_t tpp = (blockDim.x >> 5) * STEM_DG_TILES;    // tiles per block and pass
-    // Work items are (pass of tpp tiles, residue class).  A block owns a contiguous run of passes and
+    float *scr = reinterpret_cast<float *>(wfrag + (size_t)taps * ncb * 256) + warp * 256;   // [32 columns][8]
+    const uint32_t wpb = blockDim.x >> 5;                      // windows per block and pass
+    // Work items are (pass of wpb windows, residue class).  A block owns a contiguous run of passes and
     // visits every class of a pass before the next pass: the classes of one pass, and neighbouring
     // passes, read the same rows of dZ, and every block meets the classes equally often although they
     // have different tap counts.
-    const int wt_max = ((w_in + stride_w - 1) / stride_w + 15) / 16;
-    const uint32_t ipc = ((uint32_t)n * ((h_in + stride_h - 1) / stride_h) * wt_max + tpp - 1) / tpp;
+    const int wt_max = ((w_in + stride_w - 1) / stride_w + OUTW - 1) / OUTW;
+    const uint32_t ipc = ((uint32_t)n * ((h_in + stride_h - 1) / stride_h) * wt_max + wpb - 1) / wpb;
     const uint32_t ncls = (uint32_t)(stride_h * stride_w);
     const uint32_t run = (ipc + gridDim.x - 1) / gridDim.x;
     const uint32_t pass_end = min(ipc, (blockIdx.x + 1) * run);
@@ -150,102 +157,140 @@ __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_
         const int a = cls / stride_w, b = cls % stride_w;
         if (a >= h_in || b >= w_in) continue;
         const int hi_n = (h_in - a + stride_h - 1) / stride_h, wj_n = (w_in - b + stride_w - 1) / stride_w;
-        const int wt_n = (wj_n + 15) / 16;                     // tiles along a row
-        const uint32_t total = (uint32_t)n * hi_n * wt_n;
+        const int wt_n = (wj_n + OUTW - 1) / OUTW;             // windows along a row
+        const uint32_t idx = (item / ncls) * wpb + warp;
+        if (idx >= (uint32_t)n * hi_n * wt_n) continue;        // whole warp
+        const uint32_t t1 = idx / (uint32_t)wt_n;
+        const int jbase = (int)(idx - t1 * (uint32_t)wt_n) * OUTW;
+        const int img = (int)(t1 / (uint32_t)hi_n);
+        const int h = (int)(t1 - (uint32_t)img * (uint32_t)hi_n) * stride_h + a;
         const int r0 = (a + pad_h) % stride_h, q0 = (b + pad_w) % stride_w;
-        bool live[STEM_DG_TILES];
-        int img[STEM_DG_TILES], h[STEM_DG_TILES], j0[STEM_DG_TILES];
-        float acc[STEM_DG_TILES][4];
+        const int nu = q0 < kw ? (kw - q0 + stride_w - 1) / stride_w : 0;   // <= NU
+        // tap u (q = q0 + u stride_w) pairs output pixel j with column j + (b + pad_w - q0) / stride_w - u;
+        // window column p holds dZ column col0 + p, so tap u's product for pixel jbase + l sits at l + NU-1 - u
+        const int col0 = jbase + (b + pad_w - q0) / stride_w - (NU - 1);
+        float acc[NU][2][4];
 #pragma unroll
-        for (int tl = 0; tl < STEM_DG_TILES; ++tl) {
-            const uint32_t idx = (item / ncls) * tpp + warp * STEM_DG_TILES + tl;
-            live[tl] = idx < total;
-            const uint32_t id = live[tl] ? idx : 0u;
-            const uint32_t t1 = id / (uint32_t)wt_n;
-            j0[tl] = (int)(id - t1 * (uint32_t)wt_n) * 16;
-            img[tl] = (int)(t1 / (uint32_t)hi_n);
-            h[tl] = (int)(t1 - (uint32_t)img[tl] * (uint32_t)hi_n) * stride_h + a;
+        for (int u = 0; u < NU; ++u)
 #pragma unroll
-            for (int c = 0; c < 4; ++c) acc[tl][c] = 0.f;
-        }
-        if (!live[0]) continue;                                // tiles of a warp are consecutive
+            for (int tl = 0; tl < 2; ++tl)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) acc[u][tl][c] = 0.f;
         for (int cb = 0; cb < ncb; ++cb) {
             for (int r = r0; r < kh; r += stride_h) {
-                // h + pad_h - r and w + pad_w - q are multiples of the stride inside a class, also when negative
-                const uint4 *row[STEM_DG_TILES];
-                bool row_ok[STEM_DG_TILES];
+                // h + pad_h - r is a multiple of the stride inside a class, also when negative
+                const int ho = (h + pad_h - r) / stride_h;
+                if (ho < 0 || ho >= h_out) continue;
+                const uint4 *row = dz + ((size_t)(img * h_out + ho) * w_out) * v + cb * 8 + t;
+                uint4 alo[2][2], ahi[2][2];                    // columns g / g + 8 of a tile, chunks t / t + 4
 #pragma unroll
-                for (int tl = 0; tl < STEM_DG_TILES; ++tl) {
-                    const int ho = (h[tl] + pad_h - r) / stride_h;
-                    row_ok[tl] = live[tl] && ho >= 0 && ho < h_out;
-                    row[tl] = dz + ((size_t)(img[tl] * h_out + (row_ok[tl] ? ho : 0)) * w_out) * v + cb * 8 + t;
+                for (int tl = 0; tl < 2; ++tl) {
+                    const int wo = col0 + tl * 16 + g;
+                    const bool lo_ok = wo >= 0 && wo < w_out, hi_ok = wo + 8 >= 0 && wo + 8 < w_out;
+                    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+                    alo[tl][0] = lo_ok ? __ldg(row + (size_t)wo * v) : zero;
+                    alo[tl][1] = lo_ok ? __ldg(row + (size_t)wo * v + 4) : zero;
+                    ahi[tl][0] = hi_ok ? __ldg(row + (size_t)(wo + 8) * v) : zero;
+                    ahi[tl][1] = hi_ok ? __ldg(row + (size_t)(wo + 8) * v + 4) : zero;
                 }
-                for (int q = q0; q < kw; q += stride_w) {
-                    uint4 alo[STEM_DG_TILES][2], ahi[STEM_DG_TILES][2];   // pixels g / g + 8, chunks t / t + 4
 #pragma unroll
-                    for (int tl = 0; tl < STEM_DG_TILES; ++tl) {
-                        const int wo = (j0[tl] * stride_w + b + pad_w - q) / stride_w + g;
-                        const bool lo_ok = row_ok[tl] && wo >= 0 && wo < w_out;
-                        const bool hi_ok = row_ok[tl] && wo + 8 >= 0 && wo + 8 < w_out;
-                        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-                        alo[tl][0] = lo_ok ? __ldg(row[tl] + (size_t)wo * v) : zero;
-                        alo[tl][1] = lo_ok ? __ldg(row[tl] + (size_t)wo * v + 4) : zero;
-                        ahi[tl][0] = hi_ok ? __ldg(row[tl] + (size_t)(wo + 8) * v) : zero;
-                        ahi[tl][1] = hi_ok ? __ldg(row[tl] + (size_t)(wo + 8) * v + 4) : zero;
-                    }
-                    const uint32_t *wf = wfrag + ((size_t)(r * kw + q) * ncb + cb) * 256 + lane;
-                    uint32_t bf[4][2];
+                for (int u = 0; u < NU; ++u) {
+                    if (u < nu) {                              // the same for the whole warp
+                        const uint32_t *wf = wfrag + ((size_t)(r * kw + q0 + u * stride_w) * ncb + cb) * 256 + lane;
+                        uint32_t bf[4][2];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        bf[k][0] = wf[k * 64];
-                        bf[k][1] = wf[k * 64 + 32];
-                    }
+                        for (int k = 0; k < 4; ++k) {
+                            bf[k][0] = wf[k * 64];
+                            bf[k][1] = wf[k * 64 + 32];
+                        }
 #pragma unroll
-                    for (int tl = 0; tl < STEM_DG_TILES; ++tl) {
-                        if (row_ok[tl]) {                      // the same for the whole warp
-                            mma_16x8x16_bf16(acc[tl], alo[tl][0].x, ahi[tl][0].x, alo[tl][1].x, ahi[tl][1].x, bf[0][0], bf[0][1]);
-                            mma_16x8x16_bf16(acc[tl], alo[tl][0].y, ahi[tl][0].y, alo[tl][1].y, ahi[tl][1].y, bf[1][0], bf[1][1]);
-                            mma_16x8x16_bf16(acc[tl], alo[tl][0].z, ahi[tl][0].z, alo[tl][1].z, ahi[tl][1].z, bf[2][0], bf[2][1]);
-                            mma_16x8x16_bf16(acc[tl], alo[tl][0].w, ahi[tl][0].w, alo[tl][1].w, ahi[tl][1].w, bf[3][0], bf[3][1]);
+                        for (int tl = 0; tl < 2; ++tl) {
+                            mma_16x8x16_bf16(acc[u][tl], alo[tl][0].x, ahi[tl][0].x, alo[tl][1].x, ahi[tl][1].x, bf[0][0], bf[0][1]);
+                            mma_16x8x16_bf16(acc[u][tl], alo[tl][0].y, ahi[tl][0].y, alo[tl][1].y, ahi[tl][1].y, bf[1][0], bf[1][1]);
+                            mma_16x8x16_bf16(acc[u][tl], alo[tl][0].z, ahi[tl][0].z, alo[tl][1].z, ahi[tl][1].z, bf[2][0], bf[2][1]);
+                            mma_16x8x16_bf16(acc[u][tl], alo[tl][0].w, ahi[tl][0].w, alo[tl][1].w, ahi[tl][1].w, bf[3][0], bf[3][1]);
                         }
                     }
                 }
             }
         }
-        // accumulator registers: (pixel g, channels 2t and 2t+1), (pixel g + 8, the same channels)
+        // Shift and add: accumulator registers are (column g, channels 2t, 2t+1) and (column g + 8, same);
+        // lane l then owns output pixel jbase + l with all 8 channels.
+        float res[8];
 #pragma unroll
-        for (int tl = 0; tl < STEM_DG_TILES; ++tl) {
-            if (!live[tl]) continue;
+        for (int c = 0; c < 8; ++c) res[c] = 0.f;
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                const int j = j0[tl] + g + 8 * half;
-                if (j >= wj_n) continue;
-                __nv_bfloat16 *dst = dx + ((size_t)(img[tl] * h_in + h[tl]) * w_in + j * stride_w + b) * c_in;
-                if (2 * t < c_in) dst[2 * t] = __float2bfloat16_rn(acc[tl][2 * half]);
-                if (2 * t + 1 < c_in) dst[2 * t + 1] = __float2bfloat16_rn(acc[tl][2 * half + 1]);
+        for (int u = 0; u < NU; ++u) {
+            if (u < nu) {
+                __syncwarp();
+#pragma unroll
+                for (int tl = 0; tl < 2; ++tl)
+#pragma unroll
+                    for (int half = 0; half < 2; ++half)
+                        *reinterpret_cast<float2 *>(scr + (tl * 16 + g + 8 * half) * 8 + 2 * t) =
+                            make_float2(acc[u][tl][2 * half], acc[u][tl][2 * half + 1]);
+                __syncwarp();
+                if (lane < OUTW) {
+                    const float4 *src = reinterpret_cast<const float4 *>(scr + (lane + NU - 1 - u) * 8);
+                    const float4 x0 = src[0], x1 = src[1];
+                    res[0] += x0.x; res[1] += x0.y; res[2] += x0.z; res[3] += x0.w;
+                    res[4] += x1.x; res[5] += x1.y; res[6] += x1.z; res[7] += x1.w;
+                }
             }
+        }
+        const int j = jbase + lane;
+        if (lane < OUTW && j < wj_n) {
+            __nv_bfloat16 *dst = dx + ((size_t)(img * h_in + h) * w_in + j * stride_w + b) * c_in;
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+                if (c < c_in) dst[c] = __float2bfloat16_rn(res[c]);
         }
     }
 }
 
 bool stem_dgrad_eligible(const Problem &pb) {
-    return stem_eligible(pb) && (size_t)pb.kh * pb.kw * (pb.c_out / 64) * 1024 <= 160 * 1024;
+    return stem_eligible(pb) && (size_t)pb.kh * pb.kw * (pb.c_out / 64) * 1024 + 8192 <= 160 * 1024;
 }
 
 cudaError_t launch_stem_dgrad(const Problem &pb, const void *dz, const void *w, const float *s_vec, void *dx,
                               cudaStream_t st) {
-    const size_t smem = (size_t)pb.kh * pb.kw * (pb.c_out / 64) * 1024;
+    const size_t smem = (size_t)pb.kh * pb.kw * (pb.c_out / 64) * 1024 + 8192;   // fragments + 1 KB per warp
     static bool attr = false;
     if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(stem_dgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(stem_dgrad_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(stem_dgrad_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(stem_dgrad_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(stem_dgrad_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
         if (e != cudaSuccess) return e;
         attr = true;
     }
+    const int nu = (pb.kw + pb.stride_w - 1) / pb.stride_w;    // taps per kernel row in the fullest class
+    const void *fn = nu <= 1   ? (const void *)stem_dgrad_kernel<1>
+                     : nu <= 2 ? (const void *)stem_dgrad_kernel<2>
+                     : nu <= 4 ? (const void *)stem_dgrad_kernel<4>
+                               : (const void *)stem_dgrad_kernel<8>;
+    int per_sm = 0, dev = 0, sms = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, 256, smem);
+    if (e == cudaSuccess) e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) return cudaErrorLaunchOutOfResources;
     const long long passes = ((long long)pb.n * pb.h_in * pb.w_in + 255) / 256;
-    const unsigned grid = (unsigned)(passes < 148 * 3 ? passes : 148 * 3);   // three resident blocks per SM
-    stem_dgrad_kernel<<<grid, 256, smem, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.c_out, pb.kh,
-                                               pb.kw, pb.stride_h, pb.stride_w, pb.pad_h, pb.pad_w, (const uint4 *)dz,
-                                               (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)dx);
+    const long long resident = (long long)per_sm * sms;        // one wave of persistent blocks
+    const unsigned grid = (unsigned)(passes < resident ? passes : resident);
+#define CONVBN_STEM_DGRAD(NU_)                                                                                   \
+    stem_dgrad_kernel<NU_><<<grid, 256, smem, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.c_out, \
+                                                    pb.kh, pb.kw, pb.stride_h, pb.stride_w, pb.pad_h, pb.pad_w,   \
+                                                    (const uint4 *)dz, (const __nv_bfloat16 *)w, s_vec,           \
+                                                    (__nv_bfloat16 *)dx)
+    if (nu <= 1) CONVBN_STEM_DGRAD(1);
+    else if (nu <= 2) CONVBN_STEM_DGRAD(2);
+    else if (nu <= 4) CONVBN_STEM_DGRAD(4);
+    else CONVBN_STEM_DGRAD(8);
+#undef CONVBN_STEM_DGRAD
     return cudaGetLastError();
 }
 

@@ -54,6 +54,7 @@ SMALL = [
     # narrow-input (stem) path: 4 and 8 input channels, two output-channel chunk groups, stride 1 and 3
     L("b_stem_c4", 1, 4, 19, 23, 128, 5, 5, pad=2),
     L("b_stem_c8_s3", 2, 8, 25, 22, 64, 3, 3, stride=3, pad=1),
+    L("b_stem_3x3_s2", 1, 3, 41, 70, 64, 3, 3, stride=2, pad=1),
 ]
 
 EXPECTED_PATH = {   # the specialised kernels must actually be the ones that ran
