@@ -122,6 +122,236 @@ __global__ void __launch_bounds__(256) dw_fwd_kernel(DwShape s, const uint4 *__r
     }
 }
 
+// Unit stride and dilation, KH x KW known at compile time.  One thread: 8 channels x TW output columns,
+// walking down `th` output rows.  Every input row of the band is loaded and widened to fp32 once and
+// feeds the KH output rows it reaches, whose accumulators rotate through KH register slots; an output
+// row is stored when its last input row has been added.
+template <int TW, int KH, int KW>
+__global__ void __launch_bounds__(256, KH <= 3 ? 2 : 1) dw_stream_kernel(DwShape s, const uint4 *__restrict__ x,
+                                                        const __nv_bfloat16 *__restrict__ w,
+                                                        const float *__restrict__ bias, uint4 *__restrict__ z,
+                                                        int th) {
+    extern __shared__ float w_s[];                   // [taps][C]
+    constexpr int PF = 3;                            // rows of look-ahead for the L2 prefetch
+    const int v = s.c / 8;
+    stage_weights(w_s, w, KH * KW, s.c);
+    const uint32_t wgroups = (uint32_t)(s.w_out + TW - 1) / TW, bands = (uint32_t)(s.h_out + th - 1) / th;
+    const uint32_t total = (uint32_t)s.n * bands * wgroups * v;
+    for (uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        uint32_t t = idx / (uint32_t)v;
+        const int cv = (int)(idx - t * (uint32_t)v);
+        const uint32_t t1 = t / wgroups;
+        const int wo0 = (int)(t - t1 * wgroups) * TW;
+        const uint32_t n = t1 / bands;
+        const int ho0 = (int)(t1 - n * bands) * th;
+        const int rows = min(th, s.h_out - ho0);
+        float bv[8];
+        if (bias) {
+            const float4 b0 = *reinterpret_cast<const float4 *>(bias + cv * 8);
+            const float4 b1 = *reinterpret_cast<const float4 *>(bias + cv * 8 + 4);
+            bv[0] = b0.x; bv[1] = b0.y; bv[2] = b0.z; bv[3] = b0.w; bv[4] = b1.x; bv[5] = b1.y; bv[6] = b1.z; bv[7] = b1.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) bv[e] = 0.f;
+        }
+        float acc[KH][TW][8];
+#pragma unroll
+        for (int sl = 0; sl < KH; ++sl)
+#pragma unroll
+            for (int j = 0; j < TW; ++j)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[sl][j][e] = bv[e];
+        const float *wch = w_s + cv * 8;
+        const int wi0 = wo0 - s.pad_w;
+        const uint4 *xcol = x + ((size_t)n * s.h_in * s.w_in) * v + cv;
+        uint4 *zcol = z + ((size_t)(n * s.h_out + ho0) * s.w_out + wo0) * v + cv;
+        // step k brings input row ho0 - pad_h + k, which is tap row r of output row ho0 + k - r;
+        // output row o of the band lives in slot o % KH, and k0 is a multiple of KH
+        for (int k0 = 0; k0 < rows + KH - 1; k0 += KH) {
+#pragma unroll
+            for (int ph = 0; ph < KH; ++ph) {
+                const int k = k0 + ph;
+                if (k < rows + KH - 1) {
+                    const int hi = ho0 - s.pad_h + k;
+                    if (k + PF < rows + KH - 1 && hi + PF >= 0 && hi + PF < s.h_in) {
+                        // ask L2 for the row needed PF steps from now: the loads below then find it there
+                        const uint4 *prow = xcol + (size_t)(hi + PF) * s.w_in * v;
+#pragma unroll
+                        for (int j = 0; j < TW + KW - 1; ++j) {
+                            const int wi = wi0 + j;
+                            if (wi >= 0 && wi < s.w_in) asm volatile("prefetch.global.L2 [%0];" ::"l"(prow + (size_t)wi * v));
+                        }
+                    }
+                    if (hi >= 0 && hi < s.h_in) {
+                        const uint4 *xrow = xcol + (size_t)hi * s.w_in * v;
+                        float xs[TW + KW - 1][8];
+#pragma unroll
+                        for (int j = 0; j < TW + KW - 1; ++j) {
+                            const int wi = wi0 + j;
+                            unpack8((wi >= 0 && wi < s.w_in) ? __ldg(xrow + (size_t)wi * v) : make_uint4(0, 0, 0, 0), xs[j]);
+                        }
+#pragma unroll
+                        for (int r = 0; r < KH; ++r) {
+                            const int o = k - r;
+                            if (o >= 0 && o < rows) {
+                                const int sl = (ph - r + KH) % KH;
+#pragma unroll
+                                for (int q = 0; q < KW; ++q) {
+                                    const float4 w0 = *reinterpret_cast<const float4 *>(wch + (r * KW + q) * s.c);
+                                    const float4 w1 = *reinterpret_cast<const float4 *>(wch + (r * KW + q) * s.c + 4);
+                                    const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+                                    for (int j = 0; j < TW; ++j)
+#pragma unroll
+                                        for (int e = 0; e < 8; ++e) acc[sl][j][e] = fmaf(xs[j + q][e], wv[e], acc[sl][j][e]);
+                                }
+                            }
+                        }
+                    }
+                    const int od = k - (KH - 1);               // the output row that is complete now
+                    if (od >= 0) {
+                        const int sl = (ph + 1) % KH;
+#pragma unroll
+                        for (int j = 0; j < TW; ++j) {
+                            if (wo0 + j < s.w_out) zcol[((size_t)od * s.w_out + j) * v] = pack8(acc[sl][j]);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) acc[sl][j][e] = bv[e];
+                        }
+                    }
+                }
+            }
+        }
+    }
+}
+
+// ---- packed fp32 arithmetic (two lanes per instruction, sm_100) ------------------------------------
+typedef unsigned long long f32x2;
+
+__device__ __forceinline__ f32x2 pair(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+// two bf16 in one word -> two fp32
+__device__ __forceinline__ f32x2 widen(uint32_t u) { return pair(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u)); }
+// two fp32 -> two bf16 in one word (round to nearest even)
+__device__ __forceinline__ uint32_t narrow(f32x2 p) {
+    float lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
+    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&h);
+}
+
+// Unit stride and dilation, small KH x KW known at compile time.  One thread: 4 channels x TW output
+// columns, walking down `th` output rows, with its KH x KW x 4 weights in registers.  Every input row
+// of the band is loaded once (the next row's loads are issued before the current row's arithmetic),
+// widened to fp32 once and added into the KH output rows it reaches, whose accumulators rotate through
+// KH register slots; an output row is stored when its last input row has been added.  The arithmetic
+// is packed fp32 (two channels per FMA instruction).
+template <int TW, int KH, int KW>
+__global__ void __launch_bounds__(256, 2) dw_stream4_kernel(DwShape s, const uint2 *__restrict__ x,
+                                                            const __nv_bfloat16 *__restrict__ w,
+                                                            const float *__restrict__ bias, uint2 *__restrict__ z,
+                                                            int th) {
+    extern __shared__ float w_s[];                   // [taps][C]
+    constexpr int NX = TW + KW - 1;
+    const int v = s.c / 4;
+    stage_weights(w_s, w, KH * KW, s.c);
+    const uint32_t wgroups = (uint32_t)(s.w_out + TW - 1) / TW, bands = (uint32_t)(s.h_out + th - 1) / th;
+    const uint32_t total = (uint32_t)s.n * bands * wgroups * v;
+    for (uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        uint32_t t = idx / (uint32_t)v;
+        const int cv = (int)(idx - t * (uint32_t)v);
+        const uint32_t t1 = t / wgroups;
+        const int wo0 = (int)(t - t1 * wgroups) * TW;
+        const uint32_t n = t1 / bands;
+        const int ho0 = (int)(t1 - n * bands) * th;
+        const int rows = min(th, s.h_out - ho0);
+        f32x2 wr[KH * KW][2];
+#pragma unroll
+        for (int tp = 0; tp < KH * KW; ++tp) {
+            const float4 f = *reinterpret_cast<const float4 *>(w_s + tp * s.c + cv * 4);
+            wr[tp][0] = pair(f.x, f.y);
+            wr[tp][1] = pair(f.z, f.w);
+        }
+        f32x2 bv[2] = {pair(0.f, 0.f), pair(0.f, 0.f)};
+        if (bias) {
+            const float4 f = *reinterpret_cast<const float4 *>(bias + cv * 4);
+            bv[0] = pair(f.x, f.y);
+            bv[1] = pair(f.z, f.w);
+        }
+        f32x2 acc[KH][TW][2];
+#pragma unroll
+        for (int sl = 0; sl < KH; ++sl)
+#pragma unroll
+            for (int j = 0; j < TW; ++j) acc[sl][j][0] = bv[0], acc[sl][j][1] = bv[1];
+        const int wi0 = wo0 - s.pad_w;
+        bool col_ok[NX];
+#pragma unroll
+        for (int j = 0; j < NX; ++j) col_ok[j] = wi0 + j >= 0 && wi0 + j < s.w_in;
+        // row pointer at column wi0 (may lie left of the row: only dereferenced where col_ok)
+        const uint2 *xrow = x + ((ptrdiff_t)((size_t)n * s.h_in + 0) * s.w_in + wi0) * v + cv;
+        const ptrdiff_t pitch = (ptrdiff_t)s.w_in * v;
+        uint2 *zrow = z + ((size_t)(n * s.h_out + ho0) * s.w_out + wo0) * v + cv;
+        const uint2 zero = make_uint2(0u, 0u);
+        uint2 nxt[NX];
+        {
+            const int hi = ho0 - s.pad_h;
+            const bool ok = hi >= 0 && hi < s.h_in;
+#pragma unroll
+            for (int j = 0; j < NX; ++j) nxt[j] = (ok && col_ok[j]) ? __ldg(xrow + hi * pitch + (ptrdiff_t)j * v) : zero;
+        }
+        // step k brings input row ho0 - pad_h + k, which is tap row r of output row ho0 + k - r;
+        // output row o of the band lives in slot o % KH, and k0 is a multiple of KH
+        for (int k0 = 0; k0 < rows + KH - 1; k0 += KH) {
+#pragma unroll
+            for (int ph = 0; ph < KH; ++ph) {
+                const int k = k0 + ph;
+                if (k < rows + KH - 1) {
+                    f32x2 xs[NX][2];
+#pragma unroll
+                    for (int j = 0; j < NX; ++j) xs[j][0] = widen(nxt[j].x), xs[j][1] = widen(nxt[j].y);
+                    {
+                        const int hi = ho0 - s.pad_h + k + 1;
+                        const bool ok = k + 1 < rows + KH - 1 && hi >= 0 && hi < s.h_in;
+#pragma unroll
+                        for (int j = 0; j < NX; ++j)
+                            nxt[j] = (ok && col_ok[j]) ? __ldg(xrow + hi * pitch + (ptrdiff_t)j * v) : zero;
+                    }
+#pragma unroll
+                    for (int r = 0; r < KH; ++r) {
+                        if (k - r >= 0) {                      // rows past the band only reach slots never stored
+                            const int sl = (ph - r + KH) % KH;
+#pragma unroll
+                            for (int q = 0; q < KW; ++q)
+#pragma unroll
+                                for (int j = 0; j < TW; ++j) {
+                                    acc[sl][j][0] = fma2(xs[j + q][0], wr[r * KW + q][0], acc[sl][j][0]);
+                                    acc[sl][j][1] = fma2(xs[j + q][1], wr[r * KW + q][1], acc[sl][j][1]);
+                                }
+                        }
+                    }
+                    const int od = k - (KH - 1);               // the output row that is complete now
+                    if (od >= 0) {
+                        const int sl = (ph + 1) % KH;
+#pragma unroll
+                        for (int j = 0; j < TW; ++j) {
+                            if (wo0 + j < s.w_out)
+                                zrow[((size_t)od * s.w_out + j) * v] = make_uint2(narrow(acc[sl][j][0]), narrow(acc[sl][j][1]));
+                            acc[sl][j][0] = bv[0], acc[sl][j][1] = bv[1];
+                        }
+                    }
+                }
+            }
+        }
+    }
+}
+
 // dX[n,h,w,c] = sum over taps with (h + p - r d) divisible by the stride of omega'[c,r,q] dZ[n,ho,wo,c].
 __global__ void __launch_bounds__(256) dw_dgrad_kernel(DwShape s, const uint4 *__restrict__ dz,
                                                        const __nv_bfloat16 *__restrict__ w,
@@ -322,7 +552,30 @@ cudaError_t launch_dw_fwd(const Problem &pb, const void *x, const void *w, const
     const bool unit_w = pb.stride_w == 1 && pb.dil_w == 1;
     static bool a3 = false, a5 = false, a0 = false;
     cudaError_t e;
-    if (unit_w && pb.kw == 3) {
+    const bool unit = unit_w && pb.stride_h == 1 && pb.dil_h == 1 && pb.kh == pb.kw && pb.pad_h >= 0 && pb.pad_w >= 0;
+    if (unit && (pb.kh == 3 || pb.kh == 5)) {
+        // rows per thread: as tall as still leaves every SM a few blocks
+        int th = 8;
+        auto threads = [&](int t) {
+            return (long long)pb.n * ((pb.h_out + t - 1) / t) * ((pb.w_out + 1) / 2) * (pb.c_in / 8);
+        };
+        while (th > 1 && threads(th) < 148LL * 256 * 4) th /= 2;
+        static bool s3 = false, s5 = false;
+        if (pb.kh == 3) {
+            auto threads4 = [&](int t) {
+                return (long long)pb.n * ((pb.h_out + t - 1) / t) * ((pb.w_out + 1) / 2) * (pb.c_in / 4);
+            };
+            th = 16;
+            while (th > 1 && threads4(th) < 148LL * 256 * 4) th /= 2;
+            if ((e = set_smem_once(dw_stream4_kernel<2, 3, 3>, &s3)) != cudaSuccess) return e;
+            dw_stream4_kernel<2, 3, 3><<<dw_grid(threads4(th)), 256, smem, st>>>(s, (const uint2 *)x, (const __nv_bfloat16 *)w,
+                                                                                bias, (uint2 *)z, th);
+        } else {
+            if ((e = set_smem_once(dw_stream_kernel<2, 5, 5>, &s5)) != cudaSuccess) return e;
+            dw_stream_kernel<2, 5, 5><<<dw_grid(threads(th)), 256, smem, st>>>(s, (const uint4 *)x, (const __nv_bfloat16 *)w,
+                                                                              bias, (uint4 *)z, th);
+        }
+    } else if (unit_w && pb.kw == 3) {
         if ((e = set_smem_once(dw_fwd_kernel<4, 3>, &a3)) != cudaSuccess) return e;
         dw_fwd_kernel<4, 3><<<dw_grid(total), 256, smem, st>>>(s, (const uint4 *)x, (const __nv_bfloat16 *)w, bias,
                                                                 (uint4 *)z);
