@@ -5,7 +5,10 @@
 //   forward        Z[n,h,w,c]  = b'[c] + sum_{r,q} omega'[c,r,q] X[n, h s - p + r d, w s - p + q d, c]   (Sec. 3.1/3.3)
 //   backward data  dX = omega'_rot (*) dZ   (Sec. 3.2.1), gathered per dX element
 //   backward weight domega'[c,r,q] = sum_{n,h,w} dZ[n,h,w,c] X[n, ...]   (Sec. 3.2.1), per-slice partials
+#include <cstdlib>
+
 #include "kernels.h"
+#include "packed_f32.cuh"
 
 namespace convbn {
 
@@ -224,42 +227,91 @@ __global__ void __launch_bounds__(256, KH <= 3 ? 2 : 1) dw_stream_kernel(DwShape
     }
 }
 
-// ---- packed fp32 arithmetic (two lanes per instruction, sm_100) ------------------------------------
-typedef unsigned long long f32x2;
-
-__device__ __forceinline__ f32x2 pair(float lo, float hi) {
-    f32x2 r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
-    f32x2 d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-// two bf16 in one word -> two fp32
-__device__ __forceinline__ f32x2 widen(uint32_t u) { return pair(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u)); }
-// two fp32 -> two bf16 in one word (round to nearest even)
-__device__ __forceinline__ uint32_t narrow(f32x2 p) {
-    float lo, hi;
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
-    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<const uint32_t *>(&h);
-}
-
 // Unit stride and dilation, small KH x KW known at compile time.  One thread: 4 channels x TW output
 // columns, walking down `th` output rows, with its KH x KW x 4 weights in registers.  Every input row
-// of the band is loaded once (the next row's loads are issued before the current row's arithmetic),
-// widened to fp32 once and added into the KH output rows it reaches, whose accumulators rotate through
-// KH register slots; an output row is stored when its last input row has been added.  The arithmetic
-// is packed fp32 (two channels per FMA instruction).
+// of the band is loaded once, KH rows ahead of its use, into a ring of KH register rows, widened to
+// fp32 once and added into the KH output rows it reaches, whose accumulators rotate through KH register
+// slots; an output row starts from the bias in its first FMA and is stored when its last input row has
+// been added.  Both rings are indexed statically (the row loop is unrolled KH times).  The arithmetic
+// is packed fp32 (two channels per FMA instruction).  EDGE: the thread's columns touch the left or right
+// border and need per-column guards.
+template <int TW, int KH, int KW, bool EDGE>
+__device__ __forceinline__ void dw_stream4_item(const DwShape &s, const uint2 *__restrict__ xp, ptrdiff_t pitch,
+                                                ptrdiff_t colstep, uint2 *__restrict__ zp, ptrdiff_t zpitch,
+                                                int hi0, int rows, int wi0, int wo0, const f32x2 (&wr)[KH * KW][2],
+                                                const f32x2 (&bv)[2]) {
+    constexpr int NX = TW + KW - 1;
+    const uint2 zero = make_uint2(0u, 0u);
+    bool col_ok[NX];
+#pragma unroll
+    for (int j = 0; j < NX; ++j) col_ok[j] = !EDGE || (wi0 + j >= 0 && wi0 + j < s.w_in);
+    bool out_ok[TW];
+#pragma unroll
+    for (int j = 0; j < TW; ++j) out_ok[j] = !EDGE || wo0 + j < s.w_out;
+    const int steps = rows + KH - 1;                           // input rows of the band
+    uint2 raw[KH][NX];
+    f32x2 acc[KH][TW][2];
+#pragma unroll
+    for (int sl = 0; sl < KH; ++sl) {
+        const int hi = hi0 + sl;
+        const bool ok = sl < steps && hi >= 0 && hi < s.h_in;
+#pragma unroll
+        for (int j = 0; j < NX; ++j) raw[sl][j] = (ok && col_ok[j]) ? __ldg(xp + hi * pitch + j * colstep) : zero;
+#pragma unroll
+        for (int j = 0; j < TW; ++j) acc[sl][j][0] = acc[sl][j][1] = 0ull;
+    }
+    // step k brings input row hi0 + k, which is tap row r of output row k - r of the band; output row o
+    // lives in slot o % KH, input row k in ring row k % KH, and k0 is a multiple of KH
+    for (int k0 = 0; k0 < steps; k0 += KH) {
+#pragma unroll
+        for (int ph = 0; ph < KH; ++ph) {
+            const int k = k0 + ph;
+            if (k < steps) {
+                f32x2 xs[NX][2];
+#pragma unroll
+                for (int j = 0; j < NX; ++j) xs[j][0] = widen(raw[ph][j].x), xs[j][1] = widen(raw[ph][j].y);
+                {
+                    const int hi = hi0 + k + KH;
+                    if (k + KH < steps && hi >= 0 && hi < s.h_in) {
+#pragma unroll
+                        for (int j = 0; j < NX; ++j)
+                            raw[ph][j] = col_ok[j] ? __ldg(xp + hi * pitch + j * colstep) : zero;
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < NX; ++j) raw[ph][j] = zero;
+                    }
+                }
+                // tap row 0 opens output row k in slot ph (from the bias); rows before the band's first
+                // or past its last only reach slots that are re-opened before, or never reach, a store
+#pragma unroll
+                for (int r = 0; r < KH; ++r) {
+                    const int sl = (ph - r + KH) % KH;
+#pragma unroll
+                    for (int q = 0; q < KW; ++q)
+#pragma unroll
+                        for (int j = 0; j < TW; ++j) {
+                            acc[sl][j][0] = fma2(xs[j + q][0], wr[r * KW + q][0], (r == 0 && q == 0) ? bv[0] : acc[sl][j][0]);
+                            acc[sl][j][1] = fma2(xs[j + q][1], wr[r * KW + q][1], (r == 0 && q == 0) ? bv[1] : acc[sl][j][1]);
+                        }
+                }
+                if (k >= KH - 1) {                             // output row k - (KH - 1) is complete
+                    const int sl = (ph + 1) % KH;
+                    uint2 *zr = zp + (k - (KH - 1)) * zpitch;
+#pragma unroll
+                    for (int j = 0; j < TW; ++j)
+                        if (out_ok[j]) zr[j * colstep] = make_uint2(narrow(acc[sl][j][0]), narrow(acc[sl][j][1]));
+                }
+            }
+        }
+    }
+}
+
 template <int TW, int KH, int KW>
 __global__ void __launch_bounds__(256, 2) dw_stream4_kernel(DwShape s, const uint2 *__restrict__ x,
                                                             const __nv_bfloat16 *__restrict__ w,
                                                             const float *__restrict__ bias, uint2 *__restrict__ z,
                                                             int th) {
     extern __shared__ float w_s[];                   // [taps][C]
-    constexpr int NX = TW + KW - 1;
     const int v = s.c / 4;
     stage_weights(w_s, w, KH * KW, s.c);
     const uint32_t wgroups = (uint32_t)(s.w_out + TW - 1) / TW, bands = (uint32_t)(s.h_out + th - 1) / th;
@@ -279,76 +331,24 @@ __global__ void __launch_bounds__(256, 2) dw_stream4_kernel(DwShape s, const uin
             wr[tp][0] = pair(f.x, f.y);
             wr[tp][1] = pair(f.z, f.w);
         }
-        f32x2 bv[2] = {pair(0.f, 0.f), pair(0.f, 0.f)};
+        f32x2 bv[2] = {0ull, 0ull};
         if (bias) {
             const float4 f = *reinterpret_cast<const float4 *>(bias + cv * 4);
             bv[0] = pair(f.x, f.y);
             bv[1] = pair(f.z, f.w);
         }
-        f32x2 acc[KH][TW][2];
-#pragma unroll
-        for (int sl = 0; sl < KH; ++sl)
-#pragma unroll
-            for (int j = 0; j < TW; ++j) acc[sl][j][0] = bv[0], acc[sl][j][1] = bv[1];
         const int wi0 = wo0 - s.pad_w;
-        bool col_ok[NX];
-#pragma unroll
-        for (int j = 0; j < NX; ++j) col_ok[j] = wi0 + j >= 0 && wi0 + j < s.w_in;
-        // row pointer at column wi0 (may lie left of the row: only dereferenced where col_ok)
-        const uint2 *xrow = x + ((ptrdiff_t)((size_t)n * s.h_in + 0) * s.w_in + wi0) * v + cv;
-        const ptrdiff_t pitch = (ptrdiff_t)s.w_in * v;
-        uint2 *zrow = z + ((size_t)(n * s.h_out + ho0) * s.w_out + wo0) * v + cv;
-        const uint2 zero = make_uint2(0u, 0u);
-        uint2 nxt[NX];
-        {
-            const int hi = ho0 - s.pad_h;
-            const bool ok = hi >= 0 && hi < s.h_in;
-#pragma unroll
-            for (int j = 0; j < NX; ++j) nxt[j] = (ok && col_ok[j]) ? __ldg(xrow + hi * pitch + (ptrdiff_t)j * v) : zero;
-        }
-        // step k brings input row ho0 - pad_h + k, which is tap row r of output row ho0 + k - r;
-        // output row o of the band lives in slot o % KH, and k0 is a multiple of KH
-        for (int k0 = 0; k0 < rows + KH - 1; k0 += KH) {
-#pragma unroll
-            for (int ph = 0; ph < KH; ++ph) {
-                const int k = k0 + ph;
-                if (k < rows + KH - 1) {
-                    f32x2 xs[NX][2];
-#pragma unroll
-                    for (int j = 0; j < NX; ++j) xs[j][0] = widen(nxt[j].x), xs[j][1] = widen(nxt[j].y);
-                    {
-                        const int hi = ho0 - s.pad_h + k + 1;
-                        const bool ok = k + 1 < rows + KH - 1 && hi >= 0 && hi < s.h_in;
-#pragma unroll
-                        for (int j = 0; j < NX; ++j)
-                            nxt[j] = (ok && col_ok[j]) ? __ldg(xrow + hi * pitch + (ptrdiff_t)j * v) : zero;
-                    }
-#pragma unroll
-                    for (int r = 0; r < KH; ++r) {
-                        if (k - r >= 0) {                      // rows past the band only reach slots never stored
-                            const int sl = (ph - r + KH) % KH;
-#pragma unroll
-                            for (int q = 0; q < KW; ++q)
-#pragma unroll
-                                for (int j = 0; j < TW; ++j) {
-                                    acc[sl][j][0] = fma2(xs[j + q][0], wr[r * KW + q][0], acc[sl][j][0]);
-                                    acc[sl][j][1] = fma2(xs[j + q][1], wr[r * KW + q][1], acc[sl][j][1]);
-                                }
-                        }
-                    }
-                    const int od = k - (KH - 1);               // the output row that is complete now
-                    if (od >= 0) {
-                        const int sl = (ph + 1) % KH;
-#pragma unroll
-                        for (int j = 0; j < TW; ++j) {
-                            if (wo0 + j < s.w_out)
-                                zrow[((size_t)od * s.w_out + j) * v] = make_uint2(narrow(acc[sl][j][0]), narrow(acc[sl][j][1]));
-                            acc[sl][j][0] = bv[0], acc[sl][j][1] = bv[1];
-                        }
-                    }
-                }
-            }
-        }
+        // pointer to (image n, row 0, column wi0): may lie outside the row, and is only dereferenced
+        // at columns and rows that are inside
+        const uint2 *xp = x + ((ptrdiff_t)n * s.h_in * s.w_in + wi0) * v + cv;
+        uint2 *zp = z + ((size_t)(n * s.h_out + ho0) * s.w_out + wo0) * v + cv;
+        const bool edge = wi0 < 0 || wi0 + TW + KW - 1 > s.w_in || wo0 + TW > s.w_out;
+        if (edge)
+            dw_stream4_item<TW, KH, KW, true>(s, xp, (ptrdiff_t)s.w_in * v, v, zp, (ptrdiff_t)s.w_out * v, ho0 - s.pad_h,
+                                              rows, wi0, wo0, wr, bv);
+        else
+            dw_stream4_item<TW, KH, KW, false>(s, xp, (ptrdiff_t)s.w_in * v, v, zp, (ptrdiff_t)s.w_out * v,
+                                               ho0 - s.pad_h, rows, wi0, wo0, wr, bv);
     }
 }
 
@@ -552,6 +552,8 @@ cudaError_t launch_dw_fwd(const Problem &pb, const void *x, const void *w, const
     const bool unit_w = pb.stride_w == 1 && pb.dil_w == 1;
     static bool a3 = false, a5 = false, a0 = false;
     cudaError_t e;
+    static const bool no_tma = getenv("CONVBN_NO_DW_TMA") != nullptr;
+    if (!no_tma && dw_tma_eligible(pb)) return launch_dw_tma(pb, x, w, bias, z, st);
     const bool unit = unit_w && pb.stride_h == 1 && pb.dil_h == 1 && pb.kh == pb.kw && pb.pad_h >= 0 && pb.pad_w >= 0;
     if (unit && (pb.kh == 3 || pb.kh == 5)) {
         // rows per thread: as tall as still leaves every SM a few blocks

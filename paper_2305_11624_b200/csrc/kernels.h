@@ -120,6 +120,10 @@ cudaError_t launch_stem_fwd(const Problem &pb, const void *x_packed, const void 
 
 // ---- depthwise (groups = C_in = C_out) bandwidth kernels, bf16 NHWC, C multiple of 8 -----------
 bool dw_eligible(const Problem &pb);
+// 3x3, unit stride and dilation, C <= 256: TMA-fed streaming kernel (forward; backward data with rotated taps)
+bool dw_tma_eligible(const Problem &pb);
+cudaError_t launch_dw_tma(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
+                          cudaStream_t st);
 bool dw_wgrad_supported(const Problem &pb);     // tap counts the register-tiled kernel is built for
 cudaError_t launch_dw_fwd(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
                           cudaStream_t st);

@@ -23,6 +23,9 @@ bool make_tmap_im2col_bf16(CUtensorMap *tm, const void *base, int n, int h, int 
 // General tiled map over bf16 data: rank <= 5, dims / byte strides (strides[0] unused) / box, 128-byte swizzle.
 bool make_tmap_tiled_bf16(CUtensorMap *tm, const void *base, int rank, const unsigned long long *dims,
                           const unsigned long long *strides_bytes, const unsigned int *box);
+// The same without swizzle: the box lands in shared memory in plain row-major order.
+bool make_tmap_tiled_bf16_linear(CUtensorMap *tm, const void *base, int rank, const unsigned long long *dims,
+                                 const unsigned long long *strides_bytes, const unsigned int *box);
 
 namespace ptx {
 

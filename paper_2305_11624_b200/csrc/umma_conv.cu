@@ -413,16 +413,26 @@ bool make_tmap_im2col_bf16(CUtensorMap *tm, const void *base, int n, int h, int 
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-bool make_tmap_tiled_bf16(CUtensorMap *tm, const void *base, int rank, const unsigned long long *dims,
-                          const unsigned long long *strides_bytes, const unsigned int *box) {
+static bool encode_tiled_bf16(CUtensorMap *tm, const void *base, int rank, const unsigned long long *dims,
+                              const unsigned long long *strides_bytes, const unsigned int *box, CUtensorMapSwizzle sw) {
     if (!load_encoders() || rank < 1 || rank > 5) return false;
     cuuint64_t d[5], st[4];
     cuuint32_t bx[5], es[5];
     for (int i = 0; i < rank; ++i) { d[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
     for (int i = 1; i < rank; ++i) st[i - 1] = strides_bytes[i];
     return g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), d, st, bx,
-                          es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+                          es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool make_tmap_tiled_bf16(CUtensorMap *tm, const void *base, int rank, const unsigned long long *dims,
+                          const unsigned long long *strides_bytes, const unsigned int *box) {
+    return encode_tiled_bf16(tm, base, rank, dims, strides_bytes, box, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
+bool make_tmap_tiled_bf16_linear(CUtensorMap *tm, const void *base, int rank, const unsigned long long *dims,
+                                 const unsigned long long *strides_bytes, const unsigned int *box) {
+    return encode_tiled_bf16(tm, base, rank, dims, strides_bytes, box, CU_TENSOR_MAP_SWIZZLE_NONE);
 }
 
 bool umma_conv_eligible(const UmmaConvShape &s) {
