@@ -125,7 +125,7 @@ struct Plan {
     size_t xpk = 0, wst = 0;   // small-C_in layers: packed input [n][hp][wp][8], expanded weights [C_out][kh][64]
     bool stem = false;
     size_t wbd = 0;        // block-diagonal expanded weights [C_out][taps][64], storage dtype
-    bool umma_wgrad = false, dw_wgrad = false, grouped_wgrad = false;
+    bool umma_wgrad = false, dw_wgrad = false, dw_tma_wgrad = false, grouped_wgrad = false;
     UmmaWgradPlan uw;
 };
 
@@ -146,6 +146,8 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
     if (pl.dw_wgrad) {
         pl.splits = dw_wgrad_splits(pb);
         part_bytes = wrows * pl.splits * sizeof(float);
+        pl.dw_tma_wgrad = dw_tma_eligible(pb) && getenv("CONVBN_NO_DW_TMA") == nullptr;
+        if (pl.dw_tma_wgrad && dw_tma_wgrad_partial_bytes(pb) > part_bytes) part_bytes = dw_tma_wgrad_partial_bytes(pb);
     }
     pl.stem = stem_path(d, pb);
     const size_t xpk_bytes = pl.stem ? stem_packed_bytes(pb) : 0, wst_bytes = pl.stem ? stem_weight_bytes(pb) : 0;
@@ -441,7 +443,7 @@ int run_param_grads(const convbn_desc *d, const Problem &pb, const Plan &pl, con
     float *partials = (float *)at(ws, pl.partials), *bsum = (float *)at(ws, pl.bsum);
     const bool need_bsum = vec3 || db;
     const bool tc = pl.grouped_wgrad || pl.umma_wgrad || pl.stem;   // tensor-core paths sum dZ inside the GEMM
-    if (need_bsum && !tc)
+    if (need_bsum && !tc && !pl.dw_tma_wgrad)
         LAUNCH("channel_sum", launch_channel_sum_partial(pb, d->dtype, d->layout, dz, bsum, pl.bsplits, st));
     if (pl.stem) {
         LAUNCH("stem_pack", launch_stem_pack(pb, x, at(ws, pl.xpk), st));
@@ -463,6 +465,11 @@ int run_param_grads(const convbn_desc *d, const Problem &pb, const Plan &pl, con
                                                                    dotpart, counters, db, dgamma, dbeta, need_bsum,
                                                                    st));
         *which = "umma";
+    } else if (pl.dw_tma_wgrad) {
+        int nparts = 0;
+        LAUNCH("dw_wgrad", launch_dw_tma_wgrad(pb, dz, x, partials, &nparts, st));
+        LAUNCH("dw_wgrad_finish", launch_dw_wgrad_finish(pb, partials, nparts, w, vec3, b, mean, dw, db, dgamma, dbeta, st));
+        *which = "depthwise";
     } else {
         if (pl.dw_wgrad)
             LAUNCH("dw_wgrad", launch_dw_wgrad(pb, dz, x, partials, pl.splits, st));

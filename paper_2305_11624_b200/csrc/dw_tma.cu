@@ -42,12 +42,16 @@ __device__ __forceinline__ bool try_wait_u32(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ void arrive_u32(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+// lane 0 of the warp arrives; a predicated instruction, so the warp does not branch
+__device__ __forceinline__ void arrive_lane0(uint32_t bar, int lane) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.eq.s32 p, %1, 0;\n\t@p mbarrier.arrive.shared::cta.b64 _, [%0];\n\t}" ::"r"(bar),
+        "r"(lane)
+        : "memory");
 }
-// Out-of-line part of a wait: polls for at most two seconds, and gives up early when another role has
-// set the abort flag.  Returns false on give-up.
-__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+// Slow part of a wait: polls for at most two seconds, and gives up early when another role has set the
+// abort flag.  Returns false on give-up.
+__device__ __forceinline__ bool wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
     const uint64_t t0 = globaltimer_ns();
     uint32_t spins = 0;
     while (true) {
@@ -186,7 +190,7 @@ __global__ void __launch_bounds__(288, 2) dw_tma_kernel(const __grid_constant__ 
                             xs[j][1] = widen(q.y);
                         }
                         __syncwarp();
-                        if (lane == 0) arrive_u32(empty0 + slot * 8);
+                        arrive_lane0(empty0 + slot * 8, lane);
                         ++slot;
                         slot_off += (uint32_t)g.stage_stride;
                         if (slot_off == ring_bytes) { slot = 0; slot_off = 0; par ^= 1u; }
@@ -221,6 +225,204 @@ __global__ void __launch_bounds__(288, 2) dw_tma_kernel(const __grid_constant__ 
     if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
 }
 
+// ---- backward weight ---------------------------------------------------------------------------------
+//   domega'[c,r,q] = sum_{n,h,w} dZ[n,h,w,c] X[n, h - p + r, w - p + q, c],   sum dZ[.,c]      (Sec. 3.2.1)
+// The same row stream with two boxes per ring slot: the X row (with halo columns) and the dZ row of the
+// same step.  X row k of a band meets dZ rows k, k-1, k-2 (tap rows 0, 1, 2), so every consumer keeps the
+// last KH dZ rows of its columns in KH rotating register slots and its KH x KW x 4 sums (plus the sum of
+// dZ) in registers across all the items of the block.  At the end the thread columns are added in
+// column order through shared memory, and the block writes one partial row: part[block][c][KH KW + 1].
+template <int TW, int KH, int KW>
+__global__ void __launch_bounds__(256, 2) dw_tma_wgrad_kernel(const __grid_constant__ CUtensorMap tx,
+                                                              const __grid_constant__ CUtensorMap tdz, DwTmaGeom g,
+                                                              float *__restrict__ part, int *err) {
+    constexpr int NX = TW + KW - 1, NACC = KH * KW + 1;
+    extern __shared__ uint8_t dw_smem_raw[];
+    uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dw_smem_raw) + 127) & ~(uintptr_t)127);
+    DwTmaCtl *ctl = reinterpret_cast<DwTmaCtl *>(base);
+    uint8_t *ring = base + ((sizeof(DwTmaCtl) + 127) / 128) * 128;
+    volatile int *abort_flag = &ctl->abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < g.stages; ++i) {
+            mbar_init(&ctl->full[i], 1);
+            mbar_init(&ctl->empty[i], (uint32_t)g.consumer_warps);
+        }
+        ctl->abort_flag = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+    const uint32_t items = (uint32_t)g.n * g.bands * g.strips;
+    const int bwo = g.cols_t * TW;                             // dZ columns per strip
+    const uint32_t x_bytes = (uint32_t)(bwo + KW - 1) * g.c * 2, dz_bytes = (uint32_t)bwo * g.c * 2;
+    const uint32_t dz_off = (x_bytes + 127u) & ~127u;          // dZ row behind the X row in a slot
+    const int v = g.c / 4;
+    const int cv = (int)threadIdx.x % v, tc = (int)threadIdx.x / v;
+    const bool active = warp < g.consumer_warps && tc < g.cols_t;
+    f32x2 acc[NACC][2];
+#pragma unroll
+    for (int t = 0; t < NACC; ++t) acc[t][0] = acc[t][1] = 0ull;
+    if (warp == g.consumer_warps) {
+        // ---- producer ----
+        if (lane == 0) {
+            prefetch_tensormap(&tx);
+            prefetch_tensormap(&tdz);
+            uint32_t slot = 0, par = 0;
+            bool ok = true;
+            for (uint32_t it = blockIdx.x; it < items && ok; it += gridDim.x) {
+                const int strip = (int)(it % (uint32_t)g.strips);
+                const uint32_t t1 = it / (uint32_t)g.strips;
+                const int band = (int)(t1 % (uint32_t)g.bands), img = (int)(t1 / (uint32_t)g.bands);
+                const int rows = min(g.th, g.h_out - band * g.th), steps = rows + KH - 1;
+                const int wo0 = strip * bwo, ho0 = band * g.th;
+                for (int k = 0; k < steps; ++k) {
+                    if (!mbar_wait_bounded(&ctl->empty[slot], par ^ 1u, abort_flag)) { ok = false; break; }
+                    uint8_t *dst = ring + (size_t)slot * g.stage_stride;
+                    mbar_arrive_expect_tx(&ctl->full[slot], x_bytes + (k < rows ? dz_bytes : 0u));
+                    tma_load_4d(dst, &tx, &ctl->full[slot], 0, wo0 - g.pad_w, ho0 - g.pad_h + k, img);
+                    if (k < rows) tma_load_4d(dst + dz_off, &tdz, &ctl->full[slot], 0, wo0, ho0 + k, img);
+                    if (++slot == (uint32_t)g.stages) { slot = 0; par ^= 1u; }
+                }
+            }
+            if (!ok) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+        }
+    } else {
+        // ---- consumers ----
+        const uint32_t col_bytes = (uint32_t)g.c * 2;
+        uint32_t x_addr[NX], dz_addr[TW];
+#pragma unroll
+        for (int j = 0; j < NX; ++j)
+            x_addr[j] = smem_u32(ring) + (uint32_t)((active ? tc : 0) * TW + j) * col_bytes + (uint32_t)cv * 8;
+#pragma unroll
+        for (int j = 0; j < TW; ++j)
+            dz_addr[j] = smem_u32(ring) + dz_off + (uint32_t)((active ? tc : 0) * TW + j) * col_bytes + (uint32_t)cv * 8;
+        const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+        const uint32_t ring_bytes = (uint32_t)g.stages * g.stage_stride;
+        const f32x2 ones = pair(1.f, 1.f);
+        uint32_t slot = 0, slot_off = 0, par = 0;
+        bool ok = true;
+        for (uint32_t it = blockIdx.x; it < items && ok; it += gridDim.x) {
+            const uint32_t t1 = it / (uint32_t)g.strips;
+            const int band = (int)(t1 % (uint32_t)g.bands);
+            const int rows = min(g.th, g.h_out - band * g.th);
+            int steps = rows + KH - 1;
+            f32x2 dzw[KH][TW][2];                              // dZ row o of the band lives in slot o % KH
+#pragma unroll
+            for (int sl = 0; sl < KH; ++sl)
+#pragma unroll
+                for (int j = 0; j < TW; ++j) dzw[sl][j][0] = dzw[sl][j][1] = 0ull;
+            for (int k0 = 0; k0 < steps; k0 += KH) {
+#pragma unroll
+                for (int ph = 0; ph < KH; ++ph) {
+                    const int k = k0 + ph;
+                    if (k < steps) {
+                        if (!try_wait_u32(full0 + slot * 8, par) && !wait_slow(full0 + slot * 8, par, abort_flag)) {
+                            ok = false;
+                            steps = 0;                         // leaves both loops
+                        } else {
+                            f32x2 xs[NX][2];
+#pragma unroll
+                            for (int j = 0; j < NX; ++j) {
+                                const uint2 q = lds_u2(x_addr[j] + slot_off);
+                                xs[j][0] = widen(q.x);
+                                xs[j][1] = widen(q.y);
+                            }
+                            if (k < rows) {                    // same for the whole block
+#pragma unroll
+                                for (int j = 0; j < TW; ++j) {
+                                    const uint2 q = lds_u2(dz_addr[j] + slot_off);
+                                    dzw[ph][j][0] = widen(q.x);
+                                    dzw[ph][j][1] = widen(q.y);
+                                    acc[KH * KW][0] = fma2(dzw[ph][j][0], ones, acc[KH * KW][0]);
+                                    acc[KH * KW][1] = fma2(dzw[ph][j][1], ones, acc[KH * KW][1]);
+                                }
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < TW; ++j) dzw[ph][j][0] = dzw[ph][j][1] = 0ull;
+                            }
+                            __syncwarp();
+                            arrive_lane0(empty0 + slot * 8, lane);
+                            ++slot;
+                            slot_off += (uint32_t)g.stage_stride;
+                            if (slot_off == ring_bytes) { slot = 0; slot_off = 0; par ^= 1u; }
+                            // X row k is tap row r of dZ row k - r (slot (ph - r) mod KH; zero outside the band)
+#pragma unroll
+                            for (int r = 0; r < KH; ++r) {
+                                const int sl = (ph - r + KH) % KH;
+#pragma unroll
+                                for (int q = 0; q < KW; ++q)
+#pragma unroll
+                                    for (int j = 0; j < TW; ++j) {
+                                        acc[r * KW + q][0] = fma2(dzw[sl][j][0], xs[j + q][0], acc[r * KW + q][0]);
+                                        acc[r * KW + q][1] = fma2(dzw[sl][j][1], xs[j + q][1], acc[r * KW + q][1]);
+                                    }
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+    }
+    // ---- add the thread columns (in column order) and write the block's partial row ----
+    __syncthreads();                                           // every row has been consumed: the ring is free
+    float *red = reinterpret_cast<float *>(ring);              // [cols_t][C / 4][NACC][4]
+    if (active) {
+        float *mine = red + ((size_t)tc * v + cv) * (NACC * 4);
+#pragma unroll
+        for (int t = 0; t < NACC; ++t) {
+            float a, b, c2, d;
+            asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(acc[t][0]));
+            asm("mov.b64 {%0, %1}, %2;" : "=f"(c2), "=f"(d) : "l"(acc[t][1]));
+            *reinterpret_cast<float4 *>(mine + t * 4) = make_float4(a, b, c2, d);
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < g.c * NACC; i += blockDim.x) {
+        const int c = i / NACC, t = i - c * NACC;
+        float sum = 0.f;
+        for (int col = 0; col < g.cols_t; ++col) sum += red[((size_t)col * v + c / 4) * (NACC * 4) + t * 4 + (c & 3)];
+        part[(size_t)blockIdx.x * g.c * NACC + i] = sum;
+    }
+}
+
+// Adds the block partials in block order and forms the parameter gradients (Table 2, Tune row):
+//   domega = s domega', dbeta = sum dZ, db = s dbeta, dgamma = r (sum_k domega' omega + dbeta (b - mu_hat)).
+// vec3 == NULL: domega = domega', db = sum dZ.  One block per channel; warp t sums tap t (warp KH KW: dZ).
+template <int TAPS>
+__global__ void __launch_bounds__(32 * (TAPS + 1)) dw_wgrad_finish_kernel(int c_total, int nparts,
+                                                                           const float *__restrict__ part,
+                                                                           const __nv_bfloat16 *__restrict__ w,
+                                                                           const float *__restrict__ vec3,
+                                                                           const float *__restrict__ b,
+                                                                           const float *__restrict__ mean,
+                                                                           float *__restrict__ dw, float *__restrict__ db,
+                                                                           float *__restrict__ dgamma,
+                                                                           float *__restrict__ dbeta) {
+    __shared__ float tot[TAPS + 1];
+    const int c = blockIdx.x, t = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float sum = 0.f;
+    for (int p = lane; p < nparts; p += 32) sum += part[((size_t)p * c_total + c) * (TAPS + 1) + t];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+    if (lane == 0) tot[t] = sum;
+    __syncthreads();
+    if (threadIdx.x < TAPS) dw[(size_t)c * TAPS + threadIdx.x] = (vec3 ? vec3[c] : 1.f) * tot[threadIdx.x];
+    if (threadIdx.x == 0) {
+        const float dsum = tot[TAPS];
+        if (vec3) {
+            float dot = 0.f;
+            for (int k = 0; k < TAPS; ++k) dot = fmaf(tot[k], __bfloat162float(w[(size_t)c * TAPS + k]), dot);
+            const float s = vec3[c], r = vec3[2 * c_total + c];
+            dbeta[c] = dsum;
+            if (db) db[c] = s * dsum;
+            dgamma[c] = r * (dot + dsum * ((b ? b[c] : 0.f) - mean[c]));
+        } else if (db) {
+            db[c] = dsum;
+        }
+    }
+}
+
 }  // namespace
 
 bool dw_tma_eligible(const Problem &pb) {
@@ -230,23 +432,26 @@ bool dw_tma_eligible(const Problem &pb) {
            pb.pin * pb.c_in < (1LL << 31);
 }
 
-cudaError_t launch_dw_tma(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
-                          cudaStream_t st) {
-    constexpr int TW = 2, KH = 3, KW = 3;
+// Strip width, ring depth, band height and grid for a stream of `bytes_per_col_row` bytes per output
+// column and row (X box plus, for the backward-weight kernel, the dZ box).
+static cudaError_t dw_tma_geometry(const Problem &pb, int tw, int kh, int kw, bool with_dz, DwTmaGeom *out,
+                                   unsigned *grid) {
+    const int max_consumers = with_dz ? 224 : 256;            // consumer threads; the producer warp comes on top
     DwTmaGeom g{};
     g.n = pb.n; g.c = pb.c_in; g.h_in = pb.h_in; g.w_in = pb.w_in; g.h_out = pb.h_out; g.w_out = pb.w_out;
     g.pad_h = pb.pad_h; g.pad_w = pb.pad_w;
     const int v = pb.c_in / 4;
-    const int tcols = (pb.w_out + TW - 1) / TW;               // thread columns in a row
-    int cols_max = 256 / v;                                    // at most 256 consumer threads
+    const int tcols = (pb.w_out + tw - 1) / tw;                // thread columns in a row
+    int cols_max = max_consumers / v;
     if (cols_max < 1) cols_max = 1;
-    if (cols_max > 254 / TW) cols_max = 254 / TW;              // box width (cols TW + KW - 1) <= 256
+    if (cols_max > 254 / tw) cols_max = 254 / tw;              // box width (cols tw + kw - 1) <= 256
     if (cols_max > tcols) cols_max = tcols;
     g.strips = (tcols + cols_max - 1) / cols_max;
     g.cols_t = (tcols + g.strips - 1) / g.strips;
     g.consumer_warps = (g.cols_t * v + 31) / 32;
-    g.row_bytes = (g.cols_t * TW + KW - 1) * pb.c_in * 2;
+    g.row_bytes = (g.cols_t * tw + kw - 1) * pb.c_in * 2;
     g.stage_stride = (g.row_bytes + 127) / 128 * 128;
+    if (with_dz) g.stage_stride += (g.cols_t * tw * pb.c_in * 2 + 127) / 128 * 128;
     g.stages = (int)((96 * 1024) / g.stage_stride);
     if (g.stages > kDwMaxStages) g.stages = kDwMaxStages;
     if (g.stages < 4) return cudaErrorInvalidValue;
@@ -261,32 +466,87 @@ cudaError_t launch_dw_tma(const Problem &pb, const void *x, const void *w, const
     for (int th = 4; th <= pb.h_out; ++th) {
         const long long bands = (pb.h_out + th - 1) / th;
         const long long per_block = ((long long)pb.n * bands * g.strips + resident - 1) / resident;
-        const long long cost = per_block * (th + KH - 1);
+        const long long cost = per_block * (th + kh - 1);
         if (best < 0 || cost < best) { best = cost; g.th = th; }
     }
-    if (pb.h_out < 4) g.th = pb.h_out;
     g.bands = (pb.h_out + g.th - 1) / g.th;
     const long long items = (long long)pb.n * g.bands * g.strips;
-    const unsigned grid = (unsigned)(items < resident ? items : resident);
+    *grid = (unsigned)(items < resident ? items : resident);
+    *out = g;
+    return cudaSuccess;
+}
 
+static bool dw_tma_map(CUtensorMap *tm, const void *base, int n, int h, int w, int c, int box_w) {
+    const unsigned long long dims[4] = {(unsigned long long)c, (unsigned long long)w, (unsigned long long)h,
+                                        (unsigned long long)n};
+    const unsigned long long str[4] = {0, (unsigned long long)c * 2, (unsigned long long)w * c * 2,
+                                       (unsigned long long)h * w * c * 2};
+    const unsigned int box[4] = {(unsigned)c, (unsigned)box_w, 1, 1};
+    return make_tmap_tiled_bf16_linear(tm, base, 4, dims, str, box);
+}
+
+static size_t dw_tma_smem(const DwTmaGeom &g) {
+    return 128 + ((sizeof(DwTmaCtl) + 127) / 128) * 128 + (size_t)g.stages * g.stage_stride;
+}
+
+cudaError_t launch_dw_tma(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
+                          cudaStream_t st) {
+    constexpr int TW = 2, KH = 3, KW = 3;
+    DwTmaGeom g;
+    unsigned grid = 0;
+    cudaError_t e = dw_tma_geometry(pb, TW, KH, KW, false, &g, &grid);
+    if (e != cudaSuccess) return e;
     CUtensorMap tx;
-    const unsigned long long dims[4] = {(unsigned long long)pb.c_in, (unsigned long long)pb.w_in,
-                                        (unsigned long long)pb.h_in, (unsigned long long)pb.n};
-    const unsigned long long str[4] = {0, (unsigned long long)pb.c_in * 2, (unsigned long long)pb.w_in * pb.c_in * 2,
-                                       (unsigned long long)pb.h_in * pb.w_in * pb.c_in * 2};
-    const unsigned int box[4] = {(unsigned)pb.c_in, (unsigned)(g.cols_t * TW + KW - 1), 1, 1};
-    if (!make_tmap_tiled_bf16_linear(&tx, x, 4, dims, str, box)) return cudaErrorInvalidValue;
+    if (!dw_tma_map(&tx, x, pb.n, pb.h_in, pb.w_in, pb.c_in, g.cols_t * TW + KW - 1)) return cudaErrorInvalidValue;
     int *err = nullptr;
     if ((e = error_word_address(&err)) != cudaSuccess) return e;
-    const size_t smem = 128 + ((sizeof(DwTmaCtl) + 127) / 128) * 128 + (size_t)g.stages * g.stage_stride;
     static bool attr = false;
     if (!attr) {
         e = cudaFuncSetAttribute(dw_tma_kernel<TW, KH, KW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024);
         if (e != cudaSuccess) return e;
         attr = true;
     }
-    dw_tma_kernel<TW, KH, KW><<<grid, (g.consumer_warps + 1) * 32, smem, st>>>(tx, g, (const __nv_bfloat16 *)w, bias,
-                                                                              (uint2 *)z, err);
+    dw_tma_kernel<TW, KH, KW><<<grid, (g.consumer_warps + 1) * 32, dw_tma_smem(g), st>>>(
+        tx, g, (const __nv_bfloat16 *)w, bias, (uint2 *)z, err);
+    return cudaGetLastError();
+}
+
+// Partial rows the backward-weight kernel writes: one per block, [C][KH KW + 1] floats each.
+size_t dw_tma_wgrad_partial_bytes(const Problem &pb) {
+    DwTmaGeom g;
+    unsigned grid = 0;
+    if (dw_tma_geometry(pb, 2, 3, 3, true, &g, &grid) != cudaSuccess) return 0;
+    return (size_t)grid * pb.c_in * 10 * sizeof(float);
+}
+
+cudaError_t launch_dw_tma_wgrad(const Problem &pb, const void *dz, const void *x, float *part, int *nparts,
+                                cudaStream_t st) {
+    constexpr int TW = 2, KH = 3, KW = 3;
+    DwTmaGeom g;
+    unsigned grid = 0;
+    cudaError_t e = dw_tma_geometry(pb, TW, KH, KW, true, &g, &grid);
+    if (e != cudaSuccess) return e;
+    CUtensorMap tx, tdz;
+    if (!dw_tma_map(&tx, x, pb.n, pb.h_in, pb.w_in, pb.c_in, g.cols_t * TW + KW - 1)) return cudaErrorInvalidValue;
+    if (!dw_tma_map(&tdz, dz, pb.n, pb.h_out, pb.w_out, pb.c_in, g.cols_t * TW)) return cudaErrorInvalidValue;
+    int *err = nullptr;
+    if ((e = error_word_address(&err)) != cudaSuccess) return e;
+    static bool attr = false;
+    if (!attr) {
+        e = cudaFuncSetAttribute(dw_tma_wgrad_kernel<TW, KH, KW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024);
+        if (e != cudaSuccess) return e;
+        attr = true;
+    }
+    dw_tma_wgrad_kernel<TW, KH, KW><<<grid, (g.consumer_warps + 1) * 32, dw_tma_smem(g), st>>>(tx, tdz, g, part, err);
+    *nparts = (int)grid;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_dw_wgrad_finish(const Problem &pb, const float *part, int nparts, const void *w, const float *vec3,
+                                   const float *b, const float *mean, float *dw, float *db, float *dgamma,
+                                   float *dbeta, cudaStream_t st) {
+    dw_wgrad_finish_kernel<9><<<pb.c_in, 32 * 10, 0, st>>>(pb.c_in, nparts, part, (const __nv_bfloat16 *)w, vec3, b, mean,
+                                                         dw, db, dgamma, dbeta);
     return cudaGetLastError();
 }
 

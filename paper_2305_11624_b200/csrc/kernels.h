@@ -124,6 +124,13 @@ bool dw_eligible(const Problem &pb);
 bool dw_tma_eligible(const Problem &pb);
 cudaError_t launch_dw_tma(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
                           cudaStream_t st);
+// backward weight on the same stream: block partials [nparts][C][10] (9 taps, then sum dZ), then the finish
+size_t dw_tma_wgrad_partial_bytes(const Problem &pb);
+cudaError_t launch_dw_tma_wgrad(const Problem &pb, const void *dz, const void *x, float *part, int *nparts,
+                                cudaStream_t st);
+cudaError_t launch_dw_wgrad_finish(const Problem &pb, const float *part, int nparts, const void *w, const float *vec3,
+                                   const float *b, const float *mean, float *dw, float *db, float *dgamma,
+                                   float *dbeta, cudaStream_t st);
 bool dw_wgrad_supported(const Problem &pb);     // tap counts the register-tiled kernel is built for
 cudaError_t launch_dw_fwd(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
                           cudaStream_t st);
