@@ -340,17 +340,20 @@ __global__ void __launch_bounds__(1024) wgrad_epilogue_fused_kernel(
     const size_t slice = (size_t)kdim * c_out;
     {
         const int k = k0 + ty;
-        float a0 = 0.f, a1 = 0.f;
+        // eight independent sums per thread keep eight loads in flight; they are added in a fixed order
+        float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         if (k < kdim) {
             const float *src = part + (size_t)k * c_out + co0 + tx;
             int sp = tz;
-            for (; sp + SL < splits; sp += 2 * SL) {
-                a0 += src[(size_t)sp * slice];
-                a1 += src[(size_t)(sp + SL) * slice];
+            for (; sp + 7 * SL < splits; sp += 8 * SL) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) a[u] += __ldcg(src + (size_t)(sp + u * SL) * slice);
             }
-            if (sp < splits) a0 += src[(size_t)sp * slice];
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (sp + u * SL < splits) a[u] += __ldcg(src + (size_t)(sp + u * SL) * slice);
         }
-        tile[tz][ty][tx] = a0 + a1;
+        tile[tz][ty][tx] = ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
     }
     __syncthreads();
     if (threadIdx.x < 32 * KR) {
