@@ -314,7 +314,8 @@ cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
 // ---- epilogue over k-major partials ------------------------------------------------------------
 // One kernel finishes every parameter gradient (Table 2, Tune row) from the fp32 partial tiles:
 //   block (bx, by): 32 output channels x KR k rows x SL lanes over the pixel slices (KR SL = 32,
-//   1024 threads): (8, 4) when there are few slices, (2, 16) when there are many
+//   up to 1024 threads), REP such row groups one after the other: (8, 4) when there are few slices, (2, 16)
+//   when there are many, (8, 1) x 4 with 256 threads when there are few slices and thousands of blocks
 //     acc[k][co] = sum_split part[split][k][co]        (each lane a strided subset, lanes added in order)
 //     dw[co][k]  = s[co] acc                           (transposed through shared memory)
 //     dotpart[by][co] = sum over the block's k rows of acc * w[co][k]
@@ -323,23 +324,31 @@ cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
 //   tree, so the result does not depend on which block came last:
 //     dbeta = sum dZ,  db = s dbeta,  dgamma = r (sum_k domega' omega + dbeta (b - mu_hat))
 //   plain mode (vec3 == NULL): dw = acc, db = sum dZ if requested.
-template <int KR, int SL>
-__global__ void __launch_bounds__(1024) wgrad_epilogue_fused_kernel(
+template <int KR, int SL, int REP>
+__global__ void __launch_bounds__(32 * KR * SL) wgrad_epilogue_fused_kernel(
     int c_out, int kdim, const float *__restrict__ part, int splits, const float *__restrict__ bsum, int bsplits,
     const __nv_bfloat16 *__restrict__ w, const float *__restrict__ vec3, const float *__restrict__ b,
     const float *__restrict__ mean, float *__restrict__ dw, float *__restrict__ dotpart,
     unsigned int *__restrict__ counters, float *__restrict__ db, float *__restrict__ dgamma,
     float *__restrict__ dbeta, int need_sums) {
-    static_assert(KR * SL == 32, "one block is 32 x 32 threads");
-    __shared__ float tile[SL][KR][33];
+    static_assert(KR * SL <= 32, "at most 32 warps per block");
+    __shared__ float tile[REP][SL][KR][33];
     __shared__ int is_last;
     pdl_wait();
     pdl_launch_dependents();
     const int tx = threadIdx.x & 31, ty = (threadIdx.x >> 5) % KR, tz = (threadIdx.x >> 5) / KR;
-    const int co0 = blockIdx.x * 32, k0 = blockIdx.y * KR;
+    const int co0 = blockIdx.x * 32, k0 = blockIdx.y * (KR * REP);   // REP groups of KR rows per block
     const size_t slice = (size_t)kdim * c_out;
-    {
-        const int k = k0 + ty;
+    // the weights the second phase multiplies with are requested now, together with the partials
+    float wv[REP];
+#pragma unroll
+    for (int rep = 0; rep < REP; ++rep) {
+        const int k = k0 + rep * KR + (int)(threadIdx.x % KR), co = co0 + (int)(threadIdx.x / KR);
+        wv[rep] = (vec3 && threadIdx.x < 32 * KR && k < kdim) ? __bfloat162float(w[(size_t)co * kdim + k]) : 0.f;
+    }
+#pragma unroll
+    for (int rep = 0; rep < REP; ++rep) {
+        const int k = k0 + rep * KR + ty;
         // eight independent sums per thread keep eight loads in flight; they are added in a fixed order
         float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         if (k < kdim) {
@@ -353,19 +362,23 @@ __global__ void __launch_bounds__(1024) wgrad_epilogue_fused_kernel(
             for (int u = 0; u < 8; ++u)
                 if (sp + u * SL < splits) a[u] += __ldcg(src + (size_t)(sp + u * SL) * slice);
         }
-        tile[tz][ty][tx] = ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
+        tile[rep][tz][ty][tx] = ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
     }
     __syncthreads();
     if (threadIdx.x < 32 * KR) {
-        const int kk = threadIdx.x % KR, cl = threadIdx.x / KR, k = k0 + kk, co = co0 + cl;
+        const int kk = threadIdx.x % KR, cl = threadIdx.x / KR, co = co0 + cl;
         float d = 0.f;
-        if (k < kdim) {
-            float v = 0.f;
 #pragma unroll
-            for (int z = 0; z < SL; ++z) v += tile[z][kk][cl];
-            const size_t o = (size_t)co * kdim + k;
-            dw[o] = (vec3 ? vec3[co] : 1.f) * v;
-            if (vec3) d = v * __bfloat162float(w[o]);
+        for (int rep = 0; rep < REP; ++rep) {
+            const int k = k0 + rep * KR + kk;
+            if (k < kdim) {
+                float v = 0.f;
+#pragma unroll
+                for (int z = 0; z < SL; ++z) v += tile[rep][z][kk][cl];
+                const size_t o = (size_t)co * kdim + k;
+                dw[o] = (vec3 ? vec3[co] : 1.f) * v;
+                d = fmaf(v, wv[rep], d);
+            }
         }
         if (vec3) {
 #pragma unroll
@@ -384,8 +397,8 @@ __global__ void __launch_bounds__(1024) wgrad_epilogue_fused_kernel(
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    const int warp = threadIdx.x >> 5, lane = tx;
-    const int co = co0 + warp;                      // 32 warps, one per channel
+    const int lane = tx;
+    for (int co = co0 + (int)(threadIdx.x >> 5); co < co0 + 32; co += KR * SL) {   // a warp per channel
     float dsum = 0.f, dot = 0.f;
     for (int sp = lane; sp < bsplits; sp += 32) dsum += __ldcg(bsum + (size_t)sp * c_out + co);
     if (vec3)
@@ -404,6 +417,7 @@ __global__ void __launch_bounds__(1024) wgrad_epilogue_fused_kernel(
             dgamma[co] = r * (dot + dsum * ((b ? b[co] : 0.f) - mean[co]));
         }
     }
+    }
     if (threadIdx.x == 0) counters[blockIdx.x] = 0;   // leave the counter clean for the next call
 }
 
@@ -414,17 +428,17 @@ cudaError_t launch_wgrad_epilogue_fused(const Problem &pb, const UmmaWgradPlan &
     const dim3 grid(pb.c_out / 32, pl.kt);
     const int ns = need_sums ? 1 : 0;
     static bool carve_a = false, carve_b = false;
-    prefer_max_shared_once(wgrad_epilogue_fused_kernel<8, 4>, &carve_a);
-    prefer_max_shared_once(wgrad_epilogue_fused_kernel<2, 16>, &carve_b);
-    if (pl.kr == 32)
-        return launch_pdl(wgrad_epilogue_fused_kernel<32, 1>, grid, dim3(1024), 0, st, pb.c_out, pb.kdim, partials,
+    prefer_max_shared_once(wgrad_epilogue_fused_kernel<8, 4, 1>, &carve_a);
+    prefer_max_shared_once(wgrad_epilogue_fused_kernel<2, 16, 1>, &carve_b);
+    if (pl.kr == 32)                                  // 4 groups of 8 rows, 256 threads: several blocks per SM
+        return launch_pdl(wgrad_epilogue_fused_kernel<8, 1, 4>, grid, dim3(256), 0, st, pb.c_out, pb.kdim, partials,
                           pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw, dotpart, counters, db,
                           dgamma, dbeta, ns);
     if (pl.kr == 8)
-        return launch_pdl(wgrad_epilogue_fused_kernel<8, 4>, grid, dim3(1024), 0, st, pb.c_out, pb.kdim, partials,
+        return launch_pdl(wgrad_epilogue_fused_kernel<8, 4, 1>, grid, dim3(1024), 0, st, pb.c_out, pb.kdim, partials,
                           pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw, dotpart, counters, db,
                           dgamma, dbeta, ns);
-    return launch_pdl(wgrad_epilogue_fused_kernel<2, 16>, grid, dim3(1024), 0, st, pb.c_out, pb.kdim, partials,
+    return launch_pdl(wgrad_epilogue_fused_kernel<2, 16, 1>, grid, dim3(1024), 0, st, pb.c_out, pb.kdim, partials,
                       pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw, dotpart, counters, db,
                       dgamma, dbeta, ns);
 }
