@@ -325,7 +325,10 @@ int run_conv_fwd(const convbn_desc *d, const Problem &pb, const void *x, const v
                           -pb.pad_h, -pb.pad_w, pb.stride_h, pb.stride_w, pb.dil_h, pb.dil_w, 1};
         if (!umma_conv_eligible(s)) return CONVBN_EUNSUPPORTED;
         LAUNCH("expand_blockdiag", launch_expand_blockdiag(pb, w, nullptr, wbd_scratch, false, st));
-        LAUNCH("grouped_fwd", launch_umma_conv(s, x, wbd_scratch, bias, z, st));
+        if (umma_strip_eligible(s))
+            LAUNCH("grouped_fwd", launch_umma_strip_conv(s, x, wbd_scratch, bias, z, st));
+        else
+            LAUNCH("grouped_fwd", launch_umma_conv(s, x, wbd_scratch, bias, z, st));
         *which = "grouped-umma";
     } else if (umma_fwd_shape(d, pb, &s)) {
         if (umma_strip_eligible(s)) {
@@ -359,7 +362,10 @@ int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, cons
                           pb.dil_w, 1};
         if (!umma_conv_eligible(s)) return CONVBN_EUNSUPPORTED;
         LAUNCH("expand_blockdiag", launch_expand_blockdiag(pb, w, scale, wbd_scratch, true, st));
-        LAUNCH("grouped_dgrad", launch_umma_conv(s, dz, wbd_scratch, nullptr, dx, st));
+        if (umma_strip_eligible(s))
+            LAUNCH("grouped_dgrad", launch_umma_strip_conv(s, dz, wbd_scratch, nullptr, dx, st));
+        else
+            LAUNCH("grouped_dgrad", launch_umma_conv(s, dz, wbd_scratch, nullptr, dx, st));
         *which = "grouped-umma";
     } else if (strided_dgrad_ok(d, pb)) {
         // Strided backward data, one stride-1 GEMM per residue class (a, b) of the input position:

@@ -31,6 +31,7 @@ struct StripGemm {
     int tiles_h, tiles_w;
     uint32_t strip_bytes;             // one patch buffer (multiple of 1024)
     int nacc;                         // accumulator sets in tensor memory (1 or 2)
+    int blockdiag;                    // grouped conv as block-diagonal 64-channel GEMMs: output block j reads input chunk j
     uint32_t tmem_cols;
     __nv_bfloat16 *out;
     BnFold fold;
@@ -58,7 +59,8 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
     float *scale_s = bias_s + g.cn;
     const bool fold = g.fold.gamma != nullptr;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int cchunks = g.ca / 64, taps = g.kh * g.kw;
+    const int cchunks = g.blockdiag ? 1 : g.ca / 64, taps = g.kh * g.kw;
+    const int w_ca = g.blockdiag ? 64 : g.ca;          // K extent of one tap in the weight matrix
     const uint32_t n_tiles = (uint32_t)g.cn / BN;
     const uint32_t sp_tiles = (uint32_t)g.n * g.tiles_h * g.tiles_w;
     const uint32_t total_tiles = sp_tiles * n_tiles;
@@ -123,8 +125,8 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
                 for (int cc = 0; cc < cchunks; ++cc) {
                     if (!mbar_wait_bounded(&ctl->strip_empty[sb], ph ^ 1u, abort_flag)) { ok = false; break; }
                     mbar_arrive_expect_tx(&ctl->strip_full[sb], bytes);
-                    tma_load_4d(strips + (size_t)sb * g.strip_bytes, &tm_act, &ctl->strip_full[sb], cc * 64,
-                                w0 + g.lower_w, h0 + g.lower_h, img);
+                    tma_load_4d(strips + (size_t)sb * g.strip_bytes, &tm_act, &ctl->strip_full[sb],
+                                g.blockdiag ? n0 : cc * 64, w0 + g.lower_w, h0 + g.lower_h, img);
                     if (++sb == 2) { sb = 0; ph ^= 1u; }
                 }
             }
@@ -145,7 +147,7 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
                     for (int tap = 0; tap < taps; ++tap) {
                         if (!mbar_wait_bounded(&ctl->b_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
                         mbar_arrive_expect_tx(&ctl->b_full[s], kBBytes);
-                        tma_load_2d(bring + (size_t)s * kBBytes, &tm_w, &ctl->b_full[s], tap * g.ca + cc * 64, n0);
+                        tma_load_2d(bring + (size_t)s * kBBytes, &tm_w, &ctl->b_full[s], tap * w_ca + cc * 64, n0);
                         if (++s == kSBStages) { s = 0; ph ^= 1u; }
                     }
             }
@@ -268,15 +270,32 @@ namespace {
 
 struct StripPlan { bool ok = false; int bn = 64, R = 0, CW = 0, Wt = 0, nmb = 0, nacc = 2, tiles_w = 1 << 20; uint32_t strip_bytes = 0; size_t smem = 0; };
 
+int strip_sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0, v = 0;
+        n = (cudaGetDevice(&dev) == cudaSuccess &&
+             cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) ? v : 148;
+    }
+    return n;
+}
+
 StripPlan plan_strip(const UmmaConvShape &s) {
     StripPlan best;
-    if (s.stride_h != 1 || s.stride_w != 1 || s.dil_h != 1 || s.dil_w != 1 || s.blockdiag || s.out_sw) return best;
+    if (s.stride_h != 1 || s.stride_w != 1 || s.dil_h != 1 || s.dil_w != 1 || s.out_sw) return best;
+    if (s.blockdiag && s.ca != s.cn) return best;
     if (s.taps_h * s.taps_w < 2 || s.ca % 64 || s.cn % 64 || s.cn > 4096 || s.wo < 14 || s.ho < 2) return best;
     if ((long long)s.n * s.ho * s.wo >= (1LL << 30)) return best;
-    const int bn = (s.cn % 128 == 0) ? 128 : 64;
+    const int bn = (s.cn % 128 == 0 && !s.blockdiag) ? 128 : 64;
     const int nmb_max = 512 / bn / 2;                      // two accumulator sets
     const int tiles_w_min = (s.wo + (256 - s.taps_w + 1) - 1) / (256 - s.taps_w + 1);
-    double best_eff = 0.0, best_score = -1.0;
+    // Among the tilings that keep at least 70 % of the MMA rows useful, take the one with the lowest
+    // estimated time: rounds over the SMs x (the larger of the tile's MMA issue time and its shared-memory
+    // fill time, plus a fixed cost per tile).  The weight tiles are streamed again for every tile, so small
+    // tiles pay for them many times over.
+    const int cchunks = s.blockdiag ? 1 : s.ca / 64, taps = s.taps_h * s.taps_w;
+    const int n_tiles = s.cn / bn, sms = strip_sm_count();
+    double best_eff = 0.0, best_cost = -1.0;
     for (int tiles_w = tiles_w_min; tiles_w < tiles_w_min + 4; ++tiles_w) {
     const int cw = (s.wo + tiles_w - 1) / tiles_w, wt = cw + s.taps_w - 1;
     if (cw < 8) break;
@@ -288,13 +307,16 @@ StripPlan plan_strip(const UmmaConvShape &s) {
         const size_t smem = 1024 + 2 * (size_t)sbytes + (size_t)kSBStages * bn * 128 + sizeof(StripCtl) +
                             2 * (size_t)s.cn * sizeof(float) + 32;
         if (smem > 224 * 1024) break;
-        // useful fraction of the MMA rows, derated by the halo rows that are loaded again by the next tile
         const int tiles_h = (s.ho + r - 1) / r;
         const double eff = (double)s.ho * s.wo / ((double)tiles_h * tiles_w * nmb * 128.0);
-        // prefer the useful fraction; among equals fewer column tiles (less halo), then taller tiles
-        const double score = eff - 0.01 * (tiles_w - tiles_w_min) + 1e-4 * r;
-        if (score > best_score) {
-            best_score = score;
+        if (eff < 0.70) continue;
+        const double mma_clk = (double)nmb * taps * cchunks * 4 * (bn == 64 ? 67.0 : 128.0);
+        const double fill_clk = ((double)(r + s.taps_h - 1) * wt * 128.0 + (double)taps * bn * 128.0) * cchunks / 32.0;
+        const double tile_clk = (mma_clk > fill_clk ? mma_clk : fill_clk) + 1500.0;
+        const long long tiles = (long long)s.n * tiles_h * tiles_w * n_tiles;
+        const double cost = (double)((tiles + sms - 1) / sms) * tile_clk;
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
             best_eff = eff;
             best.ok = true; best.bn = bn; best.R = r; best.CW = cw; best.Wt = wt; best.nmb = nmb;
             best.strip_bytes = sbytes; best.smem = smem; best.tiles_w = tiles_w;
@@ -329,15 +351,6 @@ bool make_tmap_nhwc_box(CUtensorMap *tm, const void *base, int n, int h, int w, 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int strip_sm_count() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0, v = 0;
-        n = (cudaGetDevice(&dev) == cudaSuccess &&
-             cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) ? v : 148;
-    }
-    return n;
-}
 
 template <int BN>
 cudaError_t launch_strip(const CUtensorMap &ta, const CUtensorMap &tw, const StripGemm &g, size_t smem,
@@ -374,6 +387,7 @@ cudaError_t launch_umma_strip_conv(const UmmaConvShape &s, const void *act, cons
     g.tiles_h = (s.ho + pl.R - 1) / pl.R; g.tiles_w = (s.wo + pl.CW - 1) / pl.CW;
     g.strip_bytes = pl.strip_bytes;
     g.nacc = 2;
+    g.blockdiag = s.blockdiag;
     int cols = 2 * pl.nmb * pl.bn, p2 = 32;
     while (p2 < cols) p2 <<= 1;
     g.tmem_cols = (uint32_t)p2;
@@ -381,7 +395,7 @@ cudaError_t launch_umma_strip_conv(const UmmaConvShape &s, const void *act, cons
     g.fold = fold ? *fold : BnFold{nullptr, nullptr, nullptr, nullptr, nullptr, 0.f, nullptr};
     CUtensorMap ta, tw;
     if (!make_tmap_nhwc_box(&ta, act, s.n, s.ha, s.wa, s.ca, pl.Wt, g.rows_in)) return cudaErrorInvalidValue;
-    if (!make_tmap_matrix_bf16(&tw, wmat, s.cn, (long long)s.taps_h * s.taps_w * s.ca, pl.bn, 64))
+    if (!make_tmap_matrix_bf16(&tw, wmat, s.cn, (long long)s.taps_h * s.taps_w * (s.blockdiag ? 64 : s.ca), pl.bn, 64))
         return cudaErrorInvalidValue;
     int *err = nullptr;
     cudaError_t e = error_word_address(&err);

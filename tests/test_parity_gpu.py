@@ -51,6 +51,8 @@ SMALL = [
     L("b_grouped_cg4", 1, 64, 10, 12, 64, 3, 3, pad=1, groups=16),
     L("b_grouped_cg32_s2", 2, 128, 11, 9, 128, 3, 3, stride=2, pad=1, groups=4),
     L("b_dw_5x5", 1, 48, 11, 13, 48, 5, 5, pad=2, groups=48),
+    # grouped, wide enough for the patch-reuse kernel (block-diagonal mode): two 64-channel blocks
+    L("b_grouped_wide", 2, 128, 17, 22, 128, 3, 3, pad=1, groups=16),
     L("b_dw_nopad", 3, 32, 13, 37, 32, 3, 3, pad=0, groups=32),
     L("b_dw_wide_c", 1, 256, 9, 21, 256, 3, 3, pad=1, groups=256),
     # narrow-input (stem) path: 4 and 8 input channels, two output-channel chunk groups, stride 1 and 3
