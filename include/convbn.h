@@ -196,9 +196,11 @@ size_t convbn_host_step_arena_bytes(const convbn_desc *desc);
 /* Forward, backward-data and backward-weight of one block (the three Tune-row calls above, Sec. 3.4
  * and Table 2) with every tensor in HOST memory: x, dz, w, b (NULL = no bias), gamma, beta,
  * run_mean, run_var are host inputs; z, dx, dw, db (NULL iff b is NULL), dgamma, dbeta are host
- * outputs, in the dtype / layout conventions above.  Copies are asynchronous on `stream` (use
- * page-locked host memory for them to overlap); outputs are valid once the stream has been
- * synchronised.  `device_arena` is caller-owned DEVICE scratch of at least
+ * outputs, in the dtype / layout conventions above.  Copies are asynchronous (use page-locked host
+ * memory for them to overlap): everything is ordered on `stream`, except that dZ is uploaded on a
+ * second, library-owned stream (one per device, created on the first call there) so that it crosses
+ * the bus while Z comes back; `stream` waits for it before the backward kernels.  Outputs are valid,
+ * and the host inputs may be reused, once `stream` has been synchronised.  `device_arena` is caller-owned DEVICE scratch of at least
  * convbn_host_step_arena_bytes(desc) bytes, 256-byte aligned. */
 int convbn_tune_step_host(const convbn_desc *desc, const void *x, const void *dz, const void *w,
                           const float *b, const float *gamma, const float *beta,

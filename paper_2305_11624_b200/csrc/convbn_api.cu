@@ -759,6 +759,29 @@ size_t convbn_host_step_arena_bytes(const convbn_desc *desc) {
     return make_host_arena(desc, pb).total;
 }
 
+namespace {
+// Second copy lane of convbn_tune_step_host: one stream and two events per device, made on first use.
+// The upload of dZ runs there while the forward kernels and the download of Z run on the caller's
+// stream, so the two PCIe directions are busy at the same time.
+struct CopyLane { cudaStream_t stream = nullptr; cudaEvent_t inputs_queued = nullptr, dz_ready = nullptr; };
+CopyLane g_copy_lane[64];
+std::mutex g_copy_lane_mu;
+
+int copy_lane(CopyLane **out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return CONVBN_ECUDA;
+    CopyLane &l = g_copy_lane[dev];
+    if (!l.stream) {
+        if (cudaStreamCreateWithFlags(&l.stream, cudaStreamNonBlocking) != cudaSuccess) { l.stream = nullptr; return CONVBN_ECUDA; }
+        if (cudaEventCreateWithFlags(&l.inputs_queued, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&l.dz_ready, cudaEventDisableTiming) != cudaSuccess)
+            return CONVBN_ECUDA;
+    }
+    *out = &l;
+    return CONVBN_OK;
+}
+}  // namespace
+
 int convbn_tune_step_host(const convbn_desc *desc, const void *x, const void *dz, const void *w,
                           const float *b, const float *gamma, const float *beta,
                           const float *run_mean, const float *run_var, void *z, void *dx, float *dw,
@@ -790,11 +813,22 @@ int convbn_tune_step_host(const convbn_desc *desc, const void *x, const void *dz
     CU(h2d(ar.var, run_var, vb));
     if (b) CU(h2d(ar.b, b, vb));
     const float *db_dev = b ? (const float *)(d + ar.b) : nullptr;
-    CK(convbn_tune_fwd(desc, d + ar.x, d + ar.w, db_dev, (const float *)(d + ar.gamma),
-                       (const float *)(d + ar.beta), (const float *)(d + ar.mean),
-                       (const float *)(d + ar.var), d + ar.z, d + ar.saved, d + ar.ws, ar.ws_bytes, stream));
-    CU(d2h(z, ar.z, ar.z_bytes));
-    CU(h2d(ar.dz, dz, ar.z_bytes));
+    {
+        // dZ goes up on the second lane, after the inputs above (and after everything queued earlier on
+        // `stream`, which may still read the arena), while the forward pass and the download of Z run here
+        std::lock_guard<std::mutex> lk(g_copy_lane_mu);
+        CopyLane *lane = nullptr;
+        CK(copy_lane(&lane));
+        CU(cudaEventRecord(lane->inputs_queued, st));
+        CU(cudaStreamWaitEvent(lane->stream, lane->inputs_queued, 0));
+        CU(cudaMemcpyAsync(d + ar.dz, dz, ar.z_bytes, cudaMemcpyHostToDevice, lane->stream));
+        CU(cudaEventRecord(lane->dz_ready, lane->stream));
+        CK(convbn_tune_fwd(desc, d + ar.x, d + ar.w, db_dev, (const float *)(d + ar.gamma),
+                           (const float *)(d + ar.beta), (const float *)(d + ar.mean),
+                           (const float *)(d + ar.var), d + ar.z, d + ar.saved, d + ar.ws, ar.ws_bytes, stream));
+        CU(d2h(z, ar.z, ar.z_bytes));
+        CU(cudaStreamWaitEvent(st, lane->dz_ready, 0));
+    }
     CK(convbn_tune_bwd_data(desc, d + ar.dz, d + ar.w, d + ar.saved, d + ar.dx, d + ar.ws, ar.ws_bytes, stream));
     CU(d2h(dx, ar.dx, ar.x_bytes));
     CK(convbn_tune_bwd_weight(desc, d + ar.dz, d + ar.x, d + ar.w, db_dev, (const float *)(d + ar.mean),

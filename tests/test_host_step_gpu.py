@@ -1,0 +1,45 @@
+"""convbn_tune_step_host (host buffers in, host buffers out) against the fp64 oracle."""
+import numpy as np
+import pytest
+
+from paper_2305_11624_b200 import inputs as I
+
+import parity
+
+pytestmark = pytest.mark.gpu
+
+SPECS = [
+    I.LayerSpec("h_3x3", 2, 64, 18, 20, 128, 3, 3, pad=1),
+    I.LayerSpec("h_bias_f32", 2, 8, 9, 7, 12, 3, 3, pad=1, dtype="f32", layout="nchw", bias=True),
+    I.LayerSpec("h_dw", 1, 32, 13, 17, 32, 3, 3, pad=1, groups=32),
+]
+
+
+@pytest.mark.parametrize("spec", SPECS, ids=lambda s: s.name)
+def test_host_step(spec):
+    import torch
+    from paper_2305_11624_b200 import convbn as C
+    from paper_2305_11624_b200.harness import Block
+
+    t = parity.make_inputs(spec, 77)
+    ref = parity.oracle_tune(spec, t)
+    blk = Block(spec, device="cuda:0", modes=("tune",))
+    blk.load(t)                                        # device copies are only the templates of the host ones
+    pin = lambda a: None if a is None else a.detach().cpu().pin_memory()
+    out = lambda a: None if a is None else torch.zeros(a.shape, dtype=a.dtype).pin_memory()
+    ins = [pin(a) for a in (blk.x, blk.dz, blk.w, blk.b, blk.gamma, blk.beta, blk.mu_hat, blk.var_hat)]
+    outs = [out(a) for a in (blk.z, blk.dx, blk.dw, blk.db, blk.dgamma, blk.dbeta)]
+    arena = torch.empty(C.convbn_host_step_arena_bytes(blk.desc), dtype=torch.uint8, device="cuda:0")
+    for _ in range(2):                                 # twice: the second call reuses the arena and the copy lane
+        C.convbn_tune_step_host(blk.desc, *ins, *outs, arena)
+        torch.cuda.synchronize()
+        C.convbn_check()
+    # put the host results where Block.fetch reads them, to reuse its layout conversions
+    for name, h in zip(("z", "dx", "dw", "db", "dgamma", "dbeta"), outs):
+        if h is not None:
+            getattr(blk, name).copy_(h)
+    names = ["z", "dx", "dw", "dgamma", "dbeta"] + (["db"] if spec.bias else [])
+    got = {k: blk.fetch(k) for k in names}
+    if not spec.bias:
+        got["db"] = None
+    parity.compare(got, ref, parity.TOL[spec.dtype], parity.TUNE_OUTPUTS, spec.name)
