@@ -377,6 +377,28 @@ int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, cons
         if (any_empty &&
             cudaMemsetAsync(dx, 0, (size_t)pb.pin * pb.c_in * elem_size(d->dtype), st) != cudaSuccess)
             return CONVBN_ECUDA;
+        // one launch writes every class's weight matrix (when the kernel has at most 64 taps)
+        const bool merged = pb.kh * pb.kw <= 64;
+        if (merged) {
+            ClassTapTable where;
+            memset(&where, 0, sizeof(where));
+            size_t eoff = 0;
+            for (int a = 0; a < pb.stride_h && a < pb.h_in; ++a)
+                for (int b2 = 0; b2 < pb.stride_w && b2 < pb.w_in; ++b2) {
+                    const ClassTaps ch = class_taps(a, pb.pad_h, pb.kh, pb.stride_h);
+                    const ClassTaps cw = class_taps(b2, pb.pad_w, pb.kw, pb.stride_w);
+                    if (ch.count == 0 || cw.count == 0) continue;
+                    for (int mh = 0; mh < ch.count; ++mh)
+                        for (int mw = 0; mw < cw.count; ++mw) {
+                            const int tap = (ch.r_max - pb.stride_h * mh) * pb.kw + (cw.r_max - pb.stride_w * mw);
+                            where.offset[tap] = (long long)eoff;
+                            where.count[tap] = ch.count * cw.count;
+                            where.pos[tap] = mh * cw.count + mw;
+                        }
+                    eoff += (size_t)ch.count * cw.count * pb.c_in * pb.c_out;
+                }
+            LAUNCH("reparam_dgrad", launch_reparam_dgrad_classes(pb, w, scale, w_scratch, where, st));
+        }
         size_t woff = 0;
         for (int a = 0; a < pb.stride_h && a < pb.h_in; ++a)
             for (int b2 = 0; b2 < pb.stride_w && b2 < pb.w_in; ++b2) {
@@ -393,8 +415,9 @@ int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, cons
                 cs.out_sh = pb.stride_h * pb.w_in * pb.c_in;
                 cs.out_sw = pb.stride_w * pb.c_in;
                 if (!umma_conv_eligible(cs)) return CONVBN_EUNSUPPORTED;
-                LAUNCH("reparam_dgrad", launch_reparam_dgrad_class(pb, w, scale, wc, ch.count, cw.count, ch.r_max,
-                                                                   cw.r_max, pb.stride_h, pb.stride_w, st));
+                if (!merged)
+                    LAUNCH("reparam_dgrad", launch_reparam_dgrad_class(pb, w, scale, wc, ch.count, cw.count, ch.r_max,
+                                                                       cw.r_max, pb.stride_h, pb.stride_w, st));
                 LAUNCH("umma_dgrad", launch_umma_conv(cs, dz, wc, nullptr,
                                                       (char *)dx + ((size_t)a * pb.w_in + b2) * pb.c_in *
                                                                        elem_size(d->dtype), st));

@@ -69,6 +69,14 @@ cudaError_t launch_reparam_dgrad(const Problem &pb, const void *w, const float *
                                  cudaStream_t st);
 // One parity class of a strided backward-data pass: w_t[ci][mh][mw][co] = s[co] w[co][r][q][ci] with
 // r = r_max - step_h mh, q = q_max - step_w mw for mh < th, mw < tw.
+// Per-tap placement for launch_reparam_dgrad_classes (strided backward data, at most 64 taps).
+struct ClassTapTable {
+    long long offset[64];   // element offset of the tap's class matrix in the scratch buffer
+    int count[64];          // taps of that class (0: unused tap)
+    int pos[64];            // position of the tap inside its class, row-major over (tap row, tap column)
+};
+cudaError_t launch_reparam_dgrad_classes(const Problem &pb, const void *w, const float *s_vec, void *w_t,
+                                         const ClassTapTable &where, cudaStream_t st);
 cudaError_t launch_reparam_dgrad_class(const Problem &pb, const void *w, const float *s_vec, void *w_t, int th,
                                        int tw, int r_max, int q_max, int step_h, int step_w, cudaStream_t st);
 

@@ -172,6 +172,42 @@ cudaError_t launch_reparam_dgrad_class(const Problem &pb, const void *w, const f
                       step_h, step_w, th * tw, (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t, pb.kh * pb.kw);
 }
 
+// All residue classes of a strided backward pass in one launch: tap t of the kernel belongs to exactly
+// one class; `where` gives, per tap, the element offset of its class matrix in w_t, the class's tap
+// count and the tap's position in the class (count 0: the tap is not used).
+__global__ void __launch_bounds__(256) reparam_dgrad_classes_kernel(int c_out, int c_in, ClassTapTable where,
+                                                                    const __nv_bfloat16 *__restrict__ w,
+                                                                    const float *__restrict__ s_vec,
+                                                                    __nv_bfloat16 *__restrict__ w_t, int taps) {
+    __shared__ float tile[32][33];
+    pdl_wait();
+    pdl_launch_dependents();
+    const int tap = blockIdx.z, ctaps = where.count[tap], ct = where.pos[tap];
+    if (ctaps == 0) return;
+    __nv_bfloat16 *dst = w_t + where.offset[tap];
+    const int co0 = blockIdx.y * 32, ci0 = blockIdx.x * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int j = ty; j < 32; j += 8) {
+        const int co = co0 + j, ci = ci0 + tx;
+        if (co < c_out && ci < c_in)
+            tile[j][tx] = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((long long)co * taps + tap) * c_in + ci]);
+    }
+    __syncthreads();
+    for (int j = ty; j < 32; j += 8) {
+        const int ci = ci0 + j, co = co0 + tx;
+        if (co < c_out && ci < c_in) dst[((long long)ci * ctaps + ct) * c_out + co] = __float2bfloat16_rn(tile[tx][j]);
+    }
+}
+
+cudaError_t launch_reparam_dgrad_classes(const Problem &pb, const void *w, const float *s_vec, void *w_t,
+                                         const ClassTapTable &where, cudaStream_t st) {
+    dim3 grid((pb.c_in + 31) / 32, (pb.c_out + 31) / 32, pb.kh * pb.kw);
+    static bool carve = false;
+    prefer_max_shared_once(reparam_dgrad_classes_kernel, &carve);
+    return launch_pdl(reparam_dgrad_classes_kernel, grid, dim3(256), 0, st, pb.c_out, pb.c_in, where,
+                      (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t, pb.kh * pb.kw);
+}
+
 cudaError_t launch_reparam_dgrad(const Problem &pb, const void *w, const float *s_vec, void *w_t,
                                  cudaStream_t st) {
     dim3 grid((pb.c_in + 31) / 32, (pb.c_out + 31) / 32, pb.kh * pb.kw);
