@@ -319,6 +319,10 @@ int run_conv_fwd(const convbn_desc *d, const Problem &pb, const void *x, const v
         LAUNCH("stem_expand", launch_stem_expand_weights(pb, w, nullptr, at(ws, pl.wst), st));
         LAUNCH("stem_fwd", launch_stem_fwd(pb, at(ws, pl.xpk), at(ws, pl.wst), bias, z, st));
         *which = "umma-stem";
+    } else if (grouped_path(d, pb) && grouped8_eligible(pb)) {
+        // 8 channels per group: warp-level MMAs on the (already folded) weights as they are
+        LAUNCH("grouped_fwd", launch_grouped8_fwd(pb, x, w, bias, z, st));
+        *which = "grouped-mma";
     } else if (grouped_path(d, pb)) {
         // block-diagonal GEMM: expand the (already folded) weights, then the dense tensor-core kernel
         s = UmmaConvShape{pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.c_out, pb.kh, pb.kw,
@@ -356,6 +360,10 @@ int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, cons
     if (stem_path(d, pb) && stem_dgrad_eligible(pb)) {
         LAUNCH("stem_dgrad", launch_stem_dgrad(pb, dz, w, scale, dx, st));
         *which = "stem-simt";
+    } else if (grouped_path(d, pb) && grouped8_eligible(pb)) {
+        LAUNCH("grouped_flip", launch_grouped8_flip_weights(pb, w, scale, wbd_scratch, st));
+        LAUNCH("grouped_dgrad", launch_grouped8_dgrad(pb, dz, wbd_scratch, dx, st));
+        *which = "grouped-mma";
     } else if (grouped_path(d, pb) && pb.stride_h == 1 && pb.stride_w == 1) {
         s = UmmaConvShape{pb.n, pb.h_out, pb.w_out, pb.c_out, pb.h_in, pb.w_in, pb.c_in, pb.kh, pb.kw,
                           pb.pad_h - (pb.kh - 1) * pb.dil_h, pb.pad_w - (pb.kw - 1) * pb.dil_w, 1, 1, pb.dil_h,

@@ -1,0 +1,270 @@
+// Grouped convolution with 8 channels per group (C_in/G = C_out/G = 8), bf16 NHWC, unit stride and dilation:
+//   Z[p, 8g + o] = b'[8g + o] + sum_{tap, ci} omega'[8g + o][tap][ci] X[p + tap, 8g + ci]     (Sec. 3.1 / 3.3)
+// and, with rotated and transposed weights, the backward-data pass (Sec. 3.2.1).
+// One group is a GEMM with N = 8 and K = 8 per tap (about 36 FLOP per byte moved): far too narrow for a
+// 128-row tcgen05 tile, whose block-diagonal emulation spends 8x the MMA work and was bound by it, but an
+// exact fit for the warp-level m16n8k16 MMA: 16 pixels x (2 taps x 8 input channels) x 8 output channels.
+// The kernel is organised around the memory stream.  Work item = (image, band of R output rows, 64-channel
+// chunk); a producer warp brings the item's input patch ((R + kh - 1) rows x (W + kw - 1) columns x 64
+// channels, zero fill outside the image) into a ring of shared-memory stages with one TMA box (128-byte
+// swizzle).  Compute warp w owns group w of the chunk: its A fragments are ldmatrix loads of [pixel][8
+// channels] rows at the tap's shifted start address (virtual pixels, row pitch W + kw - 1: the outputs of
+// the halo columns are computed and dropped), which the swizzle makes bank-conflict free; its B fragments
+// (the group's 8 x 8 weights per tap) sit in registers for the whole item; results go straight to global
+// memory as bf16 pairs.
+#include "kernels.h"
+#include "mma_sync.cuh"
+#include "sm100_ptx.cuh"
+
+namespace convbn {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int kGMaxStages = 8;
+constexpr int kGMaxKSteps = 5;       // up to 10 taps (3 x 3), two per k-step; the loops over them are unrolled
+constexpr int kGThreads = 288;       // 8 compute warps + the producer warp
+constexpr int kGTiles = 4;           // 16-pixel MMA tiles a warp works on at a time
+
+struct GroupedCtl {
+    uint64_t full[kGMaxStages], empty[kGMaxStages];
+    int abort_flag;
+};
+
+struct GroupedGeom {
+    int n, ho, wo, c, kh, kw, lower_h, lower_w;
+    int R, Wt, rows_in, tiles_h;
+    int stages;
+    uint32_t patch_bytes;      // bytes one TMA box writes
+    uint32_t stage_stride;     // allocation per stage (multiple of 1024, includes the read-ahead tail)
+};
+
+__global__ void __launch_bounds__(kGThreads) grouped8_conv_kernel(const __grid_constant__ CUtensorMap tm_act,
+                                                                 const GroupedGeom g,
+                                                                 const __nv_bfloat16 *__restrict__ w,
+                                                                 const float *__restrict__ bias,
+                                                                 __nv_bfloat16 *__restrict__ out, int *err) {
+    extern __shared__ uint8_t grouped_smem_raw[];
+    uint8_t *ring = (uint8_t *)(((uintptr_t)grouped_smem_raw + 1023) & ~(uintptr_t)1023);
+    GroupedCtl *ctl = (GroupedCtl *)(ring + (size_t)g.stages * g.stage_stride);
+    volatile int *abort_flag = &ctl->abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int taps = g.kh * g.kw, ksteps = (taps + 1) / 2, chunks = g.c / 64;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < g.stages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 8); }
+        ctl->abort_flag = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+    const uint32_t items = (uint32_t)g.n * g.tiles_h * chunks;   // chunk fastest: the chunks of a patch run together
+    if (warp == 8) {
+        if (lane == 0) {
+            prefetch_tensormap(&tm_act);
+            uint32_t s = 0, ph = 0;
+            bool ok = true;
+            for (uint32_t it = blockIdx.x; it < items; it += gridDim.x) {
+                const int cc = (int)(it % (uint32_t)chunks);
+                const uint32_t t1 = it / (uint32_t)chunks;
+                const int h0 = (int)(t1 % (uint32_t)g.tiles_h) * g.R, img = (int)(t1 / (uint32_t)g.tiles_h);
+                if (!mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+                mbar_arrive_expect_tx(&ctl->full[s], g.patch_bytes);
+                tma_load_4d(ring + (size_t)s * g.stage_stride, &tm_act, &ctl->full[s], cc * 64, g.lower_w,
+                            h0 + g.lower_h, img);
+                if (++s == (uint32_t)g.stages) { s = 0; ph ^= 1u; }
+            }
+            if (!ok) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+        }
+        return;
+    }
+    // ---- compute warps: warp = group inside the 64-channel chunk ----
+    const int gr = lane >> 2, t = lane & 3;
+    // ldmatrix.x4: lanes 0-7 address the rows of matrix 0 (pixels 0-7, first tap), 8-15 matrix 1 (pixels
+    // 8-15, first tap), 16-23 matrix 2 (pixels 0-7, second tap), 24-31 matrix 3 (pixels 8-15, second tap)
+    const int lm_pix = (lane & 7) + ((lane >> 3) & 1) * 8, lm_tap = lane >> 4;
+    const int npix = g.R * g.Wt;                               // virtual pixels of a full band
+    uint32_t s = 0, ph = 0;
+    bool ok = true;
+    for (uint32_t it = blockIdx.x; it < items && ok; it += gridDim.x) {
+        const int cc = (int)(it % (uint32_t)chunks);
+        const uint32_t t1 = it / (uint32_t)chunks;
+        const int h0 = (int)(t1 % (uint32_t)g.tiles_h) * g.R, img = (int)(t1 / (uint32_t)g.tiles_h);
+        const int ch0 = cc * 64 + warp * 8;                    // first channel of this warp's group
+        // B fragments: k = 8 (tap in the step) + ci, n = output channel gr; lane holds ci = 2t, 2t + 1
+        uint32_t bf[kGMaxKSteps][2];
+        const __nv_bfloat16 *wrow = w + ((size_t)(ch0 + gr) * taps) * 8 + 2 * t;
+#pragma unroll
+        for (int ks = 0; ks < kGMaxKSteps; ++ks) {
+            bf[ks][0] = 2 * ks < taps ? *reinterpret_cast<const uint32_t *>(wrow + (size_t)(2 * ks) * 8) : 0u;
+            bf[ks][1] = 2 * ks + 1 < taps ? *reinterpret_cast<const uint32_t *>(wrow + (size_t)(2 * ks + 1) * 8) : 0u;
+        }
+        const float b0 = bias ? bias[ch0 + 2 * t] : 0.f, b1 = bias ? bias[ch0 + 2 * t + 1] : 0.f;
+        if (!mbar_wait_bounded(&ctl->full[s], ph, abort_flag)) { ok = false; break; }
+        const uint32_t patch = smem_u32(ring + (size_t)s * g.stage_stride);
+        // four 16-pixel tiles at a time: their MMA chains are independent, so the loads of one overlap
+        // the arithmetic of the others
+        for (int v0 = 0; v0 < npix; v0 += 16 * kGTiles) {
+            float acc[kGTiles][4];
+#pragma unroll
+            for (int u = 0; u < kGTiles; ++u) { acc[u][0] = b0; acc[u][1] = b1; acc[u][2] = b0; acc[u][3] = b1; }
+            int r = 0, q = 0;                                  // tap 2 ks
+#pragma unroll
+            for (int ks = 0; ks < kGMaxKSteps; ++ks) {
+                if (ks >= ksteps) break;                       // the same for every lane
+                int r1 = r, q1 = q + 1;                        // tap 2 ks + 1
+                if (q1 == g.kw) { q1 = 0; ++r1; }
+                const bool second = lm_tap && 2 * ks + 1 < taps;   // an absent second tap re-reads the first (weights 0)
+                const int v = v0 + lm_pix + (second ? r1 * g.Wt + q1 : r * g.Wt + q);
+                // tiles are 16 rows = 2048 bytes apart, which leaves the swizzle term unchanged
+                const uint32_t addr = patch + (uint32_t)v * 128u + (uint32_t)((warp ^ (v & 7)) << 4);
+                uint32_t a[kGTiles][4];
+#pragma unroll
+                for (int u = 0; u < kGTiles; ++u) ldmatrix_x4(a[u][0], a[u][1], a[u][2], a[u][3], addr + (uint32_t)u * 2048u);
+#pragma unroll
+                for (int u = 0; u < kGTiles; ++u) mma_16x8x16_bf16(acc[u], a[u][0], a[u][1], a[u][2], a[u][3], bf[ks][0], bf[ks][1]);
+                r = r1; q = q1 + 1;
+                if (q >= g.kw) { q -= g.kw; ++r; }
+            }
+            // rows gr and gr + 8 of tile u are virtual pixels v0 + 16 u + gr (+ 8): walk them without dividing again
+            int ti = (v0 + gr) / g.Wt, tj = (v0 + gr) - ti * g.Wt;
+#pragma unroll
+            for (int u = 0; u < kGTiles; ++u)
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int h = h0 + ti;
+                    if (ti < g.R && tj < g.wo && h < g.ho) {
+                        const __nv_bfloat162 o2 = __floats2bfloat162_rn(acc[u][2 * half], acc[u][2 * half + 1]);
+                        *reinterpret_cast<__nv_bfloat162 *>(out + ((size_t)((size_t)img * g.ho + h) * g.wo + tj) * g.c + ch0 + 2 * t) = o2;
+                    }
+                    tj += 8;
+                    while (tj >= g.Wt) { tj -= g.Wt; ++ti; }
+                }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ctl->empty[s]);
+        if (++s == (uint32_t)g.stages) { s = 0; ph ^= 1u; }
+    }
+    if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+}
+
+// Backward-data operand: wt[8g + ci][taps - 1 - tap][o] = s[8g + o] w[8g + o][tap][ci]
+__global__ void __launch_bounds__(256) grouped8_flip_weights_kernel(int c, int taps, const __nv_bfloat16 *__restrict__ w,
+                                                                   const float *__restrict__ s_vec,
+                                                                   __nv_bfloat16 *__restrict__ wt) {
+    const int total = c * taps * 8;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+        const int o = i & 7, tap_o = (i >> 3) % taps, row = (i >> 3) / taps;   // row = 8g + ci
+        const int co = (row & ~7) + o, ci = row & 7, tap = taps - 1 - tap_o;
+        wt[i] = __float2bfloat16_rn((s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((size_t)co * taps + tap) * 8 + ci]));
+    }
+}
+
+struct GroupedPlan { bool ok = false; GroupedGeom g; size_t smem = 0; unsigned grid = 0; };
+
+GroupedPlan plan_grouped8(int n, int h_in, int w_in, int c, int ho, int wo, int kh, int kw, int lower_h, int lower_w) {
+    GroupedPlan pl;
+    (void)h_in; (void)w_in;
+    const int wt = wo + kw - 1;
+    if (wt > 256 || kh * kw > 2 * kGMaxKSteps || c % 64) return pl;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) sms = v;
+    }
+    // The compute warps of one block (8, two per scheduler) cannot hide the ldmatrix -> MMA latency on
+    // their own, so the bands are kept small enough for two or three blocks per SM.  Estimated time:
+    // rounds over the resident blocks x input pixels of a band, derated for the SM being shared.
+    double best = -1.0;
+    for (int r = 1; r <= ho && r + kh - 1 <= 256; ++r) {
+        const int rows_in = r + kh - 1;
+        // stage = the box, plus what the last group of tiles reads past it
+        const size_t px = (size_t)((r * wt + 16 * kGTiles - 1) / (16 * kGTiles) * (16 * kGTiles)) + (size_t)(kh - 1) * wt + kw;
+        const size_t need = px > (size_t)rows_in * wt ? px : (size_t)rows_in * wt;
+        const size_t stride = (need * 128 + 1023) / 1024 * 1024;
+        const int tiles_h = (ho + r - 1) / r;
+        const long long items = (long long)n * tiles_h * (c / 64);
+        for (int stages = 2; stages <= 4; ++stages) {
+            const size_t smem = 1024 + (size_t)stages * stride + sizeof(GroupedCtl);
+            if (smem > 220 * 1024) break;
+            int bps = (int)((226 * 1024) / (smem + 1024));
+            if (bps > 3) bps = 3;
+            if (bps < 1) break;
+            const long long slots = (long long)sms * bps;
+            const double share = bps == 1 ? 1.9 : (bps == 2 ? 1.25 : 1.0);     // time per item relative to 3 blocks per SM
+            const double cost = (double)((items + slots - 1) / slots) * bps * (rows_in * (double)wt + 40.0) * share *
+                                (stages == 2 ? 1.1 : 1.0);
+            if (best < 0 || cost < best) {
+                best = cost;
+                pl.ok = true;
+                pl.g.R = r; pl.g.Wt = wt; pl.g.rows_in = rows_in; pl.g.tiles_h = tiles_h; pl.g.stages = stages;
+                pl.g.patch_bytes = (uint32_t)((size_t)rows_in * wt * 128);
+                pl.g.stage_stride = (uint32_t)stride;
+                pl.smem = smem;
+                pl.grid = (unsigned)(items < slots ? items : slots);
+            }
+        }
+    }
+    pl.g.n = n; pl.g.ho = ho; pl.g.wo = wo; pl.g.c = c; pl.g.kh = kh; pl.g.kw = kw;
+    pl.g.lower_h = lower_h; pl.g.lower_w = lower_w;
+    return pl;
+}
+
+}  // namespace
+
+bool grouped8_eligible(const Problem &pb) {
+    static const bool off = getenv("CONVBN_NO_GROUPED_MMA") != nullptr;
+    if (off) return false;
+    return pb.groups > 1 && pb.cg == 8 && pb.cog == 8 && pb.c_in % 64 == 0 && pb.stride_h == 1 && pb.stride_w == 1 &&
+           pb.dil_h == 1 && pb.dil_w == 1 && pb.kh * pb.kw <= 2 * kGMaxKSteps && pb.w_out + pb.kw - 1 <= 256 &&
+           pb.w_in + pb.kw - 1 <= 256 && pb.pad_h <= 128 && pb.pad_w <= 128 && pb.p < (1LL << 30) &&
+           pb.pin < (1LL << 30);
+}
+
+// act: [n][ha][wa][c]; out: [n][ho][wo][c]; w: [c][kh kw][8] (row = output channel of this pass)
+static cudaError_t launch_grouped8(int n, int ha, int wa, int c, int ho, int wo, int kh, int kw, int lower_h,
+                                   int lower_w, const void *act, const void *w, const float *bias, void *out,
+                                   cudaStream_t st) {
+    const GroupedPlan pl = plan_grouped8(n, ha, wa, c, ho, wo, kh, kw, lower_h, lower_w);
+    if (!pl.ok) return cudaErrorInvalidValue;
+    CUtensorMap ta;
+    const unsigned long long dims[4] = {(unsigned long long)c, (unsigned long long)wa, (unsigned long long)ha,
+                                        (unsigned long long)n};
+    const unsigned long long str[4] = {0, (unsigned long long)c * 2, (unsigned long long)wa * c * 2,
+                                       (unsigned long long)ha * wa * c * 2};
+    const unsigned int box[4] = {64, (unsigned)pl.g.Wt, (unsigned)pl.g.rows_in, 1};
+    if (!make_tmap_tiled_bf16(&ta, act, 4, dims, str, box)) return cudaErrorInvalidValue;
+    int *err = nullptr;
+    cudaError_t e = error_word_address(&err);
+    if (e != cudaSuccess) return e;
+    static bool attr = false;
+    if (!attr) {
+        e = cudaFuncSetAttribute(grouped8_conv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        if (e != cudaSuccess) return e;
+        attr = true;
+    }
+    grouped8_conv_kernel<<<pl.grid, kGThreads, pl.smem, st>>>(ta, pl.g, (const __nv_bfloat16 *)w, bias,
+                                                             (__nv_bfloat16 *)out, err);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_grouped8_fwd(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
+                                cudaStream_t st) {
+    return launch_grouped8(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.kh, pb.kw, -pb.pad_h, -pb.pad_w, x, w,
+                           bias, z, st);
+}
+
+cudaError_t launch_grouped8_flip_weights(const Problem &pb, const void *w, const float *s_vec, void *wt,
+                                         cudaStream_t st) {
+    const int total = pb.c_out * pb.kh * pb.kw * 8;
+    grouped8_flip_weights_kernel<<<(total + 255) / 256, 256, 0, st>>>(pb.c_out, pb.kh * pb.kw, (const __nv_bfloat16 *)w,
+                                                                     s_vec, (__nv_bfloat16 *)wt);
+    return cudaGetLastError();
+}
+
+// dX = omega'_rot (*) dZ: the same kernel on the mirrored problem, weights from launch_grouped8_flip_weights
+cudaError_t launch_grouped8_dgrad(const Problem &pb, const void *dz, const void *wt, void *dx, cudaStream_t st) {
+    return launch_grouped8(pb.n, pb.h_out, pb.w_out, pb.c_out, pb.h_in, pb.w_in, pb.kh, pb.kw, pb.pad_h - (pb.kh - 1),
+                           pb.pad_w - (pb.kw - 1), dz, wt, nullptr, dx, st);
+}
+
+}  // namespace convbn

@@ -152,6 +152,13 @@ cudaError_t launch_dw_wgrad(const Problem &pb, const void *dz, const void *x, fl
 // For C_in/G = C_out/G = cg dividing 64 and C a multiple of 64, every 64-channel block is a dense
 // 64 -> 64 convolution whose weight matrix is zero outside the cg x cg diagonal blocks.
 bool grouped_bd_eligible(const Problem &pb);
+// 8 channels per group, unit stride and dilation, at most 10 taps: warp-level MMAs fed by a TMA patch ring
+bool grouped8_eligible(const Problem &pb);
+cudaError_t launch_grouped8_fwd(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
+                                cudaStream_t st);
+cudaError_t launch_grouped8_flip_weights(const Problem &pb, const void *w, const float *s_vec, void *wt,
+                                         cudaStream_t st);
+cudaError_t launch_grouped8_dgrad(const Problem &pb, const void *dz, const void *wt, void *dx, cudaStream_t st);
 // wbd[co][tap][64]: omega (scaled by s_vec[co] if given) placed at its group's columns, zeros elsewhere.
 // transpose_flip = true builds the backward-data operand instead: wbd[ci][taps-1-tap][64 output channels].
 cudaError_t launch_expand_blockdiag(const Problem &pb, const void *w, const float *s_vec, void *wbd,

@@ -5,6 +5,7 @@
 // channels) per filter row r.  A 5-D strided tensor map exposes those overlapping windows to TMA, and
 // the dense tensor-core kernels run with K = kh * 64 (zeros in the unused slots of the weights).
 #include "kernels.h"
+#include "mma_sync.cuh"
 
 namespace convbn {
 
@@ -99,13 +100,6 @@ cudaError_t launch_stem_expand_weights(const Problem &pb, const void *w, const f
 // dZ: lane (g, t) reads 8-channel chunks t and t + 4 of pixels g and g + 8, and k-step k takes word k
 // of each chunk.  The B fragments (the scaled weights, rounded to bf16) are laid out in shared memory
 // in exactly that order, one 32-bit word per lane and fragment register.
-__device__ __forceinline__ void mma_16x8x16_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                                 uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
 // A warp owns 32 consecutive columns of one dZ row at a time (two MMA tiles).  With NU taps in a kernel
 // row of the class, tap u pairs output pixel j with dZ column j + const - u, so instead of loading
 // shifted A fragments per tap the warp keeps one accumulator per tap over the un-shifted columns and

@@ -53,6 +53,9 @@ SMALL = [
     L("b_dw_5x5", 1, 48, 11, 13, 48, 5, 5, pad=2, groups=48),
     # grouped, wide enough for the patch-reuse kernel (block-diagonal mode): two 64-channel blocks
     L("b_grouped_wide", 2, 128, 17, 22, 128, 3, 3, pad=1, groups=16),
+    # 8 channels per group on warp-level MMAs: no padding, a 1x3 kernel (odd tap count), a bias
+    L("b_grouped8_nopad", 1, 64, 12, 19, 64, 3, 3, pad=0, groups=8, bias=True),
+    L("b_grouped8_1x3", 2, 128, 6, 33, 128, 1, 3, pad=1, groups=16),
     L("b_dw_nopad", 3, 32, 13, 37, 32, 3, 3, pad=0, groups=32),
     L("b_dw_wide_c", 1, 256, 9, 21, 256, 3, 3, pad=1, groups=256),
     # narrow-input (stem) path: 4 and 8 input channels, two output-channel chunk groups, stride 1 and 3
@@ -64,7 +67,7 @@ SMALL = [
 EXPECTED_PATH = {   # the specialised kernels must actually be the ones that ran
     "b_1x1_a": ("umma", "umma", "umma"), "b_3x3_a": ("umma-strip", "umma-strip", "umma"),
     "b_3x3_s2": ("umma", "umma-strided", "umma"), "b_dw": ("depthwise", "depthwise", "depthwise"),
-    "b_grouped": ("grouped-umma", "grouped-umma", "grouped-umma"), "b_odd_c": ("direct", "direct", "direct"),
+    "b_grouped": ("grouped-mma", "grouped-mma", "grouped-umma"), "b_odd_c": ("direct", "direct", "direct"),
     "b_strip_wide": ("umma-strip", "umma-strip", "umma"), "b_strip_bn128": ("umma-strip", "umma-strip", "umma"),
     "b_1x1_s2": ("umma", "umma-strided", "umma"), "b_grouped_cg32_s2": ("grouped-umma", "direct", "grouped-umma"),
     "f32_bias": ("direct", "direct", "direct"),
