@@ -99,6 +99,23 @@ __global__ void __launch_bounds__(kGThreads) grouped8_conv_kernel(const __grid_c
             bf[ks][1] = 2 * ks + 1 < taps ? *reinterpret_cast<const uint32_t *>(wrow + (size_t)(2 * ks + 1) * 8) : 0u;
         }
         const float b0 = bias ? bias[ch0 + 2 * t] : 0.f, b1 = bias ? bias[ch0 + 2 * t + 1] : 0.f;
+        // this lane's ldmatrix row of k-step ks, relative to the tile start: its pixel plus the shift of its tap
+        int vrow[kGMaxKSteps];
+        {
+            int r = 0, q = 0;                                  // tap 2 ks
+#pragma unroll
+            for (int ks = 0; ks < kGMaxKSteps; ++ks) {
+                int r1 = r, q1 = q + 1;                        // tap 2 ks + 1
+                if (q1 == g.kw) { q1 = 0; ++r1; }
+                const bool second = lm_tap && 2 * ks + 1 < taps;   // an absent second tap re-reads the first (weights 0)
+                vrow[ks] = lm_pix + (second ? r1 * g.Wt + q1 : r * g.Wt + q);
+                r = r1; q = q1 + 1;
+                if (q >= g.kw) { q -= g.kw; ++r; }
+            }
+        }
+        const int rows_here = min(g.R, g.ho - h0);
+        __nv_bfloat16 *obase = out + ((size_t)((size_t)img * g.ho + h0) * g.wo) * g.c + ch0 + 2 * t;
+        const int wrap_elems = (g.wo - g.Wt) * g.c;            // output offset of (row + 1, column - Wt)
         if (!mbar_wait_bounded(&ctl->full[s], ph, abort_flag)) { ok = false; break; }
         const uint32_t patch = smem_u32(ring + (size_t)s * g.stage_stride);
         // four 16-pixel tiles at a time: their MMA chains are independent, so the loads of one overlap
@@ -107,14 +124,10 @@ __global__ void __launch_bounds__(kGThreads) grouped8_conv_kernel(const __grid_c
             float acc[kGTiles][4];
 #pragma unroll
             for (int u = 0; u < kGTiles; ++u) { acc[u][0] = b0; acc[u][1] = b1; acc[u][2] = b0; acc[u][3] = b1; }
-            int r = 0, q = 0;                                  // tap 2 ks
 #pragma unroll
             for (int ks = 0; ks < kGMaxKSteps; ++ks) {
                 if (ks >= ksteps) break;                       // the same for every lane
-                int r1 = r, q1 = q + 1;                        // tap 2 ks + 1
-                if (q1 == g.kw) { q1 = 0; ++r1; }
-                const bool second = lm_tap && 2 * ks + 1 < taps;   // an absent second tap re-reads the first (weights 0)
-                const int v = v0 + lm_pix + (second ? r1 * g.Wt + q1 : r * g.Wt + q);
+                const int v = v0 + vrow[ks];
                 // tiles are 16 rows = 2048 bytes apart, which leaves the swizzle term unchanged
                 const uint32_t addr = patch + (uint32_t)v * 128u + (uint32_t)((warp ^ (v & 7)) << 4);
                 uint32_t a[kGTiles][4];
@@ -122,22 +135,19 @@ __global__ void __launch_bounds__(kGThreads) grouped8_conv_kernel(const __grid_c
                 for (int u = 0; u < kGTiles; ++u) ldmatrix_x4(a[u][0], a[u][1], a[u][2], a[u][3], addr + (uint32_t)u * 2048u);
 #pragma unroll
                 for (int u = 0; u < kGTiles; ++u) mma_16x8x16_bf16(acc[u], a[u][0], a[u][1], a[u][2], a[u][3], bf[ks][0], bf[ks][1]);
-                r = r1; q = q1 + 1;
-                if (q >= g.kw) { q -= g.kw; ++r; }
             }
-            // rows gr and gr + 8 of tile u are virtual pixels v0 + 16 u + gr (+ 8): walk them without dividing again
+            // rows gr and gr + 8 of tile u are virtual pixels v0 + 16 u + gr (+ 8): walk them, 8 pixels a step
             int ti = (v0 + gr) / g.Wt, tj = (v0 + gr) - ti * g.Wt;
+            ptrdiff_t off = ((ptrdiff_t)ti * g.wo + tj) * g.c;
 #pragma unroll
             for (int u = 0; u < kGTiles; ++u)
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
-                    const int h = h0 + ti;
-                    if (ti < g.R && tj < g.wo && h < g.ho) {
-                        const __nv_bfloat162 o2 = __floats2bfloat162_rn(acc[u][2 * half], acc[u][2 * half + 1]);
-                        *reinterpret_cast<__nv_bfloat162 *>(out + ((size_t)((size_t)img * g.ho + h) * g.wo + tj) * g.c + ch0 + 2 * t) = o2;
-                    }
+                    if (ti < rows_here && tj < g.wo)
+                        *reinterpret_cast<__nv_bfloat162 *>(obase + off) = __floats2bfloat162_rn(acc[u][2 * half], acc[u][2 * half + 1]);
                     tj += 8;
-                    while (tj >= g.Wt) { tj -= g.Wt; ++ti; }
+                    off += 8 * g.c;
+                    if (tj >= g.Wt) { tj -= g.Wt; ++ti; off += wrap_elems; }
                 }
         }
         __syncwarp();
@@ -165,7 +175,7 @@ GroupedPlan plan_grouped8(int n, int h_in, int w_in, int c, int ho, int wo, int 
     GroupedPlan pl;
     (void)h_in; (void)w_in;
     const int wt = wo + kw - 1;
-    if (wt > 256 || kh * kw > 2 * kGMaxKSteps || c % 64) return pl;
+    if (wt > 256 || wt < 8 || kh * kw > 2 * kGMaxKSteps || c % 64) return pl;
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) {
         int v = 0;
