@@ -125,7 +125,7 @@ struct Plan {
     size_t xpk = 0, wst = 0;   // small-C_in layers: packed input [n][hp][wp][8], expanded weights [C_out][kh][64]
     bool stem = false;
     size_t wbd = 0;        // block-diagonal expanded weights [C_out][taps][64], storage dtype
-    bool umma_wgrad = false, dw_wgrad = false, dw_tma_wgrad = false, grouped_wgrad = false;
+    bool umma_wgrad = false, dw_wgrad = false, dw_tma_wgrad = false, grouped_wgrad = false, grouped8_wgrad = false;
     UmmaWgradPlan uw;
 };
 
@@ -158,6 +158,12 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
         pl.uw = umma_wgrad_plan(pb);
         pl.bsplits = pl.uw.splits;
         part_bytes = (size_t)pl.uw.splits * (pb.c_out / 64) * pb.kh * pb.kw * 64 * 64 * sizeof(float);
+        const int slots = grouped8_eligible(pb) ? grouped8_wgrad_slots(pb) : 0;
+        if (slots > 0) {
+            pl.grouped8_wgrad = true;
+            pl.bsplits = slots;
+            part_bytes = (size_t)slots * wrows * sizeof(float);
+        }
     }
     if (pl.stem) {
         pl.umma_wgrad = false;
@@ -488,6 +494,11 @@ int run_param_grads(const convbn_desc *d, const Problem &pb, const Plan &pl, con
         LAUNCH("wgrad_epilogue_stem", launch_wgrad_epilogue_stem(pb, pl.uw, partials, bsum, w, vec3, b, mean, dw, db,
                                                                  dgamma, dbeta, need_bsum, st));
         *which = "umma-stem";
+    } else if (pl.grouped8_wgrad) {
+        LAUNCH("grouped_wgrad", launch_grouped8_wgrad(pb, dz, x, partials, bsum, st));
+        LAUNCH("grouped_wgrad_finish", launch_grouped8_wgrad_finish(pb, partials, bsum, w, vec3, b, mean, dw, db,
+                                                                    dgamma, dbeta, st));
+        *which = "grouped-mma";
     } else if (pl.grouped_wgrad) {
         LAUNCH("grouped_wgrad", launch_umma_wgrad(pb, pl.uw, dz, x, partials, bsum, nullptr, st));
         LAUNCH("wgrad_epilogue_bd", launch_wgrad_epilogue_bd(pb, partials, pl.uw.splits, need_bsum ? bsum : nullptr,

@@ -157,6 +157,185 @@ __global__ void __launch_bounds__(kGThreads) grouped8_conv_kernel(const __grid_c
     if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
 }
 
+// ---- backward weight -----------------------------------------------------------------------------------
+//   domega'[8g + o][tap][ci] = sum_p dZ[p][8g + o] X[p + tap][8g + ci],   sum_p dZ[p][8g + o]      (Sec. 3.2.1)
+// The same patch stream with two boxes per stage: the X patch and the dZ band, the latter on the same
+// virtual-pixel grid (row pitch W + kw - 1, its extra columns lie outside the tensor and arrive as zeros,
+// so the products of the halo positions vanish).  Per group and 16 virtual pixels: K = the pixels,
+// M = (2 taps x 8 input channels), N = 8 output channels; both operands come out of shared memory with
+// transposing ldmatrix loads, and a sixth MMA against a matrix of ones gives sum dZ.  A block keeps one
+// 64-channel chunk for its whole life, so the sums stay in registers across its bands; at the end every
+// warp writes its group's partial block: part[slot][C][taps 8], bsum[slot][C].
+__global__ void __launch_bounds__(kGThreads) grouped8_wgrad_kernel(const __grid_constant__ CUtensorMap tm_x,
+                                                                  const __grid_constant__ CUtensorMap tm_dz,
+                                                                  const GroupedGeom g, uint32_t dz_off, int slots,
+                                                                  float *__restrict__ part, float *__restrict__ bsum,
+                                                                  int *err) {
+    extern __shared__ uint8_t grouped_smem_raw[];
+    uint8_t *ring = (uint8_t *)(((uintptr_t)grouped_smem_raw + 1023) & ~(uintptr_t)1023);
+    GroupedCtl *ctl = (GroupedCtl *)(ring + (size_t)g.stages * g.stage_stride);
+    volatile int *abort_flag = &ctl->abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int taps = g.kh * g.kw, ksteps = (taps + 1) / 2, chunks = g.c / 64;
+    // the regions TMA never writes (read-ahead tails, the gap between the two boxes) are read as operands:
+    // they have to hold zeros, not whatever the last kernel left there
+    for (uint32_t i = threadIdx.x; i < (uint32_t)g.stages * g.stage_stride / 16; i += kGThreads)
+        reinterpret_cast<uint4 *>(ring)[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < g.stages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 8); }
+        ctl->abort_flag = 0;
+        fence_barrier_init();
+    }
+    fence_proxy_async_smem();
+    __syncthreads();
+    const int cc = (int)(blockIdx.x % (uint32_t)chunks), slot = (int)(blockIdx.x / (uint32_t)chunks);
+    const uint32_t items = (uint32_t)g.n * g.tiles_h;          // bands of this chunk
+    const uint32_t x_bytes = g.patch_bytes, dz_bytes = (uint32_t)g.R * g.Wt * 128u;
+    float acc[kGMaxKSteps][4], accs[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int ks = 0; ks < kGMaxKSteps; ++ks) acc[ks][0] = acc[ks][1] = acc[ks][2] = acc[ks][3] = 0.f;
+    if (warp == 8) {
+        if (lane == 0) {
+            prefetch_tensormap(&tm_x);
+            prefetch_tensormap(&tm_dz);
+            uint32_t s = 0, ph = 0;
+            bool ok = true;
+            for (uint32_t it = (uint32_t)slot; it < items; it += (uint32_t)slots) {
+                const int h0 = (int)(it % (uint32_t)g.tiles_h) * g.R, img = (int)(it / (uint32_t)g.tiles_h);
+                if (!mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+                uint8_t *dst = ring + (size_t)s * g.stage_stride;
+                mbar_arrive_expect_tx(&ctl->full[s], x_bytes + dz_bytes);
+                tma_load_4d(dst, &tm_x, &ctl->full[s], cc * 64, g.lower_w, h0 + g.lower_h, img);
+                tma_load_4d(dst + dz_off, &tm_dz, &ctl->full[s], cc * 64, 0, h0, img);
+                if (++s == (uint32_t)g.stages) { s = 0; ph ^= 1u; }
+            }
+            if (!ok) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+        }
+        return;
+    }
+    const int gr = lane >> 2, t = lane & 3;
+    // A: matrix 0 = pixels 0-7 of the first tap, 1 = pixels 0-7 of the second, 2 / 3 = pixels 8-15
+    const int lm_pix = (lane & 7) + (lane >> 4) * 8, lm_tap = (lane >> 3) & 1;
+    int vrow[kGMaxKSteps];
+    {
+        int r = 0, q = 0;
+#pragma unroll
+        for (int ks = 0; ks < kGMaxKSteps; ++ks) {
+            int r1 = r, q1 = q + 1;
+            if (q1 == g.kw) { q1 = 0; ++r1; }
+            const bool second = lm_tap && 2 * ks + 1 < taps;   // an absent second tap re-reads the first (its rows are dropped)
+            vrow[ks] = lm_pix + (second ? r1 * g.Wt + q1 : r * g.Wt + q);
+            r = r1; q = q1 + 1;
+            if (q >= g.kw) { q -= g.kw; ++r; }
+        }
+    }
+    const int npix = g.R * g.Wt;
+    const uint32_t ones = 0x3F803F80u;                         // bf16 1.0 twice
+    uint32_t s = 0, ph = 0;
+    bool ok = true;
+    for (uint32_t it = (uint32_t)slot; it < items && ok; it += (uint32_t)slots) {
+        if (!mbar_wait_bounded(&ctl->full[s], ph, abort_flag)) { ok = false; break; }
+        const uint32_t xpatch = smem_u32(ring + (size_t)s * g.stage_stride), dzpatch = xpatch + dz_off;
+        for (int v0 = 0; v0 < npix; v0 += 16) {
+            uint32_t b0, b1;
+            {
+                const int v = v0 + (lane & 15);
+                ldmatrix_x2_trans(b0, b1, dzpatch + (uint32_t)v * 128u + (uint32_t)((warp ^ (v & 7)) << 4));
+            }
+            mma_16x8x16_bf16(accs, ones, ones, ones, ones, b0, b1);
+#pragma unroll
+            for (int ks = 0; ks < kGMaxKSteps; ++ks) {
+                if (ks >= ksteps) break;
+                const int v = v0 + vrow[ks];
+                uint32_t a0, a1, a2, a3;
+                ldmatrix_x4_trans(a0, a1, a2, a3, xpatch + (uint32_t)v * 128u + (uint32_t)((warp ^ (v & 7)) << 4));
+                mma_16x8x16_bf16(acc[ks], a0, a1, a2, a3, b0, b1);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ctl->empty[s]);
+        if (++s == (uint32_t)g.stages) { s = 0; ph ^= 1u; }
+    }
+    if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+    // accumulator registers: (row gr = input channel of the first tap, columns 2t, 2t + 1 = output channels),
+    // (row gr + 8 = the same input channel of the second tap)
+    const int ch0 = cc * 64 + warp * 8, kdim = taps * 8;
+    float *prow0 = part + ((size_t)slot * g.c + ch0 + 2 * t) * kdim, *prow1 = prow0 + kdim;
+#pragma unroll
+    for (int ks = 0; ks < kGMaxKSteps; ++ks) {
+        if (2 * ks < taps) {
+            prow0[(2 * ks) * 8 + gr] = acc[ks][0];
+            prow1[(2 * ks) * 8 + gr] = acc[ks][1];
+        }
+        if (2 * ks + 1 < taps) {
+            prow0[(2 * ks + 1) * 8 + gr] = acc[ks][2];
+            prow1[(2 * ks + 1) * 8 + gr] = acc[ks][3];
+        }
+    }
+    if (gr == 0) {
+        bsum[(size_t)slot * g.c + ch0 + 2 * t] = accs[0];
+        bsum[(size_t)slot * g.c + ch0 + 2 * t + 1] = accs[1];
+    }
+}
+
+// Adds the block partials and forms the parameter gradients (Table 2, Tune row):
+//   domega = s domega', dbeta = sum dZ, db = s dbeta, dgamma = r (sum_k domega' omega + dbeta (b - mu_hat)).
+// vec3 == NULL: domega = domega', db = sum dZ.  One block per output channel: thread (k, j) adds slots
+// j, j + ng, ... of entry k (a slot's kdim <= 80 entries are contiguous, so the loads coalesce), the ng
+// slot groups are then added in order, and the last group column does the same for sum dZ.
+__global__ void __launch_bounds__(256) grouped8_wgrad_finish_kernel(int c, int kdim, int slots,
+                                                                   const float *__restrict__ part,
+                                                                   const float *__restrict__ bsum,
+                                                                   const __nv_bfloat16 *__restrict__ w,
+                                                                   const float *__restrict__ vec3,
+                                                                   const float *__restrict__ b,
+                                                                   const float *__restrict__ mean,
+                                                                   float *__restrict__ dw, float *__restrict__ db,
+                                                                   float *__restrict__ dgamma,
+                                                                   float *__restrict__ dbeta) {
+    __shared__ float red[256];
+    __shared__ float dots[96];
+    const int co = blockIdx.x;
+    const int ng = 256 / (kdim + 1);                 // slot groups; column kdim of each group sums dZ
+    const int k = threadIdx.x % (kdim + 1), j = threadIdx.x / (kdim + 1);
+    float sum = 0.f;
+    if (j < ng) {
+        if (k < kdim) {
+#pragma unroll 8
+            for (int sl = j; sl < slots; sl += ng) sum += __ldcg(part + ((size_t)sl * c + co) * kdim + k);
+        } else {
+#pragma unroll 8
+            for (int sl = j; sl < slots; sl += ng) sum += __ldcg(bsum + (size_t)sl * c + co);
+        }
+    }
+    red[threadIdx.x] = sum;
+    __syncthreads();
+    const float s = vec3 ? vec3[co] : 1.f;
+    if (threadIdx.x <= kdim) {
+        float tot = 0.f;
+        for (int jj = 0; jj < ng; ++jj) tot += red[jj * (kdim + 1) + threadIdx.x];
+        if (threadIdx.x < kdim) {
+            dw[(size_t)co * kdim + threadIdx.x] = s * tot;
+            dots[threadIdx.x] = vec3 ? tot * __bfloat162float(w[(size_t)co * kdim + threadIdx.x]) : 0.f;
+        } else {
+            dots[kdim] = tot;                        // sum dZ
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float d = 0.f;
+        for (int i = 0; i < kdim; ++i) d += dots[i];
+        const float dsum = dots[kdim];
+        if (vec3) {
+            dbeta[co] = dsum;
+            if (db) db[co] = s * dsum;
+            dgamma[co] = vec3[2 * c + co] * (d + dsum * ((b ? b[co] : 0.f) - mean[co]));
+        } else if (db) {
+            db[co] = dsum;
+        }
+    }
+}
+
 // Backward-data operand: wt[8g + ci][taps - 1 - tap][o] = s[8g + o] w[8g + o][tap][ci]
 __global__ void __launch_bounds__(256) grouped8_flip_weights_kernel(int c, int taps, const __nv_bfloat16 *__restrict__ w,
                                                                    const float *__restrict__ s_vec,
@@ -169,9 +348,10 @@ __global__ void __launch_bounds__(256) grouped8_flip_weights_kernel(int c, int t
     }
 }
 
-struct GroupedPlan { bool ok = false; GroupedGeom g; size_t smem = 0; unsigned grid = 0; };
+struct GroupedPlan { bool ok = false; GroupedGeom g; size_t smem = 0; unsigned grid = 0; uint32_t dz_off = 0; int bps = 1; };
 
-GroupedPlan plan_grouped8(int n, int h_in, int w_in, int c, int ho, int wo, int kh, int kw, int lower_h, int lower_w) {
+GroupedPlan plan_grouped8(int n, int h_in, int w_in, int c, int ho, int wo, int kh, int kw, int lower_h, int lower_w,
+                          bool with_dz = false) {
     GroupedPlan pl;
     (void)h_in; (void)w_in;
     const int wt = wo + kw - 1;
@@ -190,7 +370,9 @@ GroupedPlan plan_grouped8(int n, int h_in, int w_in, int c, int ho, int wo, int 
         // stage = the box, plus what the last group of tiles reads past it
         const size_t px = (size_t)((r * wt + 16 * kGTiles - 1) / (16 * kGTiles) * (16 * kGTiles)) + (size_t)(kh - 1) * wt + kw;
         const size_t need = px > (size_t)rows_in * wt ? px : (size_t)rows_in * wt;
-        const size_t stride = (need * 128 + 1023) / 1024 * 1024;
+        size_t stride = (need * 128 + 1023) / 1024 * 1024;
+        const size_t dz_off = stride;                          // the dZ band sits behind the X patch
+        if (with_dz) stride += ((size_t)((r * wt + 15) / 16 * 16) * 128 + 1023) / 1024 * 1024;
         const int tiles_h = (ho + r - 1) / r;
         const long long items = (long long)n * tiles_h * (c / 64);
         for (int stages = 2; stages <= 4; ++stages) {
@@ -209,6 +391,8 @@ GroupedPlan plan_grouped8(int n, int h_in, int w_in, int c, int ho, int wo, int 
                 pl.g.R = r; pl.g.Wt = wt; pl.g.rows_in = rows_in; pl.g.tiles_h = tiles_h; pl.g.stages = stages;
                 pl.g.patch_bytes = (uint32_t)((size_t)rows_in * wt * 128);
                 pl.g.stage_stride = (uint32_t)stride;
+                pl.dz_off = (uint32_t)dz_off;
+                pl.bps = bps;
                 pl.smem = smem;
                 pl.grid = (unsigned)(items < slots ? items : slots);
             }
@@ -275,6 +459,77 @@ cudaError_t launch_grouped8_flip_weights(const Problem &pb, const void *w, const
 cudaError_t launch_grouped8_dgrad(const Problem &pb, const void *dz, const void *wt, void *dx, cudaStream_t st) {
     return launch_grouped8(pb.n, pb.h_out, pb.w_out, pb.c_out, pb.h_in, pb.w_in, pb.kh, pb.kw, pb.pad_h - (pb.kh - 1),
                            pb.pad_w - (pb.kw - 1), dz, wt, nullptr, dx, st);
+}
+
+// Blocks per 64-channel chunk of the backward-weight kernel = partial rows it writes.
+static GroupedPlan plan_grouped8_wgrad(const Problem &pb, int *slots) {
+    GroupedPlan pl = plan_grouped8(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.kh, pb.kw, -pb.pad_h, -pb.pad_w,
+                                   true);
+    if (!pl.ok) return pl;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) sms = v;
+    }
+    const int chunks = pb.c_in / 64;
+    long long per_chunk = (long long)sms * pl.bps / chunks;
+    const long long bands = (long long)pb.n * pl.g.tiles_h;
+    if (per_chunk > bands) per_chunk = bands;
+    if (per_chunk < 1) per_chunk = 1;
+    *slots = (int)per_chunk;
+    pl.grid = (unsigned)(per_chunk * chunks);
+    return pl;
+}
+
+int grouped8_wgrad_slots(const Problem &pb) {
+    int slots = 0;
+    return plan_grouped8_wgrad(pb, &slots).ok ? slots : 0;
+}
+
+// part: [slots][C][taps 8] floats, bsum: [slots][C] floats (slots = grouped8_wgrad_slots)
+cudaError_t launch_grouped8_wgrad(const Problem &pb, const void *dz, const void *x, float *part, float *bsum,
+                                  cudaStream_t st) {
+    int slots = 0;
+    const GroupedPlan pl = plan_grouped8_wgrad(pb, &slots);
+    if (!pl.ok) return cudaErrorInvalidValue;
+    CUtensorMap tx, tdz;
+    {
+        const unsigned long long dims[4] = {(unsigned long long)pb.c_in, (unsigned long long)pb.w_in,
+                                            (unsigned long long)pb.h_in, (unsigned long long)pb.n};
+        const unsigned long long str[4] = {0, (unsigned long long)pb.c_in * 2, (unsigned long long)pb.w_in * pb.c_in * 2,
+                                           (unsigned long long)pb.h_in * pb.w_in * pb.c_in * 2};
+        const unsigned int box[4] = {64, (unsigned)pl.g.Wt, (unsigned)pl.g.rows_in, 1};
+        if (!make_tmap_tiled_bf16(&tx, x, 4, dims, str, box)) return cudaErrorInvalidValue;
+    }
+    {
+        const unsigned long long dims[4] = {(unsigned long long)pb.c_out, (unsigned long long)pb.w_out,
+                                            (unsigned long long)pb.h_out, (unsigned long long)pb.n};
+        const unsigned long long str[4] = {0, (unsigned long long)pb.c_out * 2, (unsigned long long)pb.w_out * pb.c_out * 2,
+                                           (unsigned long long)pb.h_out * pb.w_out * pb.c_out * 2};
+        const unsigned int box[4] = {64, (unsigned)pl.g.Wt, (unsigned)pl.g.R, 1};
+        if (!make_tmap_tiled_bf16(&tdz, dz, 4, dims, str, box)) return cudaErrorInvalidValue;
+    }
+    int *err = nullptr;
+    cudaError_t e = error_word_address(&err);
+    if (e != cudaSuccess) return e;
+    static bool attr = false;
+    if (!attr) {
+        e = cudaFuncSetAttribute(grouped8_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        if (e != cudaSuccess) return e;
+        attr = true;
+    }
+    grouped8_wgrad_kernel<<<pl.grid, kGThreads, pl.smem, st>>>(tx, tdz, pl.g, pl.dz_off, slots, part, bsum, err);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_grouped8_wgrad_finish(const Problem &pb, const float *part, const float *bsum, const void *w,
+                                         const float *vec3, const float *b, const float *mean, float *dw, float *db,
+                                         float *dgamma, float *dbeta, cudaStream_t st) {
+    const int slots = grouped8_wgrad_slots(pb);
+    if (slots <= 0) return cudaErrorInvalidValue;
+    grouped8_wgrad_finish_kernel<<<pb.c_out, 256, 0, st>>>(pb.c_out, pb.kh * pb.kw * 8, slots, part, bsum,
+                                                         (const __nv_bfloat16 *)w, vec3, b, mean, dw, db, dgamma, dbeta);
+    return cudaGetLastError();
 }
 
 }  // namespace convbn

@@ -159,6 +159,13 @@ cudaError_t launch_grouped8_fwd(const Problem &pb, const void *x, const void *w,
 cudaError_t launch_grouped8_flip_weights(const Problem &pb, const void *w, const float *s_vec, void *wt,
                                          cudaStream_t st);
 cudaError_t launch_grouped8_dgrad(const Problem &pb, const void *dz, const void *wt, void *dx, cudaStream_t st);
+// backward weight: part [slots][C][taps 8] and bsum [slots][C] floats, slots = grouped8_wgrad_slots(pb)
+int grouped8_wgrad_slots(const Problem &pb);
+cudaError_t launch_grouped8_wgrad(const Problem &pb, const void *dz, const void *x, float *part, float *bsum,
+                                  cudaStream_t st);
+cudaError_t launch_grouped8_wgrad_finish(const Problem &pb, const float *part, const float *bsum, const void *w,
+                                         const float *vec3, const float *b, const float *mean, float *dw, float *db,
+                                         float *dgamma, float *dbeta, cudaStream_t st);
 // wbd[co][tap][64]: omega (scaled by s_vec[co] if given) placed at its group's columns, zeros elsewhere.
 // transpose_flip = true builds the backward-data operand instead: wbd[ci][taps-1-tap][64 output channels].
 cudaError_t launch_expand_blockdiag(const Problem &pb, const void *w, const float *s_vec, void *wbd,

