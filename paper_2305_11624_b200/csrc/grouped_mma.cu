@@ -300,13 +300,10 @@ __global__ void __launch_bounds__(256) grouped8_wgrad_finish_kernel(int c, int k
     const int k = threadIdx.x % (kdim + 1), j = threadIdx.x / (kdim + 1);
     float sum = 0.f;
     if (j < ng) {
-        if (k < kdim) {
-#pragma unroll 8
-            for (int sl = j; sl < slots; sl += ng) sum += __ldcg(part + ((size_t)sl * c + co) * kdim + k);
-        } else {
-#pragma unroll 8
-            for (int sl = j; sl < slots; sl += ng) sum += __ldcg(bsum + (size_t)sl * c + co);
-        }
+        if (k < kdim)
+            for (int sl = j; sl < slots; sl += ng) sum += part[((size_t)sl * c + co) * kdim + k];
+        else
+            for (int sl = j; sl < slots; sl += ng) sum += bsum[(size_t)sl * c + co];
     }
     red[threadIdx.x] = sum;
     __syncthreads();
