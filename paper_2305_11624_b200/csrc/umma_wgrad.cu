@@ -397,26 +397,50 @@ __global__ void __launch_bounds__(32 * KR * SL) wgrad_epilogue_fused_kernel(
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    const int lane = tx;
-    for (int co = co0 + (int)(threadIdx.x >> 5); co < co0 + 32; co += KR * SL) {   // a warp per channel
-    float dsum = 0.f, dot = 0.f;
-    for (int sp = lane; sp < bsplits; sp += 32) dsum += __ldcg(bsum + (size_t)sp * c_out + co);
-    if (vec3)
-        for (int t = lane; t < (int)gridDim.y; t += 32) dot += __ldcg(dotpart + (size_t)t * c_out + co);
-    for (int o = 16; o > 0; o >>= 1) {
-        dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
-        dot += __shfl_xor_sync(0xffffffffu, dot, o);
-    }
-    if (lane == 0) {
-        if (!vec3) {
-            if (db) db[co] = dsum;
-        } else {
-            const float s = vec3[co], r = vec3[2 * c_out + co];
-            dbeta[co] = dsum;
-            if (db) db[co] = s * dsum;
-            dgamma[co] = r * (dot + dsum * ((b ? b[co] : 0.f) - mean[co]));
+    // Thread (channel ch, row group grp) adds rows grp, grp + ngrp, ... of the dZ sums and of the dot
+    // partials: a row's 32 channels are one 128-byte read, a thread's (up to eight) rows are requested
+    // together, and the groups are then added in order: one memory round trip instead of one per row.
+    {
+        __shared__ float fin[2][32][33];
+        const int ch = tx, grp = (int)(threadIdx.x >> 5), ngrp = KR * SL;
+        float ds = 0.f, dt = 0.f;
+        for (int base = grp; base < bsplits; base += ngrp * 8) {
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int sp = base + u * ngrp;
+                v[u] = sp < bsplits ? __ldcg(bsum + (size_t)sp * c_out + co0 + ch) : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) ds += v[u];
         }
-    }
+        if (vec3)
+            for (int base = grp; base < (int)gridDim.y; base += ngrp * 8) {
+                float v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int t = base + u * ngrp;
+                    v[u] = t < (int)gridDim.y ? __ldcg(dotpart + (size_t)t * c_out + co0 + ch) : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) dt += v[u];
+            }
+        fin[0][grp][ch] = ds;
+        fin[1][grp][ch] = dt;
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            const int co = co0 + ch;
+            float dsum = 0.f, dot = 0.f;
+            for (int gq = 0; gq < ngrp; ++gq) { dsum += fin[0][gq][ch]; dot += fin[1][gq][ch]; }
+            if (!vec3) {
+                if (db) db[co] = dsum;
+            } else {
+                const float s = vec3[co], r = vec3[2 * c_out + co];
+                dbeta[co] = dsum;
+                if (db) db[co] = s * dsum;
+                dgamma[co] = r * (dot + dsum * ((b ? b[co] : 0.f) - mean[co]));
+            }
+        }
     }
     if (threadIdx.x == 0) counters[blockIdx.x] = 0;   // leave the counter clean for the next call
 }
