@@ -325,13 +325,16 @@ cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
 //     dbeta = sum dZ,  db = s dbeta,  dgamma = r (sum_k domega' omega + dbeta (b - mu_hat))
 //   plain mode (vec3 == NULL): dw = acc, db = sum dZ if requested.
 template <int KR, int SL, int REP>
-__global__ void __launch_bounds__(32 * KR * SL) wgrad_epilogue_fused_kernel(
+__global__ void __launch_bounds__(32 * KR * SL, SL == 16 ? 2 : (KR * SL == 8 ? 4 : 1)) wgrad_epilogue_fused_kernel(
     int c_out, int kdim, const float *__restrict__ part, int splits, const float *__restrict__ bsum, int bsplits,
     const __nv_bfloat16 *__restrict__ w, const float *__restrict__ vec3, const float *__restrict__ b,
     const float *__restrict__ mean, float *__restrict__ dw, float *__restrict__ dotpart,
     unsigned int *__restrict__ counters, float *__restrict__ db, float *__restrict__ dgamma,
     float *__restrict__ dbeta, int need_sums) {
     static_assert(KR * SL <= 32, "at most 32 warps per block");
+    // loads in flight per thread: the (2, 16) shape has the most blocks and is held to 32 registers, so
+    // that two of its 1024-thread blocks share an SM
+    constexpr int NB = SL == 16 ? 4 : 8;
     __shared__ float tile[REP][SL][KR][33];
     __shared__ int is_last;
     pdl_wait();
@@ -349,20 +352,25 @@ __global__ void __launch_bounds__(32 * KR * SL) wgrad_epilogue_fused_kernel(
 #pragma unroll
     for (int rep = 0; rep < REP; ++rep) {
         const int k = k0 + rep * KR + ty;
-        // eight independent sums per thread keep eight loads in flight; they are added in a fixed order
-        float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        // NB independent sums per thread keep NB loads in flight; they are added in a fixed order
+        float a[NB];
+#pragma unroll
+        for (int u = 0; u < NB; ++u) a[u] = 0.f;
         if (k < kdim) {
             const float *src = part + (size_t)k * c_out + co0 + tx;
             int sp = tz;
-            for (; sp + 7 * SL < splits; sp += 8 * SL) {
+            for (; sp + (NB - 1) * SL < splits; sp += NB * SL) {
 #pragma unroll
-                for (int u = 0; u < 8; ++u) a[u] += __ldcg(src + (size_t)(sp + u * SL) * slice);
+                for (int u = 0; u < NB; ++u) a[u] += __ldcg(src + (size_t)(sp + u * SL) * slice);
             }
 #pragma unroll
-            for (int u = 0; u < 8; ++u)
+            for (int u = 0; u < NB; ++u)
                 if (sp + u * SL < splits) a[u] += __ldcg(src + (size_t)(sp + u * SL) * slice);
         }
-        tile[rep][tz][ty][tx] = ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
+        float tot = 0.f;
+#pragma unroll
+        for (int u = 0; u < NB; ++u) tot += a[u];
+        tile[rep][tz][ty][tx] = tot;
     }
     __syncthreads();
     if (threadIdx.x < 32 * KR) {
@@ -398,32 +406,32 @@ __global__ void __launch_bounds__(32 * KR * SL) wgrad_epilogue_fused_kernel(
     if (!is_last) return;
     __threadfence();
     // Thread (channel ch, row group grp) adds rows grp, grp + ngrp, ... of the dZ sums and of the dot
-    // partials: a row's 32 channels are one 128-byte read, a thread's (up to eight) rows are requested
+    // partials: a row's 32 channels are one 128-byte read, a thread's (up to NB) rows are requested
     // together, and the groups are then added in order: one memory round trip instead of one per row.
     {
         __shared__ float fin[2][32][33];
         const int ch = tx, grp = (int)(threadIdx.x >> 5), ngrp = KR * SL;
         float ds = 0.f, dt = 0.f;
-        for (int base = grp; base < bsplits; base += ngrp * 8) {
-            float v[8];
+        for (int base = grp; base < bsplits; base += ngrp * NB) {
+            float v[NB];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int u = 0; u < NB; ++u) {
                 const int sp = base + u * ngrp;
                 v[u] = sp < bsplits ? __ldcg(bsum + (size_t)sp * c_out + co0 + ch) : 0.f;
             }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) ds += v[u];
+            for (int u = 0; u < NB; ++u) ds += v[u];
         }
         if (vec3)
-            for (int base = grp; base < (int)gridDim.y; base += ngrp * 8) {
-                float v[8];
+            for (int base = grp; base < (int)gridDim.y; base += ngrp * NB) {
+                float v[NB];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
+                for (int u = 0; u < NB; ++u) {
                     const int t = base + u * ngrp;
                     v[u] = t < (int)gridDim.y ? __ldcg(dotpart + (size_t)t * c_out + co0 + ch) : 0.f;
                 }
 #pragma unroll
-                for (int u = 0; u < 8; ++u) dt += v[u];
+                for (int u = 0; u < NB; ++u) dt += v[u];
             }
         fin[0][grp][ch] = ds;
         fin[1][grp][ch] = dt;
