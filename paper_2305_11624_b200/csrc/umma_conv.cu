@@ -117,6 +117,8 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
     }
     // Everything above touched only this CTA's own shared / tensor memory.  Global memory (inputs that
     // an earlier kernel may still be writing, outputs it may still be reading) comes after this wait.
+    // the tensor maps are kernel parameters, not data of an earlier kernel: fetch them before the wait
+    if (threadIdx.x == 0) { prefetch_tensormap(&tm_act); prefetch_tensormap(&tm_w); prefetch_tensormap(&tm_out); }
     pdl_wait();
     pdl_launch_dependents();
     if (fold) {
@@ -144,7 +146,6 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
         // ---------------- TMA producer ----------------
         // The whole warp runs the loop; lane 0 arms the barrier and loads the activation tile, lane 1
         // loads the weight tile, so the two copies are issued in parallel.
-        if (lane == 0) { prefetch_tensormap(&tm_act); prefetch_tensormap(&tm_w); }
         uint32_t it = 0;                         // k-blocks issued so far
         int s = 0;                               // ring slot and its phase, advanced incrementally
         uint32_t ph = 0;

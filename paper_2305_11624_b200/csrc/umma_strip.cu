@@ -79,6 +79,8 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
         tmem_alloc(&ctl->tmem_base, g.tmem_cols);
         tmem_relinquish();
     }
+    // the tensor maps are kernel parameters, not data of an earlier kernel: fetch them before the wait
+    if (threadIdx.x == 0) { prefetch_tensormap(&tm_act); prefetch_tensormap(&tm_w); }
     pdl_wait();
     pdl_launch_dependents();
     if (fold) {
@@ -114,7 +116,6 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
     if (warp == 0) {
         // ---------------- patch loader: one TMA copy per (tile, channel chunk) ----------------
         if (elect_one()) {
-            prefetch_tensormap(&tm_act);
             int sb = 0;
             uint32_t ph = 0;
             const uint32_t bytes = (uint32_t)g.rows_in * g.Wt * 128u;
@@ -137,7 +138,6 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
     } else if (warp == 1) {
         // ---------------- weight-tile loader ----------------
         if (elect_one()) {
-            prefetch_tensormap(&tm_w);
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;

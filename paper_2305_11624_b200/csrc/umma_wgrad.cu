@@ -80,6 +80,8 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
         tmem_alloc(&ctl->tmem_base, BN);
         tmem_relinquish();
     }
+    // the tensor maps are kernel parameters, not data of an earlier kernel: fetch them before the wait
+    if (threadIdx.x == 0) { prefetch_tensormap(&tm_x); prefetch_tensormap(&tm_dz); }
     pdl_wait();                 // global memory only after every earlier kernel has finished
     pdl_launch_dependents();
     // counters of the epilogue kernel that runs after this one start from zero
@@ -101,7 +103,6 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
 
     if (warp == 0) {
         // The whole warp runs the loop; lanes 0-1 load the two X slices, lanes 2.. the dZ boxes.
-        if (lane == 0) { prefetch_tensormap(&tm_x); prefetch_tensormap(&tm_dz); }
         const uint32_t tx_bytes = (uint32_t)(a_chunks + b_chunks) * kChunkBytes;
         // this lane's X slice: k = tap * c_in + ci is fixed for the whole CTA
         const int kk = k0 + (lane & 1) * 64;
