@@ -233,7 +233,7 @@ __global__ void __launch_bounds__(288, 2) dw_tma_kernel(const __grid_constant__ 
 // dZ) in registers across all the items of the block.  At the end the thread columns are added in
 // column order through shared memory, and the block writes one partial row: part[block][c][KH KW + 1].
 template <int TW, int KH, int KW>
-__global__ void __launch_bounds__(256, 2) dw_tma_wgrad_kernel(const __grid_constant__ CUtensorMap tx,
+__global__ void __launch_bounds__(288, 2) dw_tma_wgrad_kernel(const __grid_constant__ CUtensorMap tx,
                                                               const __grid_constant__ CUtensorMap tdz, DwTmaGeom g,
                                                               float *__restrict__ part, int *err) {
     constexpr int NX = TW + KW - 1, NACC = KH * KW + 1;
@@ -436,7 +436,7 @@ bool dw_tma_eligible(const Problem &pb) {
 // column and row (X box plus, for the backward-weight kernel, the dZ box).
 static cudaError_t dw_tma_geometry(const Problem &pb, int tw, int kh, int kw, bool with_dz, DwTmaGeom *out,
                                    unsigned *grid) {
-    const int max_consumers = with_dz ? 224 : 256;            // consumer threads; the producer warp comes on top
+    const int max_consumers = with_dz ? 256 : 256;            // consumer threads; the producer warp comes on top
     DwTmaGeom g{};
     g.n = pb.n; g.c = pb.c_in; g.h_in = pb.h_in; g.w_in = pb.w_in; g.h_out = pb.h_out; g.w_out = pb.w_out;
     g.pad_h = pb.pad_h; g.pad_w = pb.pad_w;
