@@ -42,6 +42,12 @@ __device__ __forceinline__ bool try_wait_u32(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// 8-byte global store under a predicate (a predicated instruction: no branch, no reconvergence point)
+__device__ __forceinline__ void stg_u2_if(void *ptr, uint32_t x, uint32_t y, bool on) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.s32 p, %3, 0;\n\t@p st.global.v2.b32 [%0], {%1, %2};\n\t}" ::"l"(ptr), "r"(x),
+                 "r"(y), "r"((int)on)
+                 : "memory");
+}
 // lane 0 of the warp arrives; a predicated instruction, so the warp does not branch
 __device__ __forceinline__ void arrive_lane0(uint32_t bar, int lane) {
     asm volatile(
@@ -210,11 +216,12 @@ __global__ void __launch_bounds__(288, 2) dw_tma_kernel(const __grid_constant__ 
                                                          (r == 0 && q == 0) ? bv[1] : acc[sl][j][1]);
                                 }
                         }
-                        if (k >= KH - 1) {                     // output row k - (KH - 1) is complete
+                        {                                      // output row k - (KH - 1) is complete from k = KH - 1 on
                             const int sl = (ph + 1) % KH;
+                            const bool row_done = k >= KH - 1;
 #pragma unroll
                             for (int j = 0; j < TW; ++j)
-                                if (out_ok[j]) zr[(ptrdiff_t)j * v] = make_uint2(narrow(acc[sl][j][0]), narrow(acc[sl][j][1]));
+                                stg_u2_if(zr + (ptrdiff_t)j * v, narrow(acc[sl][j][0]), narrow(acc[sl][j][1]), row_done && out_ok[j]);
                         }
                         zr += zpitch;
                     }
