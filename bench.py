@@ -301,10 +301,13 @@ def run_ours(args):
     peaks, peak_src = load_peaks()
     tag2layer = {shape_tag(b.spec): b for b in blocks[0]}
     kernels = []
+    phase_ms = {}                                    # (layer tag, phase) -> milliseconds over the eager pass
     for name, (count, total_ms) in prof.items():
-        fam, _, tag = name.partition("@")
+        fam, _, rest = name.partition("@")
+        tag, _, phase = rest.partition("#")
         kernels.append({"kernel": fam, "layer": tag2layer[tag].spec.name if tag in tag2layer else tag,
                         "launches": count, "total_ms": total_ms, "_tag": tag})
+        phase_ms[(tag, phase)] = phase_ms.get((tag, phase), 0.0) + total_ms
     kernels.sort(key=lambda k: -k["total_ms"])
     all_ms = sum(k["total_ms"] for k in kernels) or 1.0
     for k in kernels:
@@ -339,6 +342,22 @@ def run_ours(args):
                              "algorithmic_bytes": by, "algorithmic_flops": fl, "share_of_step": top["share"]})
     for k in kernels:
         k.pop("_tag")
+    # every layer and phase (all kernels of the call, weight re-layouts and epilogues included) against its
+    # own roofline: the larger of FLOPs / tensor peak (dense bf16 only) and algorithmic bytes / copy bandwidth
+    per_layer = []
+    hbm, tc = peaks["hbm_gbs"], peaks["bf16_tflops_sustained"]
+    for (tag, phase), tot in sorted(phase_ms.items()):
+        b = tag2layer.get(tag)
+        kind = {"fwd": "fwd", "bwd_data": "dgrad", "bwd_weight": "wgrad"}.get(phase)
+        if b is None or kind is None:
+            continue
+        us = tot / args.steps * 1e3
+        fl, by = b.flops_per_phase(), kernel_bytes(kind, b.spec, (b.h_out, b.w_out))
+        t_hbm = by / (hbm * 1e9) * 1e6
+        t_tc = fl / (tc * 1e12) * 1e6 if (b.spec.dtype == "bf16" and b.spec.groups == 1) else 0.0
+        per_layer.append({"layer": b.spec.name, "phase": phase, "us": round(us, 2),
+                          "bound": "tensor" if t_tc > t_hbm else "hbm", "roof_us": round(max(t_hbm, t_tc), 2),
+                          "frac": round(max(t_hbm, t_tc) / us, 3) if us > 0 else None})
 
     # ---- Tune against the Eval- and Deploy-mode paths built from the same kernels (the paper's
     # comparison: Table 2, Fig. 3), eager calls, forward + full backward of every layer per step
@@ -406,7 +425,7 @@ def run_ours(args):
                           "note": "same steps as plain library calls with per-kernel CUDA events (source of `kernels` and `roofline`)"},
                 "clocks": sampler.summary(), "e2e": e2e,
                 "gpu_launches": sum(k["launches"] for k in kernels),
-                "roofline": roofline, "cpu_baseline": cpu, "modes": modes, "kernels": kernels[:12],
+                "roofline": roofline, "cpu_baseline": cpu, "modes": modes, "kernels": kernels[:12], "per_layer": per_layer,
                 "activation_bytes": {b.spec.name: {m: b.saved_bytes(m) for m in ("tune", "eval", "deploy")}
                                      for b in blocks[0]}}
         print(json.dumps(line), flush=True)

@@ -213,7 +213,8 @@ int convbn_tune_step_host(const convbn_desc *desc, const void *x, const void *dz
 /* After convbn_profile_begin(), every kernel this library launches (from any thread) is bracketed
  * by a pair of CUDA events on its stream.  convbn_profile_end() stops that, synchronises the
  * device and writes one line per kernel family into `report` (host buffer, NUL-terminated,
- * truncated to report_bytes): "<name> <launches> <total milliseconds>\n".  At most 65536
+ * truncated to report_bytes): "<name> <launches> <total milliseconds>\n", where <name> is
+ * "<kernel family>@<shape key of the layer>#<phase of the call>".  At most 65536
  * launches are recorded between begin and end; later ones run unrecorded. */
 int convbn_profile_begin(void);
 int convbn_profile_end(char *report, size_t report_bytes);

@@ -22,6 +22,7 @@ thread_local const char *t_last_kernel[CONVBN_PHASE_COUNT] = {"none", "none", "n
 // ---- optional per-kernel timing (CUDA events around every launch this library makes) ----------
 struct ProfRec { cudaEvent_t a, b; std::string name; };
 thread_local char t_prof_tag[96] = "";   // shape key of the API call in progress
+thread_local const char *t_prof_phase = "";   // its phase: fwd, bwd_data, bwd_weight (Eval / Deploy: their own names)
 struct Profiler {
     bool on = false;
     std::vector<ProfRec> recs;
@@ -40,7 +41,7 @@ struct ProfScope {
         if (!g_prof.on || g_prof.recs.size() >= kProfCap) return;
         if (cudaEventCreate(&rec.a) != cudaSuccess) return;
         if (cudaEventCreate(&rec.b) != cudaSuccess) { cudaEventDestroy(rec.a); return; }
-        rec.name = std::string(name) + "@" + t_prof_tag;
+        rec.name = std::string(name) + "@" + t_prof_tag + "#" + t_prof_phase;
         cudaEventRecord(rec.a, st);
         live = true;
     }
@@ -450,12 +451,17 @@ int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, cons
         if (pb.stride_h == 1 && pb.stride_w == 1) {
             // dX = omega'_rot (*) dZ is itself a stride-1 depthwise convolution of dZ with the rotated
             // taps and padding (k-1) d - p: run the forward kernel on the mirrored problem.
-            LAUNCH("rescale_weight", launch_rescale_weight(pb, d->dtype, w, scale, w_scratch, st, true));
             Problem mp = pb;
             mp.h_in = pb.h_out; mp.w_in = pb.w_out; mp.h_out = pb.h_in; mp.w_out = pb.w_in;
             mp.pad_h = (pb.kh - 1) * pb.dil_h - pb.pad_h; mp.pad_w = (pb.kw - 1) * pb.dil_w - pb.pad_w;
             mp.p = pb.pin; mp.pin = pb.p;
-            LAUNCH("dw_dgrad", launch_dw_fwd(mp, dz, w_scratch, nullptr, dx, st));
+            if (dw_tma_eligible(mp) && getenv("CONVBN_NO_DW_TMA") == nullptr) {
+                // the streaming kernel scales and reverses the taps itself
+                LAUNCH("dw_dgrad", launch_dw_tma(mp, dz, w, nullptr, dx, st, nullptr, scale, true));
+            } else {
+                LAUNCH("rescale_weight", launch_rescale_weight(pb, d->dtype, w, scale, w_scratch, st, true));
+                LAUNCH("dw_dgrad", launch_dw_fwd(mp, dz, w_scratch, nullptr, dx, st));
+            }
         } else {
             const void *wd = w;
             if (scale) {
@@ -566,6 +572,7 @@ int convbn_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const
                     const float *run_var, void *z, void *saved, void *workspace,
                     size_t workspace_bytes, void *stream) {
     Problem pb;
+    t_prof_phase = "fwd";
     CK(make_problem(desc, &pb));
     CK(check_pair(desc));
     if (!x || !w || !gamma || !beta || !run_mean || !run_var || !z || !saved) return CONVBN_EINVAL;
@@ -600,6 +607,13 @@ int convbn_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const
         }
         return CONVBN_OK;
     }
+    if (dw_path(desc, pb) && dw_tma_eligible(pb) && getenv("CONVBN_NO_DW_TMA") == nullptr) {
+        // depthwise 3x3: the fold is formed inside the streaming kernel from the raw weights
+        const BnFold fold{gamma, beta, run_mean, run_var, b, pb.eps, vec3};
+        LAUNCH("dw_fwd", launch_dw_tma(pb, x, w, nullptr, z, st, &fold));
+        t_last_kernel[CONVBN_PHASE_TUNE_FWD] = "depthwise";
+        return CONVBN_OK;
+    }
     LAUNCH("reparam", launch_reparam(pb, desc->dtype, desc->layout, w, b, gamma, beta, run_mean, run_var, vec3, wf,
                       nullptr, st));
     CK(run_conv_fwd(desc, pb, x, wf, vec3 + pb.c_out, z, pl, workspace, st, &t_last_kernel[CONVBN_PHASE_TUNE_FWD]));
@@ -609,6 +623,7 @@ int convbn_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const
 int convbn_tune_bwd_data(const convbn_desc *desc, const void *dz, const void *w, const void *saved,
                          void *dx, void *workspace, size_t workspace_bytes, void *stream) {
     Problem pb;
+    t_prof_phase = "bwd_data";
     CK(make_problem(desc, &pb));
     CK(check_pair(desc));
     if (!dz || !w || !saved || !dx) return CONVBN_EINVAL;
@@ -628,6 +643,7 @@ int convbn_tune_bwd_weight(const convbn_desc *desc, const void *dz, const void *
                            float *db, float *dgamma, float *dbeta, void *workspace,
                            size_t workspace_bytes, void *stream) {
     Problem pb;
+    t_prof_phase = "bwd_weight";
     CK(make_problem(desc, &pb));
     CK(check_pair(desc));
     if (!dz || !x || !w || !run_mean || !saved || !dw || !dgamma || !dbeta) return CONVBN_EINVAL;
@@ -649,6 +665,7 @@ int convbn_eval_fwd(const convbn_desc *desc, const void *x, const void *w, const
                     const float *run_var, void *z, void *y_saved, void *workspace,
                     size_t workspace_bytes, void *stream) {
     Problem pb;
+    t_prof_phase = "eval_fwd";
     CK(make_problem(desc, &pb));
     CK(check_pair(desc));
     if (!x || !w || !gamma || !beta || !run_mean || !run_var || !z || !y_saved) return CONVBN_EINVAL;
@@ -673,6 +690,7 @@ int convbn_eval_bwd(const convbn_desc *desc, const void *dz, const void *x, cons
                     void *dx, float *dw, float *db, float *dgamma, float *dbeta, void *workspace,
                     size_t workspace_bytes, void *stream) {
     Problem pb;
+    t_prof_phase = "eval_bwd";
     CK(make_problem(desc, &pb));
     CK(check_pair(desc));
     if (!dz || !x || !y_saved || !w || !gamma || !run_mean || !run_var || !dx || !dw || !dgamma || !dbeta)
@@ -701,6 +719,7 @@ int convbn_deploy_prepare(const convbn_desc *desc, const void *w, const float *b
                           const float *beta, const float *run_mean, const float *run_var,
                           void *w_fused, float *b_fused, void *stream) {
     Problem pb;
+    t_prof_phase = "deploy_prepare";
     CK(make_problem(desc, &pb));
     CK(check_pair(desc));
     if (!w || !gamma || !beta || !run_mean || !run_var || !w_fused || !b_fused) return CONVBN_EINVAL;
@@ -717,6 +736,7 @@ int convbn_deploy_fwd(const convbn_desc *desc, const void *x, const void *w_fuse
                       const float *b_fused, void *z, void *workspace, size_t workspace_bytes,
                       void *stream) {
     Problem pb;
+    t_prof_phase = "deploy_fwd";
     CK(make_problem(desc, &pb));
     CK(check_pair(desc));
     if (!x || !w_fused || !b_fused || !z) return CONVBN_EINVAL;
@@ -733,6 +753,7 @@ int convbn_deploy_bwd(const convbn_desc *desc, const void *dz, const void *x, co
                       void *dx, float *dw_fused, float *db_fused, void *workspace,
                       size_t workspace_bytes, void *stream) {
     Problem pb;
+    t_prof_phase = "deploy_bwd";
     CK(make_problem(desc, &pb));
     CK(check_pair(desc));
     if (!dz || !x || !w_fused || !dx || !dw_fused || !db_fused) return CONVBN_EINVAL;
@@ -918,6 +939,7 @@ int convbn_tune_bwd_weight_noalloc(const convbn_desc *desc, const void *dz, cons
                                    const void *saved, float *dw, float *db, float *dgamma,
                                    float *dbeta, void *stream) {
     Problem pb;
+    t_prof_phase = "bwd_weight";
     CK(make_problem(desc, &pb));
     CK(check_pair(desc));
     const size_t need = make_plan(desc, pb, CONVBN_PHASE_TUNE_BWD_WEIGHT).total;

@@ -83,8 +83,9 @@ struct DwTmaGeom {
 template <int TW, int KH, int KW>
 __global__ void __launch_bounds__(288, 2) dw_tma_kernel(const __grid_constant__ CUtensorMap tx, DwTmaGeom g,
                                                         const __nv_bfloat16 *__restrict__ w,
-                                                        const float *__restrict__ bias, uint2 *__restrict__ z,
-                                                        int *err) {
+                                                        const float *__restrict__ bias, const BnFold fold,
+                                                        const float *__restrict__ scale, int reverse_taps,
+                                                        uint2 *__restrict__ z, int *err) {
     constexpr int NX = TW + KW - 1;
     extern __shared__ uint8_t dw_smem_raw[];
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dw_smem_raw) + 127) & ~(uintptr_t)127);
@@ -133,19 +134,35 @@ __global__ void __launch_bounds__(288, 2) dw_tma_kernel(const __grid_constant__ 
     f32x2 wr[KH * KW][2];
     f32x2 bv[2] = {0ull, 0ull};
     if (active) {
+        // Per-channel factor of the taps: the BN fold formed here (forward, Sec. 3.3: s = gamma / sqrt(var +
+        // eps), b' = (b - mu) s + beta; omega stays unrounded), or the saved s (backward data), or 1.
+        float sc[4] = {1.f, 1.f, 1.f, 1.f}, bf[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int c = cv * 4 + e;
+            if (fold.gamma) {
+                const float r = 1.0f / sqrtf(fold.var[c] + fold.eps);
+                sc[e] = fold.gamma[c] * r;
+                bf[e] = ((fold.b ? fold.b[c] : 0.f) - fold.mean[c]) * sc[e] + fold.beta[c];
+                if (blockIdx.x == 0 && tc == 0 && fold.vec3) {
+                    fold.vec3[c] = sc[e]; fold.vec3[g.c + c] = bf[e]; fold.vec3[2 * g.c + c] = r;
+                }
+            } else {
+                if (scale) sc[e] = scale[c];
+                if (bias) bf[e] = bias[c];
+            }
+        }
 #pragma unroll
         for (int tp = 0; tp < KH * KW; ++tp) {
+            const int src = reverse_taps ? KH * KW - 1 - tp : tp;
             float f[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) f[e] = __bfloat162float(w[(size_t)(cv * 4 + e) * (KH * KW) + tp]);
+            for (int e = 0; e < 4; ++e) f[e] = sc[e] * __bfloat162float(w[(size_t)(cv * 4 + e) * (KH * KW) + src]);
             wr[tp][0] = pair(f[0], f[1]);
             wr[tp][1] = pair(f[2], f[3]);
         }
-        if (bias) {
-            const float4 f = *reinterpret_cast<const float4 *>(bias + cv * 4);
-            bv[0] = pair(f.x, f.y);
-            bv[1] = pair(f.z, f.w);
-        }
+        bv[0] = pair(bf[0], bf[1]);
+        bv[1] = pair(bf[2], bf[3]);
     } else {
 #pragma unroll
         for (int tp = 0; tp < KH * KW; ++tp) wr[tp][0] = wr[tp][1] = 0ull;
@@ -496,8 +513,11 @@ static size_t dw_tma_smem(const DwTmaGeom &g) {
     return 128 + ((sizeof(DwTmaCtl) + 127) / 128) * 128 + (size_t)g.stages * g.stage_stride;
 }
 
+// fold != NULL: Tune forward from the raw weights and BN parameters (writes the saved vectors too);
+// scale != NULL: taps multiplied by scale[c]; reverse_taps: taps read in reverse order (the rotated
+// kernel of the backward-data pass on the mirrored problem).
 cudaError_t launch_dw_tma(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
-                          cudaStream_t st) {
+                          cudaStream_t st, const BnFold *fold, const float *scale, bool reverse_taps) {
     constexpr int TW = 2, KH = 3, KW = 3;
     DwTmaGeom g;
     unsigned grid = 0;
@@ -513,8 +533,9 @@ cudaError_t launch_dw_tma(const Problem &pb, const void *x, const void *w, const
         if (e != cudaSuccess) return e;
         attr = true;
     }
+    const BnFold none{nullptr, nullptr, nullptr, nullptr, nullptr, 0.f, nullptr};
     dw_tma_kernel<TW, KH, KW><<<grid, (g.consumer_warps + 1) * 32, dw_tma_smem(g), st>>>(
-        tx, g, (const __nv_bfloat16 *)w, bias, (uint2 *)z, err);
+        tx, g, (const __nv_bfloat16 *)w, bias, fold ? *fold : none, scale, reverse_taps ? 1 : 0, (uint2 *)z, err);
     return cudaGetLastError();
 }
 

@@ -131,7 +131,8 @@ bool dw_eligible(const Problem &pb);
 // 3x3, unit stride and dilation, C <= 256: TMA-fed streaming kernel (forward; backward data with rotated taps)
 bool dw_tma_eligible(const Problem &pb);
 cudaError_t launch_dw_tma(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
-                          cudaStream_t st);
+                          cudaStream_t st, const BnFold *fold = nullptr, const float *scale = nullptr,
+                          bool reverse_taps = false);
 // backward weight on the same stream: block partials [nparts][C][10] (9 taps, then sum dZ), then the finish
 size_t dw_tma_wgrad_partial_bytes(const Problem &pb);
 cudaError_t launch_dw_tma_wgrad(const Problem &pb, const void *dz, const void *x, float *part, int *nparts,
