@@ -229,8 +229,9 @@ int convbn_check(void *stream);
 /* Static, NUL-terminated description of a status code. */
 const char *convbn_status_string(int status);
 
-/* Name of the kernel family the last call of `phase` selected on this thread ("direct",
- * "umma", "depthwise", ...), for logs and tests.  Static string, never NULL. */
+/* Name of the kernel family the last call of `phase` selected on this thread, for logs and tests:
+ * "direct", "umma", "umma-strip", "umma-strided", "umma-stem", "stem-mma", "depthwise",
+ * "grouped-mma", "grouped-umma".  Static string, never NULL. */
 const char *convbn_last_kernel(int phase);
 
 #ifdef __cplusplus

@@ -366,7 +366,7 @@ int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, cons
     UmmaConvShape s;
     if (stem_path(d, pb) && stem_dgrad_eligible(pb)) {
         LAUNCH("stem_dgrad", launch_stem_dgrad(pb, dz, w, scale, dx, st));
-        *which = "stem-simt";
+        *which = "stem-mma";
     } else if (grouped_path(d, pb) && grouped8_eligible(pb)) {
         LAUNCH("grouped_flip", launch_grouped8_flip_weights(pb, w, scale, wbd_scratch, st));
         LAUNCH("grouped_dgrad", launch_grouped8_dgrad(pb, dz, wbd_scratch, dx, st));
