@@ -1,5 +1,5 @@
 // Inline-PTX wrappers for the sm_100a features the tensor-core kernels use: mbarriers with
-// bounded waits, TMA tensor loads (tiled and im2col mode, never multicast), tcgen05 tensor-memory
+// bounded waits, TMA tensor loads (tiled and im2col mode; every CTA loads its own tiles), tcgen05 tensor-memory
 // allocation, MMA issue, commit and accumulator loads, and the shared-memory / instruction
 // descriptor encodings of tcgen05.mma.
 #pragma once
