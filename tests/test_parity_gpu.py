@@ -56,6 +56,9 @@ SMALL = [
     # 8 channels per group on warp-level MMAs: no padding, a 1x3 kernel (odd tap count), a bias
     L("b_grouped8_nopad", 1, 64, 12, 19, 64, 3, 3, pad=0, groups=8, bias=True),
     L("b_grouped8_1x3", 2, 128, 6, 33, 128, 1, 3, pad=1, groups=16),
+    L("b_grouped8_2x2", 1, 64, 11, 14, 64, 2, 2, pad=0, groups=8),
+    # depthwise 3x3 too narrow for the TMA row stream (W_out < 8): the register-streaming kernel
+    L("b_dw_narrow", 2, 32, 9, 6, 32, 3, 3, pad=1, groups=32),
     L("b_dw_nopad", 3, 32, 13, 37, 32, 3, 3, pad=0, groups=32),
     L("b_dw_wide_c", 1, 256, 9, 21, 256, 3, 3, pad=1, groups=256),
     # narrow-input (stem) path: 4 and 8 input channels, two output-channel chunk groups, stride 1 and 3
