@@ -170,32 +170,44 @@ __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_
             for (int tl = 0; tl < 2; ++tl)
 #pragma unroll
                 for (int c = 0; c < 4; ++c) acc[u][tl][c] = 0.f;
+        // this lane's four dZ columns of the window (tile 0 / 1, rows g / g + 8): validity and offset inside
+        // a dZ row are the same for every kernel row, only the row changes
+        bool col_ok[2][2];
+        int col_off[2][2];
+#pragma unroll
+        for (int tl = 0; tl < 2; ++tl)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const int wo = col0 + tl * 16 + g + 8 * hh;
+                col_ok[tl][hh] = wo >= 0 && wo < w_out;
+                col_off[tl][hh] = col_ok[tl][hh] ? wo * v + t : 0;
+            }
+        const uint4 *img_base = dz + (size_t)img * h_out * w_out * v;
+        const int wstep = stride_w * ncb * 256;                // fragment words between two taps of a class
         for (int cb = 0; cb < ncb; ++cb) {
             for (int r = r0; r < kh; r += stride_h) {
                 // h + pad_h - r is a multiple of the stride inside a class, also when negative
                 const int ho = (h + pad_h - r) / stride_h;
                 if (ho < 0 || ho >= h_out) continue;
-                const uint4 *row = dz + ((size_t)(img * h_out + ho) * w_out) * v + cb * 8 + t;
+                const uint4 *row = img_base + (size_t)ho * w_out * v + cb * 8;
                 uint4 alo[2][2], ahi[2][2];                    // columns g / g + 8 of a tile, chunks t / t + 4
+                const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
                 for (int tl = 0; tl < 2; ++tl) {
-                    const int wo = col0 + tl * 16 + g;
-                    const bool lo_ok = wo >= 0 && wo < w_out, hi_ok = wo + 8 >= 0 && wo + 8 < w_out;
-                    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-                    alo[tl][0] = lo_ok ? __ldg(row + (size_t)wo * v) : zero;
-                    alo[tl][1] = lo_ok ? __ldg(row + (size_t)wo * v + 4) : zero;
-                    ahi[tl][0] = hi_ok ? __ldg(row + (size_t)(wo + 8) * v) : zero;
-                    ahi[tl][1] = hi_ok ? __ldg(row + (size_t)(wo + 8) * v + 4) : zero;
+                    alo[tl][0] = col_ok[tl][0] ? __ldg(row + col_off[tl][0]) : zero;
+                    alo[tl][1] = col_ok[tl][0] ? __ldg(row + col_off[tl][0] + 4) : zero;
+                    ahi[tl][0] = col_ok[tl][1] ? __ldg(row + col_off[tl][1]) : zero;
+                    ahi[tl][1] = col_ok[tl][1] ? __ldg(row + col_off[tl][1] + 4) : zero;
                 }
+                const uint32_t *wf = wfrag + ((r * kw + q0) * ncb + cb) * 256 + lane;
 #pragma unroll
                 for (int u = 0; u < NU; ++u) {
                     if (u < nu) {                              // the same for the whole warp
-                        const uint32_t *wf = wfrag + ((size_t)(r * kw + q0 + u * stride_w) * ncb + cb) * 256 + lane;
                         uint32_t bf[4][2];
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
-                            bf[k][0] = wf[k * 64];
-                            bf[k][1] = wf[k * 64 + 32];
+                            bf[k][0] = wf[u * wstep + k * 64];
+                            bf[k][1] = wf[u * wstep + k * 64 + 32];
                         }
 #pragma unroll
                         for (int tl = 0; tl < 2; ++tl) {
