@@ -244,11 +244,21 @@ UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
     const int bn = bd ? 64 : wgrad_bn(pb);
     const long long kd = bd ? (long long)pb.kh * pb.kw * 64 : pb.kdim;
     const long long m_tiles = (kd / 64 + 1 + 1) / 2, n_tiles = (pb.c_out + bn - 1) / bn;   // + the ones slice
-    const long long target = 148;
-    long long splits = (target + m_tiles * n_tiles - 1) / (m_tiles * n_tiles);
+    // Resident CTAs: the 64- and 128-wide tiles run two CTAs per SM (their stage rings are sized for it,
+    // launch_w), which measured 25-40 % faster than one CTA with a deeper ring; 256-wide tiles own an SM.
+    // The slice count minimises  rounds over the resident slots x (pixels per slice + a fixed cost per
+    // CTA, in pixels) + a small cost per slice for the epilogue that adds the slices up; a grid a few
+    // CTAs larger than the slots would otherwise run a second, nearly empty round.
+    const long long slots = 148 * (bn == 256 ? 1 : 2), tiles = m_tiles * n_tiles;
     const long long max_splits = (pb.p + 4 * kWP - 1) / (4 * kWP);     // at least 256 pixels per slice
-    if (splits > max_splits) splits = max_splits;
-    if (splits < 1) splits = 1;
+    long long splits = 1;
+    double best_cost = -1.0;
+    for (long long sp = 1; sp <= max_splits; ++sp) {
+        const long long rounds = (tiles * sp + slots - 1) / slots;
+        const double cost = (double)rounds * ((double)pb.p / (double)sp + 384.0) + 4.0 * (double)sp;
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; splits = sp; }
+        if (tiles * sp > 4 * slots) break;
+    }
     long long per = (pb.p + splits - 1) / splits;
     per = (per + kWP - 1) / kWP * kWP;
     pl.per_split = per;
@@ -266,7 +276,7 @@ static cudaError_t launch_w(const CUtensorMap &tx, const CUtensorMap &tdz, Wgrad
                             const Problem &pb, float *partials, float *bsum, unsigned int *counters, int *err,
                             cudaStream_t st) {
     constexpr size_t stage = 2 * kChunkBytes + (BN / 64) * kChunkBytes;
-    int stages = BN == 256 ? 4 : 4;
+    int stages = BN == 128 ? 3 : 4;                    // 128-wide: 3 x 32 KB, so that two CTAs share an SM
     const long long max_kb = (pl.per_split + kWP - 1) / kWP;
     if (stages > max_kb) stages = (int)max_kb;
     g.stages = stages;
