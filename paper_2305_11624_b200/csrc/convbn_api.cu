@@ -134,7 +134,9 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
     Plan pl;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-    const size_t wbytes = (size_t)pb.c_out * pb.kdim * elem_size(d->dtype);
+    size_t wbytes = (size_t)pb.c_out * pb.kdim * elem_size(d->dtype);
+    // the sub-pixel backward-data path of small-C_in layers keeps its (zero-padded) weight matrix there
+    if (stem_path(d, pb) && subpixel_weight_bytes(pb) > wbytes) wbytes = subpixel_weight_bytes(pb);
     const size_t wrows = (size_t)pb.c_out * pb.kdim;
     pl.splits = direct_wgrad_splits(pb);
     pl.bsplits = channel_sum_splits(pb);
@@ -364,7 +366,13 @@ int run_conv_fwd(const convbn_desc *d, const Problem &pb, const void *x, const v
 int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, const void *w, const float *scale,
                    void *w_scratch, void *wbd_scratch, void *dx, cudaStream_t st, const char **which) {
     UmmaConvShape s;
-    if (stem_path(d, pb) && stem_dgrad_eligible(pb)) {
+    if (stem_path(d, pb) && subpixel_dgrad_shape(pb, &s) && umma_strip_eligible(s)) {
+        // stride 2, C_in <= 4: one stride-1 convolution over dZ whose 16 output columns are the four
+        // parity classes of the input position
+        LAUNCH("subpixel_weights", launch_subpixel_weights(pb, w, scale, w_scratch, st));
+        LAUNCH("stem_dgrad", launch_umma_strip_conv(s, dz, w_scratch, nullptr, dx, st));
+        *which = "umma-subpixel";
+    } else if (stem_path(d, pb) && stem_dgrad_eligible(pb)) {
         LAUNCH("stem_dgrad", launch_stem_dgrad(pb, dz, w, scale, dx, st));
         *which = "stem-mma";
     } else if (grouped_path(d, pb) && grouped8_eligible(pb)) {

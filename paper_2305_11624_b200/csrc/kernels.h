@@ -46,6 +46,11 @@ struct UmmaConvShape {
     // out + n out_sn + i out_sh + j out_sw (elements) instead of densely.
     long long out_sn = 0;
     int out_sh = 0, out_sw = 0;
+    // Sub-pixel output (stride-2 backward data of a layer with at most 4 input channels, strip kernel only,
+    // cn = 16): output "pixel" (n, i, j) holds the 2 x 2 input positions (2 i + a, 2 j + b); GEMM column
+    // 8 a + b sub_cin + ci is written to out[n][2 i + a][2 j + b][ci] of a [n][sub_hin][sub_win][sub_cin]
+    // tensor (positions outside it are dropped).  0: off.
+    int sub_cin = 0, sub_hin = 0, sub_win = 0;
 };
 bool umma_conv_eligible(const UmmaConvShape &s);
 // BatchNorm parameters for in-kernel reparameterisation: the kernel forms s and b' per output channel,
@@ -63,6 +68,16 @@ cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void
 bool umma_strip_eligible(const UmmaConvShape &s);
 cudaError_t launch_umma_strip_conv(const UmmaConvShape &s, const void *act, const void *wmat, const float *bias,
                                    void *out, cudaStream_t st, const BnFold *fold = nullptr);
+// Backward data of a stride-2 layer with C_in <= 4 as ONE stride-1 convolution over dZ (Sec. 3.2.1: the
+// transposed convolution, regrouped by the parity of the input position): the four parity classes of an
+// input position become 4 C_in output columns of a GEMM whose taps are the dZ offsets any class needs;
+// taps a class does not meet have zero weights.  subpixel_dgrad_shape fills the strip-kernel shape and
+// returns false when the layer does not qualify; the weight matrix is [16][taps_h taps_w C_out] bf16,
+// row 8 a + b C_in + ci, entry s[co] w[co][r][q][ci] with r = a + pad_h - 2 d (d = the tap's dZ row offset).
+bool subpixel_dgrad_shape(const Problem &pb, UmmaConvShape *s);
+size_t subpixel_weight_bytes(const Problem &pb);
+cudaError_t launch_subpixel_weights(const Problem &pb, const void *w, const float *s_vec, void *wsub,
+                                    cudaStream_t st);
 // Weight operand of the backward-data GEMM: w_t[ci][taps-1-tap][co] = s[co] w[co][tap][ci]
 // (s_vec == NULL: unscaled).  bf16, groups = 1.
 cudaError_t launch_reparam_dgrad(const Problem &pb, const void *w, const float *s_vec, void *w_t,

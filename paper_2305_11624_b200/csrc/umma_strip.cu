@@ -33,6 +33,7 @@ struct StripGemm {
     int nacc;                         // accumulator sets in tensor memory (1 or 2)
     int blockdiag;                    // grouped conv as block-diagonal 64-channel GEMMs: output block j reads input chunk j
     uint32_t tmem_cols;
+    int sub_cin, sub_hin, sub_win;    // sub-pixel output mode (BN = 16), see UmmaConvShape
     __nv_bfloat16 *out;
     BnFold fold;
 };
@@ -220,6 +221,37 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
                 const bool valid = ti < g.R && tj < g.CW && h < g.ho && wq < g.wo;
                 __nv_bfloat16 *orow = g.out + ((size_t)((size_t)img * g.ho + (valid ? h : 0)) * g.wo + (valid ? wq : 0)) * g.cn + n0;
                 const uint32_t t_row = tmem_base + (a * (uint32_t)g.nmb + (uint32_t)mb) * BN + ((uint32_t)(quarter * 32) << 16);
+                if constexpr (BN == 16) {
+                    // sub-pixel mode: columns 8 a2 + e (e = b cin + ci) go to input row 2 h + a2, elements
+                    // e of the 2 cin consecutive values that start at column 2 wq
+                    uint32_t vv[16];
+                    tmem_ld_32x16(t_row, vv);
+                    tmem_ld_wait();
+                    if (valid) {
+                        const int cin = g.sub_cin;
+                        int lim = (g.sub_win - 2 * wq) * cin;          // elements left in the row
+                        if (lim > 2 * cin) lim = 2 * cin;
+                        const bool pairs = ((g.sub_win * cin) & 1) == 0;   // every row start is 4-byte aligned
+#pragma unroll
+                        for (int a2 = 0; a2 < 2; ++a2) {
+                            const int hh = 2 * h + a2;
+                            if (hh < g.sub_hin) {
+                                __nv_bfloat16 *dst = g.out + (((size_t)img * g.sub_hin + hh) * g.sub_win + (size_t)(2 * wq)) * cin;
+#pragma unroll
+                                for (int e = 0; e < 8; e += 2) {
+                                    const float f0 = __uint_as_float(vv[a2 * 8 + e]), f1 = __uint_as_float(vv[a2 * 8 + e + 1]);
+                                    if (pairs && e + 1 < lim) {
+                                        const __nv_bfloat162 hh2 = __floats2bfloat162_rn(f0, f1);
+                                        *(__nv_bfloat162 *)(dst + e) = hh2;
+                                    } else {
+                                        if (e < lim) dst[e] = __float2bfloat16_rn(f0);
+                                        if (e + 1 < lim) dst[e + 1] = __float2bfloat16_rn(f1);
+                                    }
+                                }
+                            }
+                        }
+                    }
+                } else {
 #pragma unroll 1
                 for (int c0 = 0; c0 < BN; c0 += 32) {
                     uint32_t vv[32];
@@ -253,6 +285,7 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
                         }
                     }
                 }
+                }
             }
             // this warp has read all it needs from the accumulator set
             tc_fence_before_sync();
@@ -284,9 +317,11 @@ StripPlan plan_strip(const UmmaConvShape &s) {
     StripPlan best;
     if (s.stride_h != 1 || s.stride_w != 1 || s.dil_h != 1 || s.dil_w != 1 || s.out_sw) return best;
     if (s.blockdiag && s.ca != s.cn) return best;
-    if (s.taps_h * s.taps_w < 2 || s.ca % 64 || s.cn % 64 || s.cn > 4096 || s.wo < 14 || s.ho < 2) return best;
+    const bool sub = s.sub_cin > 0;
+    if (sub && (s.cn != 16 || s.blockdiag)) return best;
+    if (s.taps_h * s.taps_w < 2 || s.ca % 64 || (!sub && s.cn % 64) || s.cn > 4096 || s.wo < 14 || s.ho < 2) return best;
     if ((long long)s.n * s.ho * s.wo >= (1LL << 30)) return best;
-    const int bn = (s.cn % 128 == 0 && !s.blockdiag) ? 128 : 64;
+    const int bn = sub ? 16 : ((s.cn % 128 == 0 && !s.blockdiag) ? 128 : 64);
     const int nmb_max = 512 / bn / 2;                      // two accumulator sets
     const int tiles_w_min = (s.wo + (256 - s.taps_w + 1) - 1) / (256 - s.taps_w + 1);
     // Among the tilings that keep at least 70 % of the MMA rows useful, take the one with the lowest
@@ -310,7 +345,7 @@ StripPlan plan_strip(const UmmaConvShape &s) {
         const int tiles_h = (s.ho + r - 1) / r;
         const double eff = (double)s.ho * s.wo / ((double)tiles_h * tiles_w * nmb * 128.0);
         if (eff < 0.70) continue;
-        const double mma_clk = (double)nmb * taps * cchunks * 4 * (bn == 64 ? 67.0 : 128.0);
+        const double mma_clk = (double)nmb * taps * cchunks * 4 * (bn == 16 ? 40.0 : (bn == 64 ? 67.0 : 128.0));
         const double fill_clk = ((double)(r + s.taps_h - 1) * wt * 128.0 + (double)taps * bn * 128.0) * cchunks / 32.0;
         const double tile_clk = (mma_clk > fill_clk ? mma_clk : fill_clk) + 1500.0;
         const long long tiles = (long long)s.n * tiles_h * tiles_w * n_tiles;
@@ -388,6 +423,7 @@ cudaError_t launch_umma_strip_conv(const UmmaConvShape &s, const void *act, cons
     g.strip_bytes = pl.strip_bytes;
     g.nacc = 2;
     g.blockdiag = s.blockdiag;
+    g.sub_cin = s.sub_cin; g.sub_hin = s.sub_hin; g.sub_win = s.sub_win;
     int cols = 2 * pl.nmb * pl.bn, p2 = 32;
     while (p2 < cols) p2 <<= 1;
     g.tmem_cols = (uint32_t)p2;
@@ -400,8 +436,77 @@ cudaError_t launch_umma_strip_conv(const UmmaConvShape &s, const void *act, cons
     int *err = nullptr;
     cudaError_t e = error_word_address(&err);
     if (e != cudaSuccess) return e;
+    if (pl.bn == 16) return launch_strip<16>(ta, tw, g, pl.smem, bias, err, st);
     if (pl.bn == 64) return launch_strip<64>(ta, tw, g, pl.smem, bias, err, st);
     return launch_strip<128>(ta, tw, g, pl.smem, bias, err, st);
+}
+
+// ---- stride-2 backward data of a small-C_in layer as a sub-pixel convolution -------------------------
+namespace {
+
+// dZ row offsets d = (a + pad - r) / 2 over both parities a and all taps r with a + pad - r even
+void subpixel_range(int pad, int k, int *dmin, int *dmax) {
+    bool any = false;
+    for (int a = 0; a < 2; ++a)
+        for (int r = 0; r < k; ++r) {
+            const int t = a + pad - r;
+            if (t & 1) continue;
+            const int d = t / 2;                       // t even: exact
+            if (!any || d < *dmin) *dmin = d;
+            if (!any || d > *dmax) *dmax = d;
+            any = true;
+        }
+}
+
+__global__ void subpixel_weights_kernel(const __nv_bfloat16 *__restrict__ w, const float *__restrict__ s_vec,
+                                        __nv_bfloat16 *__restrict__ wsub, int c_out, int cin, int kh, int kw,
+                                        int pad_h, int pad_w, int th, int tw, int dmin_h, int dmin_w) {
+    pdl_wait();
+    pdl_launch_dependents();
+    const int total = 16 * th * tw * c_out;
+    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        const int co = idx % c_out;
+        int t = idx / c_out;
+        const int tq = t % tw; t /= tw;
+        const int tr = t % th;
+        const int row = t / th, a = row >> 3, e = row & 7, b = e / cin, ci = e - b * cin;
+        const int r = a + pad_h - 2 * (dmin_h + tr), q = b + pad_w - 2 * (dmin_w + tq);
+        float v = 0.f;
+        if (b < 2 && r >= 0 && r < kh && q >= 0 && q < kw)
+            v = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[(((size_t)co * kh + r) * kw + q) * cin + ci]);
+        wsub[idx] = __float2bfloat16_rn(v);
+    }
+}
+
+}  // namespace
+
+bool subpixel_dgrad_shape(const Problem &pb, UmmaConvShape *s) {
+    if (pb.groups != 1 || pb.c_in > 4 || pb.stride_h != 2 || pb.stride_w != 2 || pb.dil_h != 1 || pb.dil_w != 1)
+        return false;
+    if (pb.c_out % 64 || pb.c_out > 1024 || pb.kh > 32 || pb.kw > 32 || pb.pin >= (1LL << 30)) return false;
+    int dmin_h = 0, dmax_h = 0, dmin_w = 0, dmax_w = 0;
+    subpixel_range(pb.pad_h, pb.kh, &dmin_h, &dmax_h);
+    subpixel_range(pb.pad_w, pb.kw, &dmin_w, &dmax_w);
+    *s = UmmaConvShape{pb.n, pb.h_out, pb.w_out, pb.c_out, (pb.h_in + 1) / 2, (pb.w_in + 1) / 2, 16,
+                       dmax_h - dmin_h + 1, dmax_w - dmin_w + 1, dmin_h, dmin_w, 1, 1, 1, 1};
+    s->sub_cin = pb.c_in; s->sub_hin = pb.h_in; s->sub_win = pb.w_in;
+    return true;
+}
+
+size_t subpixel_weight_bytes(const Problem &pb) {
+    UmmaConvShape s;
+    if (!subpixel_dgrad_shape(pb, &s)) return 0;
+    return (size_t)16 * s.taps_h * s.taps_w * pb.c_out * sizeof(__nv_bfloat16);
+}
+
+cudaError_t launch_subpixel_weights(const Problem &pb, const void *w, const float *s_vec, void *wsub,
+                                    cudaStream_t st) {
+    UmmaConvShape s;
+    if (!subpixel_dgrad_shape(pb, &s)) return cudaErrorInvalidValue;
+    const int total = 16 * s.taps_h * s.taps_w * pb.c_out;
+    return launch_pdl(subpixel_weights_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st,
+                      (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)wsub, pb.c_out, pb.c_in, pb.kh, pb.kw,
+                      pb.pad_h, pb.pad_w, s.taps_h, s.taps_w, s.lower_h, s.lower_w);
 }
 
 }  // namespace convbn

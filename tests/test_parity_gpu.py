@@ -65,6 +65,12 @@ SMALL = [
     L("b_stem_c4", 1, 4, 19, 23, 128, 5, 5, pad=2),
     L("b_stem_c8_s3", 2, 8, 25, 22, 64, 3, 3, stride=3, pad=1),
     L("b_stem_3x3_s2", 1, 3, 41, 70, 64, 3, 3, stride=2, pad=1),
+    # stride-2 backward data of narrow inputs as a sub-pixel convolution: one input channel with odd sizes
+    # (unpaired stores), four channels with two output-channel chunks, no padding with input rows beyond
+    # twice the output height
+    L("b_sub_c1_odd", 2, 1, 33, 45, 64, 5, 5, stride=2, pad=2),
+    L("b_sub_c4", 1, 4, 40, 64, 128, 7, 7, stride=2, pad=3),
+    L("b_sub_nopad", 1, 3, 38, 52, 64, 4, 4, stride=2, pad=0),
 ]
 
 EXPECTED_PATH = {   # the specialised kernels must actually be the ones that ran
@@ -74,6 +80,8 @@ EXPECTED_PATH = {   # the specialised kernels must actually be the ones that ran
     "b_strip_wide": ("umma-strip", "umma-strip", "umma"), "b_strip_bn128": ("umma-strip", "umma-strip", "umma"),
     "b_1x1_s2": ("umma", "umma-strided", "umma"), "b_grouped_cg32_s2": ("grouped-umma", "direct", "grouped-umma"),
     "f32_bias": ("direct", "direct", "direct"),
+    "b_stem_like": ("umma-stem", "stem-mma", "umma-stem"), "b_sub_c1_odd": ("umma-stem", "umma-subpixel", "umma-stem"),
+    "b_sub_c4": ("umma-stem", "umma-subpixel", "umma-stem"), "b_sub_nopad": ("umma-stem", "umma-subpixel", "umma-stem"),
 }
 
 
