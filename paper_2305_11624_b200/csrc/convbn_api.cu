@@ -136,7 +136,8 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
     size_t wbytes = (size_t)pb.c_out * pb.kdim * elem_size(d->dtype);
     // the sub-pixel backward-data path of small-C_in layers keeps its (zero-padded) weight matrix there
-    if (stem_path(d, pb) && subpixel_weight_bytes(pb) > wbytes) wbytes = subpixel_weight_bytes(pb);
+    if (!force_direct() && d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && subpixel_weight_bytes(pb) > wbytes)
+        wbytes = subpixel_weight_bytes(pb);
     const size_t wrows = (size_t)pb.c_out * pb.kdim;
     pl.splits = direct_wgrad_splits(pb);
     pl.bsplits = channel_sum_splits(pb);
@@ -390,6 +391,12 @@ int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, cons
         else
             LAUNCH("grouped_dgrad", launch_umma_conv(s, dz, wbd_scratch, nullptr, dx, st));
         *which = "grouped-umma";
+    } else if (strided_dgrad_ok(d, pb) && subpixel_wide_shape(pb, &s) && umma_strip_eligible(s)) {
+        // stride 2: the four parity classes of the input position as column blocks of ONE stride-1
+        // convolution over dZ (one launch, the dZ patch staged once, absent taps skipped)
+        LAUNCH("subpixel_weights", launch_subpixel_weights(pb, w, scale, w_scratch, st));
+        LAUNCH("strip_dgrad", launch_umma_strip_conv(s, dz, w_scratch, nullptr, dx, st));
+        *which = "umma-subpixel";
     } else if (strided_dgrad_ok(d, pb)) {
         // Strided backward data, one stride-1 GEMM per residue class (a, b) of the input position:
         // rows h = stride_h i + a only meet taps r with (a + pad_h - r) divisible by stride_h, at output

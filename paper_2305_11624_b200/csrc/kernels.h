@@ -51,6 +51,11 @@ struct UmmaConvShape {
     // 8 a + b sub_cin + ci is written to out[n][2 i + a][2 j + b][ci] of a [n][sub_hin][sub_win][sub_cin]
     // tensor (positions outside it are dropped).  0: off.
     int sub_cin = 0, sub_hin = 0, sub_win = 0;
+    // The same regrouping for wide layers (sub_cin a multiple of 64, cn = 4 sub_cin): GEMM columns
+    // [cls sub_cin, (cls + 1) sub_cin), cls = 2 a + b, are the channels of input position (2 i + a, 2 j + b);
+    // bit t of sub_mask[cls] says that tap t = tr taps_w + tq has weights for that class (other taps are
+    // skipped, not multiplied by zeros).
+    unsigned sub_mask[4] = {0, 0, 0, 0};
 };
 bool umma_conv_eligible(const UmmaConvShape &s);
 // BatchNorm parameters for in-kernel reparameterisation: the kernel forms s and b' per output channel,
@@ -75,6 +80,9 @@ cudaError_t launch_umma_strip_conv(const UmmaConvShape &s, const void *act, cons
 // returns false when the layer does not qualify; the weight matrix is [16][taps_h taps_w C_out] bf16,
 // row 8 a + b C_in + ci, entry s[co] w[co][r][q][ci] with r = a + pad_h - 2 d (d = the tap's dZ row offset).
 bool subpixel_dgrad_shape(const Problem &pb, UmmaConvShape *s);
+// Wide variant (C_in, C_out multiples of 64, stride 2): weight matrix [4 C_in][taps_h taps_w C_out], row
+// (2 a + b) C_in + ci.  Replaces one GEMM launch per parity class by one launch.
+bool subpixel_wide_shape(const Problem &pb, UmmaConvShape *s);
 size_t subpixel_weight_bytes(const Problem &pb);
 cudaError_t launch_subpixel_weights(const Problem &pb, const void *w, const float *s_vec, void *wsub,
                                     cudaStream_t st);

@@ -33,7 +33,9 @@ struct StripGemm {
     int nacc;                         // accumulator sets in tensor memory (1 or 2)
     int blockdiag;                    // grouped conv as block-diagonal 64-channel GEMMs: output block j reads input chunk j
     uint32_t tmem_cols;
-    int sub_cin, sub_hin, sub_win;    // sub-pixel output mode (BN = 16), see UmmaConvShape
+    int sub_cin, sub_hin, sub_win;    // sub-pixel output mode, see UmmaConvShape
+    int sub_wide;                     // 1: wide sub-pixel mode (BN = 64 / 128), n-tile -> parity class
+    uint32_t sub_mask[4];             // taps with weights, per class
     __nv_bfloat16 *out;
     BnFold fold;
 };
@@ -144,8 +146,10 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
             bool ok = true;
             for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
                 const int n0 = (int)(t % n_tiles) * BN;
+                const uint32_t mask = g.sub_wide ? g.sub_mask[n0 / g.sub_cin] : 0xffffffffu;
                 for (int cc = 0; cc < cchunks && ok; ++cc)
                     for (int tap = 0; tap < taps; ++tap) {
+                        if (!((mask >> tap) & 1u)) continue;
                         if (!mbar_wait_bounded(&ctl->b_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
                         mbar_arrive_expect_tx(&ctl->b_full[s], kBBytes);
                         tma_load_2d(bring + (size_t)s * kBBytes, &tm_w, &ctl->b_full[s], tap * w_ca + cc * 64, n0);
@@ -167,12 +171,15 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
                 if (!mbar_wait_bounded(&ctl->tmem_empty[a], (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d0 = tmem_base + a * (uint32_t)(g.nmb * BN);
+                const uint32_t mask = g.sub_wide ? g.sub_mask[(int)(t % n_tiles) * BN / g.sub_cin] : 0xffffffffu;
+                uint32_t started = 0;                   // 0 until the tile's first MMAs have been issued
                 for (int cc = 0; cc < cchunks && ok; ++cc) {
                     if (!mbar_wait_bounded(&ctl->strip_full[sb], sph, abort_flag)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint32_t patch = smem_u32(strips + (size_t)sb * g.strip_bytes);
                     int r = 0, q = 0;
                     for (int tap = 0; tap < taps; ++tap) {
+                        if (!((mask >> tap) & 1u)) { if (++q == g.kw) { q = 0; ++r; } continue; }
                         if (!mbar_wait_bounded(&ctl->b_full[s], bph, abort_flag)) { ok = false; break; }
                         tc_fence_after_sync();
                         const uint32_t b_addr = smem_u32(bring + (size_t)s * kBBytes);
@@ -185,8 +192,9 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
                             for (int mb = 0; mb < g.nmb; ++mb)
                                 umma_bf16_ss(d0 + (uint32_t)(mb * BN),
                                              smem_desc_sw128(patch + (uint32_t)mb * (128u * 128u) + shift + k * 32, 16, 1024),
-                                             bd, idesc, (cc | tap | k) ? 1u : 0u);
+                                             bd, idesc, (started | (uint32_t)k) ? 1u : 0u);
                         }
+                        started = 1;
                         umma_commit(&ctl->b_empty[s]);
                         if (++s == kSBStages) { s = 0; bph ^= 1u; }
                         if (++q == g.kw) { q = 0; ++r; }
@@ -220,6 +228,14 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
                 const int h = h0 + ti, wq = w0 + tj;
                 const bool valid = ti < g.R && tj < g.CW && h < g.ho && wq < g.wo;
                 __nv_bfloat16 *orow = g.out + ((size_t)((size_t)img * g.ho + (valid ? h : 0)) * g.wo + (valid ? wq : 0)) * g.cn + n0;
+                bool store = valid;
+                if (BN != 16 && g.sub_wide) {
+                    // this n-tile holds channels [c_off, c_off + BN) of input position (2 h + a2, 2 wq + b2)
+                    const int cls = n0 / g.sub_cin, c_off = n0 - cls * g.sub_cin;
+                    const int hh = 2 * h + (cls >> 1), ww = 2 * wq + (cls & 1);
+                    store = valid && hh < g.sub_hin && ww < g.sub_win;
+                    orow = g.out + (((size_t)img * g.sub_hin + (store ? hh : 0)) * g.sub_win + (store ? ww : 0)) * g.sub_cin + c_off;
+                }
                 const uint32_t t_row = tmem_base + (a * (uint32_t)g.nmb + (uint32_t)mb) * BN + ((uint32_t)(quarter * 32) << 16);
                 if constexpr (BN == 16) {
                     // sub-pixel mode: columns 8 a2 + e (e = b cin + ci) go to input row 2 h + a2, elements
@@ -257,7 +273,7 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
                     uint32_t vv[32];
                     tmem_ld_32x32(t_row + (uint32_t)c0, vv);
                     tmem_ld_wait();
-                    if (valid) {
+                    if (store) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 8) {
                             float f[8];
@@ -317,11 +333,13 @@ StripPlan plan_strip(const UmmaConvShape &s) {
     StripPlan best;
     if (s.stride_h != 1 || s.stride_w != 1 || s.dil_h != 1 || s.dil_w != 1 || s.out_sw) return best;
     if (s.blockdiag && s.ca != s.cn) return best;
-    const bool sub = s.sub_cin > 0;
-    if (sub && (s.cn != 16 || s.blockdiag)) return best;
+    const bool sub = s.sub_cin > 0 && s.cn == 16, sub_wide = s.sub_cin > 0 && !sub;
+    if (s.sub_cin > 0 && s.blockdiag) return best;
+    if (sub_wide && (s.sub_cin % 64 || s.cn != 4 * s.sub_cin)) return best;
     if (s.taps_h * s.taps_w < 2 || s.ca % 64 || (!sub && s.cn % 64) || s.cn > 4096 || s.wo < 14 || s.ho < 2) return best;
     if ((long long)s.n * s.ho * s.wo >= (1LL << 30)) return best;
-    const int bn = sub ? 16 : ((s.cn % 128 == 0 && !s.blockdiag) ? 128 : 64);
+    // wide sub-pixel mode: an n-tile must not straddle two parity classes
+    const int bn = sub ? 16 : (sub_wide ? (s.sub_cin % 128 == 0 ? 128 : 64) : ((s.cn % 128 == 0 && !s.blockdiag) ? 128 : 64));
     const int nmb_max = 512 / bn / 2;                      // two accumulator sets
     const int tiles_w_min = (s.wo + (256 - s.taps_w + 1) - 1) / (256 - s.taps_w + 1);
     // Among the tilings that keep at least 70 % of the MMA rows useful, take the one with the lowest
@@ -424,6 +442,8 @@ cudaError_t launch_umma_strip_conv(const UmmaConvShape &s, const void *act, cons
     g.nacc = 2;
     g.blockdiag = s.blockdiag;
     g.sub_cin = s.sub_cin; g.sub_hin = s.sub_hin; g.sub_win = s.sub_win;
+    g.sub_wide = (s.sub_cin > 0 && s.cn != 16) ? 1 : 0;
+    for (int c = 0; c < 4; ++c) g.sub_mask[c] = s.sub_mask[c];
     int cols = 2 * pl.nmb * pl.bn, p2 = 32;
     while (p2 < cols) p2 <<= 1;
     g.tmem_cols = (uint32_t)p2;
@@ -480,6 +500,54 @@ __global__ void subpixel_weights_kernel(const __nv_bfloat16 *__restrict__ w, con
 
 }  // namespace
 
+namespace {
+__global__ void subpixel_wide_weights_kernel(const __nv_bfloat16 *__restrict__ w, const float *__restrict__ s_vec,
+                                             __nv_bfloat16 *__restrict__ wsub, int c_out, int cin, int kh, int kw,
+                                             int pad_h, int pad_w, int th, int tw, int dmin_h, int dmin_w) {
+    pdl_wait();
+    pdl_launch_dependents();
+    const long long total = 4LL * cin * th * tw * c_out;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int co = (int)(idx % c_out);
+        long long t = idx / c_out;
+        const int tq = (int)(t % tw); t /= tw;
+        const int tr = (int)(t % th); t /= th;
+        const int ci = (int)(t % cin), cls = (int)(t / cin), a = cls >> 1, b = cls & 1;
+        const int r = a + pad_h - 2 * (dmin_h + tr), q = b + pad_w - 2 * (dmin_w + tq);
+        float v = 0.f;
+        if (r >= 0 && r < kh && q >= 0 && q < kw)
+            v = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[(((size_t)co * kh + r) * kw + q) * cin + ci]);
+        wsub[idx] = __float2bfloat16_rn(v);
+    }
+}
+}  // namespace
+
+bool subpixel_wide_shape(const Problem &pb, UmmaConvShape *s) {
+    if (pb.groups != 1 || pb.stride_h != 2 || pb.stride_w != 2 || pb.dil_h != 1 || pb.dil_w != 1) return false;
+    if (pb.c_in % 64 || pb.c_out % 64 || pb.c_in > 1024 || pb.kh < 2 || pb.kw < 2 || pb.kh > 8 || pb.kw > 8) return false;
+    if (pb.pin >= (1LL << 30) || pb.p >= (1LL << 30)) return false;
+    int dmin_h = 0, dmax_h = 0, dmin_w = 0, dmax_w = 0;
+    subpixel_range(pb.pad_h, pb.kh, &dmin_h, &dmax_h);
+    subpixel_range(pb.pad_w, pb.kw, &dmin_w, &dmax_w);
+    const int th = dmax_h - dmin_h + 1, tw = dmax_w - dmin_w + 1;
+    if (th * tw > 32) return false;
+    *s = UmmaConvShape{pb.n, pb.h_out, pb.w_out, pb.c_out, (pb.h_in + 1) / 2, (pb.w_in + 1) / 2, 4 * pb.c_in,
+                       th, tw, dmin_h, dmin_w, 1, 1, 1, 1};
+    s->sub_cin = pb.c_in; s->sub_hin = pb.h_in; s->sub_win = pb.w_in;
+    for (int cls = 0; cls < 4; ++cls) {
+        unsigned m = 0;
+        for (int tr = 0; tr < th; ++tr)
+            for (int tq = 0; tq < tw; ++tq) {
+                const int r = (cls >> 1) + pb.pad_h - 2 * (dmin_h + tr), q = (cls & 1) + pb.pad_w - 2 * (dmin_w + tq);
+                if (r >= 0 && r < pb.kh && q >= 0 && q < pb.kw) m |= 1u << (tr * tw + tq);
+            }
+        if (!m) return false;                          // a class without taps: its outputs are plain zeros
+        s->sub_mask[cls] = m;
+    }
+    return true;
+}
+
 bool subpixel_dgrad_shape(const Problem &pb, UmmaConvShape *s) {
     if (pb.groups != 1 || pb.c_in > 4 || pb.stride_h != 2 || pb.stride_w != 2 || pb.dil_h != 1 || pb.dil_w != 1)
         return false;
@@ -495,14 +563,22 @@ bool subpixel_dgrad_shape(const Problem &pb, UmmaConvShape *s) {
 
 size_t subpixel_weight_bytes(const Problem &pb) {
     UmmaConvShape s;
-    if (!subpixel_dgrad_shape(pb, &s)) return 0;
-    return (size_t)16 * s.taps_h * s.taps_w * pb.c_out * sizeof(__nv_bfloat16);
+    if (subpixel_dgrad_shape(pb, &s)) return (size_t)16 * s.taps_h * s.taps_w * pb.c_out * sizeof(__nv_bfloat16);
+    if (subpixel_wide_shape(pb, &s)) return (size_t)s.cn * s.taps_h * s.taps_w * pb.c_out * sizeof(__nv_bfloat16);
+    return 0;
 }
 
 cudaError_t launch_subpixel_weights(const Problem &pb, const void *w, const float *s_vec, void *wsub,
                                     cudaStream_t st) {
     UmmaConvShape s;
-    if (!subpixel_dgrad_shape(pb, &s)) return cudaErrorInvalidValue;
+    if (!subpixel_dgrad_shape(pb, &s)) {
+        if (!subpixel_wide_shape(pb, &s)) return cudaErrorInvalidValue;
+        const long long total = (long long)s.cn * s.taps_h * s.taps_w * pb.c_out;
+        const long long blocks = (total + 255) / 256;
+        return launch_pdl(subpixel_wide_weights_kernel, dim3((unsigned)(blocks < 2368 ? blocks : 2368)), dim3(256), 0, st,
+                          (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)wsub, pb.c_out, pb.c_in, pb.kh, pb.kw,
+                          pb.pad_h, pb.pad_w, s.taps_h, s.taps_w, s.lower_h, s.lower_w);
+    }
     const int total = 16 * s.taps_h * s.taps_w * pb.c_out;
     return launch_pdl(subpixel_weights_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st,
                       (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)wsub, pb.c_out, pb.c_in, pb.kh, pb.kw,

@@ -71,6 +71,10 @@ SMALL = [
     L("b_sub_c1_odd", 2, 1, 33, 45, 64, 5, 5, stride=2, pad=2),
     L("b_sub_c4", 1, 4, 40, 64, 128, 7, 7, stride=2, pad=3),
     L("b_sub_nopad", 1, 3, 38, 52, 64, 4, 4, stride=2, pad=0),
+    # the same regrouping for wide stride-2 layers: 128-column tiles; 64-column tiles with three
+    # output-channel chunks, a 5x5 kernel and odd sizes
+    L("b_sub_wide", 1, 128, 40, 58, 128, 3, 3, stride=2, pad=1),
+    L("b_sub_wide_5x5", 1, 64, 37, 61, 192, 5, 5, stride=2, pad=2),
 ]
 
 EXPECTED_PATH = {   # the specialised kernels must actually be the ones that ran
@@ -81,6 +85,7 @@ EXPECTED_PATH = {   # the specialised kernels must actually be the ones that ran
     "b_1x1_s2": ("umma", "umma-strided", "umma"), "b_grouped_cg32_s2": ("grouped-umma", "direct", "grouped-umma"),
     "f32_bias": ("direct", "direct", "direct"),
     "b_stem_like": ("umma-stem", "stem-mma", "umma-stem"), "b_sub_c1_odd": ("umma-stem", "umma-subpixel", "umma-stem"),
+    "b_sub_wide": ("umma", "umma-subpixel", "umma"), "b_sub_wide_5x5": ("umma", "umma-subpixel", "umma"),
     "b_sub_c4": ("umma-stem", "umma-subpixel", "umma-stem"), "b_sub_nopad": ("umma-stem", "umma-subpixel", "umma-stem"),
 }
 
