@@ -64,11 +64,12 @@ def kernel_bytes(kind, spec, out_hw):
 
 # DRAM bytes (read + write) per launch from the ncu capture summarised in
 # profiles/config1_gemm_kernels_ncu_full.md; None for kernels changed or not captured since.
-NCU_TRAFFIC = {("umma_fwd", "c1a"): 51.71e6, ("umma_dgrad", "c1a"): 13.80e6,
-               ("strip_fwd", "c1b"): 12.96e6, ("strip_dgrad", "c1b"): 12.96e6,
-               ("umma_fwd", "c1c"): 13.86e6, ("umma_dgrad", "c1c"): 51.94e6, ("umma_wgrad", "c1c"): 66.19e6,
+NCU_TRAFFIC = {("umma_fwd", "c1a"): 51.71e6, ("umma_dgrad", "c1a"): 13.80e6, ("umma_wgrad", "c1a"): 65.09e6,
+               ("strip_fwd", "c1b"): 12.96e6, ("strip_dgrad", "c1b"): 12.96e6, ("umma_wgrad", "c1b"): 25.71e6,
+               ("umma_fwd", "c1c"): 13.86e6, ("umma_dgrad", "c1c"): 51.94e6, ("umma_wgrad", "c1c"): 65.54e6,
                ("dw_fwd", "c4a"): 262.4e6, ("dw_dgrad", "c4a"): 261.0e6, ("dw_wgrad", "c4a"): 312.3e6,
-               ("grouped_dgrad", "c4b"): 29.1e6, ("grouped_wgrad", "c4b"): 51.8e6}
+               ("grouped_dgrad", "c4b"): 29.1e6, ("grouped_wgrad", "c4b"): 51.8e6,
+               ("stem_dgrad", "c2s"): 109.5e6}
 
 KIND_OF = {"strip_fwd": "fwd", "strip_dgrad": "dgrad", "direct_fwd": "fwd", "direct_dgrad": "dgrad", "direct_wgrad": "wgrad",
            "umma_fwd": "fwd", "umma_dgrad": "dgrad", "umma_wgrad": "wgrad",
