@@ -173,7 +173,7 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
         pl.umma_wgrad = false;
         pl.uw = stem_wgrad_plan(pb);
         pl.bsplits = pl.uw.splits;
-        part_bytes = (size_t)pl.uw.splits * pb.kh * 64 * pb.c_out * sizeof(float);
+        part_bytes = (size_t)pl.uw.splits * stem_krows(pb) * 64 * pb.c_out * sizeof(float);
     }
     if (pl.umma_wgrad) {
         pl.uw = umma_wgrad_plan(pb);

@@ -127,9 +127,13 @@ cudaError_t launch_wgrad_epilogue_fused(const Problem &pb, const UmmaWgradPlan &
 
 // ---- first-layer convolutions with C_in <= 8 (see stem_kernels.cu) -------------------------------
 bool stem_eligible(const Problem &pb);
-void stem_geometry(const Problem &pb, int *hp, int *wp);     // extent of the packed, zero-bordered input
-size_t stem_packed_bytes(const Problem &pb);                 // [n][hp][wp][8] bf16
-size_t stem_weight_bytes(const Problem &pb);                 // [C_out][kh][64] bf16
+void stem_geometry(const Problem &pb, int *hp, int *wp);     // extent of the packed, zero-bordered input (packed pixels)
+bool stem_s2d(const Problem &pb);                            // stride 2, C_in <= 4: 2 x 2 pixel blocks per packed pixel
+int stem_krows(const Problem &pb);                           // 64-wide K rows per output pixel: kh, or ceil(kh / 2)
+// byte strides of the 5-D window view {64, w_out, h_out, krows, n} of the packed input
+void stem_window_strides(const Problem &pb, unsigned long long str[5]);
+size_t stem_packed_bytes(const Problem &pb);                 // [n][hp][wp][8] bf16, or [n][hp][wp][2][2][4]
+size_t stem_weight_bytes(const Problem &pb);                 // [C_out][krows][64] bf16
 cudaError_t launch_stem_pack(const Problem &pb, const void *x, void *x_packed, cudaStream_t st);
 cudaError_t launch_stem_expand_weights(const Problem &pb, const void *w, const float *s_vec, void *wst,
                                        cudaStream_t st);
@@ -137,7 +141,7 @@ cudaError_t launch_stem_expand_weights(const Problem &pb, const void *w, const f
 bool stem_dgrad_eligible(const Problem &pb);
 cudaError_t launch_stem_dgrad(const Problem &pb, const void *dz, const void *w, const float *s_vec, void *dx,
                               cudaStream_t st);
-// Weight gradient of a stem layer on the packed input: partials [splits][kh * 64][C_out] (padded k rows),
+// Weight gradient of a stem layer on the packed input: partials [splits][krows * 64][C_out] (padded k rows),
 // bsum [splits][C_out]; the epilogue gathers the real kh x kw x C_in entries.
 UmmaWgradPlan stem_wgrad_plan(const Problem &pb);
 cudaError_t launch_stem_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const void *dz, const void *x_packed,

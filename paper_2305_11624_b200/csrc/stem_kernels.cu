@@ -4,6 +4,7 @@
 // pixels a filter row touches are 128 contiguous bytes: one K row of 64 "channels" (8 pixels x 8
 // channels) per filter row r.  A 5-D strided tensor map exposes those overlapping windows to TMA, and
 // the dense tensor-core kernels run with K = kh * 64 (zeros in the unused slots of the weights).
+// Stride-2 layers with at most 4 channels use a denser space-to-depth packing (see stem_s2d below).
 #include "kernels.h"
 #include "mma_sync.cuh"
 
@@ -15,7 +16,23 @@ bool stem_eligible(const Problem &pb) {
            pb.p < (1LL << 30) && pb.pin < (1LL << 30);
 }
 
+// Stride-2 layers with C_in <= 4 are packed "space to depth" instead: a packed pixel holds the 2 x 2 block
+// of padded input pixels (2 I + a, 2 J + b) as [a][b][4 channels] = 16 values (32 bytes).  Tap (r, q) of
+// output (ho, wo) is then element (r & 1, q & 1) of packed pixel (ho + r / 2, wo + q / 2), and the four
+// packed pixels wo .. wo + 3 of packed row ho + tr are 128 contiguous bytes: one K row of 64 per PAIR of
+// filter rows, K = ceil(kh / 2) * 64 instead of kh * 64 (7 x 7: 256 instead of 448, 57 % of it real taps).
+bool stem_s2d(const Problem &pb) { return pb.stride_h == 2 && pb.stride_w == 2 && pb.c_in <= 4; }
+
+int stem_krows(const Problem &pb) { return stem_s2d(pb) ? (pb.kh + 1) / 2 : pb.kh; }
+
 void stem_geometry(const Problem &pb, int *hp, int *wp) {
+    if (stem_s2d(pb)) {
+        const int need_h = (pb.h_out - 1) + stem_krows(pb), need_w = (pb.w_out - 1) + 4;
+        const int have_h = (pb.h_in + 2 * pb.pad_h + 1) / 2, have_w = (pb.w_in + 2 * pb.pad_w + 1) / 2;
+        *hp = need_h > have_h ? need_h : have_h;
+        *wp = need_w > have_w ? need_w : have_w;
+        return;
+    }
     const int need_h = (pb.h_out - 1) * pb.stride_h + pb.kh, need_w = (pb.w_out - 1) * pb.stride_w + 8;
     const int have_h = pb.h_in + 2 * pb.pad_h, have_w = pb.w_in + 2 * pb.pad_w;
     *hp = need_h > have_h ? need_h : have_h;
@@ -25,10 +42,53 @@ void stem_geometry(const Problem &pb, int *hp, int *wp) {
 size_t stem_packed_bytes(const Problem &pb) {
     int hp, wp;
     stem_geometry(pb, &hp, &wp);
-    return (size_t)pb.n * hp * wp * 16;
+    return (size_t)pb.n * hp * wp * (stem_s2d(pb) ? 32 : 16);
 }
 
-size_t stem_weight_bytes(const Problem &pb) { return (size_t)pb.c_out * pb.kh * 64 * 2; }
+void stem_window_strides(const Problem &pb, unsigned long long str[5]) {
+    int hp, wp;
+    stem_geometry(pb, &hp, &wp);
+    if (stem_s2d(pb)) {      // one packed pixel per output column, one packed row per output row and per K row
+        str[0] = 0; str[1] = 32; str[2] = (unsigned long long)wp * 32; str[3] = (unsigned long long)wp * 32;
+        str[4] = (unsigned long long)hp * wp * 32;
+    } else {
+        str[0] = 0; str[1] = (unsigned long long)pb.stride_w * 16; str[2] = (unsigned long long)pb.stride_h * wp * 16;
+        str[3] = (unsigned long long)wp * 16; str[4] = (unsigned long long)hp * wp * 16;
+    }
+}
+
+size_t stem_weight_bytes(const Problem &pb) { return (size_t)pb.c_out * stem_krows(pb) * 64 * 2; }
+
+// xp[n][hp][wp][a][b][4] = x[n][2 I + a - pad_h][2 J + b - pad_w][c] inside the image, 0 elsewhere
+__global__ void __launch_bounds__(256) stem_pack_s2d_kernel(int n, int h_in, int w_in, int c_in, int pad_h, int pad_w,
+                                                            int hp, int wp, const __nv_bfloat16 *__restrict__ x,
+                                                            uint4 *__restrict__ xp) {
+    const long long total = (long long)n * hp * wp * 2;          // one thread per (packed pixel, a)
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        const int a = (int)(i & 1);
+        const long long pix = i >> 1;
+        const int wq = (int)(pix % wp);
+        const long long t = pix / wp;
+        const int hq = (int)(t % hp), img = (int)(t / hp);
+        const int h = 2 * hq + a - pad_h;
+        unsigned short v[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        if (h >= 0 && h < h_in) {
+#pragma unroll
+            for (int b = 0; b < 2; ++b) {
+                const int w = 2 * wq + b - pad_w;
+                if (w >= 0 && w < w_in) {
+                    const unsigned short *src = (const unsigned short *)x + (((long long)img * h_in + h) * w_in + w) * c_in;
+                    for (int c = 0; c < c_in; ++c) v[b * 4 + c] = src[c];
+                }
+            }
+        }
+        uint4 q;
+        q.x = v[0] | ((uint32_t)v[1] << 16); q.y = v[2] | ((uint32_t)v[3] << 16);
+        q.z = v[4] | ((uint32_t)v[5] << 16); q.w = v[6] | ((uint32_t)v[7] << 16);
+        xp[i] = q;
+    }
+}
 
 // xp[n][hp][wp][8] = x[n][h - pad_h][w - pad_w][c] inside the image, 0 in the border and for c >= C_in
 __global__ void __launch_bounds__(256) stem_pack_kernel(int n, int h_in, int w_in, int c_in, int pad_h, int pad_w,
@@ -56,25 +116,32 @@ __global__ void __launch_bounds__(256) stem_pack_kernel(int n, int h_in, int w_i
 cudaError_t launch_stem_pack(const Problem &pb, const void *x, void *xp, cudaStream_t st) {
     int hp, wp;
     stem_geometry(pb, &hp, &wp);
-    const long long total = (long long)pb.n * hp * wp;
+    const long long total = (long long)pb.n * hp * wp * (stem_s2d(pb) ? 2 : 1);
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
+    if (stem_s2d(pb)) {
+        stem_pack_s2d_kernel<<<(int)blocks, 256, 0, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.pad_h, pb.pad_w, hp, wp,
+                                                          (const __nv_bfloat16 *)x, (uint4 *)xp);
+        return cudaGetLastError();
+    }
     stem_pack_kernel<<<(int)blocks, 256, 0, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.pad_h, pb.pad_w, hp, wp,
                                                   (const __nv_bfloat16 *)x, (uint4 *)xp);
     return cudaGetLastError();
 }
 
-// wst[co][r][q * 8 + c] = scale[co] * w[co][r][q][c]  (q < kw, c < C_in), zero elsewhere
-__global__ void __launch_bounds__(256) stem_expand_weights_kernel(int c_out, int kh, int kw, int c_in,
-                                                                  const __nv_bfloat16 *__restrict__ w,
+// wst[co][r][q * 8 + c] = scale[co] * w[co][r][q][c]  (q < kw, c < C_in), zero elsewhere; space-to-depth
+// packing (s2d): wst[co][tr][tq * 16 + a * 8 + b * 4 + c] with r = 2 tr + a, q = 2 tq + b
+__global__ void __launch_bounds__(256) stem_expand_weights_kernel(int c_out, int kh, int kw, int c_in, int krows,
+                                                                  int s2d, const __nv_bfloat16 *__restrict__ w,
                                                                   const float *__restrict__ s_vec,
                                                                   __nv_bfloat16 *__restrict__ wst) {
-    const int total = c_out * kh * 64;
+    const int total = c_out * krows * 64;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
-        const int j = i & 63, r = (i >> 6) % kh, co = (i >> 6) / kh;
-        const int q = j >> 3, c = j & 7;
+        const int j = i & 63, kr = (i >> 6) % krows, co = (i >> 6) / krows;
+        const int r = s2d ? 2 * kr + ((j >> 3) & 1) : kr;
+        const int q = s2d ? 2 * (j >> 4) + ((j >> 2) & 1) : j >> 3, c = s2d ? (j & 3) : (j & 7);
         float v = 0.f;
-        if (q < kw && c < c_in)
+        if (r < kh && q < kw && c < c_in)
             v = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[(((long long)co * kh + r) * kw + q) * c_in + c]);
         wst[i] = __float2bfloat16_rn(v);
     }
@@ -82,9 +149,9 @@ __global__ void __launch_bounds__(256) stem_expand_weights_kernel(int c_out, int
 
 cudaError_t launch_stem_expand_weights(const Problem &pb, const void *w, const float *s_vec, void *wst,
                                        cudaStream_t st) {
-    const int total = pb.c_out * pb.kh * 64;
-    stem_expand_weights_kernel<<<(total + 255) / 256, 256, 0, st>>>(pb.c_out, pb.kh, pb.kw, pb.c_in,
-                                                                    (const __nv_bfloat16 *)w, s_vec,
+    const int total = pb.c_out * stem_krows(pb) * 64;
+    stem_expand_weights_kernel<<<(total + 255) / 256, 256, 0, st>>>(pb.c_out, pb.kh, pb.kw, pb.c_in, stem_krows(pb),
+                                                                    stem_s2d(pb) ? 1 : 0, (const __nv_bfloat16 *)w, s_vec,
                                                                     (__nv_bfloat16 *)wst);
     return cudaGetLastError();
 }

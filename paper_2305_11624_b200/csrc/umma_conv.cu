@@ -546,13 +546,12 @@ cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void
 }
 
 // Forward pass of a small-C_in layer on the packed input (see stem_kernels.cu): tiles of 8 x 16 output
-// pixels, K = kh rows of 64, weights resident.
+// pixels, K = stem_krows rows of 64, weights resident.
 cudaError_t launch_stem_fwd(const Problem &pb, const void *x_packed, const void *wst, const float *bias, void *out,
                             cudaStream_t st, const BnFold *fold) {
-    int hp, wp;
-    stem_geometry(pb, &hp, &wp);
+    const int krows = stem_krows(pb);
     ConvGemm g;
-    g.ho = pb.h_out; g.wo = pb.w_out; g.cn = pb.c_out; g.ca = 64; g.taps_h = pb.kh; g.taps_w = 1;
+    g.ho = pb.h_out; g.wo = pb.w_out; g.cn = pb.c_out; g.ca = 64; g.taps_h = krows; g.taps_w = 1;
     g.lower_h = g.lower_w = 0; g.stride_h = g.stride_w = g.dil_h = g.dil_w = 1;
     g.stem = 1; g.stem_tw = 16; g.stem_th = 8;
     g.stem_tiles_w = (pb.w_out + 15) / 16; g.stem_tiles_h = (pb.h_out + 7) / 8;
@@ -562,10 +561,9 @@ cudaError_t launch_stem_fwd(const Problem &pb, const void *x_packed, const void 
     CUtensorMap ta, tw, tout;
     {   // overlapping windows: 64 elements (8 pixels x 8 channels) starting at every output column
         const unsigned long long dims[5] = {64, (unsigned long long)pb.w_out, (unsigned long long)pb.h_out,
-                                            (unsigned long long)pb.kh, (unsigned long long)pb.n};
-        const unsigned long long str[5] = {0, (unsigned long long)pb.stride_w * 16,
-                                           (unsigned long long)pb.stride_h * wp * 16, (unsigned long long)wp * 16,
-                                           (unsigned long long)hp * wp * 16};
+                                            (unsigned long long)krows, (unsigned long long)pb.n};
+        unsigned long long str[5];
+        stem_window_strides(pb, str);
         const unsigned int box[5] = {64, 16, 8, 1, 1};
         if (!make_tmap_tiled_bf16(&ta, x_packed, 5, dims, str, box)) return cudaErrorInvalidValue;
     }
@@ -578,7 +576,7 @@ cudaError_t launch_stem_fwd(const Problem &pb, const void *x_packed, const void 
         const unsigned int box[4] = {64, 16, 2, 1};
         if (!make_tmap_tiled_bf16(&tout, out, 4, dims, str, box)) return cudaErrorInvalidValue;
     }
-    if (!make_tmap_matrix_bf16(&tw, wst, pb.c_out, (long long)pb.kh * 64, 64, kBK)) return cudaErrorInvalidValue;
+    if (!make_tmap_matrix_bf16(&tw, wst, pb.c_out, (long long)krows * 64, 64, kBK)) return cudaErrorInvalidValue;
     int *err = nullptr;
     cudaError_t e = error_word_address(&err);
     if (e != cudaSuccess) return e;

@@ -491,7 +491,7 @@ UmmaWgradPlan stem_wgrad_plan(const Problem &pb) {
     UmmaWgradPlan pl;
     const int bn = wgrad_bn(pb);
     const long long patches = (long long)pb.n * ((pb.h_out + 3) / 4) * ((pb.w_out + 15) / 16);
-    const long long m_tiles = (pb.kh + 2) / 2, n_tiles = (pb.c_out + bn - 1) / bn;
+    const long long m_tiles = (stem_krows(pb) + 2) / 2, n_tiles = (pb.c_out + bn - 1) / bn;
     long long splits = (148 + m_tiles * n_tiles - 1) / (m_tiles * n_tiles);
     if (splits > (patches + 3) / 4) splits = (patches + 3) / 4;
     if (splits < 1) splits = 1;
@@ -502,25 +502,23 @@ UmmaWgradPlan stem_wgrad_plan(const Problem &pb) {
     return pl;
 }
 
-// partials: [splits][kh * 64][C_out]; bsum: [splits][C_out]
+// partials: [splits][krows * 64][C_out]; bsum: [splits][C_out]
 cudaError_t launch_stem_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const void *dz, const void *x_packed,
                               float *partials, float *bsum, cudaStream_t st) {
-    int hp, wp;
-    stem_geometry(pb, &hp, &wp);
+    const int krows = stem_krows(pb);
     WgradGemm g;
     g.ho = pb.h_out; g.wo = pb.w_out; g.c_in = 64; g.c_out = pb.c_out; g.taps_w = 1;
     g.lower_h = g.lower_w = 0; g.stride_h = g.stride_w = g.dil_h = g.dil_w = 1;
-    g.kdim = pb.kh * 64;
+    g.kdim = krows * 64;
     g.stem = 1; g.stem_tiles_w = (pb.w_out + 15) / 16; g.stem_tiles_h = (pb.h_out + 3) / 4;
     g.p = (long long)pb.n * g.stem_tiles_h * g.stem_tiles_w * kWP;
     g.per_split = pl.per_split; g.stages = 1; g.blockdiag = 0;
     CUtensorMap tx, tdz;
     {
         const unsigned long long dims[5] = {64, (unsigned long long)pb.w_out, (unsigned long long)pb.h_out,
-                                            (unsigned long long)pb.kh, (unsigned long long)pb.n};
-        const unsigned long long str[5] = {0, (unsigned long long)pb.stride_w * 16,
-                                           (unsigned long long)pb.stride_h * wp * 16, (unsigned long long)wp * 16,
-                                           (unsigned long long)hp * wp * 16};
+                                            (unsigned long long)krows, (unsigned long long)pb.n};
+        unsigned long long str[5];
+        stem_window_strides(pb, str);
         const unsigned int box[5] = {64, 16, 4, 1, 1};
         if (!make_tmap_tiled_bf16(&tx, x_packed, 5, dims, str, box)) return cudaErrorInvalidValue;
     }
@@ -544,9 +542,9 @@ cudaError_t launch_stem_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
     return launch_w<256>(tx, tdz, g, pl, q, partials, bsum, nullptr, err, st);
 }
 
-// One block per output channel: gathers the kh x kw x C_in real entries out of the kh x 64 padded rows,
+// One block per output channel: gathers the kh x kw x C_in real entries out of the krows x 64 padded rows,
 // adds the slices in order and finishes domega, db, dgamma, dbeta (Table 2, Tune row) or the plain sums.
-__global__ void __launch_bounds__(256) wgrad_epilogue_stem_kernel(int c_out, int kh, int kw, int c_in,
+__global__ void __launch_bounds__(256) wgrad_epilogue_stem_kernel(int c_out, int kh, int kw, int c_in, int krows, int s2d,
                                                                  const float *__restrict__ part, int splits,
                                                                  const float *__restrict__ bsum,
                                                                  const __nv_bfloat16 *__restrict__ w,
@@ -558,12 +556,13 @@ __global__ void __launch_bounds__(256) wgrad_epilogue_stem_kernel(int c_out, int
                                                                  float *__restrict__ dbeta, int need_sums) {
     __shared__ float red[256];
     const int co = blockIdx.x, kdim = kh * kw * c_in;
-    const size_t slice = (size_t)kh * 64 * c_out;
+    const size_t slice = (size_t)krows * 64 * c_out;
     const float s = vec3 ? vec3[co] : 1.f;
     float dot = 0.f;
     for (int k = threadIdx.x; k < kdim; k += blockDim.x) {
         const int c = k % c_in, t = k / c_in, q = t % kw, r = t / kw;
-        const size_t o = ((size_t)r * 64 + q * 8 + c) * c_out + co;
+        const size_t o = (s2d ? (size_t)(r >> 1) * 64 + (q >> 1) * 16 + (r & 1) * 8 + (q & 1) * 4 + c
+                              : (size_t)r * 64 + q * 8 + c) * c_out + co;
         float acc = 0.f;
         for (int sp = 0; sp < splits; ++sp) acc += part[(size_t)sp * slice + o];
         dw[(size_t)co * kdim + k] = s * acc;
@@ -597,7 +596,7 @@ cudaError_t launch_wgrad_epilogue_stem(const Problem &pb, const UmmaWgradPlan &p
                                        const float *bsum, const void *w, const float *vec3, const float *b,
                                        const float *mean, float *dw, float *db, float *dgamma, float *dbeta,
                                        bool need_sums, cudaStream_t st) {
-    wgrad_epilogue_stem_kernel<<<pb.c_out, 256, 0, st>>>(pb.c_out, pb.kh, pb.kw, pb.c_in, partials, pl.splits, bsum,
+    wgrad_epilogue_stem_kernel<<<pb.c_out, 256, 0, st>>>(pb.c_out, pb.kh, pb.kw, pb.c_in, stem_krows(pb), stem_s2d(pb) ? 1 : 0, partials, pl.splits, bsum,
                                                          (const __nv_bfloat16 *)w, vec3, b, mean, dw, db, dgamma, dbeta,
                                                          need_sums ? 1 : 0);
     return cudaGetLastError();
