@@ -129,6 +129,7 @@ cudaError_t launch_wgrad_epilogue_fused(const Problem &pb, const UmmaWgradPlan &
 bool stem_eligible(const Problem &pb);
 void stem_geometry(const Problem &pb, int *hp, int *wp);     // extent of the packed, zero-bordered input (packed pixels)
 bool stem_s2d(const Problem &pb);                            // stride 2, C_in <= 4: 2 x 2 pixel blocks per packed pixel
+bool stem_ones_in_pack(const Problem &pb);                   // the packed input carries a constant-1 slot (sum dZ row 3)
 int stem_krows(const Problem &pb);                           // 64-wide K rows per output pixel: kh, or ceil(kh / 2)
 // byte strides of the 5-D window view {64, w_out, h_out, krows, n} of the packed input
 void stem_window_strides(const Problem &pb, unsigned long long str[5]);

@@ -25,6 +25,12 @@ bool stem_s2d(const Problem &pb) { return pb.stride_h == 2 && pb.stride_w == 2 &
 
 int stem_krows(const Problem &pb) { return stem_s2d(pb) ? (pb.kh + 1) / 2 : pb.kh; }
 
+// With at most 3 channels the fourth channel slot of a packed pixel is free: the packing kernel writes the
+// constant 1 into slot (a, b, c) = (0, 0, 3), where the forward weights are zero.  In the weight-gradient
+// GEMM row 3 of the k rows is then sum_p dZ[p][co], and the separate slice of ones (a third of that
+// kernel's CTAs for a 7 x 7 stem) is not needed.
+bool stem_ones_in_pack(const Problem &pb) { return stem_s2d(pb) && pb.c_in <= 3; }
+
 void stem_geometry(const Problem &pb, int *hp, int *wp) {
     if (stem_s2d(pb)) {
         const int need_h = (pb.h_out - 1) + stem_krows(pb), need_w = (pb.w_out - 1) + 4;
@@ -61,7 +67,8 @@ size_t stem_weight_bytes(const Problem &pb) { return (size_t)pb.c_out * stem_kro
 
 // xp[n][hp][wp][a][b][4] = x[n][2 I + a - pad_h][2 J + b - pad_w][c] inside the image, 0 elsewhere
 __global__ void __launch_bounds__(256) stem_pack_s2d_kernel(int n, int h_in, int w_in, int c_in, int pad_h, int pad_w,
-                                                            int hp, int wp, const __nv_bfloat16 *__restrict__ x,
+                                                            int hp, int wp, int ones,
+                                                            const __nv_bfloat16 *__restrict__ x,
                                                             uint4 *__restrict__ xp) {
     const long long total = (long long)n * hp * wp * 2;          // one thread per (packed pixel, a)
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
@@ -73,6 +80,7 @@ __global__ void __launch_bounds__(256) stem_pack_s2d_kernel(int n, int h_in, int
         const int hq = (int)(t % hp), img = (int)(t / hp);
         const int h = 2 * hq + a - pad_h;
         unsigned short v[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        if (ones && a == 0) v[3] = 0x3F80;                       // bf16 1.0 in slot (0, 0, 3), border included
         if (h >= 0 && h < h_in) {
 #pragma unroll
             for (int b = 0; b < 2; ++b) {
@@ -121,7 +129,8 @@ cudaError_t launch_stem_pack(const Problem &pb, const void *x, void *xp, cudaStr
     if (blocks > 148 * 16) blocks = 148 * 16;
     if (stem_s2d(pb)) {
         stem_pack_s2d_kernel<<<(int)blocks, 256, 0, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.pad_h, pb.pad_w, hp, wp,
-                                                          (const __nv_bfloat16 *)x, (uint4 *)xp);
+                                                          stem_ones_in_pack(pb) ? 1 : 0, (const __nv_bfloat16 *)x,
+                                                          (uint4 *)xp);
         return cudaGetLastError();
     }
     stem_pack_kernel<<<(int)blocks, 256, 0, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.pad_h, pb.pad_w, hp, wp,

@@ -33,6 +33,7 @@ struct WgradGemm {
     // Small-C_in ("stem") mode: tm_x is the 5-D window view of the packed input (one 64-wide slice per
     // filter row), tm_dz a 4-D map of dZ; a "pixel block" is a 4 x 16 patch of output pixels.
     int stem, stem_tiles_w, stem_tiles_h;
+    int no_ones;            // 1: no slice of ones (the packed stem input carries a constant-1 slot instead)
 };
 
 struct WgradSmemCtl {
@@ -65,7 +66,7 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
     // accumulator rows are sum_p dZ[p][co], the per-channel sums needed for dbeta (Table 2), for free.
     const int nch = g.kdim / 64, c_first = k0 / 64;
     const int a_chunks = nch - c_first >= 2 ? 2 : (nch - c_first >= 1 ? 1 : 0);   // slices loaded by TMA
-    const int ones_slot = (c_first == nch) ? 0 : (c_first + 1 == nch ? 1 : -1);
+    const int ones_slot = g.no_ones ? -1 : ((c_first == nch) ? 0 : (c_first + 1 == nch ? 1 : -1));
     int b_chunks = (g.c_out - n0) / 64;
     if (b_chunks > BN / 64) b_chunks = BN / 64;
     volatile int *abort_flag = &ctl->abort_flag;
@@ -190,7 +191,7 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
             tc_fence_after_sync();
             const int k = k0 + quarter * 32 + lane;
             const bool row_ok = k < g.kdim;
-            const bool sum_row = (k == g.kdim);             // first row of the ones slice
+            const bool sum_row = !g.no_ones && (k == g.kdim);   // first row of the ones slice
             float *brow = bsum + (size_t)blockIdx.z * g.c_out + n0;
             float *orow = g.blockdiag
                               ? partials + (((size_t)blockIdx.z * gridDim.y + blockIdx.y) * g.kdim + (row_ok ? k : 0)) * 64
@@ -292,7 +293,8 @@ static cudaError_t launch_w(const CUtensorMap &tx, const CUtensorMap &tdz, Wgrad
     }
     static bool carve = false;
     prefer_max_shared_once(umma_wgrad_kernel<BN>, &carve);
-    dim3 grid((unsigned)((g.kdim / 64 + 2) / 2), (unsigned)((pb.c_out + BN - 1) / BN), (unsigned)pl.splits);
+    dim3 grid((unsigned)((g.kdim / 64 + (g.no_ones ? 1 : 2)) / 2), (unsigned)((pb.c_out + BN - 1) / BN),
+              (unsigned)pl.splits);
     return launch_pdl(umma_wgrad_kernel<BN>, grid, dim3(kWThreads), smem, st, tx, tdz, g, partials, bsum, counters,
                       pb.c_out / 32, err);
 }
@@ -304,7 +306,7 @@ cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
     g.lower_h = -pb.pad_h; g.lower_w = -pb.pad_w; g.stride_h = pb.stride_h; g.stride_w = pb.stride_w;
     g.dil_h = pb.dil_h; g.dil_w = pb.dil_w; g.kdim = pb.kdim; g.p = pb.p; g.per_split = pl.per_split; g.stages = 1;
     g.blockdiag = pb.groups > 1 ? 1 : 0;
-    g.stem = 0; g.stem_tiles_w = g.stem_tiles_h = 1;
+    g.stem = 0; g.stem_tiles_w = g.stem_tiles_h = 1; g.no_ones = 0;
     if (g.blockdiag) { g.c_in = 64; g.kdim = pb.kh * pb.kw * 64; }
     const int upper_h = g.lower_h + (pb.h_out - 1) * pb.stride_h - (pb.h_in - 1);
     const int upper_w = g.lower_w + (pb.w_out - 1) * pb.stride_w - (pb.w_in - 1);
@@ -491,7 +493,7 @@ UmmaWgradPlan stem_wgrad_plan(const Problem &pb) {
     UmmaWgradPlan pl;
     const int bn = wgrad_bn(pb);
     const long long patches = (long long)pb.n * ((pb.h_out + 3) / 4) * ((pb.w_out + 15) / 16);
-    const long long m_tiles = (stem_krows(pb) + 2) / 2, n_tiles = (pb.c_out + bn - 1) / bn;
+    const long long m_tiles = (stem_krows(pb) + (stem_ones_in_pack(pb) ? 1 : 2)) / 2, n_tiles = (pb.c_out + bn - 1) / bn;
     long long splits = (148 + m_tiles * n_tiles - 1) / (m_tiles * n_tiles);
     if (splits > (patches + 3) / 4) splits = (patches + 3) / 4;
     if (splits < 1) splits = 1;
@@ -511,6 +513,7 @@ cudaError_t launch_stem_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
     g.lower_h = g.lower_w = 0; g.stride_h = g.stride_w = g.dil_h = g.dil_w = 1;
     g.kdim = krows * 64;
     g.stem = 1; g.stem_tiles_w = (pb.w_out + 15) / 16; g.stem_tiles_h = (pb.h_out + 3) / 4;
+    g.no_ones = stem_ones_in_pack(pb) ? 1 : 0;
     g.p = (long long)pb.n * g.stem_tiles_h * g.stem_tiles_w * kWP;
     g.per_split = pl.per_split; g.stages = 1; g.blockdiag = 0;
     CUtensorMap tx, tdz;
@@ -545,6 +548,7 @@ cudaError_t launch_stem_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
 // One block per output channel: gathers the kh x kw x C_in real entries out of the krows x 64 padded rows,
 // adds the slices in order and finishes domega, db, dgamma, dbeta (Table 2, Tune row) or the plain sums.
 __global__ void __launch_bounds__(256) wgrad_epilogue_stem_kernel(int c_out, int kh, int kw, int c_in, int krows, int s2d,
+                                                                 int sum_row,
                                                                  const float *__restrict__ part, int splits,
                                                                  const float *__restrict__ bsum,
                                                                  const __nv_bfloat16 *__restrict__ w,
@@ -570,7 +574,8 @@ __global__ void __launch_bounds__(256) wgrad_epilogue_stem_kernel(int c_out, int
     }
     float bs = 0.f;
     if (need_sums)
-        for (int sp = threadIdx.x; sp < splits; sp += blockDim.x) bs += bsum[(size_t)sp * c_out + co];
+        for (int sp = threadIdx.x; sp < splits; sp += blockDim.x)   // sum dZ: its own array, or k row `sum_row`
+            bs += sum_row >= 0 ? part[(size_t)sp * slice + (size_t)sum_row * c_out + co] : bsum[(size_t)sp * c_out + co];
     red[threadIdx.x] = dot;
     __syncthreads();
     for (int o = 128; o > 0; o >>= 1) { if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o]; __syncthreads(); }
@@ -596,7 +601,8 @@ cudaError_t launch_wgrad_epilogue_stem(const Problem &pb, const UmmaWgradPlan &p
                                        const float *bsum, const void *w, const float *vec3, const float *b,
                                        const float *mean, float *dw, float *db, float *dgamma, float *dbeta,
                                        bool need_sums, cudaStream_t st) {
-    wgrad_epilogue_stem_kernel<<<pb.c_out, 256, 0, st>>>(pb.c_out, pb.kh, pb.kw, pb.c_in, stem_krows(pb), stem_s2d(pb) ? 1 : 0, partials, pl.splits, bsum,
+    wgrad_epilogue_stem_kernel<<<pb.c_out, 256, 0, st>>>(pb.c_out, pb.kh, pb.kw, pb.c_in, stem_krows(pb), stem_s2d(pb) ? 1 : 0,
+                                                         stem_ones_in_pack(pb) ? 3 : -1, partials, pl.splits, bsum,
                                                          (const __nv_bfloat16 *)w, vec3, b, mean, dw, db, dgamma, dbeta,
                                                          need_sums ? 1 : 0);
     return cudaGetLastError();
