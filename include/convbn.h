@@ -230,7 +230,7 @@ int convbn_check(void *stream);
 const char *convbn_status_string(int status);
 
 /* Name of the kernel family the last call of `phase` selected on this thread, for logs and tests:
- * "direct", "umma", "umma-strip", "umma-strided", "umma-stem", "stem-mma", "depthwise",
+ * "direct", "umma", "umma-strip", "umma-strided", "umma-subpixel", "umma-stem", "stem-mma", "depthwise",
  * "grouped-mma", "grouped-umma".  Static string, never NULL. */
 const char *convbn_last_kernel(int phase);
 
