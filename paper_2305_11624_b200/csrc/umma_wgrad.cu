@@ -362,6 +362,26 @@ __global__ void __launch_bounds__(32 * KR * SL, SL == 16 ? 2 : (KR * SL == 8 ? 4
         const int k = k0 + rep * KR + (int)(threadIdx.x % KR), co = co0 + (int)(threadIdx.x / KR);
         wv[rep] = (vec3 && threadIdx.x < 32 * KR && k < kdim) ? __bfloat162float(w[(size_t)co * kdim + k]) : 0.f;
     }
+    constexpr int NBF = REP > 1 ? 32 / REP : 1;      // slices the preloading path below can take
+    if (SL == 1 && REP > 1 && splits <= NBF) {
+        // few slices, several row groups: request every value of every group before the first use, so that
+        // REP x splits loads are in flight per thread instead of `splits`; same order of additions as below
+        float a[REP][NBF];
+#pragma unroll
+        for (int rep = 0; rep < REP; ++rep) {
+            const int k = k0 + rep * KR + ty;
+            const float *src = part + (size_t)k * c_out + co0 + tx;
+#pragma unroll
+            for (int u = 0; u < NBF; ++u) a[rep][u] = (k < kdim && u < splits) ? __ldcg(src + (size_t)u * slice) : 0.f;
+        }
+#pragma unroll
+        for (int rep = 0; rep < REP; ++rep) {
+            float tot = 0.f;
+#pragma unroll
+            for (int u = 0; u < NBF; ++u) tot += a[rep][u];
+            tile[rep][tz][ty][tx] = tot;
+        }
+    } else
 #pragma unroll
     for (int rep = 0; rep < REP; ++rep) {
         const int k = k0 + rep * KR + ty;
