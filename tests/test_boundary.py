@@ -50,6 +50,24 @@ def test_out_shape_and_sizes():
     assert C.convbn_workspace_bytes(d, 99) == 0
 
 
+def test_workspace_sizes_of_the_benchmark_layers():
+    """Every phase of every benchmark layer asks for a 256-byte multiple; the parameter-gradient scratch
+    (partial tiles per pixel slice) stays within a few tens of MiB, and that of the headline configuration's
+    layers within the 16 MiB of the no-allocation entry point."""
+    from paper_2305_11624_b200 import inputs as I
+    from paper_2305_11624_b200.harness import make_desc
+    for ci, layers in I.CONFIGS.items():
+        for sp in layers:
+            d = make_desc(sp)
+            for ph in (C.PHASE_TUNE_FWD, C.PHASE_TUNE_BWD_DATA, C.PHASE_TUNE_BWD_WEIGHT):
+                ws = C.convbn_workspace_bytes(d, ph)
+                assert ws % 256 == 0 and ws < 64 << 20, (sp.name, ph, ws)
+            wsw = C.convbn_workspace_bytes(d, C.PHASE_TUNE_BWD_WEIGHT)
+            assert wsw > 0, sp.name
+            if ci == 1:
+                assert wsw <= 16 << 20, (sp.name, wsw)
+
+
 @pytest.mark.parametrize("kw", [
     dict(n=0), dict(c_in=-1), dict(kh=0), dict(stride_h=0), dict(dil_w=0), dict(pad_h=-1),
     dict(groups=3), dict(groups=0), dict(h_in=1, w_in=1, pad_h=0, pad_w=0), dict(dtype=7),
