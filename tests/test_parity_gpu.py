@@ -132,7 +132,9 @@ def test_tune_is_deterministic_and_leaves_inputs_alone():
         assert torch.equal(getattr(blk, k), v), k
 
 
-@pytest.mark.parametrize("spec", [SMALL[0], SMALL[8], SMALL[10], SMALL[17], SMALL[19]], ids=lambda s: s.name)
+@pytest.mark.parametrize("spec", [SMALL[0], SMALL[8], SMALL[10], SMALL[17], SMALL[19]] +
+                         [sp for sp in SMALL if sp.name in ("b_stem_3x3_s2", "b_sub_c4", "b_sub_wide")],
+                         ids=lambda s: s.name)
 def test_eval_and_deploy_comparators(spec):
     """Eval and Deploy entry points against the oracle's Eval-row and Deploy-row equations, and
     the paper's claim Z_eval = Z_deploy = Z_tune on the device outputs themselves."""
