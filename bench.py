@@ -2,19 +2,24 @@
 """Benchmark of the Tune-mode ConvBN hot path on B200.
 
 A step is one pass of the whole path - convbn_tune_fwd, convbn_tune_bwd_data and
-convbn_tune_bwd_weight - over every layer of the workload (default: the ResNet-50 stage-2
-bottleneck chain, bf16 NHWC, N=32 at 56x56).  The metric is fwd+bwd TFLOP/s with
-FLOPs = 3 phases x 2 P C_out (C_in/G) kh kw per layer.
+convbn_tune_bwd_weight - over every layer of a configuration.  With no ``--workload`` all five
+configurations run in one process and ONE JSON line is printed: ``value`` is the fwd+bwd TFLOP/s
+over the three dense bf16 configurations (1-3: total FLOPs / total time), ``per_config`` holds
+every configuration on its own (config 4 in GB/s against the copy bandwidth, config 0 as a
+latency).  FLOPs = 3 phases x 2 P C_out (C_in/G) kh kw per layer.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload 1]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload i]
 
-Under torchrun every rank runs its own replica of the workload on its own batch (the path needs
-no exchange between samples), times it with CUDA events, and rank 0 prints one JSON line with the
-max-over-ranks time.  ``--impl reference`` times the fp64 CPU oracle instead (rank 0 only).
+Under torchrun every rank runs its own replica on its own batch (the path needs no exchange
+between samples), times it with CUDA events, and rank 0 prints the line with the max-over-ranks
+time; ``--gpus N`` without a launcher starts the N ranks itself.  ``--impl reference`` times the
+fp64 CPU oracle instead (rank 0 only).
 """
 import argparse
 import json
+import math
 import os
+import subprocess
 import sys
 import threading
 import time
@@ -33,6 +38,7 @@ WORKLOAD_NAMES = {
     3: "config3: detection-backbone 3x3 layers at 800x1333, bf16 NHWC, N=2",
     4: "config4: depthwise 3x3 C=96 at 112x112 and grouped 3x3 G=32 256->256 at 28x28, bf16 NHWC, N=64",
 }
+DENSE = (1, 2, 3)          # the configurations behind `value`
 
 
 def load_peaks():
@@ -59,23 +65,21 @@ def kernel_bytes(kind, spec, out_hw):
         return z + wel * es + x
     if kind == "wgrad":    # read dZ and X, write fp32 domega'
         return z + x + wel * 4
+    if kind == "bwd":      # fused backward: dZ and X read once, dX and fp32 domega' written
+        return z + 2 * x + wel * es + wel * 4
     raise KeyError(kind)
 
 
-# DRAM bytes (read + write) per launch from the ncu capture summarised in
-# profiles/config1_gemm_kernels_ncu_full.md; None for kernels changed or not captured since.
-NCU_TRAFFIC = {("umma_fwd", "c1a"): 51.71e6, ("umma_dgrad", "c1a"): 13.80e6, ("umma_wgrad", "c1a"): 65.09e6,
-               ("strip_fwd", "c1b"): 12.96e6, ("strip_dgrad", "c1b"): 12.96e6, ("umma_wgrad", "c1b"): 25.71e6,
-               ("umma_fwd", "c1c"): 13.86e6, ("umma_dgrad", "c1c"): 51.94e6, ("umma_wgrad", "c1c"): 65.54e6,
-               ("dw_fwd", "c4a"): 262.4e6, ("dw_dgrad", "c4a"): 261.0e6, ("dw_wgrad", "c4a"): 312.3e6,
-               ("grouped_dgrad", "c4b"): 29.1e6, ("grouped_wgrad", "c4b"): 51.8e6,
-               ("stem_dgrad", "c2s"): 109.5e6}
+# DRAM bytes (read + write) per launch, from ncu captures of the kernels as they are now; a kernel that
+# changed after its capture has no entry (traffic: null).  key: (kernel family, layer).
+NCU_TRAFFIC = {}
 
 KIND_OF = {"strip_fwd": "fwd", "strip_dgrad": "dgrad", "direct_fwd": "fwd", "direct_dgrad": "dgrad", "direct_wgrad": "wgrad",
-           "umma_fwd": "fwd", "umma_dgrad": "dgrad", "umma_wgrad": "wgrad",
+           "umma_fwd": "fwd", "umma_dgrad": "dgrad", "umma_wgrad": "wgrad", "umma_bwd": "bwd",
            "dw_fwd": "fwd", "dw_dgrad": "dgrad", "dw_wgrad": "wgrad",
            "grouped_fwd": "fwd", "grouped_dgrad": "dgrad", "grouped_wgrad": "wgrad",
            "stem_fwd": "fwd", "stem_dgrad": "dgrad", "stem_wgrad": "wgrad"}
+PHASE_KIND = {"fwd": "fwd", "bwd_data": "dgrad", "bwd_weight": "wgrad", "bwd": "bwd"}
 
 
 def shape_tag(spec):
@@ -86,7 +90,7 @@ def shape_tag(spec):
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons of one GPU through NVML (read-only) while running."""
 
-    def __init__(self, uuid, period=0.01):
+    def __init__(self, uuid, period=0.005):
         super().__init__(daemon=True)
         self.period, self.stop_flag = period, threading.Event()
         self.sm, self.reasons, self.sm_max, self.ok = [], set(), None, False
@@ -125,6 +129,11 @@ class ClockSampler(threading.Thread):
                 pass
             self.stop_flag.wait(self.period)
 
+    def finish(self):
+        self.stop_flag.set()
+        self.join()
+        return self.summary()
+
     def summary(self):
         if not self.ok or not self.sm:
             return {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": ["nvml-unavailable"]}
@@ -135,6 +144,26 @@ class ClockSampler(threading.Thread):
                  "ApplicationsClocksSetting": "applications_clocks_setting"}
         return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.sm_max, "samples": len(s),
                 "reasons": sorted(snake[r] for r in self.reasons)}
+
+
+def merge_clocks(summaries):
+    """One clocks object over several timed regions: median of the medians, union of the reasons."""
+    ok = [c for c in summaries if c.get("sm_mhz") is not None]
+    if not ok:
+        return summaries[0] if summaries else {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvml-unavailable"]}
+    med = sorted(c["sm_mhz"] for c in ok)
+    return {"sm_mhz": med[len(med) // 2], "sm_max_mhz": ok[0]["sm_max_mhz"],
+            "samples": sum(c.get("samples", 0) for c in ok),
+            "reasons": sorted(set(r for c in ok for r in c["reasons"]))}
+
+
+def tensor_peak(peaks, clocks):
+    """The measured bf16 peak that applies: the burst figure while the sampled SM clock stays within
+    5 % of its maximum with no power cap, else the sustained one."""
+    burst, sus = peaks["bf16_tflops"], peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+    sm, mx = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    at_max = sm is not None and mx and sm >= 0.95 * mx and "sw_power_cap" not in clocks.get("reasons", [])
+    return (burst, "burst") if at_max or sm is None else (sus, "sustained")
 
 
 # ---- multi-rank bookkeeping (replicas: every rank runs the whole workload on its own batch) -------
@@ -152,6 +181,19 @@ def max_over_ranks(value, device=None):
 def whole_job_value(flops_per_step, steps, ms_max, world):
     """Aggregate TFLOP/s of `world` replicas that each did `steps` steps within `ms_max` milliseconds."""
     return world * flops_per_step * steps / (ms_max * 1e-3) / 1e12
+
+
+def spawn_ranks(args):
+    """`--gpus N` without a launcher: start N ranks of this script under torch.distributed.run."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")           # the communicator's rank count stays in the log
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd, env=env)
 
 
 # ---- the CPU oracle, timed (reported baseline and the --impl reference arm) ----------------------
@@ -183,15 +225,19 @@ def run_reference(args):
     if rank != 0:
         return
     batch = args.ref_batch
-    times, flops, cores = oracle_step_time(args.workload, batch, args.warmup + args.steps)
-    timed = times[args.warmup:]
-    per = sum(timed) / len(timed)
+    workloads = [args.workload] if args.workload is not None else list(DENSE)
+    per, flops, cores = 0.0, 0.0, 0
+    for wl in workloads:
+        times, fl, cores = oracle_step_time(wl, batch, args.warmup + args.steps)
+        timed = times[args.warmup:]
+        per += sum(timed) / len(timed)
+        flops += fl
     val = flops / per / 1e12
     sample = "fp64 oracle, Tune fwd+bwd of every layer of the workload on a batch of %d samples per step" % batch
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": per * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": {"workload": WORKLOAD_NAMES[args.workload], "sample": sample},
+            "data": "synthetic", "config": {"workload": "; ".join(WORKLOAD_NAMES[w] for w in workloads), "sample": sample},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -199,39 +245,81 @@ def run_reference(args):
 
 
 # ---- the CUDA path ------------------------------------------------------------------------------
-def run_ours(args):
-    import torch
-    import torch.distributed as dist
-    import __graft_entry__ as G
-    from paper_2305_11624_b200 import convbn as C
-    from paper_2305_11624_b200 import inputs as I
-    from paper_2305_11624_b200.harness import Block
+class Ctx:
+    pass
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-    if rank == 0:
-        G.build()
-    if world > 1:
-        dist.barrier()
-    C.lib()
 
-    layers = I.CONFIGS[args.workload]
-    sets = max(1, args.buffer_sets)
-    blocks = [[Block(sp, device=dev) for sp in layers] for _ in range(sets)]
+def measured_activation_bytes(ctx, layers, mode):
+    """Peak of torch's allocator over forward (every layer) then backward (reverse order) of the layers, minus
+    what was allocated before: what a framework holding these layers keeps alive between the two passes plus
+    the transients of a call.  Outputs, `saved` state and per-call scratch are allocated inside the region;
+    an input whose shape matches the previous layer's output IS that output (a chain)."""
+    torch, C, Block = ctx.torch, ctx.C, ctx.Block
+    dev = ctx.dev
+    blks = [Block(sp, device=dev, modes=(mode,), allocate="params") for sp in layers]
+    for i, b in enumerate(blks):
+        b.randomize_params(1000 + i)
+    es = lambda b: 2 if b.spec.dtype == "bf16" else 4
+    new = lambda n, dt: torch.empty(int(n), dtype=dt, device=dev)
+    torch.cuda.synchronize()
+    torch.cuda.reset_peak_memory_stats(dev)
+    base = torch.cuda.memory_allocated(dev)
+    x = None
+    for b in blks:
+        nx = math.prod(b.x_shape)
+        if x is None or x.numel() != nx or x.dtype != b.tdtype:
+            x = new(nx, b.tdtype).normal_()
+        b.x = x
+        b.z = new(math.prod(b.z_shape), b.tdtype)
+        if mode == "tune":
+            b.saved = new(max(16, C.convbn_saved_bytes(b.desc, C.MODE_TUNE)), torch.uint8)
+            b.with_scratch(C.PHASE_TUNE_FWD, b.tune_fwd)
+        else:
+            b.y_saved = new(C.convbn_saved_bytes(b.desc, C.MODE_EVAL), torch.uint8)
+            b.with_scratch(C.PHASE_EVAL_FWD, b.eval_fwd)
+        x = b.z
+        b.z = None                      # the output lives on only as the next layer's input (or the loss's)
+    dz = torch.empty_like(x).normal_()
+    del x
+    for b in reversed(blks):
+        if dz.numel() != math.prod(b.z_shape):
+            dz = new(math.prod(b.z_shape), b.tdtype).normal_()
+        b.dz = dz
+        b.dx = new(math.prod(b.x_shape), b.tdtype)
+        if mode == "tune":
+            b.with_scratch(C.PHASE_TUNE_BWD_DATA, b.tune_bwd_data)
+            b.with_scratch(C.PHASE_TUNE_BWD_WEIGHT, b.tune_bwd_weight)
+            b.saved = None
+        else:
+            b.with_scratch(C.PHASE_EVAL_BWD, b.eval_bwd)
+            b.y_saved = None
+        dz = b.dx
+        b.x = b.dz = b.dx = None
+    torch.cuda.synchronize()
+    C.convbn_check()
+    peak = torch.cuda.max_memory_allocated(dev) - base
+    del blks, dz
+    return int(peak)
+
+
+def bench_config(ctx, wl):
+    """Everything measured on one configuration; returns its per_config entry (rank 0) plus raw sums."""
+    args, torch, C, I, Block = ctx.args, ctx.torch, ctx.C, ctx.I, ctx.Block
+    dev, rank, world, peaks, peak_src = ctx.dev, ctx.rank, ctx.world, ctx.peaks, ctx.peak_src
+    dist = ctx.dist
+    layers = I.CONFIGS[wl]
+    probe = [Block(sp, device=dev) for sp in layers]
+    step_flops = sum(3 * b.flops_per_phase() for b in probe)
+    footprint = sum(t.numel() * t.element_size() for b in probe for t in (b.x, b.dz, b.z, b.dx))
+    two_pass_bytes = sum(kernel_bytes(k, b.spec, (b.h_out, b.w_out)) for b in probe for k in ("fwd", "dgrad", "wgrad"))
+    l2 = int(torch.cuda.get_device_properties(dev).L2_cache_size)
+    sets = args.buffer_sets if args.buffer_sets > 0 else max(2, min(16, int(math.ceil(2.0 * l2 / footprint)) + 1))
+    blocks = [probe] + [[Block(sp, device=dev) for sp in layers] for _ in range(sets - 1)]
     for si, bs in enumerate(blocks):
         for li, b in enumerate(bs):
-            b.randomize(I.config_seed(args.workload, li) + 7919 * (rank * sets + si))
-    step_flops = sum(3 * b.flops_per_phase() for b in blocks[0])
-    footprint = sum(t.numel() * t.element_size() for b in blocks[0] for t in (b.x, b.dz, b.z, b.dx))
-
+            b.randomize(I.config_seed(wl, li) + 7919 * (rank * sets + si))
     stream = torch.cuda.current_stream()
+    calls_per_step = 3 * len(layers)
 
     def step(i):
         for b in blocks[i % sets]:
@@ -242,17 +330,13 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(args.warmup):
+    for i in range(max(args.warmup, sets)):
         step(i)
     C.convbn_check()
     barrier()
-    uuid = str(torch.cuda.get_device_properties(dev).uuid)
-    sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
-    sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
-    # ---- timed region: K steps, each a replay of the CUDA graph of one step (one graph per buffer
-    # set), so the layers' ~15 launches per step cost no host time; --no-graph times eager calls.
+    # ---- timed region: K steps, each a replay of the CUDA graph of one step (one graph per buffer set), so
+    # the launches of a step cost no host time; --no-graph times eager calls.
     graphs, launch_mode = None, "eager library calls"
     if not args.no_graph:
         try:
@@ -269,18 +353,27 @@ def run_ours(args):
             launch_mode = "CUDA graph replay (one captured step per buffer set)"
         except Exception as exc:  # capture unsupported: say so and time eager calls
             graphs, launch_mode = None, "eager library calls (graph capture failed: %r)" % (exc,)
-    barrier()
-    e0.record(stream)
-    for i in range(args.steps):
-        if graphs:
-            graphs[(args.warmup + i) % sets].replay()
-        else:
-            step(args.warmup + i)
-    e1.record(stream)
-    barrier()
-    ms = max_over_ranks(e0.elapsed_time(e1), dev)
-    value = whole_job_value(step_flops, args.steps, ms, world)
 
+    def timed(n_sets):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for i in range(3):                      # a few untimed replays settle clocks and caches
+            graphs[i % n_sets].replay() if graphs else step(i % n_sets)
+        barrier()
+        e0.record(stream)
+        for i in range(args.steps):
+            if graphs:
+                graphs[i % n_sets].replay()
+            else:
+                step(i % n_sets)
+        e1.record(stream)
+        barrier()
+        return max_over_ranks(e0.elapsed_time(e1), dev)
+
+    uuid = str(torch.cuda.get_device_properties(dev).uuid)
+    sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+    sampler.start()
+    ms = timed(sets)                            # cold: rotating sets, together larger than twice the L2
+    ms_warm = timed(1)                          # warm: the same buffers every step
     # ---- second pass, same K steps as eager calls with a CUDA-event pair around every kernel: the
     # per-kernel durations behind the roofline object (events cannot be read back out of a graph)
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -288,20 +381,29 @@ def run_ours(args):
     barrier()
     f0.record(stream)
     for i in range(args.steps):
-        step(args.warmup + i)
+        step(i)
     f1.record(stream)
     barrier()
     prof = C.convbn_profile_end()
     eager_ms = max_over_ranks(f0.elapsed_time(f1), dev)
-    sampler.stop_flag.set()
-    sampler.join()
+    clocks = sampler.finish()
     C.convbn_check()
+    # host time of a library call (descriptor checks, plans, tensor maps, launches), GPU work queued behind
+    hsteps = max(1, min(args.steps, 256 // calls_per_step))
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(hsteps):
+        step(i)
+    host_us = (time.perf_counter() - t0) / (hsteps * calls_per_step) * 1e6
+    torch.cuda.synchronize()
 
-    # ---- roofline of the dominant kernel -----------------------------------------------------
-    peaks, peak_src = load_peaks()
+    # ---- rooflines ---------------------------------------------------------------------------------
+    hbm = peaks["hbm_gbs"]
+    tc, tc_kind = tensor_peak(peaks, clocks)
+    tc_burst, tc_sus = peaks["bf16_tflops"], peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+    ridge = tc_burst * 1e12 / (hbm * 1e9)               # FLOP per byte above which the tensor peak bounds
     tag2layer = {shape_tag(b.spec): b for b in blocks[0]}
-    kernels = []
-    phase_ms = {}                                    # (layer tag, phase) -> milliseconds over the eager pass
+    kernels, phase_ms = [], {}
     for name, (count, total_ms) in prof.items():
         fam, _, rest = name.partition("@")
         tag, _, phase = rest.partition("#")
@@ -312,60 +414,90 @@ def run_ours(args):
     all_ms = sum(k["total_ms"] for k in kernels) or 1.0
     for k in kernels:
         k["share"] = k["total_ms"] / all_ms
-    roofline = None
-    if kernels:
-        top = kernels[0]
+
+    def roofline_of(top):
         b = tag2layer.get(top["_tag"])
         kind = KIND_OF.get(top["kernel"])
+        if b is None or not kind:
+            return None
         # a pass that takes several launches of this kernel per step (one per residue class of a strided
         # backward pass) is judged as a whole: its algorithmic bytes and FLOPs are those of the pass
         per_step = max(1, round(top["launches"] / args.steps))
         dur = top["total_ms"] / top["launches"] * per_step * 1e-3
-        if b is not None and kind:
-            fl = b.flops_per_phase()
-            by = kernel_bytes(kind, b.spec, (b.h_out, b.w_out))
-            hbm, tc = peaks["hbm_gbs"], peaks["bf16_tflops_sustained"]
-            dense_bf16 = b.spec.dtype == "bf16" and b.spec.groups == 1
-            tensor_bound = dense_bf16 and (fl / by) > (tc * 1e12) / (hbm * 1e9)
-            if tensor_bound:
-                ach = fl / dur / 1e12
-                roofline = {"bound": "tensor", "achieved": ach, "peak": tc, "unit": "TFLOP/s",
-                            "frac": ach / tc, "traffic": NCU_TRAFFIC.get((top["kernel"], top["layer"])),
-                            "peak_source": peak_src + " bf16 sustained (kernel timed inside a long step)"}
-            else:
-                ach = by / dur / 1e9
-                roofline = {"bound": "hbm", "achieved": ach, "peak": hbm, "unit": "GB/s",
-                            "frac": ach / hbm, "traffic": NCU_TRAFFIC.get((top["kernel"], top["layer"])),
-                            "peak_source": peak_src + " copy bandwidth"}
-            roofline.update({"kernel": top["kernel"], "layer": top["layer"], "us_per_launch": dur * 1e6 / per_step,
-                             "launches_per_step": per_step, "us_per_step": dur * 1e6,
-                             "algorithmic_bytes": by, "algorithmic_flops": fl, "share_of_step": top["share"]})
-    for k in kernels:
-        k.pop("_tag")
+        fl = b.flops_per_phase() * (2 if kind == "bwd" else 1)
+        by = kernel_bytes(kind, b.spec, (b.h_out, b.w_out))
+        dense_bf16 = b.spec.dtype == "bf16" and b.spec.groups == 1
+        traffic = NCU_TRAFFIC.get((top["kernel"], top["layer"]))
+        if dense_bf16 and fl / by > ridge:
+            ach = fl / dur / 1e12
+            r = {"bound": "tensor", "achieved": ach, "peak": tc, "unit": "TFLOP/s", "frac": ach / tc,
+                 "traffic": traffic, "peak_source": "%s bf16 %s peak (clocks %s MHz of %s, reasons %s)"
+                 % (peak_src, tc_kind, clocks.get("sm_mhz"), clocks.get("sm_max_mhz"), clocks.get("reasons")),
+                 "frac_of_burst": ach / tc_burst, "frac_of_sustained": ach / tc_sus}
+        else:
+            ach = by / dur / 1e9
+            r = {"bound": "hbm", "achieved": ach, "peak": hbm, "unit": "GB/s", "frac": ach / hbm,
+                 "traffic": traffic, "peak_source": peak_src + " copy bandwidth"}
+        r.update({"kernel": top["kernel"], "layer": top["layer"], "us_per_launch": dur * 1e6 / per_step,
+                  "launches_per_step": per_step, "us_per_step": dur * 1e6, "algorithmic_bytes": by,
+                  "algorithmic_flops": fl, "share_of_step": top["share"], "total_ms": top["total_ms"],
+                  "timing": "CUDA-event pair around each launch on the launching stream, eager pass"})
+        return r
+
+    roofline = roofline_of(kernels[0]) if kernels else None
     # every layer and phase (all kernels of the call, weight re-layouts and epilogues included) against its
     # own roofline: the larger of FLOPs / tensor peak (dense bf16 only) and algorithmic bytes / copy bandwidth
     per_layer = []
-    hbm, tc = peaks["hbm_gbs"], peaks["bf16_tflops_sustained"]
     for (tag, phase), tot in sorted(phase_ms.items()):
         b = tag2layer.get(tag)
-        kind = {"fwd": "fwd", "bwd_data": "dgrad", "bwd_weight": "wgrad"}.get(phase)
+        kind = PHASE_KIND.get(phase)
         if b is None or kind is None:
             continue
         us = tot / args.steps * 1e3
-        fl, by = b.flops_per_phase(), kernel_bytes(kind, b.spec, (b.h_out, b.w_out))
+        fl = b.flops_per_phase() * (2 if kind == "bwd" else 1)
+        by = kernel_bytes(kind, b.spec, (b.h_out, b.w_out))
         t_hbm = by / (hbm * 1e9) * 1e6
         t_tc = fl / (tc * 1e12) * 1e6 if (b.spec.dtype == "bf16" and b.spec.groups == 1) else 0.0
         per_layer.append({"layer": b.spec.name, "phase": phase, "us": round(us, 2),
                           "bound": "tensor" if t_tc > t_hbm else "hbm", "roof_us": round(max(t_hbm, t_tc), 2),
                           "frac": round(max(t_hbm, t_tc) / us, 3) if us > 0 else None})
+    launches_per_step = sum(k["launches"] for k in kernels) / float(args.steps)
+    for k in kernels:
+        k.pop("_tag")
 
-    # ---- Tune against the Eval- and Deploy-mode paths built from the same kernels (the paper's
-    # comparison: Table 2, Fig. 3), eager calls, forward + full backward of every layer per step
-    modes = None
+    out = {"workload": WORKLOAD_NAMES[wl], "layers": [b.spec.name for b in blocks[0]],
+           "ms_per_step": ms / args.steps, "ms_per_step_warm": ms_warm / args.steps,
+           "tflops": whole_job_value(step_flops, args.steps, ms, world),
+           "gbs_two_pass": world * two_pass_bytes * args.steps / (ms * 1e-3) / 1e9,
+           "frac_of_copy_bandwidth": world * two_pass_bytes * args.steps / (ms * 1e-3) / 1e9 / hbm / world,
+           "flops_per_step": step_flops, "two_pass_bytes_per_step": two_pass_bytes,
+           "l2": "cold: %d rotating buffer sets of %.0f MB (activations) against an L2 of %.0f MB; warm: one set"
+                 % (sets, footprint / 1e6, l2 / 1e6),
+           "launch": launch_mode, "launches_per_step": launches_per_step, "host_us_per_call": round(host_us, 2),
+           "eager_ms_per_step": eager_ms / args.steps, "clocks": clocks, "roofline": roofline,
+           "kernels": kernels[:10], "per_layer": per_layer,
+           "activation_bytes": {b.spec.name: {m: b.saved_bytes(m) for m in ("tune", "eval", "deploy")}
+                                for b in blocks[0]}}
+    if wl == 0:
+        out["latency_us_per_step"] = ms / args.steps * 1e3
+    gpu_launches = sum(k["launches"] for k in kernels)
+
+    # ---- end to end through the host-buffer entry point ---------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(ctx, blocks[0], stream, step_flops)
+        out["e2e"] = e2e
+    del graphs
+    blocks = [blocks[0]]
+    torch.cuda.empty_cache()
+
+    # ---- Tune against the Eval- and Deploy-mode paths built from the same kernels (the paper's comparison:
+    # Table 2, Fig. 3), eager calls, forward + full backward of every layer per step; and the measured
+    # allocator peak of a forward-hold-backward pass, Tune against Eval (Sec. 3.4, Appendix M)
     if not args.no_modes and rank == 0:
         mblocks = [Block(sp, device=dev, modes=("tune", "eval", "deploy")) for sp in layers]
         for li, b in enumerate(mblocks):
-            b.randomize(I.config_seed(args.workload, li) + 17)
+            b.randomize(I.config_seed(wl, li) + 17)
             b.deploy_prepare()
 
         def run_mode(m):
@@ -391,52 +523,33 @@ def run_ours(args):
             torch.cuda.synchronize()
             modes[m] = {"ms_per_step": m0.elapsed_time(m1) / ksteps,
                         "saved_bytes": sum(b.saved_bytes(m) for b in mblocks)}
-        modes["note"] = "eager calls, %d steps each; saved_bytes = X plus what the mode keeps for backward" % ksteps
+        modes["note"] = "eager calls, %d steps each; saved_bytes = X plus what the mode keeps for backward (analytic)" % ksteps
         C.convbn_check()
         del mblocks
+        torch.cuda.empty_cache()
+        meas = {m: measured_activation_bytes(ctx, layers, m) for m in ("tune", "eval")}
+        meas["note"] = ("torch.cuda.max_memory_allocated minus the bytes allocated before, over forward of every "
+                        "layer then backward in reverse order; outputs, saved state and per-call scratch allocated inside")
+        out["modes"] = modes
+        out["activation_bytes_measured"] = meas
+    del blocks, probe
+    torch.cuda.empty_cache()
 
-    # ---- end to end through the host-buffer entry point ---------------------------------------
-    e2e = None
-    if not args.no_e2e:
-        e2e = run_e2e(args, torch, C, blocks[0], dev, stream, world, step_flops)
-
-    # ---- CPU baseline (rank 0, single GPU only) ------------------------------------------------
-    cpu = None
+    # ---- CPU baseline (rank 0, single GPU only): the oracle as it stands, one full step of this config ----
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        full = layers[0].n
-        times, fl, cores = oracle_step_time(args.workload, full, 2)  # ~2 x 3 s on 16 cores
-        cpu = {"value": fl / min(times) / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": "one full step (all %d samples of every layer) of the fp64 oracle, best of 2, %.1f s"
-                         % (full, min(times))}
-
-    if rank == 0:
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None,
-                "dtype": "bf16" if layers[0].dtype == "bf16" else "f32", "data": "synthetic",
-                "config": {"workload": WORKLOAD_NAMES[args.workload],
-                           "layers": [b.spec.name for b in blocks[0]],
-                           "l2": "step footprint %.0f MB of activations > L2; %d rotating buffer sets"
-                                 % (footprint / 1e6, sets),
-                           "flops_per_step": step_flops, "parallelism": "replicas x%d" % world,
-                           "launch": launch_mode},
-                "eager": {"ms_per_step": eager_ms / args.steps,
-                          "value": world * step_flops * args.steps / (eager_ms * 1e-3) / 1e12,
-                          "note": "same steps as plain library calls with per-kernel CUDA events (source of `kernels` and `roofline`)"},
-                "clocks": sampler.summary(), "e2e": e2e,
-                "gpu_launches": sum(k["launches"] for k in kernels),
-                "roofline": roofline, "cpu_baseline": cpu, "modes": modes, "kernels": kernels[:12], "per_layer": per_layer,
-                "activation_bytes": {b.spec.name: {m: b.saved_bytes(m) for m in ("tune", "eval", "deploy")}
-                                     for b in blocks[0]}}
-        print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+        times, fl, cores = oracle_step_time(wl, layers[0].n, 1)
+        out["cpu_baseline"] = {"value": fl / times[0] / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+                               "seconds": times[0], "flops": fl,
+                               "sample": "one full step (all %d samples of every layer) of the fp64 oracle, %.1f s"
+                                         % (layers[0].n, times[0])}
+    out["_raw"] = {"ms": ms, "flops": step_flops, "gpu_launches": gpu_launches, "bytes": two_pass_bytes}
+    return out
 
 
-def run_e2e(args, torch, C, blks, dev, stream, world, step_flops):
+def run_e2e(ctx, blks, stream, step_flops):
     """The same step through convbn_tune_step_host: inputs in pinned host memory, every output
     copied back, copies inside the timed region."""
-    import torch.distributed as dist
+    args, torch, C, dev, world, dist = ctx.args, ctx.torch, ctx.C, ctx.dev, ctx.world, ctx.dist
     host = []
     h2d = d2h = 0
     for b in blks:
@@ -465,26 +578,97 @@ def run_e2e(args, torch, C, blks, dev, stream, world, step_flops):
         step()
     e1.record(stream)
     torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(e0.elapsed_time(e1), dev)
     return {"value": world * step_flops * steps / (ms * 1e-3) / 1e12, "unit": UNIT,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": steps,
             "ms_per_step": ms / steps}
 
 
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import __graft_entry__ as G
+    from paper_2305_11624_b200 import convbn as C
+    from paper_2305_11624_b200 import inputs as I
+    from paper_2305_11624_b200.harness import Block
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        G.build()
+    if world > 1:
+        dist.barrier()
+    C.lib()
+    ctx = Ctx()
+    ctx.args, ctx.torch, ctx.C, ctx.I, ctx.Block, ctx.dist = args, torch, C, I, Block, dist
+    ctx.dev, ctx.rank, ctx.world = dev, rank, world
+    ctx.peaks, ctx.peak_src = load_peaks()
+
+    workloads = [args.workload] if args.workload is not None else [0, 1, 2, 3, 4]
+    per_config = [bench_config(ctx, wl) for wl in workloads]
+    headline = [c for wl, c in zip(workloads, per_config) if wl in DENSE] or per_config
+    raw = [c.pop("_raw") for c in per_config]
+    hraw = [r for wl, r in zip(workloads, raw) if wl in DENSE] or raw
+    ms_total = sum(r["ms"] for r in hraw)                       # K steps of every headline configuration
+    flops_total = sum(r["flops"] for r in hraw)
+    value = whole_job_value(flops_total, args.steps, ms_total, world)
+    # the dominant kernel of the headline configurations: the one with the largest total time
+    roofs = [c["roofline"] for c in headline if c.get("roofline")]
+    roofline = max(roofs, key=lambda r: r["total_ms"]) if roofs else None
+    e2e = None
+    es = [c["e2e"] for c in headline if c.get("e2e")]
+    if es:
+        e2e_ms = sum(e["ms_per_step"] for e in es)
+        e2e = {"value": world * flops_total / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": sum(e["h2d_bytes_per_step"] for e in es),
+               "d2h_bytes_per_step": sum(e["d2h_bytes_per_step"] for e in es),
+               "ms_per_step": e2e_ms, "steps": es[0]["steps"],
+               "note": "convbn_tune_step_host per layer: pinned host inputs up, every output down, inside the timed region"}
+    cpu = None
+    cs = [c["cpu_baseline"] for c in headline if c.get("cpu_baseline")]
+    if cs:
+        secs, fl = sum(c["seconds"] for c in cs), sum(c["flops"] for c in cs)
+        cpu = {"value": fl / secs / 1e12, "unit": UNIT, "cores": cs[0]["cores"], "kind": "oracle",
+               "sample": "one full step of every headline configuration of the fp64 oracle as it stands, %.1f s" % secs}
+    if rank == 0:
+        names = [WORKLOAD_NAMES[w] for w in workloads]
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16" if any(w != 0 for w in workloads) else "f32", "data": "synthetic",
+                "config": {"workload": "; ".join(names),
+                           "value_over": "configs %s (dense bf16): total FLOPs / total time of one step of each"
+                                         % ", ".join(str(w) for w in workloads if w in DENSE or len(workloads) == 1),
+                           "l2": "inputs larger than L2: per configuration, rotating buffer sets that together exceed "
+                                 "twice the L2 (see per_config[].l2); warm numbers beside them",
+                           "flops_per_step": flops_total, "parallelism": "replicas x%d" % world,
+                           "launch": headline[0]["launch"]},
+                "clocks": merge_clocks([c["clocks"] for c in per_config]), "e2e": e2e,
+                "gpu_launches": sum(r["gpu_launches"] for r in raw),
+                "roofline": roofline, "cpu_baseline": cpu, "per_config": per_config}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=1, choices=sorted(WORKLOAD_NAMES))
-    ap.add_argument("--buffer-sets", type=int, default=2)
+    ap.add_argument("--workload", type=int, default=None, choices=sorted(WORKLOAD_NAMES),
+                    help="one configuration only (default: all five)")
+    ap.add_argument("--buffer-sets", type=int, default=0, help="rotating buffer sets (0: enough to exceed twice the L2)")
     ap.add_argument("--e2e-steps", type=int, default=5)
-    ap.add_argument("--ref-batch", type=int, default=4, help="samples per step of the reference arm")
+    ap.add_argument("--ref-batch", type=int, default=2, help="samples per step of the reference arm")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-modes", action="store_true", help="skip the Tune / Eval / Deploy comparison")
     ap.add_argument("--no-graph", action="store_true", help="time eager library calls instead of graph replays")
@@ -494,6 +678,8 @@ def main():
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
     else:
         run_ours(args)
 

@@ -95,7 +95,9 @@ int convbn_out_shape(const convbn_desc *desc, int *h_out, int *w_out);
  * Returns 0 for an invalid descriptor. */
 size_t convbn_saved_bytes(const convbn_desc *desc, int mode);
 
-/* Scratch bytes a call of `phase` (convbn_phase) needs.  0 for an invalid descriptor/phase. */
+/* Scratch bytes a call of `phase` (convbn_phase) needs.  0 for an invalid descriptor/phase.
+ * The split of the work over the SMs enters the size, so query it with the device that will run the
+ * call current (with no device present the size for a 148-SM part is returned). */
 size_t convbn_workspace_bytes(const convbn_desc *desc, int phase);
 
 /* ---- Tune mode (Sec. 3.4; Table 2, Tune row) --------------------------------------------- */

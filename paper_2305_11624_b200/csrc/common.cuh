@@ -64,10 +64,21 @@ cudaError_t read_and_clear_error_word(int *host_value); // synchronous
 // running: their set-up (barriers, tensor memory, descriptor prefetch) then overlaps its tail.  They
 // call pdl_wait() before their first access to global memory, which returns only once every earlier
 // kernel has completed and flushed; launched the plain way, pdl_wait() returns at once.
+// Invariant for kernels that own tensor memory: pdl_launch_dependents() comes only after the CTA's
+// tcgen05.alloc has completed (after the block barrier that follows it).  A dependent CTA that became
+// resident on the same SM earlier could take the columns first and then sit in its pdl_wait() for this
+// grid, while this CTA's allocation blocks behind it.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-bool pdl_enabled();   // false when CONVBN_NO_PDL=1
+// ---- per-device facts ------------------------------------------------------------------------------
+// Function attributes, the SM count and symbol addresses belong to a device, not to the process, so
+// every cache below is keyed by the ordinal of the CURRENT device.
+constexpr int kMaxDevices = 64;
+int current_device_slot();      // ordinal of the current device in [0, kMaxDevices), 0 when none can be queried
+int device_sm_count();          // SMs of the current device; 148 (B200) when no device is present (host-only sizing)
+struct PerDevice { bool done[kMaxDevices] = {}; };
+
 
 template <class... KArgs, class... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
@@ -79,20 +90,30 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = pdl_enabled() ? 1 : 0;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
-// Ask for the largest shared-memory carve-out for a kernel, once.  The tensor-core kernels need it;
-// the small kernels launched between them ask for the same split so that the SMs are not
+// Ask for the largest shared-memory carve-out for a kernel, once per device.  The tensor-core kernels
+// need it; the small kernels launched between them ask for the same split so that the SMs are not
 // re-partitioned (which drains them) at every kernel boundary of a training step.
 template <class K>
-inline void prefer_max_shared_once(K kernel, bool *done) {
-    if (*done) return;
+inline void prefer_max_shared_once(K kernel, PerDevice *flag) {
+    bool &done = flag->done[current_device_slot()];
+    if (done) return;
     cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    *done = true;
+    done = true;
+}
+// Raise a kernel's dynamic shared-memory limit, once per device.
+template <class K>
+inline cudaError_t max_dynamic_smem_once(K kernel, int bytes, PerDevice *flag) {
+    bool &done = flag->done[current_device_slot()];
+    if (done) return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) done = true;
+    return e;
 }
 
 static inline int ceil_div_i(long long a, long long b) { return (int)((a + b - 1) / b); }

@@ -98,17 +98,12 @@ int check_pair(const convbn_desc *d) {
     return CONVBN_EUNSUPPORTED;
 }
 
-bool force_direct() {
-    static const bool v = [] { const char *e = getenv("CONVBN_FORCE_DIRECT"); return e && e[0] == '1'; }();
-    return v;
-}
-
 bool stem_path(const convbn_desc *d, const Problem &pb) {
-    return !force_direct() && d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && stem_eligible(pb);
+    return d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && stem_eligible(pb);
 }
 
 bool grouped_path(const convbn_desc *d, const Problem &pb) {
-    return !force_direct() && d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && grouped_bd_eligible(pb);
+    return d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && grouped_bd_eligible(pb);
 }
 
 // Workspace carve-up of one phase.  Offsets are multiples of 256 bytes.
@@ -136,21 +131,21 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
     size_t wbytes = (size_t)pb.c_out * pb.kdim * elem_size(d->dtype);
     // the sub-pixel backward-data path of small-C_in layers keeps its (zero-padded) weight matrix there
-    if (!force_direct() && d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && subpixel_weight_bytes(pb) > wbytes)
+    if (d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && subpixel_weight_bytes(pb) > wbytes)
         wbytes = subpixel_weight_bytes(pb);
     const size_t wrows = (size_t)pb.c_out * pb.kdim;
     pl.splits = direct_wgrad_splits(pb);
     pl.bsplits = channel_sum_splits(pb);
     pl.bn_splits = pl.bsplits;                      // pixel slices of the Eval-mode BatchNorm backward
-    pl.umma_wgrad = !force_direct() && d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC &&
+    pl.umma_wgrad = d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC &&
                     umma_wgrad_eligible(pb);
     size_t part_bytes = wrows * pl.splits * sizeof(float), dot_bytes = 0;
-    pl.dw_wgrad = !force_direct() && d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && dw_eligible(pb) &&
+    pl.dw_wgrad = d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && dw_eligible(pb) &&
                   dw_wgrad_supported(pb);
     if (pl.dw_wgrad) {
         pl.splits = dw_wgrad_splits(pb);
         part_bytes = wrows * pl.splits * sizeof(float);
-        pl.dw_tma_wgrad = dw_tma_eligible(pb) && getenv("CONVBN_NO_DW_TMA") == nullptr;
+        pl.dw_tma_wgrad = dw_tma_eligible(pb);
         if (pl.dw_tma_wgrad && dw_tma_wgrad_partial_bytes(pb) > part_bytes) part_bytes = dw_tma_wgrad_partial_bytes(pb);
     }
     pl.stem = stem_path(d, pb);
@@ -275,12 +270,12 @@ int check_ws(const Plan &pl, const void *ws, size_t ws_bytes) {
 inline char *at(void *ws, size_t off) { return (char *)ws + off; }
 
 bool dw_path(const convbn_desc *d, const Problem &pb) {
-    return !force_direct() && d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && dw_eligible(pb);
+    return d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && dw_eligible(pb);
 }
 
 // Tensor-core eligibility of the forward convolution and its GEMM shape.
 bool umma_fwd_shape(const convbn_desc *d, const Problem &pb, UmmaConvShape *s) {
-    if (force_direct() || d->dtype != CONVBN_BF16 || d->layout != CONVBN_NHWC || pb.groups != 1) return false;
+    if (d->dtype != CONVBN_BF16 || d->layout != CONVBN_NHWC || pb.groups != 1) return false;
     *s = UmmaConvShape{pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.c_out, pb.kh, pb.kw,
                        -pb.pad_h, -pb.pad_w, pb.stride_h, pb.stride_w, pb.dil_h, pb.dil_w};
     return umma_conv_eligible(*s);
@@ -288,7 +283,7 @@ bool umma_fwd_shape(const convbn_desc *d, const Problem &pb, UmmaConvShape *s) {
 
 // Backward data as a stride-1 convolution of dZ with the rotated, channel-swapped omega'.
 bool umma_dgrad_shape(const convbn_desc *d, const Problem &pb, UmmaConvShape *s) {
-    if (force_direct() || d->dtype != CONVBN_BF16 || d->layout != CONVBN_NHWC || pb.groups != 1) return false;
+    if (d->dtype != CONVBN_BF16 || d->layout != CONVBN_NHWC || pb.groups != 1) return false;
     if (pb.stride_h != 1 || pb.stride_w != 1) return false;
     *s = UmmaConvShape{pb.n, pb.h_out, pb.w_out, pb.c_out, pb.h_in, pb.w_in, pb.c_in, pb.kh, pb.kw,
                        pb.pad_h - (pb.kh - 1) * pb.dil_h, pb.pad_w - (pb.kw - 1) * pb.dil_w, 1, 1, pb.dil_h,
@@ -310,7 +305,7 @@ ClassTaps class_taps(int a, int pad, int k, int stride) {
 }
 
 bool strided_dgrad_ok(const convbn_desc *d, const Problem &pb) {
-    if (force_direct() || d->dtype != CONVBN_BF16 || d->layout != CONVBN_NHWC || pb.groups != 1) return false;
+    if (d->dtype != CONVBN_BF16 || d->layout != CONVBN_NHWC || pb.groups != 1) return false;
     if (pb.stride_h == 1 && pb.stride_w == 1) return false;
     if (pb.dil_h != 1 || pb.dil_w != 1 || pb.stride_h > 4 || pb.stride_w > 4) return false;
     return pb.c_out % 64 == 0 && pb.c_in % 8 == 0 && pb.c_in >= 64 && pb.c_in <= 4096 &&
@@ -470,7 +465,7 @@ int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, cons
             mp.h_in = pb.h_out; mp.w_in = pb.w_out; mp.h_out = pb.h_in; mp.w_out = pb.w_in;
             mp.pad_h = (pb.kh - 1) * pb.dil_h - pb.pad_h; mp.pad_w = (pb.kw - 1) * pb.dil_w - pb.pad_w;
             mp.p = pb.pin; mp.pin = pb.p;
-            if (dw_tma_eligible(mp) && getenv("CONVBN_NO_DW_TMA") == nullptr) {
+            if (dw_tma_eligible(mp)) {
                 // the streaming kernel scales and reverses the taps itself
                 LAUNCH("dw_dgrad", launch_dw_tma(mp, dz, w, nullptr, dx, st, nullptr, scale, true));
             } else {
@@ -622,7 +617,7 @@ int convbn_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const
         }
         return CONVBN_OK;
     }
-    if (dw_path(desc, pb) && dw_tma_eligible(pb) && getenv("CONVBN_NO_DW_TMA") == nullptr) {
+    if (dw_path(desc, pb) && dw_tma_eligible(pb)) {
         // depthwise 3x3: the fold is formed inside the streaming kernel from the raw weights
         const BnFold fold{gamma, beta, run_mean, run_var, b, pb.eps, vec3};
         LAUNCH("dw_fwd", launch_dw_tma(pb, x, w, nullptr, z, st, &fold));

@@ -129,7 +129,7 @@ static cudaError_t dispatch(int dtype, int layout, F f) {
 
 static int grid_for(long long total) {
     long long b = (total + 255) / 256;
-    const long long cap = 148LL * 64;
+    const long long cap = (long long)device_sm_count() * 64;
     return (int)(b < 1 ? 1 : (b > cap ? cap : b));
 }
 
@@ -155,7 +155,7 @@ cudaError_t launch_direct_dgrad(const Problem &pb, int dtype, int layout, const 
 
 int direct_wgrad_splits(const Problem &pb) {
     const long long rows = (long long)pb.c_out * pb.kdim;
-    long long want = (148LL * 2048 * 2 + rows - 1) / rows;   // about two full waves of threads
+    long long want = ((long long)device_sm_count() * 2048 * 2 + rows - 1) / rows;   // about two full waves of threads
     long long cap = pb.p / 32;                                // at least 32 pixels per slice
     if (cap < 1) cap = 1;
     if (want > cap) want = cap;

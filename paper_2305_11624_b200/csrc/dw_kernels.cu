@@ -524,17 +524,12 @@ DwShape dw_shape(const Problem &pb) {
 
 int dw_grid(long long total) {
     long long b = (total + 255) / 256;
-    const long long cap = 148LL * 32;
+    const long long cap = (long long)device_sm_count() * 32;
     return (int)(b < 1 ? 1 : (b > cap ? cap : b));
 }
 
 template <class K>
-cudaError_t set_smem_once(K kernel, bool *done) {
-    if (*done) return cudaSuccess;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-    if (e == cudaSuccess) *done = true;
-    return e;
-}
+cudaError_t set_smem_once(K kernel, PerDevice *done) { return max_dynamic_smem_once(kernel, 96 * 1024, done); }
 
 }  // namespace
 
@@ -550,10 +545,9 @@ cudaError_t launch_dw_fwd(const Problem &pb, const void *x, const void *w, const
     const size_t smem = (size_t)pb.kh * pb.kw * pb.c_in * sizeof(float);
     const long long total = (long long)pb.n * pb.h_out * ((pb.w_out + 3) / 4) * (pb.c_in / 8);
     const bool unit_w = pb.stride_w == 1 && pb.dil_w == 1;
-    static bool a3 = false, a5 = false, a0 = false;
+    static PerDevice a3, a5, a0;
     cudaError_t e;
-    static const bool no_tma = getenv("CONVBN_NO_DW_TMA") != nullptr;
-    if (!no_tma && dw_tma_eligible(pb)) return launch_dw_tma(pb, x, w, bias, z, st);
+    if (dw_tma_eligible(pb)) return launch_dw_tma(pb, x, w, bias, z, st);
     const bool unit = unit_w && pb.stride_h == 1 && pb.dil_h == 1 && pb.kh == pb.kw && pb.pad_h >= 0 && pb.pad_w >= 0;
     if (unit && (pb.kh == 3 || pb.kh == 5)) {
         // rows per thread: as tall as still leaves every SM a few blocks
@@ -561,14 +555,14 @@ cudaError_t launch_dw_fwd(const Problem &pb, const void *x, const void *w, const
         auto threads = [&](int t) {
             return (long long)pb.n * ((pb.h_out + t - 1) / t) * ((pb.w_out + 1) / 2) * (pb.c_in / 8);
         };
-        while (th > 1 && threads(th) < 148LL * 256 * 4) th /= 2;
-        static bool s3 = false, s5 = false;
+        while (th > 1 && threads(th) < (long long)device_sm_count() * 256 * 4) th /= 2;
+        static PerDevice s3, s5;
         if (pb.kh == 3) {
             auto threads4 = [&](int t) {
                 return (long long)pb.n * ((pb.h_out + t - 1) / t) * ((pb.w_out + 1) / 2) * (pb.c_in / 4);
             };
             th = 16;
-            while (th > 1 && threads4(th) < 148LL * 256 * 4) th /= 2;
+            while (th > 1 && threads4(th) < (long long)device_sm_count() * 256 * 4) th /= 2;
             if ((e = set_smem_once(dw_stream4_kernel<2, 3, 3>, &s3)) != cudaSuccess) return e;
             dw_stream4_kernel<2, 3, 3><<<dw_grid(threads4(th)), 256, smem, st>>>(s, (const uint2 *)x, (const __nv_bfloat16 *)w,
                                                                                 bias, (uint2 *)z, th);
@@ -596,7 +590,7 @@ cudaError_t launch_dw_fwd(const Problem &pb, const void *x, const void *w, const
 cudaError_t launch_dw_dgrad(const Problem &pb, const void *dz, const void *w, void *dx, cudaStream_t st) {
     const DwShape s = dw_shape(pb);
     const size_t smem = (size_t)pb.kh * pb.kw * pb.c_in * sizeof(float);
-    static bool attr = false;
+    static PerDevice attr;
     cudaError_t e = set_smem_once(dw_dgrad_kernel, &attr);
     if (e != cudaSuccess) return e;
     const long long total = pb.pin * (pb.c_in / 8);
@@ -605,7 +599,7 @@ cudaError_t launch_dw_dgrad(const Problem &pb, const void *dz, const void *w, vo
 }
 
 int dw_wgrad_splits(const Problem &pb) {
-    long long want = 148 * 8;
+    long long want = (long long)device_sm_count() * 8;
     const long long cap = (pb.p + 63) / 64;
     if (want > cap) want = cap;
     if (want < 1) want = 1;

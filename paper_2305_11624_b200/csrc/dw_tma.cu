@@ -527,12 +527,8 @@ cudaError_t launch_dw_tma(const Problem &pb, const void *x, const void *w, const
     if (!dw_tma_map(&tx, x, pb.n, pb.h_in, pb.w_in, pb.c_in, g.cols_t * TW + KW - 1)) return cudaErrorInvalidValue;
     int *err = nullptr;
     if ((e = error_word_address(&err)) != cudaSuccess) return e;
-    static bool attr = false;
-    if (!attr) {
-        e = cudaFuncSetAttribute(dw_tma_kernel<TW, KH, KW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024);
-        if (e != cudaSuccess) return e;
-        attr = true;
-    }
+    static PerDevice attr;
+    if ((e = max_dynamic_smem_once(dw_tma_kernel<TW, KH, KW>, 110 * 1024, &attr)) != cudaSuccess) return e;
     const BnFold none{nullptr, nullptr, nullptr, nullptr, nullptr, 0.f, nullptr};
     dw_tma_kernel<TW, KH, KW><<<grid, (g.consumer_warps + 1) * 32, dw_tma_smem(g), st>>>(
         tx, g, (const __nv_bfloat16 *)w, bias, fold ? *fold : none, scale, reverse_taps ? 1 : 0, (uint2 *)z, err);
@@ -559,12 +555,8 @@ cudaError_t launch_dw_tma_wgrad(const Problem &pb, const void *dz, const void *x
     if (!dw_tma_map(&tdz, dz, pb.n, pb.h_out, pb.w_out, pb.c_in, g.cols_t * TW)) return cudaErrorInvalidValue;
     int *err = nullptr;
     if ((e = error_word_address(&err)) != cudaSuccess) return e;
-    static bool attr = false;
-    if (!attr) {
-        e = cudaFuncSetAttribute(dw_tma_wgrad_kernel<TW, KH, KW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024);
-        if (e != cudaSuccess) return e;
-        attr = true;
-    }
+    static PerDevice attr;
+    if ((e = max_dynamic_smem_once(dw_tma_wgrad_kernel<TW, KH, KW>, 110 * 1024, &attr)) != cudaSuccess) return e;
     dw_tma_wgrad_kernel<TW, KH, KW><<<grid, (g.consumer_warps + 1) * 32, dw_tma_smem(g), st>>>(tx, tdz, g, part, err);
     *nparts = (int)grid;
     return cudaGetLastError();

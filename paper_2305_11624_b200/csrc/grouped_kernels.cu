@@ -38,7 +38,7 @@ cudaError_t launch_expand_blockdiag(const Problem &pb, const void *w, const floa
                                     bool transpose_flip, cudaStream_t st) {
     const long long total = (long long)pb.c_out * pb.kh * pb.kw * 64;
     long long blocks = (total + 255) / 256;
-    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (blocks > device_sm_count() * 8) blocks = device_sm_count() * 8;
     expand_blockdiag_kernel<<<(int)blocks, 256, 0, st>>>(pb.c_out, pb.kh * pb.kw, pb.cg, (const __nv_bfloat16 *)w,
                                                          s_vec, (__nv_bfloat16 *)wbd, transpose_flip ? 1 : 0);
     return cudaGetLastError();

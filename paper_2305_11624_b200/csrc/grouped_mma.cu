@@ -353,11 +353,7 @@ GroupedPlan plan_grouped8(int n, int h_in, int w_in, int c, int ho, int wo, int 
     (void)h_in; (void)w_in;
     const int wt = wo + kw - 1;
     if (wt > 256 || wt < 8 || kh * kw > 2 * kGMaxKSteps || c % 64) return pl;
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) {
-        int v = 0;
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) sms = v;
-    }
+    const int sms = device_sm_count();
     // The compute warps of one block (8, two per scheduler) cannot hide the ldmatrix -> MMA latency on
     // their own, so the bands are kept small enough for two or three blocks per SM.  Estimated time:
     // rounds over the resident blocks x input pixels of a band, derated for the SM being shared.
@@ -403,8 +399,6 @@ GroupedPlan plan_grouped8(int n, int h_in, int w_in, int c, int ho, int wo, int 
 }  // namespace
 
 bool grouped8_eligible(const Problem &pb) {
-    static const bool off = getenv("CONVBN_NO_GROUPED_MMA") != nullptr;
-    if (off) return false;
     return pb.groups > 1 && pb.cg == 8 && pb.cog == 8 && pb.c_in % 64 == 0 && pb.stride_h == 1 && pb.stride_w == 1 &&
            pb.dil_h == 1 && pb.dil_w == 1 && pb.kh * pb.kw <= 2 * kGMaxKSteps && pb.w_out + pb.kw - 1 <= 256 &&
            pb.w_in + pb.kw - 1 <= 256 && pb.pad_h <= 128 && pb.pad_w <= 128 && pb.p < (1LL << 30) &&
@@ -427,12 +421,8 @@ static cudaError_t launch_grouped8(int n, int ha, int wa, int c, int ho, int wo,
     int *err = nullptr;
     cudaError_t e = error_word_address(&err);
     if (e != cudaSuccess) return e;
-    static bool attr = false;
-    if (!attr) {
-        e = cudaFuncSetAttribute(grouped8_conv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-        if (e != cudaSuccess) return e;
-        attr = true;
-    }
+    static PerDevice attr;
+    if ((e = max_dynamic_smem_once(grouped8_conv_kernel, 220 * 1024, &attr)) != cudaSuccess) return e;
     grouped8_conv_kernel<<<pl.grid, kGThreads, pl.smem, st>>>(ta, pl.g, (const __nv_bfloat16 *)w, bias,
                                                              (__nv_bfloat16 *)out, err);
     return cudaGetLastError();
@@ -463,11 +453,7 @@ static GroupedPlan plan_grouped8_wgrad(const Problem &pb, int *slots) {
     GroupedPlan pl = plan_grouped8(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.kh, pb.kw, -pb.pad_h, -pb.pad_w,
                                    true);
     if (!pl.ok) return pl;
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) {
-        int v = 0;
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) sms = v;
-    }
+    const int sms = device_sm_count();
     const int chunks = pb.c_in / 64;
     long long per_chunk = (long long)sms * pl.bps / chunks;
     const long long bands = (long long)pb.n * pl.g.tiles_h;
@@ -509,12 +495,8 @@ cudaError_t launch_grouped8_wgrad(const Problem &pb, const void *dz, const void 
     int *err = nullptr;
     cudaError_t e = error_word_address(&err);
     if (e != cudaSuccess) return e;
-    static bool attr = false;
-    if (!attr) {
-        e = cudaFuncSetAttribute(grouped8_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-        if (e != cudaSuccess) return e;
-        attr = true;
-    }
+    static PerDevice attr;
+    if ((e = max_dynamic_smem_once(grouped8_wgrad_kernel, 220 * 1024, &attr)) != cudaSuccess) return e;
     grouped8_wgrad_kernel<<<pl.grid, kGThreads, pl.smem, st>>>(tx, tdz, pl.g, pl.dz_off, slots, part, bsum, err);
     return cudaGetLastError();
 }

@@ -138,7 +138,8 @@ size_t stem_weight_bytes(const Problem &pb);                 // [C_out][krows][6
 cudaError_t launch_stem_pack(const Problem &pb, const void *x, void *x_packed, cudaStream_t st);
 cudaError_t launch_stem_expand_weights(const Problem &pb, const void *w, const float *s_vec, void *wst,
                                        cudaStream_t st);
-// Backward data of a stem layer (fp32 FMA kernel; scale folded into the weights it stages).
+// Backward data of a stem layer on warp-level MMAs (m16n8k16, fp32 accumulation; the scale is folded into
+// the weight fragments it stages).  Used for the narrow-input shapes the sub-pixel GEMM does not take.
 bool stem_dgrad_eligible(const Problem &pb);
 cudaError_t launch_stem_dgrad(const Problem &pb, const void *dz, const void *w, const float *s_vec, void *dx,
                               cudaStream_t st);

@@ -8,9 +8,23 @@ namespace convbn {
 
 __device__ int g_error_word = 0;
 
-bool pdl_enabled() {
-    static const bool v = [] { const char *e = getenv("CONVBN_NO_PDL"); return !(e && e[0] == '1'); }();
-    return v;
+int current_device_slot() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    return dev;
+}
+
+int device_sm_count() {
+    static int cache[kMaxDevices] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 148; }
+    if (dev < 0 || dev >= kMaxDevices) dev = 0;
+    if (!cache[dev]) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
+        cache[dev] = v;
+    }
+    return cache[dev];
 }
 
 // The address is looked up once per device and cached, so launches make no runtime query
@@ -166,7 +180,7 @@ __global__ void __launch_bounds__(256) reparam_dgrad_class_kernel(int c_out, int
 cudaError_t launch_reparam_dgrad_class(const Problem &pb, const void *w, const float *s_vec, void *w_t, int th,
                                        int tw, int r_max, int q_max, int step_h, int step_w, cudaStream_t st) {
     dim3 grid((pb.c_in + 31) / 32, (pb.c_out + 31) / 32, th * tw);
-    static bool carve = false;
+    static PerDevice carve;
     prefer_max_shared_once(reparam_dgrad_class_kernel, &carve);
     return launch_pdl(reparam_dgrad_class_kernel, grid, dim3(256), 0, st, pb.c_out, pb.c_in, pb.kw, tw, r_max, q_max,
                       step_h, step_w, th * tw, (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t, pb.kh * pb.kw);
@@ -202,7 +216,7 @@ __global__ void __launch_bounds__(256) reparam_dgrad_classes_kernel(int c_out, i
 cudaError_t launch_reparam_dgrad_classes(const Problem &pb, const void *w, const float *s_vec, void *w_t,
                                          const ClassTapTable &where, cudaStream_t st) {
     dim3 grid((pb.c_in + 31) / 32, (pb.c_out + 31) / 32, pb.kh * pb.kw);
-    static bool carve = false;
+    static PerDevice carve;
     prefer_max_shared_once(reparam_dgrad_classes_kernel, &carve);
     return launch_pdl(reparam_dgrad_classes_kernel, grid, dim3(256), 0, st, pb.c_out, pb.c_in, where,
                       (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t, pb.kh * pb.kw);
@@ -211,7 +225,7 @@ cudaError_t launch_reparam_dgrad_classes(const Problem &pb, const void *w, const
 cudaError_t launch_reparam_dgrad(const Problem &pb, const void *w, const float *s_vec, void *w_t,
                                  cudaStream_t st) {
     dim3 grid((pb.c_in + 31) / 32, (pb.c_out + 31) / 32, pb.kh * pb.kw);
-    static bool carve = false;
+    static PerDevice carve;
     prefer_max_shared_once(reparam_dgrad_kernel, &carve);
     return launch_pdl(reparam_dgrad_kernel, grid, dim3(256), 0, st, pb.c_out, pb.c_in, pb.kh * pb.kw,
                       (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t);
@@ -473,13 +487,13 @@ cudaError_t launch_bn_eval_fwd(const Problem &pb, int dtype, int layout, const v
         const int v = pb.c_out / 8, block = (256 / v) * v;
         const long long vecs = pb.p * v;
         long long nb = (vecs + block - 1) / block;
-        if (nb > 148 * 16) nb = 148 * 16;
+        if (nb > device_sm_count() * 16) nb = device_sm_count() * 16;
         bn_eval_fwd_nhwc8_kernel<<<(int)nb, block, 0, st>>>(pb.c_out, vecs, (const uint4 *)y, vec3, (uint4 *)z);
         return cudaGetLastError();
     }
     const long long total = pb.p * pb.c_out, hw = (long long)pb.h_out * pb.w_out;
     long long blocks = (total + 255) / 256;
-    if (blocks > 148 * 32) blocks = 148 * 32;
+    if (blocks > device_sm_count() * 32) blocks = device_sm_count() * 32;
     if (dtype == CONVBN_F32 && layout == CONVBN_NCHW)
         bn_eval_fwd_kernel<float, NCHW><<<(int)blocks, 256, 0, st>>>(pb.c_out, hw, total, (const float *)y, vec3, (float *)z);
     else if (dtype == CONVBN_BF16 && layout == CONVBN_NHWC)

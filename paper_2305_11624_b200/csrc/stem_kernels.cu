@@ -126,7 +126,7 @@ cudaError_t launch_stem_pack(const Problem &pb, const void *x, void *xp, cudaStr
     stem_geometry(pb, &hp, &wp);
     const long long total = (long long)pb.n * hp * wp * (stem_s2d(pb) ? 2 : 1);
     long long blocks = (total + 255) / 256;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks > device_sm_count() * 16) blocks = device_sm_count() * 16;
     if (stem_s2d(pb)) {
         stem_pack_s2d_kernel<<<(int)blocks, 256, 0, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.pad_h, pb.pad_w, hp, wp,
                                                           stem_ones_in_pack(pb) ? 1 : 0, (const __nv_bfloat16 *)x,
@@ -337,8 +337,8 @@ bool stem_dgrad_eligible(const Problem &pb) {
 cudaError_t launch_stem_dgrad(const Problem &pb, const void *dz, const void *w, const float *s_vec, void *dx,
                               cudaStream_t st) {
     const size_t smem = (size_t)pb.kh * pb.kw * (pb.c_out / 64) * 1024 + 8192;   // fragments + 1 KB per warp
-    static bool attr = false;
-    if (!attr) {
+    static PerDevice attr;
+    if (!attr.done[current_device_slot()]) {
         cudaError_t e = cudaFuncSetAttribute(stem_dgrad_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(stem_dgrad_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
@@ -347,7 +347,7 @@ cudaError_t launch_stem_dgrad(const Problem &pb, const void *dz, const void *w, 
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(stem_dgrad_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
         if (e != cudaSuccess) return e;
-        attr = true;
+        attr.done[current_device_slot()] = true;
     }
     const int nu = (pb.kw + pb.stride_w - 1) / pb.stride_w;    // taps per kernel row in the fullest class
     const void *fn = nu <= 1   ? (const void *)stem_dgrad_kernel<1>

@@ -120,7 +120,6 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
     // the tensor maps are kernel parameters, not data of an earlier kernel: fetch them before the wait
     if (threadIdx.x == 0) { prefetch_tensormap(&tm_act); prefetch_tensormap(&tm_w); prefetch_tensormap(&tm_out); }
     pdl_wait();
-    pdl_launch_dependents();
     if (fold) {
         // On-the-fly reparameterisation (Sec. 3.3 / 3.4): s = gamma / sqrt(var + eps), b' = (b - mu) s + beta.
         // s multiplies the fp32 accumulator (the associative law of Sec. 3.2.2), so omega is used unrounded.
@@ -140,6 +139,7 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    pdl_launch_dependents();       // only now: this CTA owns its tensor-memory columns
     const uint32_t tmem_base = ctl->tmem_base;
 
     if (warp == 0) {
@@ -447,18 +447,7 @@ bool umma_conv_eligible(const UmmaConvShape &s) {
     return true;
 }
 
-static int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
-            n = v;
-        else
-            n = 148;
-    }
-    return n;
-}
+static int sm_count() { return device_sm_count(); }
 
 template <int BN>
 static cudaError_t launch_bn(const CUtensorMap &ta, const CUtensorMap &tw, const CUtensorMap &tout, ConvGemm g,
@@ -483,14 +472,9 @@ static cudaError_t launch_bn(const CUtensorMap &ta, const CUtensorMap &tw, const
     if (stages > kMaxStages) stages = kMaxStages;
     g.stages = stages;
     const size_t smem = stages * stage + fixed;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(umma_conv_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             224 * 1024);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
-    static bool carve = false;
+    static PerDevice attr_done;
+    if (cudaError_t e = max_dynamic_smem_once(umma_conv_kernel<BN>, 224 * 1024, &attr_done); e != cudaSuccess) return e;
+    static PerDevice carve;
     prefer_max_shared_once(umma_conv_kernel<BN>, &carve);
     const unsigned grid = (unsigned)grid_l;
     return launch_pdl(umma_conv_kernel<BN>, dim3(grid), dim3(kConvThreads), smem, st, ta, tw, tout, g, bias, err);

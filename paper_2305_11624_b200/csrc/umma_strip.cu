@@ -85,7 +85,6 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
     // the tensor maps are kernel parameters, not data of an earlier kernel: fetch them before the wait
     if (threadIdx.x == 0) { prefetch_tensormap(&tm_act); prefetch_tensormap(&tm_w); }
     pdl_wait();
-    pdl_launch_dependents();
     if (fold) {
         for (int c = threadIdx.x; c < g.cn; c += kSThreads) {
             const float r = 1.0f / sqrtf(g.fold.var[c] + g.fold.eps);
@@ -103,6 +102,7 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    pdl_launch_dependents();       // only now: this CTA owns its tensor-memory columns
     const uint32_t tmem_base = ctl->tmem_base;
 
     // tile t -> (image, tile row, tile column, n-tile); n-tiles of one patch sit on neighbouring CTAs
@@ -319,15 +319,7 @@ namespace {
 
 struct StripPlan { bool ok = false; int bn = 64, R = 0, CW = 0, Wt = 0, nmb = 0, nacc = 2, tiles_w = 1 << 20; uint32_t strip_bytes = 0; size_t smem = 0; };
 
-int strip_sm_count() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0, v = 0;
-        n = (cudaGetDevice(&dev) == cudaSuccess &&
-             cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) ? v : 148;
-    }
-    return n;
-}
+int strip_sm_count() { return device_sm_count(); }
 
 StripPlan plan_strip(const UmmaConvShape &s) {
     StripPlan best;
@@ -408,14 +400,9 @@ bool make_tmap_nhwc_box(CUtensorMap *tm, const void *base, int n, int h, int w, 
 template <int BN>
 cudaError_t launch_strip(const CUtensorMap &ta, const CUtensorMap &tw, const StripGemm &g, size_t smem,
                          const float *bias, int *err, cudaStream_t st) {
-    static bool attr = false;
-    if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(umma_strip_conv_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             226 * 1024);
-        if (e != cudaSuccess) return e;
-        attr = true;
-    }
-    static bool carve = false;
+    static PerDevice attr;
+    if (cudaError_t e = max_dynamic_smem_once(umma_strip_conv_kernel<BN>, 226 * 1024, &attr); e != cudaSuccess) return e;
+    static PerDevice carve;
     prefer_max_shared_once(umma_strip_conv_kernel<BN>, &carve);
     const long long total = (long long)g.n * g.tiles_h * g.tiles_w * (g.cn / BN);
     const unsigned grid = (unsigned)(total < strip_sm_count() ? total : strip_sm_count());
@@ -425,8 +412,7 @@ cudaError_t launch_strip(const CUtensorMap &ta, const CUtensorMap &tw, const Str
 }  // namespace
 
 bool umma_strip_eligible(const UmmaConvShape &s) {
-    static const bool off = [] { const char *e = getenv("CONVBN_NO_STRIP"); return e && e[0] == '1'; }();
-    return !off && plan_strip(s).ok;
+    return plan_strip(s).ok;
 }
 
 cudaError_t launch_umma_strip_conv(const UmmaConvShape &s, const void *act, const void *wmat, const float *bias,

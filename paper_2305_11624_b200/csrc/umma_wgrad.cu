@@ -84,7 +84,6 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
     // the tensor maps are kernel parameters, not data of an earlier kernel: fetch them before the wait
     if (threadIdx.x == 0) { prefetch_tensormap(&tm_x); prefetch_tensormap(&tm_dz); }
     pdl_wait();                 // global memory only after every earlier kernel has finished
-    pdl_launch_dependents();
     // counters of the epilogue kernel that runs after this one start from zero
     if (counters && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
         for (int i = threadIdx.x; i < ncounters; i += kWThreads) counters[i] = 0u;
@@ -100,6 +99,7 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    pdl_launch_dependents();       // only now: this CTA owns its tensor-memory columns
     const uint32_t tmem_base = ctl->tmem_base;
 
     if (warp == 0) {
@@ -250,7 +250,7 @@ UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
     // The slice count minimises  rounds over the resident slots x (pixels per slice + a fixed cost per
     // CTA, in pixels) + a small cost per slice for the epilogue that adds the slices up; a grid a few
     // CTAs larger than the slots would otherwise run a second, nearly empty round.
-    const long long slots = 148 * (bn == 256 ? 1 : 2), tiles = m_tiles * n_tiles;
+    const long long slots = (long long)device_sm_count() * (bn == 256 ? 1 : 2), tiles = m_tiles * n_tiles;
     const long long max_splits = (pb.p + 4 * kWP - 1) / (4 * kWP);     // at least 256 pixels per slice
     long long splits = 1;
     double best_cost = -1.0;
@@ -267,7 +267,7 @@ UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
     // k rows per epilogue block (the block's other lanes split the slices): very many slices -> 2 rows x 16
     // lanes; few slices or very many blocks -> 32 rows x 1 lane (every block pays a fence and an atomic)
     const long long blocks8 = (long long)(pb.c_out / 32) * ((pb.kdim + 7) / 8);
-    pl.kr = pl.splits > 192 ? 2 : ((pl.splits <= 8 || blocks8 > 1200) && blocks8 / 4 >= 148 ? 32 : 8);
+    pl.kr = pl.splits > 192 ? 2 : ((pl.splits <= 8 || blocks8 > 1200) && blocks8 / 4 >= device_sm_count() ? 32 : 8);
     pl.kt = (pb.kdim + pl.kr - 1) / pl.kr;   // epilogue blocks along k = rows of dotpart
     return pl;
 }
@@ -284,14 +284,9 @@ static cudaError_t launch_w(const CUtensorMap &tx, const CUtensorMap &tdz, Wgrad
     size_t smem = stages * stage + 1024 + sizeof(WgradSmemCtl);
     const size_t floor_smem = (size_t)(228 * 1024) / (512 / BN + 1) + 1024;
     if (smem < floor_smem) smem = floor_smem;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(umma_wgrad_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             210 * 1024);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
-    static bool carve = false;
+    static PerDevice attr_done;
+    if (cudaError_t e = max_dynamic_smem_once(umma_wgrad_kernel<BN>, 210 * 1024, &attr_done); e != cudaSuccess) return e;
+    static PerDevice carve;
     prefer_max_shared_once(umma_wgrad_kernel<BN>, &carve);
     dim3 grid((unsigned)((g.kdim / 64 + (g.no_ones ? 1 : 2)) / 2), (unsigned)((pb.c_out + BN - 1) / BN),
               (unsigned)pl.splits);
@@ -492,7 +487,7 @@ cudaError_t launch_wgrad_epilogue_fused(const Problem &pb, const UmmaWgradPlan &
                                         float *db, float *dgamma, float *dbeta, bool need_sums, cudaStream_t st) {
     const dim3 grid(pb.c_out / 32, pl.kt);
     const int ns = need_sums ? 1 : 0;
-    static bool carve_a = false, carve_b = false;
+    static PerDevice carve_a, carve_b;
     prefer_max_shared_once(wgrad_epilogue_fused_kernel<8, 4, 1>, &carve_a);
     prefer_max_shared_once(wgrad_epilogue_fused_kernel<2, 16, 1>, &carve_b);
     if (pl.kr == 32)                                  // 4 groups of 8 rows, 256 threads: several blocks per SM
@@ -514,7 +509,7 @@ UmmaWgradPlan stem_wgrad_plan(const Problem &pb) {
     const int bn = wgrad_bn(pb);
     const long long patches = (long long)pb.n * ((pb.h_out + 3) / 4) * ((pb.w_out + 15) / 16);
     const long long m_tiles = (stem_krows(pb) + (stem_ones_in_pack(pb) ? 1 : 2)) / 2, n_tiles = (pb.c_out + bn - 1) / bn;
-    long long splits = (148 + m_tiles * n_tiles - 1) / (m_tiles * n_tiles);
+    long long splits = (device_sm_count() + m_tiles * n_tiles - 1) / (m_tiles * n_tiles);
     if (splits > (patches + 3) / 4) splits = (patches + 3) / 4;
     if (splits < 1) splits = 1;
     const long long per = (patches + splits - 1) / splits;

@@ -21,7 +21,9 @@ def make_desc(spec: I.LayerSpec) -> C.Desc:
 class Block:
     """Buffers of one layer on one device plus the calls of each mode."""
 
-    def __init__(self, spec: I.LayerSpec, device="cuda:0", modes=("tune",)):
+    def __init__(self, spec: I.LayerSpec, device="cuda:0", modes=("tune",), allocate="all"):
+        """allocate="params" makes only the parameters and their gradients: activations, saved state and
+        scratch are then assigned by the caller (memory measurements that allocate them per call)."""
         self.spec = spec
         self.desc = make_desc(spec)
         self.device = torch.device(device)
@@ -33,13 +35,17 @@ class Block:
         self.z_shape = (spec.n, spec.c_out, self.h_out, self.w_out)
         e = lambda shape, dt=self.tdtype: torch.empty(int(np.prod(shape)), dtype=dt, device=self.device)
         f = lambda: torch.empty(spec.c_out, dtype=torch.float32, device=self.device)
-        self.x, self.w, self.dz = e(self.x_shape), e(self.w_shape), e(self.z_shape)
+        self.w = e(self.w_shape)
         self.b = f() if spec.bias else None
         self.gamma, self.beta, self.mu_hat, self.var_hat = f(), f(), f(), f()
-        self.z, self.dx = e(self.z_shape), e(self.x_shape)
         self.dw = e(self.w_shape, torch.float32)
         self.db = f() if spec.bias else None
         self.dgamma, self.dbeta = f(), f()
+        self.x = self.dz = self.z = self.dx = self.saved = self.y_saved = self.workspace = None
+        if allocate == "params":
+            return
+        self.x, self.dz = e(self.x_shape), e(self.z_shape)
+        self.z, self.dx = e(self.z_shape), e(self.x_shape)
         phases = []
         if "tune" in modes:
             phases += [C.PHASE_TUNE_FWD, C.PHASE_TUNE_BWD_DATA, C.PHASE_TUNE_BWD_WEIGHT]
@@ -75,16 +81,32 @@ class Block:
 
     def randomize(self, seed: int):
         """Fill the inputs on the device with the recipe's distributions (for timing runs)."""
+        g = self.randomize_params(seed)
+        rn = lambda t, std: t.copy_((torch.randn(t.numel(), generator=g, device=self.device) * std).to(t.dtype))
+        rn(self.x, 1.0); rn(self.dz, 1.0)
+
+    def randomize_params(self, seed: int):
+        """Fill the parameters only; returns the generator for further draws."""
         g = torch.Generator(device=self.device)
         g.manual_seed(seed)
         sp = self.spec
         fan_in = (sp.c_in // sp.groups) * sp.kh * sp.kw
         rn = lambda t, std: t.copy_((torch.randn(t.numel(), generator=g, device=self.device) * std).to(t.dtype))
         ru = lambda t, lo, hi: t.copy_(torch.rand(t.numel(), generator=g, device=self.device) * (hi - lo) + lo)
-        rn(self.x, 1.0); rn(self.dz, 1.0); rn(self.w, float(np.sqrt(2.0 / fan_in)))
+        rn(self.w, float(np.sqrt(2.0 / fan_in)))
         rn(self.mu_hat, 0.1); rn(self.beta, 0.1); ru(self.var_hat, 0.5, 2.0); ru(self.gamma, 0.5, 1.5)
         if self.b is not None:
             rn(self.b, 0.01)
+        return g
+
+    def with_scratch(self, phase: int, call):
+        """Run one entry point with a workspace allocated for this call alone and released after it."""
+        self.workspace = torch.empty(max(256, C.convbn_workspace_bytes(self.desc, phase)), dtype=torch.uint8,
+                                     device=self.device)
+        try:
+            call()
+        finally:
+            self.workspace = None
 
     def fetch(self, name: str) -> np.ndarray:
         """Download a buffer as float64 in logical order."""

@@ -42,4 +42,4 @@ def test_host_step(spec):
     got = {k: blk.fetch(k) for k in names}
     if not spec.bias:
         got["db"] = None
-    parity.compare(got, ref, parity.TOL[spec.dtype], parity.TUNE_OUTPUTS, spec.name)
+    parity.compare(got, ref, parity.TOL[spec.dtype], parity.TUNE_OUTPUTS, spec.name, dtype=spec.dtype)

@@ -301,3 +301,33 @@ def test_saved_elements_follow_appendix_m():
     assert O.saved_elements(s, "deploy") == 32 * 64 * 56 * 56
     t = O.Shape(64, 512, 7, 7, 512, 3, 3, pad_h=1, pad_w=1)
     assert O.saved_elements(t, "eval") - O.saved_elements(t, "tune") == 64 * 512 * 49 - 9 * 512 * 512 < 0
+
+
+# ---- the comparator and the per-channel scale: hand values ---------------------------------
+
+def test_rel_l2_on_hand_values():
+    """The norm behind every parity verdict: ||got - ref|| / ||ref||, absolute when ref = 0."""
+    assert O.rel_l2([1.0, 0.0], [0.0, 1.0]) == pytest.approx(np.sqrt(2.0), rel=1e-15)
+    assert O.rel_l2([3.0, 4.0], [0.0, 0.0]) == 5.0              # zero reference: absolute norm
+    x = rnd(37)
+    assert O.rel_l2(x, x) == 0.0
+    assert O.rel_l2([2.0, 0.0, 0.0], [1.0, 0.0, 0.0]) == 1.0    # 100 % error on the only non-zero entry
+    assert O.rel_l2([[1.0, 2.0], [3.0, 5.0]], [[1.0, 2.0], [3.0, 4.0]]) == pytest.approx(1.0 / np.sqrt(30.0), rel=1e-15)
+    # a sign flip of the whole tensor is an error of 2, a transposed operand is seen
+    assert O.rel_l2(-x, x) == pytest.approx(2.0, rel=1e-15)
+    a = np.array([[1.0, 2.0], [3.0, 4.0]])
+    assert O.rel_l2(a.T, a) > 0.1
+
+
+def test_scale_on_hand_values():
+    """Sec. 3.3: r = 1 / sqrt(var_hat + eps), s = gamma r, with eps INSIDE the root."""
+    s = O.Shape(1, 1, 1, 1, 3, 1, 1, eps=1.0)
+    sc, r = O.scale(s, gamma=[3.0, -2.0, 0.5], var_hat=[15.0, 3.0, 0.0])
+    np.testing.assert_allclose(r, [0.25, 0.5, 1.0], rtol=1e-15)
+    np.testing.assert_allclose(sc, [0.75, -1.0, 0.5], rtol=1e-15)
+    # the same s folds the weights: omega' = s omega, b' = (b - mu) s + beta on a 1x1 block
+    w = np.array([2.0, 4.0, 8.0]).reshape(3, 1, 1, 1)
+    w_f, b_f = O.fold(s, w, np.array([1.0, 1.0, 1.0]), gamma=[3.0, -2.0, 0.5], beta=[0.5, 0.5, 0.5],
+                      mu_hat=[3.0, 0.0, -1.0], var_hat=[15.0, 3.0, 0.0])
+    np.testing.assert_allclose(w_f.ravel(), [1.5, -4.0, 4.0], rtol=1e-15)
+    np.testing.assert_allclose(b_f, [(1 - 3) * 0.75 + 0.5, -1.0 + 0.5, 2 * 0.5 + 0.5], rtol=1e-15)

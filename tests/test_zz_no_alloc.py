@@ -24,27 +24,40 @@ SPECS = [
 
 @pytest.mark.parametrize("spec", SPECS, ids=lambda s: s.name)
 def test_noalloc_matches_workspace_variant_on_two_calls(spec):
-    tol = parity.TOL[spec.dtype]
+    """Both entry points run the same kernels in the same fixed order, so the honest check is bit
+    equality with the workspace call (anything stale in the shared scratch would break it), on two
+    calls in a row, plus one comparison with the CPU oracle."""
+    t = parity.make_inputs(spec, 31)
     blk = Block(spec)
-    blk.load(parity.make_inputs(spec, 31))
+    blk.load(t)
     blk.tune_fwd()
     blk.tune_bwd_weight()
     C.convbn_check()
     names = ["dw", "dgamma", "dbeta"] + (["db"] if spec.bias else [])
     want = {k: blk.fetch(k) for k in names}
-    for call in range(2):
+    ref = parity.oracle_tune(spec, t)
+    parity.compare(dict(want, db=want.get("db")), ref, parity.TOL[spec.dtype], ("dw", "db", "dgamma", "dbeta"),
+                   spec.name + "/workspace call", dtype=spec.dtype)
+
+    def call():
         for k in names:
             getattr(blk, k).fill_(float("nan"))      # the call must rewrite every output itself
-        before = torch.cuda.memory_allocated()
         C.convbn_tune_bwd_weight_noalloc(blk.desc, blk.dz, blk.x, blk.w, blk.b, blk.mu_hat, blk.saved,
                                          blk.dw, blk.db, blk.dgamma, blk.dbeta)
         C.convbn_check()
-        assert torch.cuda.memory_allocated() == before
+
+    call()                                               # first call on this device: looks up the array's address
+    torch.cuda.synchronize()
+    # The library carries its own CUDA runtime, so torch's allocator statistics cannot see an allocation
+    # made inside it; the driver's count of free device memory can.
+    free_before = torch.cuda.mem_get_info()[0]
+    for i in range(2):
+        call()
         for k in names:
             got = blk.fetch(k)
-            assert np.all(np.isfinite(got)), (k, call)
-            err = parity.O.rel_l2(got, want[k])
-            assert err <= tol, (k, call, err)
+            assert np.array_equal(got, want[k]), (k, i, float(np.max(np.abs(got - want[k]))))
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] >= free_before, "device memory was allocated during the calls"
 
 
 def test_noalloc_refuses_layers_beyond_its_scratch():
