@@ -206,6 +206,8 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
         // ---------------- MMA issuer ----------------
         if (elect_one()) {
             constexpr uint32_t idesc = idesc_bf16_f32(kBM, BN, 0, 0);
+            const uint32_t hi = smem_desc_hi_sw128(1024);
+            const uint32_t tiles_lo = smem_desc_lo(smem_u32(tiles), 16), slab_lo = smem_desc_lo(smem_u32(slab), 16);
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
@@ -222,14 +224,14 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait_bounded(&ctl->full[s], ph, abort_flag)) { ok = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t a_addr = smem_u32(tiles + (size_t)s * kStageBytes);
-                    const uint32_t b_addr = g.resident ? smem_u32(slab + (size_t)kb * kBBytes) : a_addr + kABytes;
+                    // descriptors as halves: only the start-address field (16-byte units) moves
+                    const uint32_t a_lo = tiles_lo + (uint32_t)s * (kStageBytes >> 4);
+                    const uint32_t b_lo = g.resident ? slab_lo + (uint32_t)kb * (kBBytes >> 4) : a_lo + (kABytes >> 4);
+                    if (kb == 0) umma_bf16_ss_halves<false>(d_tmem, a_lo, hi, b_lo, hi, idesc);
+                    else umma_bf16_ss_halves<true>(d_tmem, a_lo, hi, b_lo, hi, idesc);
 #pragma unroll
-                    for (int k = 0; k < kBK / kUmmaK; ++k) {
-                        const uint64_t ad = smem_desc_sw128(a_addr + k * kUmmaK * 2, 16, 1024);
-                        const uint64_t bd = smem_desc_sw128(b_addr + k * kUmmaK * 2, 16, 1024);
-                        umma_bf16_ss(d_tmem, ad, bd, idesc, (kb | k) ? 1u : 0u);
-                    }
+                    for (int k = 1; k < kBK / kUmmaK; ++k)
+                        umma_bf16_ss_halves<true>(d_tmem, a_lo + (uint32_t)k * 2u, hi, b_lo + (uint32_t)k * 2u, hi, idesc);
                     umma_commit(&ctl->empty[s]);
                     if (++s == stages) { s = 0; ph ^= 1u; }
                 }

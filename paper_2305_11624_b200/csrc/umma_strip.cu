@@ -13,8 +13,14 @@
 //   forward        Z  = omega' (*) X + b'   (Sec. 3.1 / 3.3)   activation X,  weights omega'
 //   backward data  dX = omega'_rot (*) dZ   (Sec. 3.2.1)       activation dZ, rotated / swapped omega'
 //
-// Warps: 0 patch loader, 1 weight-tile loader (ring), 2 MMA issuer and tensor-memory owner,
-// 3-10 epilogue (two per tensor-memory lane quarter).  Every wait is bounded.
+// Warps: 0 patch loader (ring of 2-4 patch buffers), 1 weight-tile loader, 2-5 MMA issuers (warp 2 owns the
+// tensor memory), 6-21 epilogue (four per tensor-memory lane quarter).  Every wait is bounded.
+// One thread can issue a narrow MMA only every 60-100 clocks once the loop around it is counted, while a
+// 128 x 64 x 16 MMA executes in 48: the M blocks of a tile are therefore dealt to up to four issuing warps,
+// which write disjoint accumulators and each commit to the shared barriers (arrival count = issuers).
+// The weight tiles either stream through a 4-slot ring, once per tile, or - when the whole matrix of the
+// CTA's output channels fits beside the patch buffers - are loaded once and stay resident, which makes small
+// tiles (more rounds over the SMs, better balance) free of weight traffic.
 #include "kernels.h"
 #include "sm100_ptx.cuh"
 
@@ -22,8 +28,12 @@ namespace convbn {
 
 using namespace ptx;
 
-constexpr int kSThreads = 352;
-constexpr int kSBStages = 4;          // weight-tile ring depth
+constexpr int kSIssuers = 4;            // MMA-issuing warps (each owns a subset of a tile's M blocks)
+constexpr int kSEpiGroups = 4;          // epilogue warps per tensor-memory lane quarter
+constexpr int kSEpiWarp0 = 2 + kSIssuers;
+constexpr int kSThreads = 32 * (kSEpiWarp0 + 4 * kSEpiGroups);   // 2 loader, 4 issuer and 16 epilogue warps
+constexpr int kSBStages = 12;         // weight-tile ring: at most this many slots
+constexpr int kSMaxStrips = 4;        // patch buffers
 
 struct StripGemm {
     int n, ho, wo, cn, ca, kh, kw, lower_h, lower_w;
@@ -33,6 +43,10 @@ struct StripGemm {
     int nacc;                         // accumulator sets in tensor memory (1 or 2)
     int blockdiag;                    // grouped conv as block-diagonal 64-channel GEMMs: output block j reads input chunk j
     uint32_t tmem_cols;
+    int nstrips;                      // patch buffers in the ring (2 .. kSMaxStrips)
+    int bstages;                      // weight-tile ring slots in use (streaming mode)
+    int nissue;                       // issuing warps in use: min(nmb, kSIssuers)
+    int resident;                     // 1: all weight tiles stay in shared memory (one n-tile only)
     int sub_cin, sub_hin, sub_win;    // sub-pixel output mode, see UmmaConvShape
     int sub_wide;                     // 1: wide sub-pixel mode (BN = 64 / 128), n-tile -> parity class
     uint32_t sub_mask[4];             // taps with weights, per class
@@ -41,8 +55,9 @@ struct StripGemm {
 };
 
 struct StripCtl {
-    uint64_t strip_full[2], strip_empty[2];
+    uint64_t strip_full[kSMaxStrips], strip_empty[kSMaxStrips];
     uint64_t b_full[kSBStages], b_empty[kSBStages];
+    uint64_t bres_full;               // resident weights have landed
     uint64_t tmem_full[2], tmem_empty[2];
     uint32_t tmem_base;
     int abort_flag;
@@ -56,54 +71,80 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
     extern __shared__ uint8_t smem_raw[];
     constexpr uint32_t kBBytes = BN * 64 * 2;
     uint8_t *strips = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t *bring = strips + 2 * (size_t)g.strip_bytes;
-    StripCtl *ctl = (StripCtl *)(bring + (size_t)kSBStages * kBBytes);
+    uint8_t *bring = strips + (size_t)g.nstrips * g.strip_bytes;     // weight ring, or the resident weight tiles
+    const int cchunks = g.blockdiag ? 1 : g.ca / 64, taps = g.kh * g.kw;
+    const int bstages = g.bstages;
+    StripCtl *ctl = (StripCtl *)(bring + (size_t)(g.resident ? taps * cchunks : bstages) * kBBytes);
     float *bias_s = (float *)(((uintptr_t)(ctl + 1) + 15) & ~(uintptr_t)15);
     float *scale_s = bias_s + g.cn;
     const bool fold = g.fold.gamma != nullptr;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int cchunks = g.blockdiag ? 1 : g.ca / 64, taps = g.kh * g.kw;
+    const int nstrips = g.nstrips;
     const int w_ca = g.blockdiag ? 64 : g.ca;          // K extent of one tap in the weight matrix
     const uint32_t n_tiles = (uint32_t)g.cn / BN;
     const uint32_t sp_tiles = (uint32_t)g.n * g.tiles_h * g.tiles_w;
     const uint32_t total_tiles = sp_tiles * n_tiles;
     volatile int *abort_flag = &ctl->abort_flag;
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(&ctl->strip_full[s], 1); mbar_init(&ctl->strip_empty[s], 1);
-            mbar_init(&ctl->tmem_full[s], 1); mbar_init(&ctl->tmem_empty[s], 8);
+    // Set-up.  Warp 0 (thread 0) initialises the barriers and goes straight to its loads; warp 1 waits only
+    // for that (named barrier 2); the other warps allocate tensor memory and form the per-channel scale and
+    // shift, and meet on named barrier 1, on which the two loader warps merely arrive.  The first patch and
+    // the first weight tiles are therefore in flight while the rest of the set-up runs.
+    if (warp == 0) {
+        if (lane == 0) {
+            CONVBN_TRACE_POINT(0);
+            const uint32_t ni = (uint32_t)g.nissue;     // every issuer commits to the barriers its MMAs release
+            for (int s = 0; s < kSMaxStrips; ++s) { mbar_init(&ctl->strip_full[s], 1); mbar_init(&ctl->strip_empty[s], ni); }
+            for (int s = 0; s < 2; ++s) { mbar_init(&ctl->tmem_full[s], ni); mbar_init(&ctl->tmem_empty[s], 4 * kSEpiGroups); }
+            for (int s = 0; s < kSBStages; ++s) { mbar_init(&ctl->b_full[s], 1); mbar_init(&ctl->b_empty[s], ni); }
+            mbar_init(&ctl->bres_full, 1);
+            ctl->abort_flag = 0;
+            fence_barrier_init();
+            // the tensor maps are kernel parameters, not data of an earlier kernel: fetch them before the wait
+            prefetch_tensormap(&tm_act); prefetch_tensormap(&tm_w);
+            __threadfence_block();
         }
-        for (int s = 0; s < kSBStages; ++s) { mbar_init(&ctl->b_full[s], 1); mbar_init(&ctl->b_empty[s], 1); }
-        ctl->abort_flag = 0;
-        fence_barrier_init();
+        __syncwarp();
+        named_bar_arrive(2, 64);
+        named_bar_arrive(1, kSThreads);
+    } else if (warp == 1) {
+        named_bar_sync(2, 64);
+        named_bar_arrive(1, kSThreads);
     }
     if (warp == 2) {
         tmem_alloc(&ctl->tmem_base, g.tmem_cols);
         tmem_relinquish();
     }
-    // the tensor maps are kernel parameters, not data of an earlier kernel: fetch them before the wait
-    if (threadIdx.x == 0) { prefetch_tensormap(&tm_act); prefetch_tensormap(&tm_w); }
+    // Everything above touched only this CTA's own shared / tensor memory.  Global memory (inputs that an
+    // earlier kernel may still be writing, outputs it may still be reading) comes after this wait.
     pdl_wait();
-    if (fold) {
-        for (int c = threadIdx.x; c < g.cn; c += kSThreads) {
-            const float r = 1.0f / sqrtf(g.fold.var[c] + g.fold.eps);
-            const float sc = g.fold.gamma[c] * r;
-            const float bf = ((g.fold.b ? g.fold.b[c] : 0.f) - g.fold.mean[c]) * sc + g.fold.beta[c];
-            scale_s[c] = sc;
-            bias_s[c] = bf;
-            if (blockIdx.x == 0 && g.fold.vec3) {
-                g.fold.vec3[c] = sc; g.fold.vec3[g.cn + c] = bf; g.fold.vec3[2 * g.cn + c] = r;
+    if (threadIdx.x == 0) CONVBN_TRACE_POINT(1);
+    uint32_t tmem_base = 0;
+    if (warp >= 2) {
+        const int nt = kSThreads - 64, tid = (int)threadIdx.x - 64;
+        if (fold) {
+            // On-the-fly reparameterisation (Sec. 3.3 / 3.4): s = gamma / sqrt(var + eps), b' = (b - mu) s + beta;
+            // s multiplies the fp32 accumulator (the associative law of Sec. 3.2.2), so omega is used unrounded.
+            for (int c = tid; c < g.cn; c += nt) {
+                const float r = 1.0f / sqrtf(g.fold.var[c] + g.fold.eps);
+                const float sc = g.fold.gamma[c] * r;
+                const float bf = ((g.fold.b ? g.fold.b[c] : 0.f) - g.fold.mean[c]) * sc + g.fold.beta[c];
+                scale_s[c] = sc;
+                bias_s[c] = bf;
+                if (blockIdx.x == 0 && g.fold.vec3) {
+                    g.fold.vec3[c] = sc; g.fold.vec3[g.cn + c] = bf; g.fold.vec3[2 * g.cn + c] = r;
+                }
             }
+        } else if (bias) {
+            for (int c = tid; c < g.cn; c += nt) bias_s[c] = bias[c];
         }
-    } else if (bias) {
-        for (int c = threadIdx.x; c < g.cn; c += kSThreads) bias_s[c] = bias[c];
+        tc_fence_before_sync();
+        named_bar_sync(1, kSThreads);
+        tc_fence_after_sync();
+        pdl_launch_dependents();       // only now: this CTA owns its tensor-memory columns
+        tmem_base = ctl->tmem_base;
+        if (threadIdx.x == 64) CONVBN_TRACE_POINT(2);
     }
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    pdl_launch_dependents();       // only now: this CTA owns its tensor-memory columns
-    const uint32_t tmem_base = ctl->tmem_base;
 
     // tile t -> (image, tile row, tile column, n-tile); n-tiles of one patch sit on neighbouring CTAs
     auto decode = [&](uint32_t t, int &img, int &h0, int &w0, int &n0) {
@@ -129,14 +170,15 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
                 for (int cc = 0; cc < cchunks; ++cc) {
                     if (!mbar_wait_bounded(&ctl->strip_empty[sb], ph ^ 1u, abort_flag)) { ok = false; break; }
                     mbar_arrive_expect_tx(&ctl->strip_full[sb], bytes);
+                    if (t == blockIdx.x && cc == 0) CONVBN_TRACE_POINT(3);
                     tma_load_4d(strips + (size_t)sb * g.strip_bytes, &tm_act, &ctl->strip_full[sb],
                                 g.blockdiag ? n0 : cc * 64, w0 + g.lower_w, h0 + g.lower_h, img);
-                    if (++sb == 2) { sb = 0; ph ^= 1u; }
+                    if (++sb == nstrips) { sb = 0; ph ^= 1u; }
                 }
             }
             if (!ok) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
             // an issued copy always completes; give the last ones time to land before the CTA can exit
-            if (!ok) for (int s = 0; s < 2; ++s) mbar_wait_bounded(&ctl->strip_full[s], 0, nullptr, 2000000ull);
+            if (!ok) for (int s = 0; s < nstrips; ++s) mbar_wait_bounded(&ctl->strip_full[s], 0, nullptr, 2000000ull);
         }
     } else if (warp == 1) {
         // ---------------- weight-tile loader ----------------
@@ -144,6 +186,16 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
+            if (g.resident) {
+                // one n-tile, every (channel chunk, tap) tile loaded once: tile index cc taps + tap
+                if (blockIdx.x < total_tiles) {
+                    mbar_arrive_expect_tx(&ctl->bres_full, (uint32_t)(taps * cchunks) * kBBytes);
+                    for (int cc = 0; cc < cchunks; ++cc)
+                        for (int tap = 0; tap < taps; ++tap)
+                            tma_load_2d(bring + (size_t)(cc * taps + tap) * kBBytes, &tm_w, &ctl->bres_full,
+                                        tap * w_ca + cc * 64, 0);
+                }
+            } else
             for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
                 const int n0 = (int)(t % n_tiles) * BN;
                 const uint32_t mask = g.sub_wide ? g.sub_mask[n0 / g.sub_cin] : 0xffffffffu;
@@ -153,63 +205,87 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
                         if (!mbar_wait_bounded(&ctl->b_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
                         mbar_arrive_expect_tx(&ctl->b_full[s], kBBytes);
                         tma_load_2d(bring + (size_t)s * kBBytes, &tm_w, &ctl->b_full[s], tap * w_ca + cc * 64, n0);
-                        if (++s == kSBStages) { s = 0; ph ^= 1u; }
+                        if (++s == bstages) { s = 0; ph ^= 1u; }
                     }
             }
             if (!ok) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
-            if (!ok) for (int q = 0; q < kSBStages; ++q) mbar_wait_bounded(&ctl->b_full[q], 0, nullptr, 2000000ull);
+            if (!ok) for (int q = 0; q < bstages; ++q) mbar_wait_bounded(&ctl->b_full[q], 0, nullptr, 2000000ull);
         }
-    } else if (warp == 2) {
-        // ---------------- MMA issuer ----------------
-        if (elect_one()) {
+    } else if (warp < kSEpiWarp0) {
+        // ---------------- MMA issuers ----------------
+        // One thread issues every MMA, so the instructions between two MMAs bound the rate of the narrow
+        // ones (a 128 x 64 x 16 MMA takes 48 clocks, a 128 x 16 x 16 one 39): descriptors are kept as halves
+        // and only their start-address field moves.
+        const int me = warp - 2, ni = g.nissue;         // this warp issues M blocks me, me + ni, ...
+        if (me < ni && elect_one()) {
             constexpr uint32_t idesc = idesc_bf16_f32(128, BN, 0, 0);
+            const uint32_t hi = smem_desc_hi_sw128(1024);
+            const uint32_t bres_lo = smem_desc_lo(smem_u32(bring), 16);
             int sb = 0, s = 0;
             uint32_t sph = 0, bph = 0, i = 0;
             bool ok = true;
+            if (g.resident && blockIdx.x < total_tiles) {
+                ok = mbar_wait_bounded(&ctl->bres_full, 0, abort_flag);
+                tc_fence_after_sync();
+            }
             for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++i) {
                 const uint32_t a = i % (uint32_t)g.nacc, use = i / (uint32_t)g.nacc;
                 if (!mbar_wait_bounded(&ctl->tmem_empty[a], (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d0 = tmem_base + a * (uint32_t)(g.nmb * BN);
                 const uint32_t mask = g.sub_wide ? g.sub_mask[(int)(t % n_tiles) * BN / g.sub_cin] : 0xffffffffu;
-                uint32_t started = 0;                   // 0 until the tile's first MMAs have been issued
+                bool started = false;                   // false until the tile's first MMAs have been issued
                 for (int cc = 0; cc < cchunks && ok; ++cc) {
                     if (!mbar_wait_bounded(&ctl->strip_full[sb], sph, abort_flag)) { ok = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t patch = smem_u32(strips + (size_t)sb * g.strip_bytes);
-                    int r = 0, q = 0;
+                    if (i == 0 && cc == 0 && me == 0) CONVBN_TRACE_POINT(4);
+                    const uint32_t a_patch = smem_desc_lo(smem_u32(strips + (size_t)sb * g.strip_bytes), 16);
+                    uint32_t row_shift = 0;             // (r Wt + q) pixels of 128 bytes, in 16-byte units
+                    int q = 0;
                     for (int tap = 0; tap < taps; ++tap) {
-                        if (!((mask >> tap) & 1u)) { if (++q == g.kw) { q = 0; ++r; } continue; }
-                        if (!mbar_wait_bounded(&ctl->b_full[s], bph, abort_flag)) { ok = false; break; }
-                        tc_fence_after_sync();
-                        const uint32_t b_addr = smem_u32(bring + (size_t)s * kBBytes);
-                        const uint32_t shift = (uint32_t)(r * g.Wt + q) * 128u;
+                        const uint32_t a_tap = a_patch + row_shift + (uint32_t)q * 8u;
+                        if (++q == g.kw) { q = 0; row_shift += (uint32_t)g.Wt * 8u; }
+                        if (!((mask >> tap) & 1u)) continue;
+                        uint32_t b_lo;
+                        if (g.resident) {
+                            b_lo = bres_lo + (uint32_t)(cc * taps + tap) * (kBBytes >> 4);
+                        } else {
+                            if (!mbar_wait_bounded(&ctl->b_full[s], bph, abort_flag)) { ok = false; break; }
+                            tc_fence_after_sync();
+                            b_lo = smem_desc_lo(smem_u32(bring + (size_t)s * kBBytes), 16);
+                        }
                         // consecutive MMAs go to different accumulators (M blocks), so an MMA never has to
                         // wait for the previous one's accumulator update
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const uint64_t bd = smem_desc_sw128(b_addr + k * 32, 16, 1024);
-                            for (int mb = 0; mb < g.nmb; ++mb)
-                                umma_bf16_ss(d0 + (uint32_t)(mb * BN),
-                                             smem_desc_sw128(patch + (uint32_t)mb * (128u * 128u) + shift + k * 32, 16, 1024),
-                                             bd, idesc, (started | (uint32_t)k) ? 1u : 0u);
+                        if (!started) {
+                            for (int mb = me; mb < g.nmb; mb += ni)
+                                umma_bf16_ss_halves<false>(d0 + (uint32_t)(mb * BN), a_tap + (uint32_t)mb * 1024u, hi, b_lo, hi, idesc);
+                            started = true;
+                        } else {
+                            for (int mb = me; mb < g.nmb; mb += ni)
+                                umma_bf16_ss_halves<true>(d0 + (uint32_t)(mb * BN), a_tap + (uint32_t)mb * 1024u, hi, b_lo, hi, idesc);
                         }
-                        started = 1;
-                        umma_commit(&ctl->b_empty[s]);
-                        if (++s == kSBStages) { s = 0; bph ^= 1u; }
-                        if (++q == g.kw) { q = 0; ++r; }
+#pragma unroll
+                        for (int k = 1; k < 4; ++k)
+                            for (int mb = me; mb < g.nmb; mb += ni)
+                                umma_bf16_ss_halves<true>(d0 + (uint32_t)(mb * BN), a_tap + (uint32_t)mb * 1024u + (uint32_t)k * 2u, hi,
+                                                          b_lo + (uint32_t)k * 2u, hi, idesc);
+                        if (!g.resident) {
+                            umma_commit(&ctl->b_empty[s]);
+                            if (++s == bstages) { s = 0; bph ^= 1u; }
+                        }
                     }
                     if (ok) umma_commit(&ctl->strip_empty[sb]);
-                    if (++sb == 2) { sb = 0; sph ^= 1u; }
+                    if (++sb == nstrips) { sb = 0; sph ^= 1u; }
                 }
                 if (ok) umma_commit(&ctl->tmem_full[a]);
+                if (me == 0) { if (i == 0) CONVBN_TRACE_POINT(5); CONVBN_TRACE_POINT(6); }
             }
             if (!ok) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
         }
     } else {
         // ---------------- epilogue: tensor memory -> registers -> (scale, shift) -> bf16 -> global ----
         const int quarter = warp & 3;
-        const int egroup = (warp - 3) >> 2;            // M blocks egroup, egroup + 2 of every tile
+        const int egroup = (warp - kSEpiWarp0) >> 2;   // M blocks egroup, egroup + 4, ... of every tile
         uint32_t i = 0;
         for (uint32_t t = blockIdx.x; t < total_tiles; t += gridDim.x, ++i) {
             const uint32_t a = i % (uint32_t)g.nacc, use = i / (uint32_t)g.nacc;
@@ -219,9 +295,10 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
                 break;
             }
             tc_fence_after_sync();
+            if (warp == kSEpiWarp0 && lane == 0) { if (i == 0) CONVBN_TRACE_POINT(7); CONVBN_TRACE_POINT(9); }
             int img, h0, w0, n0;
             decode(t, img, h0, w0, n0);
-            for (int mb = egroup; mb < g.nmb; mb += 2) {
+            for (int mb = egroup; mb < g.nmb; mb += kSEpiGroups) {
                 const uint32_t v = (uint32_t)mb * 128u + (uint32_t)(quarter * 32 + lane);
                 const uint32_t vi = v / (uint32_t)g.Wt;
                 const int ti = (int)vi, tj = (int)(v - vi * (uint32_t)g.Wt);
@@ -307,17 +384,19 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&ctl->tmem_empty[a]);
+            if (warp == kSEpiWarp0 && lane == 0) { if (i == 0) CONVBN_TRACE_POINT(8); CONVBN_TRACE_POINT(10); }
         }
     }
     tc_fence_before_sync();
     __syncthreads();
+    if (threadIdx.x == 0) CONVBN_TRACE_POINT(11);
     if (warp == 2) tmem_dealloc(tmem_base, g.tmem_cols);
 }
 
 // ---- host side --------------------------------------------------------------------------------------
 namespace {
 
-struct StripPlan { bool ok = false; int bn = 64, R = 0, CW = 0, Wt = 0, nmb = 0, nacc = 2, tiles_w = 1 << 20; uint32_t strip_bytes = 0; size_t smem = 0; };
+struct StripPlan { bool ok = false; int bn = 64, R = 0, CW = 0, Wt = 0, nmb = 0, nacc = 2, tiles_w = 1 << 20, nstrips = 2, resident = 0, bstages = 4; uint32_t strip_bytes = 0; size_t smem = 0; };
 
 int strip_sm_count() { return device_sm_count(); }
 
@@ -336,10 +415,17 @@ StripPlan plan_strip(const UmmaConvShape &s) {
     const int tiles_w_min = (s.wo + (256 - s.taps_w + 1) - 1) / (256 - s.taps_w + 1);
     // Among the tilings that keep at least 70 % of the MMA rows useful, take the one with the lowest
     // estimated time: rounds over the SMs x (the larger of the tile's MMA issue time and its shared-memory
-    // fill time, plus a fixed cost per tile).  The weight tiles are streamed again for every tile, so small
-    // tiles pay for them many times over.
+    // fill time, plus a fixed cost per tile).  Weight tiles that do not stay resident are streamed again for
+    // every tile, so small tiles then pay for them many times over.
     const int cchunks = s.blockdiag ? 1 : s.ca / 64, taps = s.taps_h * s.taps_w;
     const int n_tiles = s.cn / bn, sms = strip_sm_count();
+    const size_t fixed = 1024 + sizeof(StripCtl) + 2 * (size_t)s.cn * sizeof(float) + 32;
+    const size_t bbytes = (size_t)bn * 128, wall = (size_t)taps * cchunks * bbytes;
+    const size_t budget = 224 * 1024;
+    // clocks per 128 x bn x 16 MMA (measured issue floors 39 / 48 / 64, plus the issue loop's own instructions)
+    const double mma1 = bn == 16 ? 41.0 : (bn == 64 ? 50.0 : 66.0);
+    // a ring slot is free again one load round trip (about 2.2 us under load) after its MMAs were committed
+    const double ring_clk = 4400.0;
     double best_eff = 0.0, best_cost = -1.0;
     for (int tiles_w = tiles_w_min; tiles_w < tiles_w_min + 4; ++tiles_w) {
     const int cw = (s.wo + tiles_w - 1) / tiles_w, wt = cw + s.taps_w - 1;
@@ -349,22 +435,38 @@ StripPlan plan_strip(const UmmaConvShape &s) {
         if (nmb > nmb_max) break;
         const size_t px = (size_t)nmb * 128 + (size_t)(s.taps_h - 1) * wt + (s.taps_w - 1);
         const uint32_t sbytes = (uint32_t)(((px * 128) + 1023) / 1024 * 1024);
-        const size_t smem = 1024 + 2 * (size_t)sbytes + (size_t)kSBStages * bn * 128 + sizeof(StripCtl) +
-                            2 * (size_t)s.cn * sizeof(float) + 32;
-        if (smem > 224 * 1024) break;
+        // resident weights when they fit beside two patch buffers (one n-tile, no per-class tap masks)
+        const bool resident = n_tiles == 1 && !sub_wide && fixed + wall + 2 * (size_t)sbytes <= budget;
+        if (!resident && fixed + 4 * bbytes + 2 * (size_t)sbytes > budget) break;
+        int nstrips = 2, bstages = 4;
+        if (resident) {
+            nstrips = (int)((budget - fixed - wall) / sbytes);
+            if (nstrips > kSMaxStrips) nstrips = kSMaxStrips;
+        } else {
+            bstages = (int)((budget - fixed - 2 * (size_t)sbytes) / bbytes);
+            if (bstages > kSBStages) bstages = kSBStages;
+            if ((long long)bstages > (long long)taps * cchunks) bstages = taps * cchunks;
+            nstrips = 2 + (int)((budget - fixed - 2 * (size_t)sbytes - (size_t)bstages * bbytes) / sbytes);
+            if (nstrips > kSMaxStrips) nstrips = kSMaxStrips;
+        }
+        const size_t smem = fixed + (resident ? wall : (size_t)bstages * bbytes) + (size_t)nstrips * sbytes;
         const int tiles_h = (s.ho + r - 1) / r;
         const double eff = (double)s.ho * s.wo / ((double)tiles_h * tiles_w * nmb * 128.0);
         if (eff < 0.70) continue;
-        const double mma_clk = (double)nmb * taps * cchunks * 4 * (bn == 16 ? 40.0 : (bn == 64 ? 67.0 : 128.0));
-        const double fill_clk = ((double)(r + s.taps_h - 1) * wt * 128.0 + (double)taps * bn * 128.0) * cchunks / 32.0;
-        const double tile_clk = (mma_clk > fill_clk ? mma_clk : fill_clk) + 1500.0;
+        double tap_clk = (double)nmb * 4 * mma1;
+        if (!resident && ring_clk / bstages > tap_clk) tap_clk = ring_clk / bstages;
+        const double mma_clk = tap_clk * taps * cchunks;
+        const double fill_clk = ((double)(r + s.taps_h - 1) * wt * 128.0 + (resident ? 0.0 : (double)taps * bbytes)) *
+                                cchunks / 32.0;
+        const double tile_clk = (mma_clk > fill_clk ? mma_clk : fill_clk) + 500.0;
         const long long tiles = (long long)s.n * tiles_h * tiles_w * n_tiles;
-        const double cost = (double)((tiles + sms - 1) / sms) * tile_clk;
+        const double cost = (double)((tiles + sms - 1) / sms) * tile_clk + (resident ? (double)wall / 32.0 : 0.0);
         if (best_cost < 0 || cost < best_cost) {
             best_cost = cost;
             best_eff = eff;
             best.ok = true; best.bn = bn; best.R = r; best.CW = cw; best.Wt = wt; best.nmb = nmb;
             best.strip_bytes = sbytes; best.smem = smem; best.tiles_w = tiles_w;
+            best.nstrips = nstrips; best.resident = resident ? 1 : 0; best.bstages = bstages;
         }
     }
     }
@@ -426,6 +528,8 @@ cudaError_t launch_umma_strip_conv(const UmmaConvShape &s, const void *act, cons
     g.tiles_h = (s.ho + pl.R - 1) / pl.R; g.tiles_w = (s.wo + pl.CW - 1) / pl.CW;
     g.strip_bytes = pl.strip_bytes;
     g.nacc = 2;
+    g.nstrips = pl.nstrips; g.resident = pl.resident; g.bstages = pl.bstages;
+    g.nissue = pl.nmb < kSIssuers ? pl.nmb : kSIssuers;
     g.blockdiag = s.blockdiag;
     g.sub_cin = s.sub_cin; g.sub_hin = s.sub_hin; g.sub_win = s.sub_win;
     g.sub_wide = (s.sub_cin > 0 && s.cn != 16) ? 1 : 0;

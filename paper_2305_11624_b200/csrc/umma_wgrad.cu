@@ -159,6 +159,8 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
     } else if (warp == 1) {
         if (elect_one()) {
             constexpr uint32_t idesc = idesc_bf16_f32(kWM, BN, 1, 1);   // both operands MN-major
+            const uint32_t hi = smem_desc_hi_sw128(1024);
+            const uint32_t tiles_lo = smem_desc_lo(smem_u32(tiles), kChunkBytes);
             bool ok = true;
             int s = 0;
             uint32_t ph = 0;
@@ -170,14 +172,15 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
                     break;
                 }
                 tc_fence_after_sync();
-                const uint32_t a_addr = smem_u32(tiles + (size_t)s * kStageBytes), b_addr = a_addr + kABytes;
+                // 16 pixels = two groups of 8 rows (1024 B apart); 64-channel slices 8192 B apart; descriptors as
+                // halves, only the start-address field (16-byte units) moves
+                const uint32_t a_lo = tiles_lo + (uint32_t)s * (kStageBytes >> 4), b_lo = a_lo + (kABytes >> 4);
+                if (kb == 0) umma_bf16_ss_halves<false>(tmem_base, a_lo, hi, b_lo, hi, idesc);
+                else umma_bf16_ss_halves<true>(tmem_base, a_lo, hi, b_lo, hi, idesc);
 #pragma unroll
-                for (int k = 0; k < kWP / kWUmmaK; ++k) {
-                    // 16 pixels = two groups of 8 rows (1024 B apart); 64-channel slices 8192 B apart
-                    const uint64_t ad = smem_desc_sw128(a_addr + k * kWUmmaK * 128, kChunkBytes, 1024);
-                    const uint64_t bd = smem_desc_sw128(b_addr + k * kWUmmaK * 128, kChunkBytes, 1024);
-                    umma_bf16_ss(tmem_base, ad, bd, idesc, (kb | k) ? 1u : 0u);
-                }
+                for (int k = 1; k < kWP / kWUmmaK; ++k)
+                    umma_bf16_ss_halves<true>(tmem_base, a_lo + (uint32_t)k * (kWUmmaK * 128 >> 4), hi,
+                                              b_lo + (uint32_t)k * (kWUmmaK * 128 >> 4), hi, idesc);
                 umma_commit(&ctl->empty[s]);
                 if (++s == stages) { s = 0; ph ^= 1u; }
             }
