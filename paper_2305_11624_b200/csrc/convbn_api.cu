@@ -317,7 +317,11 @@ int run_conv_fwd(const convbn_desc *d, const Problem &pb, const void *x, const v
                  void *z, const Plan &pl, void *ws, cudaStream_t st, const char **which) {
     UmmaConvShape s;
     void *wbd_scratch = at(ws, pl.wbd);
-    if (pl.stem) {
+    if (pl.stem && stem_window_eligible(pb)) {
+        // few input channels, stride 2: input rows staged once, windows formed by the operand addressing
+        LAUNCH("stem_fwd", launch_stem_window_fwd(pb, x, w, bias, z, st));
+        *which = "umma-stem";
+    } else if (pl.stem) {
         // few input channels: repack X (8 channels per pixel, zero border) and run the tensor-core GEMM
         // with one 64-wide K row (8 pixels x 8 channels) per filter row
         LAUNCH("stem_pack", launch_stem_pack(pb, x, at(ws, pl.xpk), st));
@@ -596,6 +600,12 @@ int convbn_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const
     float *vec3 = (float *)saved;
     void *wf = at(workspace, pl.w_scaled);
     UmmaConvShape us;
+    if (pl.stem && stem_window_eligible(pb)) {
+        const BnFold fold{gamma, beta, run_mean, run_var, b, pb.eps, vec3};
+        LAUNCH("stem_fwd", launch_stem_window_fwd(pb, x, w, nullptr, z, st, &fold));
+        t_last_kernel[CONVBN_PHASE_TUNE_FWD] = "umma-stem";
+        return CONVBN_OK;
+    }
     if (pl.stem) {
         const BnFold fold{gamma, beta, run_mean, run_var, b, pb.eps, vec3};
         LAUNCH("stem_pack", launch_stem_pack(pb, x, at(workspace, pl.xpk), st));

@@ -152,6 +152,11 @@ cudaError_t launch_wgrad_epilogue_stem(const Problem &pb, const UmmaWgradPlan &p
                                        const float *bsum, const void *w, const float *vec3, const float *b,
                                        const float *mean, float *dw, float *db, float *dgamma, float *dbeta,
                                        bool need_sums, cudaStream_t st);
+// Forward pass straight from X for stride_w = 2, C_in <= 4, C_out 64 or 128 (see stem_window.cu): input rows
+// staged once in shared memory, the im2col windows formed by the MMA operand addressing.  No packed copy.
+bool stem_window_eligible(const Problem &pb);
+cudaError_t launch_stem_window_fwd(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
+                                   cudaStream_t st, const BnFold *fold = nullptr);
 cudaError_t launch_stem_fwd(const Problem &pb, const void *x_packed, const void *wst, const float *bias, void *out,
                             cudaStream_t st, const BnFold *fold = nullptr);
 

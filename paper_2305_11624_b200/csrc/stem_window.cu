@@ -1,0 +1,393 @@
+// Forward pass of a first-layer ("stem") convolution with very few input channels, stride 2 along W
+// (e.g. 7x7 stride 2 on RGB):  Z = omega' (*) X + b'  (Sec. 3.1 / 3.3), on the sm_100a tensor cores with the
+// im2col expansion done by the MMA's own operand addressing instead of by memory traffic.
+//
+// Input rows are kept in shared memory as zero-bordered rows of 4-channel pixels (8 bytes each).  For one
+// filter row r the K values of output pixel wo are the kw x 4 values that start at padded pixel 2 wo: 16 wo
+// bytes into the row.  A K-major operand WITHOUT swizzle addresses element (m, k) at
+//     start + (m / 8) SBO + (m % 8) 16 + (k / 8) LBO + (k % 8) 2      bytes,
+// so SBO = 128 and LBO = 16 give  start + 16 m + 2 k : the 128 rows of the A tile are 128 consecutive output
+// pixels of one output row, overlapping windows of the same shared-memory row.  Each input row is loaded
+// once per tile (kh / stride_h times overall) instead of once per tap, and K per filter row is 32 (kw <= 8
+// taps x 4 channels; unused slots meet zero weights), i.e. kh x 2 MMAs of 128 x C_out x 16 per output row.
+//
+// Warps: 0-3 load input rows (16-byte global loads, repacked 3 -> 4 channels on the way), 4-7 issue MMAs
+// (round-robin over output rows, disjoint accumulators), 8-23 drain accumulators: scale, shift, bf16,
+// swizzled staging, TMA store.  Every CTA owns a contiguous range of output rows.  Every wait is bounded.
+#include "kernels.h"
+#include "sm100_ptx.cuh"
+
+namespace convbn {
+
+using namespace ptx;
+
+constexpr int kWinLoaders = 4, kWinIssuers = 4, kWinEpiGroups = 4;
+constexpr int kWinEpiWarp0 = kWinLoaders + kWinIssuers;
+constexpr int kWinThreads = 32 * (kWinEpiWarp0 + 4 * kWinEpiGroups);
+constexpr int kWinMaxStrips = 3;
+constexpr int kWinSlack = 2304;          // bytes readable past the last row of a patch (junk rows of an M block)
+
+struct WinGemm {
+    int n, h_in, w_in, c_in, h_out, w_out, c_out, kh, kw, stride_h, pad_h, pad_w;
+    int R;                 // output rows per tile
+    int rows_in;           // input rows per full tile: (R - 1) stride_h + kh
+    int pitch;             // bytes per padded input row in shared memory (multiple of 16)
+    int colblocks;         // M blocks per output row: ceil(w_out / 128)
+    int nstrips;           // patch buffers
+    uint32_t strip_bytes;  // one patch buffer (multiple of 1024)
+    int kblocks;           // 128-byte K rows of the resident weights: ceil(kh / 2)
+    long long total_rows;  // n * h_out
+    BnFold fold;
+};
+
+struct WinCtl {
+    uint64_t strip_full[kWinMaxStrips], strip_empty[kWinMaxStrips];
+    uint64_t tmem_full[8], tmem_empty[8];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+// descriptor halves of the un-swizzled K-major window operand: LBO 16 bytes, SBO 128 bytes
+__device__ __forceinline__ uint32_t win_desc_lo(uint32_t smem_addr) { return ((smem_addr >> 4) & 0x3FFFu) | (1u << 16); }
+__device__ __forceinline__ uint32_t win_desc_hi() { return 8u | (1u << 14); }
+
+// The chunk sequence of a CTA: its output rows [lo, hi) of the flattened (image, row) space, cut into
+// tiles of at most R rows that do not cross an image.  Every role walks the same sequence.
+struct WinChunk { int img, h0, rows; };
+__device__ __forceinline__ bool win_next_chunk(long long &cur, long long hi, int h_out, int R, WinChunk &c) {
+    if (cur >= hi) return false;
+    const long long img = cur / h_out;
+    const int h0 = (int)(cur - img * h_out);
+    int rows = R;
+    if (rows > h_out - h0) rows = h_out - h0;
+    if ((long long)rows > hi - cur) rows = (int)(hi - cur);
+    c.img = (int)img; c.h0 = h0; c.rows = rows;
+    cur += rows;
+    return true;
+}
+
+template <int BN, int C>
+__global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __grid_constant__ CUtensorMap tm_out,
+                                                                     const WinGemm g,
+                                                                     const __nv_bfloat16 *__restrict__ x,
+                                                                     const __nv_bfloat16 *__restrict__ w,
+                                                                     const float *__restrict__ bias, int *err) {
+    extern __shared__ uint8_t smem_raw[];
+    constexpr int NA = 512 / BN;                           // accumulators in tensor memory
+    uint8_t *strips = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *wres = strips + (size_t)g.nstrips * g.strip_bytes;          // [kblocks][BN][128 B], 128-byte swizzle
+    uint8_t *staging = wres + (size_t)g.kblocks * BN * 128;              // 16 warps x [32 rows][128 B]
+    WinCtl *ctl = (WinCtl *)(staging + 16 * 4096);
+    float *bias_s = (float *)(((uintptr_t)(ctl + 1) + 15) & ~(uintptr_t)15);
+    float *scale_s = bias_s + BN;
+    const bool fold = g.fold.gamma != nullptr;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int *abort_flag = &ctl->abort_flag;
+    // this CTA's output rows
+    const long long row_lo = g.total_rows * blockIdx.x / gridDim.x, row_hi = g.total_rows * (blockIdx.x + 1) / gridDim.x;
+
+    if (warp < kWinLoaders) {
+        if (threadIdx.x == 0) {
+            for (int s = 0; s < kWinMaxStrips; ++s) { mbar_init(&ctl->strip_full[s], 32 * kWinLoaders); mbar_init(&ctl->strip_empty[s], kWinIssuers); }
+            for (int s = 0; s < 8; ++s) { mbar_init(&ctl->tmem_full[s], 1); mbar_init(&ctl->tmem_empty[s], 4); }
+            ctl->abort_flag = 0;
+            fence_barrier_init();
+            prefetch_tensormap(&tm_out);
+            __threadfence_block();
+        }
+        // zero the patch buffers once: borders and the slack behind the last row stay zero for good
+        {
+            uint4 *p = (uint4 *)strips;
+            const int n16 = (int)((size_t)g.nstrips * g.strip_bytes / 16);
+            for (int i = threadIdx.x; i < n16; i += 32 * kWinLoaders) p[i] = make_uint4(0, 0, 0, 0);
+        }
+        __threadfence_block();
+        named_bar_sync(3, 32 * kWinLoaders);
+        named_bar_arrive(1, kWinThreads);
+    }
+    if (warp == kWinLoaders) {
+        tmem_alloc(&ctl->tmem_base, 512);
+        tmem_relinquish();
+    }
+    pdl_wait();
+    uint32_t tmem_base = 0;
+    if (warp >= kWinLoaders) {
+        if (warp >= kWinEpiWarp0) {
+            const int nt = kWinThreads - 32 * kWinEpiWarp0, tid = (int)threadIdx.x - 32 * kWinEpiWarp0;
+            if (fold) {
+                // On-the-fly reparameterisation (Sec. 3.3 / 3.4); s multiplies the fp32 accumulator (Sec. 3.2.2)
+                for (int c = tid; c < BN; c += nt) {
+                    const float r = 1.0f / sqrtf(g.fold.var[c] + g.fold.eps);
+                    const float sc = g.fold.gamma[c] * r;
+                    const float bf = ((g.fold.b ? g.fold.b[c] : 0.f) - g.fold.mean[c]) * sc + g.fold.beta[c];
+                    scale_s[c] = sc;
+                    bias_s[c] = bf;
+                    if (blockIdx.x == 0 && g.fold.vec3) {
+                        g.fold.vec3[c] = sc; g.fold.vec3[BN + c] = bf; g.fold.vec3[2 * BN + c] = r;
+                    }
+                }
+            } else {
+                for (int c = tid; c < BN; c += nt) { bias_s[c] = bias ? bias[c] : 0.f; scale_s[c] = 1.f; }
+            }
+            // resident weights: K index = r 32 + q 4 + c, two filter rows per 128-byte row, zeros in unused slots
+            const int slots = g.kblocks * BN * 64;
+            for (int i = tid; i < slots; i += nt) {
+                const int k64 = i & 63, co = (i >> 6) % BN, kb = (i >> 6) / BN;
+                const int r = kb * 2 + (k64 >> 5), q = (k64 & 31) >> 2, c = k64 & 3;
+                unsigned short v = 0;
+                if (r < g.kh && q < g.kw && c < C)
+                    v = ((const unsigned short *)w)[(((size_t)co * g.kh + r) * g.kw + q) * C + c];
+                *(unsigned short *)(wres + (size_t)kb * BN * 128 + co * 128 + ((((k64 >> 3) ^ (co & 7)) & 7) << 4) + (k64 & 7) * 2) = v;
+            }
+            fence_proxy_async_smem();
+        }
+        tc_fence_before_sync();
+        named_bar_sync(1, kWinThreads);
+        tc_fence_after_sync();
+        pdl_launch_dependents();       // only now: this CTA owns its tensor-memory columns
+        tmem_base = ctl->tmem_base;
+    }
+
+    if (warp < kWinLoaders) {
+        // ---------------- input-row loaders ----------------
+        const int ltid = threadIdx.x, chunks_w = g.w_in / 8;
+        long long cur = row_lo;
+        WinChunk ck;
+        int sb = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        while (ok && win_next_chunk(cur, row_hi, g.h_out, g.R, ck)) {
+            ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->strip_empty[sb], ph ^ 1u, abort_flag));
+            if (!ok) break;
+            uint8_t *patch = strips + (size_t)sb * g.strip_bytes;
+            const int first = ck.h0 * g.stride_h - g.pad_h, count = (ck.rows - 1) * g.stride_h + g.kh;
+            const int tasks = count * chunks_w;
+#pragma unroll 2
+            for (int t = ltid; t < tasks; t += 32 * kWinLoaders) {
+                const int pr = t / chunks_w, j = t - pr * chunks_w, h = first + pr;
+                uint2 *dst = (uint2 *)(patch + (size_t)pr * g.pitch + (size_t)(g.pad_w + 8 * j) * 8);
+                if (h < 0 || h >= g.h_in) {
+#pragma unroll
+                    for (int p = 0; p < 8; ++p) dst[p] = make_uint2(0, 0);
+                    continue;
+                }
+                const uint4 *src = (const uint4 *)(x + (((size_t)ck.img * g.h_in + h) * g.w_in + 8 * j) * C);
+                unsigned short e[8 * C];
+#pragma unroll
+                for (int v = 0; v < C; ++v) {
+                    const uint4 q4 = __ldg(src + v);
+                    e[8 * v + 0] = (unsigned short)q4.x; e[8 * v + 1] = (unsigned short)(q4.x >> 16);
+                    e[8 * v + 2] = (unsigned short)q4.y; e[8 * v + 3] = (unsigned short)(q4.y >> 16);
+                    e[8 * v + 4] = (unsigned short)q4.z; e[8 * v + 5] = (unsigned short)(q4.z >> 16);
+                    e[8 * v + 6] = (unsigned short)q4.w; e[8 * v + 7] = (unsigned short)(q4.w >> 16);
+                }
+#pragma unroll
+                for (int p = 0; p < 8; ++p) {
+                    unsigned short c0 = e[p * C], c1 = C > 1 ? e[p * C + (C > 1 ? 1 : 0)] : 0;
+                    unsigned short c2 = C > 2 ? e[p * C + (C > 2 ? 2 : 0)] : 0, c3 = C > 3 ? e[p * C + (C > 3 ? 3 : 0)] : 0;
+                    dst[p] = make_uint2((uint32_t)c0 | ((uint32_t)c1 << 16), (uint32_t)c2 | ((uint32_t)c3 << 16));
+                }
+            }
+            fence_proxy_async_smem();                  // the tensor core reads these rows through the async proxy
+            mbar_arrive(&ctl->strip_full[sb]);
+            if (++sb == g.nstrips) { sb = 0; ph ^= 1u; }
+        }
+        if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+    } else if (warp < kWinEpiWarp0) {
+        // ---------------- MMA issuers: unit u (one M block = 128 output pixels of one row) goes to issuer u % 4
+        const int me = warp - kWinLoaders;
+        if (elect_one()) {
+            constexpr uint32_t idesc = idesc_bf16_f32(128, BN, 0, 0);
+            const uint32_t a_hi = win_desc_hi(), b_hi = smem_desc_hi_sw128(1024);
+            const uint32_t wres_lo = smem_desc_lo(smem_u32(wres), 16);
+            long long cur = row_lo;
+            WinChunk ck;
+            int sb = 0;
+            uint32_t sph = 0, u = 0;
+            bool ok = true;
+            while (ok && win_next_chunk(cur, row_hi, g.h_out, g.R, ck)) {
+                const uint32_t patch_lo = win_desc_lo(smem_u32(strips + (size_t)sb * g.strip_bytes));
+                bool have_patch = false;
+                for (int i = 0; i < ck.rows && ok; ++i)
+                    for (int cb = 0; cb < g.colblocks; ++cb, ++u) {
+                        if ((int)(u % kWinIssuers) != me) continue;
+                        if (!have_patch) {
+                            if (!mbar_wait_bounded(&ctl->strip_full[sb], sph, abort_flag)) { ok = false; break; }
+                            tc_fence_after_sync();
+                            have_patch = true;
+                        }
+                        const uint32_t slot = u % NA, use = u / NA;
+                        if (!mbar_wait_bounded(&ctl->tmem_empty[slot], (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                        tc_fence_after_sync();
+                        const uint32_t d = tmem_base + slot * BN;
+                        // A: padded row (i stride_h + r), window start = pixel 2 (128 cb) -> 16 bytes per output pixel
+                        uint32_t a_lo = patch_lo + (((uint32_t)(i * g.stride_h) * (uint32_t)g.pitch + (uint32_t)cb * 2048u) >> 4);
+                        const uint32_t pitch16 = (uint32_t)g.pitch >> 4;
+                        for (int r = 0; r < g.kh; ++r, a_lo += pitch16) {
+                            const uint32_t b_lo = wres_lo + (uint32_t)(r >> 1) * (uint32_t)(BN * 128 >> 4) + (uint32_t)(r & 1) * 4u;
+                            if (r == 0) umma_bf16_ss_halves<false>(d, a_lo, a_hi, b_lo, b_hi, idesc);
+                            else umma_bf16_ss_halves<true>(d, a_lo, a_hi, b_lo, b_hi, idesc);
+                            umma_bf16_ss_halves<true>(d, a_lo + 2u, a_hi, b_lo + 2u, b_hi, idesc);
+                        }
+                        umma_commit(&ctl->tmem_full[slot]);
+                    }
+                // this issuer's share of the patch is read once its MMAs complete (arrives at once if it had none)
+                if (ok) umma_commit(&ctl->strip_empty[sb]);
+                if (++sb == g.nstrips) { sb = 0; sph ^= 1u; }
+            }
+            if (!ok) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+        }
+    } else {
+        // ---------------- epilogue: unit u goes to warp group u % 4; tensor memory -> scale, shift -> bf16 ->
+        // swizzled staging -> TMA store of [32 pixels][64 channels] (pixels beyond the row end are clipped)
+        const int quarter = warp & 3, egroup = (warp - kWinEpiWarp0) >> 2;
+        uint8_t *buf = staging + (size_t)(warp - kWinEpiWarp0) * 4096;
+        long long cur = row_lo;
+        WinChunk ck;
+        uint32_t u = 0;
+        bool ok = true;
+        while (ok && win_next_chunk(cur, row_hi, g.h_out, g.R, ck)) {
+            for (int i = 0; i < ck.rows && ok; ++i)
+                for (int cb = 0; cb < g.colblocks; ++cb, ++u) {
+                    if ((int)(u % kWinEpiGroups) != egroup) continue;
+                    const uint32_t slot = u % NA, use = u / NA;
+                    ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->tmem_full[slot], use & 1u, abort_flag));
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const int wo0 = cb * 128 + quarter * 32;
+                    const int out_row = ck.img * g.h_out + ck.h0 + i;
+                    const uint32_t t_row = tmem_base + slot * BN + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll 1
+                    for (int c0 = 0; c0 < BN; c0 += 64) {
+                        const bool live = wo0 < g.w_out;           // else the whole box lies beyond the row end
+                        if (live) {
+                            if (lane == 0) tma_store_wait_read<0>();   // the previous store no longer reads the buffer
+                            __syncwarp();
+                        }
+                        uint8_t *row = buf + lane * 128;
+#pragma unroll 1
+                        for (int half = 0; half < 2; ++half) {
+                            uint32_t v[32];
+                            if (live) {
+                                tmem_ld_32x32(t_row + (uint32_t)(c0 + 32 * half), v);
+                                tmem_ld_wait();
+                            }
+                            if (half == 1 && c0 + 64 >= BN) {
+                                // every column of this accumulator has been read: hand it back
+                                tc_fence_before_sync();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(&ctl->tmem_empty[slot]);
+                            }
+                            if (!live) continue;
+#pragma unroll
+                            for (int j = 0; j < 32; j += 8) {
+                                const int c = c0 + 32 * half + j;
+                                const float4 s0 = *(const float4 *)(scale_s + c), s1 = *(const float4 *)(scale_s + c + 4);
+                                const float4 b0 = *(const float4 *)(bias_s + c), b1 = *(const float4 *)(bias_s + c + 4);
+                                uint4 pk;
+                                __nv_bfloat162 h;
+                                h = __floats2bfloat162_rn(fmaf(__uint_as_float(v[j]), s0.x, b0.x), fmaf(__uint_as_float(v[j + 1]), s0.y, b0.y)); pk.x = *(uint32_t *)&h;
+                                h = __floats2bfloat162_rn(fmaf(__uint_as_float(v[j + 2]), s0.z, b0.z), fmaf(__uint_as_float(v[j + 3]), s0.w, b0.w)); pk.y = *(uint32_t *)&h;
+                                h = __floats2bfloat162_rn(fmaf(__uint_as_float(v[j + 4]), s1.x, b1.x), fmaf(__uint_as_float(v[j + 5]), s1.y, b1.y)); pk.z = *(uint32_t *)&h;
+                                h = __floats2bfloat162_rn(fmaf(__uint_as_float(v[j + 6]), s1.z, b1.z), fmaf(__uint_as_float(v[j + 7]), s1.w, b1.w)); pk.w = *(uint32_t *)&h;
+                                *(uint4 *)(row + (((4 * half + (j >> 3)) ^ (lane & 7)) << 4)) = pk;
+                            }
+                        }
+                        if (!live) continue;
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            tma_store_3d(&tm_out, buf, c0, wo0, out_row);
+                            tma_store_commit();
+                        }
+                    }
+                }
+        }
+        if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+        if (lane == 0) tma_store_wait_all<0>();             // global writes done before the CTA exits
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == kWinLoaders) tmem_dealloc(ctl->tmem_base, 512);
+}
+
+// ---- host side --------------------------------------------------------------------------------------
+namespace {
+
+struct WinPlan { bool ok = false; int R = 0, nstrips = 0, pitch = 0, kblocks = 0; uint32_t strip_bytes = 0; size_t smem = 0; };
+
+WinPlan plan_window(const Problem &pb) {
+    WinPlan pl;
+    if (pb.groups != 1 || pb.c_in > 4 || pb.stride_w != 2 || pb.stride_h != 2 || pb.dil_h != 1 ||
+        pb.dil_w != 1 || pb.kw > 8 || pb.kh > 16 || (pb.c_out != 64 && pb.c_out != 128) || pb.w_in % 8 ||
+        pb.pad_w > 64 || pb.pad_h > 64 || pb.p >= (1LL << 30) || pb.pin >= (1LL << 30))
+        return pl;
+    pl.pitch = (int)(((size_t)(pb.w_in + 2 * pb.pad_w) * 8 + 15) / 16 * 16);
+    pl.kblocks = (pb.kh + 1) / 2;
+    const size_t fixed = 1024 + 16 * 4096 + sizeof(WinCtl) + 2 * (size_t)pb.c_out * sizeof(float) + 32 +
+                         (size_t)pl.kblocks * pb.c_out * 128;
+    const size_t budget = 226 * 1024;
+    for (int r = pb.h_out < 8 ? pb.h_out : 8; r >= 1; --r) {
+        const size_t rows_in = (size_t)(r - 1) * pb.stride_h + pb.kh;
+        const size_t sbytes = (rows_in * pl.pitch + kWinSlack + 1023) / 1024 * 1024;
+        if (fixed + 2 * sbytes > budget) continue;
+        int ns = (int)((budget - fixed) / sbytes);
+        if (ns > kWinMaxStrips) ns = kWinMaxStrips;
+        pl.ok = true; pl.R = r; pl.nstrips = ns; pl.strip_bytes = (uint32_t)sbytes; pl.smem = fixed + (size_t)ns * sbytes;
+        break;
+    }
+    return pl;
+}
+
+template <int BN, int C>
+cudaError_t launch_window(const CUtensorMap &tout, const WinGemm &g, size_t smem, const void *x, const void *w,
+                          const float *bias, int *err, cudaStream_t st) {
+    static PerDevice attr, carve;
+    if (cudaError_t e = max_dynamic_smem_once(stem_window_fwd_kernel<BN, C>, 227 * 1024, &attr); e != cudaSuccess) return e;
+    prefer_max_shared_once(stem_window_fwd_kernel<BN, C>, &carve);
+    const long long sms = device_sm_count();
+    const unsigned grid = (unsigned)(g.total_rows < sms ? g.total_rows : sms);
+    return launch_pdl(stem_window_fwd_kernel<BN, C>, dim3(grid), dim3(kWinThreads), smem, st, tout, g,
+                      (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w, bias, err);
+}
+
+template <int BN>
+cudaError_t launch_window_c(int c_in, const CUtensorMap &tout, const WinGemm &g, size_t smem, const void *x,
+                            const void *w, const float *bias, int *err, cudaStream_t st) {
+    switch (c_in) {
+        case 1: return launch_window<BN, 1>(tout, g, smem, x, w, bias, err, st);
+        case 2: return launch_window<BN, 2>(tout, g, smem, x, w, bias, err, st);
+        case 3: return launch_window<BN, 3>(tout, g, smem, x, w, bias, err, st);
+        default: return launch_window<BN, 4>(tout, g, smem, x, w, bias, err, st);
+    }
+}
+
+}  // namespace
+
+bool stem_window_eligible(const Problem &pb) { return plan_window(pb).ok; }
+
+cudaError_t launch_stem_window_fwd(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
+                                   cudaStream_t st, const BnFold *fold) {
+    const WinPlan pl = plan_window(pb);
+    if (!pl.ok) return cudaErrorInvalidValue;
+    WinGemm g;
+    g.n = pb.n; g.h_in = pb.h_in; g.w_in = pb.w_in; g.c_in = pb.c_in; g.h_out = pb.h_out; g.w_out = pb.w_out;
+    g.c_out = pb.c_out; g.kh = pb.kh; g.kw = pb.kw; g.stride_h = pb.stride_h; g.pad_h = pb.pad_h; g.pad_w = pb.pad_w;
+    g.R = pl.R; g.rows_in = (pl.R - 1) * pb.stride_h + pb.kh; g.pitch = pl.pitch;
+    g.colblocks = (pb.w_out + 127) / 128; g.nstrips = pl.nstrips; g.strip_bytes = pl.strip_bytes;
+    g.kblocks = pl.kblocks; g.total_rows = (long long)pb.n * pb.h_out;
+    g.fold = fold ? *fold : BnFold{nullptr, nullptr, nullptr, nullptr, nullptr, 0.f, nullptr};
+    CUtensorMap tout;
+    const unsigned long long dims[3] = {(unsigned long long)pb.c_out, (unsigned long long)pb.w_out,
+                                        (unsigned long long)pb.n * pb.h_out};
+    const unsigned long long str[3] = {0, (unsigned long long)pb.c_out * 2, (unsigned long long)pb.w_out * pb.c_out * 2};
+    const unsigned int box[3] = {64, 32, 1};
+    if (!make_tmap_tiled_bf16(&tout, z, 3, dims, str, box)) return cudaErrorInvalidValue;
+    int *err = nullptr;
+    cudaError_t e = error_word_address(&err);
+    if (e != cudaSuccess) return e;
+    if (pb.c_out == 64) return launch_window_c<64>(pb.c_in, tout, g, pl.smem, x, w, bias, err, st);
+    return launch_window_c<128>(pb.c_in, tout, g, pl.smem, x, w, bias, err, st);
+}
+
+}  // namespace convbn

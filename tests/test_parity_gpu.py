@@ -71,6 +71,13 @@ SMALL = [
     L("b_sub_c1_odd", 2, 1, 33, 45, 64, 5, 5, stride=2, pad=2),
     L("b_sub_c4", 1, 4, 40, 64, 128, 7, 7, stride=2, pad=3),
     L("b_sub_nopad", 1, 3, 38, 52, 64, 4, 4, stride=2, pad=0),
+    # stem forward with the windows formed by the operand addressing (W_in a multiple of 8, stride 2): three
+    # channels with a ragged last chunk of rows, one and two channels, an output row wider than one M block,
+    # 128 output channels, a 3x3 kernel without padding
+    L("b_win_c3", 3, 3, 38, 48, 64, 7, 7, stride=2, pad=3),
+    L("b_win_c1", 1, 1, 20, 32, 64, 5, 5, stride=2, pad=2, bias=True),
+    L("b_win_c2_wide", 1, 2, 12, 272, 64, 3, 3, stride=2, pad=1),
+    L("b_win_c4_128", 2, 4, 18, 40, 128, 3, 3, stride=2, pad=0),
     # the same regrouping for wide stride-2 layers: 128-column tiles; 64-column tiles with three
     # output-channel chunks, a 5x5 kernel and odd sizes
     L("b_sub_wide", 1, 128, 40, 58, 128, 3, 3, stride=2, pad=1),
