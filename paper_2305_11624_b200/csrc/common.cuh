@@ -120,6 +120,8 @@ inline cudaError_t max_dynamic_smem_once(K kernel, int bytes, PerDevice *flag) {
 // timestamp per CTA at the marked places; in the library it compiles to nothing.
 #ifndef CONVBN_TRACE_POINT
 #define CONVBN_TRACE_POINT(id) ((void)0)
+#define CONVBN_TRACE_T0() ((void)0)            // start of a wait ...
+#define CONVBN_TRACE_ACC(id) ((void)0)         // ... whose duration is added to slot id
 #endif
 
 static inline int ceil_div_i(long long a, long long b) { return (int)((a + b - 1) / b); }

@@ -120,6 +120,7 @@ struct Plan {
     int splits = 1, bsplits = 1, bn_splits = 1;
     size_t xpk = 0, wst = 0;   // small-C_in layers: packed input [n][hp][wp][8], expanded weights [C_out][kh][64]
     bool stem = false;
+    bool stem_win_wgrad = false;   // stem weight gradient straight from X (window operand), fused epilogue
     size_t wbd = 0;        // block-diagonal expanded weights [C_out][taps][64], storage dtype
     bool umma_wgrad = false, dw_wgrad = false, dw_tma_wgrad = false, grouped_wgrad = false, grouped8_wgrad = false;
     UmmaWgradPlan uw;
@@ -169,6 +170,15 @@ Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
         pl.uw = stem_wgrad_plan(pb);
         pl.bsplits = pl.uw.splits;
         part_bytes = (size_t)pl.uw.splits * stem_krows(pb) * 64 * pb.c_out * sizeof(float);
+        if (stem_window_wgrad_eligible(pb)) {
+            pl.stem_win_wgrad = true;
+            pl.uw = UmmaWgradPlan();
+            pl.uw.splits = stem_window_wgrad_ctas(pb);
+            wgrad_epilogue_shape(pb, &pl.uw);
+            pl.bsplits = pl.uw.splits;
+            part_bytes = wrows * pl.uw.splits * sizeof(float);
+            dot_bytes = (size_t)pl.uw.kt * pb.c_out * sizeof(float);
+        }
     }
     if (pl.umma_wgrad) {
         pl.uw = umma_wgrad_plan(pb);
@@ -508,7 +518,15 @@ int run_param_grads(const convbn_desc *d, const Problem &pb, const Plan &pl, con
     const bool tc = pl.grouped_wgrad || pl.umma_wgrad || pl.stem;   // tensor-core paths sum dZ inside the GEMM
     if (need_bsum && !tc && !pl.dw_tma_wgrad)
         LAUNCH("channel_sum", launch_channel_sum_partial(pb, d->dtype, d->layout, dz, bsum, pl.bsplits, st));
-    if (pl.stem) {
+    if (pl.stem_win_wgrad) {
+        float *dotpart = (float *)at(ws, pl.dotpart);
+        unsigned int *counters = (unsigned int *)at(ws, pl.counters);
+        LAUNCH("stem_wgrad", launch_stem_window_wgrad(pb, dz, x, partials, bsum, counters, st));
+        LAUNCH("wgrad_epilogue_fused", launch_wgrad_epilogue_fused(pb, pl.uw, partials, bsum, w, vec3, b, mean, dw,
+                                                                   dotpart, counters, db, dgamma, dbeta, need_bsum,
+                                                                   st));
+        *which = "umma-stem";
+    } else if (pl.stem) {
         LAUNCH("stem_pack", launch_stem_pack(pb, x, at(ws, pl.xpk), st));
         LAUNCH("stem_wgrad", launch_stem_wgrad(pb, pl.uw, dz, at(ws, pl.xpk), partials, bsum, st));
         LAUNCH("wgrad_epilogue_stem", launch_wgrad_epilogue_stem(pb, pl.uw, partials, bsum, w, vec3, b, mean, dw, db,

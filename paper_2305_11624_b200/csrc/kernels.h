@@ -157,6 +157,15 @@ cudaError_t launch_wgrad_epilogue_stem(const Problem &pb, const UmmaWgradPlan &p
 bool stem_window_eligible(const Problem &pb);
 cudaError_t launch_stem_window_fwd(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
                                    cudaStream_t st, const BnFold *fold = nullptr);
+// Weight gradient of the same layers (C_in <= 3, C_out = 64) straight from X and dZ: one fp32 partial
+// [kdim][C_out] and one row of sums of dZ per CTA (stem_window_wgrad_ctas of them), in the layout the fused
+// epilogue of the dense weight-gradient path reads; `counters` are zeroed for it.
+bool stem_window_wgrad_eligible(const Problem &pb);
+int stem_window_wgrad_ctas(const Problem &pb);
+cudaError_t launch_stem_window_wgrad(const Problem &pb, const void *dz, const void *x, float *partials, float *bsum,
+                                     unsigned int *counters, cudaStream_t st);
+// k rows per block (kr) and row blocks (kt) of the fused epilogue for pl.splits partial tiles
+void wgrad_epilogue_shape(const Problem &pb, UmmaWgradPlan *pl);
 cudaError_t launch_stem_fwd(const Problem &pb, const void *x_packed, const void *wst, const float *bias, void *out,
                             cudaStream_t st, const BnFold *fold = nullptr);
 

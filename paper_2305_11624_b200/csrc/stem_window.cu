@@ -66,6 +66,45 @@ __device__ __forceinline__ bool win_next_chunk(long long &cur, long long hi, int
     return true;
 }
 
+// Fills `count` rows of a patch buffer with input rows first, first + 1, ... of image img: pixels of C channels
+// widened to 4 (8 bytes) behind a left border of pad_w pixels; rows outside the image are zero.  fill3 is the
+// bit pattern of channel slot 3 (C <= 3 only): 0, or bf16 1.0 when the weight-gradient GEMM takes sum dZ from it
+// (then the caller has also set it in the borders).  Called by nthreads threads with ids tid.
+template <int C>
+__device__ __forceinline__ void win_fill_patch(uint8_t *patch, const __nv_bfloat16 *__restrict__ x, int img, int first,
+                                               int count, int h_in, int w_in, int pad_w, int pitch, int tid, int nthreads,
+                                               uint32_t fill3) {
+    const int chunks_w = w_in / 8, tasks = count * chunks_w;
+    const uint32_t hi_fill = fill3 << 16;
+#pragma unroll 4
+    for (int t = tid; t < tasks; t += nthreads) {
+        const int pr = t / chunks_w, j = t - pr * chunks_w, h = first + pr;
+        uint2 *dst = (uint2 *)(patch + (size_t)pr * pitch + (size_t)(pad_w + 8 * j) * 8);
+        if (h < 0 || h >= h_in) {
+#pragma unroll
+            for (int p = 0; p < 8; ++p) dst[p] = make_uint2(0, hi_fill);
+            continue;
+        }
+        const uint4 *src = (const uint4 *)(x + (((size_t)img * h_in + h) * w_in + 8 * j) * C);
+        unsigned short e[8 * C];
+#pragma unroll
+        for (int v = 0; v < C; ++v) {
+            const uint4 q4 = __ldg(src + v);
+            e[8 * v + 0] = (unsigned short)q4.x; e[8 * v + 1] = (unsigned short)(q4.x >> 16);
+            e[8 * v + 2] = (unsigned short)q4.y; e[8 * v + 3] = (unsigned short)(q4.y >> 16);
+            e[8 * v + 4] = (unsigned short)q4.z; e[8 * v + 5] = (unsigned short)(q4.z >> 16);
+            e[8 * v + 6] = (unsigned short)q4.w; e[8 * v + 7] = (unsigned short)(q4.w >> 16);
+        }
+#pragma unroll
+        for (int p = 0; p < 8; ++p) {
+            const unsigned short c0 = e[p * C], c1 = C > 1 ? e[p * C + (C > 1 ? 1 : 0)] : (unsigned short)0;
+            const unsigned short c2 = C > 2 ? e[p * C + (C > 2 ? 2 : 0)] : (unsigned short)0;
+            const uint32_t w1 = C > 3 ? ((uint32_t)c2 | ((uint32_t)e[p * C + (C > 3 ? 3 : 0)] << 16)) : ((uint32_t)c2 | hi_fill);
+            dst[p] = make_uint2((uint32_t)c0 | ((uint32_t)c1 << 16), w1);
+        }
+    }
+}
+
 template <int BN, int C>
 __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __grid_constant__ CUtensorMap tm_out,
                                                                      const WinGemm g,
@@ -88,6 +127,7 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
 
     if (warp < kWinLoaders) {
         if (threadIdx.x == 0) {
+            CONVBN_TRACE_POINT(0);
             for (int s = 0; s < kWinMaxStrips; ++s) { mbar_init(&ctl->strip_full[s], 32 * kWinLoaders); mbar_init(&ctl->strip_empty[s], kWinIssuers); }
             for (int s = 0; s < 8; ++s) { mbar_init(&ctl->tmem_full[s], 1); mbar_init(&ctl->tmem_empty[s], 4); }
             ctl->abort_flag = 0;
@@ -110,6 +150,7 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
         tmem_relinquish();
     }
     pdl_wait();
+    if (threadIdx.x == 0) CONVBN_TRACE_POINT(1);
     uint32_t tmem_base = 0;
     if (warp >= kWinLoaders) {
         if (warp >= kWinEpiWarp0) {
@@ -129,15 +170,28 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
             } else {
                 for (int c = tid; c < BN; c += nt) { bias_s[c] = bias ? bias[c] : 0.f; scale_s[c] = 1.f; }
             }
-            // resident weights: K index = r 32 + q 4 + c, two filter rows per 128-byte row, zeros in unused slots
-            const int slots = g.kblocks * BN * 64;
-            for (int i = tid; i < slots; i += nt) {
-                const int k64 = i & 63, co = (i >> 6) % BN, kb = (i >> 6) / BN;
-                const int r = kb * 2 + (k64 >> 5), q = (k64 & 31) >> 2, c = k64 & 3;
-                unsigned short v = 0;
-                if (r < g.kh && q < g.kw && c < C)
-                    v = ((const unsigned short *)w)[(((size_t)co * g.kh + r) * g.kw + q) * C + c];
-                *(unsigned short *)(wres + (size_t)kb * BN * 128 + co * 128 + ((((k64 >> 3) ^ (co & 7)) & 7) << 4) + (k64 & 7) * 2) = v;
+            // resident weights: K index = r 32 + q 4 + c, two filter rows per 128-byte row, zeros in unused slots.
+            // Zero everything, then scatter the real entries (consecutive threads read consecutive elements; the
+            // loads of a batch are issued together).
+            {
+                uint4 *z4 = (uint4 *)wres;
+                for (int i = tid; i < g.kblocks * BN * 8; i += nt) z4[i] = make_uint4(0, 0, 0, 0);
+            }
+            named_bar_sync(4, nt);
+            const int rowlen = g.kh * g.kw * C, total = BN * rowlen;
+            const unsigned short *wsrc = (const unsigned short *)w;
+            for (int base = tid; base < total; base += 8 * nt) {
+                unsigned short val[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) val[k] = base + k * nt < total ? __ldg(wsrc + base + k * nt) : (unsigned short)0;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const int e = base + k * nt;
+                    if (e >= total) break;
+                    const int co = e / rowlen, rem = e - co * rowlen, c = rem % C, t2 = rem / C, q = t2 % g.kw, r = t2 / g.kw;
+                    const int k64 = (r & 1) * 32 + q * 4 + c, kb = r >> 1;
+                    *(unsigned short *)(wres + (size_t)kb * BN * 128 + co * 128 + ((((k64 >> 3) ^ (co & 7)) & 7) << 4) + (k64 & 7) * 2) = val[k];
+                }
             }
             fence_proxy_async_smem();
         }
@@ -146,50 +200,27 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
         tc_fence_after_sync();
         pdl_launch_dependents();       // only now: this CTA owns its tensor-memory columns
         tmem_base = ctl->tmem_base;
+        if (threadIdx.x == 32 * kWinLoaders) CONVBN_TRACE_POINT(2);
     }
 
     if (warp < kWinLoaders) {
         // ---------------- input-row loaders ----------------
-        const int ltid = threadIdx.x, chunks_w = g.w_in / 8;
+        const int ltid = threadIdx.x;
         long long cur = row_lo;
         WinChunk ck;
         int sb = 0;
         uint32_t ph = 0;
         bool ok = true;
         while (ok && win_next_chunk(cur, row_hi, g.h_out, g.R, ck)) {
+            { CONVBN_TRACE_T0();
             ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->strip_empty[sb], ph ^ 1u, abort_flag));
+            if (threadIdx.x == 0) CONVBN_TRACE_ACC(12); }
             if (!ok) break;
-            uint8_t *patch = strips + (size_t)sb * g.strip_bytes;
-            const int first = ck.h0 * g.stride_h - g.pad_h, count = (ck.rows - 1) * g.stride_h + g.kh;
-            const int tasks = count * chunks_w;
-#pragma unroll 2
-            for (int t = ltid; t < tasks; t += 32 * kWinLoaders) {
-                const int pr = t / chunks_w, j = t - pr * chunks_w, h = first + pr;
-                uint2 *dst = (uint2 *)(patch + (size_t)pr * g.pitch + (size_t)(g.pad_w + 8 * j) * 8);
-                if (h < 0 || h >= g.h_in) {
-#pragma unroll
-                    for (int p = 0; p < 8; ++p) dst[p] = make_uint2(0, 0);
-                    continue;
-                }
-                const uint4 *src = (const uint4 *)(x + (((size_t)ck.img * g.h_in + h) * g.w_in + 8 * j) * C);
-                unsigned short e[8 * C];
-#pragma unroll
-                for (int v = 0; v < C; ++v) {
-                    const uint4 q4 = __ldg(src + v);
-                    e[8 * v + 0] = (unsigned short)q4.x; e[8 * v + 1] = (unsigned short)(q4.x >> 16);
-                    e[8 * v + 2] = (unsigned short)q4.y; e[8 * v + 3] = (unsigned short)(q4.y >> 16);
-                    e[8 * v + 4] = (unsigned short)q4.z; e[8 * v + 5] = (unsigned short)(q4.z >> 16);
-                    e[8 * v + 6] = (unsigned short)q4.w; e[8 * v + 7] = (unsigned short)(q4.w >> 16);
-                }
-#pragma unroll
-                for (int p = 0; p < 8; ++p) {
-                    unsigned short c0 = e[p * C], c1 = C > 1 ? e[p * C + (C > 1 ? 1 : 0)] : 0;
-                    unsigned short c2 = C > 2 ? e[p * C + (C > 2 ? 2 : 0)] : 0, c3 = C > 3 ? e[p * C + (C > 3 ? 3 : 0)] : 0;
-                    dst[p] = make_uint2((uint32_t)c0 | ((uint32_t)c1 << 16), (uint32_t)c2 | ((uint32_t)c3 << 16));
-                }
-            }
+            win_fill_patch<C>(strips + (size_t)sb * g.strip_bytes, x, ck.img, ck.h0 * g.stride_h - g.pad_h,
+                              (ck.rows - 1) * g.stride_h + g.kh, g.h_in, g.w_in, g.pad_w, g.pitch, ltid, 32 * kWinLoaders, 0);
             fence_proxy_async_smem();                  // the tensor core reads these rows through the async proxy
             mbar_arrive(&ctl->strip_full[sb]);
+            if (threadIdx.x == 0) { if (sb == 0 && ph == 0) CONVBN_TRACE_POINT(3); CONVBN_TRACE_POINT(8); }
             if (++sb == g.nstrips) { sb = 0; ph ^= 1u; }
         }
         if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
@@ -212,12 +243,17 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
                     for (int cb = 0; cb < g.colblocks; ++cb, ++u) {
                         if ((int)(u % kWinIssuers) != me) continue;
                         if (!have_patch) {
+                            { CONVBN_TRACE_T0();
                             if (!mbar_wait_bounded(&ctl->strip_full[sb], sph, abort_flag)) { ok = false; break; }
+                            if (me == 0) CONVBN_TRACE_ACC(13); }
                             tc_fence_after_sync();
+                            if (me == 0 && u == 0) CONVBN_TRACE_POINT(4);
                             have_patch = true;
                         }
                         const uint32_t slot = u % NA, use = u / NA;
+                        { CONVBN_TRACE_T0();
                         if (!mbar_wait_bounded(&ctl->tmem_empty[slot], (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                        if (me == 0) CONVBN_TRACE_ACC(14); }
                         tc_fence_after_sync();
                         const uint32_t d = tmem_base + slot * BN;
                         // A: padded row (i stride_h + r), window start = pixel 2 (128 cb) -> 16 bytes per output pixel
@@ -233,6 +269,7 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
                     }
                 // this issuer's share of the patch is read once its MMAs complete (arrives at once if it had none)
                 if (ok) umma_commit(&ctl->strip_empty[sb]);
+                if (me == 0) { if (sb == 0 && sph == 0) CONVBN_TRACE_POINT(5); CONVBN_TRACE_POINT(6); }
                 if (++sb == g.nstrips) { sb = 0; sph ^= 1u; }
             }
             if (!ok) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
@@ -251,7 +288,9 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
                 for (int cb = 0; cb < g.colblocks; ++cb, ++u) {
                     if ((int)(u % kWinEpiGroups) != egroup) continue;
                     const uint32_t slot = u % NA, use = u / NA;
+                    { CONVBN_TRACE_T0();
                     ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->tmem_full[slot], use & 1u, abort_flag));
+                    if (warp == kWinEpiWarp0 && lane == 0) CONVBN_TRACE_ACC(15); }
                     if (!ok) break;
                     tc_fence_after_sync();
                     const int wo0 = cb * 128 + quarter * 32;
@@ -304,11 +343,216 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
                 }
         }
         if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+        if (warp == kWinEpiWarp0 && lane == 0) CONVBN_TRACE_POINT(9);
         if (lane == 0) tma_store_wait_all<0>();             // global writes done before the CTA exits
+        if (warp == kWinEpiWarp0 && lane == 0) CONVBN_TRACE_POINT(10);
     }
     tc_fence_before_sync();
     __syncthreads();
+    if (threadIdx.x == 0) CONVBN_TRACE_POINT(11);
     if (warp == kWinLoaders) tmem_dealloc(ctl->tmem_base, 512);
+}
+
+// ---- weight gradient of the same layers ---------------------------------------------------------------
+// domega'[co][r][q][c] = sum over images and output pixels of dZ[ho][wo][co] X[2 ho + r][2 wo + q][c]  (Sec. 3.2.1;
+// Table 2, Tune row), with the same zero-bordered 4-channel rows in shared memory.  For one input row the
+// A operand is MN-major without swizzle: element (m, k) with m = 4 q + c and k = wo sits at  start + 2 m + 16 k,
+// i.e. the contraction runs along the output pixels of a row and the 128 M rows are window offsets (the first
+// kw x 4 are the taps, the rest is ignored).  The B operand is the dZ row(s) that meet this input row, [wo][co]
+// in 128-byte-swizzled rows: input row 2 ho + r serves ceil(kh / 2) or floor(kh / 2) output rows at once, which
+// lie one after the other in the chunk's dZ buffer, so ONE MMA of N = 64 x (rows) updates all their taps:
+// accumulator column block j of parity class e = r & 1 holds tap r = e + 2 (T_e - 1 - j).
+// Channel slot 3 of every padded pixel holds 1.0 (C <= 3), so accumulator row m = 3 of tap 0 is sum dZ.
+// Each CTA accumulates its contiguous range of output rows in tensor memory and writes one fp32 partial
+// [k][co] plus one row of sums; the fused epilogue kernel adds the CTAs' partials in fixed order.
+constexpr int kWgR = 4;                  // output rows per chunk
+constexpr int kWgThreads = 256;          // warps 0-3 X loaders, 4 tensor memory + read-out, 5 dZ producer, 6-7 issuers
+
+struct WinWgrad {
+    int n, h_in, w_in, h_out, w_out, c_out, kh, kw, pad_h, pad_w;
+    int pitch, ksteps, T0, T1, kdim;
+    uint32_t xstrip_bytes, dzrow_bytes;
+    long long total_rows;
+};
+
+struct WinWgCtl {
+    uint64_t x_full[2], x_empty[2], dz_full[2], dz_empty[2], acc_done;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+template <int C>
+__global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __grid_constant__ CUtensorMap tm_dz,
+                                                                      const WinWgrad g,
+                                                                      const __nv_bfloat16 *__restrict__ x,
+                                                                      float *__restrict__ partials,
+                                                                      float *__restrict__ bsum,
+                                                                      unsigned int *__restrict__ counters, int ncounters,
+                                                                      int *err) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *xs = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *dzs = xs + 2 * (size_t)g.xstrip_bytes;
+    const uint32_t dzstrip = kWgR * g.dzrow_bytes;
+    uint8_t *zeros = dzs + 2 * (size_t)dzstrip;                 // 16 zero rows of 128 bytes
+    WinWgCtl *ctl = (WinWgCtl *)(zeros + 2048);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int *abort_flag = &ctl->abort_flag;
+    const long long row_lo = g.total_rows * blockIdx.x / gridDim.x, row_hi = g.total_rows * (blockIdx.x + 1) / gridDim.x;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&ctl->x_full[s], 128); mbar_init(&ctl->x_empty[s], 2);
+            mbar_init(&ctl->dz_full[s], 1); mbar_init(&ctl->dz_empty[s], 2);
+        }
+        mbar_init(&ctl->acc_done, 2);
+        ctl->abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&tm_dz);
+    }
+    // every padded pixel starts as (0, 0, 0, 1): borders, rows outside the image and the slack keep that
+    {
+        uint4 *p4 = (uint4 *)xs;
+        const int n16 = (int)(2 * (size_t)g.xstrip_bytes / 16);
+        for (int i = threadIdx.x; i < n16; i += kWgThreads) p4[i] = make_uint4(0, 0x3F800000u, 0, 0x3F800000u);
+        uint4 *z4 = (uint4 *)zeros;
+        for (int i = threadIdx.x; i < 128; i += kWgThreads) z4[i] = make_uint4(0, 0, 0, 0);
+    }
+    fence_proxy_async_smem();
+    if (warp == 4) {
+        tmem_alloc(&ctl->tmem_base, 512);
+        tmem_relinquish();
+    }
+    pdl_wait();
+    if (counters && blockIdx.x == 0)
+        for (int i = threadIdx.x; i < ncounters; i += kWgThreads) counters[i] = 0u;
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    pdl_launch_dependents();       // only now: this CTA owns its tensor-memory columns
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp < 4) {
+        // ---------------- X row loaders ----------------
+        long long cur = row_lo;
+        WinChunk ck;
+        int sb = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        while (ok && win_next_chunk(cur, row_hi, g.h_out, kWgR, ck)) {
+            ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->x_empty[sb], ph ^ 1u, abort_flag));
+            if (!ok) break;
+            win_fill_patch<C>(xs + (size_t)sb * g.xstrip_bytes, x, ck.img, ck.h0 * 2 - g.pad_h, (ck.rows - 1) * 2 + g.kh,
+                              g.h_in, g.w_in, g.pad_w, g.pitch, (int)threadIdx.x, 128, 0x3F80u);
+            fence_proxy_async_smem();
+            mbar_arrive(&ctl->x_full[sb]);
+            if (++sb == 2) { sb = 0; ph ^= 1u; }
+        }
+        if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+    } else if (warp == 5) {
+        // ---------------- dZ producer: one TMA box per output row of the chunk ----------------
+        if (elect_one()) {
+            long long cur = row_lo;
+            WinChunk ck;
+            int sb = 0, issued = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            while (ok && win_next_chunk(cur, row_hi, g.h_out, kWgR, ck)) {
+                if (!mbar_wait_bounded(&ctl->dz_empty[sb], ph ^ 1u, abort_flag)) { ok = false; break; }
+                mbar_arrive_expect_tx(&ctl->dz_full[sb], (uint32_t)ck.rows * g.dzrow_bytes);
+                for (int i = 0; i < ck.rows; ++i)
+                    tma_load_3d(dzs + (size_t)sb * dzstrip + (size_t)i * g.dzrow_bytes, &tm_dz, &ctl->dz_full[sb], 0, 0,
+                                ck.img * g.h_out + ck.h0 + i);
+                ++issued;
+                if (++sb == 2) { sb = 0; ph ^= 1u; }
+            }
+            if (!ok) {
+                atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1;
+                // let the copies already issued land (bounded) before the CTA may exit
+                for (int j = issued > 2 ? issued - 2 : 0; j < issued; ++j)
+                    mbar_wait_bounded(&ctl->dz_full[j & 1], (uint32_t)(j >> 1) & 1u, nullptr, 200000000ull);
+            }
+        }
+    } else if (warp >= 6) {
+        // ---------------- MMA issuers: warp 6 the even input rows of a patch, warp 7 the odd ones ----------------
+        const int e = warp - 6, Te = e ? g.T1 : g.T0;
+        if (elect_one()) {
+            const uint32_t acc = tmem_base + (uint32_t)e * 256u;
+            // A: MN-major, no swizzle: 8 M elements per 16 bytes, next 8 M elements 16 bytes on, next 8 pixels 128 bytes on
+            const uint32_t a_hi = (16u >> 4) | (1u << 14), a_lbo = (128u >> 4) << 16;
+            const uint32_t b_hi = smem_desc_hi_sw128(1024);
+            // all accumulator columns of this class start from zero: one MMA against 16 zero rows (block stride 0)
+            umma_bf16_ss_halves<false>(acc, ((smem_u32(xs) >> 4) & 0x3FFFu) | a_lbo, a_hi, smem_desc_lo(smem_u32(zeros), 0), b_hi,
+                                       idesc_bf16_f32(128, 64 * Te, 1, 1));
+            long long cur = row_lo;
+            WinChunk ck;
+            int sb = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            while (ok && win_next_chunk(cur, row_hi, g.h_out, kWgR, ck)) {
+                if (!mbar_wait_bounded(&ctl->x_full[sb], ph, abort_flag) || !mbar_wait_bounded(&ctl->dz_full[sb], ph, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after_sync();
+                const uint32_t xa = smem_u32(xs + (size_t)sb * g.xstrip_bytes), dza = smem_u32(dzs + (size_t)sb * dzstrip);
+                const int count = (ck.rows - 1) * 2 + g.kh;
+                for (int pr = e; pr < count; pr += 2) {
+                    const int i_max = (pr - e) >> 1;
+                    int t_lo = i_max - ck.rows + 1, t_hi = i_max;
+                    if (t_lo < 0) t_lo = 0;
+                    if (t_hi > Te - 1) t_hi = Te - 1;
+                    if (t_lo > t_hi) continue;
+                    const int nblk = t_hi - t_lo + 1, i_lo = i_max - t_hi, cb_lo = Te - 1 - t_hi;
+                    const uint32_t idesc = idesc_bf16_f32(128, 64 * nblk, 1, 1);
+                    const uint32_t d = acc + 64u * (uint32_t)cb_lo;
+                    uint32_t a_lo = (((xa + (uint32_t)pr * (uint32_t)g.pitch) >> 4) & 0x3FFFu) | a_lbo;
+                    uint32_t b_lo = smem_desc_lo(dza + (uint32_t)i_lo * g.dzrow_bytes, g.dzrow_bytes);
+                    for (int k = 0; k < g.ksteps; ++k, a_lo += 16u, b_lo += 128u)     // 16 pixels: 256 / 2048 bytes
+                        umma_bf16_ss_halves<true>(d, a_lo, a_hi, b_lo, b_hi, idesc);
+                }
+                umma_commit(&ctl->x_empty[sb]);
+                umma_commit(&ctl->dz_empty[sb]);
+                if (++sb == 2) { sb = 0; ph ^= 1u; }
+            }
+            if (ok) umma_commit(&ctl->acc_done);
+            else { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+        }
+    } else {
+        // ---------------- read-out (warp 4 = lanes 0-31 of tensor memory = window offsets m = 0 .. 31) ----------------
+        const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->acc_done, 0, abort_flag));
+        if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+        if (ok) {
+            tc_fence_after_sync();
+            const int q = lane >> 2, c = lane & 3;
+            const bool tap_ok = q < g.kw && c < C;
+            for (int e = 0; e < 2; ++e) {
+                const int Te = e ? g.T1 : g.T0;
+                for (int cbk = 0; cbk < Te; ++cbk) {
+                    const int r = e + 2 * (Te - 1 - cbk);
+                    const int k = (r * g.kw + q) * C + c;
+                    float *orow = partials + ((size_t)blockIdx.x * g.kdim + (tap_ok ? k : 0)) * 64;
+                    float *brow = bsum + (size_t)blockIdx.x * 64;
+                    const bool sum_row = C < 4 && r == 0 && lane == 3;
+#pragma unroll 1
+                    for (int c0 = 0; c0 < 64; c0 += 32) {
+                        uint32_t v[32];
+                        tmem_ld_32x32(tmem_base + (uint32_t)(e * 256 + cbk * 64 + c0), v);
+                        tmem_ld_wait();
+                        if (tap_ok) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) *(uint4 *)(orow + c0 + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                        } else if (sum_row) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) *(uint4 *)(brow + c0 + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 4) tmem_dealloc(tmem_base, 512);
 }
 
 // ---- host side --------------------------------------------------------------------------------------
@@ -365,6 +609,65 @@ cudaError_t launch_window_c(int c_in, const CUtensorMap &tout, const WinGemm &g,
 }  // namespace
 
 bool stem_window_eligible(const Problem &pb) { return plan_window(pb).ok; }
+
+namespace {
+struct WinWgPlan { bool ok = false; int pitch = 0, ksteps = 0; uint32_t xstrip = 0, dzrow = 0; size_t smem = 0; };
+WinWgPlan plan_window_wgrad(const Problem &pb) {
+    WinWgPlan pl;
+    if (!plan_window(pb).ok || pb.c_in > 3 || pb.c_out != 64 || pb.kh < 2 || pb.kh > 8 || pb.w_out > 256) return pl;
+    pl.pitch = (int)(((size_t)(pb.w_in + 2 * pb.pad_w) * 8 + 15) / 16 * 16);
+    pl.ksteps = (pb.w_out + 15) / 16;
+    pl.xstrip = (uint32_t)((((size_t)(kWgR - 1) * 2 + pb.kh) * pl.pitch + kWinSlack + 1023) / 1024 * 1024);
+    pl.dzrow = (uint32_t)pl.ksteps * 16 * 128;
+    pl.smem = 1024 + 2 * (size_t)pl.xstrip + 2 * (size_t)kWgR * pl.dzrow + 2048 + sizeof(WinWgCtl) + 64;
+    pl.ok = pl.smem <= 226 * 1024;
+    return pl;
+}
+}  // namespace
+
+bool stem_window_wgrad_eligible(const Problem &pb) { return plan_window_wgrad(pb).ok; }
+
+// (one function per channel count: the once-per-device flags must not be shared between the kernels)
+template <int C>
+static cudaError_t launch_window_wgrad(const CUtensorMap &tdz, const WinWgrad &g, size_t smem, unsigned grid, const void *x,
+                                       float *partials, float *bsum, unsigned int *counters, int *err, cudaStream_t st) {
+    static PerDevice attr, carve;
+    if (cudaError_t e = max_dynamic_smem_once(stem_window_wgrad_kernel<C>, 227 * 1024, &attr); e != cudaSuccess) return e;
+    prefer_max_shared_once(stem_window_wgrad_kernel<C>, &carve);
+    return launch_pdl(stem_window_wgrad_kernel<C>, dim3(grid), dim3(kWgThreads), smem, st, tdz, g,
+                      (const __nv_bfloat16 *)x, partials, bsum, counters, g.c_out / 32, err);
+}
+
+int stem_window_wgrad_ctas(const Problem &pb) {
+    const long long rows = (long long)pb.n * pb.h_out, sms = device_sm_count();
+    return (int)(rows < sms ? rows : sms);
+}
+
+cudaError_t launch_stem_window_wgrad(const Problem &pb, const void *dz, const void *x, float *partials, float *bsum,
+                                     unsigned int *counters, cudaStream_t st) {
+    const WinWgPlan pl = plan_window_wgrad(pb);
+    if (!pl.ok) return cudaErrorInvalidValue;
+    WinWgrad g;
+    g.n = pb.n; g.h_in = pb.h_in; g.w_in = pb.w_in; g.h_out = pb.h_out; g.w_out = pb.w_out; g.c_out = pb.c_out;
+    g.kh = pb.kh; g.kw = pb.kw; g.pad_h = pb.pad_h; g.pad_w = pb.pad_w; g.pitch = pl.pitch; g.ksteps = pl.ksteps;
+    g.T0 = (pb.kh + 1) / 2; g.T1 = pb.kh / 2; g.kdim = pb.kdim; g.xstrip_bytes = pl.xstrip; g.dzrow_bytes = pl.dzrow;
+    g.total_rows = (long long)pb.n * pb.h_out;
+    CUtensorMap tdz;
+    const unsigned long long dims[3] = {(unsigned long long)pb.c_out, (unsigned long long)pb.w_out,
+                                        (unsigned long long)pb.n * pb.h_out};
+    const unsigned long long str[3] = {0, (unsigned long long)pb.c_out * 2, (unsigned long long)pb.w_out * pb.c_out * 2};
+    const unsigned int box[3] = {64, (unsigned)pl.ksteps * 16, 1};
+    if (!make_tmap_tiled_bf16(&tdz, dz, 3, dims, str, box)) return cudaErrorInvalidValue;
+    int *err = nullptr;
+    cudaError_t e = error_word_address(&err);
+    if (e != cudaSuccess) return e;
+    const unsigned grid = (unsigned)stem_window_wgrad_ctas(pb);
+    switch (pb.c_in) {
+        case 1: return launch_window_wgrad<1>(tdz, g, pl.smem, grid, x, partials, bsum, counters, err, st);
+        case 2: return launch_window_wgrad<2>(tdz, g, pl.smem, grid, x, partials, bsum, counters, err, st);
+        default: return launch_window_wgrad<3>(tdz, g, pl.smem, grid, x, partials, bsum, counters, err, st);
+    }
+}
 
 cudaError_t launch_stem_window_fwd(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
                                    cudaStream_t st, const BnFold *fold) {

@@ -267,12 +267,16 @@ UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
     per = (per + kWP - 1) / kWP * kWP;
     pl.per_split = per;
     pl.splits = (int)((pb.p + per - 1) / per);
-    // k rows per epilogue block (the block's other lanes split the slices): very many slices -> 2 rows x 16
-    // lanes; few slices or very many blocks -> 32 rows x 1 lane (every block pays a fence and an atomic)
-    const long long blocks8 = (long long)(pb.c_out / 32) * ((pb.kdim + 7) / 8);
-    pl.kr = pl.splits > 192 ? 2 : ((pl.splits <= 8 || blocks8 > 1200) && blocks8 / 4 >= device_sm_count() ? 32 : 8);
-    pl.kt = (pb.kdim + pl.kr - 1) / pl.kr;   // epilogue blocks along k = rows of dotpart
+    wgrad_epilogue_shape(pb, &pl);
     return pl;
+}
+
+// k rows per epilogue block (the block's other lanes split the slices): very many slices -> 2 rows x 16
+// lanes; few slices or very many blocks -> 32 rows x 1 lane (every block pays a fence and an atomic)
+void wgrad_epilogue_shape(const Problem &pb, UmmaWgradPlan *pl) {
+    const long long blocks8 = (long long)(pb.c_out / 32) * ((pb.kdim + 7) / 8);
+    pl->kr = pl->splits > 192 ? 2 : ((pl->splits <= 8 || blocks8 > 1200) && blocks8 / 4 >= device_sm_count() ? 32 : 8);
+    pl->kt = (pb.kdim + pl->kr - 1) / pl->kr;   // epilogue blocks along k = rows of dotpart
 }
 
 template <int BN>
