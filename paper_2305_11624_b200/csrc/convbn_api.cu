@@ -376,7 +376,11 @@ int run_conv_fwd(const convbn_desc *d, const Problem &pb, const void *x, const v
 int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, const void *w, const float *scale,
                    void *w_scratch, void *wbd_scratch, void *dx, cudaStream_t st, const char **which) {
     UmmaConvShape s;
-    if (stem_path(d, pb) && subpixel_dgrad_shape(pb, &s) && umma_strip_eligible(s)) {
+    if (stem_path(d, pb) && stem_window_dgrad_eligible(pb)) {
+        // stride 2, C_in <= 4: scatter GEMM over dZ rows, window positions added up on chip
+        LAUNCH("stem_dgrad", launch_stem_window_dgrad(pb, dz, w, scale, dx, st));
+        *which = "umma-stem";
+    } else if (stem_path(d, pb) && subpixel_dgrad_shape(pb, &s) && umma_strip_eligible(s)) {
         // stride 2, C_in <= 4: one stride-1 convolution over dZ whose 16 output columns are the four
         // parity classes of the input position
         LAUNCH("subpixel_weights", launch_subpixel_weights(pb, w, scale, w_scratch, st));

@@ -164,6 +164,11 @@ bool stem_window_wgrad_eligible(const Problem &pb);
 int stem_window_wgrad_ctas(const Problem &pb);
 cudaError_t launch_stem_window_wgrad(const Problem &pb, const void *dz, const void *x, float *partials, float *bsum,
                                      unsigned int *counters, cudaStream_t st);
+// Backward data of the same layers (C_out = 64, W_out <= 128) as a scatter GEMM with the overlap-add of the
+// window positions done on chip (see stem_window_dgrad.cu); s_vec (NULL = 1) is folded into the weights.
+bool stem_window_dgrad_eligible(const Problem &pb);
+cudaError_t launch_stem_window_dgrad(const Problem &pb, const void *dz, const void *w, const float *s_vec, void *dx,
+                                     cudaStream_t st);
 // k rows per block (kr) and row blocks (kt) of the fused epilogue for pl.splits partial tiles
 void wgrad_epilogue_shape(const Problem &pb, UmmaWgradPlan *pl);
 cudaError_t launch_stem_fwd(const Problem &pb, const void *x_packed, const void *wst, const float *bias, void *out,

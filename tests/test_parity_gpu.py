@@ -78,6 +78,9 @@ SMALL = [
     L("b_win_c1", 1, 1, 20, 32, 64, 5, 5, stride=2, pad=2, bias=True),
     L("b_win_c2_wide", 1, 2, 12, 272, 64, 3, 3, stride=2, pad=1),
     L("b_win_c4_128", 2, 4, 18, 40, 128, 3, 3, stride=2, pad=0),
+    # ... an even kernel without padding whose last input row no output row reaches, four channels with 64 outputs
+    L("b_win_tail", 2, 3, 21, 40, 64, 4, 4, stride=2, pad=0),
+    L("b_win_c4_64", 3, 4, 26, 56, 64, 7, 7, stride=2, pad=3, bias=True),
     # the same regrouping for wide stride-2 layers: 128-column tiles; 64-column tiles with three
     # output-channel chunks, a 5x5 kernel and odd sizes
     L("b_sub_wide", 1, 128, 40, 58, 128, 3, 3, stride=2, pad=1),
