@@ -228,6 +228,13 @@ int convbn_profile_end(char *report, size_t report_bytes);
  * invalid) or CONVBN_ECUDA (the stream reported an error). */
 int convbn_check(void *stream);
 
+/* Self-test of the failure path (the paper has no counterpart): launches one block whose single bounded wait
+ * - the same mbarrier wait the tensor-core kernels use, with a limit of about 100 microseconds - is on a
+ * barrier that nobody arrives at.  The wait gives up, the kernel sets the device error word and returns
+ * normally; nothing faults and the context stays usable.  The next convbn_check(stream) therefore reports
+ * CONVBN_ETIMEOUT (and clears the word).  No copy or tensor-memory operation is in flight at any time. */
+int convbn_selftest_wait_timeout(void *stream);
+
 /* Static, NUL-terminated description of a status code. */
 const char *convbn_status_string(int status);
 

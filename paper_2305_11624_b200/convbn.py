@@ -25,7 +25,7 @@ EXPORTS = (
     "convbn_deploy_prepare", "convbn_deploy_fwd", "convbn_deploy_bwd", "convbn_check",
     "convbn_status_string", "convbn_last_kernel", "convbn_host_step_arena_bytes",
     "convbn_tune_step_host", "convbn_profile_begin", "convbn_profile_end",
-    "convbn_tune_bwd_weight_noalloc",
+    "convbn_tune_bwd_weight_noalloc", "convbn_selftest_wait_timeout",
 )
 
 
@@ -203,6 +203,11 @@ def convbn_deploy_bwd(desc, dz, x, w_fused, dx, dw_fused, db_fused, workspace=No
 
 def convbn_check(stream=None) -> None:
     _raise(lib().convbn_check(_stream(stream)), "convbn_check")
+
+
+def convbn_selftest_wait_timeout(stream=None) -> None:
+    """Queue the failure-path self-test: the next convbn_check() raises ConvBNError(ETIMEOUT)."""
+    _raise(lib().convbn_selftest_wait_timeout(_stream(stream)), "convbn_selftest_wait_timeout")
 
 
 def convbn_host_step_arena_bytes(desc: Desc) -> int:

@@ -820,6 +820,11 @@ int convbn_check(void *stream) {
     return (word & ERRW_TIMEOUT) ? CONVBN_ETIMEOUT : CONVBN_OK;
 }
 
+int convbn_selftest_wait_timeout(void *stream) {
+    if (launch_selftest_wait_timeout(100000ull, (cudaStream_t)stream) != cudaSuccess) return CONVBN_ECUDA;
+    return CONVBN_OK;
+}
+
 int convbn_profile_begin(void) {
     std::lock_guard<std::mutex> lk(g_prof_mu);
     for (auto &r : g_prof.recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }

@@ -257,4 +257,7 @@ cudaError_t launch_bn_eval_finish(const Problem &pb, const float *part_g, const 
                                   int splits, const float *gamma, const float *var, float *db,
                                   float *dgamma, float *dbeta, cudaStream_t st);
 
+// One block, one bounded wait (limit_ns) on a barrier without arrivals: sets ERRW_TIMEOUT in the error word.
+cudaError_t launch_selftest_wait_timeout(unsigned long long limit_ns, cudaStream_t st);
+
 }  // namespace convbn

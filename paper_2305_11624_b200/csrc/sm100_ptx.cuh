@@ -89,6 +89,32 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
     }
 }
 
+// The same bounded wait with the non-blocking test_wait: try_wait may park the thread for a system-defined
+// time before it reports "not yet", which adds up to a microsecond to every hand-over of a fine-grained
+// pipeline; test_wait returns at once, at the price of issue slots for the spinning warp.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_spin_bounded(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                                  uint64_t limit_ns = 2000000000ull) {
+    if (mbar_test_wait(bar, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+    uint32_t spins = 0;
+    while (true) {
+        if (mbar_test_wait(bar, parity)) return true;
+        if ((++spins & 1023u) == 0) {
+            if (abort_flag && *abort_flag) return false;
+            if (globaltimer_ns() - t0 > limit_ns) return false;
+        }
+    }
+}
+
 // ---- named barriers (ids 1-15; id 0 is __syncthreads) -------------------------------------------
 // `count` threads (a multiple of 32) take part; arrive does not wait.  A producer warp that only signals
 // fences its shared-memory writes (__threadfence_block) before it arrives.
@@ -230,6 +256,16 @@ __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&v)[16])
         : "r"(taddr)
         : "memory");
 }
+// 32 lanes x 32 consecutive columns <- the same value from every thread (used to clear accumulators).
+__device__ __forceinline__ void tmem_st_32x32_fill(uint32_t taddr, uint32_t value) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, "
+        "%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};"
+        ::"r"(taddr), "r"(value)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // ---- descriptors ---------------------------------------------------------------------------------

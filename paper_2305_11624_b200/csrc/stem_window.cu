@@ -11,8 +11,8 @@
 // once per tile (kh / stride_h times overall) instead of once per tap, and K per filter row is 32 (kw <= 8
 // taps x 4 channels; unused slots meet zero weights), i.e. kh x 2 MMAs of 128 x C_out x 16 per output row.
 //
-// Warps: 0-3 load input rows (16-byte global loads, repacked 3 -> 4 channels on the way), 4-7 issue MMAs
-// (round-robin over output rows, disjoint accumulators), 8-23 drain accumulators: scale, shift, bf16,
+// Warps: 0-7 load input rows (16-byte global loads, repacked 3 -> 4 channels on the way), 8-11 issue MMAs
+// (round-robin over output rows, disjoint accumulators), 12-23 drain accumulators: scale, shift, bf16,
 // swizzled staging, TMA store.  Every CTA owns a contiguous range of output rows.  Every wait is bounded.
 #include "kernels.h"
 #include "sm100_ptx.cuh"
@@ -21,7 +21,7 @@ namespace convbn {
 
 using namespace ptx;
 
-constexpr int kWinLoaders = 4, kWinIssuers = 4, kWinEpiGroups = 4;
+constexpr int kWinLoaders = 8, kWinIssuers = 4, kWinEpiGroups = 3;
 constexpr int kWinEpiWarp0 = kWinLoaders + kWinIssuers;
 constexpr int kWinThreads = 32 * (kWinEpiWarp0 + 4 * kWinEpiGroups);
 constexpr int kWinMaxStrips = 3;
@@ -45,6 +45,7 @@ struct WinCtl {
     uint64_t tmem_full[8], tmem_empty[8];
     uint32_t tmem_base;
     int abort_flag;
+    unsigned short slot_of[256];   // weight element (r, q, c) -> (K block << 8) | position in the 64-wide K row
 };
 
 // descriptor halves of the un-swizzled K-major window operand: LBO 16 bytes, SBO 128 bytes
@@ -115,8 +116,8 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
     constexpr int NA = 512 / BN;                           // accumulators in tensor memory
     uint8_t *strips = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *wres = strips + (size_t)g.nstrips * g.strip_bytes;          // [kblocks][BN][128 B], 128-byte swizzle
-    uint8_t *staging = wres + (size_t)g.kblocks * BN * 128;              // 16 warps x [32 rows][128 B]
-    WinCtl *ctl = (WinCtl *)(staging + 16 * 4096);
+    uint8_t *staging = wres + (size_t)g.kblocks * BN * 128;              // per epilogue warp [32 rows][128 B]
+    WinCtl *ctl = (WinCtl *)(staging + 4 * kWinEpiGroups * 4096);
     float *bias_s = (float *)(((uintptr_t)(ctl + 1) + 15) & ~(uintptr_t)15);
     float *scale_s = bias_s + BN;
     const bool fold = g.fold.gamma != nullptr;
@@ -177,9 +178,15 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
                 uint4 *z4 = (uint4 *)wres;
                 for (int i = tid; i < g.kblocks * BN * 8; i += nt) z4[i] = make_uint4(0, 0, 0, 0);
             }
-            named_bar_sync(4, nt);
             const int rowlen = g.kh * g.kw * C, total = BN * rowlen;
+            if (tid < rowlen) {                        // the only divisions of the set-up: once per weight-row position
+                const int c = tid % C, t2 = tid / C, q = t2 % g.kw, r = t2 / g.kw;
+                ctl->slot_of[tid] = (unsigned short)(((r >> 1) << 8) | ((r & 1) * 32 + q * 4 + c));
+            }
+            named_bar_sync(4, nt);
             const unsigned short *wsrc = (const unsigned short *)w;
+            // channel = e / rowlen by a multiply with the rounded-up reciprocal (e < 2^15: exact or one too large)
+            const uint32_t inv = (65536u + (uint32_t)rowlen - 1u) / (uint32_t)rowlen;
             for (int base = tid; base < total; base += 8 * nt) {
                 unsigned short val[8];
 #pragma unroll
@@ -188,8 +195,10 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
                 for (int k = 0; k < 8; ++k) {
                     const int e = base + k * nt;
                     if (e >= total) break;
-                    const int co = e / rowlen, rem = e - co * rowlen, c = rem % C, t2 = rem / C, q = t2 % g.kw, r = t2 / g.kw;
-                    const int k64 = (r & 1) * 32 + q * 4 + c, kb = r >> 1;
+                    int co = (int)(((uint32_t)e * inv) >> 16);
+                    int rem = e - co * rowlen;
+                    if (rem < 0) { --co; rem += rowlen; }
+                    const int sl = ctl->slot_of[rem], k64 = sl & 255, kb = sl >> 8;
                     *(unsigned short *)(wres + (size_t)kb * BN * 128 + co * 128 + ((((k64 >> 3) ^ (co & 7)) & 7) << 4) + (k64 & 7) * 2) = val[k];
                 }
             }
@@ -366,7 +375,8 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
 // Each CTA accumulates its contiguous range of output rows in tensor memory and writes one fp32 partial
 // [k][co] plus one row of sums; the fused epilogue kernel adds the CTAs' partials in fixed order.
 constexpr int kWgR = 4;                  // output rows per chunk
-constexpr int kWgThreads = 256;          // warps 0-3 X loaders, 4 tensor memory + read-out, 5 dZ producer, 6-7 issuers
+constexpr int kWgLoaders = 8;
+constexpr int kWgThreads = 32 * (kWgLoaders + 4);   // warps 0-7 X loaders, 8 tensor memory + read-out, 9 dZ producer, 10-11 issuers
 
 struct WinWgrad {
     int n, h_in, w_in, h_out, w_out, c_out, kh, kw, pad_h, pad_w;
@@ -401,7 +411,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 2; ++s) {
-            mbar_init(&ctl->x_full[s], 128); mbar_init(&ctl->x_empty[s], 2);
+            mbar_init(&ctl->x_full[s], 32 * kWgLoaders); mbar_init(&ctl->x_empty[s], 2);
             mbar_init(&ctl->dz_full[s], 1); mbar_init(&ctl->dz_empty[s], 2);
         }
         mbar_init(&ctl->acc_done, 2);
@@ -418,7 +428,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
         for (int i = threadIdx.x; i < 128; i += kWgThreads) z4[i] = make_uint4(0, 0, 0, 0);
     }
     fence_proxy_async_smem();
-    if (warp == 4) {
+    if (warp == kWgLoaders) {
         tmem_alloc(&ctl->tmem_base, 512);
         tmem_relinquish();
     }
@@ -431,7 +441,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
     pdl_launch_dependents();       // only now: this CTA owns its tensor-memory columns
     const uint32_t tmem_base = ctl->tmem_base;
 
-    if (warp < 4) {
+    if (warp < kWgLoaders) {
         // ---------------- X row loaders ----------------
         long long cur = row_lo;
         WinChunk ck;
@@ -442,13 +452,13 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
             ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->x_empty[sb], ph ^ 1u, abort_flag));
             if (!ok) break;
             win_fill_patch<C>(xs + (size_t)sb * g.xstrip_bytes, x, ck.img, ck.h0 * 2 - g.pad_h, (ck.rows - 1) * 2 + g.kh,
-                              g.h_in, g.w_in, g.pad_w, g.pitch, (int)threadIdx.x, 128, 0x3F80u);
+                              g.h_in, g.w_in, g.pad_w, g.pitch, (int)threadIdx.x, 32 * kWgLoaders, 0x3F80u);
             fence_proxy_async_smem();
             mbar_arrive(&ctl->x_full[sb]);
             if (++sb == 2) { sb = 0; ph ^= 1u; }
         }
         if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
-    } else if (warp == 5) {
+    } else if (warp == kWgLoaders + 1) {
         // ---------------- dZ producer: one TMA box per output row of the chunk ----------------
         if (elect_one()) {
             long long cur = row_lo;
@@ -472,9 +482,9 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
                     mbar_wait_bounded(&ctl->dz_full[j & 1], (uint32_t)(j >> 1) & 1u, nullptr, 200000000ull);
             }
         }
-    } else if (warp >= 6) {
-        // ---------------- MMA issuers: warp 6 the even input rows of a patch, warp 7 the odd ones ----------------
-        const int e = warp - 6, Te = e ? g.T1 : g.T0;
+    } else if (warp >= kWgLoaders + 2) {
+        // ---------------- MMA issuers: one warp for the even input rows of a patch, one for the odd ones ----------------
+        const int e = warp - (kWgLoaders + 2), Te = e ? g.T1 : g.T0;
         if (elect_one()) {
             const uint32_t acc = tmem_base + (uint32_t)e * 256u;
             // A: MN-major, no swizzle: 8 M elements per 16 bytes, next 8 M elements 16 bytes on, next 8 pixels 128 bytes on
@@ -518,7 +528,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
             else { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
         }
     } else {
-        // ---------------- read-out (warp 4 = lanes 0-31 of tensor memory = window offsets m = 0 .. 31) ----------------
+        // ---------------- read-out (warp 8 = lanes 0-31 of tensor memory = window offsets m = 0 .. 31) ----------------
         const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->acc_done, 0, abort_flag));
         if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
         if (ok) {
@@ -552,7 +562,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 4) tmem_dealloc(tmem_base, 512);
+    if (warp == kWgLoaders) tmem_dealloc(tmem_base, 512);
 }
 
 // ---- host side --------------------------------------------------------------------------------------
@@ -568,7 +578,7 @@ WinPlan plan_window(const Problem &pb) {
         return pl;
     pl.pitch = (int)(((size_t)(pb.w_in + 2 * pb.pad_w) * 8 + 15) / 16 * 16);
     pl.kblocks = (pb.kh + 1) / 2;
-    const size_t fixed = 1024 + 16 * 4096 + sizeof(WinCtl) + 2 * (size_t)pb.c_out * sizeof(float) + 32 +
+    const size_t fixed = 1024 + 4 * kWinEpiGroups * 4096 + sizeof(WinCtl) + 2 * (size_t)pb.c_out * sizeof(float) + 32 +
                          (size_t)pl.kblocks * pb.c_out * 128;
     const size_t budget = 226 * 1024;
     for (int r = pb.h_out < 8 ? pb.h_out : 8; r >= 1; --r) {

@@ -14,7 +14,7 @@
 // A CTA owns a contiguous range of dZ rows and the input rows 2 ho, 2 ho + 1 (padded coordinates) that go with
 // them; it also runs the (kh - 1) / 2 dZ rows before its range, whose contributions its first rows need.
 //
-// Warps: 0 dZ producer (TMA ring), 1 MMA issuer and tensor-memory owner, 2-3 help with set-up, 4-11 two
+// Warps: 0 dZ producer (TMA ring), 1 MMA issuer and tensor-memory owner, 2-3 help with set-up, 4-19 four
 // epilogue groups that take completed rows in turn.  Every wait is bounded.
 #include "kernels.h"
 #include "sm100_ptx.cuh"
@@ -23,7 +23,8 @@ namespace convbn {
 
 using namespace ptx;
 
-constexpr int kDgThreads = 384;
+constexpr int kDgGroups = 4;                 // epilogue groups of four warps
+constexpr int kDgThreads = 32 * (4 + 4 * kDgGroups);
 constexpr int kDgSlots = 6;                  // dZ rows in the TMA ring (16 KB each)
 constexpr int kDgBlocks = 16;                // accumulator blocks of 32 columns
 
@@ -39,6 +40,7 @@ struct WinDgCtl {
     uint64_t blk_full[kDgBlocks], blk_empty[kDgBlocks];
     uint32_t tmem_base;
     int abort_flag;
+    unsigned short nrow_of[256];             // weight element (r, q, c) -> row r 32 + 4 q + c of the resident matrix
 };
 
 // A segment: the rows [a, b) of image img that this CTA owns; processing starts `halo` rows earlier.
@@ -63,15 +65,16 @@ __global__ void __launch_bounds__(kDgThreads) stem_window_dgrad_kernel(const __g
     extern __shared__ uint8_t smem_raw[];
     uint8_t *dzs = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);      // kDgSlots x [128 px][128 B]
     uint8_t *wres = dzs + (size_t)kDgSlots * 16384;                                  // [kh * 32 rows][128 B], swizzled
-    float *xch = (float *)(wres + (size_t)g.kh * 32 * 128);                           // 2 groups x [6 q][4 c][128]
-    uint8_t *rowbuf = (uint8_t *)(xch + 2 * 6 * 4 * 128);                             // 2 groups x 2048 B
-    WinDgCtl *ctl = (WinDgCtl *)(rowbuf + 2 * 2048);
+    float *xch = (float *)(wres + (size_t)g.kh * 32 * 128);                           // per group [6 q][4 c][128]
+    uint8_t *rowbuf = (uint8_t *)(xch + kDgGroups * 6 * 4 * 128);                     // per group 2048 B
+    WinDgCtl *ctl = (WinDgCtl *)(rowbuf + kDgGroups * 2048);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &ctl->abort_flag;
     const long long row_lo = g.total_rows * blockIdx.x / gridDim.x, row_hi = g.total_rows * (blockIdx.x + 1) / gridDim.x;
     const int kh = g.kh;
 
     if (threadIdx.x == 0) {
+        CONVBN_TRACE_POINT(0);
         for (int s = 0; s < kDgSlots; ++s) { mbar_init(&ctl->dz_full[s], 1); mbar_init(&ctl->dz_empty[s], 1); }
         for (int s = 0; s < kDgBlocks; ++s) { mbar_init(&ctl->blk_full[s], 1); mbar_init(&ctl->blk_empty[s], 4); }
         ctl->abort_flag = 0;
@@ -87,13 +90,42 @@ __global__ void __launch_bounds__(kDgThreads) stem_window_dgrad_kernel(const __g
         // resident weights: row n = r 32 + 4 q + c, column co: s[co] w[co][r][q][c], zeros in the unused slots
         uint4 *z4 = (uint4 *)wres;
         for (int i = threadIdx.x; i < kh * 32 * 8; i += kDgThreads) z4[i] = make_uint4(0, 0, 0, 0);
-        __syncthreads();
         const int rowlen = kh * g.kw * C, total = g.c_out * rowlen;
-        for (int e = threadIdx.x; e < total; e += kDgThreads) {
-            const int co = e / rowlen, rem = e - co * rowlen, c = rem % C, t2 = rem / C, q = t2 % g.kw, r = t2 / g.kw;
-            const float v = (g.s_vec ? g.s_vec[co] : 1.f) * __bfloat162float(w[e]);
-            const int nrow = r * 32 + 4 * q + c;
-            *(__nv_bfloat16 *)(wres + (size_t)nrow * 128 + ((((co >> 3) ^ (nrow & 7)) & 7) << 4) + (co & 7) * 2) = __float2bfloat16_rn(v);
+        if ((int)threadIdx.x < rowlen) {           // the only divisions of the set-up: once per weight-row position
+            const int rem = threadIdx.x, c = rem % C, t2 = rem / C, q = t2 % g.kw, r = t2 / g.kw;
+            ctl->nrow_of[rem] = (unsigned short)(r * 32 + 4 * q + c);
+        }
+        tc_fence_before_sync();
+        __syncthreads();
+        tc_fence_after_sync();
+        // every accumulator block starts from zero (and is cleared again by whoever drains it), so that all
+        // MMAs accumulate and one dZ row needs a single MMA over its kh blocks
+        if (warp >= 4 && warp < 8) {
+            const uint32_t t0 = ctl->tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+            for (int b = 0; b < kDgBlocks; ++b) tmem_st_32x32_fill(t0 + (uint32_t)b * 32u, 0u);
+            tmem_st_wait();
+        }
+        // consecutive threads read consecutive weights; channel = e / rowlen by a multiply with the rounded-up
+        // reciprocal (e < 2^14: the estimate is exact or one too large, fixed up below)
+        const uint32_t inv = (65536u + (uint32_t)rowlen - 1u) / (uint32_t)rowlen;
+        for (int base = threadIdx.x; base < total; base += 8 * kDgThreads) {
+            float val[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {              // the loads of a batch are issued together
+                const int e = base + k * kDgThreads;
+                val[k] = e < total ? __bfloat162float(w[e]) : 0.f;
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int e = base + k * kDgThreads;
+                if (e >= total) break;
+                int co = (int)(((uint32_t)e * inv) >> 16);
+                int rem = e - co * rowlen;
+                if (rem < 0) { --co; rem += rowlen; }      // the rounded-up reciprocal can overshoot by one
+                const int nrow = ctl->nrow_of[rem];
+                const float v = (g.s_vec ? g.s_vec[co] : 1.f) * val[k];
+                *(__nv_bfloat16 *)(wres + (size_t)nrow * 128 + ((((co >> 3) ^ (nrow & 7)) & 7) << 4) + (co & 7) * 2) = __float2bfloat16_rn(v);
+            }
         }
         fence_proxy_async_smem();
     }
@@ -102,6 +134,7 @@ __global__ void __launch_bounds__(kDgThreads) stem_window_dgrad_kernel(const __g
     tc_fence_after_sync();
     pdl_launch_dependents();       // only now: this CTA owns its tensor-memory columns
     const uint32_t tmem_base = ctl->tmem_base;
+    if (threadIdx.x == 0) CONVBN_TRACE_POINT(2);
 
     if (warp == 0) {
         // ---------------- dZ producer ----------------
@@ -113,7 +146,9 @@ __global__ void __launch_bounds__(kDgThreads) stem_window_dgrad_kernel(const __g
             bool ok = true;
             while (ok && dg_next_segment(cur, row_hi, g.h_out, g.halo, sg))
                 for (int ho = sg.first; ho < sg.b; ++ho) {
+                    { CONVBN_TRACE_T0();
                     if (!mbar_wait_bounded(&ctl->dz_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+                    CONVBN_TRACE_ACC(12); }
                     mbar_arrive_expect_tx(&ctl->dz_full[s], 16384u);
                     tma_load_3d(dzs + (size_t)s * 16384, &tm_dz, &ctl->dz_full[s], 0, 0, sg.img * g.h_out + ho);
                     ++issued;
@@ -131,17 +166,15 @@ __global__ void __launch_bounds__(kDgThreads) stem_window_dgrad_kernel(const __g
             const uint32_t hi = smem_desc_hi_sw128(1024);
             const uint32_t dz_lo = smem_desc_lo(smem_u32(dzs), 16), w_lo = smem_desc_lo(smem_u32(wres), 16);
             // blocks [first, first + nb) of the ring (wrapping at 16), filter rows r0 .. r0 + nb - 1
-            auto issue = [&](uint32_t a_lo, uint32_t seq_first, int r0, int nb, bool fresh) {
+            auto issue = [&](uint32_t a_lo, uint32_t seq_first, int r0, int nb) {
                 while (nb > 0) {
                     const uint32_t blk = seq_first % kDgBlocks;
                     int run = (int)(kDgBlocks - blk);
                     if (run > nb) run = nb;
                     const uint32_t idesc = idesc_bf16_f32(128, 32 * run, 0, 0);
                     const uint32_t d = tmem_base + blk * 32u, b_lo = w_lo + (uint32_t)r0 * 256u;   // 32 rows x 128 B per r
-                    if (fresh) umma_bf16_ss_halves<false>(d, a_lo, hi, b_lo, hi, idesc);
-                    else umma_bf16_ss_halves<true>(d, a_lo, hi, b_lo, hi, idesc);
 #pragma unroll
-                    for (int k = 1; k < 4; ++k) umma_bf16_ss_halves<true>(d, a_lo + (uint32_t)k * 2u, hi, b_lo + (uint32_t)k * 2u, hi, idesc);
+                    for (int k = 0; k < 4; ++k) umma_bf16_ss_halves<true>(d, a_lo + (uint32_t)k * 2u, hi, b_lo + (uint32_t)k * 2u, hi, idesc);
                     seq_first += (uint32_t)run; r0 += run; nb -= run;
                 }
             };
@@ -157,17 +190,20 @@ __global__ void __launch_bounds__(kDgThreads) stem_window_dgrad_kernel(const __g
                     const uint32_t row0 = seq_base + 2u * (uint32_t)(ho - sg.first);
                     const int nnew = ho == sg.first ? kh : (kh < 2 ? kh : 2), nold = kh - nnew;
                     // blocks taken for rows never touched before must have been drained by their last user
+                    { CONVBN_TRACE_T0();
                     for (int j = 0; j < nnew && ok; ++j) {
                         const uint32_t sq = row0 + (uint32_t)(nold + j);
-                        if (sq >= kDgBlocks && !mbar_wait_bounded(&ctl->blk_empty[sq % kDgBlocks], ((sq / kDgBlocks) & 1u) ^ 1u, abort_flag))
+                        if (sq >= kDgBlocks && !mbar_spin_bounded(&ctl->blk_empty[sq % kDgBlocks], ((sq / kDgBlocks) & 1u) ^ 1u, abort_flag))
                             ok = false;
                     }
+                    CONVBN_TRACE_ACC(13); }
                     if (!ok) break;
-                    if (!mbar_wait_bounded(&ctl->dz_full[s], ph, abort_flag)) { ok = false; break; }
+                    { CONVBN_TRACE_T0();
+                    if (!mbar_spin_bounded(&ctl->dz_full[s], ph, abort_flag)) { ok = false; break; }
+                    CONVBN_TRACE_ACC(14); }
                     tc_fence_after_sync();
                     const uint32_t a_lo = dz_lo + (uint32_t)s * (16384u >> 4);
-                    if (nold > 0) issue(a_lo, row0, 0, nold, false);
-                    issue(a_lo, row0 + (uint32_t)nold, nold, nnew, true);
+                    issue(a_lo, row0, 0, kh);
                     umma_commit(&ctl->dz_empty[s]);
                     // rows no later dZ row of the segment reaches: 2 ho and 2 ho + 1, everything at the segment's end
                     const int ndone = ho == sg.b - 1 ? kh : (kh < 2 ? kh : 2);
@@ -176,6 +212,7 @@ __global__ void __launch_bounds__(kDgThreads) stem_window_dgrad_kernel(const __g
                     if (++s == kDgSlots) { s = 0; ph ^= 1u; }
                 }
             }
+            CONVBN_TRACE_POINT(6);
             if (!ok) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
         }
     } else if (warp >= 4) {
@@ -194,18 +231,28 @@ __global__ void __launch_bounds__(kDgThreads) stem_window_dgrad_kernel(const __g
                 const uint32_t row0 = seq_base + 2u * (uint32_t)(ho - sg.first);
                 const int ndone = ho == sg.b - 1 ? kh : (kh < 2 ? kh : 2);
                 for (int jr = 0; jr < ndone && ok; ++jr, ++done) {
-                    if ((int)(done & 1u) != grp) continue;
+                    if ((int)(done % kDgGroups) != grp) continue;
                     const uint32_t sq = row0 + (uint32_t)jr, blk = sq % kDgBlocks;
-                    ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->blk_full[blk], (sq / kDgBlocks) & 1u, abort_flag));
+                    { CONVBN_TRACE_T0();
+                    ok = __all_sync(0xffffffffu, mbar_spin_bounded(&ctl->blk_full[blk], (sq / kDgBlocks) & 1u, abort_flag));
+                    if (warp == 4 && lane == 0) CONVBN_TRACE_ACC(15); }
                     if (!ok) break;
                     tc_fence_after_sync();
                     const int rp = 2 * ho + jr, rho = rp - g.pad_h;          // padded / real input row
                     const bool stored = rp >= 2 * sg.a && (rp < 2 * sg.b || sg.b == g.h_out) && rho >= 0 && rho < g.h_in;
                     uint32_t v[32];
+                    const uint32_t taddr = tmem_base + blk * 32u + ((uint32_t)(quarter * 32) << 16);
+                    { CONVBN_TRACE_T0();
                     if (stored) {
-                        tmem_ld_32x32(tmem_base + blk * 32u + ((uint32_t)(quarter * 32) << 16), v);
+                        tmem_ld_32x32(taddr, v);
                         tmem_ld_wait();
                     }
+                    if (warp == 4 && lane == 0) CONVBN_TRACE_ACC(4); }
+                    { CONVBN_TRACE_T0();
+                    tmem_st_32x32_fill(taddr, 0u);        // the block's next user accumulates into zeros
+                    tmem_st_wait();
+                    if (warp == 4 && lane == 0) CONVBN_TRACE_ACC(5); }
+                    CONVBN_TRACE_T0();
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&ctl->blk_empty[blk]);
@@ -235,21 +282,24 @@ __global__ void __launch_bounds__(kDgThreads) stem_window_dgrad_kernel(const __g
                         uint4 *dst = (uint4 *)(dx + ((size_t)sg.img * g.h_in + rho) * g.w_in * C);
                         for (int i = gt; i < n16; i += 128) dst[i] = ((const uint4 *)rbuf)[i];
                     }
+                    if (warp == 4 && lane == 0) CONVBN_TRACE_ACC(7);
                 }
                 seq = row0 + (uint32_t)ndone;
             }
         }
+        if (warp == 4 && lane == 0) CONVBN_TRACE_POINT(10);
         if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
     }
     tc_fence_before_sync();
     __syncthreads();
+    if (threadIdx.x == 0) CONVBN_TRACE_POINT(11);
     if (warp == 1) tmem_dealloc(tmem_base, 512);
 }
 
 // ---- host side --------------------------------------------------------------------------------------
 namespace {
 size_t dgrad_window_smem(const Problem &pb) {
-    return 1024 + (size_t)kDgSlots * 16384 + (size_t)pb.kh * 32 * 128 + 2 * 6 * 4 * 128 * sizeof(float) + 2 * 2048 +
+    return 1024 + (size_t)kDgSlots * 16384 + (size_t)pb.kh * 32 * 128 + kDgGroups * 6 * 4 * 128 * sizeof(float) + kDgGroups * 2048 +
            sizeof(WinDgCtl) + 64;
 }
 

@@ -355,6 +355,24 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
     if (warp == 1) tmem_dealloc(tmem_base, 2 * BN);
 }
 
+// ---- failure-path self-test: the bounded wait of the kernels above, on a barrier nobody completes --------
+__global__ void selftest_wait_timeout_kernel(unsigned long long limit_ns, int *err) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        fence_barrier_init();
+        if (!mbar_wait_bounded(&bar, 0, nullptr, limit_ns)) atomicOr(err, ERRW_TIMEOUT);
+    }
+}
+
+cudaError_t launch_selftest_wait_timeout(unsigned long long limit_ns, cudaStream_t st) {
+    int *err = nullptr;
+    cudaError_t e = error_word_address(&err);
+    if (e != cudaSuccess) return e;
+    selftest_wait_timeout_kernel<<<1, 32, 0, st>>>(limit_ns, err);
+    return cudaGetLastError();
+}
+
 // ---- host side: tensor maps and launch ---------------------------------------------------------
 namespace {
 
