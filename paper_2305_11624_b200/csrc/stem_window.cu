@@ -184,22 +184,29 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
                 ctl->slot_of[tid] = (unsigned short)(((r >> 1) << 8) | ((r & 1) * 32 + q * 4 + c));
             }
             named_bar_sync(4, nt);
-            const unsigned short *wsrc = (const unsigned short *)w;
-            // channel = e / rowlen by a multiply with the rounded-up reciprocal (e < 2^15: exact or one too large)
+            // 16-byte loads (8 weights), all of a thread's loads issued before the first use; channel = e / rowlen
+            // by a multiply with the rounded-up reciprocal (e < 2^15: exact or one too large, fixed up)
+            const uint4 *wsrc = (const uint4 *)w;
             const uint32_t inv = (65536u + (uint32_t)rowlen - 1u) / (uint32_t)rowlen;
-            for (int base = tid; base < total; base += 8 * nt) {
-                unsigned short val[8];
+            const int n8 = total / 8;                  // BN is a multiple of 64, so total is a multiple of 8
+            for (int base = tid; base < n8; base += 4 * nt) {
+                uint4 val[4];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) val[k] = base + k * nt < total ? __ldg(wsrc + base + k * nt) : (unsigned short)0;
+                for (int k = 0; k < 4; ++k) val[k] = base + k * nt < n8 ? __ldg(wsrc + base + k * nt) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const int e = base + k * nt;
-                    if (e >= total) break;
-                    int co = (int)(((uint32_t)e * inv) >> 16);
-                    int rem = e - co * rowlen;
-                    if (rem < 0) { --co; rem += rowlen; }
-                    const int sl = ctl->slot_of[rem], k64 = sl & 255, kb = sl >> 8;
-                    *(unsigned short *)(wres + (size_t)kb * BN * 128 + co * 128 + ((((k64 >> 3) ^ (co & 7)) & 7) << 4) + (k64 & 7) * 2) = val[k];
+                for (int k = 0; k < 4; ++k) {
+                    if (base + k * nt >= n8) break;
+                    const uint32_t wd[4] = {val[k].x, val[k].y, val[k].z, val[k].w};
+#pragma unroll
+                    for (int h = 0; h < 8; ++h) {
+                        const int e = (base + k * nt) * 8 + h;
+                        int co = (int)(((uint32_t)e * inv) >> 16);
+                        int rem = e - co * rowlen;
+                        if (rem < 0) { --co; rem += rowlen; }
+                        const int sl = ctl->slot_of[rem], k64 = sl & 255, kb = sl >> 8;
+                        *(unsigned short *)(wres + (size_t)kb * BN * 128 + co * 128 + ((((k64 >> 3) ^ (co & 7)) & 7) << 4) + (k64 & 7) * 2) =
+                            (unsigned short)(wd[h >> 1] >> ((h & 1) * 16));
+                    }
                 }
             }
             fence_proxy_async_smem();

@@ -105,26 +105,30 @@ __global__ void __launch_bounds__(kDgThreads) stem_window_dgrad_kernel(const __g
             for (int b = 0; b < kDgBlocks; ++b) tmem_st_32x32_fill(t0 + (uint32_t)b * 32u, 0u);
             tmem_st_wait();
         }
-        // consecutive threads read consecutive weights; channel = e / rowlen by a multiply with the rounded-up
-        // reciprocal (e < 2^14: the estimate is exact or one too large, fixed up below)
+        // 16-byte loads (8 weights), a thread's loads issued together; channel = e / rowlen by a multiply with the
+        // rounded-up reciprocal (e < 2^14: the estimate is exact or one too large, fixed up below)
         const uint32_t inv = (65536u + (uint32_t)rowlen - 1u) / (uint32_t)rowlen;
-        for (int base = threadIdx.x; base < total; base += 8 * kDgThreads) {
-            float val[8];
+        const uint4 *wsrc = (const uint4 *)w;
+        const int n8 = total / 8;                      // C_out = 64: total is a multiple of 8
+        for (int base = threadIdx.x; base < n8; base += 2 * kDgThreads) {
+            uint4 val[2];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {              // the loads of a batch are issued together
-                const int e = base + k * kDgThreads;
-                val[k] = e < total ? __bfloat162float(w[e]) : 0.f;
-            }
+            for (int k = 0; k < 2; ++k) val[k] = base + k * kDgThreads < n8 ? __ldg(wsrc + base + k * kDgThreads) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const int e = base + k * kDgThreads;
-                if (e >= total) break;
-                int co = (int)(((uint32_t)e * inv) >> 16);
-                int rem = e - co * rowlen;
-                if (rem < 0) { --co; rem += rowlen; }      // the rounded-up reciprocal can overshoot by one
-                const int nrow = ctl->nrow_of[rem];
-                const float v = (g.s_vec ? g.s_vec[co] : 1.f) * val[k];
-                *(__nv_bfloat16 *)(wres + (size_t)nrow * 128 + ((((co >> 3) ^ (nrow & 7)) & 7) << 4) + (co & 7) * 2) = __float2bfloat16_rn(v);
+            for (int k = 0; k < 2; ++k) {
+                if (base + k * kDgThreads >= n8) break;
+                const uint32_t wd[4] = {val[k].x, val[k].y, val[k].z, val[k].w};
+#pragma unroll
+                for (int h = 0; h < 8; ++h) {
+                    const int e = (base + k * kDgThreads) * 8 + h;
+                    int co = (int)(((uint32_t)e * inv) >> 16);
+                    int rem = e - co * rowlen;
+                    if (rem < 0) { --co; rem += rowlen; }      // the rounded-up reciprocal can overshoot by one
+                    const int nrow = ctl->nrow_of[rem];
+                    const float wv = __uint_as_float((wd[h >> 1] >> ((h & 1) * 16)) << 16);     // bf16 -> fp32
+                    const float v = (g.s_vec ? g.s_vec[co] : 1.f) * wv;
+                    *(__nv_bfloat16 *)(wres + (size_t)nrow * 128 + ((((co >> 3) ^ (nrow & 7)) & 7) << 4) + (co & 7) * 2) = __float2bfloat16_rn(v);
+                }
             }
         }
         fence_proxy_async_smem();

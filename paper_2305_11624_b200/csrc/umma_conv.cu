@@ -105,6 +105,7 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
     volatile int *abort_flag = &ctl->abort_flag;
 
     if (threadIdx.x == 0) {
+        CONVBN_TRACE_POINT(0);
         for (int s = 0; s < stages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tmem_full[a], 1); mbar_init(&ctl->tmem_empty[a], 4); }
         mbar_init(&ctl->bfull, 1);
@@ -120,6 +121,7 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
     // the tensor maps are kernel parameters, not data of an earlier kernel: fetch them before the wait
     if (threadIdx.x == 0) { prefetch_tensormap(&tm_act); prefetch_tensormap(&tm_w); prefetch_tensormap(&tm_out); }
     pdl_wait();
+    if (threadIdx.x == 0) CONVBN_TRACE_POINT(1);
     if (fold) {
         // On-the-fly reparameterisation (Sec. 3.3 / 3.4): s = gamma / sqrt(var + eps), b' = (b - mu) s + beta.
         // s multiplies the fp32 accumulator (the associative law of Sec. 3.2.2), so omega is used unrounded.
@@ -141,6 +143,7 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
     tc_fence_after_sync();
     pdl_launch_dependents();       // only now: this CTA owns its tensor-memory columns
     const uint32_t tmem_base = ctl->tmem_base;
+    if (threadIdx.x == 0) CONVBN_TRACE_POINT(2);
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -177,7 +180,9 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
             const int base_w = g.lower_w + wo0 * g.stride_w, base_h = g.lower_h + ho0 * g.stride_h;
             int r = 0, q = 0, cc = 0;
             for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                { CONVBN_TRACE_T0();
                 ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->empty[s], ph ^ 1u, abort_flag));
+                if (lane == 0) CONVBN_TRACE_ACC(12); }
                 if (!ok) break;
                 uint8_t *a_dst = tiles + (size_t)s * kStageBytes, *b_dst = a_dst + kABytes;
                 if (lane == 0) {
@@ -218,11 +223,16 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
             uint32_t mt, nt;
             for (uint32_t i = 0; ok && tile_of(i, mt, nt); ++i) {
                 const uint32_t acc = i & 1u;
+                { CONVBN_TRACE_T0();
                 if (!mbar_wait_bounded(&ctl->tmem_empty[acc], ((i >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                CONVBN_TRACE_ACC(13); }
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int kb = 0; kb < num_kb; ++kb) {
+                    { CONVBN_TRACE_T0();
                     if (!mbar_wait_bounded(&ctl->full[s], ph, abort_flag)) { ok = false; break; }
+                    CONVBN_TRACE_ACC(14); }
+                    if (i == 0 && kb == 0) CONVBN_TRACE_POINT(4);
                     tc_fence_after_sync();
                     // descriptors as halves: only the start-address field (16-byte units) moves
                     const uint32_t a_lo = tiles_lo + (uint32_t)s * (kStageBytes >> 4);
@@ -236,6 +246,7 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                     if (++s == stages) { s = 0; ph ^= 1u; }
                 }
                 if (ok) umma_commit(&ctl->tmem_full[acc]);
+                CONVBN_TRACE_POINT(6);
             }
             if (!ok) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
         }
@@ -250,7 +261,9 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
         uint32_t mt, nt;
         for (uint32_t i = egroup; tile_of(i, mt, nt); i += 2) {
             const uint32_t acc = egroup;
+            CONVBN_TRACE_T0();
             const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->tmem_full[acc], (i >> 1) & 1u, abort_flag));
+            if (warp == 2 && lane == 0) CONVBN_TRACE_ACC(15);
             if (!ok) {
                 if (lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
                 break;
@@ -348,10 +361,13 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                 }
             }
         }
+        if (warp == 2 && lane == 0) CONVBN_TRACE_POINT(9);
         if (lane == 0) tma_store_wait_all<0>();             // global writes done before the CTA exits
+        if (warp == 2 && lane == 0) CONVBN_TRACE_POINT(10);
     }
     tc_fence_before_sync();
     __syncthreads();
+    if (threadIdx.x == 0) CONVBN_TRACE_POINT(11);
     if (warp == 1) tmem_dealloc(tmem_base, 2 * BN);
 }
 
