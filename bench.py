@@ -319,7 +319,7 @@ def bench_config(ctx, wl):
         for li, b in enumerate(bs):
             b.randomize(I.config_seed(wl, li) + 7919 * (rank * sets + si))
     stream = torch.cuda.current_stream()
-    calls_per_step = 3 * len(layers)
+    calls_per_step = 2 * len(layers)             # convbn_tune_fwd and convbn_tune_bwd per layer
 
     def step(i):
         for b in blocks[i % sets]:

@@ -68,7 +68,8 @@ typedef enum {
     CONVBN_PHASE_EVAL_BWD = 4,
     CONVBN_PHASE_DEPLOY_FWD = 5,
     CONVBN_PHASE_DEPLOY_BWD = 6,
-    CONVBN_PHASE_COUNT = 7
+    CONVBN_PHASE_TUNE_BWD = 7,
+    CONVBN_PHASE_COUNT = 8
 } convbn_phase;
 
 /* Problem description (paper Sec. 3.1 and the shape annotations of Appendix C; stride, padding,
@@ -129,6 +130,17 @@ int convbn_tune_bwd_weight(const convbn_desc *desc, const void *dz, const void *
                            const void *w, const float *b, const float *run_mean,
                            const void *saved, float *dw, float *db, float *dgamma,
                            float *dbeta, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Backward, both halves in one call (Table 2, Tune row; Sec. 3.2.1): dX and the parameter gradients exactly
+ * as convbn_tune_bwd_data followed by convbn_tune_bwd_weight define them, same arguments, same outputs.
+ * For the 1x1, stride-1 layers of a bottleneck (bf16 NHWC, one of C_in / C_out equal to 64 and the other
+ * 128 or 256, at least 512 pixels) one kernel reads every dZ tile from memory ONCE and feeds both the
+ * data-gradient and the weight-gradient GEMM from it (omega' = s omega is formed in shared memory and never
+ * written); every other layer runs the two calls above one after the other.  dx may not alias dz or x.
+ * Workspace: convbn_workspace_bytes(desc, CONVBN_PHASE_TUNE_BWD). */
+int convbn_tune_bwd(const convbn_desc *desc, const void *dz, const void *x, const void *w, const float *b,
+                    const float *run_mean, const void *saved, void *dx, float *dw, float *db, float *dgamma,
+                    float *dbeta, void *workspace, size_t workspace_bytes, void *stream);
 
 /* Parameter gradients for callers that cannot allocate device memory (the paper has no counterpart
  * of this call; it exists for integration reasons only).
@@ -240,7 +252,8 @@ const char *convbn_status_string(int status);
 
 /* Name of the kernel family the last call of `phase` selected on this thread, for logs and tests:
  * "direct", "umma", "umma-strip", "umma-strided", "umma-subpixel", "umma-stem", "stem-mma", "depthwise",
- * "grouped-mma", "grouped-umma".  Static string, never NULL. */
+ * "grouped-mma", "grouped-umma", and for CONVBN_PHASE_TUNE_BWD "umma-fused-bwd" or "two-calls".
+ * Static string, never NULL. */
 const char *convbn_last_kernel(int phase);
 
 #ifdef __cplusplus

@@ -17,7 +17,7 @@ F32, BF16 = 0, 1
 NCHW, NHWC = 0, 1
 MODE_TUNE, MODE_EVAL, MODE_DEPLOY = 0, 1, 2
 (PHASE_TUNE_FWD, PHASE_TUNE_BWD_DATA, PHASE_TUNE_BWD_WEIGHT, PHASE_EVAL_FWD, PHASE_EVAL_BWD,
- PHASE_DEPLOY_FWD, PHASE_DEPLOY_BWD) = range(7)
+ PHASE_DEPLOY_FWD, PHASE_DEPLOY_BWD, PHASE_TUNE_BWD) = range(8)
 
 EXPORTS = (
     "convbn_out_shape", "convbn_saved_bytes", "convbn_workspace_bytes", "convbn_tune_fwd",
@@ -25,7 +25,7 @@ EXPORTS = (
     "convbn_deploy_prepare", "convbn_deploy_fwd", "convbn_deploy_bwd", "convbn_check",
     "convbn_status_string", "convbn_last_kernel", "convbn_host_step_arena_bytes",
     "convbn_tune_step_host", "convbn_profile_begin", "convbn_profile_end",
-    "convbn_tune_bwd_weight_noalloc", "convbn_selftest_wait_timeout",
+    "convbn_tune_bwd_weight_noalloc", "convbn_selftest_wait_timeout", "convbn_tune_bwd",
 )
 
 
@@ -144,6 +144,15 @@ def convbn_tune_bwd_weight(desc, dz, x, w, b, run_mean, saved, dw, db, dgamma, d
                                         _ptr(dgamma), _ptr(dbeta), _ptr(workspace),
                                         ctypes.c_size_t(wb), _stream(stream)),
            "convbn_tune_bwd_weight")
+
+
+def convbn_tune_bwd(desc, dz, x, w, b, run_mean, saved, dx, dw, db, dgamma, dbeta, workspace=None,
+                    workspace_bytes: Optional[int] = None, stream=None):
+    wb = _nbytes(workspace) if workspace_bytes is None else workspace_bytes
+    _raise(lib().convbn_tune_bwd(ctypes.byref(desc), _ptr(dz), _ptr(x), _ptr(w), _ptr(b), _ptr(run_mean),
+                                 _ptr(saved), _ptr(dx), _ptr(dw), _ptr(db), _ptr(dgamma), _ptr(dbeta),
+                                 _ptr(workspace), ctypes.c_size_t(wb), _stream(stream)),
+           "convbn_tune_bwd")
 
 
 def convbn_tune_bwd_weight_noalloc(desc, dz, x, w, b, run_mean, saved, dw, db, dgamma, dbeta,

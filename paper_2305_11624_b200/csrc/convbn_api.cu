@@ -17,7 +17,7 @@ using namespace convbn;
 namespace {
 
 thread_local const char *t_last_kernel[CONVBN_PHASE_COUNT] = {"none", "none", "none", "none",
-                                                              "none", "none", "none"};
+                                                              "none", "none", "none", "none"};
 
 // ---- optional per-kernel timing (CUDA events around every launch this library makes) ----------
 struct ProfRec { cudaEvent_t a, b; std::string name; };
@@ -126,8 +126,30 @@ struct Plan {
     UmmaWgradPlan uw;
 };
 
+bool fused_bwd_path(const convbn_desc *d, const Problem &pb) {
+    return d->dtype == CONVBN_BF16 && d->layout == CONVBN_NHWC && fused_bwd1x1_eligible(pb);
+}
+
 Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
     Plan pl;
+    if (phase == CONVBN_PHASE_TUNE_BWD) {
+        if (!fused_bwd_path(d, pb)) {       // the two calls one after the other, in the same workspace
+            const Plan a = make_plan(d, pb, CONVBN_PHASE_TUNE_BWD_DATA), b2 = make_plan(d, pb, CONVBN_PHASE_TUNE_BWD_WEIGHT);
+            pl.total = a.total > b2.total ? a.total : b2.total;
+            return pl;
+        }
+        size_t o = 0;
+        auto put = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 256); return r; };
+        pl.uw.splits = fused_bwd1x1_ctas(pb);
+        wgrad_epilogue_shape(pb, &pl.uw);
+        pl.bsplits = pl.uw.splits;
+        pl.partials = put((size_t)pl.uw.splits * pb.c_out * pb.kdim * sizeof(float));
+        pl.bsum = put((size_t)pl.uw.splits * pb.c_out * sizeof(float));
+        pl.dotpart = put((size_t)pl.uw.kt * pb.c_out * sizeof(float));
+        pl.counters = put((size_t)(pb.c_out / 32 + 1) * sizeof(unsigned int));
+        pl.total = o;
+        return pl;
+    }
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
     size_t wbytes = (size_t)pb.c_out * pb.kdim * elem_size(d->dtype);
@@ -699,6 +721,40 @@ int convbn_tune_bwd_weight(const convbn_desc *desc, const void *dz, const void *
     cudaStream_t st = (cudaStream_t)stream;
     CK(run_param_grads(desc, pb, pl, dz, x, w, (const float *)saved, b, run_mean, dw, db, dgamma, dbeta,
                        workspace, st, &t_last_kernel[CONVBN_PHASE_TUNE_BWD_WEIGHT]));
+    return CONVBN_OK;
+}
+
+int convbn_tune_bwd(const convbn_desc *desc, const void *dz, const void *x, const void *w, const float *b,
+                    const float *run_mean, const void *saved, void *dx, float *dw, float *db, float *dgamma,
+                    float *dbeta, void *workspace, size_t workspace_bytes, void *stream) {
+    Problem pb;
+    t_prof_phase = "bwd";
+    CK(make_problem(desc, &pb));
+    CK(check_pair(desc));
+    if (!dz || !x || !w || !run_mean || !saved || !dx || !dw || !dgamma || !dbeta) return CONVBN_EINVAL;
+    if ((b == nullptr) != (db == nullptr)) return CONVBN_EINVAL;
+    if (!aligned(dz, 16) || !aligned(x, 16) || !aligned(w, 16) || !aligned(saved, 16) || !aligned(dx, 16) ||
+        !aligned(dw, 16) || !aligned(b, 4) || !aligned(run_mean, 4) || !aligned(db, 4) || !aligned(dgamma, 4) ||
+        !aligned(dbeta, 4))
+        return CONVBN_EALIGN;
+    const Plan pl = make_plan(desc, pb, CONVBN_PHASE_TUNE_BWD);
+    CK(check_ws(pl, workspace, workspace_bytes));
+    if (!fused_bwd_path(desc, pb)) {
+        CK(convbn_tune_bwd_data(desc, dz, w, saved, dx, workspace, workspace_bytes, stream));
+        CK(convbn_tune_bwd_weight(desc, dz, x, w, b, run_mean, saved, dw, db, dgamma, dbeta, workspace, workspace_bytes,
+                                  stream));
+        t_last_kernel[CONVBN_PHASE_TUNE_BWD] = "two-calls";
+        return CONVBN_OK;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    float *partials = (float *)at(workspace, pl.partials), *bsum = (float *)at(workspace, pl.bsum);
+    float *dotpart = (float *)at(workspace, pl.dotpart);
+    unsigned int *counters = (unsigned int *)at(workspace, pl.counters);
+    const float *vec3 = (const float *)saved;
+    LAUNCH("umma_bwd", launch_fused_bwd1x1(pb, dz, x, w, vec3, dx, partials, bsum, counters, st));
+    LAUNCH("wgrad_epilogue_fused", launch_wgrad_epilogue_fused(pb, pl.uw, partials, bsum, w, vec3, b, run_mean, dw, dotpart,
+                                                               counters, db, dgamma, dbeta, true, st));
+    t_last_kernel[CONVBN_PHASE_TUNE_BWD] = "umma-fused-bwd";
     return CONVBN_OK;
 }
 

@@ -257,6 +257,14 @@ cudaError_t launch_bn_eval_finish(const Problem &pb, const float *part_g, const 
                                   int splits, const float *gamma, const float *var, float *db,
                                   float *dgamma, float *dbeta, cudaStream_t st);
 
+// ---- fused backward of 1x1 stride-1 layers (see umma_bwd1x1.cu) ----------------------------------------
+// dX plus one fp32 partial [C_in][C_out] and one row of sums of dZ per CTA (fused_bwd1x1_ctas of them), in the
+// layout the fused epilogue reads; `counters` are zeroed for it.  vec3 = saved [s | b' | r].
+bool fused_bwd1x1_eligible(const Problem &pb);
+int fused_bwd1x1_ctas(const Problem &pb);
+cudaError_t launch_fused_bwd1x1(const Problem &pb, const void *dz, const void *x, const void *w, const float *vec3,
+                                void *dx, float *partials, float *bsum, unsigned int *counters, cudaStream_t st);
+
 // One block, one bounded wait (limit_ns) on a barrier without arrivals: sets ERRW_TIMEOUT in the error word.
 cudaError_t launch_selftest_wait_timeout(unsigned long long limit_ns, cudaStream_t st);
 

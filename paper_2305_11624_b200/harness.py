@@ -48,7 +48,7 @@ class Block:
         self.z, self.dx = e(self.z_shape), e(self.x_shape)
         phases = []
         if "tune" in modes:
-            phases += [C.PHASE_TUNE_FWD, C.PHASE_TUNE_BWD_DATA, C.PHASE_TUNE_BWD_WEIGHT]
+            phases += [C.PHASE_TUNE_FWD, C.PHASE_TUNE_BWD_DATA, C.PHASE_TUNE_BWD_WEIGHT, C.PHASE_TUNE_BWD]
             self.saved = torch.empty(max(16, C.convbn_saved_bytes(self.desc, C.MODE_TUNE)),
                                      dtype=torch.uint8, device=self.device)
         if "eval" in modes:
@@ -138,10 +138,13 @@ class Block:
                                  self.dw, self.db, self.dgamma, self.dbeta, self.workspace,
                                  stream=stream)
 
+    def tune_bwd(self, stream=None):
+        C.convbn_tune_bwd(self.desc, self.dz, self.x, self.w, self.b, self.mu_hat, self.saved, self.dx, self.dw,
+                          self.db, self.dgamma, self.dbeta, self.workspace, stream=stream)
+
     def tune_step(self, stream=None):
         self.tune_fwd(stream)
-        self.tune_bwd_data(stream)
-        self.tune_bwd_weight(stream)
+        self.tune_bwd(stream)
 
     # ---- Eval mode -------------------------------------------------------------------------
     def eval_fwd(self, stream=None):
