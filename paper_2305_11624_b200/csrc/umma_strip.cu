@@ -21,6 +21,8 @@
 // The weight tiles either stream through a 4-slot ring, once per tile, or - when the whole matrix of the
 // CTA's output channels fits beside the patch buffers - are loaded once and stay resident, which makes small
 // tiles (more rounds over the SMs, better balance) free of weight traffic.
+#include <string.h>
+
 #include "kernels.h"
 #include "sm100_ptx.cuh"
 
@@ -400,7 +402,27 @@ struct StripPlan { bool ok = false; int bn = 64, R = 0, CW = 0, Wt = 0, nmb = 0,
 
 int strip_sm_count() { return device_sm_count(); }
 
+StripPlan plan_strip_search(const UmmaConvShape &s);
+
+// The search below runs a double loop over tile shapes and is asked for several times per library call
+// (eligibility, workspace size, launch): its result is cached per thread, keyed by the shape and the SM count.
 StripPlan plan_strip(const UmmaConvShape &s) {
+    struct Entry { UmmaConvShape key; int sms; StripPlan plan; bool used; };
+    thread_local Entry cache[16] = {};
+    thread_local int next = 0;
+    const int sms = strip_sm_count();
+    for (const Entry &e : cache)
+        if (e.used && e.sms == sms && memcmp(&e.key, &s, sizeof(UmmaConvShape)) == 0) return e.plan;
+    Entry &slot = cache[next];
+    next = (next + 1) % 16;
+    memcpy(&slot.key, &s, sizeof(UmmaConvShape));
+    slot.sms = sms;
+    slot.plan = plan_strip_search(s);
+    slot.used = true;
+    return slot.plan;
+}
+
+StripPlan plan_strip_search(const UmmaConvShape &s) {
     StripPlan best;
     if (s.stride_h != 1 || s.stride_w != 1 || s.dil_h != 1 || s.dil_w != 1 || s.out_sw) return best;
     if (s.blockdiag && s.ca != s.cn) return best;
