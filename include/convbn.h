@@ -87,6 +87,15 @@ typedef struct convbn_desc {
  * CONVBN_EINVAL if the descriptor is inconsistent or the output would be empty. */
 int convbn_out_shape(const convbn_desc *desc, int *h_out, int *w_out);
 
+/* Linear-BN block (Sec. 3.2.2, last sentence: the associative law holds for a linear layer followed by
+ * BatchNorm too): Y = X W^T + b on a [rows, in_features] matrix, W [out_features, in_features], BatchNorm over
+ * the features.  That is the 1x1 block on `rows` images of one pixel, and in both supported layouts the
+ * matrices already have the memory order the convolution entry points expect (X row-major [rows][in],
+ * W row-major [out][in], Z [rows][out]).  Fills `desc` (host) so that every Tune / Eval / Deploy entry point
+ * above serves the Linear-BN block; dtype CONVBN_BF16 selects the NHWC convention, CONVBN_F32 NCHW.
+ * CONVBN_EINVAL for non-positive sizes or an unknown dtype. */
+int convbn_linear_desc(int rows, int in_features, int out_features, int dtype, double eps, convbn_desc *desc);
+
 /* Bytes of the opaque `saved` buffer that a forward call of `mode` (convbn_mode) writes for its
  * backward calls - the activation kept beside X (Sec. 3.3 / 3.4, Appendix M memory analysis):
  *   TUNE   : three fp32 vectors s, b', r (omega' is re-formed from omega in backward, it is

@@ -25,7 +25,7 @@ EXPORTS = (
     "convbn_deploy_prepare", "convbn_deploy_fwd", "convbn_deploy_bwd", "convbn_check",
     "convbn_status_string", "convbn_last_kernel", "convbn_host_step_arena_bytes",
     "convbn_tune_step_host", "convbn_profile_begin", "convbn_profile_end",
-    "convbn_tune_bwd_weight_noalloc", "convbn_selftest_wait_timeout", "convbn_tune_bwd",
+    "convbn_tune_bwd_weight_noalloc", "convbn_selftest_wait_timeout", "convbn_tune_bwd", "convbn_linear_desc",
 )
 
 
@@ -109,6 +109,14 @@ def convbn_out_shape(desc: Desc):
     _raise(lib().convbn_out_shape(ctypes.byref(desc), ctypes.byref(ho), ctypes.byref(wo)),
            "convbn_out_shape")
     return ho.value, wo.value
+
+
+def convbn_linear_desc(rows: int, in_features: int, out_features: int, dtype: int = BF16, eps: float = 1e-5) -> Desc:
+    """Descriptor under which the convolution entry points compute a Linear-BN block on a [rows, in] matrix."""
+    d = Desc()
+    _raise(lib().convbn_linear_desc(ctypes.c_int(rows), ctypes.c_int(in_features), ctypes.c_int(out_features),
+                                    ctypes.c_int(dtype), ctypes.c_double(eps), ctypes.byref(d)), "convbn_linear_desc")
+    return d
 
 
 def convbn_saved_bytes(desc: Desc, mode: int) -> int:

@@ -608,6 +608,19 @@ int convbn_out_shape(const convbn_desc *desc, int *h_out, int *w_out) {
     return CONVBN_OK;
 }
 
+int convbn_linear_desc(int rows, int in_features, int out_features, int dtype, double eps, convbn_desc *desc) {
+    if (!desc || rows <= 0 || in_features <= 0 || out_features <= 0 || !(eps >= 0.0)) return CONVBN_EINVAL;
+    if (dtype != CONVBN_F32 && dtype != CONVBN_BF16) return CONVBN_EINVAL;
+    memset(desc, 0, sizeof(*desc));
+    desc->n = rows; desc->c_in = in_features; desc->h_in = 1; desc->w_in = 1;
+    desc->c_out = out_features; desc->kh = 1; desc->kw = 1;
+    desc->stride_h = desc->stride_w = desc->dil_h = desc->dil_w = desc->groups = 1;
+    desc->dtype = dtype;
+    desc->layout = dtype == CONVBN_BF16 ? CONVBN_NHWC : CONVBN_NCHW;
+    desc->eps = eps;
+    return CONVBN_OK;
+}
+
 size_t convbn_saved_bytes(const convbn_desc *desc, int mode) {
     Problem pb;
     if (make_problem(desc, &pb) != CONVBN_OK) return 0;
