@@ -323,10 +323,28 @@ def bench_config(ctx, wl):
             b.randomize(I.config_seed(wl, li) + 7919 * (rank * sets + si))
     stream = torch.cuda.current_stream()
     calls_per_step = 2 * len(layers)             # convbn_tune_fwd and convbn_tune_bwd per layer
+    # --dp-allreduce: the layers' parameter gradients are views of one fp32 bucket per buffer set, summed over
+    # the ranks at the end of every step (the only exchange data-parallel Tune mode needs); default: replicas
+    buckets = None
+    if args.dp_allreduce and world > 1:
+        from paper_2305_11624_b200.dataparallel import GradientBucket
+        buckets = []
+        for bs in blocks:
+            sizes = GradientBucket.sizes_for([(b.spec.name, b.spec.c_out, b.dw.numel() // b.spec.c_out, b.db is not None)
+                                              for b in bs])
+            bk = GradientBucket(sizes, device=dev)
+            for b in bs:
+                b.dw, b.dgamma, b.dbeta = (bk.views[b.spec.name + k] for k in (".dw", ".dgamma", ".dbeta"))
+                if b.db is not None:
+                    b.db = bk.views[b.spec.name + ".db"]
+            buckets.append(bk)
 
     def step(i):
         for b in blocks[i % sets]:
             b.tune_step(stream)
+        if buckets:
+            buckets[i % sets].all_reduce_async()
+            buckets[i % sets].wait()
 
     def barrier():
         if world > 1:
@@ -341,7 +359,7 @@ def bench_config(ctx, wl):
     # ---- timed region: K steps, each a replay of the CUDA graph of one step (one graph per buffer set), so
     # the launches of a step cost no host time; --no-graph times eager calls.
     graphs, launch_mode = None, "eager library calls"
-    if not args.no_graph:
+    if not args.no_graph and not buckets:        # (the collective is issued eagerly, outside a captured graph)
         try:
             graphs = []
             for si in range(sets):
@@ -651,7 +669,9 @@ def run_ours(args):
                                          % ", ".join(str(w) for w in workloads if w in DENSE or len(workloads) == 1),
                            "l2": "inputs larger than L2: per configuration, rotating buffer sets that together exceed "
                                  "twice the L2 (see per_config[].l2); warm numbers beside them",
-                           "flops_per_step": flops_total, "parallelism": "replicas x%d" % world,
+                           "flops_per_step": flops_total,
+                           "parallelism": ("data parallel x%d, gradient all-reduce per step" if args.dp_allreduce and world > 1
+                                           else "replicas x%d") % world,
                            "launch": headline[0]["launch"]},
                 "clocks": merge_clocks([c["clocks"] for c in per_config]), "e2e": e2e,
                 "gpu_launches": sum(r["gpu_launches"] for r in raw),
@@ -676,6 +696,8 @@ def main():
     ap.add_argument("--no-modes", action="store_true", help="skip the Tune / Eval / Deploy comparison")
     ap.add_argument("--no-graph", action="store_true", help="time eager library calls instead of graph replays")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--dp-allreduce", action="store_true",
+                    help="with N > 1 ranks: sum the parameter gradients over the ranks every step (default: replicas)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
