@@ -1,12 +1,13 @@
 #!/usr/bin/env python
 """Benchmark of the Tune-mode ConvBN hot path on B200.
 
-A step is one pass of the whole path - convbn_tune_fwd, convbn_tune_bwd_data and
-convbn_tune_bwd_weight - over every layer of a configuration.  With no ``--workload`` all five
+A step is one pass of the whole path - convbn_tune_fwd, then convbn_tune_bwd (input and parameter
+gradients in one call) - over every layer of a configuration.  With no ``--workload`` all five
 configurations run in one process and ONE JSON line is printed: ``value`` is the fwd+bwd TFLOP/s
 over the three dense bf16 configurations (1-3: total FLOPs / total time), ``per_config`` holds
 every configuration on its own (config 4 in GB/s against the copy bandwidth, config 0 as a
-latency).  FLOPs = 3 phases x 2 P C_out (C_in/G) kh kw per layer.
+latency), ``backbone`` a whole ResNet-50 (batch 32 at 224x224) replayed in Tune, Eval and Deploy mode
+with time per iteration and peak memory.  FLOPs = 3 phases x 2 P C_out (C_in/G) kh kw per layer.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload i]
 
@@ -605,6 +606,28 @@ def run_e2e(ctx, blks, stream, step_flops):
             "ms_per_step": ms / steps}
 
 
+def run_backbone(ctx, batch=32, size=224, iters=10):
+    """Forward + backward of all 53 ConvBN blocks of a ResNet-50 with their ReLUs and skip connections, in each
+    mode: time per iteration and peak bytes above parameters, gradients and inputs (Sec. 3.4, Fig. 3)."""
+    torch = ctx.torch
+    from paper_2305_11624_b200.backbone import BackboneReplay, resnet50_plan
+    stem, plan = resnet50_plan(size)
+    out = {"network": "ResNet-50 ConvBN blocks + ReLU + skip connections (max-pool replaced by synthetic tensors)",
+           "batch": batch, "image": size, "dtype": "bf16", "iters": iters, "modes": {}}
+    for mode in ("tune", "eval", "deploy"):
+        rp = BackboneReplay(batch, plan, mode, stem_hw=stem, device=ctx.dev)
+        ms, peak, how = rp.measure(iters=iters, warmup=3)
+        out["modes"][mode] = {"ms_per_iter": ms, "peak_bytes": peak, "tflops": rp.flops / ms / 1e9, "timing": how}
+        out["flops_per_iter"] = rp.flops
+        out["conv_bn_blocks"] = len(rp.layers)
+        del rp
+        torch.cuda.empty_cache()
+    m = out["modes"]
+    out["tune_vs_eval"] = {"time": m["tune"]["ms_per_iter"] / m["eval"]["ms_per_iter"],
+                           "peak_memory": m["tune"]["peak_bytes"] / m["eval"]["peak_bytes"]}
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -658,6 +681,11 @@ def run_ours(args):
         secs, fl = sum(c["seconds"] for c in cs), sum(c["flops"] for c in cs)
         cpu = {"value": fl / secs / 1e12, "unit": UNIT, "cores": cs[0]["cores"], "kind": "oracle",
                "sample": "one full step of every headline configuration of the fp64 oracle as it stands, %.1f s" % secs}
+    backbone = None
+    if rank == 0 and args.workload is None and not args.no_backbone:
+        backbone = run_backbone(ctx)
+    if world > 1:
+        dist.barrier()
     if rank == 0:
         names = [WORKLOAD_NAMES[w] for w in workloads]
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -675,7 +703,7 @@ def run_ours(args):
                            "launch": headline[0]["launch"]},
                 "clocks": merge_clocks([c["clocks"] for c in per_config]), "e2e": e2e,
                 "gpu_launches": sum(r["gpu_launches"] for r in raw),
-                "roofline": roofline, "cpu_baseline": cpu, "per_config": per_config}
+                "roofline": roofline, "cpu_baseline": cpu, "backbone": backbone, "per_config": per_config}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -696,6 +724,7 @@ def main():
     ap.add_argument("--no-modes", action="store_true", help="skip the Tune / Eval / Deploy comparison")
     ap.add_argument("--no-graph", action="store_true", help="time eager library calls instead of graph replays")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-backbone", action="store_true", help="skip the whole-ResNet-50 replay in the three modes")
     ap.add_argument("--dp-allreduce", action="store_true",
                     help="with N > 1 ranks: sum the parameter gradients over the ranks every step (default: replicas)")
     args = ap.parse_args()

@@ -25,7 +25,7 @@ EXPORTS = (
     "convbn_deploy_prepare", "convbn_deploy_fwd", "convbn_deploy_bwd", "convbn_check",
     "convbn_status_string", "convbn_last_kernel", "convbn_host_step_arena_bytes",
     "convbn_tune_step_host", "convbn_profile_begin", "convbn_profile_end",
-    "convbn_tune_bwd_weight_noalloc", "convbn_selftest_wait_timeout", "convbn_tune_bwd", "convbn_linear_desc",
+    "convbn_tune_bwd_weight_noalloc", "convbn_selftest_wait_timeout", "convbn_tune_bwd", "convbn_linear_desc", "convbn_relu", "convbn_add_relu", "convbn_relu_bwd", "convbn_add",
 )
 
 
@@ -216,6 +216,31 @@ def convbn_deploy_bwd(desc, dz, x, w_fused, dx, dw_fused, db_fused, workspace=No
                                    _ptr(dw_fused), _ptr(db_fused), _ptr(workspace),
                                    ctypes.c_size_t(wb), _stream(stream)),
            "convbn_deploy_bwd")
+
+
+def _dtype_of(t) -> int:
+    import torch
+    return BF16 if t.dtype == torch.bfloat16 else F32
+
+
+def convbn_relu(a, out, stream=None):
+    _raise(lib().convbn_relu(ctypes.c_int(_dtype_of(a)), _ptr(a), _ptr(out), ctypes.c_longlong(a.numel()), _stream(stream)),
+           "convbn_relu")
+
+
+def convbn_add_relu(a, b, out, stream=None):
+    _raise(lib().convbn_add_relu(ctypes.c_int(_dtype_of(a)), _ptr(a), _ptr(b), _ptr(out), ctypes.c_longlong(a.numel()),
+                                 _stream(stream)), "convbn_add_relu")
+
+
+def convbn_relu_bwd(a, y, out, stream=None):
+    _raise(lib().convbn_relu_bwd(ctypes.c_int(_dtype_of(a)), _ptr(a), _ptr(y), _ptr(out), ctypes.c_longlong(a.numel()),
+                                 _stream(stream)), "convbn_relu_bwd")
+
+
+def convbn_add(a, b, out, stream=None):
+    _raise(lib().convbn_add(ctypes.c_int(_dtype_of(a)), _ptr(a), _ptr(b), _ptr(out), ctypes.c_longlong(a.numel()),
+                            _stream(stream)), "convbn_add")
 
 
 def convbn_check(stream=None) -> None:

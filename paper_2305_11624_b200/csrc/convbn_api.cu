@@ -889,6 +889,26 @@ int convbn_check(void *stream) {
     return (word & ERRW_TIMEOUT) ? CONVBN_ETIMEOUT : CONVBN_OK;
 }
 
+static int glue_call(int mode, int dtype, const void *a, const void *b, void *out, long long count, void *stream) {
+    if (!a || !out || (mode != 0 && !b) || count < 0) return CONVBN_EINVAL;
+    if (dtype != CONVBN_F32 && dtype != CONVBN_BF16) return CONVBN_EINVAL;
+    if (!aligned(a, 16) || !aligned(out, 16) || !aligned(b, 16)) return CONVBN_EALIGN;
+    if (count == 0) return CONVBN_OK;
+    return launch_glue(mode, dtype, a, b, out, count, (cudaStream_t)stream) == cudaSuccess ? CONVBN_OK : CONVBN_ECUDA;
+}
+int convbn_relu(int dtype, const void *a, void *out, long long count, void *stream) {
+    return glue_call(0, dtype, a, nullptr, out, count, stream);
+}
+int convbn_add_relu(int dtype, const void *a, const void *b, void *out, long long count, void *stream) {
+    return glue_call(1, dtype, a, b, out, count, stream);
+}
+int convbn_relu_bwd(int dtype, const void *a, const void *y, void *out, long long count, void *stream) {
+    return glue_call(2, dtype, a, y, out, count, stream);
+}
+int convbn_add(int dtype, const void *a, const void *b, void *out, long long count, void *stream) {
+    return glue_call(3, dtype, a, b, out, count, stream);
+}
+
 int convbn_selftest_wait_timeout(void *stream) {
     if (launch_selftest_wait_timeout(100000ull, (cudaStream_t)stream) != cudaSuccess) return CONVBN_ECUDA;
     return CONVBN_OK;

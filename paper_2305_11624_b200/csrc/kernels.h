@@ -265,6 +265,9 @@ int fused_bwd1x1_ctas(const Problem &pb);
 cudaError_t launch_fused_bwd1x1(const Problem &pb, const void *dz, const void *x, const void *w, const float *vec3,
                                 void *dx, float *partials, float *bsum, unsigned int *counters, cudaStream_t st);
 
+// ---- elementwise glue between blocks (glue_kernels.cu): mode 0 relu(a), 1 relu(a + b), 2 a masked by b > 0, 3 a + b
+cudaError_t launch_glue(int mode, int dtype, const void *a, const void *b, void *out, long long count, cudaStream_t st);
+
 // One block, one bounded wait (limit_ns) on a barrier without arrivals: sets ERRW_TIMEOUT in the error word.
 cudaError_t launch_selftest_wait_timeout(unsigned long long limit_ns, cudaStream_t st);
 
