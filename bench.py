@@ -6,7 +6,7 @@ gradients in one call) - over every layer of a configuration.  With no ``--workl
 configurations run in one process and ONE JSON line is printed: ``value`` is the fwd+bwd TFLOP/s
 over the three dense bf16 configurations (1-3: total FLOPs / total time), ``per_config`` holds
 every configuration on its own (config 4 in GB/s against the copy bandwidth, config 0 as a
-latency), ``backbone`` a whole ResNet-50 (batch 32 at 224x224) replayed in Tune, Eval and Deploy mode
+latency), ``backbone`` a whole ResNet-50 (batch 32 and 256 at 224x224, batch 32 at 448x448) replayed in Tune, Eval and Deploy mode
 with time per iteration and peak memory.  FLOPs = 3 phases x 2 P C_out (C_in/G) kh kw per layer.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload i]
@@ -606,6 +606,13 @@ def run_e2e(ctx, blks, stream, step_flops):
             "ms_per_step": ms / steps}
 
 
+BACKBONE_CASES = ((32, 224), (256, 224), (32, 448))
+
+
+def run_backbones(ctx):
+    return [run_backbone(ctx, b, s, iters=10 if b * s * s <= 32 * 224 * 224 else 4) for b, s in BACKBONE_CASES]
+
+
 def run_backbone(ctx, batch=32, size=224, iters=10):
     """Forward + backward of all 53 ConvBN blocks of a ResNet-50 with their ReLUs and skip connections, in each
     mode: time per iteration and peak bytes above parameters, gradients and inputs (Sec. 3.4, Fig. 3)."""
@@ -683,7 +690,7 @@ def run_ours(args):
                "sample": "one full step of every headline configuration of the fp64 oracle as it stands, %.1f s" % secs}
     backbone = None
     if rank == 0 and args.workload is None and not args.no_backbone:
-        backbone = run_backbone(ctx)
+        backbone = run_backbones(ctx)
     if world > 1:
         dist.barrier()
     if rank == 0:

@@ -231,7 +231,7 @@ int convbn_tune_step_host(const convbn_desc *desc, const void *x, const void *dz
                           float *db, float *dgamma, float *dbeta, void *device_arena,
                           size_t arena_bytes, void *stream);
 
-/* ---- glue between blocks (Sec. 3.1: "not affected by the activation function or skip connection") ------ */
+/* ---- glue between blocks (Sec. 3.1: what surrounds a ConvBN block stays as it is) ------ */
 
 /* Elementwise operations a residual network places between its ConvBN blocks, on `count` elements of `dtype`
  * (convbn_dtype), all pointers device, 16-byte aligned; `out` may alias `a` (in place) or `b`.
@@ -239,7 +239,8 @@ int convbn_tune_step_host(const convbn_desc *desc, const void *x, const void *dz
  *   convbn_add_relu      out = max(a + b, 0)                    (the end of a residual block)
  *   convbn_relu_bwd      out = a where y > 0, else 0            (a: gradient of the ReLU output y)
  *   convbn_add           out = a + b                            (gradients meeting at a fork)
- * CONVBN_EINVAL for NULL pointers, a negative count or an unknown dtype; CONVBN_EALIGN; CONVBN_ECUDA. */
+ * A count of 0 is a no-op that looks at no pointer.  CONVBN_EINVAL for a negative count, an unknown dtype or (count > 0)
+ * a NULL pointer; CONVBN_EALIGN; CONVBN_ECUDA. */
 int convbn_relu(int dtype, const void *a, void *out, long long count, void *stream);
 int convbn_add_relu(int dtype, const void *a, const void *b, void *out, long long count, void *stream);
 int convbn_relu_bwd(int dtype, const void *a, const void *y, void *out, long long count, void *stream);

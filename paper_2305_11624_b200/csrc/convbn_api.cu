@@ -890,10 +890,10 @@ int convbn_check(void *stream) {
 }
 
 static int glue_call(int mode, int dtype, const void *a, const void *b, void *out, long long count, void *stream) {
-    if (!a || !out || (mode != 0 && !b) || count < 0) return CONVBN_EINVAL;
-    if (dtype != CONVBN_F32 && dtype != CONVBN_BF16) return CONVBN_EINVAL;
-    if (!aligned(a, 16) || !aligned(out, 16) || !aligned(b, 16)) return CONVBN_EALIGN;
+    if (count < 0 || (dtype != CONVBN_F32 && dtype != CONVBN_BF16)) return CONVBN_EINVAL;
     if (count == 0) return CONVBN_OK;
+    if (!a || !out || (mode != 0 && !b)) return CONVBN_EINVAL;
+    if (!aligned(a, 16) || !aligned(out, 16) || !aligned(b, 16)) return CONVBN_EALIGN;
     return launch_glue(mode, dtype, a, b, out, count, (cudaStream_t)stream) == cudaSuccess ? CONVBN_OK : CONVBN_ECUDA;
 }
 int convbn_relu(int dtype, const void *a, void *out, long long count, void *stream) {

@@ -114,3 +114,41 @@ def test_resnet50_plan_has_53_blocks():
     stem, plan = resnet50_plan(224)
     rp_layers = 1 + sum(3 + (1 if (b.stride > 1 or b.c_in != b.c_out) else 0) for b in plan)
     assert rp_layers == 53 and plan[0].hw == (56, 56) and plan[-1].hw == (7, 7) and plan[-1].c_out == 2048
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("count", [0, 1, 7, 8, 4099, 148 * 1024 * 9 + 3])
+def test_glue_operations_are_exact(dtype, count):
+    """ReLU, add + ReLU, ReLU backward and add: one rounding of an exactly representable result, so bit equality
+    with the same operation in numpy float64 rounded once to the storage type; ragged counts and in-place use."""
+    from paper_2305_11624_b200 import convbn as C
+    g = torch.Generator(device="cuda:0"); g.manual_seed(count + 1)
+    pad = count + 8                    # keep a guard band behind the data: nothing past `count` may be written
+    a = torch.randn(pad, generator=g, device="cuda:0").to(dtype)
+    b = torch.randn(pad, generator=g, device="cuda:0").to(dtype)
+    y = torch.randn(pad, generator=g, device="cuda:0").to(dtype)
+    f = lambda t: t.float().cpu().numpy().astype(np.float64)
+    back = lambda r: torch.from_numpy(r).to(dtype).float().numpy()     # round to nearest even, once
+    fa, fb, fy = f(a), f(b), f(y)
+    guard = -7.0
+    for name, call, ref in (("relu", lambda o: C.convbn_relu(a, o), np.maximum(fa, 0)),
+                            ("add_relu", lambda o: C.convbn_add_relu(a, b, o), np.maximum(fa + fb, 0)),
+                            ("relu_bwd", lambda o: C.convbn_relu_bwd(a, y, o), fa * (fy > 0)),
+                            ("add", lambda o: C.convbn_add(a, b, o), fa + fb)):
+        out = torch.full((pad,), guard, dtype=dtype, device="cuda:0")
+        view = out[:count]
+        if count == 0:
+            view = out[:0]
+        # the binding takes the count from the first operand
+        args_a, args_b, args_y = a[:count], b[:count], y[:count]
+        {"relu": lambda: C.convbn_relu(args_a, view), "add_relu": lambda: C.convbn_add_relu(args_a, args_b, view),
+         "relu_bwd": lambda: C.convbn_relu_bwd(args_a, args_y, view), "add": lambda: C.convbn_add(args_a, args_b, view)}[name]()
+        C.convbn_check()
+        got = out.float().cpu().numpy()
+        assert np.array_equal(got[:count], back(ref[:count]) + 0.0), name       # (+0.0: -0 and +0 compare equal anyway)
+        assert np.all(got[count:] == guard), name
+    if count:
+        inplace = a[:count].clone()
+        C.convbn_add_relu(inplace, b[:count], inplace)
+        C.convbn_check()
+        assert np.array_equal(inplace.float().cpu().numpy(), back(np.maximum(fa + fb, 0)[:count]))
