@@ -36,13 +36,14 @@ constexpr int kSEpiWarp0 = 2 + kSIssuers;
 constexpr int kSThreads = 32 * (kSEpiWarp0 + 4 * kSEpiGroups);   // 2 loader, 4 issuer and 16 epilogue warps
 constexpr int kSBStages = 12;         // weight-tile ring: at most this many slots
 constexpr int kSMaxStrips = 4;        // patch buffers
+constexpr int kSMaxAcc = 4;           // accumulator sets (tiles in flight between the issuers and the epilogue)
 
 struct StripGemm {
     int n, ho, wo, cn, ca, kh, kw, lower_h, lower_w;
     int R, CW, Wt, rows_in, nmb;      // tile rows / columns, patch width, patch rows, M blocks of 128
     int tiles_h, tiles_w;
     uint32_t strip_bytes;             // one patch buffer (multiple of 1024)
-    int nacc;                         // accumulator sets in tensor memory (1 or 2)
+    int nacc;                         // accumulator sets in tensor memory (2 .. kSMaxAcc)
     int blockdiag;                    // grouped conv as block-diagonal 64-channel GEMMs: output block j reads input chunk j
     uint32_t tmem_cols;
     int nstrips;                      // patch buffers in the ring (2 .. kSMaxStrips)
@@ -60,10 +61,22 @@ struct StripCtl {
     uint64_t strip_full[kSMaxStrips], strip_empty[kSMaxStrips];
     uint64_t b_full[kSBStages], b_empty[kSBStages];
     uint64_t bres_full;               // resident weights have landed
-    uint64_t tmem_full[2], tmem_empty[2];
+    uint64_t tmem_full[kSMaxAcc], tmem_empty[kSMaxAcc];
     uint32_t tmem_base;
     int abort_flag;
 };
+
+// One stage of a 4 x 4 transpose inside a quad of lanes: the lane whose bit is set gives `lo` and takes the partner's
+// `hi` in its place; the other lane gives `hi` and takes the partner's `lo`.
+__device__ __forceinline__ void quad_swap(uint4 &lo, uint4 &hi, int mask, bool upper) {
+    const uint4 send = upper ? lo : hi;
+    uint4 recv;
+    recv.x = __shfl_xor_sync(0xffffffffu, send.x, mask);
+    recv.y = __shfl_xor_sync(0xffffffffu, send.y, mask);
+    recv.z = __shfl_xor_sync(0xffffffffu, send.z, mask);
+    recv.w = __shfl_xor_sync(0xffffffffu, send.w, mask);
+    if (upper) lo = recv; else hi = recv;
+}
 
 template <int BN>
 __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid_constant__ CUtensorMap tm_act,
@@ -97,7 +110,7 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
             CONVBN_TRACE_POINT(0);
             const uint32_t ni = (uint32_t)g.nissue;     // every issuer commits to the barriers its MMAs release
             for (int s = 0; s < kSMaxStrips; ++s) { mbar_init(&ctl->strip_full[s], 1); mbar_init(&ctl->strip_empty[s], ni); }
-            for (int s = 0; s < 2; ++s) { mbar_init(&ctl->tmem_full[s], ni); mbar_init(&ctl->tmem_empty[s], 4 * kSEpiGroups); }
+            for (int s = 0; s < kSMaxAcc; ++s) { mbar_init(&ctl->tmem_full[s], ni); mbar_init(&ctl->tmem_empty[s], 4 * kSEpiGroups); }
             for (int s = 0; s < kSBStages; ++s) { mbar_init(&ctl->b_full[s], 1); mbar_init(&ctl->b_empty[s], ni); }
             mbar_init(&ctl->bres_full, 1);
             ctl->abort_flag = 0;
@@ -347,38 +360,56 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
                         }
                     }
                 } else {
+                // A lane holds one pixel's row of the accumulator; 32 lanes storing 16 bytes each, 2 BN bytes apart,
+                // would touch 32 lines per instruction.  The four lanes of a quad transpose their 4 x 4 blocks of
+                // 16-byte chunks instead, so that every store instruction writes 64 contiguous bytes per quad.
+                const int quad0 = lane & ~3, qc = lane & 3;
+                const unsigned long long optr = (unsigned long long)(uintptr_t)orow;
+                __nv_bfloat16 *rowp[4];
+                bool rowok[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const unsigned long long pk64 = __shfl_sync(0xffffffffu, optr, quad0 + k);
+                    rowp[k] = (__nv_bfloat16 *)(uintptr_t)pk64;
+                    rowok[k] = __shfl_sync(0xffffffffu, (int)store, quad0 + k) != 0;
+                }
 #pragma unroll 1
                 for (int c0 = 0; c0 < BN; c0 += 32) {
                     uint32_t vv[32];
                     tmem_ld_32x32(t_row + (uint32_t)c0, vv);
                     tmem_ld_wait();
-                    if (store) {
+                    uint4 pk[4];
 #pragma unroll
-                        for (int j = 0; j < 32; j += 8) {
-                            float f[8];
+                    for (int j = 0; j < 32; j += 8) {
+                        float f[8];
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(vv[j + e]);
-                            if (fold) {
-                                const float4 s0 = *(const float4 *)(scale_s + n0 + c0 + j);
-                                const float4 s1 = *(const float4 *)(scale_s + n0 + c0 + j + 4);
-                                f[0] *= s0.x; f[1] *= s0.y; f[2] *= s0.z; f[3] *= s0.w;
-                                f[4] *= s1.x; f[5] *= s1.y; f[6] *= s1.z; f[7] *= s1.w;
-                            }
-                            if (bias || fold) {
-                                const float4 b0 = *(const float4 *)(bias_s + n0 + c0 + j);
-                                const float4 b1 = *(const float4 *)(bias_s + n0 + c0 + j + 4);
-                                f[0] += b0.x; f[1] += b0.y; f[2] += b0.z; f[3] += b0.w;
-                                f[4] += b1.x; f[5] += b1.y; f[6] += b1.z; f[7] += b1.w;
-                            }
-                            uint4 pk;
-                            __nv_bfloat162 hh;
-                            hh = __floats2bfloat162_rn(f[0], f[1]); pk.x = *(uint32_t *)&hh;
-                            hh = __floats2bfloat162_rn(f[2], f[3]); pk.y = *(uint32_t *)&hh;
-                            hh = __floats2bfloat162_rn(f[4], f[5]); pk.z = *(uint32_t *)&hh;
-                            hh = __floats2bfloat162_rn(f[6], f[7]); pk.w = *(uint32_t *)&hh;
-                            *(uint4 *)(orow + c0 + j) = pk;
+                        for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(vv[j + e]);
+                        if (fold) {
+                            const float4 s0 = *(const float4 *)(scale_s + n0 + c0 + j);
+                            const float4 s1 = *(const float4 *)(scale_s + n0 + c0 + j + 4);
+                            f[0] *= s0.x; f[1] *= s0.y; f[2] *= s0.z; f[3] *= s0.w;
+                            f[4] *= s1.x; f[5] *= s1.y; f[6] *= s1.z; f[7] *= s1.w;
                         }
+                        if (bias || fold) {
+                            const float4 b0 = *(const float4 *)(bias_s + n0 + c0 + j);
+                            const float4 b1 = *(const float4 *)(bias_s + n0 + c0 + j + 4);
+                            f[0] += b0.x; f[1] += b0.y; f[2] += b0.z; f[3] += b0.w;
+                            f[4] += b1.x; f[5] += b1.y; f[6] += b1.z; f[7] += b1.w;
+                        }
+                        __nv_bfloat162 hh;
+                        hh = __floats2bfloat162_rn(f[0], f[1]); pk[j >> 3].x = *(uint32_t *)&hh;
+                        hh = __floats2bfloat162_rn(f[2], f[3]); pk[j >> 3].y = *(uint32_t *)&hh;
+                        hh = __floats2bfloat162_rn(f[4], f[5]); pk[j >> 3].z = *(uint32_t *)&hh;
+                        hh = __floats2bfloat162_rn(f[6], f[7]); pk[j >> 3].w = *(uint32_t *)&hh;
                     }
+                    // butterfly transpose: afterwards pk[k] of lane (quad0 + c) is chunk c of row (quad0 + k)
+                    quad_swap(pk[0], pk[1], 1, (lane & 1) != 0);
+                    quad_swap(pk[2], pk[3], 1, (lane & 1) != 0);
+                    quad_swap(pk[0], pk[2], 2, (lane & 2) != 0);
+                    quad_swap(pk[1], pk[3], 2, (lane & 2) != 0);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        if (rowok[k]) *(uint4 *)(rowp[k] + c0 + qc * 8) = pk[k];
                 }
                 }
             }
@@ -482,6 +513,8 @@ StripPlan plan_strip_search(const UmmaConvShape &s) {
                                 cchunks / 32.0;
         const double tile_clk = (mma_clk > fill_clk ? mma_clk : fill_clk) + 500.0;
         const long long tiles = (long long)s.n * tiles_h * tiles_w * n_tiles;
+        // (Tiles of fewer than four M blocks were measured and lose: with two blocks in flight the MMAs of one
+        // accumulator wait for each other, 75 clocks per 128 x 64 x 16 MMA instead of 57, and the tile count grows.)
         const double cost = (double)((tiles + sms - 1) / sms) * tile_clk + (resident ? (double)wall / 32.0 : 0.0);
         if (best_cost < 0 || cost < best_cost) {
             best_cost = cost;
@@ -489,6 +522,7 @@ StripPlan plan_strip_search(const UmmaConvShape &s) {
             best.ok = true; best.bn = bn; best.R = r; best.CW = cw; best.Wt = wt; best.nmb = nmb;
             best.strip_bytes = sbytes; best.smem = smem; best.tiles_w = tiles_w;
             best.nstrips = nstrips; best.resident = resident ? 1 : 0; best.bstages = bstages;
+            best.nacc = 512 / (bn * nmb) < kSMaxAcc ? 512 / (bn * nmb) : kSMaxAcc;
         }
     }
     }
@@ -549,14 +583,14 @@ cudaError_t launch_umma_strip_conv(const UmmaConvShape &s, const void *act, cons
     g.R = pl.R; g.CW = pl.CW; g.Wt = pl.Wt; g.rows_in = pl.R + s.taps_h - 1; g.nmb = pl.nmb;
     g.tiles_h = (s.ho + pl.R - 1) / pl.R; g.tiles_w = (s.wo + pl.CW - 1) / pl.CW;
     g.strip_bytes = pl.strip_bytes;
-    g.nacc = 2;
+    g.nacc = pl.nacc;
     g.nstrips = pl.nstrips; g.resident = pl.resident; g.bstages = pl.bstages;
     g.nissue = pl.nmb < kSIssuers ? pl.nmb : kSIssuers;
     g.blockdiag = s.blockdiag;
     g.sub_cin = s.sub_cin; g.sub_hin = s.sub_hin; g.sub_win = s.sub_win;
     g.sub_wide = (s.sub_cin > 0 && s.cn != 16) ? 1 : 0;
     for (int c = 0; c < 4; ++c) g.sub_mask[c] = s.sub_mask[c];
-    int cols = 2 * pl.nmb * pl.bn, p2 = 32;
+    int cols = pl.nacc * pl.nmb * pl.bn, p2 = 32;
     while (p2 < cols) p2 <<= 1;
     g.tmem_cols = (uint32_t)p2;
     g.out = (__nv_bfloat16 *)out;
