@@ -74,7 +74,7 @@ def kernel_bytes(kind, spec, out_hw):
 # DRAM bytes (read + write) per launch, from ncu captures of the kernels as they are now; a kernel that
 # changed after its capture has no entry (traffic: null).  key: (kernel family, layer).
 NCU_TRAFFIC = {("stem_fwd", "c2s"): 63.19e6, ("stem_dgrad", "c2s"): 116.28e6, ("stem_wgrad", "c2s"): 126.66e6,
-               ("umma_bwd", "c1a"): 76.34e6, ("strip_fwd", "c1b"): 12.96e6, ("strip_dgrad", "c1b"): 12.96e6,
+               ("umma_bwd", "c1a"): 76.34e6,
                ("umma_fwd", "c2a"): 14.99e6, ("umma_dgrad", "c2a"): 5.35e6, ("umma_wgrad", "c2a"): 16.10e6,
                ("umma_fwd", "c2b"): 7.98e6}
 
