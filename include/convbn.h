@@ -231,6 +231,31 @@ int convbn_tune_step_host(const convbn_desc *desc, const void *x, const void *dz
                           float *db, float *dgamma, float *dbeta, void *device_arena,
                           size_t arena_bytes, void *stream);
 
+/* ---- TransposedConv-BN in Tune mode (Sec. 3.2.2: the rewrite holds for any linear layer in front of a frozen BatchNorm;
+ *      Sec. 3.3 definitions; Table 2, Tune row, with the transposed convolution in place of the convolution) ------------
+ *
+ * `desc` describes the TRANSPOSED convolution in its own terms: input [n][c_in][h_in][w_in] (logical), output
+ * [n][c_out][h_out][w_out] with h_out = (h_in - 1) stride_h - 2 pad_h + dil_h (kh - 1) + 1 (no output padding), input pixel
+ * (hi, wi) adding x[ci] w[ci][co][r][q] to output pixel (hi stride_h - pad_h + r dil_h, wi stride_w - pad_w + q dil_w).
+ * Weights: NHWC descriptors [c_in][kh][kw][c_out/groups], NCHW descriptors [c_in][c_out/groups][kh][kw] (the layout of
+ * the convolution this layer transposes, whose c_out is this c_in).  BatchNorm vectors, `saved` ([s | b' | r],
+ * 3 c_out floats) and parameter gradients as in the convolution calls; dw has the layout of w, fp32.
+ *   Z  = convT(X, s w) + b'                      convbn_tconv_tune_fwd  (writes z and saved)
+ *   dX, dw = s dw', db = s dbeta, dgamma = r (sum dw' w + dbeta (b - mu_hat)), dbeta = sum dZ
+ *                                                convbn_tconv_tune_bwd  (b and db both NULL or both non-NULL)
+ * The transposed convolution runs on the kernels of the convolution it transposes (forward = that layer's backward data,
+ * input gradient = its forward, weight gradient = its weight gradient with the two tensors exchanged); the scale, the bias
+ * and the per-channel sums are separate small kernels.  One workspace size serves both calls.  Pointers: device, 16-byte
+ * aligned (vectors 4), workspace 256.  Errors as for the convolution calls; nothing is launched after an error. */
+int convbn_tconv_out_shape(const convbn_desc *desc, int *h_out, int *w_out);
+size_t convbn_tconv_workspace_bytes(const convbn_desc *desc);
+int convbn_tconv_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const float *b, const float *gamma,
+                          const float *beta, const float *run_mean, const float *run_var, void *z, void *saved,
+                          void *workspace, size_t workspace_bytes, void *stream);
+int convbn_tconv_tune_bwd(const convbn_desc *desc, const void *dz, const void *x, const void *w, const float *b,
+                          const float *run_mean, const void *saved, void *dx, float *dw, float *db, float *dgamma,
+                          float *dbeta, void *workspace, size_t workspace_bytes, void *stream);
+
 /* ---- glue between blocks (Sec. 3.1: what surrounds a ConvBN block stays as it is) ------ */
 
 /* Elementwise operations a residual network places between its ConvBN blocks, on `count` elements of `dtype`

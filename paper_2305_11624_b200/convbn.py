@@ -26,6 +26,7 @@ EXPORTS = (
     "convbn_status_string", "convbn_last_kernel", "convbn_host_step_arena_bytes",
     "convbn_tune_step_host", "convbn_profile_begin", "convbn_profile_end",
     "convbn_tune_bwd_weight_noalloc", "convbn_selftest_wait_timeout", "convbn_tune_bwd", "convbn_linear_desc", "convbn_relu", "convbn_add_relu", "convbn_relu_bwd", "convbn_add",
+    "convbn_tconv_out_shape", "convbn_tconv_workspace_bytes", "convbn_tconv_tune_fwd", "convbn_tconv_tune_bwd",
 )
 
 
@@ -161,6 +162,34 @@ def convbn_tune_bwd(desc, dz, x, w, b, run_mean, saved, dx, dw, db, dgamma, dbet
                                  _ptr(saved), _ptr(dx), _ptr(dw), _ptr(db), _ptr(dgamma), _ptr(dbeta),
                                  _ptr(workspace), ctypes.c_size_t(wb), _stream(stream)),
            "convbn_tune_bwd")
+
+
+def convbn_tconv_out_shape(desc):
+    h, w = ctypes.c_int(0), ctypes.c_int(0)
+    _raise(lib().convbn_tconv_out_shape(ctypes.byref(desc), ctypes.byref(h), ctypes.byref(w)), "convbn_tconv_out_shape")
+    return h.value, w.value
+
+
+def convbn_tconv_workspace_bytes(desc) -> int:
+    f = lib().convbn_tconv_workspace_bytes
+    f.restype = ctypes.c_size_t
+    return int(f(ctypes.byref(desc)))
+
+
+def convbn_tconv_tune_fwd(desc, x, w, b, gamma, beta, run_mean, run_var, z, saved, workspace=None,
+                          workspace_bytes: Optional[int] = None, stream=None):
+    wb = _nbytes(workspace) if workspace_bytes is None else workspace_bytes
+    _raise(lib().convbn_tconv_tune_fwd(ctypes.byref(desc), _ptr(x), _ptr(w), _ptr(b), _ptr(gamma), _ptr(beta),
+                                       _ptr(run_mean), _ptr(run_var), _ptr(z), _ptr(saved), _ptr(workspace),
+                                       ctypes.c_size_t(wb), _stream(stream)), "convbn_tconv_tune_fwd")
+
+
+def convbn_tconv_tune_bwd(desc, dz, x, w, b, run_mean, saved, dx, dw, db, dgamma, dbeta, workspace=None,
+                          workspace_bytes: Optional[int] = None, stream=None):
+    wb = _nbytes(workspace) if workspace_bytes is None else workspace_bytes
+    _raise(lib().convbn_tconv_tune_bwd(ctypes.byref(desc), _ptr(dz), _ptr(x), _ptr(w), _ptr(b), _ptr(run_mean),
+                                       _ptr(saved), _ptr(dx), _ptr(dw), _ptr(db), _ptr(dgamma), _ptr(dbeta),
+                                       _ptr(workspace), ctypes.c_size_t(wb), _stream(stream)), "convbn_tconv_tune_bwd")
 
 
 def convbn_tune_bwd_weight_noalloc(desc, dz, x, w, b, run_mean, saved, dw, db, dgamma, dbeta,

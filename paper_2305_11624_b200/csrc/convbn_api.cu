@@ -882,6 +882,134 @@ int convbn_deploy_bwd(const convbn_desc *desc, const void *dz, const void *x, co
     return CONVBN_OK;
 }
 
+// ---- TransposedConv-BN -----------------------------------------------------------------------------
+namespace {
+
+// The convolution a transposed convolution transposes: its input is the transposed layer's OUTPUT.
+struct TconvView {
+    convbn_desc conv;          // descriptor of that convolution
+    Problem pb;                // and its problem
+    int h_out, w_out;          // output extent of the transposed layer
+    size_t wcount;             // weight elements
+    size_t off_w, off_zero, off_dwp, off_bsum, off_inner, total;
+    int bsplits;
+    Problem sum_pb;            // a 1x1 problem whose output is the transposed layer's output (for the channel sums)
+    Plan fwd, bwd;             // plans of the inner convolution: plain forward, plain backward
+};
+
+int tconv_view(const convbn_desc *d, TconvView *v) {
+    if (!d) return CONVBN_EINVAL;
+    if (d->n <= 0 || d->c_in <= 0 || d->h_in <= 0 || d->w_in <= 0 || d->c_out <= 0 || d->kh <= 0 || d->kw <= 0 ||
+        d->stride_h <= 0 || d->stride_w <= 0 || d->pad_h < 0 || d->pad_w < 0 || d->dil_h <= 0 || d->dil_w <= 0 ||
+        d->groups <= 0)
+        return CONVBN_EINVAL;
+    const long long ho = (long long)(d->h_in - 1) * d->stride_h - 2LL * d->pad_h + (long long)d->dil_h * (d->kh - 1) + 1;
+    const long long wo = (long long)(d->w_in - 1) * d->stride_w - 2LL * d->pad_w + (long long)d->dil_w * (d->kw - 1) + 1;
+    if (ho <= 0 || wo <= 0 || ho > (1 << 24) || wo > (1 << 24)) return CONVBN_EINVAL;
+    v->h_out = (int)ho; v->w_out = (int)wo;
+    v->conv = *d;
+    v->conv.c_in = d->c_out; v->conv.c_out = d->c_in; v->conv.h_in = (int)ho; v->conv.w_in = (int)wo;
+    CK(make_problem(&v->conv, &v->pb));
+    CK(check_pair(&v->conv));
+    if (v->pb.h_out != d->h_in || v->pb.w_out != d->w_in) return CONVBN_EINVAL;
+    convbn_desc one = *d;
+    one.c_in = d->c_out; one.h_in = (int)ho; one.w_in = (int)wo; one.kh = one.kw = 1;
+    one.stride_h = one.stride_w = one.dil_h = one.dil_w = 1; one.pad_h = one.pad_w = 0; one.groups = 1;
+    CK(make_problem(&one, &v->sum_pb));
+    v->bsplits = channel_sum_splits(v->sum_pb);
+    v->fwd = make_plan(&v->conv, v->pb, CONVBN_PHASE_DEPLOY_FWD);
+    v->bwd = make_plan(&v->conv, v->pb, CONVBN_PHASE_DEPLOY_BWD);
+    v->wcount = (size_t)d->c_in * (d->c_out / d->groups) * d->kh * d->kw;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { const size_t at0 = off; off += (bytes + 255) / 256 * 256; return at0; };
+    v->off_w = take(v->wcount * elem_size(d->dtype));
+    v->off_zero = take((size_t)d->c_in * sizeof(float));
+    v->off_dwp = take(v->wcount * sizeof(float));
+    v->off_bsum = take((size_t)v->bsplits * d->c_out * sizeof(float));
+    v->off_inner = off;
+    v->total = off + (v->fwd.total > v->bwd.total ? v->fwd.total : v->bwd.total);
+    return CONVBN_OK;
+}
+
+}  // namespace
+
+int convbn_tconv_out_shape(const convbn_desc *desc, int *h_out, int *w_out) {
+    TconvView v;
+    CK(tconv_view(desc, &v));
+    if (!h_out || !w_out) return CONVBN_EINVAL;
+    *h_out = v.h_out; *w_out = v.w_out;
+    return CONVBN_OK;
+}
+
+size_t convbn_tconv_workspace_bytes(const convbn_desc *desc) {
+    TconvView v;
+    return tconv_view(desc, &v) == CONVBN_OK ? v.total : 0;
+}
+
+int convbn_tconv_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const float *b, const float *gamma,
+                          const float *beta, const float *run_mean, const float *run_var, void *z, void *saved,
+                          void *workspace, size_t workspace_bytes, void *stream) {
+    TconvView v;
+    t_prof_phase = "tconv_fwd";
+    CK(tconv_view(desc, &v));
+    if (!x || !w || !gamma || !beta || !run_mean || !run_var || !z || !saved) return CONVBN_EINVAL;
+    if (!aligned(x, 16) || !aligned(w, 16) || !aligned(z, 16) || !aligned(saved, 16) || !aligned(b, 4) ||
+        !aligned(gamma, 4) || !aligned(beta, 4) || !aligned(run_mean, 4) || !aligned(run_var, 4))
+        return CONVBN_EALIGN;
+    if (!workspace || workspace_bytes < v.total) return CONVBN_EWORKSPACE;
+    if (!aligned(workspace, 256)) return CONVBN_EALIGN;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool nhwc = desc->layout == CONVBN_NHWC;
+    const int taps = desc->kh * desc->kw, cig = desc->c_in / desc->groups, cog = desc->c_out / desc->groups;
+    float *vec3 = (float *)saved;
+    void *wf = at(workspace, v.off_w), *inner = at(workspace, v.off_inner);
+    LAUNCH("tconv_vec3", launch_tconv_vec3(desc->c_out, (float)desc->eps, b, gamma, beta, run_mean, run_var, vec3, st));
+    LAUNCH("tconv_rescale", launch_tconv_rescale(desc->dtype, nhwc, (long long)v.wcount, taps, cig, cog, w, vec3, wf, st));
+    // Z = omega' scattered over X: the backward-data pass of the convolution with the same weights
+    const char *which = nullptr;
+    CK(run_conv_dgrad(&v.conv, v.pb, x, wf, nullptr, at(inner, v.bwd.w_scaled), at(inner, v.bwd.wbd), z, st, &which));
+    const long long count = (long long)desc->n * desc->c_out * v.h_out * v.w_out;
+    LAUNCH("tconv_bias", launch_tconv_bias(desc->dtype, nhwc, count, desc->c_out, (long long)v.h_out * v.w_out,
+                                           vec3 + desc->c_out, z, st));
+    return CONVBN_OK;
+}
+
+int convbn_tconv_tune_bwd(const convbn_desc *desc, const void *dz, const void *x, const void *w, const float *b,
+                          const float *run_mean, const void *saved, void *dx, float *dw, float *db, float *dgamma,
+                          float *dbeta, void *workspace, size_t workspace_bytes, void *stream) {
+    TconvView v;
+    t_prof_phase = "tconv_bwd";
+    CK(tconv_view(desc, &v));
+    if (!dz || !x || !w || !run_mean || !saved || !dx || !dw || !dgamma || !dbeta) return CONVBN_EINVAL;
+    if ((b == nullptr) != (db == nullptr)) return CONVBN_EINVAL;
+    if (!aligned(dz, 16) || !aligned(x, 16) || !aligned(w, 16) || !aligned(saved, 16) || !aligned(dx, 16) ||
+        !aligned(dw, 16) || !aligned(b, 4) || !aligned(run_mean, 4) || !aligned(db, 4) || !aligned(dgamma, 4) ||
+        !aligned(dbeta, 4))
+        return CONVBN_EALIGN;
+    if (!workspace || workspace_bytes < v.total) return CONVBN_EWORKSPACE;
+    if (!aligned(workspace, 256)) return CONVBN_EALIGN;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool nhwc = desc->layout == CONVBN_NHWC;
+    const int taps = desc->kh * desc->kw, cig = desc->c_in / desc->groups, cog = desc->c_out / desc->groups;
+    const float *vec3 = (const float *)saved;
+    void *wf = at(workspace, v.off_w), *inner = at(workspace, v.off_inner);
+    float *zero = (float *)at(workspace, v.off_zero), *dwp = (float *)at(workspace, v.off_dwp);
+    float *bsum = (float *)at(workspace, v.off_bsum);
+    // omega' is re-formed from omega and the saved scale (Sec. 3.4: Tune mode keeps X and a few vectors)
+    LAUNCH("tconv_rescale", launch_tconv_rescale(desc->dtype, nhwc, (long long)v.wcount, taps, cig, cog, w, vec3, wf, st));
+    CU(cudaMemsetAsync(zero, 0, (size_t)desc->c_in * sizeof(float), st));
+    // dX gathers dZ through omega': the forward pass of that convolution, without a bias
+    const char *which = nullptr;
+    CK(run_conv_fwd(&v.conv, v.pb, dz, wf, zero, dx, v.fwd, inner, st, &which));
+    // domega' contracts X with windows of dZ: that convolution's weight gradient with the two tensors exchanged
+    CK(run_param_grads(&v.conv, v.pb, v.bwd, x, dz, wf, nullptr, nullptr, nullptr, dwp, nullptr, nullptr, nullptr, inner,
+                       st, &which));
+    LAUNCH("channel_sum", launch_channel_sum_partial(v.sum_pb, desc->dtype, desc->layout, dz, bsum, v.bsplits, st));
+    LAUNCH("tconv_epilogue", launch_tconv_param_epilogue(desc->dtype, nhwc, desc->c_out, taps, cig, cog, dwp, w, vec3, b,
+                                                         run_mean, bsum, v.bsplits, dw, db, dgamma, dbeta, st));
+    return CONVBN_OK;
+}
+
 int convbn_check(void *stream) {
     if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return CONVBN_ECUDA;
     int word = 0;

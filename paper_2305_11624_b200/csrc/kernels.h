@@ -271,4 +271,19 @@ cudaError_t launch_glue(int mode, int dtype, const void *a, const void *b, void 
 // One block, one bounded wait (limit_ns) on a barrier without arrivals: sets ERRW_TIMEOUT in the error word.
 cudaError_t launch_selftest_wait_timeout(unsigned long long limit_ns, cudaStream_t st);
 
+// ---- TransposedConv-BN: pointwise pieces around the convolution kernels (tconv_kernels.cu) ---------------
+// Weights [C_in][taps][C_out/G] (nhwc) or [C_in][C_out/G][taps]; the scale belongs to the output channel
+// co = (ci / cig) cog + j.
+cudaError_t launch_tconv_vec3(int c_out, float eps, const float *b, const float *gamma, const float *beta,
+                              const float *mean, const float *var, float *vec3, cudaStream_t st);
+cudaError_t launch_tconv_rescale(int dtype, bool nhwc, long long count, int taps, int cig, int cog, const void *w,
+                                 const float *s, void *w_out, cudaStream_t st);
+cudaError_t launch_tconv_bias(int dtype, bool nhwc, long long count, int c, long long hw, const float *bias, void *z,
+                              cudaStream_t st);
+// dwp: fp32 domega' in the weight layout; bsum: [bsplits][C_out] partial sums of dZ
+cudaError_t launch_tconv_param_epilogue(int dtype, bool nhwc, int c_out, int taps, int cig, int cog, const float *dwp,
+                                        const void *w, const float *vec3, const float *b, const float *mean,
+                                        const float *bsum, int bsplits, float *dw, float *db, float *dgamma,
+                                        float *dbeta, cudaStream_t st);
+
 }  // namespace convbn

@@ -116,3 +116,91 @@ def test_gradients_match_finite_differences(case):
     np.testing.assert_allclose(g["dbeta"], dz.sum(axis=(0, 2, 3)))
     s, _ = T.scale(p["gamma"], p["var_hat"], 1e-5)
     np.testing.assert_allclose(g["db"], s * g["dbeta"])
+
+
+# ---- the library against the oracle ----------------------------------------------------------------------------
+GPU_CASES = [  # (dtype, n, c_in, h, w, c_out, k, stride, pad, dil, groups, bias)
+    ("f32", 2, 3, 4, 5, 4, 3, 1, 0, 1, 1, True),
+    ("f32", 1, 4, 5, 4, 6, 2, 2, 0, 1, 1, True),
+    ("f32", 2, 4, 3, 4, 2, 3, 2, 1, 1, 2, False),
+    ("f32", 1, 2, 3, 3, 2, 3, 1, 2, 2, 1, True),
+    ("bf16", 2, 128, 28, 28, 64, 2, 2, 0, 1, 1, False),     # U-Net up-sampling: kernel = stride = 2
+    ("bf16", 2, 64, 16, 20, 64, 4, 2, 1, 1, 1, True),       # kernel 4, stride 2, pad 1
+    ("bf16", 2, 64, 30, 30, 128, 3, 1, 1, 1, 1, False),     # stride 1: the strip kernel on both passes
+    ("bf16", 3, 64, 9, 11, 64, 3, 2, 1, 1, 2, True),        # two groups, ragged extent
+    ("bf16", 1, 256, 56, 56, 128, 2, 2, 0, 1, 1, False),    # several tiles per CTA
+]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("case", GPU_CASES, ids=lambda c: "%s_c%d_%dx%d_o%d_k%d_s%d_g%d" % (c[0], c[2], c[3], c[4], c[5], c[6], c[7], c[10]))
+def test_library_matches_the_oracle(case):
+    import parity
+    from paper_2305_11624_b200 import convbn as C
+    from paper_2305_11624_b200 import inputs as I
+    dtype, n, ci, h, w, co, k, st, pad, dil, grp, bias = case
+    bf = dtype == "bf16"
+    lay = "nhwc" if bf else "nchw"
+    rnd = (lambda a: I.round_bf16(a.astype(np.float32)).astype(np.float64)) if bf else (lambda a: a.astype(np.float32).astype(np.float64))
+    x = rnd(_rnd(1, n, ci, h, w))
+    wt = rnd(_rnd(2, ci, co // grp, k, k) * np.sqrt(2.0 / (ci // grp * k * k)))
+    ho, wo = T.out_hw(h, w, k, k, st, pad, dil)
+    dz = rnd(_rnd(3, n, co, ho, wo))
+    f32 = lambda a: a.astype(np.float32).astype(np.float64)
+    p = {key: f32(val) for key, val in _params(4, co).items()}
+    b = f32(_rnd(5, co) * 0.01) if bias else None
+    kw = dict(stride=st, pad=pad, dil=dil, groups=grp)
+    ref = T.tune_forward(x, wt, b, eps=1e-5, **p, **kw)
+    ref.update(T.tune_backward(dz, x, wt, b, p["gamma"], p["mu_hat"], p["var_hat"], 1e-5, **kw))
+
+    dev = "cuda:0"
+    tdt = torch.bfloat16 if bf else torch.float32
+    up = lambda a, dt=torch.float32: torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).reshape(-1).to(dt).to(dev)
+    desc = C.Desc.make(n, ci, h, w, co, k, k, st, st, pad, pad, dil, dil, grp, C.BF16 if bf else C.F32, C.NHWC if bf else C.NCHW, 1e-5)
+    assert C.convbn_tconv_out_shape(desc) == (ho, wo)
+    X, W, DZ = up(I.act_to_layout(x, lay), tdt), up(I.weight_to_layout(wt, lay), tdt), up(I.act_to_layout(dz, lay), tdt)
+    G, Bt, M, V = (up(p[key]) for key in ("gamma", "beta", "mu_hat", "var_hat"))
+    Bv = up(b) if bias else None
+    Z = torch.full((n * co * ho * wo,), float("nan"), dtype=tdt, device=dev)
+    DX = torch.full((x.size,), float("nan"), dtype=tdt, device=dev)
+    DW = torch.full((wt.size,), float("nan"), device=dev)
+    DB = torch.full((co,), float("nan"), device=dev) if bias else None
+    DG, DBt = torch.full((co,), float("nan"), device=dev), torch.full((co,), float("nan"), device=dev)
+    saved = torch.empty(3 * co, device=dev)
+    ws = torch.empty(max(256, C.convbn_tconv_workspace_bytes(desc)), dtype=torch.uint8, device=dev)
+    C.convbn_tconv_tune_fwd(desc, X, W, Bv, G, Bt, M, V, Z, saved, ws)
+    C.convbn_tconv_tune_bwd(desc, DZ, X, W, Bv, M, saved, DX, DW, DB, DG, DBt, ws)
+    C.convbn_check()
+    dn = lambda t: t.float().cpu().numpy().astype(np.float64)
+    got = {"z": I.act_from_layout(dn(Z), lay, (n, co, ho, wo)), "dx": I.act_from_layout(dn(DX), lay, x.shape),
+           "dw": I.weight_from_layout(dn(DW), lay, wt.shape), "dgamma": dn(DG), "dbeta": dn(DBt)}
+    if bias:
+        got["db"] = dn(DB)
+    tol = parity.TOL[dtype]
+    errs = {key: O.rel_l2(val, ref[key]) for key, val in got.items()}
+    print(errs)
+    assert all(np.isfinite(v) and v <= tol for v in errs.values()), errs
+    # per element, on the activations (z carries two bf16 roundings: the convolution's and the bias add's)
+    for key in ("z", "dx"):
+        assert parity.elem_excess(got[key], ref[key], parity.ELEM_BOUND[dtype], channel_axis=1) <= 1.0, key
+
+
+def test_tconv_symbols_and_argument_checks():
+    from paper_2305_11624_b200 import convbn as C
+    d = C.Desc.make(1, 8, 4, 4, 8, 3, 3, 2, 2, 1, 1)
+    assert C.convbn_tconv_out_shape(d) == (7, 7)
+    assert C.convbn_tconv_workspace_bytes(d) > 0
+    bad = C.Desc.make(1, 8, 2, 2, 8, 1, 1, 1, 1, 3, 3)          # padding eats the whole output
+    with pytest.raises(C.ConvBNError):
+        C.convbn_tconv_out_shape(bad)
+    assert C.convbn_tconv_workspace_bytes(bad) == 0
+    with pytest.raises(C.ConvBNError) as e:                      # NULL pointers are refused before any launch
+        C.convbn_tconv_tune_fwd(d, None, None, None, None, None, None, None, None, None, None, 0, stream=0)
+    assert e.value.status == C.EINVAL
+    ok = 4096                                                    # fake aligned addresses: checks come before any launch
+    with pytest.raises(C.ConvBNError) as e:
+        C.convbn_tconv_tune_fwd(d, ok, ok, None, ok, ok, ok, ok, ok, ok, None, 0, stream=0)
+    assert e.value.status == C.EWORKSPACE
+    with pytest.raises(C.ConvBNError) as e:
+        C.convbn_tconv_tune_bwd(d, ok, ok, ok, ok, ok, ok, ok, ok, None, ok, ok, ok, 1 << 30, stream=0)
+    assert e.value.status == C.EINVAL                            # b without db
