@@ -72,11 +72,13 @@ def kernel_bytes(kind, spec, out_hw):
 
 
 # DRAM bytes (read + write) per launch, from ncu captures of the kernels as they are now; a kernel that
-# changed after its capture has no entry (traffic: null).  key: (kernel family, layer).
-NCU_TRAFFIC = {("stem_fwd", "c2s"): 63.19e6, ("stem_dgrad", "c2s"): 116.28e6, ("stem_wgrad", "c2s"): 126.66e6,
-               ("umma_bwd", "c1a"): 76.34e6,
-               ("umma_fwd", "c2a"): 14.99e6, ("umma_dgrad", "c2a"): 5.35e6, ("umma_wgrad", "c2a"): 16.10e6,
-               ("umma_fwd", "c2b"): 7.98e6}
+# changed after its capture has no entry (traffic: null).  key: (kernel family, layer) -> (bytes, summary file).
+_P1, _P2S, _P2D = ("profiles/config1_kernels_ncu_full.md", "profiles/config2_stem_window_kernels_ncu_full.md",
+                   "profiles/config2_dense_gemm_ncu_full.md")
+NCU_TRAFFIC = {("stem_fwd", "c2s"): (63.19e6, _P2S), ("stem_dgrad", "c2s"): (116.28e6, _P2S), ("stem_wgrad", "c2s"): (126.66e6, _P2S),
+               ("umma_bwd", "c1a"): (76.0e6, _P1), ("strip_fwd", "c1b"): (13.0e6, _P1), ("strip_dgrad", "c1b"): (13.0e6, _P1),
+               ("umma_fwd", "c2a"): (14.99e6, _P2D), ("umma_dgrad", "c2a"): (5.35e6, _P2D), ("umma_wgrad", "c2a"): (16.10e6, _P2D),
+               ("umma_fwd", "c2b"): (7.98e6, _P2D)}
 
 KIND_OF = {"strip_fwd": "fwd", "strip_dgrad": "dgrad", "direct_fwd": "fwd", "direct_dgrad": "dgrad", "direct_wgrad": "wgrad",
            "umma_fwd": "fwd", "umma_dgrad": "dgrad", "umma_wgrad": "wgrad", "umma_bwd": "bwd",
@@ -449,7 +451,7 @@ def bench_config(ctx, wl):
         fl = b.flops_per_phase() * (2 if kind == "bwd" else 1)
         by = kernel_bytes(kind, b.spec, (b.h_out, b.w_out))
         dense_bf16 = b.spec.dtype == "bf16" and b.spec.groups == 1
-        traffic = NCU_TRAFFIC.get((top["kernel"], top["layer"]))
+        traffic, traffic_from = NCU_TRAFFIC.get((top["kernel"], top["layer"]), (None, None))
         if dense_bf16 and fl / by > ridge:
             ach = fl / dur / 1e12
             r = {"bound": "tensor", "achieved": ach, "peak": tc, "unit": "TFLOP/s", "frac": ach / tc,
@@ -463,6 +465,7 @@ def bench_config(ctx, wl):
         r.update({"kernel": top["kernel"], "layer": top["layer"], "us_per_launch": dur * 1e6 / per_step,
                   "launches_per_step": per_step, "us_per_step": dur * 1e6, "algorithmic_bytes": by,
                   "algorithmic_flops": fl, "share_of_step": top["share"], "total_ms": top["total_ms"],
+                  "traffic_from": traffic_from,
                   "timing": "CUDA-event pair around each launch on the launching stream, eager pass"})
         return r
 
