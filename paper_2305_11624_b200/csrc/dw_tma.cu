@@ -81,7 +81,7 @@ struct DwTmaGeom {
 };
 
 template <int TW, int KH, int KW>
-__global__ void __launch_bounds__(288, 2) dw_tma_kernel(const __grid_constant__ CUtensorMap tx, DwTmaGeom g,
+__global__ void __launch_bounds__(TW >= 4 ? 384 : 288, TW >= 4 ? 1 : 2) dw_tma_kernel(const __grid_constant__ CUtensorMap tx, DwTmaGeom g,
                                                         const __nv_bfloat16 *__restrict__ w,
                                                         const float *__restrict__ bias, const BnFold fold,
                                                         const float *__restrict__ scale, int reverse_taps,
@@ -257,7 +257,7 @@ __global__ void __launch_bounds__(288, 2) dw_tma_kernel(const __grid_constant__ 
 // dZ) in registers across all the items of the block.  At the end the thread columns are added in
 // column order through shared memory, and the block writes one partial row: part[block][c][KH KW + 1].
 template <int TW, int KH, int KW>
-__global__ void __launch_bounds__(288, 2) dw_tma_wgrad_kernel(const __grid_constant__ CUtensorMap tx,
+__global__ void __launch_bounds__(TW >= 4 ? 384 : 288, TW >= 4 ? 1 : 2) dw_tma_wgrad_kernel(const __grid_constant__ CUtensorMap tx,
                                                               const __grid_constant__ CUtensorMap tdz, DwTmaGeom g,
                                                               float *__restrict__ part, int *err) {
     constexpr int NX = TW + KW - 1, NACC = KH * KW + 1;
@@ -460,7 +460,10 @@ bool dw_tma_eligible(const Problem &pb) {
 // column and row (X box plus, for the backward-weight kernel, the dZ box).
 static cudaError_t dw_tma_geometry(const Problem &pb, int tw, int kh, int kw, bool with_dz, DwTmaGeom *out,
                                    unsigned *grid) {
-    const int max_consumers = with_dz ? 256 : 256;            // consumer threads; the producer warp comes on top
+    // consumer threads (the producer warp comes on top): two blocks of 256 per SM, or one block of 352 when a
+    // thread owns four columns (its accumulators need the registers of a whole SM's worth of fewer threads)
+    const int max_consumers = tw >= 4 ? 352 : 256;
+    const size_t ring_budget = tw >= 4 ? 192 * 1024 : 96 * 1024;
     DwTmaGeom g{};
     g.n = pb.n; g.c = pb.c_in; g.h_in = pb.h_in; g.w_in = pb.w_in; g.h_out = pb.h_out; g.w_out = pb.w_out;
     g.pad_h = pb.pad_h; g.pad_w = pb.pad_w;
@@ -476,14 +479,14 @@ static cudaError_t dw_tma_geometry(const Problem &pb, int tw, int kh, int kw, bo
     g.row_bytes = (g.cols_t * tw + kw - 1) * pb.c_in * 2;
     g.stage_stride = (g.row_bytes + 127) / 128 * 128;
     if (with_dz) g.stage_stride += (g.cols_t * tw * pb.c_in * 2 + 127) / 128 * 128;
-    g.stages = (int)((96 * 1024) / g.stage_stride);
+    g.stages = (int)(ring_budget / g.stage_stride);
     if (g.stages > kDwMaxStages) g.stages = kDwMaxStages;
     if (g.stages < 4) return cudaErrorInvalidValue;
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    const long long resident = 2LL * sms;
+    const long long resident = (tw >= 4 ? 1LL : 2LL) * sms;
     // band height: the one that minimises (items per block, rounded up) x (input rows per item)
     long long best = -1;
     g.th = pb.h_out;
@@ -518,7 +521,7 @@ static size_t dw_tma_smem(const DwTmaGeom &g) {
 // kernel of the backward-data pass on the mirrored problem).
 cudaError_t launch_dw_tma(const Problem &pb, const void *x, const void *w, const float *bias, void *z,
                           cudaStream_t st, const BnFold *fold, const float *scale, bool reverse_taps) {
-    constexpr int TW = 2, KH = 3, KW = 3;
+    constexpr int TW = 4, KH = 3, KW = 3;
     DwTmaGeom g;
     unsigned grid = 0;
     cudaError_t e = dw_tma_geometry(pb, TW, KH, KW, false, &g, &grid);
@@ -528,7 +531,7 @@ cudaError_t launch_dw_tma(const Problem &pb, const void *x, const void *w, const
     int *err = nullptr;
     if ((e = error_word_address(&err)) != cudaSuccess) return e;
     static PerDevice attr;
-    if ((e = max_dynamic_smem_once(dw_tma_kernel<TW, KH, KW>, 110 * 1024, &attr)) != cudaSuccess) return e;
+    if ((e = max_dynamic_smem_once(dw_tma_kernel<TW, KH, KW>, 210 * 1024, &attr)) != cudaSuccess) return e;
     const BnFold none{nullptr, nullptr, nullptr, nullptr, nullptr, 0.f, nullptr};
     dw_tma_kernel<TW, KH, KW><<<grid, (g.consumer_warps + 1) * 32, dw_tma_smem(g), st>>>(
         tx, g, (const __nv_bfloat16 *)w, bias, fold ? *fold : none, scale, reverse_taps ? 1 : 0, (uint2 *)z, err);
@@ -539,13 +542,13 @@ cudaError_t launch_dw_tma(const Problem &pb, const void *x, const void *w, const
 size_t dw_tma_wgrad_partial_bytes(const Problem &pb) {
     DwTmaGeom g;
     unsigned grid = 0;
-    if (dw_tma_geometry(pb, 2, 3, 3, true, &g, &grid) != cudaSuccess) return 0;
+    if (dw_tma_geometry(pb, 4, 3, 3, true, &g, &grid) != cudaSuccess) return 0;
     return (size_t)grid * pb.c_in * 10 * sizeof(float);
 }
 
 cudaError_t launch_dw_tma_wgrad(const Problem &pb, const void *dz, const void *x, float *part, int *nparts,
                                 cudaStream_t st) {
-    constexpr int TW = 2, KH = 3, KW = 3;
+    constexpr int TW = 4, KH = 3, KW = 3;
     DwTmaGeom g;
     unsigned grid = 0;
     cudaError_t e = dw_tma_geometry(pb, TW, KH, KW, true, &g, &grid);
@@ -556,7 +559,7 @@ cudaError_t launch_dw_tma_wgrad(const Problem &pb, const void *dz, const void *x
     int *err = nullptr;
     if ((e = error_word_address(&err)) != cudaSuccess) return e;
     static PerDevice attr;
-    if ((e = max_dynamic_smem_once(dw_tma_wgrad_kernel<TW, KH, KW>, 110 * 1024, &attr)) != cudaSuccess) return e;
+    if ((e = max_dynamic_smem_once(dw_tma_wgrad_kernel<TW, KH, KW>, 210 * 1024, &attr)) != cudaSuccess) return e;
     dw_tma_wgrad_kernel<TW, KH, KW><<<grid, (g.consumer_warps + 1) * 32, dw_tma_smem(g), st>>>(tx, tdz, g, part, err);
     *nparts = (int)grid;
     return cudaGetLastError();

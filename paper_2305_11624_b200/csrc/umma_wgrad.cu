@@ -275,7 +275,7 @@ UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
 // lanes; few slices or very many blocks -> 32 rows x 1 lane (every block pays a fence and an atomic)
 void wgrad_epilogue_shape(const Problem &pb, UmmaWgradPlan *pl) {
     const long long blocks8 = (long long)(pb.c_out / 32) * ((pb.kdim + 7) / 8);
-    pl->kr = pl->splits > 192 ? 2 : ((pl->splits <= 8 || blocks8 > 1200) && blocks8 / 4 >= device_sm_count() ? 32 : 8);
+    pl->kr = pl->splits > 192 ? 2 : ((pl->splits <= 8 || blocks8 > 600) && blocks8 / 4 >= device_sm_count() ? 32 : 8);
     pl->kt = (pb.kdim + pl->kr - 1) / pl->kr;   // epilogue blocks along k = rows of dotpart
 }
 
