@@ -57,6 +57,7 @@ __global__ void __launch_bounds__(kGThreads) grouped8_conv_kernel(const __grid_c
         fence_barrier_init();
     }
     __syncthreads();
+    if (threadIdx.x == 0) { CONVBN_TRACE_POINT(0); }
     const uint32_t items = (uint32_t)g.n * g.tiles_h * chunks;   // chunk fastest: the chunks of a patch run together
     if (warp == 8) {
         if (lane == 0) {
@@ -117,6 +118,7 @@ __global__ void __launch_bounds__(kGThreads) grouped8_conv_kernel(const __grid_c
         __nv_bfloat16 *obase = out + ((size_t)((size_t)img * g.ho + h0) * g.wo) * g.c + ch0 + 2 * t;
         const int wrap_elems = (g.wo - g.Wt) * g.c;            // output offset of (row + 1, column - Wt)
         if (!mbar_wait_bounded(&ctl->full[s], ph, abort_flag)) { ok = false; break; }
+        if (threadIdx.x == 0) { if (it == blockIdx.x) CONVBN_TRACE_POINT(1); CONVBN_TRACE_POINT(3); }
         const uint32_t patch = smem_u32(ring + (size_t)s * g.stage_stride);
         // four 16-pixel tiles at a time: their MMA chains are independent, so the loads of one overlap
         // the arithmetic of the others
@@ -152,6 +154,7 @@ __global__ void __launch_bounds__(kGThreads) grouped8_conv_kernel(const __grid_c
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&ctl->empty[s]);
+        if (threadIdx.x == 0) { if (it == blockIdx.x) CONVBN_TRACE_POINT(2); CONVBN_TRACE_POINT(4); }
         if (++s == (uint32_t)g.stages) { s = 0; ph ^= 1u; }
     }
     if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
