@@ -56,7 +56,11 @@ typedef enum {
     CONVBN_ECAPACITY = 7     /* problem too large for the library's built-in scratch */
 } convbn_status;
 
-typedef enum { CONVBN_F32 = 0, CONVBN_BF16 = 1 } convbn_dtype;
+/* Storage type of x, w, z, dz, dx.  CONVBN_F16 (IEEE half; the paper's mixed-precision rows, Table 4) is implemented for
+ * the Tune-mode calls of dense NHWC layers whose channel counts are multiples of 64 (the tensor-core paths: fp16 operands,
+ * fp32 accumulation, fp32 parameter gradients) and for the elementwise glue; every other call returns CONVBN_EUNSUPPORTED
+ * for it. */
+typedef enum { CONVBN_F32 = 0, CONVBN_BF16 = 1, CONVBN_F16 = 2 } convbn_dtype;
 typedef enum { CONVBN_NCHW = 0, CONVBN_NHWC = 1 } convbn_layout;
 typedef enum { CONVBN_MODE_TUNE = 0, CONVBN_MODE_EVAL = 1, CONVBN_MODE_DEPLOY = 2 } convbn_mode;
 

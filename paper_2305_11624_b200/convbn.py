@@ -13,7 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIBRARY = os.path.join(_HERE, "libconvbn.so")
 
 OK, EINVAL, EUNSUPPORTED, EWORKSPACE, EALIGN, ECUDA, ETIMEOUT, ECAPACITY = range(8)
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2
 NCHW, NHWC = 0, 1
 MODE_TUNE, MODE_EVAL, MODE_DEPLOY = 0, 1, 2
 (PHASE_TUNE_FWD, PHASE_TUNE_BWD_DATA, PHASE_TUNE_BWD_WEIGHT, PHASE_EVAL_FWD, PHASE_EVAL_BWD,
@@ -249,7 +249,7 @@ def convbn_deploy_bwd(desc, dz, x, w_fused, dx, dw_fused, db_fused, workspace=No
 
 def _dtype_of(t) -> int:
     import torch
-    return BF16 if t.dtype == torch.bfloat16 else F32
+    return {torch.bfloat16: BF16, torch.float16: F16}.get(t.dtype, F32)
 
 
 def convbn_relu(a, out, stream=None):

@@ -3,8 +3,11 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+
+#include <type_traits>
 
 #include "../../include/convbn.h"
 
@@ -49,9 +52,43 @@ __host__ __device__ __forceinline__ void w_row_decode(int k, int cg, int kh, int
 
 __device__ __forceinline__ float to_f32(float v) { return v; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float to_f32(__half v) { return __half2float(v); }
 template <class T> __device__ __forceinline__ T from_f32(float v);
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+template <> __device__ __forceinline__ __half from_f32<__half>(float v) { return __float2half_rn(v); }
+
+// ---- the two 16-bit storage types ---------------------------------------------------------------------
+// The tensor-core kernels move 16-bit elements without looking at them (TMA, shared memory, MMA operands);
+// only four things depend on whether those bits are bf16 or IEEE half: the operand-format field of the MMA
+// instruction descriptor, the conversion of results, the conversion of weights that are rescaled on the way,
+// and the constant 1.  Kernels carry an `f16` flag (0: bf16, 1: half) instead of a second instantiation.
+__device__ __forceinline__ uint32_t pack2_h16(float a, float b, int f16) {
+    if (f16) { const __half2 h = __floats2half2_rn(a, b); return *reinterpret_cast<const uint32_t *>(&h); }
+    const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<const uint32_t *>(&h);
+}
+// The same with the type fixed at compile time, for the epilogue loops (one uniform branch per tile picks the loop).
+template <bool F16>
+__device__ __forceinline__ uint32_t pack2_t(float a, float b) {
+    if constexpr (F16) { const __half2 h = __floats2half2_rn(a, b); return *reinterpret_cast<const uint32_t *>(&h); }
+    else { const __nv_bfloat162 h = __floats2bfloat162_rn(a, b); return *reinterpret_cast<const uint32_t *>(&h); }
+}
+__device__ __forceinline__ uint16_t pack1_h16(float a, int f16) {
+    if (f16) { const __half h = __float2half_rn(a); return *reinterpret_cast<const uint16_t *>(&h); }
+    const __nv_bfloat16 h = __float2bfloat16_rn(a);
+    return *reinterpret_cast<const uint16_t *>(&h);
+}
+__device__ __forceinline__ float unpack_h16(uint16_t bits, int f16) {
+    if (f16) return __half2float(*reinterpret_cast<const __half *>(&bits));
+    return __uint_as_float((uint32_t)bits << 16);
+}
+__device__ __forceinline__ float load_h16(const void *p, int f16) { return unpack_h16(*reinterpret_cast<const uint16_t *>(p), f16); }
+__host__ __device__ constexpr uint32_t one_h16(int f16) { return f16 ? 0x3C00u : 0x3F80u; }
+// The storage type of the call in progress on this host thread (set by the entry points, read by the
+// launchers when they fill their kernels' parameter records).
+void set_call_f16(int f16);
+int call_f16();
 
 // Device error word: kernels that give up on a bounded wait OR a non-zero code into it.  The word
 // lives in one translation unit; kernels elsewhere get its device address as an argument.

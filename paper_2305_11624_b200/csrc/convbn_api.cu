@@ -67,7 +67,7 @@ int make_problem(const convbn_desc *d, Problem *pb) {
     const long long eh = (long long)d->h_in + 2LL * d->pad_h - (long long)d->dil_h * (d->kh - 1) - 1;
     const long long ew = (long long)d->w_in + 2LL * d->pad_w - (long long)d->dil_w * (d->kw - 1) - 1;
     if (eh < 0 || ew < 0) return CONVBN_EINVAL;
-    if (d->dtype != CONVBN_F32 && d->dtype != CONVBN_BF16) return CONVBN_EINVAL;
+    if (d->dtype != CONVBN_F32 && d->dtype != CONVBN_BF16 && d->dtype != CONVBN_F16) return CONVBN_EINVAL;
     if (d->layout != CONVBN_NCHW && d->layout != CONVBN_NHWC) return CONVBN_EINVAL;
     pb->n = d->n; pb->c_in = d->c_in; pb->h_in = d->h_in; pb->w_in = d->w_in;
     pb->c_out = d->c_out; pb->kh = d->kh; pb->kw = d->kw;
@@ -344,6 +344,33 @@ bool strided_dgrad_ok(const convbn_desc *d, const Problem &pb) {
            pb.pin < (1LL << 31) - 256;
 }
 
+// CONVBN_F16 calls.  IEEE half runs on the 16-bit tensor-core paths only: the descriptor is checked for them, then
+// the call proceeds as its bf16 twin with the half flag set for the launchers (operand format of the MMAs,
+// conversions of results and of rescaled weights, the constant 1).  The flag is cleared when the call returns.
+struct HalfCall {
+    convbn_desc d;
+    const convbn_desc *use;
+    int status = CONVBN_OK;
+    bool set_here = false;         // an entry point called from another one must not clear the caller's flag
+    explicit HalfCall(const convbn_desc *desc) : use(desc) {
+        if (!desc || desc->dtype != CONVBN_F16) return;
+        d = *desc;
+        d.dtype = CONVBN_BF16;
+        use = &d;
+        Problem pb;
+        status = make_problem(&d, &pb);
+        if (status != CONVBN_OK) return;
+        UmmaConvShape s;
+        const bool dense = d.layout == CONVBN_NHWC && pb.groups == 1 && pb.c_in % 64 == 0 && pb.c_out % 64 == 0 &&
+                           umma_fwd_shape(&d, pb, &s) && (umma_dgrad_shape(&d, pb, &s) || strided_dgrad_ok(&d, pb)) &&
+                           make_plan(&d, pb, CONVBN_PHASE_TUNE_BWD_WEIGHT).umma_wgrad;
+        if (!dense) { status = CONVBN_EUNSUPPORTED; return; }
+        set_call_f16(1);
+        set_here = true;
+    }
+    ~HalfCall() { if (set_here) set_call_f16(0); }
+};
+
 // Forward convolution with whatever weights / bias the mode folded: tensor cores when eligible.
 int run_conv_fwd(const convbn_desc *d, const Problem &pb, const void *x, const void *w, const float *bias,
                  void *z, const Plan &pl, void *ws, cudaStream_t st, const char **which) {
@@ -610,18 +637,21 @@ int convbn_out_shape(const convbn_desc *desc, int *h_out, int *w_out) {
 
 int convbn_linear_desc(int rows, int in_features, int out_features, int dtype, double eps, convbn_desc *desc) {
     if (!desc || rows <= 0 || in_features <= 0 || out_features <= 0 || !(eps >= 0.0)) return CONVBN_EINVAL;
-    if (dtype != CONVBN_F32 && dtype != CONVBN_BF16) return CONVBN_EINVAL;
+    if (dtype != CONVBN_F32 && dtype != CONVBN_BF16 && dtype != CONVBN_F16) return CONVBN_EINVAL;
     memset(desc, 0, sizeof(*desc));
     desc->n = rows; desc->c_in = in_features; desc->h_in = 1; desc->w_in = 1;
     desc->c_out = out_features; desc->kh = 1; desc->kw = 1;
     desc->stride_h = desc->stride_w = desc->dil_h = desc->dil_w = desc->groups = 1;
     desc->dtype = dtype;
-    desc->layout = dtype == CONVBN_BF16 ? CONVBN_NHWC : CONVBN_NCHW;
+    desc->layout = dtype == CONVBN_F32 ? CONVBN_NCHW : CONVBN_NHWC;
     desc->eps = eps;
     return CONVBN_OK;
 }
 
 size_t convbn_saved_bytes(const convbn_desc *desc, int mode) {
+    HalfCall half(desc);
+    if (half.status != CONVBN_OK) return 0;
+    desc = half.use;
     Problem pb;
     if (make_problem(desc, &pb) != CONVBN_OK) return 0;
     switch (mode) {
@@ -632,6 +662,9 @@ size_t convbn_saved_bytes(const convbn_desc *desc, int mode) {
 }
 
 size_t convbn_workspace_bytes(const convbn_desc *desc, int phase) {
+    HalfCall half(desc);
+    if (half.status != CONVBN_OK) return 0;
+    desc = half.use;
     Problem pb;
     if (phase < 0 || phase >= CONVBN_PHASE_COUNT) return 0;
     if (make_problem(desc, &pb) != CONVBN_OK) return 0;
@@ -642,6 +675,9 @@ int convbn_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const
                     const float *gamma, const float *beta, const float *run_mean,
                     const float *run_var, void *z, void *saved, void *workspace,
                     size_t workspace_bytes, void *stream) {
+    HalfCall half(desc);              // CONVBN_F16: checked here, then run as the 16-bit path with the half flag set
+    if (half.status != CONVBN_OK) return half.status;
+    desc = half.use;
     Problem pb;
     t_prof_phase = "fwd";
     CK(make_problem(desc, &pb));
@@ -699,6 +735,9 @@ int convbn_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const
 
 int convbn_tune_bwd_data(const convbn_desc *desc, const void *dz, const void *w, const void *saved,
                          void *dx, void *workspace, size_t workspace_bytes, void *stream) {
+    HalfCall half(desc);              // CONVBN_F16: checked here, then run as the 16-bit path with the half flag set
+    if (half.status != CONVBN_OK) return half.status;
+    desc = half.use;
     Problem pb;
     t_prof_phase = "bwd_data";
     CK(make_problem(desc, &pb));
@@ -719,6 +758,9 @@ int convbn_tune_bwd_weight(const convbn_desc *desc, const void *dz, const void *
                            const float *b, const float *run_mean, const void *saved, float *dw,
                            float *db, float *dgamma, float *dbeta, void *workspace,
                            size_t workspace_bytes, void *stream) {
+    HalfCall half(desc);              // CONVBN_F16: checked here, then run as the 16-bit path with the half flag set
+    if (half.status != CONVBN_OK) return half.status;
+    desc = half.use;
     Problem pb;
     t_prof_phase = "bwd_weight";
     CK(make_problem(desc, &pb));
@@ -740,6 +782,9 @@ int convbn_tune_bwd_weight(const convbn_desc *desc, const void *dz, const void *
 int convbn_tune_bwd(const convbn_desc *desc, const void *dz, const void *x, const void *w, const float *b,
                     const float *run_mean, const void *saved, void *dx, float *dw, float *db, float *dgamma,
                     float *dbeta, void *workspace, size_t workspace_bytes, void *stream) {
+    HalfCall half(desc);              // CONVBN_F16: checked here, then run as the 16-bit path with the half flag set
+    if (half.status != CONVBN_OK) return half.status;
+    desc = half.use;
     Problem pb;
     t_prof_phase = "bwd";
     CK(make_problem(desc, &pb));
@@ -1018,7 +1063,7 @@ int convbn_check(void *stream) {
 }
 
 static int glue_call(int mode, int dtype, const void *a, const void *b, void *out, long long count, void *stream) {
-    if (count < 0 || (dtype != CONVBN_F32 && dtype != CONVBN_BF16)) return CONVBN_EINVAL;
+    if (count < 0 || (dtype != CONVBN_F32 && dtype != CONVBN_BF16 && dtype != CONVBN_F16)) return CONVBN_EINVAL;
     if (count == 0) return CONVBN_OK;
     if (!a || !out || (mode != 0 && !b)) return CONVBN_EINVAL;
     if (!aligned(a, 16) || !aligned(out, 16) || !aligned(b, 16)) return CONVBN_EALIGN;

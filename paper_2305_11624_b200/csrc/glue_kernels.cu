@@ -1,7 +1,7 @@
 // Elementwise glue between ConvBN blocks of a residual network: ReLU and the skip-connection add.  They are not
 // part of the block (Sec. 3.1: the block is unaffected by the activation function or skip connection that
 // follows it), but a whole-backbone replay needs them between the blocks, on the same stream and without
-// allocations.  bf16 or fp32 storage, fp32 arithmetic, 16-byte accesses, grid-stride loops.
+// allocations.  bf16, half or fp32 storage, fp32 arithmetic, 16-byte accesses, grid-stride loops.
 #include "kernels.h"
 
 namespace convbn {
@@ -10,6 +10,7 @@ namespace {
 
 template <class T> struct Vec;
 template <> struct Vec<__nv_bfloat16> { static constexpr int n = 8; };
+template <> struct Vec<__half> { static constexpr int n = 8; };
 template <> struct Vec<float> { static constexpr int n = 4; };
 
 template <class T>
@@ -18,7 +19,10 @@ __device__ __forceinline__ void load_vec(const T *p, float (&f)[Vec<T>::n]) {
     if constexpr (Vec<T>::n == 8) {
         const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(w[i] << 16); f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u); }
+        for (int i = 0; i < 4; ++i) {
+            f[2 * i] = unpack_h16((uint16_t)(w[i] & 0xFFFFu), sizeof(T) == 2 && !__is_same(T, __nv_bfloat16));
+            f[2 * i + 1] = unpack_h16((uint16_t)(w[i] >> 16), sizeof(T) == 2 && !__is_same(T, __nv_bfloat16));
+        }
     } else {
         f[0] = __uint_as_float(q.x); f[1] = __uint_as_float(q.y); f[2] = __uint_as_float(q.z); f[3] = __uint_as_float(q.w);
     }
@@ -29,7 +33,7 @@ __device__ __forceinline__ void store_vec(T *p, const float (&f)[Vec<T>::n]) {
     if constexpr (Vec<T>::n == 8) {
         uint32_t w[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) { const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]); w[i] = *(const uint32_t *)&h; }
+        for (int i = 0; i < 4; ++i) w[i] = pack2_h16(f[2 * i], f[2 * i + 1], !__is_same(T, __nv_bfloat16));
         q = make_uint4(w[0], w[1], w[2], w[3]);
     } else {
         q = make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
@@ -84,6 +88,15 @@ cudaError_t launch_glue_t(const void *a, const void *b, void *out, long long cou
 }  // namespace
 
 cudaError_t launch_glue(int mode, int dtype, const void *a, const void *b, void *out, long long count, cudaStream_t st) {
+    if (dtype == CONVBN_F16) {
+        switch (mode) {
+            case 0: return launch_glue_t<__half, 0>(a, b, out, count, st);
+            case 1: return launch_glue_t<__half, 1>(a, b, out, count, st);
+            case 2: return launch_glue_t<__half, 2>(a, b, out, count, st);
+            case 3: return launch_glue_t<__half, 3>(a, b, out, count, st);
+            default: return cudaErrorInvalidValue;
+        }
+    }
     const bool bf = dtype == CONVBN_BF16;
     switch (mode) {
         case 0: return bf ? launch_glue_t<__nv_bfloat16, 0>(a, b, out, count, st) : launch_glue_t<float, 0>(a, b, out, count, st);

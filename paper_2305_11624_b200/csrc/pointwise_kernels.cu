@@ -8,6 +8,10 @@ namespace convbn {
 
 __device__ int g_error_word = 0;
 
+namespace { thread_local int t_call_f16 = 0; }
+void set_call_f16(int f16) { t_call_f16 = f16 ? 1 : 0; }
+int call_f16() { return t_call_f16; }
+
 int current_device_slot() {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
@@ -133,7 +137,7 @@ cudaError_t launch_rescale_weight(const Problem &pb, int dtype, const void *w, c
 __global__ void __launch_bounds__(256) reparam_dgrad_kernel(int c_out, int c_in, int taps,
                                                             const __nv_bfloat16 *__restrict__ w,
                                                             const float *__restrict__ s_vec,
-                                                            __nv_bfloat16 *__restrict__ w_t) {
+                                                            __nv_bfloat16 *__restrict__ w_t, int f16) {
     __shared__ float tile[32][33];
     pdl_wait();
     pdl_launch_dependents();
@@ -142,13 +146,13 @@ __global__ void __launch_bounds__(256) reparam_dgrad_kernel(int c_out, int c_in,
     for (int j = ty; j < 32; j += 8) {
         const int co = co0 + j, ci = ci0 + tx;
         if (co < c_out && ci < c_in)
-            tile[j][tx] = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((long long)co * taps + tap) * c_in + ci]);
+            tile[j][tx] = (s_vec ? s_vec[co] : 1.f) * load_h16(w + ((long long)co * taps + tap) * c_in + ci, f16);
     }
     __syncthreads();
     for (int j = ty; j < 32; j += 8) {
         const int ci = ci0 + j, co = co0 + tx;
         if (co < c_out && ci < c_in)
-            w_t[((long long)ci * taps + (taps - 1 - tap)) * c_out + co] = __float2bfloat16_rn(tile[tx][j]);
+            reinterpret_cast<uint16_t *>(w_t)[((long long)ci * taps + (taps - 1 - tap)) * c_out + co] = pack1_h16(tile[tx][j], f16);
     }
 }
 
@@ -156,7 +160,7 @@ __global__ void __launch_bounds__(256) reparam_dgrad_class_kernel(int c_out, int
                                                                   int q_max, int step_h, int step_w, int ctaps,
                                                                   const __nv_bfloat16 *__restrict__ w,
                                                                   const float *__restrict__ s_vec,
-                                                                  __nv_bfloat16 *__restrict__ w_t, int taps) {
+                                                                  __nv_bfloat16 *__restrict__ w_t, int taps, int f16) {
     __shared__ float tile[32][33];
     pdl_wait();
     pdl_launch_dependents();
@@ -167,13 +171,13 @@ __global__ void __launch_bounds__(256) reparam_dgrad_class_kernel(int c_out, int
     for (int j = ty; j < 32; j += 8) {
         const int co = co0 + j, ci = ci0 + tx;
         if (co < c_out && ci < c_in)
-            tile[j][tx] = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((long long)co * taps + tap) * c_in + ci]);
+            tile[j][tx] = (s_vec ? s_vec[co] : 1.f) * load_h16(w + ((long long)co * taps + tap) * c_in + ci, f16);
     }
     __syncthreads();
     for (int j = ty; j < 32; j += 8) {
         const int ci = ci0 + j, co = co0 + tx;
         if (co < c_out && ci < c_in)
-            w_t[((long long)ci * ctaps + ct) * c_out + co] = __float2bfloat16_rn(tile[tx][j]);
+            reinterpret_cast<uint16_t *>(w_t)[((long long)ci * ctaps + ct) * c_out + co] = pack1_h16(tile[tx][j], f16);
     }
 }
 
@@ -183,7 +187,7 @@ cudaError_t launch_reparam_dgrad_class(const Problem &pb, const void *w, const f
     static PerDevice carve;
     prefer_max_shared_once(reparam_dgrad_class_kernel, &carve);
     return launch_pdl(reparam_dgrad_class_kernel, grid, dim3(256), 0, st, pb.c_out, pb.c_in, pb.kw, tw, r_max, q_max,
-                      step_h, step_w, th * tw, (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t, pb.kh * pb.kw);
+                      step_h, step_w, th * tw, (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t, pb.kh * pb.kw, call_f16());
 }
 
 // All residue classes of a strided backward pass in one launch: tap t of the kernel belongs to exactly
@@ -192,7 +196,7 @@ cudaError_t launch_reparam_dgrad_class(const Problem &pb, const void *w, const f
 __global__ void __launch_bounds__(256) reparam_dgrad_classes_kernel(int c_out, int c_in, ClassTapTable where,
                                                                     const __nv_bfloat16 *__restrict__ w,
                                                                     const float *__restrict__ s_vec,
-                                                                    __nv_bfloat16 *__restrict__ w_t, int taps) {
+                                                                    __nv_bfloat16 *__restrict__ w_t, int taps, int f16) {
     __shared__ float tile[32][33];
     pdl_wait();
     pdl_launch_dependents();
@@ -204,12 +208,12 @@ __global__ void __launch_bounds__(256) reparam_dgrad_classes_kernel(int c_out, i
     for (int j = ty; j < 32; j += 8) {
         const int co = co0 + j, ci = ci0 + tx;
         if (co < c_out && ci < c_in)
-            tile[j][tx] = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((long long)co * taps + tap) * c_in + ci]);
+            tile[j][tx] = (s_vec ? s_vec[co] : 1.f) * load_h16(w + ((long long)co * taps + tap) * c_in + ci, f16);
     }
     __syncthreads();
     for (int j = ty; j < 32; j += 8) {
         const int ci = ci0 + j, co = co0 + tx;
-        if (co < c_out && ci < c_in) dst[((long long)ci * ctaps + ct) * c_out + co] = __float2bfloat16_rn(tile[tx][j]);
+        if (co < c_out && ci < c_in) reinterpret_cast<uint16_t *>(dst)[((long long)ci * ctaps + ct) * c_out + co] = pack1_h16(tile[tx][j], f16);
     }
 }
 
@@ -219,7 +223,7 @@ cudaError_t launch_reparam_dgrad_classes(const Problem &pb, const void *w, const
     static PerDevice carve;
     prefer_max_shared_once(reparam_dgrad_classes_kernel, &carve);
     return launch_pdl(reparam_dgrad_classes_kernel, grid, dim3(256), 0, st, pb.c_out, pb.c_in, where,
-                      (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t, pb.kh * pb.kw);
+                      (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t, pb.kh * pb.kw, call_f16());
 }
 
 cudaError_t launch_reparam_dgrad(const Problem &pb, const void *w, const float *s_vec, void *w_t,
@@ -228,7 +232,7 @@ cudaError_t launch_reparam_dgrad(const Problem &pb, const void *w, const float *
     static PerDevice carve;
     prefer_max_shared_once(reparam_dgrad_kernel, &carve);
     return launch_pdl(reparam_dgrad_kernel, grid, dim3(256), 0, st, pb.c_out, pb.c_in, pb.kh * pb.kw,
-                      (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t);
+                      (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)w_t, call_f16());
 }
 
 // ---- per-channel partial sums over pixel slices (Appendix B) --------------------------------

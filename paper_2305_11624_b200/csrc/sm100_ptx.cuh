@@ -314,6 +314,10 @@ __host__ __device__ constexpr uint32_t idesc_bf16_f32(int m, int n, int a_mn_maj
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
            ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
+// The same with IEEE half operands when f16 != 0 (A and B format 0 = f16; both operands always share one type).
+__host__ __device__ constexpr uint32_t idesc_h16_f32(int m, int n, int a_mn_major, int b_mn_major, int f16) {
+    return idesc_bf16_f32(m, n, a_mn_major, b_mn_major) & (f16 ? ~((7u << 7) | (7u << 10)) : ~0u);
+}
 
 }  // namespace ptx
 }  // namespace convbn

@@ -26,6 +26,7 @@ struct FusedBwd {
     long long p;            // pixels
     int m_tiles;            // ceil(p / 128)
     const float *vec3;      // saved [s | b' | r]
+    int f16;                // 16-bit storage type: 0 bf16, 1 IEEE half
 };
 
 struct FbCtl {
@@ -85,7 +86,8 @@ __global__ void __launch_bounds__(kFbThreads) fused_bwd1x1_kernel(const __grid_c
         tmem_relinquish();
     }
     {
-        const uint4 one4 = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
+        const uint32_t one2 = one_h16(g.f16) * 0x10001u;
+        const uint4 one4 = make_uint4(one2, one2, one2, one2);
         for (int i = threadIdx.x; i < 1024 / 16; i += kFbThreads) ((uint4 *)ones)[i] = one4;
     }
     pdl_wait();
@@ -101,9 +103,8 @@ __global__ void __launch_bounds__(kFbThreads) fused_bwd1x1_kernel(const __grid_c
         uint32_t out[4];
 #pragma unroll
         for (int h = 0; h < 4; ++h) {
-            const float lo = __uint_as_float(in[h] << 16) * sc, hi = __uint_as_float(in[h] & 0xFFFF0000u) * sc;
-            const __nv_bfloat162 pk = __floats2bfloat162_rn(lo, hi);
-            out[h] = *(const uint32_t *)&pk;
+            const float lo = unpack_h16((uint16_t)(in[h] & 0xFFFFu), g.f16) * sc, hi = unpack_h16((uint16_t)(in[h] >> 16), g.f16) * sc;
+            out[h] = pack2_h16(lo, hi, g.f16);
         }
         *(uint4 *)(wres + (size_t)(ci >> 6) * (CO * 128) + co * 128 + (((((ci & 63) >> 3) ^ (co & 7)) & 7) << 4)) =
             make_uint4(out[0], out[1], out[2], out[3]);
@@ -143,9 +144,9 @@ __global__ void __launch_bounds__(kFbThreads) fused_bwd1x1_kernel(const __grid_c
         if (elect_one()) {
             const uint32_t hi = smem_desc_hi_sw128(1024);
             constexpr uint32_t kBox16 = kFbBox >> 4;
-            constexpr uint32_t idesc_dx = idesc_bf16_f32(128, CI, 0, 1);            // A = dZ (K-major), B = omega' (MN-major)
-            constexpr uint32_t idesc_dw = idesc_bf16_f32(128, S::kNarrow, 1, 1);    // both operands MN-major
-            constexpr uint32_t idesc_sum = idesc_bf16_f32(128, S::kWideIn ? CO : 16, 1, 1);
+            const uint32_t idesc_dx = idesc_h16_f32(128, CI, 0, 1, g.f16);          // A = dZ (K-major), B = omega' (MN-major)
+            const uint32_t idesc_dw = idesc_h16_f32(128, S::kNarrow, 1, 1, g.f16);  // both operands MN-major
+            const uint32_t idesc_sum = idesc_h16_f32(128, S::kWideIn ? CO : 16, 1, 1, g.f16);
             const uint32_t w_lo = smem_desc_lo(smem_u32(wres), CO * 128);           // N blocks CO * 128 bytes apart
             // a tile of ones of any extent: one 8 x 128-byte group, block stride 0, row-group stride 0
             const uint32_t ones_lo = smem_desc_lo(smem_u32(ones), 0), ones_hi = smem_desc_hi_sw128(0);
@@ -230,16 +231,19 @@ __global__ void __launch_bounds__(kFbThreads) fused_bwd1x1_kernel(const __grid_c
                 if (lane == 0) tma_store_wait_read<0>();
                 __syncwarp();
                 uint8_t *row = buf_s + lane * 128;
-#pragma unroll
-                for (int j = 0; j < 64; j += 8) {
-                    uint4 pk;
-                    __nv_bfloat162 h;
-                    h = __floats2bfloat162_rn(__uint_as_float(v[j]), __uint_as_float(v[j + 1])); pk.x = *(uint32_t *)&h;
-                    h = __floats2bfloat162_rn(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])); pk.y = *(uint32_t *)&h;
-                    h = __floats2bfloat162_rn(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5])); pk.z = *(uint32_t *)&h;
-                    h = __floats2bfloat162_rn(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7])); pk.w = *(uint32_t *)&h;
-                    *(uint4 *)(row + ((((j >> 3) ^ (lane & 7)) & 7) << 4)) = pk;
-                }
+                auto pack_rows = [&](auto half_tag) {
+                    constexpr bool H = decltype(half_tag)::value;
+    #pragma unroll
+                    for (int j = 0; j < 64; j += 8) {
+                        uint4 pk;
+                        pk.x = pack2_t<H>(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
+                        pk.y = pack2_t<H>(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                        pk.z = pack2_t<H>(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5]));
+                        pk.w = pack2_t<H>(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7]));
+                        *(uint4 *)(row + ((((j >> 3) ^ (lane & 7)) & 7) << 4)) = pk;
+                    }
+                };
+                if (g.f16) pack_rows(std::true_type{}); else pack_rows(std::false_type{});
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
@@ -337,7 +341,7 @@ cudaError_t launch_fused_bwd1x1(const Problem &pb, const void *dz, const void *x
                                 float *partials, float *bsum, unsigned int *counters, cudaStream_t st) {
     if (!fused_bwd1x1_eligible(pb)) return cudaErrorInvalidValue;
     FusedBwd g;
-    g.p = pb.p; g.m_tiles = (int)((pb.p + 127) / 128); g.vec3 = vec3;
+    g.p = pb.p; g.m_tiles = (int)((pb.p + 127) / 128); g.vec3 = vec3; g.f16 = call_f16();
     CUtensorMap tdz, tx, tdx;
     if (!make_tmap_matrix_bf16(&tdz, dz, pb.p, pb.c_out, 128, 64)) return cudaErrorInvalidValue;
     if (!make_tmap_matrix_bf16(&tx, x, pb.p, pb.c_in, 128, 64)) return cudaErrorInvalidValue;

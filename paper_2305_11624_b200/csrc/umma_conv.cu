@@ -47,6 +47,7 @@ struct ConvGemm {
     // row r), tiles are stem_th x stem_tw output patches (stem_th * stem_tw = 128), the output map is 4-D.
     int stem, stem_tw, stem_th, stem_tiles_w, stem_tiles_h;
     int resident;            // 1: the CTA's whole weight slab [BN][K] stays in shared memory (loaded once)
+    int f16;                 // 16-bit storage type: 0 bf16, 1 IEEE half
     BnFold fold;             // fold.gamma != NULL: scale and shift formed in the kernel from the BN parameters
 };
 
@@ -210,7 +211,7 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (elect_one()) {
-            constexpr uint32_t idesc = idesc_bf16_f32(kBM, BN, 0, 0);
+            const uint32_t idesc = idesc_h16_f32(kBM, BN, 0, 0, g.f16);
             const uint32_t hi = smem_desc_hi_sw128(1024);
             const uint32_t tiles_lo = smem_desc_lo(smem_u32(tiles), 16), slab_lo = smem_desc_lo(smem_u32(slab), 16);
             int s = 0;
@@ -303,11 +304,10 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                         for (int j = 0; j < 64; j += 8) {
                             if (c0 + j < ncols) {
                                 uint4 pk;
-                                __nv_bfloat162 h;
-                                h = __floats2bfloat162_rn(__uint_as_float(v[j]), __uint_as_float(v[j + 1])); pk.x = *(uint32_t *)&h;
-                                h = __floats2bfloat162_rn(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])); pk.y = *(uint32_t *)&h;
-                                h = __floats2bfloat162_rn(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5])); pk.z = *(uint32_t *)&h;
-                                h = __floats2bfloat162_rn(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7])); pk.w = *(uint32_t *)&h;
+                                pk.x = pack2_h16(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), g.f16);
+                                pk.y = pack2_h16(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]), g.f16);
+                                pk.z = pack2_h16(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5]), g.f16);
+                                pk.w = pack2_h16(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7]), g.f16);
                                 *(uint4 *)(srow + c0 + j) = pk;
                             }
                         }
@@ -319,31 +319,34 @@ __global__ void __launch_bounds__(kConvThreads) umma_conv_kernel(const __grid_co
                     if (lane == 0) tma_store_wait_read<0>();
                     __syncwarp();
                     uint8_t *row = buf + lane * 128;
-#pragma unroll
-                    for (int j = 0; j < 64; j += 8) {
-                        float f[8];
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[j + e]);
-                        if (fold) {
-                            const float4 s0 = *(const float4 *)(scale_s + n0 + c0 + j);
-                            const float4 s1 = *(const float4 *)(scale_s + n0 + c0 + j + 4);
-                            f[0] *= s0.x; f[1] *= s0.y; f[2] *= s0.z; f[3] *= s0.w;
-                            f[4] *= s1.x; f[5] *= s1.y; f[6] *= s1.z; f[7] *= s1.w;
+                    auto pack_rows = [&](auto half_tag) {
+                        constexpr bool H = decltype(half_tag)::value;
+    #pragma unroll
+                        for (int j = 0; j < 64; j += 8) {
+                            float f[8];
+    #pragma unroll
+                            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[j + e]);
+                            if (fold) {
+                                const float4 s0 = *(const float4 *)(scale_s + n0 + c0 + j);
+                                const float4 s1 = *(const float4 *)(scale_s + n0 + c0 + j + 4);
+                                f[0] *= s0.x; f[1] *= s0.y; f[2] *= s0.z; f[3] *= s0.w;
+                                f[4] *= s1.x; f[5] *= s1.y; f[6] *= s1.z; f[7] *= s1.w;
+                            }
+                            if (bias || fold) {
+                                const float4 b0 = *(const float4 *)(bias_s + n0 + c0 + j);
+                                const float4 b1 = *(const float4 *)(bias_s + n0 + c0 + j + 4);
+                                f[0] += b0.x; f[1] += b0.y; f[2] += b0.z; f[3] += b0.w;
+                                f[4] += b1.x; f[5] += b1.y; f[6] += b1.z; f[7] += b1.w;
+                            }
+                            uint4 pk;
+                            pk.x = pack2_t<H>(f[0], f[1]);
+                            pk.y = pack2_t<H>(f[2], f[3]);
+                            pk.z = pack2_t<H>(f[4], f[5]);
+                            pk.w = pack2_t<H>(f[6], f[7]);
+                            *(uint4 *)(row + ((((j >> 3) ^ (lane & 7)) & 7) << 4)) = pk;
                         }
-                        if (bias || fold) {
-                            const float4 b0 = *(const float4 *)(bias_s + n0 + c0 + j);
-                            const float4 b1 = *(const float4 *)(bias_s + n0 + c0 + j + 4);
-                            f[0] += b0.x; f[1] += b0.y; f[2] += b0.z; f[3] += b0.w;
-                            f[4] += b1.x; f[5] += b1.y; f[6] += b1.z; f[7] += b1.w;
-                        }
-                        uint4 pk;
-                        __nv_bfloat162 h;
-                        h = __floats2bfloat162_rn(f[0], f[1]); pk.x = *(uint32_t *)&h;
-                        h = __floats2bfloat162_rn(f[2], f[3]); pk.y = *(uint32_t *)&h;
-                        h = __floats2bfloat162_rn(f[4], f[5]); pk.z = *(uint32_t *)&h;
-                        h = __floats2bfloat162_rn(f[6], f[7]); pk.w = *(uint32_t *)&h;
-                        *(uint4 *)(row + ((((j >> 3) ^ (lane & 7)) & 7) << 4)) = pk;
-                    }
+                    };
+                    if (g.f16) pack_rows(std::true_type{}); else pack_rows(std::false_type{});
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
@@ -540,6 +543,7 @@ cudaError_t launch_umma_conv(const UmmaConvShape &s, const void *act, const void
     g.lower_h = s.lower_h; g.lower_w = s.lower_w; g.stride_h = s.stride_h; g.stride_w = s.stride_w;
     g.dil_h = s.dil_h; g.dil_w = s.dil_w; g.p = (long long)s.n * s.ho * s.wo; g.stages = 1;
     g.blockdiag = s.blockdiag;
+    g.f16 = call_f16();
     g.stem = 0; g.stem_tw = g.stem_th = g.stem_tiles_w = g.stem_tiles_h = 1;
     g.fold = fold ? *fold : BnFold{nullptr, nullptr, nullptr, nullptr, nullptr, 0.f, nullptr};
     g.out_strided = s.out_sw ? (__nv_bfloat16 *)out : nullptr;
@@ -577,6 +581,7 @@ cudaError_t launch_stem_fwd(const Problem &pb, const void *x_packed, const void 
     g.stem_tiles_w = (pb.w_out + 15) / 16; g.stem_tiles_h = (pb.h_out + 7) / 8;
     g.p = (long long)pb.n * g.stem_tiles_h * g.stem_tiles_w * kBM;      // m-tiles x 128 (patches, ragged edges clipped)
     g.stages = 1; g.blockdiag = 0; g.out_strided = nullptr; g.out_sn = 0; g.out_sh = g.out_sw = 0;
+    g.f16 = 0;                      // the packed-stem path is bf16 only
     g.fold = fold ? *fold : BnFold{nullptr, nullptr, nullptr, nullptr, nullptr, 0.f, nullptr};
     CUtensorMap ta, tw, tout;
     {   // overlapping windows: 64 elements (8 pixels x 8 channels) starting at every output column

@@ -50,6 +50,7 @@ struct StripGemm {
     int bstages;                      // weight-tile ring slots in use (streaming mode)
     int nissue;                       // issuing warps in use: min(nmb, kSIssuers)
     int resident;                     // 1: all weight tiles stay in shared memory (one n-tile only)
+    int f16;                          // 16-bit storage type: 0 bf16, 1 IEEE half
     int sub_cin, sub_hin, sub_win;    // sub-pixel output mode, see UmmaConvShape
     int sub_wide;                     // 1: wide sub-pixel mode (BN = 64 / 128), n-tile -> parity class
     uint32_t sub_mask[4];             // taps with weights, per class
@@ -233,7 +234,7 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
         // and only their start-address field moves.
         const int me = warp - 2, ni = g.nissue;         // this warp issues M blocks me, me + ni, ...
         if (me < ni && elect_one()) {
-            constexpr uint32_t idesc = idesc_bf16_f32(128, BN, 0, 0);
+            const uint32_t idesc = idesc_h16_f32(128, BN, 0, 0, g.f16);
             const uint32_t hi = smem_desc_hi_sw128(1024);
             const uint32_t bres_lo = smem_desc_lo(smem_u32(bring), 16);
             int sb = 0, s = 0;
@@ -379,29 +380,32 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
                     tmem_ld_32x32(t_row + (uint32_t)c0, vv);
                     tmem_ld_wait();
                     uint4 pk[4];
-#pragma unroll
-                    for (int j = 0; j < 32; j += 8) {
-                        float f[8];
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(vv[j + e]);
-                        if (fold) {
-                            const float4 s0 = *(const float4 *)(scale_s + n0 + c0 + j);
-                            const float4 s1 = *(const float4 *)(scale_s + n0 + c0 + j + 4);
-                            f[0] *= s0.x; f[1] *= s0.y; f[2] *= s0.z; f[3] *= s0.w;
-                            f[4] *= s1.x; f[5] *= s1.y; f[6] *= s1.z; f[7] *= s1.w;
+                    auto pack_chunk = [&](auto half_tag) {
+                        constexpr bool H = decltype(half_tag)::value;
+    #pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            float f[8];
+    #pragma unroll
+                            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(vv[j + e]);
+                            if (fold) {
+                                const float4 s0 = *(const float4 *)(scale_s + n0 + c0 + j);
+                                const float4 s1 = *(const float4 *)(scale_s + n0 + c0 + j + 4);
+                                f[0] *= s0.x; f[1] *= s0.y; f[2] *= s0.z; f[3] *= s0.w;
+                                f[4] *= s1.x; f[5] *= s1.y; f[6] *= s1.z; f[7] *= s1.w;
+                            }
+                            if (bias || fold) {
+                                const float4 b0 = *(const float4 *)(bias_s + n0 + c0 + j);
+                                const float4 b1 = *(const float4 *)(bias_s + n0 + c0 + j + 4);
+                                f[0] += b0.x; f[1] += b0.y; f[2] += b0.z; f[3] += b0.w;
+                                f[4] += b1.x; f[5] += b1.y; f[6] += b1.z; f[7] += b1.w;
+                            }
+                            pk[j >> 3].x = pack2_t<H>(f[0], f[1]);
+                            pk[j >> 3].y = pack2_t<H>(f[2], f[3]);
+                            pk[j >> 3].z = pack2_t<H>(f[4], f[5]);
+                            pk[j >> 3].w = pack2_t<H>(f[6], f[7]);
                         }
-                        if (bias || fold) {
-                            const float4 b0 = *(const float4 *)(bias_s + n0 + c0 + j);
-                            const float4 b1 = *(const float4 *)(bias_s + n0 + c0 + j + 4);
-                            f[0] += b0.x; f[1] += b0.y; f[2] += b0.z; f[3] += b0.w;
-                            f[4] += b1.x; f[5] += b1.y; f[6] += b1.z; f[7] += b1.w;
-                        }
-                        __nv_bfloat162 hh;
-                        hh = __floats2bfloat162_rn(f[0], f[1]); pk[j >> 3].x = *(uint32_t *)&hh;
-                        hh = __floats2bfloat162_rn(f[2], f[3]); pk[j >> 3].y = *(uint32_t *)&hh;
-                        hh = __floats2bfloat162_rn(f[4], f[5]); pk[j >> 3].z = *(uint32_t *)&hh;
-                        hh = __floats2bfloat162_rn(f[6], f[7]); pk[j >> 3].w = *(uint32_t *)&hh;
-                    }
+                    };
+                    if (g.f16) pack_chunk(std::true_type{}); else pack_chunk(std::false_type{});
                     // butterfly transpose: afterwards pk[k] of lane (quad0 + c) is chunk c of row (quad0 + k)
                     quad_swap(pk[0], pk[1], 1, (lane & 1) != 0);
                     quad_swap(pk[2], pk[3], 1, (lane & 1) != 0);
@@ -584,6 +588,7 @@ cudaError_t launch_umma_strip_conv(const UmmaConvShape &s, const void *act, cons
     g.tiles_h = (s.ho + pl.R - 1) / pl.R; g.tiles_w = (s.wo + pl.CW - 1) / pl.CW;
     g.strip_bytes = pl.strip_bytes;
     g.nacc = pl.nacc;
+    g.f16 = call_f16();
     g.nstrips = pl.nstrips; g.resident = pl.resident; g.bstages = pl.bstages;
     g.nissue = pl.nmb < kSIssuers ? pl.nmb : kSIssuers;
     g.blockdiag = s.blockdiag;
@@ -649,7 +654,7 @@ __global__ void subpixel_weights_kernel(const __nv_bfloat16 *__restrict__ w, con
 namespace {
 __global__ void subpixel_wide_weights_kernel(const __nv_bfloat16 *__restrict__ w, const float *__restrict__ s_vec,
                                              __nv_bfloat16 *__restrict__ wsub, int c_out, int cin, int kh, int kw,
-                                             int pad_h, int pad_w, int th, int tw, int dmin_h, int dmin_w) {
+                                             int pad_h, int pad_w, int th, int tw, int dmin_h, int dmin_w, int f16) {
     pdl_wait();
     pdl_launch_dependents();
     const long long total = 4LL * cin * th * tw * c_out;
@@ -663,8 +668,8 @@ __global__ void subpixel_wide_weights_kernel(const __nv_bfloat16 *__restrict__ w
         const int r = a + pad_h - 2 * (dmin_h + tr), q = b + pad_w - 2 * (dmin_w + tq);
         float v = 0.f;
         if (r >= 0 && r < kh && q >= 0 && q < kw)
-            v = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[(((size_t)co * kh + r) * kw + q) * cin + ci]);
-        wsub[idx] = __float2bfloat16_rn(v);
+            v = (s_vec ? s_vec[co] : 1.f) * load_h16(w + (((size_t)co * kh + r) * kw + q) * cin + ci, f16);
+        reinterpret_cast<uint16_t *>(wsub)[idx] = pack1_h16(v, f16);
     }
 }
 }  // namespace
@@ -723,7 +728,7 @@ cudaError_t launch_subpixel_weights(const Problem &pb, const void *w, const floa
         const long long blocks = (total + 255) / 256;
         return launch_pdl(subpixel_wide_weights_kernel, dim3((unsigned)(blocks < 2368 ? blocks : 2368)), dim3(256), 0, st,
                           (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)wsub, pb.c_out, pb.c_in, pb.kh, pb.kw,
-                          pb.pad_h, pb.pad_w, s.taps_h, s.taps_w, s.lower_h, s.lower_w);
+                          pb.pad_h, pb.pad_w, s.taps_h, s.taps_w, s.lower_h, s.lower_w, call_f16());
     }
     const int total = 16 * s.taps_h * s.taps_w * pb.c_out;
     return launch_pdl(subpixel_weights_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st,

@@ -34,6 +34,7 @@ struct WgradGemm {
     // filter row), tm_dz a 4-D map of dZ; a "pixel block" is a 4 x 16 patch of output pixels.
     int stem, stem_tiles_w, stem_tiles_h;
     int no_ones;            // 1: no slice of ones (the packed stem input carries a constant-1 slot instead)
+    int f16;                // 16-bit storage type: 0 bf16, 1 IEEE half
 };
 
 struct WgradSmemCtl {
@@ -88,8 +89,9 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
     if (counters && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
         for (int i = threadIdx.x; i < ncounters; i += kWThreads) counters[i] = 0u;
     if (ones_slot >= 0) {
-        // bf16 1.0 everywhere (invariant under the swizzle); TMA never writes this slice
-        const uint4 ones = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
+        // 1.0 everywhere (invariant under the swizzle); TMA never writes this slice
+        const uint32_t one2 = one_h16(g.f16) * 0x10001u;
+        const uint4 ones = make_uint4(one2, one2, one2, one2);
         for (int s = 0; s < stages; ++s) {
             uint4 *dst = (uint4 *)(tiles + (size_t)s * kStageBytes + (size_t)ones_slot * kChunkBytes);
             for (int i = threadIdx.x; i < (int)(kChunkBytes / 16); i += kWThreads) dst[i] = ones;
@@ -158,7 +160,7 @@ __global__ void __launch_bounds__(kWThreads) umma_wgrad_kernel(const __grid_cons
         }
     } else if (warp == 1) {
         if (elect_one()) {
-            constexpr uint32_t idesc = idesc_bf16_f32(kWM, BN, 1, 1);   // both operands MN-major
+            const uint32_t idesc = idesc_h16_f32(kWM, BN, 1, 1, g.f16);   // both operands MN-major
             const uint32_t hi = smem_desc_hi_sw128(1024);
             const uint32_t tiles_lo = smem_desc_lo(smem_u32(tiles), kChunkBytes);
             bool ok = true;
@@ -308,7 +310,7 @@ cudaError_t launch_umma_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
     g.lower_h = -pb.pad_h; g.lower_w = -pb.pad_w; g.stride_h = pb.stride_h; g.stride_w = pb.stride_w;
     g.dil_h = pb.dil_h; g.dil_w = pb.dil_w; g.kdim = pb.kdim; g.p = pb.p; g.per_split = pl.per_split; g.stages = 1;
     g.blockdiag = pb.groups > 1 ? 1 : 0;
-    g.stem = 0; g.stem_tiles_w = g.stem_tiles_h = 1; g.no_ones = 0;
+    g.stem = 0; g.stem_tiles_w = g.stem_tiles_h = 1; g.no_ones = 0; g.f16 = call_f16();
     if (g.blockdiag) { g.c_in = 64; g.kdim = pb.kh * pb.kw * 64; }
     const int upper_h = g.lower_h + (pb.h_out - 1) * pb.stride_h - (pb.h_in - 1);
     const int upper_w = g.lower_w + (pb.w_out - 1) * pb.stride_w - (pb.w_in - 1);
@@ -345,7 +347,7 @@ __global__ void __launch_bounds__(32 * KR * SL, SL == 16 ? 2 : (KR * SL == 8 ? 4
     const __nv_bfloat16 *__restrict__ w, const float *__restrict__ vec3, const float *__restrict__ b,
     const float *__restrict__ mean, float *__restrict__ dw, float *__restrict__ dotpart,
     unsigned int *__restrict__ counters, float *__restrict__ db, float *__restrict__ dgamma,
-    float *__restrict__ dbeta, int need_sums) {
+    float *__restrict__ dbeta, int need_sums, int f16) {
     static_assert(KR * SL <= 32, "at most 32 warps per block");
     // loads in flight per thread: the (2, 16) shape has the most blocks and is held to 32 registers, so
     // that two of its 1024-thread blocks share an SM
@@ -362,7 +364,7 @@ __global__ void __launch_bounds__(32 * KR * SL, SL == 16 ? 2 : (KR * SL == 8 ? 4
 #pragma unroll
     for (int rep = 0; rep < REP; ++rep) {
         const int k = k0 + rep * KR + (int)(threadIdx.x % KR), co = co0 + (int)(threadIdx.x / KR);
-        wv[rep] = (vec3 && threadIdx.x < 32 * KR && k < kdim) ? __bfloat162float(w[(size_t)co * kdim + k]) : 0.f;
+        wv[rep] = (vec3 && threadIdx.x < 32 * KR && k < kdim) ? load_h16(w + (size_t)co * kdim + k, f16) : 0.f;
     }
     constexpr int NBF = REP > 1 ? 32 / REP : 1;      // slices the preloading path below can take
     if (SL == 1 && REP > 1 && splits <= NBF) {
@@ -500,14 +502,14 @@ cudaError_t launch_wgrad_epilogue_fused(const Problem &pb, const UmmaWgradPlan &
     if (pl.kr == 32)                                  // 4 groups of 8 rows, 256 threads: several blocks per SM
         return launch_pdl(wgrad_epilogue_fused_kernel<8, 1, 4>, grid, dim3(256), 0, st, pb.c_out, pb.kdim, partials,
                           pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw, dotpart, counters, db,
-                          dgamma, dbeta, ns);
+                          dgamma, dbeta, ns, call_f16());
     if (pl.kr == 8)
         return launch_pdl(wgrad_epilogue_fused_kernel<8, 4, 1>, grid, dim3(1024), 0, st, pb.c_out, pb.kdim, partials,
                           pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw, dotpart, counters, db,
-                          dgamma, dbeta, ns);
+                          dgamma, dbeta, ns, call_f16());
     return launch_pdl(wgrad_epilogue_fused_kernel<2, 16, 1>, grid, dim3(1024), 0, st, pb.c_out, pb.kdim, partials,
                       pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw, dotpart, counters, db,
-                      dgamma, dbeta, ns);
+                      dgamma, dbeta, ns, call_f16());
 }
 
 // ---- small-C_in ("stem") layers -------------------------------------------------------------------
@@ -536,6 +538,7 @@ cudaError_t launch_stem_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
     g.kdim = krows * 64;
     g.stem = 1; g.stem_tiles_w = (pb.w_out + 15) / 16; g.stem_tiles_h = (pb.h_out + 3) / 4;
     g.no_ones = stem_ones_in_pack(pb) ? 1 : 0;
+    g.f16 = 0;                      // the packed-stem path is bf16 only
     g.p = (long long)pb.n * g.stem_tiles_h * g.stem_tiles_w * kWP;
     g.per_split = pl.per_split; g.stages = 1; g.blockdiag = 0;
     CUtensorMap tx, tdz;

@@ -13,7 +13,7 @@ from . import inputs as I
 
 
 def make_desc(spec: I.LayerSpec) -> C.Desc:
-    return C.Desc.make(dtype=C.BF16 if spec.dtype == "bf16" else C.F32,
+    return C.Desc.make(dtype={"bf16": C.BF16, "f16": C.F16}.get(spec.dtype, C.F32),
                        layout=C.NHWC if spec.layout == "nhwc" else C.NCHW, eps=spec.eps,
                        **spec.dims())
 
@@ -28,7 +28,7 @@ class Block:
         self.desc = make_desc(spec)
         self.device = torch.device(device)
         self.h_out, self.w_out = C.convbn_out_shape(self.desc)
-        self.tdtype = torch.bfloat16 if spec.dtype == "bf16" else torch.float32
+        self.tdtype = {"bf16": torch.bfloat16, "f16": torch.float16}.get(spec.dtype, torch.float32)
         cg = spec.c_in // spec.groups
         self.x_shape = (spec.n, spec.c_in, spec.h_in, spec.w_in)
         self.w_shape = (spec.c_out, cg, spec.kh, spec.kw)
@@ -176,7 +176,7 @@ class Block:
 
     def saved_bytes(self, mode: str) -> int:
         """Bytes kept from forward to backward beside nothing else: X plus the mode's extra."""
-        es = 2 if self.spec.dtype == "bf16" else 4
+        es = 2 if self.spec.dtype in ("bf16", "f16") else 4
         xb = int(np.prod(self.x_shape)) * es
         m = {"tune": C.MODE_TUNE, "eval": C.MODE_EVAL, "deploy": C.MODE_DEPLOY}[mode]
         return xb + C.convbn_saved_bytes(self.desc, m)

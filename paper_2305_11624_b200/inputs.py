@@ -86,7 +86,7 @@ def round_bf16(a: np.ndarray) -> np.ndarray:
 
 @dataclass(frozen=True)
 class LayerSpec:
-    """One ConvBN layer: sizes, storage type (``"f32"``/``"bf16"``), memory layout
+    """One ConvBN layer: sizes, storage type (``"f32"``/``"bf16"``/``"f16"``), memory layout
     (``"nchw"``/``"nhwc"``) and whether the convolution has a bias."""
     name: str
     n: int
@@ -174,6 +174,9 @@ def make_block(spec: LayerSpec, seed: int, out_hw: Tuple[int, int]) -> Dict[str,
     t["var_hat"] = uniform(seed, _TAGS["var_hat"], spec.c_out, 0.5, 2.0)
     t["gamma"] = uniform(seed, _TAGS["gamma"], spec.c_out, 0.5, 1.5)
     t["beta"] = normal(seed, _TAGS["beta"], spec.c_out) * np.float32(0.1)
+    if spec.dtype == "f16":
+        for k in ("x", "w", "dz"):
+            t[k] = t[k].astype(np.float16).astype(np.float32)          # numpy rounds to nearest even
     if spec.dtype == "bf16":
         for k in ("x", "w", "dz"):
             t[k] = round_bf16(t[k])

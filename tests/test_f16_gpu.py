@@ -1,0 +1,92 @@
+"""IEEE-half storage (the paper's mixed-precision rows, Table 4): Tune-mode forward and backward of dense layers on
+the tensor-core paths against the fp64 oracle, inputs rounded to half on the host; unsupported calls are refused."""
+import numpy as np
+import pytest
+import torch
+
+import parity
+from paper_2305_11624_b200 import convbn as C
+from paper_2305_11624_b200 import inputs as I
+from paper_2305_11624_b200.harness import Block, make_desc
+
+pytestmark = pytest.mark.gpu
+L = I.LayerSpec
+
+SHAPES = [
+    L("h_1x1_256_64", 2, 256, 28, 28, 64, 1, 1, dtype="f16"),                       # fused single-read backward
+    L("h_1x1_64_256", 2, 64, 28, 28, 256, 1, 1, dtype="f16", bias=True),
+    L("h_1x1_512_128", 3, 512, 14, 14, 128, 1, 1, dtype="f16"),                      # two-call backward
+    L("h_3x3_64", 2, 64, 30, 30, 64, 3, 3, pad=1, dtype="f16"),                      # strip kernel
+    L("h_3x3_128_256", 2, 128, 20, 36, 256, 3, 3, pad=1, dtype="f16", bias=True),
+    L("h_3x3_s2_128", 2, 128, 40, 42, 128, 3, 3, stride=2, pad=1, dtype="f16"),      # sub-pixel backward data
+    L("h_3x3_256_7x7", 4, 256, 7, 7, 256, 3, 3, pad=1, dtype="f16"),                 # small images: im2col GEMM
+    L("h_1x1_s2_256_512", 2, 256, 14, 14, 512, 1, 1, stride=2, dtype="f16"),         # residue-class backward data
+    L("h_5x5_64_d2", 1, 64, 24, 24, 64, 5, 5, pad=4, dil=2, dtype="f16"),
+]
+
+
+@pytest.mark.parametrize("spec", SHAPES, ids=lambda s: s.name)
+def test_half_tune_against_the_oracle(spec):
+    t = parity.make_inputs(spec, 4321)
+    assert np.array_equal(t["x"], t["x"].astype(np.float16).astype(np.float32))      # the oracle reads what the GPU reads
+    ref = parity.oracle_tune(spec, t)
+    got = parity.run_tune_gpu(spec, t)
+    errs = parity.compare(got, ref, parity.TOL["f16"], parity.TUNE_OUTPUTS, spec.name, dtype="f16")
+    print(spec.name, got["_kernels"], {k: "%.1e" % v for k, v in errs.items()})
+    assert all(k.startswith("umma") for k in got["_kernels"]), got["_kernels"]
+    # the one-call backward gives the same numbers
+    blk = Block(spec, modes=("tune",))
+    blk.load(t)
+    blk.tune_fwd(); blk.tune_bwd()
+    C.convbn_check()
+    two = {k: blk.fetch(k) for k in ("dx", "dw", "dgamma", "dbeta")}
+    parity.compare(two, ref, parity.TOL["f16"], ("dx", "dw", "dgamma", "dbeta"), spec.name + " one call", dtype="f16")
+
+
+def test_half_is_not_bf16():
+    """The same bits read as the other 16-bit type give another tensor: a kernel that ignored the flag would fail."""
+    spec = L("h_flag", 1, 64, 16, 16, 64, 3, 3, pad=1, dtype="f16")
+    t = parity.make_inputs(spec, 7)
+    got = parity.run_tune_gpu(spec, t)
+    wrong = L("b_flag", 1, 64, 16, 16, 64, 3, 3, pad=1, dtype="bf16")
+    blk = Block(wrong, modes=("tune",))
+    hb = Block(spec, modes=("tune",)); hb.load(t)
+    for name in ("x", "w", "dz"):
+        getattr(blk, name).view(torch.int16).copy_(getattr(hb, name).view(torch.int16))      # half bits in bf16 buffers
+    for name in ("gamma", "beta", "mu_hat", "var_hat"):
+        getattr(blk, name).copy_(getattr(hb, name))
+    blk.tune_fwd()
+    C.convbn_check()
+    z_bits_as_bf16 = blk.z.view(torch.int16).cpu().numpy()
+    hb.tune_fwd()
+    assert not np.array_equal(z_bits_as_bf16, hb.z.view(torch.int16).cpu().numpy())
+    assert np.isfinite(got["z"]).all()
+
+
+@pytest.mark.parametrize("spec,call", [
+    (L("h_dw", 1, 64, 16, 16, 64, 3, 3, pad=1, groups=64, dtype="f16"), "tune"),
+    (L("h_stem", 1, 3, 32, 32, 64, 7, 7, stride=2, pad=3, dtype="f16"), "tune"),
+    (L("h_odd", 1, 48, 16, 16, 64, 3, 3, pad=1, dtype="f16"), "tune"),
+    (L("h_eval", 1, 64, 16, 16, 64, 3, 3, pad=1, dtype="f16"), "eval"),
+], ids=lambda v: v.name if isinstance(v, L) else v)
+def test_unsupported_half_calls_are_refused(spec, call):
+    d = make_desc(spec)
+    if call == "tune":
+        assert C.convbn_workspace_bytes(d, C.PHASE_TUNE_FWD) == 0
+        with pytest.raises(C.ConvBNError) as e:
+            C.convbn_tune_fwd(d, 4096, 4096, None, 4096, 4096, 4096, 4096, 4096, 4096, 4096, 1 << 20, stream=0)
+    else:
+        with pytest.raises(C.ConvBNError) as e:
+            C.convbn_eval_fwd(d, 4096, 4096, None, 4096, 4096, 4096, 4096, 4096, 4096, 4096, 1 << 20, stream=0)
+    assert e.value.status == C.EUNSUPPORTED
+
+
+def test_half_glue_and_linear():
+    a = torch.randn(4099, device="cuda:0").half(); b = torch.randn(4099, device="cuda:0").half()
+    out = torch.empty_like(a)
+    C.convbn_add_relu(a, b, out)
+    C.convbn_check()
+    ref = torch.relu(a.float() + b.float()).half()
+    assert torch.equal(out, ref)
+    d = C.convbn_linear_desc(1000, 128, 64, C.F16)
+    assert (d.layout, d.dtype, d.c_in, d.c_out) == (C.NHWC, C.F16, 128, 64)
