@@ -278,6 +278,8 @@ UmmaWgradPlan umma_wgrad_plan(const Problem &pb) {
 void wgrad_epilogue_shape(const Problem &pb, UmmaWgradPlan *pl) {
     const long long blocks8 = (long long)(pb.c_out / 32) * ((pb.kdim + 7) / 8);
     pl->kr = pl->splits > 192 ? 2 : ((pl->splits <= 8 || blocks8 > 600) && blocks8 / 4 >= device_sm_count() ? 32 : 8);
+    // very large weight matrices in few slices: 8 groups of 8 rows per block halve the blocks (and their fences) again
+    if (pl->kr == 32 && pl->splits <= 4 && blocks8 / 8 >= 2 * device_sm_count()) pl->kr = 64;
     pl->kt = (pb.kdim + pl->kr - 1) / pl->kr;   // epilogue blocks along k = rows of dotpart
 }
 
@@ -499,6 +501,10 @@ cudaError_t launch_wgrad_epilogue_fused(const Problem &pb, const UmmaWgradPlan &
     static PerDevice carve_a, carve_b;
     prefer_max_shared_once(wgrad_epilogue_fused_kernel<8, 4, 1>, &carve_a);
     prefer_max_shared_once(wgrad_epilogue_fused_kernel<2, 16, 1>, &carve_b);
+    if (pl.kr == 64)
+        return launch_pdl(wgrad_epilogue_fused_kernel<8, 1, 8>, grid, dim3(256), 0, st, pb.c_out, pb.kdim, partials,
+                          pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw, dotpart, counters, db,
+                          dgamma, dbeta, ns, call_f16());
     if (pl.kr == 32)                                  // 4 groups of 8 rows, 256 threads: several blocks per SM
         return launch_pdl(wgrad_epilogue_fused_kernel<8, 1, 4>, grid, dim3(256), 0, st, pb.c_out, pb.kdim, partials,
                           pl.splits, bsum, pl.splits, (const __nv_bfloat16 *)w, vec3, b, mean, dw, dotpart, counters, db,
