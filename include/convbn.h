@@ -149,7 +149,10 @@ int convbn_tune_bwd_weight(const convbn_desc *desc, const void *dz, const void *
  * For the 1x1, stride-1 layers of a bottleneck (bf16 NHWC, one of C_in / C_out equal to 64 and the other
  * 128 or 256, at least 512 pixels) one kernel reads every dZ tile from memory ONCE and feeds both the
  * data-gradient and the weight-gradient GEMM from it (omega' = s omega is formed in shared memory and never
- * written); every other layer runs the two calls above one after the other.  dx may not alias dz or x.
+ * written); every other layer runs the two passes above SIDE BY SIDE: the parameter-gradient pass on a stream the library
+ * owns (one per device and host thread, created on first use), forked from `stream` at the start of the call and joined
+ * into it before the call returns, so the caller sees plain stream order (and a stream capture stays well-formed); each
+ * pass has its own region of the workspace.  dx may not alias dz or x.
  * Workspace: convbn_workspace_bytes(desc, CONVBN_PHASE_TUNE_BWD). */
 int convbn_tune_bwd(const convbn_desc *desc, const void *dz, const void *x, const void *w, const float *b,
                     const float *run_mean, const void *saved, void *dx, float *dw, float *db, float *dgamma,

@@ -133,9 +133,10 @@ bool fused_bwd_path(const convbn_desc *d, const Problem &pb) {
 Plan make_plan(const convbn_desc *d, const Problem &pb, int phase) {
     Plan pl;
     if (phase == CONVBN_PHASE_TUNE_BWD) {
-        if (!fused_bwd_path(d, pb)) {       // the two calls one after the other, in the same workspace
+        if (!fused_bwd_path(d, pb)) {       // the two passes run side by side: each has its own region
             const Plan a = make_plan(d, pb, CONVBN_PHASE_TUNE_BWD_DATA), b2 = make_plan(d, pb, CONVBN_PHASE_TUNE_BWD_WEIGHT);
-            pl.total = a.total > b2.total ? a.total : b2.total;
+            pl.w_scaled = align_up(a.total, 256);          // here: offset of the backward-weight region
+            pl.total = pl.w_scaled + b2.total;
             return pl;
         }
         size_t o = 0;
@@ -779,6 +780,32 @@ int convbn_tune_bwd_weight(const convbn_desc *desc, const void *dz, const void *
     return CONVBN_OK;
 }
 
+}  // extern "C"
+
+namespace {
+// Side lane of convbn_tune_bwd: one stream and two events per device and host thread, made on first use.  The
+// parameter-gradient pass (GEMM + epilogue) runs there while the input-gradient pass (weight re-layout + GEMM) runs
+// on the caller's stream; the caller's stream waits for the lane before the call returns, so stream order is what
+// the caller sees.  (Per thread: two threads sharing the events could wait on each other's fork points.)
+struct SideLane { cudaStream_t stream = nullptr; cudaEvent_t fork = nullptr, join = nullptr; };
+thread_local SideLane t_side_lane[kMaxDevices];
+
+int side_lane(SideLane **out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CONVBN_ECUDA;
+    SideLane &l = t_side_lane[dev];
+    if (!l.stream) {
+        if (cudaStreamCreateWithFlags(&l.stream, cudaStreamNonBlocking) != cudaSuccess) { l.stream = nullptr; return CONVBN_ECUDA; }
+        if (cudaEventCreateWithFlags(&l.fork, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&l.join, cudaEventDisableTiming) != cudaSuccess)
+            return CONVBN_ECUDA;
+    }
+    *out = &l;
+    return CONVBN_OK;
+}
+}  // namespace
+
+extern "C" {
 int convbn_tune_bwd(const convbn_desc *desc, const void *dz, const void *x, const void *w, const float *b,
                     const float *run_mean, const void *saved, void *dx, float *dw, float *db, float *dgamma,
                     float *dbeta, void *workspace, size_t workspace_bytes, void *stream) {
@@ -798,11 +825,25 @@ int convbn_tune_bwd(const convbn_desc *desc, const void *dz, const void *x, cons
     const Plan pl = make_plan(desc, pb, CONVBN_PHASE_TUNE_BWD);
     CK(check_ws(pl, workspace, workspace_bytes));
     if (!fused_bwd_path(desc, pb)) {
-        CK(convbn_tune_bwd_data(desc, dz, w, saved, dx, workspace, workspace_bytes, stream));
-        CK(convbn_tune_bwd_weight(desc, dz, x, w, b, run_mean, saved, dw, db, dgamma, dbeta, workspace, workspace_bytes,
-                                  stream));
+        void *ws_w = workspace ? at(workspace, pl.w_scaled) : nullptr;
+        const size_t bytes_d = pl.w_scaled, bytes_w = pl.total - pl.w_scaled;
         t_last_kernel[CONVBN_PHASE_TUNE_BWD] = "two-calls";
-        return CONVBN_OK;
+        if (g_prof.on) {                 // per-kernel timing wants one stream
+            CK(convbn_tune_bwd_data(desc, dz, w, saved, dx, workspace, bytes_d, stream));
+            return convbn_tune_bwd_weight(desc, dz, x, w, b, run_mean, saved, dw, db, dgamma, dbeta, ws_w, bytes_w, stream);
+        }
+        SideLane *lane = nullptr;
+        CK(side_lane(&lane));
+        cudaStream_t st = (cudaStream_t)stream;
+        CU(cudaEventRecord(lane->fork, st));
+        CU(cudaStreamWaitEvent(lane->stream, lane->fork, 0));
+        const int sw = convbn_tune_bwd_weight(desc, dz, x, w, b, run_mean, saved, dw, db, dgamma, dbeta, ws_w, bytes_w,
+                                              lane->stream);
+        // whatever happened on the lane, the caller's stream joins it again (a capture must not be left forked)
+        const bool joined = cudaEventRecord(lane->join, lane->stream) == cudaSuccess;
+        const int sd = convbn_tune_bwd_data(desc, dz, w, saved, dx, workspace, bytes_d, stream);
+        if (!joined || cudaStreamWaitEvent(st, lane->join, 0) != cudaSuccess) return CONVBN_ECUDA;
+        return sw != CONVBN_OK ? sw : sd;
     }
     cudaStream_t st = (cudaStream_t)stream;
     float *partials = (float *)at(workspace, pl.partials), *bsum = (float *)at(workspace, pl.bsum);
