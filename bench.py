@@ -1,8 +1,9 @@
 #!/usr/bin/env python
 """Benchmark of the Tune-mode ConvBN hot path on B200.
 
-A step is one pass of the whole path - convbn_tune_fwd, then convbn_tune_bwd (input and parameter
-gradients in one call) - over every layer of a configuration.  With no ``--workload`` all five
+A step is one pass of the whole path - convbn_tune_fwd, then convbn_tune_bwd_begin (input gradient on the
+caller's stream, parameter gradients on the library's side stream) - over every layer of a configuration,
+closed by one convbn_tune_bwd_join (``--join-per-layer``: convbn_tune_bwd, which joins in every call).  With no ``--workload`` all five
 configurations run in one process and ONE JSON line is printed: ``value`` is the fwd+bwd TFLOP/s
 over the three dense bf16 configurations (1-3: total FLOPs / total time), ``per_config`` holds
 every configuration on its own (config 4 in GB/s against the copy bandwidth, config 0 as a
@@ -343,9 +344,15 @@ def bench_config(ctx, wl):
                     b.db = bk.views[b.spec.name + ".db"]
             buckets.append(bk)
 
+    # Parameter gradients off the critical path: every layer's backward call leaves its weight-gradient pass on the
+    # library's side stream and the step joins once at its end (--join-per-layer: every call joins before it returns).
+    defer = not args.join_per_layer
+
     def step(i):
         for b in blocks[i % sets]:
-            b.tune_step(stream)
+            b.tune_step(stream, defer_join=defer)
+        if defer:
+            C.convbn_tune_bwd_join(stream)
         if buckets:
             buckets[i % sets].all_reduce_async()
             buckets[i % sets].wait()
@@ -370,7 +377,9 @@ def bench_config(ctx, wl):
                 gr = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(gr):
                     for b in blocks[si]:
-                        b.tune_step()
+                        b.tune_step(defer_join=defer)
+                    if defer:
+                        C.convbn_tune_bwd_join()
                 graphs.append(gr)
             for gr in graphs:
                 gr.replay()
@@ -378,6 +387,9 @@ def bench_config(ctx, wl):
             launch_mode = "CUDA graph replay (one captured step per buffer set)"
         except Exception as exc:  # capture unsupported: say so and time eager calls
             graphs, launch_mode = None, "eager library calls (graph capture failed: %r)" % (exc,)
+
+    launch_mode += ("; parameter-gradient passes on the library's side stream, one join per step" if defer
+                    else "; every backward call joins its parameter-gradient pass")
 
     def timed(n_sets):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -735,6 +747,8 @@ def main():
     ap.add_argument("--no-modes", action="store_true", help="skip the Tune / Eval / Deploy comparison")
     ap.add_argument("--no-graph", action="store_true", help="time eager library calls instead of graph replays")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--join-per-layer", action="store_true",
+                    help="every backward call joins its parameter-gradient pass before returning (default: one join per step)")
     ap.add_argument("--no-backbone", action="store_true", help="skip the whole-ResNet-50 replay in the three modes")
     ap.add_argument("--dp-allreduce", action="store_true",
                     help="with N > 1 ranks: sum the parameter gradients over the ranks every step (default: replicas)")

@@ -238,6 +238,20 @@ int convbn_tune_step_host(const convbn_desc *desc, const void *x, const void *dz
                           float *db, float *dgamma, float *dbeta, void *device_arena,
                           size_t arena_bytes, void *stream);
 
+/* Backward with the parameter gradients off the critical path (what a training step wants: dX feeds the layer below at
+ * once, domega, db, dgamma, dbeta are needed by the optimiser only).  convbn_tune_bwd_begin takes the arguments of
+ * convbn_tune_bwd and computes the same values, but returns with the parameter-gradient pass (the weight-gradient GEMM
+ * and its epilogue, or for the single-kernel 1x1 path the epilogue alone) still running on the library's side stream:
+ * when work queued on `stream` after the call runs, dx is complete, while dw, db, dgamma, dbeta and the workspace belong
+ * to the library until convbn_tune_bwd_join(stream) has been called and the work it queues on `stream` has been reached.
+ * convbn_tune_bwd_join makes `stream` wait for every pass begun by the calling host thread on the current device; it is
+ * cheap, may be called with nothing pending, and must be called before a stream capture that contains begin calls ends.
+ * Errors as for convbn_tune_bwd. */
+int convbn_tune_bwd_begin(const convbn_desc *desc, const void *dz, const void *x, const void *w, const float *b,
+                          const float *run_mean, const void *saved, void *dx, float *dw, float *db, float *dgamma,
+                          float *dbeta, void *workspace, size_t workspace_bytes, void *stream);
+int convbn_tune_bwd_join(void *stream);
+
 /* ---- TransposedConv-BN in Tune mode (Sec. 3.2.2: the rewrite holds for any linear layer in front of a frozen BatchNorm;
  *      Sec. 3.3 definitions; Table 2, Tune row, with the transposed convolution in place of the convolution) ------------
  *

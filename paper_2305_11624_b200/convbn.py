@@ -26,6 +26,7 @@ EXPORTS = (
     "convbn_status_string", "convbn_last_kernel", "convbn_host_step_arena_bytes",
     "convbn_tune_step_host", "convbn_profile_begin", "convbn_profile_end",
     "convbn_tune_bwd_weight_noalloc", "convbn_selftest_wait_timeout", "convbn_tune_bwd", "convbn_linear_desc", "convbn_relu", "convbn_add_relu", "convbn_relu_bwd", "convbn_add",
+    "convbn_tune_bwd_begin", "convbn_tune_bwd_join",
     "convbn_tconv_out_shape", "convbn_tconv_workspace_bytes", "convbn_tconv_tune_fwd", "convbn_tconv_tune_bwd",
 )
 
@@ -162,6 +163,20 @@ def convbn_tune_bwd(desc, dz, x, w, b, run_mean, saved, dx, dw, db, dgamma, dbet
                                  _ptr(saved), _ptr(dx), _ptr(dw), _ptr(db), _ptr(dgamma), _ptr(dbeta),
                                  _ptr(workspace), ctypes.c_size_t(wb), _stream(stream)),
            "convbn_tune_bwd")
+
+
+def convbn_tune_bwd_begin(desc, dz, x, w, b, run_mean, saved, dx, dw, db, dgamma, dbeta, workspace=None,
+                          workspace_bytes: Optional[int] = None, stream=None):
+    """convbn_tune_bwd that returns with the parameter-gradient pass still running on the library's side lane."""
+    wb = _nbytes(workspace) if workspace_bytes is None else workspace_bytes
+    _raise(lib().convbn_tune_bwd_begin(ctypes.byref(desc), _ptr(dz), _ptr(x), _ptr(w), _ptr(b), _ptr(run_mean),
+                                       _ptr(saved), _ptr(dx), _ptr(dw), _ptr(db), _ptr(dgamma), _ptr(dbeta),
+                                       _ptr(workspace), ctypes.c_size_t(wb), _stream(stream)), "convbn_tune_bwd_begin")
+
+
+def convbn_tune_bwd_join(stream=None) -> None:
+    """Make `stream` wait for every parameter-gradient pass begun by this thread on the current device."""
+    _raise(lib().convbn_tune_bwd_join(_stream(stream)), "convbn_tune_bwd_join")
 
 
 def convbn_tconv_out_shape(desc):

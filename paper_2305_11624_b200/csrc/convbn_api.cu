@@ -806,9 +806,9 @@ int side_lane(SideLane **out) {
 }  // namespace
 
 extern "C" {
-int convbn_tune_bwd(const convbn_desc *desc, const void *dz, const void *x, const void *w, const float *b,
-                    const float *run_mean, const void *saved, void *dx, float *dw, float *db, float *dgamma,
-                    float *dbeta, void *workspace, size_t workspace_bytes, void *stream) {
+static int tune_bwd_impl(const convbn_desc *desc, const void *dz, const void *x, const void *w, const float *b,
+                         const float *run_mean, const void *saved, void *dx, float *dw, float *db, float *dgamma,
+                         float *dbeta, void *workspace, size_t workspace_bytes, void *stream, bool defer_join) {
     HalfCall half(desc);              // CONVBN_F16: checked here, then run as the 16-bit path with the half flag set
     if (half.status != CONVBN_OK) return half.status;
     desc = half.use;
@@ -828,7 +828,7 @@ int convbn_tune_bwd(const convbn_desc *desc, const void *dz, const void *x, cons
         void *ws_w = workspace ? at(workspace, pl.w_scaled) : nullptr;
         const size_t bytes_d = pl.w_scaled, bytes_w = pl.total - pl.w_scaled;
         t_last_kernel[CONVBN_PHASE_TUNE_BWD] = "two-calls";
-        if (g_prof.on) {                 // per-kernel timing wants one stream
+        if (g_prof.on && !defer_join) {  // per-kernel timing wants one stream
             CK(convbn_tune_bwd_data(desc, dz, w, saved, dx, workspace, bytes_d, stream));
             return convbn_tune_bwd_weight(desc, dz, x, w, b, run_mean, saved, dw, db, dgamma, dbeta, ws_w, bytes_w, stream);
         }
@@ -842,7 +842,8 @@ int convbn_tune_bwd(const convbn_desc *desc, const void *dz, const void *x, cons
         // whatever happened on the lane, the caller's stream joins it again (a capture must not be left forked)
         const bool joined = cudaEventRecord(lane->join, lane->stream) == cudaSuccess;
         const int sd = convbn_tune_bwd_data(desc, dz, w, saved, dx, workspace, bytes_d, stream);
-        if (!joined || cudaStreamWaitEvent(st, lane->join, 0) != cudaSuccess) return CONVBN_ECUDA;
+        if (!joined) return CONVBN_ECUDA;
+        if (!defer_join && cudaStreamWaitEvent(st, lane->join, 0) != cudaSuccess) return CONVBN_ECUDA;
         return sw != CONVBN_OK ? sw : sd;
     }
     cudaStream_t st = (cudaStream_t)stream;
@@ -851,9 +852,44 @@ int convbn_tune_bwd(const convbn_desc *desc, const void *dz, const void *x, cons
     unsigned int *counters = (unsigned int *)at(workspace, pl.counters);
     const float *vec3 = (const float *)saved;
     LAUNCH("umma_bwd", launch_fused_bwd1x1(pb, dz, x, w, vec3, dx, partials, bsum, counters, st));
+    t_last_kernel[CONVBN_PHASE_TUNE_BWD] = "umma-fused-bwd";
+    if (defer_join) {
+        // dX is complete on the caller's stream; the parameter gradients are finished on the side lane
+        SideLane *lane = nullptr;
+        CK(side_lane(&lane));
+        CU(cudaEventRecord(lane->fork, st));
+        CU(cudaStreamWaitEvent(lane->stream, lane->fork, 0));
+        cudaStream_t st = lane->stream;
+        LAUNCH("wgrad_epilogue_fused", launch_wgrad_epilogue_fused(pb, pl.uw, partials, bsum, w, vec3, b, run_mean, dw,
+                                                                   dotpart, counters, db, dgamma, dbeta, true, st));
+        CU(cudaEventRecord(lane->join, lane->stream));
+        return CONVBN_OK;
+    }
     LAUNCH("wgrad_epilogue_fused", launch_wgrad_epilogue_fused(pb, pl.uw, partials, bsum, w, vec3, b, run_mean, dw, dotpart,
                                                                counters, db, dgamma, dbeta, true, st));
-    t_last_kernel[CONVBN_PHASE_TUNE_BWD] = "umma-fused-bwd";
+    return CONVBN_OK;
+}
+
+int convbn_tune_bwd(const convbn_desc *desc, const void *dz, const void *x, const void *w, const float *b,
+                    const float *run_mean, const void *saved, void *dx, float *dw, float *db, float *dgamma,
+                    float *dbeta, void *workspace, size_t workspace_bytes, void *stream) {
+    return tune_bwd_impl(desc, dz, x, w, b, run_mean, saved, dx, dw, db, dgamma, dbeta, workspace, workspace_bytes, stream,
+                         false);
+}
+
+int convbn_tune_bwd_begin(const convbn_desc *desc, const void *dz, const void *x, const void *w, const float *b,
+                          const float *run_mean, const void *saved, void *dx, float *dw, float *db, float *dgamma,
+                          float *dbeta, void *workspace, size_t workspace_bytes, void *stream) {
+    return tune_bwd_impl(desc, dz, x, w, b, run_mean, saved, dx, dw, db, dgamma, dbeta, workspace, workspace_bytes, stream,
+                         true);
+}
+
+int convbn_tune_bwd_join(void *stream) {
+    SideLane *lane = nullptr;
+    CK(side_lane(&lane));
+    // the lane is one stream: its last join point covers every pass begun before it
+    CU(cudaEventRecord(lane->join, lane->stream));
+    CU(cudaStreamWaitEvent((cudaStream_t)stream, lane->join, 0));
     return CONVBN_OK;
 }
 

@@ -142,9 +142,18 @@ class Block:
         C.convbn_tune_bwd(self.desc, self.dz, self.x, self.w, self.b, self.mu_hat, self.saved, self.dx, self.dw,
                           self.db, self.dgamma, self.dbeta, self.workspace, stream=stream)
 
-    def tune_step(self, stream=None):
+    def tune_bwd_begin(self, stream=None):
+        """Backward with the parameter-gradient pass left running on the library's side lane; dw, db, dgamma, dbeta and
+        the workspace belong to it until C.convbn_tune_bwd_join(stream)."""
+        C.convbn_tune_bwd_begin(self.desc, self.dz, self.x, self.w, self.b, self.mu_hat, self.saved, self.dx, self.dw,
+                                self.db, self.dgamma, self.dbeta, self.workspace, stream=stream)
+
+    def tune_step(self, stream=None, defer_join=False):
         self.tune_fwd(stream)
-        self.tune_bwd(stream)
+        if defer_join:
+            self.tune_bwd_begin(stream)
+        else:
+            self.tune_bwd(stream)
 
     # ---- Eval mode -------------------------------------------------------------------------
     def eval_fwd(self, stream=None):

@@ -54,3 +54,52 @@ def test_tune_bwd_is_deterministic():
         outs.append({k: getattr(blk, k).clone() for k in ("dx", "dw", "dgamma", "dbeta")})
     for k in outs[0]:
         assert torch.equal(outs[0][k], outs[1][k]), k
+
+
+def test_begin_join_gives_the_bits_of_the_synchronous_call():
+    """convbn_tune_bwd_begin leaves the parameter-gradient passes of several layers on the side lane; after one
+    convbn_tune_bwd_join every output equals the synchronous call's bit for bit (the kernels and their order of
+    additions are the same), inside and outside a captured graph."""
+    import torch
+    specs = [s for s, _ in SPECS[:6]]
+    blks = []
+    for i, spec in enumerate(specs):
+        b = Block(spec)
+        b.load(parity.make_inputs(spec, 40 + i))
+        b.tune_fwd()
+        b.tune_bwd()
+        blks.append(b)
+    torch.cuda.synchronize()
+    names = ("dx", "dw", "dgamma", "dbeta")
+    want = [{k: getattr(b, k).clone() for k in names} for b in blks]
+
+    def poison():
+        for b in blks:
+            for k in names:
+                getattr(b, k).fill_(float("nan"))
+
+    poison()
+    for b in blks:
+        b.tune_bwd_begin()
+    C.convbn_tune_bwd_join()
+    torch.cuda.synchronize()
+    C.convbn_check()
+    for b, w in zip(blks, want):
+        for k in names:
+            assert torch.equal(getattr(b, k), w[k]), (b.spec.name, k)
+    C.convbn_tune_bwd_join()                               # nothing pending: a no-op
+
+    poison()
+    torch.cuda.synchronize()
+    gr = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(gr):
+        for b in blks:
+            b.tune_bwd_begin()
+        C.convbn_tune_bwd_join()
+    poison()
+    gr.replay()
+    torch.cuda.synchronize()
+    C.convbn_check()
+    for b, w in zip(blks, want):
+        for k in names:
+            assert torch.equal(getattr(b, k), w[k]), (b.spec.name, k, "graph")
