@@ -637,8 +637,9 @@ def run_backbone(ctx, batch=32, size=224, iters=10):
     stem, plan = resnet50_plan(size)
     out = {"network": "ResNet-50 ConvBN blocks + ReLU + skip connections (max-pool replaced by synthetic tensors)",
            "batch": batch, "image": size, "dtype": "bf16", "iters": iters, "modes": {}}
-    for mode in ("tune", "eval", "deploy"):
-        rp = BackboneReplay(batch, plan, mode, stem_hw=stem, device=ctx.dev)
+    for mode in ("tune", "eval", "deploy", "tune_async"):
+        # tune_async: Tune mode with the parameter-gradient passes joined once per bottleneck instead of per call
+        rp = BackboneReplay(batch, plan, mode.split("_")[0], stem_hw=stem, device=ctx.dev, async_param_grads=mode == "tune_async")
         ms, peak, how = rp.measure(iters=iters, warmup=3)
         out["modes"][mode] = {"ms_per_iter": ms, "peak_bytes": peak, "tflops": rp.flops / ms / 1e9, "timing": how}
         out["flops_per_iter"] = rp.flops

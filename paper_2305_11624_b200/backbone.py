@@ -82,12 +82,20 @@ class _Layer:
         z, b.z = b.z, None
         return z
 
-    def backward(self, dz):
-        """Gradient with respect to the block's input; drops what the block kept for it."""
+    def backward(self, dz, held=None):
+        """Gradient with respect to the block's input; drops what the block kept for it.  With `held` (a list, Tune
+        mode) the parameter-gradient pass stays on the library's side stream: what it still reads (dZ, X, the saved
+        vectors, the scratch) is parked in `held` until the caller has joined."""
         b = self.blk
         b.dz = dz
         b.dx = torch.empty(self.in_elems, dtype=b.tdtype, device=b.device)
-        if self.mode == "tune":
+        if self.mode == "tune" and held is not None:
+            b.workspace = torch.empty(max(256, C.convbn_workspace_bytes(b.desc, C.PHASE_TUNE_BWD)), dtype=torch.uint8,
+                                      device=b.device)
+            b.tune_bwd_begin()
+            held.append((b.workspace, b.saved, b.x, b.dz))
+            b.workspace = b.saved = None
+        elif self.mode == "tune":
             b.with_scratch(C.PHASE_TUNE_BWD, b.tune_bwd)
             b.saved = None
         elif self.mode == "eval":
@@ -101,8 +109,9 @@ class _Layer:
 
 class BackboneReplay:
     def __init__(self, batch: int, plan: List[Bottleneck], mode: str, stem_hw: Optional[Tuple[int, int]] = None,
-                 device="cuda:0", seed: int = 0):
+                 device="cuda:0", seed: int = 0, async_param_grads: bool = False):
         assert mode in ("tune", "eval", "deploy")
+        self.async_param_grads = async_param_grads
         self.mode, self.batch, self.device = mode, batch, torch.device(device)
         self.dtype = torch.bfloat16
         n, k = batch, seed
@@ -164,17 +173,23 @@ class BackboneReplay:
         if keep is not None:
             keep["out"] = x.clone()
         g = ins["g"].clone()
+        # Tune mode: the parameter gradients of a bottleneck's blocks run beside its input-gradient chain and are
+        # joined once per bottleneck, after which what they were reading can be released
+        held = [] if self.mode == "tune" and self.async_param_grads else None
         for (c1, c2, c3, ds), (xin, a, b, out) in zip(reversed(self.blocks), reversed(relu_outs)):
             C.convbn_relu_bwd(g, out, g)                       # through the block's final ReLU; g feeds both branches
-            gb = c3.backward(g); C.convbn_relu_bwd(gb, b, gb)
-            ga = c2.backward(gb); C.convbn_relu_bwd(ga, a, ga)
-            gx = c1.backward(ga)
+            gb = c3.backward(g, held); C.convbn_relu_bwd(gb, b, gb)
+            ga = c2.backward(gb, held); C.convbn_relu_bwd(ga, a, ga)
+            gx = c1.backward(ga, held)
             if ds is not None:
-                gs = ds.backward(g)
+                gs = ds.backward(g, held)
                 C.convbn_add(gx, gs, gx)
                 del gs
             else:
                 C.convbn_add(gx, g, gx)
+            if held is not None:
+                C.convbn_tune_bwd_join()
+                held.clear()
             g = gx
             del gb, ga
         relu_outs.clear()

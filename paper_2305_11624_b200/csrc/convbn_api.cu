@@ -803,6 +803,26 @@ int side_lane(SideLane **out) {
     *out = &l;
     return CONVBN_OK;
 }
+
+// `side(lane stream)` and `main_pass()` side by side, the caller's stream joined to the lane before return.
+// Under the profiler (per-kernel event pairs on one stream) they run one after the other.
+template <class Side, class Main>
+int side_by_side(cudaStream_t st, Side &&side, Main &&main_pass) {
+    if (g_prof.on) {
+        CK(main_pass());
+        return side(st);
+    }
+    SideLane *lane = nullptr;
+    CK(side_lane(&lane));
+    CU(cudaEventRecord(lane->fork, st));
+    CU(cudaStreamWaitEvent(lane->stream, lane->fork, 0));
+    const int ss = side(lane->stream);
+    // whatever happened on the lane, the caller's stream joins it again (a capture must not be left forked)
+    const bool joined = cudaEventRecord(lane->join, lane->stream) == cudaSuccess;
+    const int sm = main_pass();
+    if (!joined || cudaStreamWaitEvent(st, lane->join, 0) != cudaSuccess) return CONVBN_ECUDA;
+    return ss != CONVBN_OK ? ss : sm;
+}
 }  // namespace
 
 extern "C" {
@@ -940,12 +960,18 @@ int convbn_eval_bwd(const convbn_desc *desc, const void *dz, const void *x, cons
     LAUNCH("bn_eval_bwd", launch_bn_eval_bwd(pb, desc->dtype, desc->layout, dz, y_saved, gamma, run_mean, run_var, dy, pg,
                           pbm, pl.bn_splits, st));
     LAUNCH("bn_eval_finish", launch_bn_eval_finish(pb, pg, pbm, pl.bn_splits, gamma, run_var, db, dgamma, dbeta, st));
-    CK(run_conv_dgrad(desc, pb, dy, w, nullptr, at(workspace, pl.w_scaled), at(workspace, pl.wbd), dx, st,
-                      &t_last_kernel[CONVBN_PHASE_EVAL_BWD]));
-    const char *unused = nullptr;
-    CK(run_param_grads(desc, pb, pl, dy, x, w, nullptr, nullptr, nullptr, dw, nullptr, nullptr, nullptr, workspace,
-                       st, &unused));
-    return CONVBN_OK;
+    // dX and domega both start from dY and use separate regions of the workspace: side by side, as in Tune mode
+    return side_by_side(
+        st,
+        [&](cudaStream_t lane) {
+            const char *unused = nullptr;
+            return run_param_grads(desc, pb, pl, dy, x, w, nullptr, nullptr, nullptr, dw, nullptr, nullptr, nullptr, workspace,
+                                   lane, &unused);
+        },
+        [&]() {
+            return run_conv_dgrad(desc, pb, dy, w, nullptr, at(workspace, pl.w_scaled), at(workspace, pl.wbd), dx, st,
+                                  &t_last_kernel[CONVBN_PHASE_EVAL_BWD]);
+        });
 }
 
 int convbn_deploy_prepare(const convbn_desc *desc, const void *w, const float *b, const float *gamma,
@@ -996,12 +1022,17 @@ int convbn_deploy_bwd(const convbn_desc *desc, const void *dz, const void *x, co
     const Plan pl = make_plan(desc, pb, CONVBN_PHASE_DEPLOY_BWD);
     CK(check_ws(pl, workspace, workspace_bytes));
     cudaStream_t st = (cudaStream_t)stream;
-    CK(run_conv_dgrad(desc, pb, dz, w_fused, nullptr, at(workspace, pl.w_scaled), at(workspace, pl.wbd), dx, st,
-                      &t_last_kernel[CONVBN_PHASE_DEPLOY_BWD]));
-    const char *unused = nullptr;
-    CK(run_param_grads(desc, pb, pl, dz, x, w_fused, nullptr, nullptr, nullptr, dw_fused, db_fused, nullptr, nullptr,
-                       workspace, st, &unused));
-    return CONVBN_OK;
+    return side_by_side(
+        st,
+        [&](cudaStream_t lane) {
+            const char *unused = nullptr;
+            return run_param_grads(desc, pb, pl, dz, x, w_fused, nullptr, nullptr, nullptr, dw_fused, db_fused, nullptr, nullptr,
+                                   workspace, lane, &unused);
+        },
+        [&]() {
+            return run_conv_dgrad(desc, pb, dz, w_fused, nullptr, at(workspace, pl.w_scaled), at(workspace, pl.wbd), dx, st,
+                                  &t_last_kernel[CONVBN_PHASE_DEPLOY_BWD]);
+        });
 }
 
 // ---- TransposedConv-BN -----------------------------------------------------------------------------

@@ -117,6 +117,20 @@ def test_modes_agree_and_eval_keeps_more():
     assert peaks["eval"] > 1.3 * max(peaks["tune"], peaks["deploy"]), peaks
 
 
+def test_async_parameter_gradients_give_the_same_bits():
+    outs = []
+    for flag in (False, True):
+        rp = BackboneReplay(2, PLAN, "tune", seed=3, async_param_grads=flag)
+        ins = rp.make_inputs(5)
+        keep = {}
+        rp.forward_backward(ins, keep)
+        torch.cuda.synchronize()
+        outs.append((keep["out"], keep["dx"], [l.blk.dw.clone() for l in rp.layers], [l.blk.dgamma.clone() for l in rp.layers]))
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    for a, b in zip(outs[0][2] + outs[0][3], outs[1][2] + outs[1][3]):
+        assert torch.equal(a, b)
+
+
 def test_resnet50_plan_has_53_blocks():
     stem, plan = resnet50_plan(224)
     rp_layers = 1 + sum(3 + (1 if (b.stride > 1 or b.c_in != b.c_out) else 0) for b in plan)
