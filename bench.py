@@ -3,7 +3,8 @@
 
 A step is one pass of the whole path - convbn_tune_fwd, then convbn_tune_bwd_begin (input gradient on the
 caller's stream, parameter gradients on the library's side stream) - over every layer of a configuration,
-closed by one convbn_tune_bwd_join (``--join-per-layer``: convbn_tune_bwd, which joins in every call).  With no ``--workload`` all five
+closed by one convbn_tune_bwd_join (``--join-per-layer``: convbn_tune_bwd, which joins in every call;
+``--order training``: every forward call first, then every backward call).  With no ``--workload`` all five
 configurations run in one process and ONE JSON line is printed: ``value`` is the fwd+bwd TFLOP/s
 over the three dense bf16 configurations (1-3: total FLOPs / total time), ``per_config`` holds
 every configuration on its own (config 4 in GB/s against the copy bandwidth, config 0 as a
@@ -348,11 +349,26 @@ def bench_config(ctx, wl):
     # library's side stream and the step joins once at its end (--join-per-layer: every call joins before it returns).
     defer = not args.join_per_layer
 
+    def run_layers(bs, st=None):
+        """One step over the layers `bs`.  Deferred mode follows the order of a training step: every forward call,
+        each followed by the preparation of its backward weights on the library's prepare stream; then every backward
+        call (input gradients on the caller's stream, parameter gradients on the side stream); one join."""
+        if not defer:
+            for b in bs:
+                b.tune_step(st)
+            return
+        if args.order == "layer":
+            for b in bs:
+                b.tune_step(st, defer_join=True)
+        else:
+            for b in bs:
+                b.tune_fwd(st)
+            for b in bs:
+                b.tune_bwd_begin(st)
+        C.convbn_tune_bwd_join(st)
+
     def step(i):
-        for b in blocks[i % sets]:
-            b.tune_step(stream, defer_join=defer)
-        if defer:
-            C.convbn_tune_bwd_join(stream)
+        run_layers(blocks[i % sets], stream)
         if buckets:
             buckets[i % sets].all_reduce_async()
             buckets[i % sets].wait()
@@ -376,10 +392,7 @@ def bench_config(ctx, wl):
             for si in range(sets):
                 gr = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(gr):
-                    for b in blocks[si]:
-                        b.tune_step(defer_join=defer)
-                    if defer:
-                        C.convbn_tune_bwd_join()
+                    run_layers(blocks[si])
                 graphs.append(gr)
             for gr in graphs:
                 gr.replay()
@@ -388,7 +401,9 @@ def bench_config(ctx, wl):
         except Exception as exc:  # capture unsupported: say so and time eager calls
             graphs, launch_mode = None, "eager library calls (graph capture failed: %r)" % (exc,)
 
-    launch_mode += ("; parameter-gradient passes on the library's side stream, one join per step" if defer
+    launch_mode += ("; %s; parameter-gradient passes on the library's side stream, one join per step"
+                    % ("forward then backward of each layer in turn" if args.order == "layer"
+                       else "every forward call, then every backward call") if defer
                     else "; every backward call joins its parameter-gradient pass")
 
     def timed(n_sets):
@@ -411,6 +426,20 @@ def bench_config(ctx, wl):
     sampler.start()
     ms = timed(sets)                            # cold: rotating sets, together larger than twice the L2
     ms_warm = timed(1)                          # warm: the same buffers every step
+    # the other orders of the same step, for comparison: every forward call before every backward call (what a
+    # training step does: the forward phase then has nothing to overlap with), and one stream joined in every call
+    ms_other = {}
+    if graphs and defer and args.order == "layer":
+        keep_graphs = graphs
+        for name, order, dfr in (("training_order", "training", True), ("join_per_layer", "layer", False)):
+            args.order, defer, graphs = order, dfr, []
+            for si in range(sets):
+                gr = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gr):
+                    run_layers(blocks[si])
+                graphs.append(gr)
+            ms_other[name] = timed(sets) / args.steps
+        args.order, defer, graphs = "layer", True, keep_graphs
     # ---- second pass, same K steps as eager calls with a CUDA-event pair around every kernel: the
     # per-kernel durations behind the roofline object (events cannot be read back out of a graph)
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -511,6 +540,7 @@ def bench_config(ctx, wl):
            "flops_per_step": step_flops, "two_pass_bytes_per_step": two_pass_bytes,
            "l2": "cold: %d rotating buffer sets of %.0f MB (activations) against an L2 of %.0f MB; warm: one set"
                  % (sets, footprint / 1e6, l2 / 1e6),
+           "ms_per_step_other_orders": ms_other,
            "launch": launch_mode, "launches_per_step": launches_per_step, "host_us_per_call": round(host_us, 2),
            "eager_ms_per_step": eager_ms / args.steps, "clocks": clocks, "roofline": roofline,
            "kernels": kernels[:10], "per_layer": per_layer,
@@ -748,6 +778,9 @@ def main():
     ap.add_argument("--no-modes", action="store_true", help="skip the Tune / Eval / Deploy comparison")
     ap.add_argument("--no-graph", action="store_true", help="time eager library calls instead of graph replays")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--order", default="layer", choices=["layer", "training"],
+                    help="layer: forward then backward of each layer in turn; training: every forward call, then every "
+                         "backward call")
     ap.add_argument("--join-per-layer", action="store_true",
                     help="every backward call joins its parameter-gradient pass before returning (default: one join per step)")
     ap.add_argument("--no-backbone", action="store_true", help="skip the whole-ResNet-50 replay in the three modes")

@@ -787,7 +787,11 @@ namespace {
 // parameter-gradient pass (GEMM + epilogue) runs there while the input-gradient pass (weight re-layout + GEMM) runs
 // on the caller's stream; the caller's stream waits for the lane before the call returns, so stream order is what
 // the caller sees.  (Per thread: two threads sharing the events could wait on each other's fork points.)
-struct SideLane { cudaStream_t stream = nullptr; cudaEvent_t fork = nullptr, join = nullptr; };
+struct SideLane {
+    cudaStream_t stream = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+    bool pending = false;          // passes begun there that no stream has joined yet
+};
 thread_local SideLane t_side_lane[kMaxDevices];
 
 int side_lane(SideLane **out) {
@@ -848,7 +852,7 @@ static int tune_bwd_impl(const convbn_desc *desc, const void *dz, const void *x,
         void *ws_w = workspace ? at(workspace, pl.w_scaled) : nullptr;
         const size_t bytes_d = pl.w_scaled, bytes_w = pl.total - pl.w_scaled;
         t_last_kernel[CONVBN_PHASE_TUNE_BWD] = "two-calls";
-        if (g_prof.on && !defer_join) {  // per-kernel timing wants one stream
+        if (g_prof.on) {                 // per-kernel timing wants one stream, deferred or not
             CK(convbn_tune_bwd_data(desc, dz, w, saved, dx, workspace, bytes_d, stream));
             return convbn_tune_bwd_weight(desc, dz, x, w, b, run_mean, saved, dw, db, dgamma, dbeta, ws_w, bytes_w, stream);
         }
@@ -863,7 +867,8 @@ static int tune_bwd_impl(const convbn_desc *desc, const void *dz, const void *x,
         const bool joined = cudaEventRecord(lane->join, lane->stream) == cudaSuccess;
         const int sd = convbn_tune_bwd_data(desc, dz, w, saved, dx, workspace, bytes_d, stream);
         if (!joined) return CONVBN_ECUDA;
-        if (!defer_join && cudaStreamWaitEvent(st, lane->join, 0) != cudaSuccess) return CONVBN_ECUDA;
+        if (defer_join) lane->pending = true;
+        else if (cudaStreamWaitEvent(st, lane->join, 0) != cudaSuccess) return CONVBN_ECUDA;
         return sw != CONVBN_OK ? sw : sd;
     }
     cudaStream_t st = (cudaStream_t)stream;
@@ -873,7 +878,7 @@ static int tune_bwd_impl(const convbn_desc *desc, const void *dz, const void *x,
     const float *vec3 = (const float *)saved;
     LAUNCH("umma_bwd", launch_fused_bwd1x1(pb, dz, x, w, vec3, dx, partials, bsum, counters, st));
     t_last_kernel[CONVBN_PHASE_TUNE_BWD] = "umma-fused-bwd";
-    if (defer_join) {
+    if (defer_join && !g_prof.on) {
         // dX is complete on the caller's stream; the parameter gradients are finished on the side lane
         SideLane *lane = nullptr;
         CK(side_lane(&lane));
@@ -883,6 +888,7 @@ static int tune_bwd_impl(const convbn_desc *desc, const void *dz, const void *x,
         LAUNCH("wgrad_epilogue_fused", launch_wgrad_epilogue_fused(pb, pl.uw, partials, bsum, w, vec3, b, run_mean, dw,
                                                                    dotpart, counters, db, dgamma, dbeta, true, st));
         CU(cudaEventRecord(lane->join, lane->stream));
+        lane->pending = true;
         return CONVBN_OK;
     }
     LAUNCH("wgrad_epilogue_fused", launch_wgrad_epilogue_fused(pb, pl.uw, partials, bsum, w, vec3, b, run_mean, dw, dotpart,
@@ -907,9 +913,13 @@ int convbn_tune_bwd_begin(const convbn_desc *desc, const void *dz, const void *x
 int convbn_tune_bwd_join(void *stream) {
     SideLane *lane = nullptr;
     CK(side_lane(&lane));
-    // the lane is one stream: its last join point covers every pass begun before it
-    CU(cudaEventRecord(lane->join, lane->stream));
-    CU(cudaStreamWaitEvent((cudaStream_t)stream, lane->join, 0));
+    // the lane is one stream: its last join point covers every pass begun before it.  With nothing pending the
+    // lane is left alone (inside a stream capture it may not be part of the capture at all).
+    if (lane->pending) {
+        CU(cudaEventRecord(lane->join, lane->stream));
+        CU(cudaStreamWaitEvent((cudaStream_t)stream, lane->join, 0));
+        lane->pending = false;
+    }
     return CONVBN_OK;
 }
 
