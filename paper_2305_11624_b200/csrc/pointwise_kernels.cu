@@ -156,31 +156,6 @@ __global__ void __launch_bounds__(256) reparam_dgrad_kernel(int c_out, int c_in,
     }
 }
 
-// The same for channel counts that are multiples of 64: 64 x 64 tiles, two elements per access, so that both the
-// reads (along C_in) and the writes (along C_out) are 128 contiguous bytes per warp instruction.
-__global__ void __launch_bounds__(256) reparam_dgrad64_kernel(int c_out, int c_in, int taps,
-                                                              const uint32_t *__restrict__ w2,
-                                                              const float *__restrict__ s_vec,
-                                                              uint32_t *__restrict__ w_t2, int f16) {
-    __shared__ float tile[64][65];
-    pdl_wait();
-    pdl_launch_dependents();
-    const int tap = blockIdx.z, co0 = blockIdx.y * 64, ci0 = blockIdx.x * 64;
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    for (int j = ty; j < 64; j += 8) {
-        const int co = co0 + j;
-        const float sc = s_vec ? s_vec[co] : 1.f;
-        const uint32_t v = w2[(((long long)co * taps + tap) * c_in + ci0) / 2 + tx];
-        tile[j][2 * tx] = sc * unpack_h16((uint16_t)(v & 0xFFFFu), f16);
-        tile[j][2 * tx + 1] = sc * unpack_h16((uint16_t)(v >> 16), f16);
-    }
-    __syncthreads();
-    for (int j = ty; j < 64; j += 8) {
-        const int ci = ci0 + j;
-        w_t2[(((long long)ci * taps + (taps - 1 - tap)) * c_out + co0) / 2 + tx] = pack2_h16(tile[2 * tx][j], tile[2 * tx + 1][j], f16);
-    }
-}
-
 __global__ void __launch_bounds__(256) reparam_dgrad_class_kernel(int c_out, int c_in, int kw, int tw, int r_max,
                                                                   int q_max, int step_h, int step_w, int ctaps,
                                                                   const __nv_bfloat16 *__restrict__ w,
@@ -253,12 +228,6 @@ cudaError_t launch_reparam_dgrad_classes(const Problem &pb, const void *w, const
 
 cudaError_t launch_reparam_dgrad(const Problem &pb, const void *w, const float *s_vec, void *w_t,
                                  cudaStream_t st) {
-    if (pb.c_in % 64 == 0 && pb.c_out % 64 == 0) {
-        static PerDevice carve64;
-        prefer_max_shared_once(reparam_dgrad64_kernel, &carve64);
-        return launch_pdl(reparam_dgrad64_kernel, dim3(pb.c_in / 64, pb.c_out / 64, pb.kh * pb.kw), dim3(256), 0, st, pb.c_out,
-                          pb.c_in, pb.kh * pb.kw, (const uint32_t *)w, s_vec, (uint32_t *)w_t, call_f16());
-    }
     dim3 grid((pb.c_in + 31) / 32, (pb.c_out + 31) / 32, pb.kh * pb.kw);
     static PerDevice carve;
     prefer_max_shared_once(reparam_dgrad_kernel, &carve);
