@@ -424,7 +424,11 @@ int run_conv_fwd(const convbn_desc *d, const Problem &pb, const void *x, const v
 // Backward data.  `scale` (C_out floats or NULL) is folded into the weights on the way:
 // w_scratch receives omega' in the layout the chosen kernel wants.
 int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, const void *w, const float *scale,
-                   void *w_scratch, void *wbd_scratch, void *dx, cudaStream_t st, const char **which) {
+                   void *w_scratch, void *wbd_scratch, void *dx, cudaStream_t st, const char **which,
+                   const float *out_bias = nullptr, bool *bias_done = nullptr) {
+    // out_bias (C_in floats, optional): added to dX by the paths whose epilogue can do it; *bias_done says whether it was
+    // (the transposed-convolution forward pass is this pass plus a bias)
+    if (bias_done) *bias_done = false;
     UmmaConvShape s;
     if (stem_path(d, pb) && stem_window_dgrad_eligible(pb)) {
         // stride 2, C_in <= 4: scatter GEMM over dZ rows, window positions added up on chip
@@ -519,12 +523,13 @@ int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, cons
     } else if (umma_dgrad_shape(d, pb, &s)) {
         LAUNCH("reparam_dgrad", launch_reparam_dgrad(pb, w, scale, w_scratch, st));
         if (umma_strip_eligible(s)) {
-            LAUNCH("strip_dgrad", launch_umma_strip_conv(s, dz, w_scratch, nullptr, dx, st));
+            LAUNCH("strip_dgrad", launch_umma_strip_conv(s, dz, w_scratch, out_bias, dx, st));
             *which = "umma-strip";
         } else {
-            LAUNCH("umma_dgrad", launch_umma_conv(s, dz, w_scratch, nullptr, dx, st));
+            LAUNCH("umma_dgrad", launch_umma_conv(s, dz, w_scratch, out_bias, dx, st));
             *which = "umma";
         }
+        if (bias_done && out_bias) *bias_done = true;
     } else if (dw_path(d, pb)) {
         if (pb.stride_h == 1 && pb.stride_w == 1) {
             // dX = omega'_rot (*) dZ is itself a stride-1 depthwise convolution of dZ with the rotated
@@ -1130,10 +1135,14 @@ int convbn_tconv_tune_fwd(const convbn_desc *desc, const void *x, const void *w,
     LAUNCH("tconv_rescale", launch_tconv_rescale(desc->dtype, nhwc, (long long)v.wcount, taps, cig, cog, w, vec3, wf, st));
     // Z = omega' scattered over X: the backward-data pass of the convolution with the same weights
     const char *which = nullptr;
-    CK(run_conv_dgrad(&v.conv, v.pb, x, wf, nullptr, at(inner, v.bwd.w_scaled), at(inner, v.bwd.wbd), z, st, &which));
-    const long long count = (long long)desc->n * desc->c_out * v.h_out * v.w_out;
-    LAUNCH("tconv_bias", launch_tconv_bias(desc->dtype, nhwc, count, desc->c_out, (long long)v.h_out * v.w_out,
-                                           vec3 + desc->c_out, z, st));
+    bool bias_done = false;          // unit-stride tensor-core layers add b' in the GEMM's own epilogue (one rounding)
+    CK(run_conv_dgrad(&v.conv, v.pb, x, wf, nullptr, at(inner, v.bwd.w_scaled), at(inner, v.bwd.wbd), z, st, &which,
+                      vec3 + desc->c_out, &bias_done));
+    if (!bias_done) {
+        const long long count = (long long)desc->n * desc->c_out * v.h_out * v.w_out;
+        LAUNCH("tconv_bias", launch_tconv_bias(desc->dtype, nhwc, count, desc->c_out, (long long)v.h_out * v.w_out,
+                                               vec3 + desc->c_out, z, st));
+    }
     return CONVBN_OK;
 }
 
