@@ -86,12 +86,17 @@ def compare(got: dict, ref: dict, tol: float, names, label="", dtype=None, grads
     return errs
 
 
-def run_tune_gpu(spec, t, device="cuda:0"):
+def run_tune_gpu(spec, t, device="cuda:0", deferred=False):
+    """Tune forward + backward through the library.  deferred=False: the three separate calls; True: the calls a
+    benchmark step makes (convbn_tune_fwd, convbn_tune_bwd_begin, convbn_tune_bwd_join)."""
     from paper_2305_11624_b200.harness import Block
     from paper_2305_11624_b200 import convbn as C
     blk = Block(spec, device=device, modes=("tune",))
     blk.load(t)
-    blk.tune_fwd(); blk.tune_bwd_data(); blk.tune_bwd_weight()
+    if deferred:
+        blk.tune_fwd(); blk.tune_bwd_begin(); C.convbn_tune_bwd_join()
+    else:
+        blk.tune_fwd(); blk.tune_bwd_data(); blk.tune_bwd_weight()
     C.convbn_check()
     names = ["z", "dx", "dw", "dgamma", "dbeta"] + (["db"] if spec.bias else [])
     out = {k: blk.fetch(k) for k in names}

@@ -121,6 +121,9 @@ def test_tune_benchmark_configs_full_size(ci, li, spec):
     got = parity.run_tune_gpu(spec, t)
     errs = parity.compare(got, ref, parity.TOL[spec.dtype], parity.TUNE_OUTPUTS, spec.name, dtype=spec.dtype)
     print(spec.name, got["_kernels"], {k: "%.2e" % v for k, v in errs.items()})
+    # the calls a benchmark step makes (backward in one call, parameter gradients joined afterwards), same bounds
+    got = parity.run_tune_gpu(spec, t, deferred=True)
+    parity.compare(got, ref, parity.TOL[spec.dtype], parity.TUNE_OUTPUTS, spec.name + " (begin / join)", dtype=spec.dtype)
 
 
 def test_tune_is_deterministic_and_leaves_inputs_alone():
