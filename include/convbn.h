@@ -116,7 +116,7 @@ size_t convbn_workspace_bytes(const convbn_desc *desc, int phase);
 
 /* ---- Tune mode (Sec. 3.4; Table 2, Tune row) --------------------------------------------- */
 
-/* Forward: forms s, b' and omega' from the CURRENT parameters ("on the fly"), then
+/* Forward: forms s, b' and omega' from the CURRENT parameters at every call, then
  *     Z = omega' (*) X + b'.
  * in : x [activation], w [weight], b [C_out] or NULL (= no conv bias), gamma, beta, run_mean,
  *      run_var [C_out]
