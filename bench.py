@@ -667,9 +667,11 @@ def run_backbone(ctx, batch=32, size=224, iters=10):
     stem, plan = resnet50_plan(size)
     out = {"network": "ResNet-50 ConvBN blocks + ReLU + skip connections (max-pool replaced by synthetic tensors)",
            "batch": batch, "image": size, "dtype": "bf16", "iters": iters, "modes": {}}
-    for mode in ("tune", "eval", "deploy", "tune_async"):
-        # tune_async: Tune mode with the parameter-gradient passes joined once per bottleneck instead of per call
-        rp = BackboneReplay(batch, plan, mode.split("_")[0], stem_hw=stem, device=ctx.dev, async_param_grads=mode == "tune_async")
+    for mode in ("tune", "eval", "deploy", "tune_async", "tune_f16"):
+        # tune_async: Tune mode with the parameter-gradient passes joined once per bottleneck instead of per call;
+        # tune_f16: Tune mode with IEEE-half storage (the paper's mixed-precision rows)
+        rp = BackboneReplay(batch, plan, mode.split("_")[0], stem_hw=stem, device=ctx.dev, async_param_grads=mode == "tune_async",
+                            dtype="f16" if mode == "tune_f16" else "bf16")
         ms, peak, how = rp.measure(iters=iters, warmup=3)
         out["modes"][mode] = {"ms_per_iter": ms, "peak_bytes": peak, "tflops": rp.flops / ms / 1e9, "timing": how}
         out["flops_per_iter"] = rp.flops

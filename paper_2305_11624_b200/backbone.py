@@ -52,8 +52,8 @@ def resnet50_plan(size: int = 224) -> Tuple[Optional[Tuple[int, int]], List[Bott
 class _Layer:
     """One ConvBN block of the chain: parameters, gradients, the calls of the chosen mode."""
 
-    def __init__(self, name, n, c_in, hw, c_out, k, stride, mode, device, seed):
-        spec = I.LayerSpec(name, n, c_in, hw[0], hw[1], c_out, k, k, stride=stride, pad=k // 2)
+    def __init__(self, name, n, c_in, hw, c_out, k, stride, mode, device, seed, dtype="bf16"):
+        spec = I.LayerSpec(name, n, c_in, hw[0], hw[1], c_out, k, k, stride=stride, pad=k // 2, dtype=dtype)
         self.blk = Block(spec, device=device, modes=(mode,), allocate="params")
         self.blk.randomize_params(seed)
         self.mode = mode
@@ -109,15 +109,16 @@ class _Layer:
 
 class BackboneReplay:
     def __init__(self, batch: int, plan: List[Bottleneck], mode: str, stem_hw: Optional[Tuple[int, int]] = None,
-                 device="cuda:0", seed: int = 0, async_param_grads: bool = False):
-        assert mode in ("tune", "eval", "deploy")
+                 device="cuda:0", seed: int = 0, async_param_grads: bool = False, dtype: str = "bf16"):
+        assert mode in ("tune", "eval", "deploy") and dtype in ("bf16", "f16")
+        assert dtype == "bf16" or mode == "tune", "IEEE half is implemented for Tune mode"
         self.async_param_grads = async_param_grads
         self.mode, self.batch, self.device = mode, batch, torch.device(device)
-        self.dtype = torch.bfloat16
+        self.dtype = torch.bfloat16 if dtype == "bf16" else torch.float16
         n, k = batch, seed
         self.stem = None
         if stem_hw is not None:
-            self.stem = _Layer("stem", n, 3, stem_hw, 64, 7, 2, mode, device, k)
+            self.stem = _Layer("stem", n, 3, stem_hw, 64, 7, 2, mode, device, k, dtype)
             k += 1
         self.blocks = []
         for i, bt in enumerate(plan):
@@ -125,12 +126,12 @@ class BackboneReplay:
             hw3 = (bt.hw[0] // bt.stride, bt.hw[1] // bt.stride) if bt.stride > 1 else bt.hw
             if bt.stride > 1:      # floor convention of a 3x3 stride-2 pad-1 convolution
                 hw3 = ((bt.hw[0] - 1) // bt.stride + 1, (bt.hw[1] - 1) // bt.stride + 1)
-            c1 = _Layer("b%d.c1" % i, n, bt.c_in, bt.hw, bt.width, 1, 1, mode, device, k)
-            c2 = _Layer("b%d.c2" % i, n, bt.width, hw2, bt.width, 3, bt.stride, mode, device, k + 1)
-            c3 = _Layer("b%d.c3" % i, n, bt.width, hw3, bt.c_out, 1, 1, mode, device, k + 2)
+            c1 = _Layer("b%d.c1" % i, n, bt.c_in, bt.hw, bt.width, 1, 1, mode, device, k, dtype)
+            c2 = _Layer("b%d.c2" % i, n, bt.width, hw2, bt.width, 3, bt.stride, mode, device, k + 1, dtype)
+            c3 = _Layer("b%d.c3" % i, n, bt.width, hw3, bt.c_out, 1, 1, mode, device, k + 2, dtype)
             ds = None
             if bt.stride > 1 or bt.c_in != bt.c_out:
-                ds = _Layer("b%d.ds" % i, n, bt.c_in, bt.hw, bt.c_out, 1, bt.stride, mode, device, k + 3)
+                ds = _Layer("b%d.ds" % i, n, bt.c_in, bt.hw, bt.c_out, 1, bt.stride, mode, device, k + 3, dtype)
             k += 4
             self.blocks.append((c1, c2, c3, ds))
         self.first = plan[0]

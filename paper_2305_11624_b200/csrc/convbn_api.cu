@@ -365,7 +365,10 @@ struct HalfCall {
         const bool dense = d.layout == CONVBN_NHWC && pb.groups == 1 && pb.c_in % 64 == 0 && pb.c_out % 64 == 0 &&
                            umma_fwd_shape(&d, pb, &s) && (umma_dgrad_shape(&d, pb, &s) || strided_dgrad_ok(&d, pb)) &&
                            make_plan(&d, pb, CONVBN_PHASE_TUNE_BWD_WEIGHT).umma_wgrad;
-        if (!dense) { status = CONVBN_EUNSUPPORTED; return; }
+        // the stride-2 stem of an image network: its three window kernels
+        const bool stem = d.layout == CONVBN_NHWC && stem_path(&d, pb) && stem_window_eligible(pb) &&
+                          stem_window_dgrad_eligible(pb) && make_plan(&d, pb, CONVBN_PHASE_TUNE_BWD_WEIGHT).stem_win_wgrad;
+        if (!dense && !stem) { status = CONVBN_EUNSUPPORTED; return; }
         set_call_f16(1);
         set_here = true;
     }

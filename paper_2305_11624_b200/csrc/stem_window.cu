@@ -37,6 +37,7 @@ struct WinGemm {
     uint32_t strip_bytes;  // one patch buffer (multiple of 1024)
     int kblocks;           // 128-byte K rows of the resident weights: ceil(kh / 2)
     long long total_rows;  // n * h_out
+    int f16;               // 16-bit storage type: 0 bf16, 1 IEEE half
     BnFold fold;
 };
 
@@ -244,7 +245,7 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
         // ---------------- MMA issuers: unit u (one M block = 128 output pixels of one row) goes to issuer u % 4
         const int me = warp - kWinLoaders;
         if (elect_one()) {
-            constexpr uint32_t idesc = idesc_bf16_f32(128, BN, 0, 0);
+            const uint32_t idesc = idesc_h16_f32(128, BN, 0, 0, g.f16);
             const uint32_t a_hi = win_desc_hi(), b_hi = smem_desc_hi_sw128(1024);
             const uint32_t wres_lo = smem_desc_lo(smem_u32(wres), 16);
             long long cur = row_lo;
@@ -340,11 +341,10 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
                                 const float4 s0 = *(const float4 *)(scale_s + c), s1 = *(const float4 *)(scale_s + c + 4);
                                 const float4 b0 = *(const float4 *)(bias_s + c), b1 = *(const float4 *)(bias_s + c + 4);
                                 uint4 pk;
-                                __nv_bfloat162 h;
-                                h = __floats2bfloat162_rn(fmaf(__uint_as_float(v[j]), s0.x, b0.x), fmaf(__uint_as_float(v[j + 1]), s0.y, b0.y)); pk.x = *(uint32_t *)&h;
-                                h = __floats2bfloat162_rn(fmaf(__uint_as_float(v[j + 2]), s0.z, b0.z), fmaf(__uint_as_float(v[j + 3]), s0.w, b0.w)); pk.y = *(uint32_t *)&h;
-                                h = __floats2bfloat162_rn(fmaf(__uint_as_float(v[j + 4]), s1.x, b1.x), fmaf(__uint_as_float(v[j + 5]), s1.y, b1.y)); pk.z = *(uint32_t *)&h;
-                                h = __floats2bfloat162_rn(fmaf(__uint_as_float(v[j + 6]), s1.z, b1.z), fmaf(__uint_as_float(v[j + 7]), s1.w, b1.w)); pk.w = *(uint32_t *)&h;
+                                pk.x = pack2_h16(fmaf(__uint_as_float(v[j]), s0.x, b0.x), fmaf(__uint_as_float(v[j + 1]), s0.y, b0.y), g.f16);
+                                pk.y = pack2_h16(fmaf(__uint_as_float(v[j + 2]), s0.z, b0.z), fmaf(__uint_as_float(v[j + 3]), s0.w, b0.w), g.f16);
+                                pk.z = pack2_h16(fmaf(__uint_as_float(v[j + 4]), s1.x, b1.x), fmaf(__uint_as_float(v[j + 5]), s1.y, b1.y), g.f16);
+                                pk.w = pack2_h16(fmaf(__uint_as_float(v[j + 6]), s1.z, b1.z), fmaf(__uint_as_float(v[j + 7]), s1.w, b1.w), g.f16);
                                 *(uint4 *)(row + (((4 * half + (j >> 3)) ^ (lane & 7)) << 4)) = pk;
                             }
                         }
@@ -390,6 +390,7 @@ struct WinWgrad {
     int pitch, ksteps, T0, T1, kdim;
     uint32_t xstrip_bytes, dzrow_bytes;
     long long total_rows;
+    int f16;               // 16-bit storage type: 0 bf16, 1 IEEE half
 };
 
 struct WinWgCtl {
@@ -430,7 +431,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
     {
         uint4 *p4 = (uint4 *)xs;
         const int n16 = (int)(2 * (size_t)g.xstrip_bytes / 16);
-        for (int i = threadIdx.x; i < n16; i += kWgThreads) p4[i] = make_uint4(0, 0x3F800000u, 0, 0x3F800000u);
+        for (int i = threadIdx.x; i < n16; i += kWgThreads) p4[i] = make_uint4(0, one_h16(g.f16) << 16, 0, one_h16(g.f16) << 16);
         uint4 *z4 = (uint4 *)zeros;
         for (int i = threadIdx.x; i < 128; i += kWgThreads) z4[i] = make_uint4(0, 0, 0, 0);
     }
@@ -459,7 +460,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
             ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->x_empty[sb], ph ^ 1u, abort_flag));
             if (!ok) break;
             win_fill_patch<C>(xs + (size_t)sb * g.xstrip_bytes, x, ck.img, ck.h0 * 2 - g.pad_h, (ck.rows - 1) * 2 + g.kh,
-                              g.h_in, g.w_in, g.pad_w, g.pitch, (int)threadIdx.x, 32 * kWgLoaders, 0x3F80u);
+                              g.h_in, g.w_in, g.pad_w, g.pitch, (int)threadIdx.x, 32 * kWgLoaders, one_h16(g.f16));
             fence_proxy_async_smem();
             mbar_arrive(&ctl->x_full[sb]);
             if (++sb == 2) { sb = 0; ph ^= 1u; }
@@ -499,7 +500,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
             const uint32_t b_hi = smem_desc_hi_sw128(1024);
             // all accumulator columns of this class start from zero: one MMA against 16 zero rows (block stride 0)
             umma_bf16_ss_halves<false>(acc, ((smem_u32(xs) >> 4) & 0x3FFFu) | a_lbo, a_hi, smem_desc_lo(smem_u32(zeros), 0), b_hi,
-                                       idesc_bf16_f32(128, 64 * Te, 1, 1));
+                                       idesc_h16_f32(128, 64 * Te, 1, 1, g.f16));
             long long cur = row_lo;
             WinChunk ck;
             int sb = 0;
@@ -520,7 +521,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
                     if (t_hi > Te - 1) t_hi = Te - 1;
                     if (t_lo > t_hi) continue;
                     const int nblk = t_hi - t_lo + 1, i_lo = i_max - t_hi, cb_lo = Te - 1 - t_hi;
-                    const uint32_t idesc = idesc_bf16_f32(128, 64 * nblk, 1, 1);
+                    const uint32_t idesc = idesc_h16_f32(128, 64 * nblk, 1, 1, g.f16);
                     const uint32_t d = acc + 64u * (uint32_t)cb_lo;
                     uint32_t a_lo = (((xa + (uint32_t)pr * (uint32_t)g.pitch) >> 4) & 0x3FFFu) | a_lbo;
                     uint32_t b_lo = smem_desc_lo(dza + (uint32_t)i_lo * g.dzrow_bytes, g.dzrow_bytes);
@@ -669,6 +670,7 @@ cudaError_t launch_stem_window_wgrad(const Problem &pb, const void *dz, const vo
     g.kh = pb.kh; g.kw = pb.kw; g.pad_h = pb.pad_h; g.pad_w = pb.pad_w; g.pitch = pl.pitch; g.ksteps = pl.ksteps;
     g.T0 = (pb.kh + 1) / 2; g.T1 = pb.kh / 2; g.kdim = pb.kdim; g.xstrip_bytes = pl.xstrip; g.dzrow_bytes = pl.dzrow;
     g.total_rows = (long long)pb.n * pb.h_out;
+    g.f16 = call_f16();
     CUtensorMap tdz;
     const unsigned long long dims[3] = {(unsigned long long)pb.c_out, (unsigned long long)pb.w_out,
                                         (unsigned long long)pb.n * pb.h_out};
@@ -696,6 +698,7 @@ cudaError_t launch_stem_window_fwd(const Problem &pb, const void *x, const void 
     g.R = pl.R; g.rows_in = (pl.R - 1) * pb.stride_h + pb.kh; g.pitch = pl.pitch;
     g.colblocks = (pb.w_out + 127) / 128; g.nstrips = pl.nstrips; g.strip_bytes = pl.strip_bytes;
     g.kblocks = pl.kblocks; g.total_rows = (long long)pb.n * pb.h_out;
+    g.f16 = call_f16();
     g.fold = fold ? *fold : BnFold{nullptr, nullptr, nullptr, nullptr, nullptr, 0.f, nullptr};
     CUtensorMap tout;
     const unsigned long long dims[3] = {(unsigned long long)pb.c_out, (unsigned long long)pb.w_out,

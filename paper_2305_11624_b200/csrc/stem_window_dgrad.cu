@@ -33,6 +33,7 @@ struct WinDgrad {
     int halo;                                // (kh - 1) / 2 dZ rows before a segment
     long long total_rows;                    // n * h_out
     const float *s_vec;                      // per-channel scale folded into the weights (NULL: 1)
+    int f16;                                 // 16-bit storage type: 0 bf16, 1 IEEE half
 };
 
 struct WinDgCtl {
@@ -125,9 +126,9 @@ __global__ void __launch_bounds__(kDgThreads) stem_window_dgrad_kernel(const __g
                     int rem = e - co * rowlen;
                     if (rem < 0) { --co; rem += rowlen; }      // the rounded-up reciprocal can overshoot by one
                     const int nrow = ctl->nrow_of[rem];
-                    const float wv = __uint_as_float((wd[h >> 1] >> ((h & 1) * 16)) << 16);     // bf16 -> fp32
+                    const float wv = unpack_h16((uint16_t)(wd[h >> 1] >> ((h & 1) * 16)), g.f16);
                     const float v = (g.s_vec ? g.s_vec[co] : 1.f) * wv;
-                    *(__nv_bfloat16 *)(wres + (size_t)nrow * 128 + ((((co >> 3) ^ (nrow & 7)) & 7) << 4) + (co & 7) * 2) = __float2bfloat16_rn(v);
+                    *(uint16_t *)(wres + (size_t)nrow * 128 + ((((co >> 3) ^ (nrow & 7)) & 7) << 4) + (co & 7) * 2) = pack1_h16(v, g.f16);
                 }
             }
         }
@@ -175,7 +176,7 @@ __global__ void __launch_bounds__(kDgThreads) stem_window_dgrad_kernel(const __g
                     const uint32_t blk = seq_first % kDgBlocks;
                     int run = (int)(kDgBlocks - blk);
                     if (run > nb) run = nb;
-                    const uint32_t idesc = idesc_bf16_f32(128, 32 * run, 0, 0);
+                    const uint32_t idesc = idesc_h16_f32(128, 32 * run, 0, 0, g.f16);
                     const uint32_t d = tmem_base + blk * 32u, b_lo = w_lo + (uint32_t)r0 * 256u;   // 32 rows x 128 B per r
 #pragma unroll
                     for (int k = 0; k < 4; ++k) umma_bf16_ss_halves<true>(d, a_lo + (uint32_t)k * 2u, hi, b_lo + (uint32_t)k * 2u, hi, idesc);
@@ -277,7 +278,7 @@ __global__ void __launch_bounds__(kDgThreads) stem_window_dgrad_kernel(const __g
 #pragma unroll
                             for (int t = 1; t < 4; ++t)
                                 if (j - t >= 0) acc += tile[((b + 2 * t - 2) * 4 + c) * 128 + j - t];
-                            if (p >= 0 && p < g.w_in) *(__nv_bfloat16 *)(rbuf + ((size_t)p * C + c) * 2) = __float2bfloat16_rn(acc);
+                            if (p >= 0 && p < g.w_in) *(uint16_t *)(rbuf + ((size_t)p * C + c) * 2) = pack1_h16(acc, g.f16);
                         }
                     }
                     named_bar_sync(bar_id, 128);
@@ -332,7 +333,7 @@ cudaError_t launch_stem_window_dgrad(const Problem &pb, const void *dz, const vo
     WinDgrad g;
     g.n = pb.n; g.h_in = pb.h_in; g.w_in = pb.w_in; g.h_out = pb.h_out; g.w_out = pb.w_out; g.c_out = pb.c_out;
     g.kh = pb.kh; g.kw = pb.kw; g.pad_h = pb.pad_h; g.pad_w = pb.pad_w; g.halo = (pb.kh - 1) / 2;
-    g.total_rows = (long long)pb.n * pb.h_out; g.s_vec = s_vec;
+    g.total_rows = (long long)pb.n * pb.h_out; g.s_vec = s_vec; g.f16 = call_f16();
     // input rows below the last one any output row reaches have no gradient: the kernel never visits them
     const int reached = 2 * (pb.h_out - 1) + pb.kh - pb.pad_h;       // first real row that is not reached
     if (reached < pb.h_in) {

@@ -33,15 +33,16 @@ def _cb_bwd(p, dz, x, w_f):
 BODY = resnet50_plan(64)[1]        # all 16 bottlenecks of a ResNet-50 on 64 x 64 images: 16 x 16 down to 2 x 2 pixels
 
 
-@pytest.mark.parametrize("mode,plan", [("tune", PLAN), ("eval", PLAN), ("deploy", PLAN), ("tune", BODY)],
-                         ids=["tune", "eval", "deploy", "tune_whole_body"])
-def test_three_bottlenecks_against_the_chained_oracle(mode, plan):
+@pytest.mark.parametrize("mode,plan,dtype", [("tune", PLAN, "bf16"), ("eval", PLAN, "bf16"), ("deploy", PLAN, "bf16"),
+                                             ("tune", BODY, "bf16"), ("tune", PLAN, "f16"), ("tune", BODY, "f16")],
+                         ids=["tune", "eval", "deploy", "tune_whole_body", "tune_half", "tune_whole_body_half"])
+def test_three_bottlenecks_against_the_chained_oracle(mode, plan, dtype):
     """The three modes compute one function with one set of input gradients (Sec. 3.3), so one oracle chain - the
     Tune formulas - checks all of them; Deploy's parameter gradients belong to the folded parameters and are left
     to the per-layer tests.  The last case chains all 52 blocks of the network body (images down to 2 x 2 pixels)."""
     PLAN = plan
     ch_in, hw0, ch_out, hw1 = plan[0].c_in, plan[0].hw, plan[-1].c_out, (plan[-1].hw[0] // plan[-1].stride, plan[-1].hw[1] // plan[-1].stride)
-    rp = BackboneReplay(2, PLAN, mode, seed=3)
+    rp = BackboneReplay(2, PLAN, mode, seed=3, dtype=dtype)
     ins = rp.make_inputs(5)
     keep = {}
     rp.forward_backward(ins, keep)
@@ -83,7 +84,7 @@ def test_three_bottlenecks_against_the_chained_oracle(mode, plan):
         dw_first = b1["dw"]
         g = gx
     depth = 3 * len(plan)           # convolutions on the longest path; rounding errors add in quadrature
-    tol = parity.TOL["bf16"] * np.sqrt(depth)
+    tol = parity.TOL[dtype] * np.sqrt(depth)
     got_out = nchw(keep["out"], ch_out, hw1)
     got_dx = nchw(keep["dx"], ch_in, hw0)
     errs = {"out": O.rel_l2(got_out, x), "dx": O.rel_l2(got_dx, g)}

@@ -22,6 +22,7 @@ SHAPES = [
     L("h_3x3_256_7x7", 4, 256, 7, 7, 256, 3, 3, pad=1, dtype="f16"),                 # small images: im2col GEMM
     L("h_1x1_s2_256_512", 2, 256, 14, 14, 512, 1, 1, stride=2, dtype="f16"),         # residue-class backward data
     L("h_5x5_64_d2", 1, 64, 24, 24, 64, 5, 5, pad=4, dil=2, dtype="f16"),
+    L("h_stem", 2, 3, 64, 80, 64, 7, 7, stride=2, pad=3, dtype="f16"),              # the three window kernels
 ]
 
 
@@ -65,7 +66,7 @@ def test_half_is_not_bf16():
 
 @pytest.mark.parametrize("spec,call", [
     (L("h_dw", 1, 64, 16, 16, 64, 3, 3, pad=1, groups=64, dtype="f16"), "tune"),
-    (L("h_stem", 1, 3, 32, 32, 64, 7, 7, stride=2, pad=3, dtype="f16"), "tune"),
+    (L("h_stem5", 1, 3, 32, 32, 64, 5, 5, stride=1, pad=2, dtype="f16"), "tune"),
     (L("h_odd", 1, 48, 16, 16, 64, 3, 3, pad=1, dtype="f16"), "tune"),
     (L("h_eval", 1, 64, 16, 16, 64, 3, 3, pad=1, dtype="f16"), "eval"),
 ], ids=lambda v: v.name if isinstance(v, L) else v)
