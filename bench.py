@@ -672,7 +672,15 @@ def run_backbone(ctx, batch=32, size=224, iters=10):
         # tune_f16: Tune mode with IEEE-half storage (the paper's mixed-precision rows)
         rp = BackboneReplay(batch, plan, mode.split("_")[0], stem_hw=stem, device=ctx.dev, async_param_grads=mode == "tune_async",
                             dtype="f16" if mode == "tune_f16" else "bf16")
-        ms, peak, how = rp.measure(iters=iters, warmup=3)
+        try:
+            ms, peak, how = rp.measure(iters=iters, warmup=3)
+        except ctx.C.ConvBNError as exc:       # half: the stem's window kernels take images up to 256 pixels wide
+            if mode != "tune_f16" or exc.status != ctx.C.EUNSUPPORTED:
+                raise
+            out["modes"][mode] = {"unsupported": str(exc)}
+            del rp
+            torch.cuda.empty_cache()
+            continue
         out["modes"][mode] = {"ms_per_iter": ms, "peak_bytes": peak, "tflops": rp.flops / ms / 1e9, "timing": how}
         out["flops_per_iter"] = rp.flops
         out["conv_bn_blocks"] = len(rp.layers)

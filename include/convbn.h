@@ -57,8 +57,8 @@ typedef enum {
 } convbn_status;
 
 /* Storage type of x, w, z, dz, dx.  CONVBN_F16 (IEEE half; the paper's mixed-precision rows, Table 4) is implemented for
- * the Tune-mode calls of dense NHWC layers whose channel counts are multiples of 64 and of the 7x7 stride-2 stem with at
- * most 4 input channels (the tensor-core paths: fp16 operands, fp32 accumulation, fp32 parameter gradients) and for the
+ * the Tune-mode calls of dense NHWC layers whose channel counts are multiples of 64 and of the stride-2 stem with at
+ * most 3 input channels on images up to 256 pixels wide (the tensor-core paths: fp16 operands, fp32 accumulation, fp32 parameter gradients) and for the
  * elementwise glue; every other call returns CONVBN_EUNSUPPORTED
  * for it. */
 typedef enum { CONVBN_F32 = 0, CONVBN_BF16 = 1, CONVBN_F16 = 2 } convbn_dtype;
