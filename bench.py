@@ -631,8 +631,10 @@ def run_e2e(ctx, blks, stream, step_flops):
         d2h += sum(t.numel() * t.element_size() for t in outs if t is not None)
 
     def step():
+        # every layer has its own arena: the next layer's inputs go up while this layer's results come down
         for desc, ins, outs, arena in host:
-            C.convbn_tune_step_host(desc, *ins, *outs, arena, stream=stream)
+            C.convbn_tune_step_host_begin(desc, *ins, *outs, arena, stream=stream)
+        C.convbn_tune_step_host_join(stream)
 
     steps = max(1, min(args.steps, args.e2e_steps))
     for _ in range(2):
@@ -738,7 +740,7 @@ def run_ours(args):
                "h2d_bytes_per_step": sum(e["h2d_bytes_per_step"] for e in es),
                "d2h_bytes_per_step": sum(e["d2h_bytes_per_step"] for e in es),
                "ms_per_step": e2e_ms, "steps": es[0]["steps"],
-               "note": "convbn_tune_step_host per layer: pinned host inputs up, every output down, inside the timed region"}
+               "note": "convbn_tune_step_host_begin per layer (its own arena each) and one join per step: pinned host inputs up, every output down, inside the timed region"}
     cpu = None
     cs = [c["cpu_baseline"] for c in headline if c.get("cpu_baseline")]
     if cs:

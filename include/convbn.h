@@ -228,16 +228,29 @@ size_t convbn_host_step_arena_bytes(const convbn_desc *desc);
  * and Table 2) with every tensor in HOST memory: x, dz, w, b (NULL = no bias), gamma, beta,
  * run_mean, run_var are host inputs; z, dx, dw, db (NULL iff b is NULL), dgamma, dbeta are host
  * outputs, in the dtype / layout conventions above.  Copies are asynchronous (use page-locked host
- * memory for them to overlap): everything is ordered on `stream`, except that dZ is uploaded on a
- * second, library-owned stream (one per device, created on the first call there) so that it crosses
- * the bus while Z comes back; `stream` waits for it before the backward kernels.  Outputs are valid,
- * and the host inputs may be reused, once `stream` has been synchronised.  `device_arena` is caller-owned DEVICE scratch of at least
- * convbn_host_step_arena_bytes(desc) bytes, 256-byte aligned. */
+ * memory for them to overlap).  The inputs go up on one library-owned stream, the results come down on another (one
+ * pair per device and host thread, created on the first call there) and the kernels run on `stream` in between, each
+ * step ordered behind what it needs: the uploads behind everything queued earlier on `stream`, the forward kernels
+ * behind X and the parameters, the backward kernels behind dZ (which crosses the bus while Z comes back), the
+ * downloads behind the kernels that produce them; finally `stream` waits for the last download.  Outputs are valid,
+ * and the host inputs may be reused, once `stream` has been synchronised.  `device_arena` is caller-owned DEVICE
+ * scratch of at least convbn_host_step_arena_bytes(desc) bytes, 256-byte aligned.
+ *
+ * convbn_tune_step_host_begin is the same call without that last wait: the next call's uploads (into ANOTHER arena)
+ * then cross the bus while this call's results come down.  Host buffers, outputs and the arena belong to the library
+ * until convbn_tune_step_host_join(stream) has made `stream` wait for every download begun by the calling host thread
+ * on the current device; a later call that reuses an arena waits for the earlier call's downloads by itself. */
 int convbn_tune_step_host(const convbn_desc *desc, const void *x, const void *dz, const void *w,
                           const float *b, const float *gamma, const float *beta,
                           const float *run_mean, const float *run_var, void *z, void *dx, float *dw,
                           float *db, float *dgamma, float *dbeta, void *device_arena,
                           size_t arena_bytes, void *stream);
+int convbn_tune_step_host_begin(const convbn_desc *desc, const void *x, const void *dz, const void *w,
+                                const float *b, const float *gamma, const float *beta,
+                                const float *run_mean, const float *run_var, void *z, void *dx, float *dw,
+                                float *db, float *dgamma, float *dbeta, void *device_arena,
+                                size_t arena_bytes, void *stream);
+int convbn_tune_step_host_join(void *stream);
 
 /* Backward with the parameter gradients off the critical path (what a training step wants: dX feeds the layer below at
  * once, domega, db, dgamma, dbeta are needed by the optimiser only).  convbn_tune_bwd_begin takes the arguments of

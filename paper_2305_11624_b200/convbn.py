@@ -24,7 +24,7 @@ EXPORTS = (
     "convbn_tune_bwd_data", "convbn_tune_bwd_weight", "convbn_eval_fwd", "convbn_eval_bwd",
     "convbn_deploy_prepare", "convbn_deploy_fwd", "convbn_deploy_bwd", "convbn_check",
     "convbn_status_string", "convbn_last_kernel", "convbn_host_step_arena_bytes",
-    "convbn_tune_step_host", "convbn_profile_begin", "convbn_profile_end",
+    "convbn_tune_step_host", "convbn_tune_step_host_begin", "convbn_tune_step_host_join", "convbn_profile_begin", "convbn_profile_end",
     "convbn_tune_bwd_weight_noalloc", "convbn_selftest_wait_timeout", "convbn_tune_bwd", "convbn_linear_desc", "convbn_relu", "convbn_add_relu", "convbn_relu_bwd", "convbn_add",
     "convbn_tune_bwd_begin", "convbn_tune_bwd_join",
     "convbn_tconv_out_shape", "convbn_tconv_workspace_bytes", "convbn_tconv_tune_fwd", "convbn_tconv_tune_bwd",
@@ -310,6 +310,23 @@ def convbn_tune_step_host(desc, x, dz, w, b, gamma, beta, run_mean, run_var, z, 
                                        _ptr(dbeta), _ptr(device_arena), ctypes.c_size_t(ab),
                                        _stream(stream)),
            "convbn_tune_step_host")
+
+
+def convbn_tune_step_host_begin(desc, x, dz, w, b, gamma, beta, run_mean, run_var, z, dx, dw, db, dgamma,
+                          dbeta, device_arena, arena_bytes: Optional[int] = None, stream=None):
+    """All tensors but ``device_arena`` are HOST tensors (page-locked for asynchronous copies)."""
+    ab = _nbytes(device_arena) if arena_bytes is None else arena_bytes
+    _raise(lib().convbn_tune_step_host_begin(ctypes.byref(desc), _ptr(x), _ptr(dz), _ptr(w), _ptr(b),
+                                       _ptr(gamma), _ptr(beta), _ptr(run_mean), _ptr(run_var),
+                                       _ptr(z), _ptr(dx), _ptr(dw), _ptr(db), _ptr(dgamma),
+                                       _ptr(dbeta), _ptr(device_arena), ctypes.c_size_t(ab),
+                                       _stream(stream)),
+           "convbn_tune_step_host_begin")
+
+
+def convbn_tune_step_host_join(stream=None) -> None:
+    """Make `stream` wait for the downloads of every convbn_tune_step_host_begin call of this thread on this device."""
+    _raise(lib().convbn_tune_step_host_join(_stream(stream)), "convbn_tune_step_host_join")
 
 
 def convbn_profile_begin() -> None:

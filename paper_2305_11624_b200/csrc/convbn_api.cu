@@ -1262,33 +1262,38 @@ size_t convbn_host_step_arena_bytes(const convbn_desc *desc) {
 }
 
 namespace {
-// Second copy lane of convbn_tune_step_host: one stream and two events per device, made on first use.
-// The upload of dZ runs there while the forward kernels and the download of Z run on the caller's
-// stream, so the two PCIe directions are busy at the same time.
-struct CopyLane { cudaStream_t stream = nullptr; cudaEvent_t inputs_queued = nullptr, dz_ready = nullptr; };
-CopyLane g_copy_lane[64];
-std::mutex g_copy_lane_mu;
+// Copy lanes of convbn_tune_step_host: an upload stream, a download stream and their events, per device and host
+// thread, made on first use.  Inputs go up on one lane, results come down on the other, the kernels run on the
+// caller's stream in between; both directions of the bus are then busy at once, within a call (dZ goes up while Z
+// comes down) and, when the caller defers the join, across calls (the next layer's X goes up while this layer's dX
+// comes down).
+struct CopyLanes {
+    cudaStream_t up = nullptr, down = nullptr;
+    cudaEvent_t start = nullptr, in = nullptr, dz = nullptr, fwd = nullptr, bwd = nullptr, done = nullptr;
+    const void *last_arena = nullptr;     // the previous call's arena: a call that reuses it waits for its downloads
+    bool pending = false;                 // downloads no stream has joined yet
+};
+thread_local CopyLanes t_copy_lanes[kMaxDevices];
 
-int copy_lane(CopyLane **out) {
+int copy_lanes(CopyLanes **out) {
     int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return CONVBN_ECUDA;
-    CopyLane &l = g_copy_lane[dev];
-    if (!l.stream) {
-        if (cudaStreamCreateWithFlags(&l.stream, cudaStreamNonBlocking) != cudaSuccess) { l.stream = nullptr; return CONVBN_ECUDA; }
-        if (cudaEventCreateWithFlags(&l.inputs_queued, cudaEventDisableTiming) != cudaSuccess ||
-            cudaEventCreateWithFlags(&l.dz_ready, cudaEventDisableTiming) != cudaSuccess)
-            return CONVBN_ECUDA;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CONVBN_ECUDA;
+    CopyLanes &l = t_copy_lanes[dev];
+    if (!l.up) {
+        if (cudaStreamCreateWithFlags(&l.up, cudaStreamNonBlocking) != cudaSuccess) { l.up = nullptr; return CONVBN_ECUDA; }
+        if (cudaStreamCreateWithFlags(&l.down, cudaStreamNonBlocking) != cudaSuccess) return CONVBN_ECUDA;
+        cudaEvent_t *ev[6] = {&l.start, &l.in, &l.dz, &l.fwd, &l.bwd, &l.done};
+        for (cudaEvent_t *e : ev)
+            if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return CONVBN_ECUDA;
     }
     *out = &l;
     return CONVBN_OK;
 }
-}  // namespace
 
-int convbn_tune_step_host(const convbn_desc *desc, const void *x, const void *dz, const void *w,
-                          const float *b, const float *gamma, const float *beta,
-                          const float *run_mean, const float *run_var, void *z, void *dx, float *dw,
-                          float *db, float *dgamma, float *dbeta, void *device_arena,
-                          size_t arena_bytes, void *stream) {
+int host_step_impl(const convbn_desc *desc, const void *x, const void *dz, const void *w, const float *b,
+                   const float *gamma, const float *beta, const float *run_mean, const float *run_var, void *z, void *dx,
+                   float *dw, float *db, float *dgamma, float *dbeta, void *device_arena, size_t arena_bytes, void *stream,
+                   bool defer_join) {
     Problem pb;
     CK(make_problem(desc, &pb));
     CK(check_pair(desc));
@@ -1299,14 +1304,21 @@ int convbn_tune_step_host(const convbn_desc *desc, const void *x, const void *dz
     if (!device_arena || arena_bytes < ar.total) return CONVBN_EWORKSPACE;
     if (!aligned(device_arena, 256)) return CONVBN_EALIGN;
     cudaStream_t st = (cudaStream_t)stream;
+    CopyLanes *ln = nullptr;
+    CK(copy_lanes(&ln));
     char *d = (char *)device_arena;
     const size_t vb = (size_t)pb.c_out * sizeof(float);
     auto h2d = [&](size_t off, const void *src, size_t bytes) {
-        return cudaMemcpyAsync(d + off, src, bytes, cudaMemcpyHostToDevice, st);
+        return cudaMemcpyAsync(d + off, src, bytes, cudaMemcpyHostToDevice, ln->up);
     };
     auto d2h = [&](void *dst, size_t off, size_t bytes) {
-        return cudaMemcpyAsync(dst, d + off, bytes, cudaMemcpyDeviceToHost, st);
+        return cudaMemcpyAsync(dst, d + off, bytes, cudaMemcpyDeviceToHost, ln->down);
     };
+    // uploads start after everything queued earlier on `stream` (which may still read the arena); an arena that
+    // the previous call used is also still being downloaded from
+    CU(cudaEventRecord(ln->start, st));
+    CU(cudaStreamWaitEvent(ln->up, ln->start, 0));
+    if (ln->pending && ln->last_arena == device_arena) CU(cudaStreamWaitEvent(ln->up, ln->done, 0));
     CU(h2d(ar.x, x, ar.x_bytes));
     CU(h2d(ar.w, w, ar.w_bytes));
     CU(h2d(ar.gamma, gamma, vb));
@@ -1314,33 +1326,65 @@ int convbn_tune_step_host(const convbn_desc *desc, const void *x, const void *dz
     CU(h2d(ar.mean, run_mean, vb));
     CU(h2d(ar.var, run_var, vb));
     if (b) CU(h2d(ar.b, b, vb));
+    CU(cudaEventRecord(ln->in, ln->up));
+    CU(h2d(ar.dz, dz, ar.z_bytes));
+    CU(cudaEventRecord(ln->dz, ln->up));
     const float *db_dev = b ? (const float *)(d + ar.b) : nullptr;
-    {
-        // dZ goes up on the second lane, after the inputs above (and after everything queued earlier on
-        // `stream`, which may still read the arena), while the forward pass and the download of Z run here
-        std::lock_guard<std::mutex> lk(g_copy_lane_mu);
-        CopyLane *lane = nullptr;
-        CK(copy_lane(&lane));
-        CU(cudaEventRecord(lane->inputs_queued, st));
-        CU(cudaStreamWaitEvent(lane->stream, lane->inputs_queued, 0));
-        CU(cudaMemcpyAsync(d + ar.dz, dz, ar.z_bytes, cudaMemcpyHostToDevice, lane->stream));
-        CU(cudaEventRecord(lane->dz_ready, lane->stream));
-        CK(convbn_tune_fwd(desc, d + ar.x, d + ar.w, db_dev, (const float *)(d + ar.gamma),
-                           (const float *)(d + ar.beta), (const float *)(d + ar.mean),
-                           (const float *)(d + ar.var), d + ar.z, d + ar.saved, d + ar.ws, ar.ws_bytes, stream));
-        CU(d2h(z, ar.z, ar.z_bytes));
-        CU(cudaStreamWaitEvent(st, lane->dz_ready, 0));
-    }
+    CU(cudaStreamWaitEvent(st, ln->in, 0));
+    CK(convbn_tune_fwd(desc, d + ar.x, d + ar.w, db_dev, (const float *)(d + ar.gamma), (const float *)(d + ar.beta),
+                       (const float *)(d + ar.mean), (const float *)(d + ar.var), d + ar.z, d + ar.saved, d + ar.ws,
+                       ar.ws_bytes, stream));
+    CU(cudaEventRecord(ln->fwd, st));
+    CU(cudaStreamWaitEvent(ln->down, ln->fwd, 0));
+    CU(d2h(z, ar.z, ar.z_bytes));
+    CU(cudaStreamWaitEvent(st, ln->dz, 0));
     CK(convbn_tune_bwd_data(desc, d + ar.dz, d + ar.w, d + ar.saved, d + ar.dx, d + ar.ws, ar.ws_bytes, stream));
+    CK(convbn_tune_bwd_weight(desc, d + ar.dz, d + ar.x, d + ar.w, db_dev, (const float *)(d + ar.mean), d + ar.saved,
+                              (float *)(d + ar.dw), b ? (float *)(d + ar.db) : nullptr, (float *)(d + ar.dgamma),
+                              (float *)(d + ar.dbeta), d + ar.ws, ar.ws_bytes, stream));
+    CU(cudaEventRecord(ln->bwd, st));
+    CU(cudaStreamWaitEvent(ln->down, ln->bwd, 0));
     CU(d2h(dx, ar.dx, ar.x_bytes));
-    CK(convbn_tune_bwd_weight(desc, d + ar.dz, d + ar.x, d + ar.w, db_dev, (const float *)(d + ar.mean),
-                              d + ar.saved, (float *)(d + ar.dw), b ? (float *)(d + ar.db) : nullptr,
-                              (float *)(d + ar.dgamma), (float *)(d + ar.dbeta), d + ar.ws, ar.ws_bytes,
-                              stream));
     CU(d2h(dw, ar.dw, ar.dw_bytes));
     CU(d2h(dgamma, ar.dgamma, vb));
     CU(d2h(dbeta, ar.dbeta, vb));
     if (db) CU(d2h(db, ar.db, vb));
+    CU(cudaEventRecord(ln->done, ln->down));
+    ln->last_arena = device_arena;
+    ln->pending = true;
+    if (!defer_join) {
+        CU(cudaStreamWaitEvent(st, ln->done, 0));
+        ln->pending = false;
+    }
+    return CONVBN_OK;
+}
+}  // namespace
+
+int convbn_tune_step_host(const convbn_desc *desc, const void *x, const void *dz, const void *w,
+                          const float *b, const float *gamma, const float *beta,
+                          const float *run_mean, const float *run_var, void *z, void *dx, float *dw,
+                          float *db, float *dgamma, float *dbeta, void *device_arena,
+                          size_t arena_bytes, void *stream) {
+    return host_step_impl(desc, x, dz, w, b, gamma, beta, run_mean, run_var, z, dx, dw, db, dgamma, dbeta, device_arena,
+                          arena_bytes, stream, false);
+}
+
+int convbn_tune_step_host_begin(const convbn_desc *desc, const void *x, const void *dz, const void *w,
+                                const float *b, const float *gamma, const float *beta,
+                                const float *run_mean, const float *run_var, void *z, void *dx, float *dw,
+                                float *db, float *dgamma, float *dbeta, void *device_arena,
+                                size_t arena_bytes, void *stream) {
+    return host_step_impl(desc, x, dz, w, b, gamma, beta, run_mean, run_var, z, dx, dw, db, dgamma, dbeta, device_arena,
+                          arena_bytes, stream, true);
+}
+
+int convbn_tune_step_host_join(void *stream) {
+    CopyLanes *ln = nullptr;
+    CK(copy_lanes(&ln));
+    if (ln->pending) {
+        CU(cudaStreamWaitEvent((cudaStream_t)stream, ln->done, 0));
+        ln->pending = false;
+    }
     return CONVBN_OK;
 }
 
