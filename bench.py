@@ -669,15 +669,15 @@ def run_backbone(ctx, batch=32, size=224, iters=10):
     stem, plan = resnet50_plan(size)
     out = {"network": "ResNet-50 ConvBN blocks + ReLU + skip connections (max-pool replaced by synthetic tensors)",
            "batch": batch, "image": size, "dtype": "bf16", "iters": iters, "modes": {}}
-    for mode in ("tune", "eval", "deploy", "tune_async", "tune_f16"):
+    for mode in ("tune", "eval", "deploy", "tune_async", "tune_f16", "eval_f16"):
         # tune_async: Tune mode with the parameter-gradient passes joined once per bottleneck instead of per call;
-        # tune_f16: Tune mode with IEEE-half storage (the paper's mixed-precision rows)
+        # tune_f16, eval_f16: IEEE-half storage (the paper's mixed-precision rows)
         rp = BackboneReplay(batch, plan, mode.split("_")[0], stem_hw=stem, device=ctx.dev, async_param_grads=mode == "tune_async",
-                            dtype="f16" if mode == "tune_f16" else "bf16")
+                            dtype="f16" if mode.endswith("_f16") else "bf16")
         try:
             ms, peak, how = rp.measure(iters=iters, warmup=3)
         except ctx.C.ConvBNError as exc:       # half: the stem's window kernels take images up to 256 pixels wide
-            if mode != "tune_f16" or exc.status != ctx.C.EUNSUPPORTED:
+            if not mode.endswith("_f16") or exc.status != ctx.C.EUNSUPPORTED:
                 raise
             out["modes"][mode] = {"unsupported": str(exc)}
             del rp

@@ -56,11 +56,12 @@ typedef enum {
     CONVBN_ECAPACITY = 7     /* problem too large for the library's built-in scratch */
 } convbn_status;
 
-/* Storage type of x, w, z, dz, dx.  CONVBN_F16 (IEEE half; the paper's mixed-precision rows, Table 4) is implemented for
- * the Tune-mode calls of dense NHWC layers whose channel counts are multiples of 64 and of the stride-2 stem with at
- * most 3 input channels on images up to 256 pixels wide (the tensor-core paths: fp16 operands, fp32 accumulation, fp32 parameter gradients) and for the
- * elementwise glue; every other call returns CONVBN_EUNSUPPORTED
- * for it. */
+/* Storage type of x, w, z, dz, dx.  CONVBN_F16 (IEEE half; the paper's mixed-precision rows, Table 4: fp16 storage, fp32
+ * accumulation, fp32 parameter gradients) is implemented for NHWC layers in all three modes, for the transposed
+ * layers and for the elementwise glue, except: depthwise layers, the grouped layers that run on the grouped kernels
+ * (channels per group a multiple of 8), and layers with at most 8 input channels other than the stride-2 stem with
+ * at most 3 input channels on images up to 256 pixels wide.  Those calls return CONVBN_EUNSUPPORTED (the size
+ * queries return 0). */
 typedef enum { CONVBN_F32 = 0, CONVBN_BF16 = 1, CONVBN_F16 = 2 } convbn_dtype;
 typedef enum { CONVBN_NCHW = 0, CONVBN_NHWC = 1 } convbn_layout;
 typedef enum { CONVBN_MODE_TUNE = 0, CONVBN_MODE_EVAL = 1, CONVBN_MODE_DEPLOY = 2 } convbn_mode;

@@ -111,7 +111,6 @@ class BackboneReplay:
     def __init__(self, batch: int, plan: List[Bottleneck], mode: str, stem_hw: Optional[Tuple[int, int]] = None,
                  device="cuda:0", seed: int = 0, async_param_grads: bool = False, dtype: str = "bf16"):
         assert mode in ("tune", "eval", "deploy") and dtype in ("bf16", "f16")
-        assert dtype == "bf16" or mode == "tune", "IEEE half is implemented for Tune mode"
         self.async_param_grads = async_param_grads
         self.mode, self.batch, self.device = mode, batch, torch.device(device)
         self.dtype = torch.bfloat16 if dtype == "bf16" else torch.float16

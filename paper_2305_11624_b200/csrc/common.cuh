@@ -74,6 +74,11 @@ __device__ __forceinline__ uint32_t pack2_t(float a, float b) {
     if constexpr (F16) { const __half2 h = __floats2half2_rn(a, b); return *reinterpret_cast<const uint32_t *>(&h); }
     else { const __nv_bfloat162 h = __floats2bfloat162_rn(a, b); return *reinterpret_cast<const uint32_t *>(&h); }
 }
+template <bool F16>
+__device__ __forceinline__ void unpack2_t(uint32_t bits, float &lo, float &hi) {
+    if constexpr (F16) { const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&bits)); lo = f.x; hi = f.y; }
+    else { lo = __uint_as_float(bits << 16); hi = __uint_as_float(bits & 0xFFFF0000u); }
+}
 __device__ __forceinline__ uint16_t pack1_h16(float a, int f16) {
     if (f16) { const __half h = __float2half_rn(a); return *reinterpret_cast<const uint16_t *>(&h); }
     const __nv_bfloat16 h = __float2bfloat16_rn(a);

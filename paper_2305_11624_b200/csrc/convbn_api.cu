@@ -345,9 +345,11 @@ bool strided_dgrad_ok(const convbn_desc *d, const Problem &pb) {
            pb.pin < (1LL << 31) - 256;
 }
 
-// CONVBN_F16 calls.  IEEE half runs on the 16-bit tensor-core paths only: the descriptor is checked for them, then
-// the call proceeds as its bf16 twin with the half flag set for the launchers (operand format of the MMAs,
-// conversions of results and of rescaled weights, the constant 1).  The flag is cleared when the call returns.
+// CONVBN_F16 calls.  IEEE half runs on every path of ungrouped NHWC layers whose kernels know the type: the dense
+// tensor-core kernels, the three window kernels of a stride-2 stem, the direct kernels and the element-wise ones.
+// The descriptor is checked for them, then the call proceeds as its bf16 twin with the half flag set for the
+// launchers (operand format of the MMAs, conversions of results and of rescaled weights, the constant 1, the
+// element type of the templated kernels).  The flag is cleared when the call returns.
 struct HalfCall {
     convbn_desc d;
     const convbn_desc *use;
@@ -361,14 +363,13 @@ struct HalfCall {
         Problem pb;
         status = make_problem(&d, &pb);
         if (status != CONVBN_OK) return;
-        UmmaConvShape s;
-        const bool dense = d.layout == CONVBN_NHWC && pb.groups == 1 && pb.c_in % 64 == 0 && pb.c_out % 64 == 0 &&
-                           umma_fwd_shape(&d, pb, &s) && (umma_dgrad_shape(&d, pb, &s) || strided_dgrad_ok(&d, pb)) &&
-                           make_plan(&d, pb, CONVBN_PHASE_TUNE_BWD_WEIGHT).umma_wgrad;
-        // the stride-2 stem of an image network: its three window kernels
-        const bool stem = d.layout == CONVBN_NHWC && stem_path(&d, pb) && stem_window_eligible(pb) &&
-                          stem_window_dgrad_eligible(pb) && make_plan(&d, pb, CONVBN_PHASE_TUNE_BWD_WEIGHT).stem_win_wgrad;
-        if (!dense && !stem) { status = CONVBN_EUNSUPPORTED; return; }
+        const Plan pw = make_plan(&d, pb, CONVBN_PHASE_TUNE_BWD_WEIGHT);
+        // depthwise and grouped kernels read bf16 only; so do the packed (non-window) stem kernels
+        const bool typed_elsewhere = grouped_path(&d, pb) || dw_path(&d, pb) || pw.grouped_wgrad || pw.grouped8_wgrad ||
+                                     pw.dw_wgrad || pw.dw_tma_wgrad;
+        const bool stem_ok = !stem_path(&d, pb) ||
+                             (stem_window_eligible(pb) && stem_window_dgrad_eligible(pb) && pw.stem_win_wgrad);
+        if (d.layout != CONVBN_NHWC || typed_elsewhere || !stem_ok) { status = CONVBN_EUNSUPPORTED; return; }
         set_call_f16(1);
         set_here = true;
     }
@@ -935,6 +936,9 @@ int convbn_eval_fwd(const convbn_desc *desc, const void *x, const void *w, const
                     const float *gamma, const float *beta, const float *run_mean,
                     const float *run_var, void *z, void *y_saved, void *workspace,
                     size_t workspace_bytes, void *stream) {
+    HalfCall half(desc);
+    if (half.status != CONVBN_OK) return half.status;
+    desc = half.use;
     Problem pb;
     t_prof_phase = "eval_fwd";
     CK(make_problem(desc, &pb));
@@ -960,6 +964,9 @@ int convbn_eval_bwd(const convbn_desc *desc, const void *dz, const void *x, cons
                     const void *w, const float *gamma, const float *run_mean, const float *run_var,
                     void *dx, float *dw, float *db, float *dgamma, float *dbeta, void *workspace,
                     size_t workspace_bytes, void *stream) {
+    HalfCall half(desc);
+    if (half.status != CONVBN_OK) return half.status;
+    desc = half.use;
     Problem pb;
     t_prof_phase = "eval_bwd";
     CK(make_problem(desc, &pb));
@@ -995,6 +1002,9 @@ int convbn_eval_bwd(const convbn_desc *desc, const void *dz, const void *x, cons
 int convbn_deploy_prepare(const convbn_desc *desc, const void *w, const float *b, const float *gamma,
                           const float *beta, const float *run_mean, const float *run_var,
                           void *w_fused, float *b_fused, void *stream) {
+    HalfCall half(desc);
+    if (half.status != CONVBN_OK) return half.status;
+    desc = half.use;
     Problem pb;
     t_prof_phase = "deploy_prepare";
     CK(make_problem(desc, &pb));
@@ -1012,6 +1022,9 @@ int convbn_deploy_prepare(const convbn_desc *desc, const void *w, const float *b
 int convbn_deploy_fwd(const convbn_desc *desc, const void *x, const void *w_fused,
                       const float *b_fused, void *z, void *workspace, size_t workspace_bytes,
                       void *stream) {
+    HalfCall half(desc);
+    if (half.status != CONVBN_OK) return half.status;
+    desc = half.use;
     Problem pb;
     t_prof_phase = "deploy_fwd";
     CK(make_problem(desc, &pb));
@@ -1029,6 +1042,9 @@ int convbn_deploy_fwd(const convbn_desc *desc, const void *x, const void *w_fuse
 int convbn_deploy_bwd(const convbn_desc *desc, const void *dz, const void *x, const void *w_fused,
                       void *dx, float *dw_fused, float *db_fused, void *workspace,
                       size_t workspace_bytes, void *stream) {
+    HalfCall half(desc);
+    if (half.status != CONVBN_OK) return half.status;
+    desc = half.use;
     Problem pb;
     t_prof_phase = "deploy_bwd";
     CK(make_problem(desc, &pb));
@@ -1102,11 +1118,24 @@ int tconv_view(const convbn_desc *d, TconvView *v) {
     return CONVBN_OK;
 }
 
+// An IEEE-half transposed layer runs as its bf16 twin: `twin` receives the descriptor to use from here on and
+// `inner` the convolution it transposes, typed half again, for HalfCall to check and to set the call's flag.
+int tconv_open(const convbn_desc *&desc, convbn_desc *twin, convbn_desc *inner, TconvView *v) {
+    if (!desc) return CONVBN_EINVAL;
+    const bool is_half = desc->dtype == CONVBN_F16;
+    if (is_half) { *twin = *desc; twin->dtype = CONVBN_BF16; desc = twin; }
+    CK(tconv_view(desc, v));
+    *inner = v->conv;
+    if (is_half) inner->dtype = CONVBN_F16;
+    return CONVBN_OK;
+}
+
 }  // namespace
 
 int convbn_tconv_out_shape(const convbn_desc *desc, int *h_out, int *w_out) {
     TconvView v;
-    CK(tconv_view(desc, &v));
+    convbn_desc twin, inner_desc;
+    CK(tconv_open(desc, &twin, &inner_desc, &v));
     if (!h_out || !w_out) return CONVBN_EINVAL;
     *h_out = v.h_out; *w_out = v.w_out;
     return CONVBN_OK;
@@ -1114,15 +1143,21 @@ int convbn_tconv_out_shape(const convbn_desc *desc, int *h_out, int *w_out) {
 
 size_t convbn_tconv_workspace_bytes(const convbn_desc *desc) {
     TconvView v;
-    return tconv_view(desc, &v) == CONVBN_OK ? v.total : 0;
+    convbn_desc twin, inner_desc;
+    if (tconv_open(desc, &twin, &inner_desc, &v) != CONVBN_OK) return 0;
+    HalfCall half(&inner_desc);
+    return half.status == CONVBN_OK ? v.total : 0;
 }
 
 int convbn_tconv_tune_fwd(const convbn_desc *desc, const void *x, const void *w, const float *b, const float *gamma,
                           const float *beta, const float *run_mean, const float *run_var, void *z, void *saved,
                           void *workspace, size_t workspace_bytes, void *stream) {
     TconvView v;
+    convbn_desc twin, inner_desc;
     t_prof_phase = "tconv_fwd";
-    CK(tconv_view(desc, &v));
+    CK(tconv_open(desc, &twin, &inner_desc, &v));
+    HalfCall half(&inner_desc);            // CONVBN_F16: the inner convolution's paths are checked, the half flag is set
+    if (half.status != CONVBN_OK) return half.status;
     if (!x || !w || !gamma || !beta || !run_mean || !run_var || !z || !saved) return CONVBN_EINVAL;
     if (!aligned(x, 16) || !aligned(w, 16) || !aligned(z, 16) || !aligned(saved, 16) || !aligned(b, 4) ||
         !aligned(gamma, 4) || !aligned(beta, 4) || !aligned(run_mean, 4) || !aligned(run_var, 4))
@@ -1153,8 +1188,11 @@ int convbn_tconv_tune_bwd(const convbn_desc *desc, const void *dz, const void *x
                           const float *run_mean, const void *saved, void *dx, float *dw, float *db, float *dgamma,
                           float *dbeta, void *workspace, size_t workspace_bytes, void *stream) {
     TconvView v;
+    convbn_desc twin, inner_desc;
     t_prof_phase = "tconv_bwd";
-    CK(tconv_view(desc, &v));
+    CK(tconv_open(desc, &twin, &inner_desc, &v));
+    HalfCall half(&inner_desc);
+    if (half.status != CONVBN_OK) return half.status;
     if (!dz || !x || !w || !run_mean || !saved || !dx || !dw || !dgamma || !dbeta) return CONVBN_EINVAL;
     if ((b == nullptr) != (db == nullptr)) return CONVBN_EINVAL;
     if (!aligned(dz, 16) || !aligned(x, 16) || !aligned(w, 16) || !aligned(saved, 16) || !aligned(dx, 16) ||
@@ -1256,6 +1294,9 @@ int convbn_profile_end(char *report, size_t report_bytes) {
 }
 
 size_t convbn_host_step_arena_bytes(const convbn_desc *desc) {
+    HalfCall half(desc);
+    if (half.status != CONVBN_OK) return 0;
+    desc = half.use;
     Problem pb;
     if (make_problem(desc, &pb) != CONVBN_OK) return 0;
     return make_host_arena(desc, pb).total;
@@ -1294,6 +1335,9 @@ int host_step_impl(const convbn_desc *desc, const void *x, const void *dz, const
                    const float *gamma, const float *beta, const float *run_mean, const float *run_var, void *z, void *dx,
                    float *dw, float *db, float *dgamma, float *dbeta, void *device_arena, size_t arena_bytes, void *stream,
                    bool defer_join) {
+    HalfCall half(desc);              // CONVBN_F16: the step runs as its bf16 twin with the half flag set
+    if (half.status != CONVBN_OK) return half.status;
+    desc = half.use;
     Problem pb;
     CK(make_problem(desc, &pb));
     CK(check_pair(desc));

@@ -123,6 +123,7 @@ __global__ void __launch_bounds__(256) direct_wgrad_kernel(Problem pb, const T *
 template <class F>
 static cudaError_t dispatch(int dtype, int layout, F f) {
     if (dtype == CONVBN_F32 && layout == CONVBN_NCHW) return f((float *)0, NCHW());
+    if (dtype == CONVBN_BF16 && layout == CONVBN_NHWC && call_f16()) return f((__half *)0, NHWC());   // a half call runs as its bf16 twin
     if (dtype == CONVBN_BF16 && layout == CONVBN_NHWC) return f((__nv_bfloat16 *)0, NHWC());
     return cudaErrorInvalidValue;
 }

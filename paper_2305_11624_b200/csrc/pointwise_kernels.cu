@@ -59,7 +59,7 @@ cudaError_t read_and_clear_error_word(int *host_value) {
 template <class F>
 static cudaError_t by_type(int dtype, F f) {
     if (dtype == CONVBN_F32) return f((float *)0);
-    if (dtype == CONVBN_BF16) return f((__nv_bfloat16 *)0);
+    if (dtype == CONVBN_BF16) return call_f16() ? f((__half *)0) : f((__nv_bfloat16 *)0);   // a half call runs as its bf16 twin
     return cudaErrorInvalidValue;
 }
 
@@ -258,9 +258,10 @@ __global__ void __launch_bounds__(256) channel_sum_partial_kernel(int c_out, int
     part[(long long)split * c_out + c] = acc;
 }
 
-// NHWC bf16 with C a multiple of 8: the tensor is a flat array of 16-byte vectors (8 channels);
-// the block size is a multiple of C/8, so a thread always sees the same 8 channels.  Per-thread
-// sums are combined per channel in thread order (fixed), one partial row per block.
+// NHWC, 16-bit elements (H: IEEE half, else bf16), C a multiple of 8: the tensor is a flat array of 16-byte
+// vectors (8 channels); the block size is a multiple of C/8, so a thread always sees the same 8 channels.
+// Per-thread sums are combined per channel in thread order (fixed), one partial row per block.
+template <bool H>
 __global__ void __launch_bounds__(256) channel_sum_nhwc8_kernel(int c_out, long long p, int pix_per_block,
                                                                 const uint4 *__restrict__ t,
                                                                 float *__restrict__ part) {
@@ -275,8 +276,10 @@ __global__ void __launch_bounds__(256) channel_sum_nhwc8_kernel(int c_out, long 
         const uint32_t u[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            acc[2 * e] += __uint_as_float(u[e] << 16);
-            acc[2 * e + 1] += __uint_as_float(u[e] & 0xFFFF0000u);
+            float lo, hi;
+            unpack2_t<H>(u[e], lo, hi);
+            acc[2 * e] += lo;
+            acc[2 * e + 1] += hi;
         }
     }
 #pragma unroll
@@ -312,7 +315,8 @@ cudaError_t launch_channel_sum_partial(const Problem &pb, int dtype, int layout,
         const int v = pb.c_out / 8;
         const int block = (256 / v) * v;
         const long long per = (pb.p + splits - 1) / splits;
-        channel_sum_nhwc8_kernel<<<splits, block, 0, st>>>(pb.c_out, pb.p, (int)per, (const uint4 *)t, part);
+        if (call_f16()) channel_sum_nhwc8_kernel<true><<<splits, block, 0, st>>>(pb.c_out, pb.p, (int)per, (const uint4 *)t, part);
+        else channel_sum_nhwc8_kernel<false><<<splits, block, 0, st>>>(pb.c_out, pb.p, (int)per, (const uint4 *)t, part);
         return cudaGetLastError();
     }
     const int threads = pb.c_out >= 256 ? 256 : ((pb.c_out + 31) / 32) * 32;
@@ -320,6 +324,9 @@ cudaError_t launch_channel_sum_partial(const Problem &pb, int dtype, int layout,
     if (dtype == CONVBN_F32 && layout == CONVBN_NCHW)
         channel_sum_partial_kernel<float, NCHW><<<grid, threads, 0, st>>>(
             pb.c_out, pb.h_out, pb.w_out, pb.p, (const float *)t, part, splits);
+    else if (dtype == CONVBN_BF16 && layout == CONVBN_NHWC && call_f16())
+        channel_sum_partial_kernel<__half, NHWC><<<grid, threads, 0, st>>>(
+            pb.c_out, pb.h_out, pb.w_out, pb.p, (const __half *)t, part, splits);
     else if (dtype == CONVBN_BF16 && layout == CONVBN_NHWC)
         channel_sum_partial_kernel<__nv_bfloat16, NHWC><<<grid, threads, 0, st>>>(
             pb.c_out, pb.h_out, pb.w_out, pb.p, (const __nv_bfloat16 *)t, part, splits);
@@ -405,8 +412,9 @@ __global__ void __launch_bounds__(256) bn_eval_fwd_kernel(int c_out, long long h
     }
 }
 
-// bf16 NHWC with C a multiple of 8: 16-byte vectors; the block size is a multiple of C / 8, so a thread
-// keeps its 8 channels (and their scale / shift in registers) over its grid-stride loop.
+// 16-bit NHWC (H: IEEE half, else bf16) with C a multiple of 8: 16-byte vectors; the block size is a multiple of
+// C / 8, so a thread keeps its 8 channels (and their scale / shift in registers) over its grid-stride loop.
+template <bool H>
 __global__ void __launch_bounds__(256) bn_eval_fwd_nhwc8_kernel(int c_out, long long vecs, const uint4 *__restrict__ y,
                                                                 const float *__restrict__ vec3,
                                                                 uint4 *__restrict__ z) {
@@ -421,10 +429,9 @@ __global__ void __launch_bounds__(256) bn_eval_fwd_nhwc8_kernel(int c_out, long 
         uint32_t o[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            const float a = fmaf(sc[2 * e], __uint_as_float(u[e] << 16), sh[2 * e]);
-            const float b2 = fmaf(sc[2 * e + 1], __uint_as_float(u[e] & 0xFFFF0000u), sh[2 * e + 1]);
-            const __nv_bfloat162 h = __floats2bfloat162_rn(a, b2);
-            o[e] = *(const uint32_t *)&h;
+            float lo, hi;
+            unpack2_t<H>(u[e], lo, hi);
+            o[e] = pack2_t<H>(fmaf(sc[2 * e], lo, sh[2 * e]), fmaf(sc[2 * e + 1], hi, sh[2 * e + 1]));
         }
         z[i] = make_uint4(o[0], o[1], o[2], o[3]);
     }
@@ -432,6 +439,7 @@ __global__ void __launch_bounds__(256) bn_eval_fwd_nhwc8_kernel(int c_out, long 
 
 // dy = s dz and per-block partial sums of dz (y - mean) r and dz, one partial row per block
 // (Table 2, Eval row); layout and block shape as above, lanes combined per channel in thread order.
+template <bool H>
 __global__ void __launch_bounds__(256) bn_eval_bwd_nhwc8_kernel(int c_out, long long p, int pix_per_block, float eps,
                                                                 const uint4 *__restrict__ dz,
                                                                 const uint4 *__restrict__ y,
@@ -460,14 +468,14 @@ __global__ void __launch_bounds__(256) bn_eval_bwd_nhwc8_kernel(int c_out, long 
         uint32_t o[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            const float d0 = __uint_as_float(ud[e] << 16), d1 = __uint_as_float(ud[e] & 0xFFFF0000u);
-            const float y0 = __uint_as_float(uy[e] << 16), y1 = __uint_as_float(uy[e] & 0xFFFF0000u);
+            float d0, d1, y0, y1;
+            unpack2_t<H>(ud[e], d0, d1);
+            unpack2_t<H>(uy[e], y0, y1);
             ag[2 * e] = fmaf(d0, (y0 - m8[2 * e]) * r8[2 * e], ag[2 * e]);
             ag[2 * e + 1] = fmaf(d1, (y1 - m8[2 * e + 1]) * r8[2 * e + 1], ag[2 * e + 1]);
             ab[2 * e] += d0;
             ab[2 * e + 1] += d1;
-            const __nv_bfloat162 h = __floats2bfloat162_rn(s8[2 * e] * d0, s8[2 * e + 1] * d1);
-            o[e] = *(const uint32_t *)&h;
+            o[e] = pack2_t<H>(s8[2 * e] * d0, s8[2 * e + 1] * d1);
         }
         dy[i] = make_uint4(o[0], o[1], o[2], o[3]);
     }
@@ -492,7 +500,8 @@ cudaError_t launch_bn_eval_fwd(const Problem &pb, int dtype, int layout, const v
         const long long vecs = pb.p * v;
         long long nb = (vecs + block - 1) / block;
         if (nb > device_sm_count() * 16) nb = device_sm_count() * 16;
-        bn_eval_fwd_nhwc8_kernel<<<(int)nb, block, 0, st>>>(pb.c_out, vecs, (const uint4 *)y, vec3, (uint4 *)z);
+        if (call_f16()) bn_eval_fwd_nhwc8_kernel<true><<<(int)nb, block, 0, st>>>(pb.c_out, vecs, (const uint4 *)y, vec3, (uint4 *)z);
+        else bn_eval_fwd_nhwc8_kernel<false><<<(int)nb, block, 0, st>>>(pb.c_out, vecs, (const uint4 *)y, vec3, (uint4 *)z);
         return cudaGetLastError();
     }
     const long long total = pb.p * pb.c_out, hw = (long long)pb.h_out * pb.w_out;
@@ -500,6 +509,8 @@ cudaError_t launch_bn_eval_fwd(const Problem &pb, int dtype, int layout, const v
     if (blocks > device_sm_count() * 32) blocks = device_sm_count() * 32;
     if (dtype == CONVBN_F32 && layout == CONVBN_NCHW)
         bn_eval_fwd_kernel<float, NCHW><<<(int)blocks, 256, 0, st>>>(pb.c_out, hw, total, (const float *)y, vec3, (float *)z);
+    else if (dtype == CONVBN_BF16 && layout == CONVBN_NHWC && call_f16())
+        bn_eval_fwd_kernel<__half, NHWC><<<(int)blocks, 256, 0, st>>>(pb.c_out, hw, total, (const __half *)y, vec3, (__half *)z);
     else if (dtype == CONVBN_BF16 && layout == CONVBN_NHWC)
         bn_eval_fwd_kernel<__nv_bfloat16, NHWC><<<(int)blocks, 256, 0, st>>>(
             pb.c_out, hw, total, (const __nv_bfloat16 *)y, vec3, (__nv_bfloat16 *)z);
@@ -544,9 +555,12 @@ cudaError_t launch_bn_eval_bwd(const Problem &pb, int dtype, int layout, const v
     if (channel_sum_fast(pb, dtype, layout)) {
         const int v = pb.c_out / 8, block = (256 / v) * v;
         const long long per = (pb.p + splits - 1) / splits;
-        bn_eval_bwd_nhwc8_kernel<<<splits, block, 0, st>>>(pb.c_out, pb.p, (int)per, pb.eps, (const uint4 *)dz,
-                                                           (const uint4 *)y, gamma, mean, var, (uint4 *)dy, part_g,
-                                                           part_b);
+        if (call_f16())
+            bn_eval_bwd_nhwc8_kernel<true><<<splits, block, 0, st>>>(pb.c_out, pb.p, (int)per, pb.eps, (const uint4 *)dz,
+                                                                     (const uint4 *)y, gamma, mean, var, (uint4 *)dy, part_g, part_b);
+        else
+            bn_eval_bwd_nhwc8_kernel<false><<<splits, block, 0, st>>>(pb.c_out, pb.p, (int)per, pb.eps, (const uint4 *)dz,
+                                                                      (const uint4 *)y, gamma, mean, var, (uint4 *)dy, part_g, part_b);
         return cudaGetLastError();
     }
     const int threads = pb.c_out >= 256 ? 256 : ((pb.c_out + 31) / 32) * 32;
@@ -555,6 +569,10 @@ cudaError_t launch_bn_eval_bwd(const Problem &pb, int dtype, int layout, const v
         bn_eval_bwd_kernel<float, NCHW><<<grid, threads, 0, st>>>(
             pb.c_out, pb.h_out, pb.w_out, pb.p, pb.eps, (const float *)dz, (const float *)y, gamma, mean,
             var, (float *)dy, part_g, part_b, splits);
+    else if (dtype == CONVBN_BF16 && layout == CONVBN_NHWC && call_f16())
+        bn_eval_bwd_kernel<__half, NHWC><<<grid, threads, 0, st>>>(
+            pb.c_out, pb.h_out, pb.w_out, pb.p, pb.eps, (const __half *)dz, (const __half *)y, gamma, mean, var,
+            (__half *)dy, part_g, part_b, splits);
     else if (dtype == CONVBN_BF16 && layout == CONVBN_NHWC)
         bn_eval_bwd_kernel<__nv_bfloat16, NHWC><<<grid, threads, 0, st>>>(
             pb.c_out, pb.h_out, pb.w_out, pb.p, pb.eps, (const __nv_bfloat16 *)dz,

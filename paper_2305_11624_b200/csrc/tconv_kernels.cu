@@ -109,6 +109,9 @@ cudaError_t launch_tconv_vec3(int c_out, float eps, const float *b, const float 
 
 cudaError_t launch_tconv_rescale(int dtype, bool nhwc, long long count, int taps, int cig, int cog, const void *w,
                                  const float *s, void *w_out, cudaStream_t st) {
+    if (dtype == CONVBN_BF16 && call_f16())     // a half call runs as its bf16 twin
+        return launch_pdl(tconv_rescale_kernel<__half>, dim3(grid_for(count)), dim3(256), 0, st, count, taps, cig, cog, nhwc,
+                          (const __half *)w, s, (__half *)w_out);
     if (dtype == CONVBN_BF16)
         return launch_pdl(tconv_rescale_kernel<__nv_bfloat16>, dim3(grid_for(count)), dim3(256), 0, st, count, taps, cig, cog,
                           nhwc, (const __nv_bfloat16 *)w, s, (__nv_bfloat16 *)w_out);
@@ -118,6 +121,8 @@ cudaError_t launch_tconv_rescale(int dtype, bool nhwc, long long count, int taps
 
 cudaError_t launch_tconv_bias(int dtype, bool nhwc, long long count, int c, long long hw, const float *bias, void *z,
                               cudaStream_t st) {
+    if (dtype == CONVBN_BF16 && call_f16())
+        return launch_pdl(tconv_bias_kernel<__half>, dim3(grid_for(count)), dim3(256), 0, st, count, c, hw, nhwc, bias, (__half *)z);
     if (dtype == CONVBN_BF16)
         return launch_pdl(tconv_bias_kernel<__nv_bfloat16>, dim3(grid_for(count)), dim3(256), 0, st, count, c, hw, nhwc, bias,
                           (__nv_bfloat16 *)z);
@@ -129,6 +134,9 @@ cudaError_t launch_tconv_param_epilogue(int dtype, bool nhwc, int c_out, int tap
                                         const float *bsum, int bsplits, float *dw, float *db, float *dgamma,
                                         float *dbeta, cudaStream_t st) {
     const dim3 grid((c_out + 31) / 32);
+    if (dtype == CONVBN_BF16 && call_f16())
+        return launch_pdl(tconv_param_epilogue_kernel<__half>, grid, dim3(256), 0, st, c_out, taps, cig, cog, nhwc, dwp,
+                          (const __half *)w, vec3, b, mean, bsum, bsplits, dw, db, dgamma, dbeta);
     if (dtype == CONVBN_BF16)
         return launch_pdl(tconv_param_epilogue_kernel<__nv_bfloat16>, grid, dim3(256), 0, st, c_out, taps, cig, cog, nhwc, dwp,
                           (const __nv_bfloat16 *)w, vec3, b, mean, bsum, bsplits, dw, db, dgamma, dbeta);

@@ -34,8 +34,10 @@ BODY = resnet50_plan(64)[1]        # all 16 bottlenecks of a ResNet-50 on 64 x 6
 
 
 @pytest.mark.parametrize("mode,plan,dtype", [("tune", PLAN, "bf16"), ("eval", PLAN, "bf16"), ("deploy", PLAN, "bf16"),
-                                             ("tune", BODY, "bf16"), ("tune", PLAN, "f16"), ("tune", BODY, "f16")],
-                         ids=["tune", "eval", "deploy", "tune_whole_body", "tune_half", "tune_whole_body_half"])
+                                             ("tune", BODY, "bf16"), ("tune", PLAN, "f16"), ("tune", BODY, "f16"),
+                                             ("eval", PLAN, "f16"), ("deploy", PLAN, "f16")],
+                         ids=["tune", "eval", "deploy", "tune_whole_body", "tune_half", "tune_whole_body_half",
+                              "eval_half", "deploy_half"])
 def test_three_bottlenecks_against_the_chained_oracle(mode, plan, dtype):
     """The three modes compute one function with one set of input gradients (Sec. 3.3), so one oracle chain - the
     Tune formulas - checks all of them; Deploy's parameter gradients belong to the folded parameters and are left

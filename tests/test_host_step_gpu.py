@@ -12,6 +12,7 @@ SPECS = [
     I.LayerSpec("h_3x3", 2, 64, 18, 20, 128, 3, 3, pad=1),
     I.LayerSpec("h_bias_f32", 2, 8, 9, 7, 12, 3, 3, pad=1, dtype="f32", layout="nchw", bias=True),
     I.LayerSpec("h_dw", 1, 32, 13, 17, 32, 3, 3, pad=1, groups=32),
+    I.LayerSpec("h_half_1x1", 2, 256, 20, 20, 64, 1, 1, dtype="f16", bias=True),
 ]
 
 

@@ -53,7 +53,8 @@ def test_linear_gradients_match_finite_differences():
 
 @pytest.mark.gpu
 @pytest.mark.parametrize("rows,cin,cout,dtype,bias", [(777, 256, 64, "bf16", False), (1000, 64, 256, "bf16", False),
-                                                      (300, 512, 192, "bf16", True), (37, 24, 10, "f32", True)])
+                                                      (300, 512, 192, "bf16", True), (37, 24, 10, "f32", True),
+                                                      (777, 256, 64, "f16", True), (37, 24, 10, "f16", False)])
 def test_linear_bn_on_the_device(rows, cin, cout, dtype, bias):
     import torch
     import parity
@@ -61,14 +62,15 @@ def test_linear_bn_on_the_device(rows, cin, cout, dtype, bias):
     from paper_2305_11624_b200 import inputs as I
     tol = parity.TOL[dtype]
     t = _draw(rows, cin, cout, bias)
-    rnd = I.round_bf16 if dtype == "bf16" else (lambda a: np.asarray(a, np.float32))
+    rnd = {"bf16": I.round_bf16, "f16": lambda a: np.asarray(a, np.float16).astype(np.float32),
+           "f32": lambda a: np.asarray(a, np.float32)}[dtype]
     dz = RNG.standard_normal((rows, cout))
     t["x"], t["w"], dz = (rnd(a.astype(np.float32)).astype(np.float64) for a in (t["x"], t["w"], dz))
     for k in ("b", "gamma", "beta", "mu_hat", "var_hat"):
         if t[k] is not None:
             t[k] = t[k].astype(np.float32).astype(np.float64)
-    desc = C.convbn_linear_desc(rows, cin, cout, C.BF16 if dtype == "bf16" else C.F32, 1e-5)
-    td = torch.bfloat16 if dtype == "bf16" else torch.float32
+    desc = C.convbn_linear_desc(rows, cin, cout, {"bf16": C.BF16, "f16": C.F16, "f32": C.F32}[dtype], 1e-5)
+    td = {"bf16": torch.bfloat16, "f16": torch.float16, "f32": torch.float32}[dtype]
     dev = lambda a, d=td: None if a is None else torch.tensor(np.asarray(a, np.float32), device="cuda").to(d).contiguous()
     x, w, dzd = dev(t["x"]), dev(t["w"]), dev(dz)
     vec = {k: dev(t[k], torch.float32) for k in ("b", "gamma", "beta", "mu_hat", "var_hat")}

@@ -147,7 +147,13 @@ def test_tune_is_deterministic_and_leaves_inputs_alone():
 
 COMPARATOR_SPECS = [SMALL[0], SMALL[8], SMALL[10], SMALL[17], SMALL[19]] + \
     [sp for sp in SMALL if sp.name in ("b_stem_3x3_s2", "b_sub_c4", "b_sub_wide")] + \
-    [I.find_layer(name)[2] for name in ("c1a", "c1b", "c1c", "c3c", "c4a")]       # benchmark layers at full size
+    [I.find_layer(name)[2] for name in ("c1a", "c1b", "c1c", "c3c", "c4a")] + \
+    [L("h_1x1_256_64", 2, 256, 28, 28, 64, 1, 1, dtype="f16"),                    # IEEE half in the three modes
+     L("h_3x3_128_256", 2, 128, 20, 36, 256, 3, 3, pad=1, dtype="f16", bias=True),
+     L("h_3x3_s2_128", 2, 128, 40, 42, 128, 3, 3, stride=2, pad=1, dtype="f16"),
+     L("h_stem", 2, 3, 64, 80, 64, 7, 7, stride=2, pad=3, dtype="f16"),
+     L("h_20_24", 2, 20, 11, 13, 24, 3, 3, stride=2, pad=1, dtype="f16", bias=True)]
+# (the benchmark layers run at full size)
 
 
 @pytest.mark.parametrize("spec", COMPARATOR_SPECS, ids=lambda s: s.name)

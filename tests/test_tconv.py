@@ -129,6 +129,9 @@ GPU_CASES = [  # (dtype, n, c_in, h, w, c_out, k, stride, pad, dil, groups, bias
     ("bf16", 2, 64, 30, 30, 128, 3, 1, 1, 1, 1, False),     # stride 1: the strip kernel on both passes
     ("bf16", 3, 64, 9, 11, 64, 3, 2, 1, 1, 2, True),        # two groups, ragged extent
     ("bf16", 1, 256, 56, 56, 128, 2, 2, 0, 1, 1, False),    # several tiles per CTA
+    ("f16", 2, 128, 28, 28, 64, 2, 2, 0, 1, 1, True),       # IEEE half: up-sampling, stride 1, and the direct kernels
+    ("f16", 2, 64, 30, 30, 128, 3, 1, 1, 1, 1, False),
+    ("f16", 2, 12, 9, 11, 20, 3, 2, 1, 1, 2, True),
 ]
 
 
@@ -139,9 +142,11 @@ def test_library_matches_the_oracle(case):
     from paper_2305_11624_b200 import convbn as C
     from paper_2305_11624_b200 import inputs as I
     dtype, n, ci, h, w, co, k, st, pad, dil, grp, bias = case
-    bf = dtype == "bf16"
+    bf = dtype in ("bf16", "f16")           # 16-bit storage, NHWC
     lay = "nhwc" if bf else "nchw"
-    rnd = (lambda a: I.round_bf16(a.astype(np.float32)).astype(np.float64)) if bf else (lambda a: a.astype(np.float32).astype(np.float64))
+    rnd = {"bf16": lambda a: I.round_bf16(a.astype(np.float32)).astype(np.float64),
+           "f16": lambda a: a.astype(np.float16).astype(np.float64),
+           "f32": lambda a: a.astype(np.float32).astype(np.float64)}[dtype]
     x = rnd(_rnd(1, n, ci, h, w))
     wt = rnd(_rnd(2, ci, co // grp, k, k) * np.sqrt(2.0 / (ci // grp * k * k)))
     ho, wo = T.out_hw(h, w, k, k, st, pad, dil)
@@ -154,9 +159,9 @@ def test_library_matches_the_oracle(case):
     ref.update(T.tune_backward(dz, x, wt, b, p["gamma"], p["mu_hat"], p["var_hat"], 1e-5, **kw))
 
     dev = "cuda:0"
-    tdt = torch.bfloat16 if bf else torch.float32
+    tdt = {"bf16": torch.bfloat16, "f16": torch.float16, "f32": torch.float32}[dtype]
     up = lambda a, dt=torch.float32: torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).reshape(-1).to(dt).to(dev)
-    desc = C.Desc.make(n, ci, h, w, co, k, k, st, st, pad, pad, dil, dil, grp, C.BF16 if bf else C.F32, C.NHWC if bf else C.NCHW, 1e-5)
+    desc = C.Desc.make(n, ci, h, w, co, k, k, st, st, pad, pad, dil, dil, grp, {"bf16": C.BF16, "f16": C.F16, "f32": C.F32}[dtype], C.NHWC if bf else C.NCHW, 1e-5)
     assert C.convbn_tconv_out_shape(desc) == (ho, wo)
     X, W, DZ = up(I.act_to_layout(x, lay), tdt), up(I.weight_to_layout(wt, lay), tdt), up(I.act_to_layout(dz, lay), tdt)
     G, Bt, M, V = (up(p[key]) for key in ("gamma", "beta", "mu_hat", "var_hat"))
