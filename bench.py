@@ -676,7 +676,7 @@ def run_backbone(ctx, batch=32, size=224, iters=10):
                             dtype="f16" if mode.endswith("_f16") else "bf16")
         try:
             ms, peak, how = rp.measure(iters=iters, warmup=3)
-        except ctx.C.ConvBNError as exc:       # half: the stem's window kernels take images up to 256 pixels wide
+        except ctx.C.ConvBNError as exc:       # a layer shape that has no half path
             if not mode.endswith("_f16") or exc.status != ctx.C.EUNSUPPORTED:
                 raise
             out["modes"][mode] = {"unsupported": str(exc)}

@@ -346,7 +346,7 @@ bool strided_dgrad_ok(const convbn_desc *d, const Problem &pb) {
 }
 
 // CONVBN_F16 calls.  IEEE half runs on every path of ungrouped NHWC layers whose kernels know the type: the dense
-// tensor-core kernels, the three window kernels of a stride-2 stem, the direct kernels and the element-wise ones.
+// tensor-core kernels, the window and packed kernels of the stems, the direct kernels and the element-wise ones.
 // The descriptor is checked for them, then the call proceeds as its bf16 twin with the half flag set for the
 // launchers (operand format of the MMAs, conversions of results and of rescaled weights, the constant 1, the
 // element type of the templated kernels).  The flag is cleared when the call returns.
@@ -364,12 +364,10 @@ struct HalfCall {
         status = make_problem(&d, &pb);
         if (status != CONVBN_OK) return;
         const Plan pw = make_plan(&d, pb, CONVBN_PHASE_TUNE_BWD_WEIGHT);
-        // depthwise and grouped kernels read bf16 only; so do the packed (non-window) stem kernels
+        // depthwise and grouped kernels read bf16 only
         const bool typed_elsewhere = grouped_path(&d, pb) || dw_path(&d, pb) || pw.grouped_wgrad || pw.grouped8_wgrad ||
                                      pw.dw_wgrad || pw.dw_tma_wgrad;
-        const bool stem_ok = !stem_path(&d, pb) ||
-                             (stem_window_eligible(pb) && stem_window_dgrad_eligible(pb) && pw.stem_win_wgrad);
-        if (d.layout != CONVBN_NHWC || typed_elsewhere || !stem_ok) { status = CONVBN_EUNSUPPORTED; return; }
+        if (d.layout != CONVBN_NHWC || typed_elsewhere) { status = CONVBN_EUNSUPPORTED; return; }
         set_call_f16(1);
         set_here = true;
     }
@@ -444,7 +442,8 @@ int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, cons
         LAUNCH("subpixel_weights", launch_subpixel_weights(pb, w, scale, w_scratch, st));
         LAUNCH("stem_dgrad", launch_umma_strip_conv(s, dz, w_scratch, nullptr, dx, st));
         *which = "umma-subpixel";
-    } else if (stem_path(d, pb) && stem_dgrad_eligible(pb)) {
+    } else if (stem_path(d, pb) && stem_dgrad_eligible(pb) && !call_f16()) {
+        // (warp-level bf16 MMAs: a half call takes the direct kernel below instead)
         LAUNCH("stem_dgrad", launch_stem_dgrad(pb, dz, w, scale, dx, st));
         *which = "stem-mma";
     } else if (grouped_path(d, pb) && grouped8_eligible(pb)) {

@@ -67,7 +67,7 @@ size_t stem_weight_bytes(const Problem &pb) { return (size_t)pb.c_out * stem_kro
 
 // xp[n][hp][wp][a][b][4] = x[n][2 I + a - pad_h][2 J + b - pad_w][c] inside the image, 0 elsewhere
 __global__ void __launch_bounds__(256) stem_pack_s2d_kernel(int n, int h_in, int w_in, int c_in, int pad_h, int pad_w,
-                                                            int hp, int wp, int ones,
+                                                            int hp, int wp, int ones, int f16,
                                                             const __nv_bfloat16 *__restrict__ x,
                                                             uint4 *__restrict__ xp) {
     const long long total = (long long)n * hp * wp * 2;          // one thread per (packed pixel, a)
@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(256) stem_pack_s2d_kernel(int n, int h_in, int
         const int hq = (int)(t % hp), img = (int)(t / hp);
         const int h = 2 * hq + a - pad_h;
         unsigned short v[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        if (ones && a == 0) v[3] = 0x3F80;                       // bf16 1.0 in slot (0, 0, 3), border included
+        if (ones && a == 0) v[3] = (unsigned short)one_h16(f16);   // 1.0 in slot (0, 0, 3), border included
         if (h >= 0 && h < h_in) {
 #pragma unroll
             for (int b = 0; b < 2; ++b) {
@@ -129,7 +129,7 @@ cudaError_t launch_stem_pack(const Problem &pb, const void *x, void *xp, cudaStr
     if (blocks > device_sm_count() * 16) blocks = device_sm_count() * 16;
     if (stem_s2d(pb)) {
         stem_pack_s2d_kernel<<<(int)blocks, 256, 0, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.pad_h, pb.pad_w, hp, wp,
-                                                          stem_ones_in_pack(pb) ? 1 : 0, (const __nv_bfloat16 *)x,
+                                                          stem_ones_in_pack(pb) ? 1 : 0, call_f16(), (const __nv_bfloat16 *)x,
                                                           (uint4 *)xp);
         return cudaGetLastError();
     }
@@ -143,7 +143,7 @@ cudaError_t launch_stem_pack(const Problem &pb, const void *x, void *xp, cudaStr
 __global__ void __launch_bounds__(256) stem_expand_weights_kernel(int c_out, int kh, int kw, int c_in, int krows,
                                                                   int s2d, const __nv_bfloat16 *__restrict__ w,
                                                                   const float *__restrict__ s_vec,
-                                                                  __nv_bfloat16 *__restrict__ wst) {
+                                                                  __nv_bfloat16 *__restrict__ wst, int f16) {
     const int total = c_out * krows * 64;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
         const int j = i & 63, kr = (i >> 6) % krows, co = (i >> 6) / krows;
@@ -151,8 +151,8 @@ __global__ void __launch_bounds__(256) stem_expand_weights_kernel(int c_out, int
         const int q = s2d ? 2 * (j >> 4) + ((j >> 2) & 1) : j >> 3, c = s2d ? (j & 3) : (j & 7);
         float v = 0.f;
         if (r < kh && q < kw && c < c_in)
-            v = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[(((long long)co * kh + r) * kw + q) * c_in + c]);
-        wst[i] = __float2bfloat16_rn(v);
+            v = (s_vec ? s_vec[co] : 1.f) * load_h16(w + (((long long)co * kh + r) * kw + q) * c_in + c, f16);
+        reinterpret_cast<uint16_t *>(wst)[i] = pack1_h16(v, f16);
     }
 }
 
@@ -161,7 +161,7 @@ cudaError_t launch_stem_expand_weights(const Problem &pb, const void *w, const f
     const int total = pb.c_out * stem_krows(pb) * 64;
     stem_expand_weights_kernel<<<(total + 255) / 256, 256, 0, st>>>(pb.c_out, pb.kh, pb.kw, pb.c_in, stem_krows(pb),
                                                                     stem_s2d(pb) ? 1 : 0, (const __nv_bfloat16 *)w, s_vec,
-                                                                    (__nv_bfloat16 *)wst);
+                                                                    (__nv_bfloat16 *)wst, call_f16());
     return cudaGetLastError();
 }
 

@@ -581,7 +581,7 @@ cudaError_t launch_stem_fwd(const Problem &pb, const void *x_packed, const void 
     g.stem_tiles_w = (pb.w_out + 15) / 16; g.stem_tiles_h = (pb.h_out + 7) / 8;
     g.p = (long long)pb.n * g.stem_tiles_h * g.stem_tiles_w * kBM;      // m-tiles x 128 (patches, ragged edges clipped)
     g.stages = 1; g.blockdiag = 0; g.out_strided = nullptr; g.out_sn = 0; g.out_sh = g.out_sw = 0;
-    g.f16 = 0;                      // the packed-stem path is bf16 only
+    g.f16 = call_f16();
     g.fold = fold ? *fold : BnFold{nullptr, nullptr, nullptr, nullptr, nullptr, 0.f, nullptr};
     CUtensorMap ta, tw, tout;
     {   // overlapping windows: 64 elements (8 pixels x 8 channels) starting at every output column

@@ -350,11 +350,10 @@ __global__ void __launch_bounds__(kSThreads) umma_strip_conv_kernel(const __grid
                                 for (int e = 0; e < 8; e += 2) {
                                     const float f0 = __uint_as_float(vv[a2 * 8 + e]), f1 = __uint_as_float(vv[a2 * 8 + e + 1]);
                                     if (pairs && e + 1 < lim) {
-                                        const __nv_bfloat162 hh2 = __floats2bfloat162_rn(f0, f1);
-                                        *(__nv_bfloat162 *)(dst + e) = hh2;
+                                        *(uint32_t *)(dst + e) = pack2_h16(f0, f1, g.f16);
                                     } else {
-                                        if (e < lim) dst[e] = __float2bfloat16_rn(f0);
-                                        if (e + 1 < lim) dst[e + 1] = __float2bfloat16_rn(f1);
+                                        if (e < lim) reinterpret_cast<uint16_t *>(dst)[e] = pack1_h16(f0, g.f16);
+                                        if (e + 1 < lim) reinterpret_cast<uint16_t *>(dst)[e + 1] = pack1_h16(f1, g.f16);
                                     }
                                 }
                             }
@@ -631,7 +630,7 @@ void subpixel_range(int pad, int k, int *dmin, int *dmax) {
 
 __global__ void subpixel_weights_kernel(const __nv_bfloat16 *__restrict__ w, const float *__restrict__ s_vec,
                                         __nv_bfloat16 *__restrict__ wsub, int c_out, int cin, int kh, int kw,
-                                        int pad_h, int pad_w, int th, int tw, int dmin_h, int dmin_w) {
+                                        int pad_h, int pad_w, int th, int tw, int dmin_h, int dmin_w, int f16) {
     pdl_wait();
     pdl_launch_dependents();
     const int total = 16 * th * tw * c_out;
@@ -644,8 +643,8 @@ __global__ void subpixel_weights_kernel(const __nv_bfloat16 *__restrict__ w, con
         const int r = a + pad_h - 2 * (dmin_h + tr), q = b + pad_w - 2 * (dmin_w + tq);
         float v = 0.f;
         if (b < 2 && r >= 0 && r < kh && q >= 0 && q < kw)
-            v = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[(((size_t)co * kh + r) * kw + q) * cin + ci]);
-        wsub[idx] = __float2bfloat16_rn(v);
+            v = (s_vec ? s_vec[co] : 1.f) * load_h16(w + (((size_t)co * kh + r) * kw + q) * cin + ci, f16);
+        reinterpret_cast<uint16_t *>(wsub)[idx] = pack1_h16(v, f16);
     }
 }
 
@@ -733,7 +732,7 @@ cudaError_t launch_subpixel_weights(const Problem &pb, const void *w, const floa
     const int total = 16 * s.taps_h * s.taps_w * pb.c_out;
     return launch_pdl(subpixel_weights_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st,
                       (const __nv_bfloat16 *)w, s_vec, (__nv_bfloat16 *)wsub, pb.c_out, pb.c_in, pb.kh, pb.kw,
-                      pb.pad_h, pb.pad_w, s.taps_h, s.taps_w, s.lower_h, s.lower_w);
+                      pb.pad_h, pb.pad_w, s.taps_h, s.taps_w, s.lower_h, s.lower_w, call_f16());
 }
 
 }  // namespace convbn

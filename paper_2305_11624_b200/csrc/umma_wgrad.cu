@@ -544,7 +544,7 @@ cudaError_t launch_stem_wgrad(const Problem &pb, const UmmaWgradPlan &pl, const 
     g.kdim = krows * 64;
     g.stem = 1; g.stem_tiles_w = (pb.w_out + 15) / 16; g.stem_tiles_h = (pb.h_out + 3) / 4;
     g.no_ones = stem_ones_in_pack(pb) ? 1 : 0;
-    g.f16 = 0;                      // the packed-stem path is bf16 only
+    g.f16 = call_f16();
     g.p = (long long)pb.n * g.stem_tiles_h * g.stem_tiles_w * kWP;
     g.per_split = pl.per_split; g.stages = 1; g.blockdiag = 0;
     CUtensorMap tx, tdz;
@@ -588,7 +588,7 @@ __global__ void __launch_bounds__(256) wgrad_epilogue_stem_kernel(int c_out, int
                                                                  const float *__restrict__ mean,
                                                                  float *__restrict__ dw, float *__restrict__ db,
                                                                  float *__restrict__ dgamma,
-                                                                 float *__restrict__ dbeta, int need_sums) {
+                                                                 float *__restrict__ dbeta, int need_sums, int f16) {
     __shared__ float red[256];
     const int co = blockIdx.x, kdim = kh * kw * c_in;
     const size_t slice = (size_t)krows * 64 * c_out;
@@ -601,7 +601,7 @@ __global__ void __launch_bounds__(256) wgrad_epilogue_stem_kernel(int c_out, int
         float acc = 0.f;
         for (int sp = 0; sp < splits; ++sp) acc += part[(size_t)sp * slice + o];
         dw[(size_t)co * kdim + k] = s * acc;
-        if (vec3) dot = fmaf(acc, __bfloat162float(w[(size_t)co * kdim + k]), dot);
+        if (vec3) dot = fmaf(acc, load_h16(w + (size_t)co * kdim + k, f16), dot);
     }
     float bs = 0.f;
     if (need_sums)
@@ -635,7 +635,7 @@ cudaError_t launch_wgrad_epilogue_stem(const Problem &pb, const UmmaWgradPlan &p
     wgrad_epilogue_stem_kernel<<<pb.c_out, 256, 0, st>>>(pb.c_out, pb.kh, pb.kw, pb.c_in, stem_krows(pb), stem_s2d(pb) ? 1 : 0,
                                                          stem_ones_in_pack(pb) ? 3 : -1, partials, pl.splits, bsum,
                                                          (const __nv_bfloat16 *)w, vec3, b, mean, dw, db, dgamma, dbeta,
-                                                         need_sums ? 1 : 0);
+                                                         need_sums ? 1 : 0, call_f16());
     return cudaGetLastError();
 }
 

@@ -152,6 +152,7 @@ COMPARATOR_SPECS = [SMALL[0], SMALL[8], SMALL[10], SMALL[17], SMALL[19]] + \
      L("h_3x3_128_256", 2, 128, 20, 36, 256, 3, 3, pad=1, dtype="f16", bias=True),
      L("h_3x3_s2_128", 2, 128, 40, 42, 128, 3, 3, stride=2, pad=1, dtype="f16"),
      L("h_stem", 2, 3, 64, 80, 64, 7, 7, stride=2, pad=3, dtype="f16"),
+     L("h_stem_w272", 2, 3, 8, 272, 64, 7, 7, stride=2, pad=3, dtype="f16", bias=True),
      L("h_20_24", 2, 20, 11, 13, 24, 3, 3, stride=2, pad=1, dtype="f16", bias=True)]
 # (the benchmark layers run at full size)
 
