@@ -77,7 +77,10 @@ typedef enum {
 } convbn_phase;
 
 /* Problem description (paper Sec. 3.1 and the shape annotations of Appendix C; stride, padding,
- * dilation and groups as in the convention above).  Plain data, read on the host. */
+ * dilation and groups as in the convention above).  Plain data, read on the host.
+ * Largest problems: X and Z at most 2^40 elements each, C_in / groups * kh * kw at most 2^30, padded input extents
+ * (h_in + 2 pad_h, w_in + 2 pad_w) and filter spans (dil (k - 1)) at most 2^30; beyond that every entry point
+ * returns CONVBN_EINVAL (the size queries 0). */
 typedef struct convbn_desc {
     int n, c_in, h_in, w_in;   /* X is [N, C_in, H_in, W_in] logically                  */
     int c_out, kh, kw;         /* omega is [C_out, C_in/groups, kh, kw] logically        */

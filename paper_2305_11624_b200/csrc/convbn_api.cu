@@ -67,6 +67,10 @@ int make_problem(const convbn_desc *d, Problem *pb) {
     const long long eh = (long long)d->h_in + 2LL * d->pad_h - (long long)d->dil_h * (d->kh - 1) - 1;
     const long long ew = (long long)d->w_in + 2LL * d->pad_w - (long long)d->dil_w * (d->kw - 1) - 1;
     if (eh < 0 || ew < 0) return CONVBN_EINVAL;
+    // padded extents and filter spans stay inside 2^30, so that every row and column index fits an int
+    if ((long long)d->h_in + 2LL * d->pad_h > (1LL << 30) || (long long)d->w_in + 2LL * d->pad_w > (1LL << 30) ||
+        (long long)d->dil_h * (d->kh - 1) > (1LL << 30) || (long long)d->dil_w * (d->kw - 1) > (1LL << 30))
+        return CONVBN_EINVAL;
     if (d->dtype != CONVBN_F32 && d->dtype != CONVBN_BF16 && d->dtype != CONVBN_F16) return CONVBN_EINVAL;
     if (d->layout != CONVBN_NCHW && d->layout != CONVBN_NHWC) return CONVBN_EINVAL;
     pb->n = d->n; pb->c_in = d->c_in; pb->h_in = d->h_in; pb->w_in = d->w_in;

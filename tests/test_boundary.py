@@ -84,6 +84,31 @@ def test_bad_descriptors_are_rejected_on_the_host(kw):
     assert e.value.status == C.EINVAL
 
 
+def test_largest_problems():
+    """The documented size limits: 2^40 elements per tensor, 2^30 weights per output channel.  One element below is
+    accepted (sizes come back, nothing overflows into a small or negative number), one above is CONVBN_EINVAL."""
+    ho, wo = ctypes.c_int(), ctypes.c_int()
+    shape = lambda d: C.lib().convbn_out_shape(ctypes.byref(d), ctypes.byref(ho), ctypes.byref(wo))
+    one = dict(kh=1, kw=1, pad_h=0, pad_w=0, dtype=C.BF16, layout=C.NHWC)
+    # 2^40 activation elements exactly: 2^15 images of 2^7 x 2^8 pixels and 2^10 channels
+    at_limit = good(n=1 << 15, c_in=1 << 10, h_in=1 << 7, w_in=1 << 8, c_out=1 << 10, **one)
+    assert shape(at_limit) == C.OK and (ho.value, wo.value) == (1 << 7, 1 << 8)
+    assert C.convbn_saved_bytes(at_limit, C.MODE_EVAL) == 2 << 40
+    assert C.convbn_saved_bytes(at_limit, C.MODE_TUNE) == 3 * 4 * (1 << 10)
+    for ph in (C.PHASE_TUNE_FWD, C.PHASE_TUNE_BWD, C.PHASE_EVAL_BWD):
+        ws = C.convbn_workspace_bytes(at_limit, ph)
+        assert 0 < ws < 3 << 40 and ws % 256 == 0, (ph, ws)      # Eval backward holds dY, a tensor of the size of Z
+    assert shape(good(n=(1 << 15) + 1, c_in=1 << 10, h_in=1 << 7, w_in=1 << 8, c_out=1 << 10, **one)) == C.EINVAL   # input
+    assert shape(good(n=(1 << 15) + 1, c_in=8, h_in=1 << 7, w_in=1 << 8, c_out=1 << 10, **one)) == C.EINVAL         # output
+    # weights per output channel: C_in kh kw <= 2^30
+    wide = dict(n=1, h_in=64, w_in=64, c_out=8, pad_h=0, pad_w=0, dtype=C.BF16, layout=C.NHWC)
+    assert shape(good(c_in=1 << 18, kh=64, kw=64, **wide)) == C.OK and (ho.value, wo.value) == (1, 1)
+    assert shape(good(c_in=(1 << 18) + 8, kh=64, kw=64, **wide)) == C.EINVAL
+    # extents that no int holds are rejected, not wrapped
+    assert shape(good(n=1, c_in=1, h_in=(1 << 31) - 1, w_in=(1 << 31) - 1, c_out=1, **one)) == C.EINVAL
+    assert shape(good(h_in=16, w_in=16, pad_h=(1 << 31) - 1, pad_w=1)) == C.EINVAL
+
+
 def test_argument_checks_before_any_launch():
     d = good()
     ws = C.convbn_workspace_bytes(d, C.PHASE_TUNE_FWD)
