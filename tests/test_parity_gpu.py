@@ -110,6 +110,32 @@ def test_tune_small(spec):
         assert got["_kernels"] == EXPECTED_PATH[spec.name], got["_kernels"]
 
 
+DEGENERATE = [sp for sp in SMALL if sp.name in ("f32_bias", "b_1x1_a", "b_3x3_a", "b_bias", "b_odd_c", "b_dw", "b_grouped",
+                                               "b_win_c3", "b_sub_wide")] + \
+    [L("h_3x3_64", 2, 64, 30, 30, 64, 3, 3, pad=1, dtype="f16", bias=True)]
+
+
+@pytest.mark.parametrize("spec", DEGENERATE, ids=lambda s: s.name)
+def test_degenerate_statistics_and_affine_parameters(spec):
+    """The cases the rewrite itself can degenerate in (Sec. 3.3 definitions): gamma = 0 (the channel's omega' vanishes, its
+    output is the constant b', its domega is zero while dgamma is not), negative gamma, a running variance of exactly
+    zero (s = gamma / sqrt(eps), some 300 times larger than elsewhere) and a large one, a large running mean."""
+    t = parity.make_inputs(spec, 4242)
+    c = spec.c_out
+    idx = np.arange(c)
+    t["gamma"] = np.where(idx % 4 == 0, 0.0, np.where(idx % 4 == 1, -t["gamma"], t["gamma"])).astype(np.float32).astype(np.float64)
+    t["var_hat"] = np.where(idx % 8 == 2, 0.0, np.where(idx % 8 == 3, 4096.0, t["var_hat"]))
+    t["mu_hat"] = np.where(idx % 8 == 5, 37.5, t["mu_hat"])
+    ref = parity.oracle_tune(spec, t)
+    assert np.all(ref["w_f"][0] == 0.0) and np.all(ref["dw"][0] == 0.0) and np.abs(ref["dgamma"][0]) > 0
+    got = parity.run_tune_gpu(spec, t)
+    parity.compare(got, ref, parity.TOL[spec.dtype], parity.TUNE_OUTPUTS, spec.name, dtype=spec.dtype)
+    assert np.all(got["dw"][0::4] == 0.0)                          # exactly
+    # a channel with gamma = 0 outputs its b' everywhere, rounded once
+    nchw_const = got["z"][:, 0]
+    assert np.ptp(nchw_const) == 0.0 and abs(nchw_const.flat[0] - ref["b_f"][0]) <= 2.0 ** -8 * abs(ref["b_f"][0])
+
+
 FULL = [(ci, li, sp) for ci, layers in I.CONFIGS.items() for li, sp in enumerate(layers)]
 
 
