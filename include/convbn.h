@@ -57,9 +57,9 @@ typedef enum {
 } convbn_status;
 
 /* Storage type of x, w, z, dz, dx.  CONVBN_F16 (IEEE half; the paper's mixed-precision rows, Table 4: fp16 storage, fp32
- * accumulation, fp32 parameter gradients) is implemented for NHWC layers in all three modes, for the transposed
- * layers and for the elementwise glue, except depthwise layers and the grouped layers that run on the grouped
- * kernels (channels per group a multiple of 8).  Those calls return CONVBN_EUNSUPPORTED (the size queries return 0). */
+ * accumulation, fp32 parameter gradients) is an NHWC storage type like CONVBN_BF16: every entry point that takes a
+ * bf16 NHWC layer takes the same layer in half.  With CONVBN_NCHW it is refused: CONVBN_EUNSUPPORTED (the size
+ * queries return 0). */
 typedef enum { CONVBN_F32 = 0, CONVBN_BF16 = 1, CONVBN_F16 = 2 } convbn_dtype;
 typedef enum { CONVBN_NCHW = 0, CONVBN_NHWC = 1 } convbn_layout;
 typedef enum { CONVBN_MODE_TUNE = 0, CONVBN_MODE_EVAL = 1, CONVBN_MODE_DEPLOY = 2 } convbn_mode;

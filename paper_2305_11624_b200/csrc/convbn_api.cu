@@ -349,9 +349,9 @@ bool strided_dgrad_ok(const convbn_desc *d, const Problem &pb) {
            pb.pin < (1LL << 31) - 256;
 }
 
-// CONVBN_F16 calls.  IEEE half runs on every path of ungrouped NHWC layers whose kernels know the type: the dense
-// tensor-core kernels, the window and packed kernels of the stems, the direct kernels and the element-wise ones.
-// The descriptor is checked for them, then the call proceeds as its bf16 twin with the half flag set for the
+// CONVBN_F16 calls.  IEEE half is an NHWC storage type like bf16 and runs on the same kernels, each of which either
+// moves 16-bit elements without looking at them or knows the type (a run-time flag or a second instantiation).
+// The descriptor is checked, then the call proceeds as its bf16 twin with the half flag set for the
 // launchers (operand format of the MMAs, conversions of results and of rescaled weights, the constant 1, the
 // element type of the templated kernels).  The flag is cleared when the call returns.
 struct HalfCall {
@@ -367,11 +367,7 @@ struct HalfCall {
         Problem pb;
         status = make_problem(&d, &pb);
         if (status != CONVBN_OK) return;
-        const Plan pw = make_plan(&d, pb, CONVBN_PHASE_TUNE_BWD_WEIGHT);
-        // depthwise and grouped kernels read bf16 only
-        const bool typed_elsewhere = grouped_path(&d, pb) || dw_path(&d, pb) || pw.grouped_wgrad || pw.grouped8_wgrad ||
-                                     pw.dw_wgrad || pw.dw_tma_wgrad;
-        if (d.layout != CONVBN_NHWC || typed_elsewhere) { status = CONVBN_EUNSUPPORTED; return; }
+        if (d.layout != CONVBN_NHWC) { status = CONVBN_EUNSUPPORTED; return; }
         set_call_f16(1);
         set_here = true;
     }

@@ -18,32 +18,30 @@ constexpr int kMaxTaps = 49;   // up to 7 x 7
 
 struct DwShape {
     int n, c, h_in, w_in, h_out, w_out, kh, kw, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w;
+    int f16;               // 16-bit storage type: 0 bf16, 1 IEEE half
 };
 
-__device__ __forceinline__ void unpack8(const uint4 &q, float (&f)[8]) {
+__device__ __forceinline__ void unpack8(const uint4 &q, float (&f)[8], int f16) {
     const uint32_t u[4] = {q.x, q.y, q.z, q.w};
+    if (f16) {
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        f[2 * e] = __uint_as_float(u[e] << 16);
-        f[2 * e + 1] = __uint_as_float(u[e] & 0xFFFF0000u);
+        for (int e = 0; e < 4; ++e) unpack2_t<true>(u[e], f[2 * e], f[2 * e + 1]);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) unpack2_t<false>(u[e], f[2 * e], f[2 * e + 1]);
     }
 }
 
-__device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
-    uint4 q;
-    __nv_bfloat162 h;
-    h = __floats2bfloat162_rn(f[0], f[1]); q.x = *(uint32_t *)&h;
-    h = __floats2bfloat162_rn(f[2], f[3]); q.y = *(uint32_t *)&h;
-    h = __floats2bfloat162_rn(f[4], f[5]); q.z = *(uint32_t *)&h;
-    h = __floats2bfloat162_rn(f[6], f[7]); q.w = *(uint32_t *)&h;
-    return q;
+__device__ __forceinline__ uint4 pack8(const float (&f)[8], int f16) {
+    return make_uint4(pack2_h16(f[0], f[1], f16), pack2_h16(f[2], f[3], f16), pack2_h16(f[4], f[5], f16),
+                      pack2_h16(f[6], f[7], f16));
 }
 
 // Stage the block's weights in shared memory as fp32 [tap][C] (global layout is [C][tap]).
-__device__ __forceinline__ void stage_weights(float *w_s, const __nv_bfloat16 *w, int taps, int c) {
+__device__ __forceinline__ void stage_weights(float *w_s, const __nv_bfloat16 *w, int taps, int c, int f16) {
     for (int i = threadIdx.x; i < taps * c; i += blockDim.x) {
         const int ch = i % c, t = i / c;
-        w_s[i] = __bfloat162float(w[(size_t)ch * taps + t]);
+        w_s[i] = load_h16(w + (size_t)ch * taps + t, f16);
     }
     __syncthreads();
 }
@@ -56,7 +54,7 @@ __global__ void __launch_bounds__(256) dw_fwd_kernel(DwShape s, const uint4 *__r
                                                      const float *__restrict__ bias, uint4 *__restrict__ z) {
     extern __shared__ float w_s[];                   // [taps][C]
     const int v = s.c / 8;
-    stage_weights(w_s, w, s.kh * s.kw, s.c);
+    stage_weights(w_s, w, s.kh * s.kw, s.c, s.f16);
     const uint32_t wgroups = (uint32_t)(s.w_out + TW - 1) / TW;
     const uint32_t total = (uint32_t)s.n * s.h_out * wgroups * v;
     for (uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
@@ -94,7 +92,7 @@ __global__ void __launch_bounds__(256) dw_fwd_kernel(DwShape s, const uint4 *__r
 #pragma unroll
                     for (int j = 0; j < TW; ++j) {
                         float xv[8];
-                        unpack8(seg[j + q], xv);
+                        unpack8(seg[j + q], xv, s.f16);
 #pragma unroll
                         for (int e = 0; e < 8; ++e) acc[j][e] = fmaf(xv[e], wv[e], acc[j][e]);
                     }
@@ -110,7 +108,7 @@ __global__ void __launch_bounds__(256) dw_fwd_kernel(DwShape s, const uint4 *__r
                         const int wi = (wo0 + j) * s.stride_w - s.pad_w + q * s.dil_w;
                         if (wi >= 0 && wi < s.w_in && wo0 + j < s.w_out) {
                             float xv[8];
-                            unpack8(__ldg(xrow + (size_t)wi * v), xv);
+                            unpack8(__ldg(xrow + (size_t)wi * v), xv, s.f16);
 #pragma unroll
                             for (int e = 0; e < 8; ++e) acc[j][e] = fmaf(xv[e], wv[e], acc[j][e]);
                         }
@@ -121,7 +119,7 @@ __global__ void __launch_bounds__(256) dw_fwd_kernel(DwShape s, const uint4 *__r
         uint4 *zrow = z + ((size_t)(n * s.h_out + ho) * s.w_out + wo0) * v + cv;
 #pragma unroll
         for (int j = 0; j < TW; ++j)
-            if (wo0 + j < s.w_out) zrow[(size_t)j * v] = pack8(acc[j]);
+            if (wo0 + j < s.w_out) zrow[(size_t)j * v] = pack8(acc[j], s.f16);
     }
 }
 
@@ -137,7 +135,7 @@ __global__ void __launch_bounds__(256, KH <= 3 ? 2 : 1) dw_stream_kernel(DwShape
     extern __shared__ float w_s[];                   // [taps][C]
     constexpr int PF = 3;                            // rows of look-ahead for the L2 prefetch
     const int v = s.c / 8;
-    stage_weights(w_s, w, KH * KW, s.c);
+    stage_weights(w_s, w, KH * KW, s.c, s.f16);
     const uint32_t wgroups = (uint32_t)(s.w_out + TW - 1) / TW, bands = (uint32_t)(s.h_out + th - 1) / th;
     const uint32_t total = (uint32_t)s.n * bands * wgroups * v;
     for (uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
@@ -191,7 +189,7 @@ __global__ void __launch_bounds__(256, KH <= 3 ? 2 : 1) dw_stream_kernel(DwShape
 #pragma unroll
                         for (int j = 0; j < TW + KW - 1; ++j) {
                             const int wi = wi0 + j;
-                            unpack8((wi >= 0 && wi < s.w_in) ? __ldg(xrow + (size_t)wi * v) : make_uint4(0, 0, 0, 0), xs[j]);
+                            unpack8((wi >= 0 && wi < s.w_in) ? __ldg(xrow + (size_t)wi * v) : make_uint4(0, 0, 0, 0), xs[j], s.f16);
                         }
 #pragma unroll
                         for (int r = 0; r < KH; ++r) {
@@ -216,7 +214,7 @@ __global__ void __launch_bounds__(256, KH <= 3 ? 2 : 1) dw_stream_kernel(DwShape
                         const int sl = (ph + 1) % KH;
 #pragma unroll
                         for (int j = 0; j < TW; ++j) {
-                            if (wo0 + j < s.w_out) zcol[((size_t)od * s.w_out + j) * v] = pack8(acc[sl][j]);
+                            if (wo0 + j < s.w_out) zcol[((size_t)od * s.w_out + j) * v] = pack8(acc[sl][j], s.f16);
 #pragma unroll
                             for (int e = 0; e < 8; ++e) acc[sl][j][e] = bv[e];
                         }
@@ -269,7 +267,7 @@ __device__ __forceinline__ void dw_stream4_item(const DwShape &s, const uint2 *_
             if (k < steps) {
                 f32x2 xs[NX][2];
 #pragma unroll
-                for (int j = 0; j < NX; ++j) xs[j][0] = widen(raw[ph][j].x), xs[j][1] = widen(raw[ph][j].y);
+                for (int j = 0; j < NX; ++j) xs[j][0] = widen_h16(raw[ph][j].x, s.f16), xs[j][1] = widen_h16(raw[ph][j].y, s.f16);
                 {
                     const int hi = hi0 + k + KH;
                     if (k + KH < steps && hi >= 0 && hi < s.h_in) {
@@ -299,7 +297,7 @@ __device__ __forceinline__ void dw_stream4_item(const DwShape &s, const uint2 *_
                     uint2 *zr = zp + (k - (KH - 1)) * zpitch;
 #pragma unroll
                     for (int j = 0; j < TW; ++j)
-                        if (out_ok[j]) zr[j * colstep] = make_uint2(narrow(acc[sl][j][0]), narrow(acc[sl][j][1]));
+                        if (out_ok[j]) zr[j * colstep] = make_uint2(narrow_h16(acc[sl][j][0], s.f16), narrow_h16(acc[sl][j][1], s.f16));
                 }
             }
         }
@@ -313,7 +311,7 @@ __global__ void __launch_bounds__(256, 2) dw_stream4_kernel(DwShape s, const uin
                                                             int th) {
     extern __shared__ float w_s[];                   // [taps][C]
     const int v = s.c / 4;
-    stage_weights(w_s, w, KH * KW, s.c);
+    stage_weights(w_s, w, KH * KW, s.c, s.f16);
     const uint32_t wgroups = (uint32_t)(s.w_out + TW - 1) / TW, bands = (uint32_t)(s.h_out + th - 1) / th;
     const uint32_t total = (uint32_t)s.n * bands * wgroups * v;
     for (uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
@@ -358,7 +356,7 @@ __global__ void __launch_bounds__(256) dw_dgrad_kernel(DwShape s, const uint4 *_
                                                        uint4 *__restrict__ dx) {
     extern __shared__ float w_s[];
     const int v = s.c / 8;
-    stage_weights(w_s, w, s.kh * s.kw, s.c);
+    stage_weights(w_s, w, s.kh * s.kw, s.c, s.f16);
     const uint32_t total = (uint32_t)s.n * s.h_in * s.w_in * v;
     for (uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
         uint32_t t = idx / (uint32_t)v;
@@ -379,13 +377,13 @@ __global__ void __launch_bounds__(256) dw_dgrad_kernel(DwShape s, const uint4 *_
                 const int wo = ws / s.stride_w;
                 if (wo >= s.w_out) continue;
                 float dv[8];
-                unpack8(__ldg(dz + ((size_t)(n * s.h_out + ho) * s.w_out + wo) * v + cv), dv);
+                unpack8(__ldg(dz + ((size_t)(n * s.h_out + ho) * s.w_out + wo) * v + cv), dv, s.f16);
                 const float *wp = w_s + (r * s.kw + q) * s.c + cv * 8;
 #pragma unroll
                 for (int e = 0; e < 8; ++e) acc[e] = fmaf(dv[e], wp[e], acc[e]);
             }
         }
-        dx[idx] = pack8(acc);
+        dx[idx] = pack8(acc, s.f16);
     }
 }
 
@@ -413,7 +411,7 @@ __global__ void __launch_bounds__(256) dw_wgrad_kernel(DwShape s, const uint4 *_
         const uint32_t n = t2 / (uint32_t)s.h_out;
         const int ho = (int)(t2 - n * (uint32_t)s.h_out);
         float dv[8];
-        unpack8(__ldg(dz + (size_t)p * v + cv), dv);
+        unpack8(__ldg(dz + (size_t)p * v + cv), dv, s.f16);
 #pragma unroll
         for (int t = 0; t < TAPS; ++t) {
             const int r = t / s.kw, q = t - r * s.kw;
@@ -421,7 +419,7 @@ __global__ void __launch_bounds__(256) dw_wgrad_kernel(DwShape s, const uint4 *_
             const int wi = wo * s.stride_w - s.pad_w + q * s.dil_w;
             if (hi >= 0 && hi < s.h_in && wi >= 0 && wi < s.w_in) {
                 float xv[8];
-                unpack8(__ldg(x + ((size_t)(n * s.h_in + hi) * s.w_in + wi) * v + cv), xv);
+                unpack8(__ldg(x + ((size_t)(n * s.h_in + hi) * s.w_in + wi) * v + cv), xv, s.f16);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) acc[t][e] = fmaf(dv[e], xv[e], acc[t][e]);
             }
@@ -485,13 +483,13 @@ __global__ void __launch_bounds__(256, 1) dw_wgrad_window_kernel(DwShape s, cons
         }
         float dv[TW][8];
 #pragma unroll
-        for (int j = 0; j < TW; ++j) unpack8(dq[j], dv[j]);
+        for (int j = 0; j < TW; ++j) unpack8(dq[j], dv[j], s.f16);
 #pragma unroll
         for (int r = 0; r < KH; ++r)
 #pragma unroll
             for (int j = 0; j < TW + KW - 1; ++j) {
                 float xv[8];
-                unpack8(seg[r][j], xv);
+                unpack8(seg[r][j], xv, s.f16);
 #pragma unroll
                 for (int q = 0; q < KW; ++q) {
                     const int o = j - q;
@@ -519,7 +517,7 @@ __global__ void __launch_bounds__(256, 1) dw_wgrad_window_kernel(DwShape s, cons
 
 DwShape dw_shape(const Problem &pb) {
     return DwShape{pb.n, pb.c_in, pb.h_in, pb.w_in, pb.h_out, pb.w_out, pb.kh, pb.kw, pb.stride_h, pb.stride_w,
-                   pb.pad_h, pb.pad_w, pb.dil_h, pb.dil_w};
+                   pb.pad_h, pb.pad_w, pb.dil_h, pb.dil_w, call_f16()};
 }
 
 int dw_grid(long long total) {

@@ -80,7 +80,7 @@ struct DwTmaGeom {
     int consumer_warps;
 };
 
-template <int TW, int KH, int KW>
+template <int TW, int KH, int KW, bool H>
 __global__ void __launch_bounds__(TW >= 4 ? 384 : 288, TW >= 4 ? 1 : 2) dw_tma_kernel(const __grid_constant__ CUtensorMap tx, DwTmaGeom g,
                                                         const __nv_bfloat16 *__restrict__ w,
                                                         const float *__restrict__ bias, const BnFold fold,
@@ -157,7 +157,7 @@ __global__ void __launch_bounds__(TW >= 4 ? 384 : 288, TW >= 4 ? 1 : 2) dw_tma_k
             const int src = reverse_taps ? KH * KW - 1 - tp : tp;
             float f[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) f[e] = sc[e] * __bfloat162float(w[(size_t)(cv * 4 + e) * (KH * KW) + src]);
+            for (int e = 0; e < 4; ++e) f[e] = sc[e] * load_h16(w + (size_t)(cv * 4 + e) * (KH * KW) + src, H ? 1 : 0);
             wr[tp][0] = pair(f[0], f[1]);
             wr[tp][1] = pair(f[2], f[3]);
         }
@@ -209,8 +209,8 @@ __global__ void __launch_bounds__(TW >= 4 ? 384 : 288, TW >= 4 ? 1 : 2) dw_tma_k
 #pragma unroll
                         for (int j = 0; j < NX; ++j) {
                             const uint2 q = lds_u2(col_addr[j] + slot_off);
-                            xs[j][0] = widen(q.x);
-                            xs[j][1] = widen(q.y);
+                            xs[j][0] = widen_t<H>(q.x);
+                            xs[j][1] = widen_t<H>(q.y);
                         }
                         __syncwarp();
                         arrive_lane0(empty0 + slot * 8, lane);
@@ -238,7 +238,7 @@ __global__ void __launch_bounds__(TW >= 4 ? 384 : 288, TW >= 4 ? 1 : 2) dw_tma_k
                             const bool row_done = k >= KH - 1;
 #pragma unroll
                             for (int j = 0; j < TW; ++j)
-                                stg_u2_if(zr + (ptrdiff_t)j * v, narrow(acc[sl][j][0]), narrow(acc[sl][j][1]), row_done && out_ok[j]);
+                                stg_u2_if(zr + (ptrdiff_t)j * v, narrow_t<H>(acc[sl][j][0]), narrow_t<H>(acc[sl][j][1]), row_done && out_ok[j]);
                         }
                         zr += zpitch;
                     }
@@ -256,7 +256,7 @@ __global__ void __launch_bounds__(TW >= 4 ? 384 : 288, TW >= 4 ? 1 : 2) dw_tma_k
 // last KH dZ rows of its columns in KH rotating register slots and its KH x KW x 4 sums (plus the sum of
 // dZ) in registers across all the items of the block.  At the end the thread columns are added in
 // column order through shared memory, and the block writes one partial row: part[block][c][KH KW + 1].
-template <int TW, int KH, int KW>
+template <int TW, int KH, int KW, bool H>
 __global__ void __launch_bounds__(TW >= 4 ? 384 : 288, TW >= 4 ? 1 : 2) dw_tma_wgrad_kernel(const __grid_constant__ CUtensorMap tx,
                                                               const __grid_constant__ CUtensorMap tdz, DwTmaGeom g,
                                                               float *__restrict__ part, int *err) {
@@ -348,15 +348,15 @@ __global__ void __launch_bounds__(TW >= 4 ? 384 : 288, TW >= 4 ? 1 : 2) dw_tma_w
 #pragma unroll
                             for (int j = 0; j < NX; ++j) {
                                 const uint2 q = lds_u2(x_addr[j] + slot_off);
-                                xs[j][0] = widen(q.x);
-                                xs[j][1] = widen(q.y);
+                                xs[j][0] = widen_t<H>(q.x);
+                                xs[j][1] = widen_t<H>(q.y);
                             }
                             if (k < rows) {                    // same for the whole block
 #pragma unroll
                                 for (int j = 0; j < TW; ++j) {
                                     const uint2 q = lds_u2(dz_addr[j] + slot_off);
-                                    dzw[ph][j][0] = widen(q.x);
-                                    dzw[ph][j][1] = widen(q.y);
+                                    dzw[ph][j][0] = widen_t<H>(q.x);
+                                    dzw[ph][j][1] = widen_t<H>(q.y);
                                     acc[KH * KW][0] = fma2(dzw[ph][j][0], ones, acc[KH * KW][0]);
                                     acc[KH * KW][1] = fma2(dzw[ph][j][1], ones, acc[KH * KW][1]);
                                 }
@@ -422,7 +422,7 @@ __global__ void __launch_bounds__(32 * (TAPS + 1)) dw_wgrad_finish_kernel(int c_
                                                                            const float *__restrict__ mean,
                                                                            float *__restrict__ dw, float *__restrict__ db,
                                                                            float *__restrict__ dgamma,
-                                                                           float *__restrict__ dbeta) {
+                                                                           float *__restrict__ dbeta, int f16) {
     __shared__ float tot[TAPS + 1];
     const int c = blockIdx.x, t = threadIdx.x >> 5, lane = threadIdx.x & 31;
     float sum = 0.f;
@@ -436,7 +436,7 @@ __global__ void __launch_bounds__(32 * (TAPS + 1)) dw_wgrad_finish_kernel(int c_
         const float dsum = tot[TAPS];
         if (vec3) {
             float dot = 0.f;
-            for (int k = 0; k < TAPS; ++k) dot = fmaf(tot[k], __bfloat162float(w[(size_t)c * TAPS + k]), dot);
+            for (int k = 0; k < TAPS; ++k) dot = fmaf(tot[k], load_h16(w + (size_t)c * TAPS + k, f16), dot);
             const float s = vec3[c], r = vec3[2 * c_total + c];
             dbeta[c] = dsum;
             if (db) db[c] = s * dsum;
@@ -530,10 +530,16 @@ cudaError_t launch_dw_tma(const Problem &pb, const void *x, const void *w, const
     if (!dw_tma_map(&tx, x, pb.n, pb.h_in, pb.w_in, pb.c_in, g.cols_t * TW + KW - 1)) return cudaErrorInvalidValue;
     int *err = nullptr;
     if ((e = error_word_address(&err)) != cudaSuccess) return e;
-    static PerDevice attr;
-    if ((e = max_dynamic_smem_once(dw_tma_kernel<TW, KH, KW>, 210 * 1024, &attr)) != cudaSuccess) return e;
+    static PerDevice attr, attr_h;        // (one flag per instantiation)
     const BnFold none{nullptr, nullptr, nullptr, nullptr, nullptr, 0.f, nullptr};
-    dw_tma_kernel<TW, KH, KW><<<grid, (g.consumer_warps + 1) * 32, dw_tma_smem(g), st>>>(
+    if (call_f16()) {
+        if ((e = max_dynamic_smem_once(dw_tma_kernel<TW, KH, KW, true>, 210 * 1024, &attr_h)) != cudaSuccess) return e;
+        dw_tma_kernel<TW, KH, KW, true><<<grid, (g.consumer_warps + 1) * 32, dw_tma_smem(g), st>>>(
+            tx, g, (const __nv_bfloat16 *)w, bias, fold ? *fold : none, scale, reverse_taps ? 1 : 0, (uint2 *)z, err);
+        return cudaGetLastError();
+    }
+    if ((e = max_dynamic_smem_once(dw_tma_kernel<TW, KH, KW, false>, 210 * 1024, &attr)) != cudaSuccess) return e;
+    dw_tma_kernel<TW, KH, KW, false><<<grid, (g.consumer_warps + 1) * 32, dw_tma_smem(g), st>>>(
         tx, g, (const __nv_bfloat16 *)w, bias, fold ? *fold : none, scale, reverse_taps ? 1 : 0, (uint2 *)z, err);
     return cudaGetLastError();
 }
@@ -558,10 +564,15 @@ cudaError_t launch_dw_tma_wgrad(const Problem &pb, const void *dz, const void *x
     if (!dw_tma_map(&tdz, dz, pb.n, pb.h_out, pb.w_out, pb.c_in, g.cols_t * TW)) return cudaErrorInvalidValue;
     int *err = nullptr;
     if ((e = error_word_address(&err)) != cudaSuccess) return e;
-    static PerDevice attr;
-    if ((e = max_dynamic_smem_once(dw_tma_wgrad_kernel<TW, KH, KW>, 210 * 1024, &attr)) != cudaSuccess) return e;
-    dw_tma_wgrad_kernel<TW, KH, KW><<<grid, (g.consumer_warps + 1) * 32, dw_tma_smem(g), st>>>(tx, tdz, g, part, err);
+    static PerDevice attr, attr_h;
     *nparts = (int)grid;
+    if (call_f16()) {
+        if ((e = max_dynamic_smem_once(dw_tma_wgrad_kernel<TW, KH, KW, true>, 210 * 1024, &attr_h)) != cudaSuccess) return e;
+        dw_tma_wgrad_kernel<TW, KH, KW, true><<<grid, (g.consumer_warps + 1) * 32, dw_tma_smem(g), st>>>(tx, tdz, g, part, err);
+        return cudaGetLastError();
+    }
+    if ((e = max_dynamic_smem_once(dw_tma_wgrad_kernel<TW, KH, KW, false>, 210 * 1024, &attr)) != cudaSuccess) return e;
+    dw_tma_wgrad_kernel<TW, KH, KW, false><<<grid, (g.consumer_warps + 1) * 32, dw_tma_smem(g), st>>>(tx, tdz, g, part, err);
     return cudaGetLastError();
 }
 
@@ -569,7 +580,7 @@ cudaError_t launch_dw_wgrad_finish(const Problem &pb, const float *part, int npa
                                    const float *b, const float *mean, float *dw, float *db, float *dgamma,
                                    float *dbeta, cudaStream_t st) {
     dw_wgrad_finish_kernel<9><<<pb.c_in, 32 * 10, 0, st>>>(pb.c_in, nparts, part, (const __nv_bfloat16 *)w, vec3, b, mean,
-                                                         dw, db, dgamma, dbeta);
+                                                         dw, db, dgamma, dbeta, call_f16());
     return cudaGetLastError();
 }
 

@@ -13,7 +13,7 @@ namespace convbn {
 __global__ void __launch_bounds__(256) expand_blockdiag_kernel(int c, int taps, int cg,
                                                                const __nv_bfloat16 *__restrict__ w,
                                                                const float *__restrict__ s_vec,
-                                                               __nv_bfloat16 *__restrict__ wbd, int transpose_flip) {
+                                                               __nv_bfloat16 *__restrict__ wbd, int transpose_flip, int f16) {
     const long long total = (long long)c * taps * 64;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
@@ -24,13 +24,13 @@ __global__ void __launch_bounds__(256) expand_blockdiag_kernel(int c, int taps, 
         if (!transpose_flip) {
             const int co = row, start = ((co & 63) / cg) * cg;
             if (j >= start && j < start + cg)
-                val = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((long long)co * taps + tap_o) * cg + (j - start)]);
+                val = (s_vec ? s_vec[co] : 1.f) * load_h16(w + ((long long)co * taps + tap_o) * cg + (j - start), f16);
         } else {
             const int ci = row, co = (ci & ~63) + j, tap = taps - 1 - tap_o;
             if ((j / cg) == ((ci & 63) / cg))
-                val = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((long long)co * taps + tap) * cg + (ci % cg)]);
+                val = (s_vec ? s_vec[co] : 1.f) * load_h16(w + ((long long)co * taps + tap) * cg + (ci % cg), f16);
         }
-        wbd[i] = __float2bfloat16_rn(val);
+        reinterpret_cast<uint16_t *>(wbd)[i] = pack1_h16(val, f16);
     }
 }
 
@@ -40,7 +40,7 @@ cudaError_t launch_expand_blockdiag(const Problem &pb, const void *w, const floa
     long long blocks = (total + 255) / 256;
     if (blocks > device_sm_count() * 8) blocks = device_sm_count() * 8;
     expand_blockdiag_kernel<<<(int)blocks, 256, 0, st>>>(pb.c_out, pb.kh * pb.kw, pb.cg, (const __nv_bfloat16 *)w,
-                                                         s_vec, (__nv_bfloat16 *)wbd, transpose_flip ? 1 : 0);
+                                                         s_vec, (__nv_bfloat16 *)wbd, transpose_flip ? 1 : 0, call_f16());
     return cudaGetLastError();
 }
 
@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(256) wgrad_epilogue_bd_kernel(int c_out, int t
                                                                const float *__restrict__ mean,
                                                                float *__restrict__ dw, float *__restrict__ db,
                                                                float *__restrict__ dgamma,
-                                                               float *__restrict__ dbeta) {
+                                                               float *__restrict__ dbeta, int f16) {
     __shared__ float red[256];
     const int co = blockIdx.x, kdim = taps * cg, nblk = c_out / 64;
     const int blk = co >> 6, col = co & 63, start = (col / cg) * cg;
@@ -69,7 +69,7 @@ __global__ void __launch_bounds__(256) wgrad_epilogue_bd_kernel(int c_out, int t
         float acc = 0.f;
         for (int sp = 0; sp < splits; ++sp) acc += part[((size_t)sp * nblk + blk) * tile + o];
         dw[(size_t)co * kdim + k] = s * acc;
-        if (vec3) dot = fmaf(acc, __bfloat162float(w[(size_t)co * kdim + k]), dot);
+        if (vec3) dot = fmaf(acc, load_h16(w + (size_t)co * kdim + k, f16), dot);
     }
     float bs = 0.f;
     if (bsum_part)
@@ -101,7 +101,7 @@ cudaError_t launch_wgrad_epilogue_bd(const Problem &pb, const float *partials, i
                                      float *dbeta, cudaStream_t st) {
     wgrad_epilogue_bd_kernel<<<pb.c_out, 256, 0, st>>>(pb.c_out, pb.kh * pb.kw, pb.cg, partials, splits, bsum_part,
                                                        bsplits, (const __nv_bfloat16 *)w, vec3, b, mean, dw, db,
-                                                       dgamma, dbeta);
+                                                       dgamma, dbeta, call_f16());
     return cudaGetLastError();
 }
 

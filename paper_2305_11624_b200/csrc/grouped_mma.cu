@@ -40,6 +40,7 @@ struct GroupedGeom {
     uint32_t stage_stride;     // allocation per stage (multiple of 1024, includes the read-ahead tail)
 };
 
+template <bool H>            // H: IEEE-half storage, else bf16
 __global__ void __launch_bounds__(kGThreads) grouped8_conv_kernel(const __grid_constant__ CUtensorMap tm_act,
                                                                  const GroupedGeom g,
                                                                  const __nv_bfloat16 *__restrict__ w,
@@ -136,7 +137,7 @@ __global__ void __launch_bounds__(kGThreads) grouped8_conv_kernel(const __grid_c
 #pragma unroll
                 for (int u = 0; u < kGTiles; ++u) ldmatrix_x4(a[u][0], a[u][1], a[u][2], a[u][3], addr + (uint32_t)u * 2048u);
 #pragma unroll
-                for (int u = 0; u < kGTiles; ++u) mma_16x8x16_bf16(acc[u], a[u][0], a[u][1], a[u][2], a[u][3], bf[ks][0], bf[ks][1]);
+                for (int u = 0; u < kGTiles; ++u) mma_16x8x16_t<H>(acc[u], a[u][0], a[u][1], a[u][2], a[u][3], bf[ks][0], bf[ks][1]);
             }
             // rows gr and gr + 8 of tile u are virtual pixels v0 + 16 u + gr (+ 8): walk them, 8 pixels a step
             int ti = (v0 + gr) / g.Wt, tj = (v0 + gr) - ti * g.Wt;
@@ -146,7 +147,7 @@ __global__ void __launch_bounds__(kGThreads) grouped8_conv_kernel(const __grid_c
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
                     if (ti < rows_here && tj < g.wo)
-                        *reinterpret_cast<__nv_bfloat162 *>(obase + off) = __floats2bfloat162_rn(acc[u][2 * half], acc[u][2 * half + 1]);
+                        *reinterpret_cast<uint32_t *>(obase + off) = pack2_t<H>(acc[u][2 * half], acc[u][2 * half + 1]);
                     tj += 8;
                     off += 8 * g.c;
                     if (tj >= g.Wt) { tj -= g.Wt; ++ti; off += wrap_elems; }
@@ -169,6 +170,7 @@ __global__ void __launch_bounds__(kGThreads) grouped8_conv_kernel(const __grid_c
 // transposing ldmatrix loads, and a sixth MMA against a matrix of ones gives sum dZ.  A block keeps one
 // 64-channel chunk for its whole life, so the sums stay in registers across its bands; at the end every
 // warp writes its group's partial block: part[slot][C][taps 8], bsum[slot][C].
+template <bool H>
 __global__ void __launch_bounds__(kGThreads) grouped8_wgrad_kernel(const __grid_constant__ CUtensorMap tm_x,
                                                                   const __grid_constant__ CUtensorMap tm_dz,
                                                                   const GroupedGeom g, uint32_t dz_off, int slots,
@@ -233,7 +235,7 @@ __global__ void __launch_bounds__(kGThreads) grouped8_wgrad_kernel(const __grid_
         }
     }
     const int npix = g.R * g.Wt;
-    const uint32_t ones = 0x3F803F80u;                         // bf16 1.0 twice
+    const uint32_t ones = one_h16(H ? 1 : 0) * 0x10001u;       // 1.0 twice
     uint32_t s = 0, ph = 0;
     bool ok = true;
     for (uint32_t it = (uint32_t)slot; it < items && ok; it += (uint32_t)slots) {
@@ -245,14 +247,14 @@ __global__ void __launch_bounds__(kGThreads) grouped8_wgrad_kernel(const __grid_
                 const int v = v0 + (lane & 15);
                 ldmatrix_x2_trans(b0, b1, dzpatch + (uint32_t)v * 128u + (uint32_t)((warp ^ (v & 7)) << 4));
             }
-            mma_16x8x16_bf16(accs, ones, ones, ones, ones, b0, b1);
+            mma_16x8x16_t<H>(accs, ones, ones, ones, ones, b0, b1);
 #pragma unroll
             for (int ks = 0; ks < kGMaxKSteps; ++ks) {
                 if (ks >= ksteps) break;
                 const int v = v0 + vrow[ks];
                 uint32_t a0, a1, a2, a3;
                 ldmatrix_x4_trans(a0, a1, a2, a3, xpatch + (uint32_t)v * 128u + (uint32_t)((warp ^ (v & 7)) << 4));
-                mma_16x8x16_bf16(acc[ks], a0, a1, a2, a3, b0, b1);
+                mma_16x8x16_t<H>(acc[ks], a0, a1, a2, a3, b0, b1);
             }
         }
         __syncwarp();
@@ -295,7 +297,7 @@ __global__ void __launch_bounds__(256) grouped8_wgrad_finish_kernel(int c, int k
                                                                    const float *__restrict__ mean,
                                                                    float *__restrict__ dw, float *__restrict__ db,
                                                                    float *__restrict__ dgamma,
-                                                                   float *__restrict__ dbeta) {
+                                                                   float *__restrict__ dbeta, int f16) {
     __shared__ float red[256];
     __shared__ float dots[96];
     const int co = blockIdx.x;
@@ -316,7 +318,7 @@ __global__ void __launch_bounds__(256) grouped8_wgrad_finish_kernel(int c, int k
         for (int jj = 0; jj < ng; ++jj) tot += red[jj * (kdim + 1) + threadIdx.x];
         if (threadIdx.x < kdim) {
             dw[(size_t)co * kdim + threadIdx.x] = s * tot;
-            dots[threadIdx.x] = vec3 ? tot * __bfloat162float(w[(size_t)co * kdim + threadIdx.x]) : 0.f;
+            dots[threadIdx.x] = vec3 ? tot * load_h16(w + (size_t)co * kdim + threadIdx.x, f16) : 0.f;
         } else {
             dots[kdim] = tot;                        // sum dZ
         }
@@ -339,12 +341,13 @@ __global__ void __launch_bounds__(256) grouped8_wgrad_finish_kernel(int c, int k
 // Backward-data operand: wt[8g + ci][taps - 1 - tap][o] = s[8g + o] w[8g + o][tap][ci]
 __global__ void __launch_bounds__(256) grouped8_flip_weights_kernel(int c, int taps, const __nv_bfloat16 *__restrict__ w,
                                                                    const float *__restrict__ s_vec,
-                                                                   __nv_bfloat16 *__restrict__ wt) {
+                                                                   __nv_bfloat16 *__restrict__ wt, int f16) {
     const int total = c * taps * 8;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
         const int o = i & 7, tap_o = (i >> 3) % taps, row = (i >> 3) / taps;   // row = 8g + ci
         const int co = (row & ~7) + o, ci = row & 7, tap = taps - 1 - tap_o;
-        wt[i] = __float2bfloat16_rn((s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((size_t)co * taps + tap) * 8 + ci]));
+        reinterpret_cast<uint16_t *>(wt)[i] =
+            pack1_h16((s_vec ? s_vec[co] : 1.f) * load_h16(w + ((size_t)co * taps + tap) * 8 + ci, f16), f16);
     }
 }
 
@@ -424,10 +427,16 @@ static cudaError_t launch_grouped8(int n, int ha, int wa, int c, int ho, int wo,
     int *err = nullptr;
     cudaError_t e = error_word_address(&err);
     if (e != cudaSuccess) return e;
-    static PerDevice attr;
-    if ((e = max_dynamic_smem_once(grouped8_conv_kernel, 220 * 1024, &attr)) != cudaSuccess) return e;
-    grouped8_conv_kernel<<<pl.grid, kGThreads, pl.smem, st>>>(ta, pl.g, (const __nv_bfloat16 *)w, bias,
-                                                             (__nv_bfloat16 *)out, err);
+    static PerDevice attr, attr_h;        // (one flag per instantiation)
+    if (call_f16()) {
+        if ((e = max_dynamic_smem_once(grouped8_conv_kernel<true>, 220 * 1024, &attr_h)) != cudaSuccess) return e;
+        grouped8_conv_kernel<true><<<pl.grid, kGThreads, pl.smem, st>>>(ta, pl.g, (const __nv_bfloat16 *)w, bias,
+                                                                       (__nv_bfloat16 *)out, err);
+        return cudaGetLastError();
+    }
+    if ((e = max_dynamic_smem_once(grouped8_conv_kernel<false>, 220 * 1024, &attr)) != cudaSuccess) return e;
+    grouped8_conv_kernel<false><<<pl.grid, kGThreads, pl.smem, st>>>(ta, pl.g, (const __nv_bfloat16 *)w, bias,
+                                                                    (__nv_bfloat16 *)out, err);
     return cudaGetLastError();
 }
 
@@ -441,7 +450,7 @@ cudaError_t launch_grouped8_flip_weights(const Problem &pb, const void *w, const
                                          cudaStream_t st) {
     const int total = pb.c_out * pb.kh * pb.kw * 8;
     grouped8_flip_weights_kernel<<<(total + 255) / 256, 256, 0, st>>>(pb.c_out, pb.kh * pb.kw, (const __nv_bfloat16 *)w,
-                                                                     s_vec, (__nv_bfloat16 *)wt);
+                                                                     s_vec, (__nv_bfloat16 *)wt, call_f16());
     return cudaGetLastError();
 }
 
@@ -498,9 +507,14 @@ cudaError_t launch_grouped8_wgrad(const Problem &pb, const void *dz, const void 
     int *err = nullptr;
     cudaError_t e = error_word_address(&err);
     if (e != cudaSuccess) return e;
-    static PerDevice attr;
-    if ((e = max_dynamic_smem_once(grouped8_wgrad_kernel, 220 * 1024, &attr)) != cudaSuccess) return e;
-    grouped8_wgrad_kernel<<<pl.grid, kGThreads, pl.smem, st>>>(tx, tdz, pl.g, pl.dz_off, slots, part, bsum, err);
+    static PerDevice attr, attr_h;
+    if (call_f16()) {
+        if ((e = max_dynamic_smem_once(grouped8_wgrad_kernel<true>, 220 * 1024, &attr_h)) != cudaSuccess) return e;
+        grouped8_wgrad_kernel<true><<<pl.grid, kGThreads, pl.smem, st>>>(tx, tdz, pl.g, pl.dz_off, slots, part, bsum, err);
+        return cudaGetLastError();
+    }
+    if ((e = max_dynamic_smem_once(grouped8_wgrad_kernel<false>, 220 * 1024, &attr)) != cudaSuccess) return e;
+    grouped8_wgrad_kernel<false><<<pl.grid, kGThreads, pl.smem, st>>>(tx, tdz, pl.g, pl.dz_off, slots, part, bsum, err);
     return cudaGetLastError();
 }
 
@@ -510,7 +524,8 @@ cudaError_t launch_grouped8_wgrad_finish(const Problem &pb, const float *part, c
     const int slots = grouped8_wgrad_slots(pb);
     if (slots <= 0) return cudaErrorInvalidValue;
     grouped8_wgrad_finish_kernel<<<pb.c_out, 256, 0, st>>>(pb.c_out, pb.kh * pb.kw * 8, slots, part, bsum,
-                                                         (const __nv_bfloat16 *)w, vec3, b, mean, dw, db, dgamma, dbeta);
+                                                         (const __nv_bfloat16 *)w, vec3, b, mean, dw, db, dgamma, dbeta,
+                                                         call_f16());
     return cudaGetLastError();
 }
 

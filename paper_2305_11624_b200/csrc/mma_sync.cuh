@@ -15,6 +15,20 @@ __device__ __forceinline__ void mma_16x8x16_bf16(float (&c)[4], uint32_t a0, uin
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// The same with IEEE-half operands, and the choice between the two at compile time.
+__device__ __forceinline__ void mma_16x8x16_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+template <bool H>
+__device__ __forceinline__ void mma_16x8x16_t(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1) {
+    if constexpr (H) mma_16x8x16_f16(c, a0, a1, a2, a3, b0, b1);
+    else mma_16x8x16_bf16(c, a0, a1, a2, a3, b0, b1);
+}
+
 // Four 8 x 8 bf16 matrices from shared memory: lanes 8i..8i+7 give the 16-byte row addresses of matrix i;
 // register i of every lane receives its two elements of matrix i in MMA fragment order.
 __device__ __forceinline__ void ldmatrix_x4(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, uint32_t smem_addr) {

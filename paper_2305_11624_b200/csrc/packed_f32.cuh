@@ -1,6 +1,7 @@
 // Packed fp32 arithmetic (two values per register pair and instruction, sm_100) and the bf16 pair
 // conversions that go with it.
 #pragma once
+#include <cuda_fp16.h>
 #include <cuda_bf16.h>
 #include <cstdint>
 
@@ -27,5 +28,22 @@ __device__ __forceinline__ uint32_t narrow(f32x2 p) {
     const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t *>(&h);
 }
+// The same for either 16-bit storage type, fixed at compile time (H: IEEE half, else bf16) or at run time.
+template <bool H>
+__device__ __forceinline__ f32x2 widen_t(uint32_t u) {
+    if constexpr (H) { const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&u)); return pair(f.x, f.y); }
+    else return widen(u);
+}
+template <bool H>
+__device__ __forceinline__ uint32_t narrow_t(f32x2 p) {
+    if constexpr (H) {
+        float lo, hi;
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
+        const __half2 h = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<const uint32_t *>(&h);
+    } else return narrow(p);
+}
+__device__ __forceinline__ f32x2 widen_h16(uint32_t u, int f16) { return f16 ? widen_t<true>(u) : widen(u); }
+__device__ __forceinline__ uint32_t narrow_h16(f32x2 p, int f16) { return f16 ? narrow_t<true>(p) : narrow(p); }
 
 }  // namespace convbn

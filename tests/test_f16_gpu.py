@@ -37,6 +37,16 @@ FALLBACK = [
     L("h_stem_w272", 2, 3, 8, 272, 64, 7, 7, stride=2, pad=3, dtype="f16", bias=True),
     L("h_stem5_s1", 1, 3, 32, 32, 64, 5, 5, stride=1, pad=2, dtype="f16"),
     L("h_stem_c8_s2", 1, 8, 20, 24, 64, 3, 3, stride=2, pad=1, dtype="f16"),
+    # depthwise: the row-streaming kernels (TMA ring; registers for narrow rows) and the general ones
+    L("h_dw", 2, 96, 14, 15, 96, 3, 3, pad=1, groups=96, dtype="f16", bias=True),
+    L("h_dw_narrow", 2, 32, 9, 6, 32, 3, 3, pad=1, groups=32, dtype="f16"),
+    L("h_dw_s2", 1, 32, 9, 9, 32, 3, 3, stride=2, pad=1, groups=32, dtype="f16"),
+    L("h_dw_5x5", 1, 48, 11, 13, 48, 5, 5, pad=2, groups=48, dtype="f16"),
+    # grouped: warp-level MMAs (8 channels per group), block-diagonal tensor-core GEMMs (other widths)
+    L("h_grouped8", 2, 256, 9, 9, 256, 3, 3, pad=1, groups=32, dtype="f16", bias=True),
+    L("h_grouped_cg4", 1, 64, 10, 12, 64, 3, 3, pad=1, groups=16, dtype="f16"),
+    L("h_grouped_cg32_s2", 2, 128, 11, 9, 128, 3, 3, stride=2, pad=1, groups=4, dtype="f16"),
+    L("h_grouped_wide", 2, 128, 17, 22, 128, 3, 3, pad=1, groups=16, dtype="f16"),
 ]
 
 
@@ -79,21 +89,25 @@ def test_half_is_not_bf16():
     assert np.isfinite(got["z"]).all()
 
 
-@pytest.mark.parametrize("spec,call", [
-    (L("h_dw", 1, 64, 16, 16, 64, 3, 3, pad=1, groups=64, dtype="f16"), "tune"),
-    (L("h_grouped", 1, 64, 16, 16, 64, 3, 3, pad=1, groups=8, dtype="f16"), "tune"),
-    (L("h_dw_eval", 1, 64, 16, 16, 64, 3, 3, pad=1, groups=64, dtype="f16"), "eval"),
-], ids=lambda v: v.name if isinstance(v, L) else v)
-def test_unsupported_half_calls_are_refused(spec, call):
-    d = make_desc(spec)
-    if call == "tune":
-        assert C.convbn_workspace_bytes(d, C.PHASE_TUNE_FWD) == 0
+def test_half_is_an_nhwc_storage_type():
+    """Half in the NCHW layout (the fp32 convention) is refused by every call, the size queries return 0."""
+    d = make_desc(L("h_nchw", 1, 64, 16, 16, 64, 3, 3, pad=1, dtype="f16", layout="nchw"))
+    assert C.convbn_workspace_bytes(d, C.PHASE_TUNE_FWD) == 0 and C.convbn_saved_bytes(d, C.MODE_EVAL) == 0
+    for call in (C.convbn_tune_fwd, C.convbn_eval_fwd):
         with pytest.raises(C.ConvBNError) as e:
-            C.convbn_tune_fwd(d, 4096, 4096, None, 4096, 4096, 4096, 4096, 4096, 4096, 4096, 1 << 20, stream=0)
-    else:
-        with pytest.raises(C.ConvBNError) as e:
-            C.convbn_eval_fwd(d, 4096, 4096, None, 4096, 4096, 4096, 4096, 4096, 4096, 4096, 1 << 20, stream=0)
-    assert e.value.status == C.EUNSUPPORTED
+            call(d, 4096, 4096, None, 4096, 4096, 4096, 4096, 4096, 4096, 4096, 1 << 20, stream=0)
+        assert e.value.status == C.EUNSUPPORTED
+
+
+@pytest.mark.parametrize("name", ["c4a", "c4b"])
+def test_half_depthwise_and_grouped_benchmark_layers_full_size(name):
+    import dataclasses
+    spec = dataclasses.replace(I.find_layer(name)[2], name=name + "_half", dtype="f16")
+    t = parity.make_inputs(spec, 99)
+    ref = parity.oracle_tune(spec, t)
+    got = parity.run_tune_gpu(spec, t, deferred=True)
+    errs = parity.compare(got, ref, parity.TOL["f16"], parity.TUNE_OUTPUTS, spec.name, dtype="f16")
+    print(spec.name, got["_kernels"], {k: "%.1e" % v for k, v in errs.items()})
 
 
 def test_half_glue_and_linear():

@@ -179,7 +179,9 @@ COMPARATOR_SPECS = [SMALL[0], SMALL[8], SMALL[10], SMALL[17], SMALL[19]] + \
      L("h_3x3_s2_128", 2, 128, 40, 42, 128, 3, 3, stride=2, pad=1, dtype="f16"),
      L("h_stem", 2, 3, 64, 80, 64, 7, 7, stride=2, pad=3, dtype="f16"),
      L("h_stem_w272", 2, 3, 8, 272, 64, 7, 7, stride=2, pad=3, dtype="f16", bias=True),
-     L("h_20_24", 2, 20, 11, 13, 24, 3, 3, stride=2, pad=1, dtype="f16", bias=True)]
+     L("h_20_24", 2, 20, 11, 13, 24, 3, 3, stride=2, pad=1, dtype="f16", bias=True),
+     L("h_dw", 2, 96, 14, 15, 96, 3, 3, pad=1, groups=96, dtype="f16", bias=True),
+     L("h_grouped8", 2, 256, 9, 9, 256, 3, 3, pad=1, groups=32, dtype="f16")]
 # (the benchmark layers run at full size)
 
 
