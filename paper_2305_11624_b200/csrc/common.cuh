@@ -62,7 +62,9 @@ template <> __device__ __forceinline__ __half from_f32<__half>(float v) { return
 // The tensor-core kernels move 16-bit elements without looking at them (TMA, shared memory, MMA operands);
 // only four things depend on whether those bits are bf16 or IEEE half: the operand-format field of the MMA
 // instruction descriptor, the conversion of results, the conversion of weights that are rescaled on the way,
-// and the constant 1.  Kernels carry an `f16` flag (0: bf16, 1: half) instead of a second instantiation.
+// and the constant 1.  Those kernels carry an `f16` flag (0: bf16, 1: half) instead of a second instantiation.
+// Kernels that do arithmetic on every element (depthwise, grouped warp-level MMAs, direct, element-wise) are
+// templates on the type or take the same flag.
 __device__ __forceinline__ uint32_t pack2_h16(float a, float b, int f16) {
     if (f16) { const __half2 h = __floats2half2_rn(a, b); return *reinterpret_cast<const uint32_t *>(&h); }
     const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);

@@ -1,5 +1,6 @@
-"""IEEE-half storage (the paper's mixed-precision rows, Table 4): forward and backward of ungrouped layers in the
-three modes against the fp64 oracle, inputs rounded to half on the host; unsupported calls are refused."""
+"""IEEE-half storage (the paper's mixed-precision rows, Table 4): Tune-mode forward and backward of every kind of NHWC
+layer against the fp64 oracle, inputs rounded to half on the host; half in the NCHW layout is refused.  (Eval and
+Deploy mode in half: the half cases of test_parity_gpu.py and test_backbone_gpu.py.)"""
 import numpy as np
 import pytest
 import torch
