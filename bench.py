@@ -81,7 +81,7 @@ NCU_TRAFFIC = {("stem_fwd", "c2s"): (63.19e6, _P2S), ("stem_dgrad", "c2s"): (116
                ("umma_bwd", "c1a"): (76.4e6, _P1), ("strip_fwd", "c1b"): (13.0e6, _P1), ("strip_dgrad", "c1b"): (13.0e6, _P1),
                ("umma_fwd", "c2a"): (14.99e6, _P2D), ("umma_dgrad", "c2a"): (5.35e6, _P2D), ("umma_wgrad", "c2a"): (16.10e6, _P2D),
                ("umma_fwd", "c2b"): (7.98e6, _P2D),
-               ("dw_fwd", "c4a"): (259.0e6, _P4), ("dw_dgrad", "c4a"): (258.6e6, _P4), ("dw_wgrad", "c4a"): (312.8e6, _P4)}
+               ("dw_fwd", "c4a"): (259.0e6, _P4), ("dw_dgrad", "c4a"): (258.7e6, _P4), ("dw_wgrad", "c4a"): (312.0e6, _P4)}
 
 KIND_OF = {"strip_fwd": "fwd", "strip_dgrad": "dgrad", "direct_fwd": "fwd", "direct_dgrad": "dgrad", "direct_wgrad": "wgrad",
            "umma_fwd": "fwd", "umma_dgrad": "dgrad", "umma_wgrad": "wgrad", "umma_bwd": "bwd",
