@@ -418,6 +418,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
     const long long row_lo = g.total_rows * blockIdx.x / gridDim.x, row_hi = g.total_rows * (blockIdx.x + 1) / gridDim.x;
 
     if (threadIdx.x == 0) {
+        CONVBN_TRACE_POINT(0);
         for (int s = 0; s < 2; ++s) {
             mbar_init(&ctl->x_full[s], 32 * kWgLoaders); mbar_init(&ctl->x_empty[s], 2);
             mbar_init(&ctl->dz_full[s], 1); mbar_init(&ctl->dz_empty[s], 2);
@@ -448,6 +449,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
     tc_fence_after_sync();
     pdl_launch_dependents();       // only now: this CTA owns its tensor-memory columns
     const uint32_t tmem_base = ctl->tmem_base;
+    if (threadIdx.x == 0) CONVBN_TRACE_POINT(1);
 
     if (warp < kWgLoaders) {
         // ---------------- X row loaders ----------------
@@ -457,7 +459,9 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
         uint32_t ph = 0;
         bool ok = true;
         while (ok && win_next_chunk(cur, row_hi, g.h_out, kWgR, ck)) {
+            CONVBN_TRACE_T0();
             ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->x_empty[sb], ph ^ 1u, abort_flag));
+            if (threadIdx.x == 0) CONVBN_TRACE_ACC(12);
             if (!ok) break;
             win_fill_patch<C>(xs + (size_t)sb * g.xstrip_bytes, x, ck.img, ck.h0 * 2 - g.pad_h, (ck.rows - 1) * 2 + g.kh,
                               g.h_in, g.w_in, g.pad_w, g.pitch, (int)threadIdx.x, 32 * kWgLoaders, one_h16(g.f16));
@@ -507,10 +511,15 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
             uint32_t ph = 0;
             bool ok = true;
             while (ok && win_next_chunk(cur, row_hi, g.h_out, kWgR, ck)) {
-                if (!mbar_wait_bounded(&ctl->x_full[sb], ph, abort_flag) || !mbar_wait_bounded(&ctl->dz_full[sb], ph, abort_flag)) {
+                CONVBN_TRACE_T0();
+                const bool got_x = mbar_wait_bounded(&ctl->x_full[sb], ph, abort_flag);
+                if (e == 0) CONVBN_TRACE_ACC(13);
+                if (!got_x || !mbar_wait_bounded(&ctl->dz_full[sb], ph, abort_flag)) {
                     ok = false;
                     break;
                 }
+                if (e == 0) CONVBN_TRACE_ACC(14);          // (x and dZ together)
+                if (e == 0 && cur - ck.rows <= row_lo) CONVBN_TRACE_POINT(2);
                 tc_fence_after_sync();
                 const uint32_t xa = smem_u32(xs + (size_t)sb * g.xstrip_bytes), dza = smem_u32(dzs + (size_t)sb * dzstrip);
                 const int count = (ck.rows - 1) * 2 + g.kh;
@@ -532,6 +541,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
                 umma_commit(&ctl->dz_empty[sb]);
                 if (++sb == 2) { sb = 0; ph ^= 1u; }
             }
+            if (e == 0) CONVBN_TRACE_POINT(3);
             if (ok) umma_commit(&ctl->acc_done);
             else { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
         }
@@ -539,6 +549,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
         // ---------------- read-out (warp 8 = lanes 0-31 of tensor memory = window offsets m = 0 .. 31) ----------------
         const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->acc_done, 0, abort_flag));
         if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+        if (lane == 0) CONVBN_TRACE_POINT(4);
         if (ok) {
             tc_fence_after_sync();
             const int q = lane >> 2, c = lane & 3;
@@ -570,6 +581,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
     }
     tc_fence_before_sync();
     __syncthreads();
+    if (threadIdx.x == 0) CONVBN_TRACE_POINT(5);
     if (warp == kWgLoaders) tmem_dealloc(tmem_base, 512);
 }
 
