@@ -442,8 +442,7 @@ int run_conv_dgrad(const convbn_desc *d, const Problem &pb, const void *dz, cons
         LAUNCH("subpixel_weights", launch_subpixel_weights(pb, w, scale, w_scratch, st));
         LAUNCH("stem_dgrad", launch_umma_strip_conv(s, dz, w_scratch, nullptr, dx, st));
         *which = "umma-subpixel";
-    } else if (stem_path(d, pb) && stem_dgrad_eligible(pb) && !call_f16()) {
-        // (warp-level bf16 MMAs: a half call takes the direct kernel below instead)
+    } else if (stem_path(d, pb) && stem_dgrad_eligible(pb)) {
         LAUNCH("stem_dgrad", launch_stem_dgrad(pb, dz, w, scale, dx, st));
         *which = "stem-mma";
     } else if (grouped_path(d, pb) && grouped8_eligible(pb)) {

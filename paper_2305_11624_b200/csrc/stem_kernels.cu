@@ -182,7 +182,7 @@ cudaError_t launch_stem_expand_weights(const Problem &pb, const void *w, const f
 // applies the shifts once at the end, through a small shared-memory scratch: every A fragment is
 // loaded once per kernel row rather than once per tap, and 32 - (NU - 1) output pixels come out of
 // each 32-column window.
-template <int NU>      // taps per kernel row and class, rounded up to 1, 2, 4 or 8
+template <int NU, bool H>      // NU: taps per kernel row and class, rounded up to 1, 2, 4 or 8; H: IEEE-half storage, else bf16
 __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_in, int c_in, int h_out, int w_out,
                                                          int c_out, int kh, int kw, int stride_h, int stride_w,
                                                          int pad_h, int pad_w, const uint4 *__restrict__ dz,
@@ -200,11 +200,10 @@ __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_
         const int co = cb * 64 + which * 32 + 8 * t + 2 * k;
         uint32_t word = 0u;
         if (g < c_in) {
-            const float w0 = (s_vec ? s_vec[co] : 1.f) * __bfloat162float(w[((size_t)co * taps + tap) * c_in + g]);
+            const float w0 = (s_vec ? s_vec[co] : 1.f) * load_h16(w + ((size_t)co * taps + tap) * c_in + g, H ? 1 : 0);
             const float w1 =
-                (s_vec ? s_vec[co + 1] : 1.f) * __bfloat162float(w[((size_t)(co + 1) * taps + tap) * c_in + g]);
-            word = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(w0)) |
-                   ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(w1)) << 16);
+                (s_vec ? s_vec[co + 1] : 1.f) * load_h16(w + ((size_t)(co + 1) * taps + tap) * c_in + g, H ? 1 : 0);
+            word = pack2_t<H>(w0, w1);
         }
         wfrag[i] = word;
     }
@@ -287,10 +286,10 @@ __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_
                         }
 #pragma unroll
                         for (int tl = 0; tl < 2; ++tl) {
-                            mma_16x8x16_bf16(acc[u][tl], alo[tl][0].x, ahi[tl][0].x, alo[tl][1].x, ahi[tl][1].x, bf[0][0], bf[0][1]);
-                            mma_16x8x16_bf16(acc[u][tl], alo[tl][0].y, ahi[tl][0].y, alo[tl][1].y, ahi[tl][1].y, bf[1][0], bf[1][1]);
-                            mma_16x8x16_bf16(acc[u][tl], alo[tl][0].z, ahi[tl][0].z, alo[tl][1].z, ahi[tl][1].z, bf[2][0], bf[2][1]);
-                            mma_16x8x16_bf16(acc[u][tl], alo[tl][0].w, ahi[tl][0].w, alo[tl][1].w, ahi[tl][1].w, bf[3][0], bf[3][1]);
+                            mma_16x8x16_t<H>(acc[u][tl], alo[tl][0].x, ahi[tl][0].x, alo[tl][1].x, ahi[tl][1].x, bf[0][0], bf[0][1]);
+                            mma_16x8x16_t<H>(acc[u][tl], alo[tl][0].y, ahi[tl][0].y, alo[tl][1].y, ahi[tl][1].y, bf[1][0], bf[1][1]);
+                            mma_16x8x16_t<H>(acc[u][tl], alo[tl][0].z, ahi[tl][0].z, alo[tl][1].z, ahi[tl][1].z, bf[2][0], bf[2][1]);
+                            mma_16x8x16_t<H>(acc[u][tl], alo[tl][0].w, ahi[tl][0].w, alo[tl][1].w, ahi[tl][1].w, bf[3][0], bf[3][1]);
                         }
                     }
                 }
@@ -325,7 +324,7 @@ __global__ void __launch_bounds__(256) stem_dgrad_kernel(int n, int h_in, int w_
             __nv_bfloat16 *dst = dx + ((size_t)(img * h_in + h) * w_in + j * stride_w + b) * c_in;
 #pragma unroll
             for (int c = 0; c < 8; ++c)
-                if (c < c_in) dst[c] = __float2bfloat16_rn(res[c]);
+                if (c < c_in) reinterpret_cast<uint16_t *>(dst)[c] = pack1_h16(res[c], H ? 1 : 0);
         }
     }
 }
@@ -337,23 +336,22 @@ bool stem_dgrad_eligible(const Problem &pb) {
 cudaError_t launch_stem_dgrad(const Problem &pb, const void *dz, const void *w, const float *s_vec, void *dx,
                               cudaStream_t st) {
     const size_t smem = (size_t)pb.kh * pb.kw * (pb.c_out / 64) * 1024 + 8192;   // fragments + 1 KB per warp
+    const int nu = (pb.kw + pb.stride_w - 1) / pb.stride_w;    // taps per kernel row in the fullest class
+    const bool half = call_f16() != 0;
+    const void *fns[2][4] = {{(const void *)stem_dgrad_kernel<1, false>, (const void *)stem_dgrad_kernel<2, false>,
+                              (const void *)stem_dgrad_kernel<4, false>, (const void *)stem_dgrad_kernel<8, false>},
+                             {(const void *)stem_dgrad_kernel<1, true>, (const void *)stem_dgrad_kernel<2, true>,
+                              (const void *)stem_dgrad_kernel<4, true>, (const void *)stem_dgrad_kernel<8, true>}};
     static PerDevice attr;
     if (!attr.done[current_device_slot()]) {
-        cudaError_t e = cudaFuncSetAttribute(stem_dgrad_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(stem_dgrad_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(stem_dgrad_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(stem_dgrad_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
-        if (e != cudaSuccess) return e;
+        for (int h = 0; h < 2; ++h)
+            for (int i = 0; i < 4; ++i)
+                if (cudaError_t e = cudaFuncSetAttribute(fns[h][i], cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+                    e != cudaSuccess)
+                    return e;
         attr.done[current_device_slot()] = true;
     }
-    const int nu = (pb.kw + pb.stride_w - 1) / pb.stride_w;    // taps per kernel row in the fullest class
-    const void *fn = nu <= 1   ? (const void *)stem_dgrad_kernel<1>
-                     : nu <= 2 ? (const void *)stem_dgrad_kernel<2>
-                     : nu <= 4 ? (const void *)stem_dgrad_kernel<4>
-                               : (const void *)stem_dgrad_kernel<8>;
+    const void *fn = fns[half ? 1 : 0][nu <= 1 ? 0 : nu <= 2 ? 1 : nu <= 4 ? 2 : 3];
     int per_sm = 0, dev = 0, sms = 0;
     cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, 256, smem);
     if (e == cudaSuccess) e = cudaGetDevice(&dev);
@@ -363,15 +361,22 @@ cudaError_t launch_stem_dgrad(const Problem &pb, const void *dz, const void *w, 
     const long long passes = ((long long)pb.n * pb.h_in * pb.w_in + 255) / 256;
     const long long resident = (long long)per_sm * sms;        // one wave of persistent blocks
     const unsigned grid = (unsigned)(passes < resident ? passes : resident);
-#define CONVBN_STEM_DGRAD(NU_)                                                                                   \
-    stem_dgrad_kernel<NU_><<<grid, 256, smem, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.c_out, \
-                                                    pb.kh, pb.kw, pb.stride_h, pb.stride_w, pb.pad_h, pb.pad_w,   \
-                                                    (const uint4 *)dz, (const __nv_bfloat16 *)w, s_vec,           \
-                                                    (__nv_bfloat16 *)dx)
-    if (nu <= 1) CONVBN_STEM_DGRAD(1);
-    else if (nu <= 2) CONVBN_STEM_DGRAD(2);
-    else if (nu <= 4) CONVBN_STEM_DGRAD(4);
-    else CONVBN_STEM_DGRAD(8);
+#define CONVBN_STEM_DGRAD(NU_, H_)                                                                                    \
+    stem_dgrad_kernel<NU_, H_><<<grid, 256, smem, st>>>(pb.n, pb.h_in, pb.w_in, pb.c_in, pb.h_out, pb.w_out, pb.c_out, \
+                                                        pb.kh, pb.kw, pb.stride_h, pb.stride_w, pb.pad_h, pb.pad_w,   \
+                                                        (const uint4 *)dz, (const __nv_bfloat16 *)w, s_vec,           \
+                                                        (__nv_bfloat16 *)dx)
+    if (half) {
+        if (nu <= 1) CONVBN_STEM_DGRAD(1, true);
+        else if (nu <= 2) CONVBN_STEM_DGRAD(2, true);
+        else if (nu <= 4) CONVBN_STEM_DGRAD(4, true);
+        else CONVBN_STEM_DGRAD(8, true);
+    } else {
+        if (nu <= 1) CONVBN_STEM_DGRAD(1, false);
+        else if (nu <= 2) CONVBN_STEM_DGRAD(2, false);
+        else if (nu <= 4) CONVBN_STEM_DGRAD(4, false);
+        else CONVBN_STEM_DGRAD(8, false);
+    }
 #undef CONVBN_STEM_DGRAD
     return cudaGetLastError();
 }

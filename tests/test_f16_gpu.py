@@ -33,7 +33,7 @@ FALLBACK = [
     L("h_20_24", 2, 20, 11, 13, 24, 3, 3, stride=2, pad=1, dtype="f16", bias=True),
     L("h_groups2", 1, 12, 9, 9, 10, 3, 3, pad=1, groups=2, dtype="f16"),
     # stems beyond the window kernels: packed forward and weight gradient; backward data by the sub-pixel route
-    # (stride 2) or the direct kernel
+    # (stride 2, at most 4 channels) or warp-level MMAs
     L("h_stem_w528", 1, 3, 8, 528, 64, 7, 7, stride=2, pad=3, dtype="f16"),
     L("h_stem_w272", 2, 3, 8, 272, 64, 7, 7, stride=2, pad=3, dtype="f16", bias=True),
     L("h_stem5_s1", 1, 3, 32, 32, 64, 5, 5, stride=1, pad=2, dtype="f16"),
