@@ -1,4 +1,4 @@
-// Per-channel and elementwise kernels: on-the-fly reparameterisation (omega', b'), per-channel
+// Per-channel and elementwise kernels: omega' and b' formed from the current parameters at each call, per-channel
 // sums, the parameter-gradient epilogue of Tune mode, and the Eval-mode BatchNorm passes.
 #include <stdlib.h>
 
