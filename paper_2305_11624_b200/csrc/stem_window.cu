@@ -371,24 +371,28 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
 
 // ---- weight gradient of the same layers ---------------------------------------------------------------
 // domega'[co][r][q][c] = sum over images and output pixels of dZ[ho][wo][co] X[2 ho + r][2 wo + q][c]  (Sec. 3.2.1;
-// Table 2, Tune row), with the same zero-bordered 4-channel rows in shared memory.  For one input row the
-// A operand is MN-major without swizzle: element (m, k) with m = 4 q + c and k = wo sits at  start + 2 m + 16 k,
-// i.e. the contraction runs along the output pixels of a row and the 128 M rows are window offsets (the first
-// kw x 4 are the taps, the rest is ignored).  The B operand is the dZ row(s) that meet this input row, [wo][co]
-// in 128-byte-swizzled rows: input row 2 ho + r serves ceil(kh / 2) or floor(kh / 2) output rows at once, which
-// lie one after the other in the chunk's dZ buffer, so ONE MMA of N = 64 x (rows) updates all their taps:
-// accumulator column block j of parity class e = r & 1 holds tap r = e + 2 (T_e - 1 - j).
-// Channel slot 3 of every padded pixel holds 1.0 (C <= 3), so accumulator row m = 3 of tap 0 is sum dZ.
-// Each CTA accumulates its contiguous range of output rows in tensor memory and writes one fp32 partial
-// [k][co] plus one row of sums; the fused epilogue kernel adds the CTAs' partials in fixed order.
+// Table 2, Tune row), with the same zero-bordered 4-channel rows in shared memory.  The contraction runs along the
+// output pixels of a row (K = 16 pixels per MMA).  The M side is dZ: a row [wo][co] in 128-byte-swizzled rows is an
+// MN-major operand of 64 rows (the channels), and two consecutive output rows of the chunk's dZ buffer make the
+// 128 rows of one MMA.  The N side is the window of one input row, MN-major without swizzle: element (n, k) with
+// n = 4 q + c and k = wo sits at  start + 2 n + 16 k, so 32 columns are the taps q = 0 .. 7 of all four channel
+// slots.  Input row 2 ho + r is tap row r of output row ho and tap row r - 2 of output row ho + 1: with the
+// accumulators of parity class e = r & 1 laid out as column blocks j of 32, lanes 0 - 63 of block j hold tap
+// r = e + 2 j (from the even rows of the chunk) and lanes 64 - 127 hold tap r = e + 2 (j - 1) (from the odd rows),
+// so ONE MMA serves both rows.  Block T_e of the lower lanes and block 0 of the upper lanes collect products that
+// belong to no tap and are never read.  Channel slot 3 of every padded pixel holds 1.0 (C <= 3), so column n = 3
+// of tap 0 is sum dZ.  Each CTA accumulates its contiguous range of output rows in tensor memory, adds the two
+// lane halves through shared memory and writes one fp32 partial [k][co] plus one row of sums; the fused epilogue
+// kernel adds the CTAs' partials in fixed order.
 constexpr int kWgR = 4;                  // output rows per chunk
 constexpr int kWgLoaders = 8;
-constexpr int kWgThreads = 32 * (kWgLoaders + 4);   // warps 0-7 X loaders, 8 tensor memory + read-out, 9 dZ producer, 10-11 issuers
+constexpr int kWgThreads = 32 * (kWgLoaders + 4);   // warps 0-7 X loaders, 8 tensor memory, 9 dZ producer, 10-11 issuers; 8-11 read out
 
 struct WinWgrad {
     int n, h_in, w_in, h_out, w_out, c_out, kh, kw, pad_h, pad_w;
     int pitch, ksteps, T0, T1, kdim;
     uint32_t xstrip_bytes, dzrow_bytes;
+    uint32_t work_bytes;   // operand buffers, at least the size of the read-out's exchange area
     long long total_rows;
     int f16;               // 16-bit storage type: 0 bf16, 1 IEEE half
 };
@@ -411,7 +415,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
     uint8_t *xs = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *dzs = xs + 2 * (size_t)g.xstrip_bytes;
     const uint32_t dzstrip = kWgR * g.dzrow_bytes;
-    uint8_t *zeros = dzs + 2 * (size_t)dzstrip;                 // 16 zero rows of 128 bytes
+    uint8_t *zeros = xs + g.work_bytes;                        // 16 zero rows of 128 bytes
     WinWgCtl *ctl = (WinWgCtl *)(zeros + 2048);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &ctl->abort_flag;
@@ -467,6 +471,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
                               g.h_in, g.w_in, g.pad_w, g.pitch, (int)threadIdx.x, 32 * kWgLoaders, one_h16(g.f16));
             fence_proxy_async_smem();
             mbar_arrive(&ctl->x_full[sb]);
+            if (threadIdx.x == 0 && cur - ck.rows <= row_lo) CONVBN_TRACE_POINT(6);
             if (++sb == 2) { sb = 0; ph ^= 1u; }
         }
         if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
@@ -480,10 +485,12 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
             bool ok = true;
             while (ok && win_next_chunk(cur, row_hi, g.h_out, kWgR, ck)) {
                 if (!mbar_wait_bounded(&ctl->dz_empty[sb], ph ^ 1u, abort_flag)) { ok = false; break; }
-                mbar_arrive_expect_tx(&ctl->dz_full[sb], (uint32_t)ck.rows * g.dzrow_bytes);
-                for (int i = 0; i < ck.rows; ++i)
+                // an odd chunk is completed by a row of zeros: a box beyond the last row of the tensor (the MMAs take rows in pairs)
+                const int boxes = (ck.rows + 1) & ~1;
+                mbar_arrive_expect_tx(&ctl->dz_full[sb], (uint32_t)boxes * g.dzrow_bytes);
+                for (int i = 0; i < boxes; ++i)
                     tma_load_3d(dzs + (size_t)sb * dzstrip + (size_t)i * g.dzrow_bytes, &tm_dz, &ctl->dz_full[sb], 0, 0,
-                                ck.img * g.h_out + ck.h0 + i);
+                                i < ck.rows ? ck.img * g.h_out + ck.h0 + i : g.n * g.h_out);
                 ++issued;
                 if (++sb == 2) { sb = 0; ph ^= 1u; }
             }
@@ -499,12 +506,13 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
         const int e = warp - (kWgLoaders + 2), Te = e ? g.T1 : g.T0;
         if (elect_one()) {
             const uint32_t acc = tmem_base + (uint32_t)e * 256u;
-            // A: MN-major, no swizzle: 8 M elements per 16 bytes, next 8 M elements 16 bytes on, next 8 pixels 128 bytes on
-            const uint32_t a_hi = (16u >> 4) | (1u << 14), a_lbo = (128u >> 4) << 16;
-            const uint32_t b_hi = smem_desc_hi_sw128(1024);
-            // all accumulator columns of this class start from zero: one MMA against 16 zero rows (block stride 0)
-            umma_bf16_ss_halves<false>(acc, ((smem_u32(xs) >> 4) & 0x3FFFu) | a_lbo, a_hi, smem_desc_lo(smem_u32(zeros), 0), b_hi,
-                                       idesc_h16_f32(128, 64 * Te, 1, 1, g.f16));
+            // window (N side): MN-major, no swizzle: 8 elements per 16 bytes, next 8 elements 16 bytes on, next 8 pixels 128 bytes on
+            const uint32_t w_hi = (16u >> 4) | (1u << 14), w_lbo = (128u >> 4) << 16;
+            const uint32_t z_hi = smem_desc_hi_sw128(1024);       // dZ (M side): 8 pixels = 1024 bytes
+            // all accumulator columns of this class start from zero: one MMA with 128 zero rows (block stride 0) on the M side
+            umma_bf16_ss_halves<false>(acc, smem_desc_lo(smem_u32(zeros), 0), z_hi, ((smem_u32(xs) >> 4) & 0x3FFFu) | w_lbo, w_hi,
+                                       idesc_h16_f32(128, 32 * (Te + 1), 1, 1, g.f16));
+            const uint32_t idesc = idesc_h16_f32(128, 32, 1, 1, g.f16);
             long long cur = row_lo;
             WinChunk ck;
             int sb = 0;
@@ -524,18 +532,17 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
                 const uint32_t xa = smem_u32(xs + (size_t)sb * g.xstrip_bytes), dza = smem_u32(dzs + (size_t)sb * dzstrip);
                 const int count = (ck.rows - 1) * 2 + g.kh;
                 for (int pr = e; pr < count; pr += 2) {
-                    const int i_max = (pr - e) >> 1;
-                    int t_lo = i_max - ck.rows + 1, t_hi = i_max;
-                    if (t_lo < 0) t_lo = 0;
-                    if (t_hi > Te - 1) t_hi = Te - 1;
-                    if (t_lo > t_hi) continue;
-                    const int nblk = t_hi - t_lo + 1, i_lo = i_max - t_hi, cb_lo = Te - 1 - t_hi;
-                    const uint32_t idesc = idesc_h16_f32(128, 64 * nblk, 1, 1, g.f16);
-                    const uint32_t d = acc + 64u * (uint32_t)cb_lo;
-                    uint32_t a_lo = (((xa + (uint32_t)pr * (uint32_t)g.pitch) >> 4) & 0x3FFFu) | a_lbo;
-                    uint32_t b_lo = smem_desc_lo(dza + (uint32_t)i_lo * g.dzrow_bytes, g.dzrow_bytes);
-                    for (int k = 0; k < g.ksteps; ++k, a_lo += 16u, b_lo += 128u)     // 16 pixels: 256 / 2048 bytes
-                        umma_bf16_ss_halves<true>(d, a_lo, a_hi, b_lo, b_hi, idesc);
+                    const int half_idx = (pr - e) >> 1;       // input row pr is tap row e + 2 (half_idx - i) of output row i
+                    for (int i = 0; i < ck.rows; i += 2) {
+                        const int t = half_idx - i;           // tap index of row i; row i + 1 (if any) takes tap t - 1
+                        const bool lower = t >= 0 && t < Te, upper = i + 1 < ck.rows && t >= 1 && t <= Te;
+                        if (!lower && !upper) continue;
+                        const uint32_t d = acc + 32u * (uint32_t)t;
+                        uint32_t z_lo = smem_desc_lo(dza + (uint32_t)i * g.dzrow_bytes, g.dzrow_bytes);
+                        uint32_t w_lo = (((xa + (uint32_t)pr * (uint32_t)g.pitch) >> 4) & 0x3FFFu) | w_lbo;
+                        for (int k = 0; k < g.ksteps; ++k, z_lo += 128u, w_lo += 16u)     // 16 pixels: 2048 / 256 bytes
+                            umma_bf16_ss_halves<true>(d, z_lo, z_hi, w_lo, w_hi, idesc);
+                    }
                 }
                 umma_commit(&ctl->x_empty[sb]);
                 umma_commit(&ctl->dz_empty[sb]);
@@ -545,37 +552,49 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
             if (ok) umma_commit(&ctl->acc_done);
             else { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
         }
-    } else {
-        // ---------------- read-out (warp 8 = lanes 0-31 of tensor memory = window offsets m = 0 .. 31) ----------------
-        const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->acc_done, 0, abort_flag));
-        if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
-        if (lane == 0) CONVBN_TRACE_POINT(4);
-        if (ok) {
+    }
+    // ---------------- read-out: warps 8 - 11 own lanes 0-31, 32-63, 64-95, 96-127 of tensor memory (lane = output channel,
+    // lower half from the even rows of the chunks, upper half from the odd rows).  The halves are added through shared
+    // memory: the lower warps hand over their odd tap rows and finish the even ones, the upper warps the reverse ----------------
+    const int rw = warp - kWgLoaders;
+    float *ex = (float *)xs;                   // exchange area [tap][n][co]: the operand buffers are free once acc_done is complete
+    const bool up_half = rw >= 2;
+    const int co = (rw & 1) * 32 + lane;
+    const uint32_t t_lane = tmem_base + ((uint32_t)((rw < 0 ? 0 : rw) * 32) << 16);
+    bool rd_ok = false;
+    if (rw >= 0) {
+        rd_ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->acc_done, 0, abort_flag));
+        if (!rd_ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
+        if (rw == 0 && lane == 0) CONVBN_TRACE_POINT(4);
+        if (rd_ok) {
             tc_fence_after_sync();
-            const int q = lane >> 2, c = lane & 3;
-            const bool tap_ok = q < g.kw && c < C;
-            for (int e = 0; e < 2; ++e) {
-                const int Te = e ? g.T1 : g.T0;
-                for (int cbk = 0; cbk < Te; ++cbk) {
-                    const int r = e + 2 * (Te - 1 - cbk);
-                    const int k = (r * g.kw + q) * C + c;
-                    float *orow = partials + ((size_t)blockIdx.x * g.kdim + (tap_ok ? k : 0)) * 64;
-                    float *brow = bsum + (size_t)blockIdx.x * 64;
-                    const bool sum_row = C < 4 && r == 0 && lane == 3;
-#pragma unroll 1
-                    for (int c0 = 0; c0 < 64; c0 += 32) {
-                        uint32_t v[32];
-                        tmem_ld_32x32(tmem_base + (uint32_t)(e * 256 + cbk * 64 + c0), v);
-                        tmem_ld_wait();
-                        if (tap_ok) {
+            const int e = up_half ? 0 : 1, Te = e ? g.T1 : g.T0;       // the class this half gives away
+            for (int t = 0; t < Te; ++t) {         // the upper lanes keep tap t in column block t + 1
+                uint32_t v[32];
+                tmem_ld_32x32(t_lane + (uint32_t)(e * 256 + 32 * (t + (up_half ? 1 : 0))), v);
+                tmem_ld_wait();
+                float *dst = ex + (size_t)((e ? g.T0 : 0) + t) * (32 * 64) + co;
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4) *(uint4 *)(orow + c0 + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                        } else if (sum_row) {
+                for (int n = 0; n < 32; ++n) dst[n * 64] = __uint_as_float(v[n]);
+            }
+        }
+    }
+    __syncthreads();                           // every warp: the halves that were given away are in the exchange area
+    if (rw >= 0 && rd_ok && !*abort_flag) {
+        const int e = up_half ? 1 : 0, Te = e ? g.T1 : g.T0;           // the class this half finishes
+        float *prow = partials + (size_t)blockIdx.x * g.kdim * 64 + co;
+        for (int t = 0; t < Te; ++t) {
+            const int r = e + 2 * t;
+            uint32_t v[32];
+            tmem_ld_32x32(t_lane + (uint32_t)(e * 256 + 32 * (t + (up_half ? 1 : 0))), v);
+            tmem_ld_wait();
+            const float *other = ex + (size_t)((e ? g.T0 : 0) + t) * (32 * 64) + co;
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4) *(uint4 *)(brow + c0 + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                        }
-                    }
-                }
+            for (int n = 0; n < 32; ++n) {
+                const int q = n >> 2, c = n & 3;
+                const float sum = __uint_as_float(v[n]) + other[n * 64];
+                if (q < g.kw && c < C) prow[(size_t)((r * g.kw + q) * C + c) * 64] = sum;
+                else if (C < 4 && r == 0 && n == 3) bsum[(size_t)blockIdx.x * 64 + co] = sum;      // sum dZ
             }
         }
     }
@@ -641,7 +660,7 @@ cudaError_t launch_window_c(int c_in, const CUtensorMap &tout, const WinGemm &g,
 bool stem_window_eligible(const Problem &pb) { return plan_window(pb).ok; }
 
 namespace {
-struct WinWgPlan { bool ok = false; int pitch = 0, ksteps = 0; uint32_t xstrip = 0, dzrow = 0; size_t smem = 0; };
+struct WinWgPlan { bool ok = false; int pitch = 0, ksteps = 0; uint32_t xstrip = 0, dzrow = 0, work = 0; size_t smem = 0; };
 WinWgPlan plan_window_wgrad(const Problem &pb) {
     WinWgPlan pl;
     if (!plan_window(pb).ok || pb.c_in > 3 || pb.c_out != 64 || pb.kh < 2 || pb.kh > 8 || pb.w_out > 256) return pl;
@@ -649,7 +668,9 @@ WinWgPlan plan_window_wgrad(const Problem &pb) {
     pl.ksteps = (pb.w_out + 15) / 16;
     pl.xstrip = (uint32_t)((((size_t)(kWgR - 1) * 2 + pb.kh) * pl.pitch + kWinSlack + 1023) / 1024 * 1024);
     pl.dzrow = (uint32_t)pl.ksteps * 16 * 128;
-    pl.smem = 1024 + 2 * (size_t)pl.xstrip + 2 * (size_t)kWgR * pl.dzrow + 2048 + sizeof(WinWgCtl) + 64;
+    pl.work = 2 * pl.xstrip + 2 * (uint32_t)kWgR * pl.dzrow;
+    if (pl.work < (uint32_t)pb.kh * 8192u) pl.work = (uint32_t)pb.kh * 8192u;       // the read-out's exchange area: kh taps x 32 x 64 floats
+    pl.smem = 1024 + (size_t)pl.work + 2048 + sizeof(WinWgCtl) + 64;
     pl.ok = pl.smem <= 226 * 1024;
     return pl;
 }
@@ -680,7 +701,7 @@ cudaError_t launch_stem_window_wgrad(const Problem &pb, const void *dz, const vo
     WinWgrad g;
     g.n = pb.n; g.h_in = pb.h_in; g.w_in = pb.w_in; g.h_out = pb.h_out; g.w_out = pb.w_out; g.c_out = pb.c_out;
     g.kh = pb.kh; g.kw = pb.kw; g.pad_h = pb.pad_h; g.pad_w = pb.pad_w; g.pitch = pl.pitch; g.ksteps = pl.ksteps;
-    g.T0 = (pb.kh + 1) / 2; g.T1 = pb.kh / 2; g.kdim = pb.kdim; g.xstrip_bytes = pl.xstrip; g.dzrow_bytes = pl.dzrow;
+    g.T0 = (pb.kh + 1) / 2; g.T1 = pb.kh / 2; g.kdim = pb.kdim; g.xstrip_bytes = pl.xstrip; g.dzrow_bytes = pl.dzrow; g.work_bytes = pl.work;
     g.total_rows = (long long)pb.n * pb.h_out;
     g.f16 = call_f16();
     CUtensorMap tdz;
