@@ -288,6 +288,22 @@ __device__ __forceinline__ uint32_t smem_desc_lo(uint32_t smem_addr, uint32_t lb
 __device__ __forceinline__ uint32_t smem_desc_hi_sw128(uint32_t sbo_bytes) {
     return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);
 }
+// D[tmem] += A[tmem] * B[smem]: the A operand (128 rows = lanes, 16-bit elements, two consecutive K elements per
+// 32-bit column: 8 columns per K = 16) is read from tensor memory, B through its shared-memory descriptor (halves).
+__device__ __forceinline__ void umma_h16_ts_acc(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tmov.b64 db, {%2, %3};\n\t"
+        "setp.eq.u32 p, %0, %0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc)
+        : "memory");
+}
+// 32 lanes x 8 consecutive 32-bit columns: thread i of the warp writes lane (base lane + i).
+__device__ __forceinline__ void tmem_st_32x32_x8(uint32_t taddr, const uint32_t (&v)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
+}
 // D[tmem] (+)= A[smem] * B[smem] with the descriptors given as halves; ACC = false overwrites D.
 template <bool ACC>
 __device__ __forceinline__ void umma_bf16_ss_halves(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,

@@ -385,12 +385,17 @@ __global__ void __launch_bounds__(kWinThreads) stem_window_fwd_kernel(const __gr
 // lane halves through shared memory and writes one fp32 partial [k][co] plus one row of sums; the fused epilogue
 // kernel adds the CTAs' partials in fixed order.
 constexpr int kWgR = 4;                  // output rows per chunk
-constexpr int kWgLoaders = 8;
-constexpr int kWgThreads = 32 * (kWgLoaders + 4);   // warps 0-7 X loaders, 8 tensor memory, 9 dZ producer, 10-11 issuers; 8-11 read out
+constexpr int kWgLoaders = 8;            // (a multiple of 4: the warps behind them own lane quarters 0, 1, 2, 3 of tensor memory in turn)
+constexpr int kWgMovers = 4;             // one warp per lane quarter
+// warps 0-7 X loaders, 8 tensor memory, 9 dZ producer, 10-11 issuers (8-11 read out), 12-15 dZ rows into tensor memory
+constexpr int kWgThreads = 32 * (kWgLoaders + 4 + kWgMovers);
+constexpr int kWgAccCols = 320;          // accumulators: two parity classes x (4 + 1) blocks of 32 columns
+constexpr int kWgMaxSlots = 4;           // ring of dZ row pairs in the remaining 192 columns
 
 struct WinWgrad {
     int n, h_in, w_in, h_out, w_out, c_out, kh, kw, pad_h, pad_w;
     int pitch, ksteps, T0, T1, kdim;
+    int nslots;            // dZ row pairs that fit tensor memory beside the accumulators (8 ksteps columns each)
     uint32_t xstrip_bytes, dzrow_bytes;
     uint32_t work_bytes;   // operand buffers, at least the size of the read-out's exchange area
     long long total_rows;
@@ -398,7 +403,7 @@ struct WinWgrad {
 };
 
 struct WinWgCtl {
-    uint64_t x_full[2], x_empty[2], dz_full[2], dz_empty[2], acc_done;
+    uint64_t x_full[2], x_empty[2], dz_full[2], dz_empty[2], a_full[kWgMaxSlots], a_empty[kWgMaxSlots], acc_done;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -425,8 +430,9 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
         CONVBN_TRACE_POINT(0);
         for (int s = 0; s < 2; ++s) {
             mbar_init(&ctl->x_full[s], 32 * kWgLoaders); mbar_init(&ctl->x_empty[s], 2);
-            mbar_init(&ctl->dz_full[s], 1); mbar_init(&ctl->dz_empty[s], 2);
+            mbar_init(&ctl->dz_full[s], 1); mbar_init(&ctl->dz_empty[s], kWgMovers);
         }
+        for (int s = 0; s < kWgMaxSlots; ++s) { mbar_init(&ctl->a_full[s], kWgMovers); mbar_init(&ctl->a_empty[s], 2); }
         mbar_init(&ctl->acc_done, 2);
         ctl->abort_flag = 0;
         fence_barrier_init();
@@ -453,6 +459,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
     tc_fence_after_sync();
     pdl_launch_dependents();       // only now: this CTA owns its tensor-memory columns
     const uint32_t tmem_base = ctl->tmem_base;
+    const uint32_t slot_cols = 8u * (uint32_t)g.ksteps;        // one dZ row pair: 8 columns per 16 pixels
     if (threadIdx.x == 0) CONVBN_TRACE_POINT(1);
 
     if (warp < kWgLoaders) {
@@ -485,12 +492,10 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
             bool ok = true;
             while (ok && win_next_chunk(cur, row_hi, g.h_out, kWgR, ck)) {
                 if (!mbar_wait_bounded(&ctl->dz_empty[sb], ph ^ 1u, abort_flag)) { ok = false; break; }
-                // an odd chunk is completed by a row of zeros: a box beyond the last row of the tensor (the MMAs take rows in pairs)
-                const int boxes = (ck.rows + 1) & ~1;
-                mbar_arrive_expect_tx(&ctl->dz_full[sb], (uint32_t)boxes * g.dzrow_bytes);
-                for (int i = 0; i < boxes; ++i)
+                mbar_arrive_expect_tx(&ctl->dz_full[sb], (uint32_t)ck.rows * g.dzrow_bytes);
+                for (int i = 0; i < ck.rows; ++i)
                     tma_load_3d(dzs + (size_t)sb * dzstrip + (size_t)i * g.dzrow_bytes, &tm_dz, &ctl->dz_full[sb], 0, 0,
-                                i < ck.rows ? ck.img * g.h_out + ck.h0 + i : g.n * g.h_out);
+                                ck.img * g.h_out + ck.h0 + i);
                 ++issued;
                 if (++sb == 2) { sb = 0; ph ^= 1u; }
             }
@@ -501,51 +506,99 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
                     mbar_wait_bounded(&ctl->dz_full[j & 1], (uint32_t)(j >> 1) & 1u, nullptr, 200000000ull);
             }
         }
+    } else if (warp >= kWgLoaders + 4) {
+        // ---------------- dZ rows into tensor memory: the M side of the MMAs.  Lane m of a pair's tile is channel m & 63 of
+        // the pair's row m >> 6; 16 pixels are 8 columns of two 16-bit elements.  (Read from tensor memory, the tile costs
+        // the MMAs no shared-memory bandwidth: every pair meets up to 2 (T + 1) input rows.) ----------------
+        const int q4 = (warp - (kWgLoaders + 4)) & 3, group = (warp - (kWgLoaders + 4)) >> 2;
+        const int m = 32 * q4 + lane, half = m >> 6, co = m & 63;
+        const uint32_t t_lane = tmem_base + ((uint32_t)(32 * q4) << 16) + (uint32_t)kWgAccCols;
+        const uint32_t in_row = (uint32_t)(co & 7) * 2u;       // byte of the channel inside its 16-byte chunk
+        long long cur = row_lo;
+        WinChunk ck;
+        int sb = 0, slot = 0;
+        uint32_t ph = 0, aph = 0;
+        bool ok = true;
+        while (ok && win_next_chunk(cur, row_hi, g.h_out, kWgR, ck)) {
+            { CONVBN_TRACE_T0();
+            ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->dz_full[sb], ph, abort_flag));
+            if (q4 == 0 && group == 0 && lane == 0) CONVBN_TRACE_ACC(15); }
+            if (!ok) break;
+            for (int i = 0; i < ck.rows; i += 2) {
+                { CONVBN_TRACE_T0();
+                ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->a_empty[slot], aph ^ 1u, abort_flag));
+                if (q4 == 0 && group == 0 && lane == 0) CONVBN_TRACE_ACC(10); }
+                if (!ok) break;
+                tc_fence_after_sync();
+                const bool have = i + half < ck.rows;           // an odd last pair has no second row: zeros
+                const uint8_t *rowb = dzs + (size_t)sb * dzstrip + (size_t)(have ? i + half : 0) * g.dzrow_bytes;
+                const uint32_t t0 = t_lane + (uint32_t)slot * slot_cols;
+                for (int k = group; k < g.ksteps; k += kWgMovers / 4) {
+                    uint32_t v[8];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        // pixels 16 k + 2 c and the next one; rows are 128-byte swizzled: chunk (co / 8) ^ (pixel & 7)
+                        const uint32_t p0 = (uint32_t)(16 * k + 2 * c);
+                        const uint32_t lo = *(const uint16_t *)(rowb + p0 * 128u + ((((uint32_t)(co >> 3) ^ (p0 & 7u)) & 7u) << 4) + in_row);
+                        const uint32_t hi = *(const uint16_t *)(rowb + (p0 + 1u) * 128u + ((((uint32_t)(co >> 3) ^ ((p0 + 1u) & 7u)) & 7u) << 4) + in_row);
+                        v[c] = have ? (lo | (hi << 16)) : 0u;
+                    }
+                    tmem_st_32x32_x8(t0 + 8u * (uint32_t)k, v);
+                }
+                tmem_st_wait();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->a_full[slot]);
+                if (++slot == g.nslots) { slot = 0; aph ^= 1u; }
+            }
+            if (!ok) break;
+            __syncwarp();                                       // the chunk's rows are in tensor memory: the buffer may be refilled
+            if (lane == 0) mbar_arrive(&ctl->dz_empty[sb]);
+            if (++sb == 2) { sb = 0; ph ^= 1u; }
+        }
+        if (!ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
     } else if (warp >= kWgLoaders + 2) {
         // ---------------- MMA issuers: one warp for the even input rows of a patch, one for the odd ones ----------------
         const int e = warp - (kWgLoaders + 2), Te = e ? g.T1 : g.T0;
         if (elect_one()) {
-            const uint32_t acc = tmem_base + (uint32_t)e * 256u;
+            const uint32_t acc = tmem_base + (uint32_t)e * (kWgAccCols / 2);
             // window (N side): MN-major, no swizzle: 8 elements per 16 bytes, next 8 elements 16 bytes on, next 8 pixels 128 bytes on
             const uint32_t w_hi = (16u >> 4) | (1u << 14), w_lbo = (128u >> 4) << 16;
-            const uint32_t z_hi = smem_desc_hi_sw128(1024);       // dZ (M side): 8 pixels = 1024 bytes
-            // all accumulator columns of this class start from zero: one MMA with 128 zero rows (block stride 0) on the M side
-            umma_bf16_ss_halves<false>(acc, smem_desc_lo(smem_u32(zeros), 0), z_hi, ((smem_u32(xs) >> 4) & 0x3FFFu) | w_lbo, w_hi,
-                                       idesc_h16_f32(128, 32 * (Te + 1), 1, 1, g.f16));
-            const uint32_t idesc = idesc_h16_f32(128, 32, 1, 1, g.f16);
+            // all accumulator columns of this class start from zero: one MMA with 128 zero rows (shared memory, block stride 0) on the M side
+            umma_bf16_ss_halves<false>(acc, smem_desc_lo(smem_u32(zeros), 0), smem_desc_hi_sw128(1024),
+                                       ((smem_u32(xs) >> 4) & 0x3FFFu) | w_lbo, w_hi, idesc_h16_f32(128, 32 * (Te + 1), 1, 1, g.f16));
+            const uint32_t idesc = idesc_h16_f32(128, 32, 0, 1, g.f16);       // M side in tensor memory (K-major), window MN-major
             long long cur = row_lo;
             WinChunk ck;
-            int sb = 0;
-            uint32_t ph = 0;
+            int sb = 0, slot = 0;
+            uint32_t ph = 0, aph = 0;
             bool ok = true;
             while (ok && win_next_chunk(cur, row_hi, g.h_out, kWgR, ck)) {
                 CONVBN_TRACE_T0();
-                const bool got_x = mbar_wait_bounded(&ctl->x_full[sb], ph, abort_flag);
+                if (!mbar_wait_bounded(&ctl->x_full[sb], ph, abort_flag)) { ok = false; break; }
                 if (e == 0) CONVBN_TRACE_ACC(13);
-                if (!got_x || !mbar_wait_bounded(&ctl->dz_full[sb], ph, abort_flag)) {
-                    ok = false;
-                    break;
-                }
-                if (e == 0) CONVBN_TRACE_ACC(14);          // (x and dZ together)
-                if (e == 0 && cur - ck.rows <= row_lo) CONVBN_TRACE_POINT(2);
-                tc_fence_after_sync();
-                const uint32_t xa = smem_u32(xs + (size_t)sb * g.xstrip_bytes), dza = smem_u32(dzs + (size_t)sb * dzstrip);
+                const uint32_t xa = smem_u32(xs + (size_t)sb * g.xstrip_bytes);
                 const int count = (ck.rows - 1) * 2 + g.kh;
-                for (int pr = e; pr < count; pr += 2) {
-                    const int half_idx = (pr - e) >> 1;       // input row pr is tap row e + 2 (half_idx - i) of output row i
-                    for (int i = 0; i < ck.rows; i += 2) {
-                        const int t = half_idx - i;           // tap index of row i; row i + 1 (if any) takes tap t - 1
+                for (int i = 0; i < ck.rows; i += 2) {
+                    if (!mbar_wait_bounded(&ctl->a_full[slot], aph, abort_flag)) { ok = false; break; }
+                    if (e == 0) CONVBN_TRACE_ACC(14);          // (x and dZ together)
+                    if (e == 0 && i == 0 && cur - ck.rows <= row_lo) CONVBN_TRACE_POINT(2);
+                    tc_fence_after_sync();
+                    const uint32_t a0 = tmem_base + (uint32_t)kWgAccCols + (uint32_t)slot * slot_cols;
+                    for (int pr = e; pr < count; pr += 2) {
+                        const int t = ((pr - e) >> 1) - i;    // input row pr is tap row e + 2 t of output row i and e + 2 (t - 1) of row i + 1
                         const bool lower = t >= 0 && t < Te, upper = i + 1 < ck.rows && t >= 1 && t <= Te;
                         if (!lower && !upper) continue;
                         const uint32_t d = acc + 32u * (uint32_t)t;
-                        uint32_t z_lo = smem_desc_lo(dza + (uint32_t)i * g.dzrow_bytes, g.dzrow_bytes);
                         uint32_t w_lo = (((xa + (uint32_t)pr * (uint32_t)g.pitch) >> 4) & 0x3FFFu) | w_lbo;
-                        for (int k = 0; k < g.ksteps; ++k, z_lo += 128u, w_lo += 16u)     // 16 pixels: 2048 / 256 bytes
-                            umma_bf16_ss_halves<true>(d, z_lo, z_hi, w_lo, w_hi, idesc);
+                        for (int k = 0; k < g.ksteps; ++k, w_lo += 16u)     // 16 pixels: 256 bytes of window, 8 columns of dZ
+                            umma_h16_ts_acc(d, a0 + 8u * (uint32_t)k, w_lo, w_hi, idesc);
                     }
+                    umma_commit(&ctl->a_empty[slot]);
+                    if (++slot == g.nslots) { slot = 0; aph ^= 1u; }
                 }
+                if (!ok) break;
                 umma_commit(&ctl->x_empty[sb]);
-                umma_commit(&ctl->dz_empty[sb]);
                 if (++sb == 2) { sb = 0; ph ^= 1u; }
             }
             if (e == 0) CONVBN_TRACE_POINT(3);
@@ -557,12 +610,13 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
     // lower half from the even rows of the chunks, upper half from the odd rows).  The halves are added through shared
     // memory: the lower warps hand over their odd tap rows and finish the even ones, the upper warps the reverse ----------------
     const int rw = warp - kWgLoaders;
+    const bool reader = rw >= 0 && rw < 4;
     float *ex = (float *)xs;                   // exchange area [tap][n][co]: the operand buffers are free once acc_done is complete
     const bool up_half = rw >= 2;
     const int co = (rw & 1) * 32 + lane;
-    const uint32_t t_lane = tmem_base + ((uint32_t)((rw < 0 ? 0 : rw) * 32) << 16);
+    const uint32_t t_lane = tmem_base + ((uint32_t)((reader ? rw : 0) * 32) << 16);
     bool rd_ok = false;
-    if (rw >= 0) {
+    if (reader) {
         rd_ok = __all_sync(0xffffffffu, mbar_wait_bounded(&ctl->acc_done, 0, abort_flag));
         if (!rd_ok && lane == 0) { atomicOr(err, ERRW_TIMEOUT); ctl->abort_flag = 1; }
         if (rw == 0 && lane == 0) CONVBN_TRACE_POINT(4);
@@ -571,7 +625,7 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
             const int e = up_half ? 0 : 1, Te = e ? g.T1 : g.T0;       // the class this half gives away
             for (int t = 0; t < Te; ++t) {         // the upper lanes keep tap t in column block t + 1
                 uint32_t v[32];
-                tmem_ld_32x32(t_lane + (uint32_t)(e * 256 + 32 * (t + (up_half ? 1 : 0))), v);
+                tmem_ld_32x32(t_lane + (uint32_t)(e * (kWgAccCols / 2) + 32 * (t + (up_half ? 1 : 0))), v);
                 tmem_ld_wait();
                 float *dst = ex + (size_t)((e ? g.T0 : 0) + t) * (32 * 64) + co;
 #pragma unroll
@@ -580,13 +634,13 @@ __global__ void __launch_bounds__(kWgThreads) stem_window_wgrad_kernel(const __g
         }
     }
     __syncthreads();                           // every warp: the halves that were given away are in the exchange area
-    if (rw >= 0 && rd_ok && !*abort_flag) {
+    if (reader && rd_ok && !*abort_flag) {
         const int e = up_half ? 1 : 0, Te = e ? g.T1 : g.T0;           // the class this half finishes
         float *prow = partials + (size_t)blockIdx.x * g.kdim * 64 + co;
         for (int t = 0; t < Te; ++t) {
             const int r = e + 2 * t;
             uint32_t v[32];
-            tmem_ld_32x32(t_lane + (uint32_t)(e * 256 + 32 * (t + (up_half ? 1 : 0))), v);
+            tmem_ld_32x32(t_lane + (uint32_t)(e * (kWgAccCols / 2) + 32 * (t + (up_half ? 1 : 0))), v);
             tmem_ld_wait();
             const float *other = ex + (size_t)((e ? g.T0 : 0) + t) * (32 * 64) + co;
 #pragma unroll
@@ -702,6 +756,8 @@ cudaError_t launch_stem_window_wgrad(const Problem &pb, const void *dz, const vo
     g.n = pb.n; g.h_in = pb.h_in; g.w_in = pb.w_in; g.h_out = pb.h_out; g.w_out = pb.w_out; g.c_out = pb.c_out;
     g.kh = pb.kh; g.kw = pb.kw; g.pad_h = pb.pad_h; g.pad_w = pb.pad_w; g.pitch = pl.pitch; g.ksteps = pl.ksteps;
     g.T0 = (pb.kh + 1) / 2; g.T1 = pb.kh / 2; g.kdim = pb.kdim; g.xstrip_bytes = pl.xstrip; g.dzrow_bytes = pl.dzrow; g.work_bytes = pl.work;
+    g.nslots = (512 - kWgAccCols) / (8 * pl.ksteps);        // at least 1: w_out <= 256 gives ksteps <= 16
+    if (g.nslots > kWgMaxSlots) g.nslots = kWgMaxSlots;
     g.total_rows = (long long)pb.n * pb.h_out;
     g.f16 = call_f16();
     CUtensorMap tdz;
