@@ -77,7 +77,7 @@ def kernel_bytes(kind, spec, out_hw):
 # changed after its capture has no entry (traffic: null).  key: (kernel family, layer) -> (bytes, summary file).
 _P1, _P2S, _P2D, _P4 = ("profiles/config1_kernels_ncu_full.md", "profiles/config2_stem_window_kernels_ncu_full.md",
                         "profiles/config2_dense_gemm_ncu_full.md", "profiles/config4a_depthwise_kernels_ncu_full.md")
-NCU_TRAFFIC = {("stem_fwd", "c2s"): (63.2e6, _P2S), ("stem_dgrad", "c2s"): (117.2e6, _P2S), ("stem_wgrad", "c2s"): (126.5e6, _P2S),
+NCU_TRAFFIC = {("stem_fwd", "c2s"): (66.3e6, _P2S), ("stem_dgrad", "c2s"): (116.6e6, _P2S), ("stem_wgrad", "c2s"): (126.9e6, _P2S),
                ("umma_bwd", "c1a"): (76.4e6, _P1), ("strip_fwd", "c1b"): (13.0e6, _P1), ("strip_dgrad", "c1b"): (13.0e6, _P1),
                ("umma_fwd", "c2a"): (14.99e6, _P2D), ("umma_dgrad", "c2a"): (5.35e6, _P2D), ("umma_wgrad", "c2a"): (16.10e6, _P2D),
                ("umma_fwd", "c2b"): (7.98e6, _P2D),
